@@ -1,0 +1,626 @@
+"""CPU oracle for the Polestar denoising step (TEST INFRASTRUCTURE ONLY).
+
+A plain, slow, float64 numpy restatement of what the decoding path computes,
+written from the paper's equations and Algorithm 1.  Nothing here is used by
+the product: only the tests, the smoke check and the benchmark's CPU-baseline
+leg import it.  It shares no code with the CUDA path.
+
+What follows the paper directly
+  * greedy reconstruction / confidence ........ Sec. 2, Eq. 1 and the sampler set
+  * semi-autoregressive block update .......... Sec. 2, Eq. 2
+  * dual-cache attention of the active block .. Sec. 2, Eq. 3
+  * drift = KL of attention rows .............. Sec. 3, Eq. 4
+  * window, block entry, layer-wise refresh ... Sec. 4.1, Algorithm 1
+  * update schedule (tau_upd, alternate full entry) ... Sec. 4.1 "Update Schedule"
+  * drift-event commit, suffix commit ......... Sec. 4.2, Algorithm 1
+  * TPF accounting ............................ Appendix D.1 "Performance Measurement"
+  * staleness metric E ........................ Appendix C.2
+
+Readings taken where the paper is silent or inconsistent (all listed again in
+the design notes of the repository):
+  * drift is measured per window position (Eq. 4, and the "top-25% token
+    positions per layer" ablation of Sec. 5.3), not per K-means centroid;
+  * KL is averaged over query heads (Appendix C.2 averages over heads);
+  * the previous distribution of a row is the last one stored for it;
+  * drift / select / sparse forward run only on refresh steps, and the single
+    test ``cum > tau_upd`` implements the schedule;
+  * block entry forwards the whole sequence when ``b % period == 0`` and the
+    window plus active block otherwise;
+  * window = [start - 2B, start) U [end, end + B), clipped to the sequence;
+  * ``>=`` comparisons as in the text of Sec. 2 / 4.2 (flag selects ``>`` as
+    printed in Algorithm 1);
+  * mean of an empty drift history is 0 (h = 0 gives raw drift, Appendix D
+    "Drift history size"); the history is cleared at block entry;
+  * a quota top-up guarantees progress within the step budget;
+  * committed suffix tokens reach the cache as a layer-0 packet at the next
+    refresh step;
+  * only rows with drift above ``drift_floor`` are top-k candidates, so zero
+    drift refreshes nothing; mode ALL takes every window row.
+
+Synthetic model (the paper fixes none of it): pre-norm Transformer without
+attention mask, RMSNorm, half-split RoPE on q and k at absolute positions,
+grouped-query attention, SwiGLU FFN, untied embedding / LM head, no biases.
+
+Parity status: no passage of the paper prints an input/output pair, so absolute
+values of the forward pass are pinned only through library special cases
+(non-causal SDPA, library KL, stable argsort), closed forms, the theory
+appendix's propositions used as invariants, and brute force ("full refresh
+equals no-cache decoding").  See tests/test_oracle_*.py.
+"""
+from __future__ import annotations
+
+import math
+from typing import Dict, List, Optional
+
+import numpy as np
+
+F64 = np.float64
+
+SELECT_TOPK_FRAC, SELECT_TOPK_COUNT, SELECT_THRESHOLD, SELECT_ALL, SELECT_NONE = range(5)
+FLAG_DRIFT_COMMIT, FLAG_SUFFIX_COMMIT, FLAG_GE_COMPARE, FLAG_NOCACHE = 1, 2, 4, 8
+
+
+# --------------------------------------------------------------------------
+# storage-precision emulation
+# --------------------------------------------------------------------------
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bfloat16 (ties to even), returned as float64."""
+    a = np.ascontiguousarray(x, dtype=np.float32)
+    u = a.view(np.uint32).astype(np.uint64)
+    lsb = (u >> 16) & 1
+    r = ((u + 0x7FFF + lsb) >> 16) << 16
+    out = r.astype(np.uint32).view(np.float32)
+    out = np.where(np.isfinite(a), out, a)
+    return out.astype(F64)
+
+
+def _ident(x):
+    return np.asarray(x, dtype=F64)
+
+
+# --------------------------------------------------------------------------
+# model pieces (synthetic model; plain definitions)
+# --------------------------------------------------------------------------
+
+def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """y = x / sqrt(mean(x^2) + eps) * gain, row-wise."""
+    x = np.asarray(x, F64)
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * np.asarray(gain, F64)
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Half-split rotary embedding.  x [R, H, dh], pos [R] absolute positions.
+
+    Pair i is (x[i], x[i + dh/2]); angle = pos * theta^(-2i/dh).
+    """
+    x = np.asarray(x, F64)
+    R, H, dh = x.shape
+    half = dh // 2
+    inv = theta ** (-(2.0 * np.arange(half, dtype=F64)) / dh)
+    ang = np.asarray(pos, F64)[:, None] * inv[None, :]
+    c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def silu(x):
+    return x / (1.0 + np.exp(-x))
+
+
+def linear(x: np.ndarray, w: np.ndarray, rowwise: bool = False) -> np.ndarray:
+    """y = x @ w.T with w stored [out, in].  ``rowwise`` evaluates one row at a
+    time so that a row's result cannot depend on which rows accompany it."""
+    x = np.asarray(x, F64)
+    w64 = np.asarray(w, F64)
+    if rowwise:
+        out = np.empty((x.shape[0], w64.shape[0]), F64)
+        for r in range(x.shape[0]):
+            out[r] = w64 @ x[r]
+        return out
+    return x @ w64.T
+
+
+def attn_logp_rows(q: np.ndarray, K: np.ndarray, rowwise: bool = False) -> np.ndarray:
+    """Log attention distribution of each query row over all keys (no mask).
+
+    q [R, n_h, dh], K [N, n_kv, dh] -> logp [R, n_h, N];
+    logp = s - logsumexp(s), s = q.k / sqrt(dh)  (Appendix B "Setup").
+    Query head h reads kv head floor(h * n_kv / n_h).
+    """
+    q = np.asarray(q, F64)
+    K = np.asarray(K, F64)
+    R, nh, dh = q.shape
+    N, nkv, _ = K.shape
+    logp = np.empty((R, nh, N), F64)
+    for h in range(nh):
+        g = (h * nkv) // nh
+        Kg = np.ascontiguousarray(K[:, g, :])
+        if rowwise:
+            for r in range(R):
+                s = (Kg @ q[r, h, :]) / math.sqrt(dh)
+                mx = np.max(s)
+                logp[r, h, :] = s - (mx + np.log(np.sum(np.exp(s - mx))))
+        else:
+            s = np.ascontiguousarray((Kg @ q[:, h, :].T).T) / math.sqrt(dh)        # [R, N]
+            mx = np.max(s, axis=1, keepdims=True)
+            lse = mx + np.log(np.sum(np.exp(s - mx), axis=1, keepdims=True))
+            logp[:, h, :] = s - lse
+    return logp
+
+
+def attn_out_rows(logp: np.ndarray, V: np.ndarray, round_p=_ident, rowwise: bool = False) -> np.ndarray:
+    """o = sum_j p_j v_j per head.  logp [R, n_h, N], V [N, n_kv, dh] -> [R, n_h*dh]."""
+    R, nh, N = logp.shape
+    V = np.asarray(V, F64)
+    nkv, dh = V.shape[1], V.shape[2]
+    o = np.empty((R, nh, dh), F64)
+    for h in range(nh):
+        g = (h * nkv) // nh
+        Vg = np.ascontiguousarray(V[:, g, :])
+        if rowwise:
+            for r in range(R):
+                o[r, h, :] = round_p(np.exp(np.ascontiguousarray(logp[r, h, :]))) @ Vg
+        else:
+            o[:, h, :] = round_p(np.exp(logp[:, h, :])) @ Vg
+    return o.reshape(R, nh * dh)
+
+
+def kl_rows(logp_new: np.ndarray, logp_old: np.ndarray) -> np.ndarray:
+    """Eq. 4 per row: mean over heads of KL(new || old) = sum_j p_j (log p_j - log p'_j).
+
+    No epsilon and no clamp: identical rows give exactly 0."""
+    p = np.exp(logp_new)
+    kl = np.sum(p * (logp_new - logp_old), axis=-1)      # [R, n_h]
+    return np.mean(kl, axis=-1)
+
+
+def select_rows(D: np.ndarray, mode: int, *, frac: float = 0.25, k: int = 0,
+                thresh: float = 0.0, floor: float = 0.0) -> np.ndarray:
+    """Stale-row selection (Sec. 4.1 top-k; Sec. 5.3 per-position variant).
+
+    Returns ascending window indices.  Candidates are rows with D > floor;
+    order (D descending, index ascending).  ALL takes every row, NONE none.
+    """
+    D = np.asarray(D, F64)
+    W = D.shape[0]
+    if mode == SELECT_ALL:
+        return np.arange(W, dtype=np.int64)
+    if mode == SELECT_NONE or W == 0:
+        return np.zeros(0, np.int64)
+    cand = [i for i in range(W) if D[i] > floor]
+    if mode == SELECT_THRESHOLD:
+        return np.array([i for i in cand if D[i] > thresh], np.int64)
+    kk = int(math.floor(frac * W + 0.5)) if mode == SELECT_TOPK_FRAC else int(k)
+    cand.sort(key=lambda i: (-D[i], i))
+    return np.array(sorted(cand[:max(kk, 0)]), np.int64)
+
+
+def confidence_rows(logits: np.ndarray, mask_id: int):
+    """Eq. 1 and the confidence of Sec. 2: y_hat = argmax over v != [MASK] (lowest id
+    on ties), c = softmax(logits over the whole vocabulary)[y_hat]."""
+    l = np.asarray(logits, F64)
+    m = np.max(l, axis=-1, keepdims=True)
+    lse = (m + np.log(np.sum(np.exp(l - m), axis=-1, keepdims=True)))[..., 0]
+    lx = l.copy()
+    lx[..., mask_id] = -np.inf
+    yhat = np.argmax(lx, axis=-1)
+    c = np.exp(np.take_along_axis(l, yhat[..., None], axis=-1)[..., 0] - lse)
+    return yhat.astype(np.int64), c
+
+
+def staleness(K, K_ref, V, V_ref) -> np.ndarray:
+    """Appendix C.2: E = 1 - (cos(K, K_ref) + cos(V, V_ref)) / 2 per row, cosine per
+    head, averaged over heads.  Inputs [R, n_kv, dh]."""
+    def cs(a, b):
+        a, b = np.asarray(a, F64), np.asarray(b, F64)
+        return np.sum(a * b, -1) / (np.linalg.norm(a, axis=-1) * np.linalg.norm(b, axis=-1))
+    return 1.0 - 0.5 * np.mean(cs(K, K_ref) + cs(V, V_ref), axis=-1)
+
+
+# --------------------------------------------------------------------------
+# commit rule (Sec. 4.2; Algorithm 1, the lines after the layer loop)
+# --------------------------------------------------------------------------
+
+def commit_rule(conf, yhat, masked, delta_now, theta_hist, *, within: bool, tau_s: float,
+                alpha: float, ge: bool, drift_commit: bool, quota: int):
+    """Decide which masked active-block rows commit.
+
+    conf, yhat, masked [B]; delta_now [B] or None (entry step); theta_hist: list of
+    earlier delta vectors (most recent last, already trimmed to h).
+    Returns dict with boolean arrays by_conf, by_drift, by_quota, commit, and
+    Delta, tau_d.
+    """
+    B = len(conf)
+    conf = np.asarray(conf, F64)
+    cmpop = (lambda a, b: a >= b) if ge else (lambda a, b: a > b)
+    by_conf = np.zeros(B, bool)
+    by_drift = np.zeros(B, bool)
+    by_quota = np.zeros(B, bool)
+    tau_d = alpha * (tau_s - conf) ** 2
+    if within and delta_now is not None:
+        mean_hist = np.mean(np.stack(theta_hist), axis=0) if len(theta_hist) else np.zeros(B)
+        Delta = np.asarray(delta_now, F64) - mean_hist
+    else:
+        Delta = np.zeros(B)
+    for j in range(B):
+        if not masked[j]:
+            continue
+        if cmpop(conf[j], tau_s):
+            by_conf[j] = True
+        elif within and drift_commit and delta_now is not None and cmpop(Delta[j], tau_d[j]):
+            by_drift[j] = True
+    commit = by_conf | by_drift
+    need = quota - int(commit.sum())
+    if need > 0:
+        rest = [j for j in range(B) if masked[j] and not commit[j]]
+        rest.sort(key=lambda j: (-conf[j], j))
+        for j in rest[:need]:
+            by_quota[j] = True
+        commit = commit | by_quota
+    return dict(by_conf=by_conf, by_drift=by_drift, by_quota=by_quota, commit=commit,
+                Delta=Delta, tau_d=tau_d)
+
+
+# --------------------------------------------------------------------------
+# geometry
+# --------------------------------------------------------------------------
+
+def block_range(p, b: int):
+    s = p.prompt_len + b * p.block
+    return s, s + p.block
+
+
+def window_positions(p, b: int):
+    """Local window of block b: prefix part, suffix part (ascending positions)."""
+    N = p.prompt_len + p.gen_len
+    s, e = block_range(p, b)
+    pre = list(range(max(0, s - p.win_prefix_blocks * p.block), s))
+    suf = list(range(e, min(N, e + p.win_suffix_blocks * p.block)))
+    return pre, suf
+
+
+# --------------------------------------------------------------------------
+# one sequence
+# --------------------------------------------------------------------------
+
+class _Seq:
+    """Decoding state of one sequence (Algorithm 1 "Cached state")."""
+
+    def __init__(self, m, w, p, prompt, rowwise=False, emulate_bf16=None):
+        self.m, self.w, self.p = m, w, p
+        self.rowwise = rowwise
+        emu = (m.dtype == 1) if emulate_bf16 is None else emulate_bf16
+        self.rnd = bf16_round if emu else _ident
+        self.N = p.prompt_len + p.gen_len
+        self.y = np.concatenate([np.asarray(prompt, np.int64),
+                                 np.full(p.gen_len, m.mask_id, np.int64)])
+        L = m.n_layers
+        self.Kc = [np.zeros((self.N, m.n_kv_heads, m.head_dim), F64) for _ in range(L)]
+        self.Vc = [np.zeros((self.N, m.n_kv_heads, m.head_dim), F64) for _ in range(L)]
+        self.Hc: List[Optional[np.ndarray]] = [None] * L
+        self.Pprev: List[Optional[np.ndarray]] = [None] * L
+        self.Aprev = None
+        self.theta: List[np.ndarray] = []
+        self.tok_at_h0 = None
+        self.cum = 0
+        self.delta = None
+        self.trace: Dict = {}
+
+    # -- layer pieces ------------------------------------------------------
+    def _qkv(self, l, x, pos):
+        m, wl, rnd = self.m, self.w["layers"][l], self.rnd
+        a = rnd(rmsnorm(x, wl["norm1"], m.rms_eps))
+        R = x.shape[0]
+        q = linear(a, wl["wq"], self.rowwise).reshape(R, m.n_heads, m.head_dim)
+        k = linear(a, wl["wk"], self.rowwise).reshape(R, m.n_kv_heads, m.head_dim)
+        v = linear(a, wl["wv"], self.rowwise).reshape(R, m.n_kv_heads, m.head_dim)
+        q = rnd(rope(q, pos, m.rope_theta))
+        k = rnd(rope(k, pos, m.rope_theta))
+        return q, k, rnd(v)
+
+    def _finish(self, l, x, logp):
+        """Rest of layer l for rows x with attention rows logp: attention output,
+        output projection + residual, SwiGLU FFN + residual."""
+        m, wl, rnd = self.m, self.w["layers"][l], self.rnd
+        o = rnd(attn_out_rows(logp, self.Vc[l], rnd, self.rowwise))
+        x1 = x + linear(o, wl["wo"], self.rowwise)
+        f = rnd(rmsnorm(x1, wl["norm2"], m.rms_eps))
+        g = rnd(silu(linear(f, wl["wg"], self.rowwise)) * linear(f, wl["wu"], self.rowwise))
+        return x1 + linear(g, wl["wd"], self.rowwise)
+
+    def _logits(self, xL):
+        m = self.m
+        a = self.rnd(rmsnorm(xL, self.w["final_norm"], m.rms_eps))
+        return linear(a, self.w["lm_head"], self.rowwise) * self.p.logit_scale
+
+    def _embed(self, pos):
+        return np.asarray(self.w["embed"], F64)[self.y[pos]] if len(pos) else \
+            np.zeros((0, self.m.d_model), F64)
+
+    # -- block entry (Sec. 4.1 "Initialization", "Block entry"; Alg. 1 entry part) ----
+    def step_entry(self, b: int):
+        m, p = self.m, self.p
+        s, e = block_range(p, b)
+        pre, suf = window_positions(p, b)
+        win = np.array(pre + suf, np.int64)
+        act = np.arange(s, e, dtype=np.int64)
+        full = (b % p.full_entry_period == 0) or bool(p.flags & FLAG_NOCACHE)
+        rows = np.arange(self.N, dtype=np.int64) if full else np.array(sorted(pre + list(act) + suf), np.int64)
+        where = {int(pz): i for i, pz in enumerate(rows)}
+        wi = np.array([where[int(z)] for z in win], np.int64)
+        ai = np.array([where[int(z)] for z in act], np.int64)
+        x = self._embed(rows)
+        tr = {"kind": "entry_full" if full else "entry_window", "x_act": [], "rows": rows}
+        for l in range(m.n_layers):
+            tr["x_act"].append(x[ai].copy())
+            self.Hc[l] = x[wi].copy()
+            q, k, v = self._qkv(l, x, rows)
+            self.Kc[l][rows] = k
+            self.Vc[l][rows] = v
+            logp = attn_logp_rows(q, self.Kc[l], self.rowwise)
+            self.Pprev[l] = logp[wi].copy()
+            if l == m.n_layers - 1:
+                self.Aprev = logp[ai].copy()
+            x = self._finish(l, x, logp)
+        tr["x_act"].append(x[ai].copy())
+        self.tok_at_h0 = self.y[win].copy()
+        self.win, self.act, self.n_pre = win, act, len(pre)
+        self.theta = []
+        self.delta = None
+        self.logits = self._logits(x[ai])
+        self.suffix_logits = None
+        self.suffix_rows = np.zeros(0, np.int64)
+        tr["logits"] = self.logits
+        self.trace = tr
+        self.within = False
+
+    # -- within-block step (Alg. 1 inner loop) ----------------------------------
+    def step_within(self, forced_sel=None):
+        m, p = self.m, self.p
+        L = m.n_layers
+        win, act = self.win, self.act
+        W = len(win)
+        refresh = (p.tau_upd < 0) or (self.cum > p.tau_upd)
+        tr = {"kind": "within", "refresh": refresh, "x_act": [], "D": [], "sel": [],
+              "patched": []}
+        U_idx = np.zeros(0, np.int64)
+        U_val = np.zeros((0, m.d_model), F64)
+        if refresh:
+            self.cum = 0
+            U_idx = np.array([i for i in range(W) if self.y[win[i]] != self.tok_at_h0[i]], np.int64)
+            U_val = self._embed(win[U_idx])
+            self.tok_at_h0 = self.y[win].copy()
+        x = self._embed(act)
+        for l in range(L):
+            tr["x_act"].append(x.copy())
+            # 1. patch the caches from the update packet of the previous layer
+            if refresh and len(U_idx):
+                self.Hc[l][U_idx] = U_val
+                _, k, v = self._qkv(l, U_val, win[U_idx])
+                self.Kc[l][win[U_idx]] = k
+                self.Vc[l][win[U_idx]] = v
+            tr["patched"].append(U_idx.copy())
+            # 2. active block over the patched cache (Eq. 3)
+            q, k, v = self._qkv(l, x, act)
+            self.Kc[l][act] = k
+            self.Vc[l][act] = v
+            logpA = attn_logp_rows(q, self.Kc[l], self.rowwise)
+            if l == L - 1:
+                self.delta = kl_rows(logpA, self.Aprev)
+                self.Aprev = logpA.copy()
+            x = self._finish(l, x, logpA)
+            # 3. drift of the window rows, selection, sparse forward -> next packet
+            if refresh:
+                qw, _, _ = self._qkv(l, self.Hc[l], win)
+                P = attn_logp_rows(qw, self.Kc[l], self.rowwise)
+                D = kl_rows(P, self.Pprev[l])
+                self.Pprev[l] = P.copy()
+                if forced_sel is not None:
+                    S = np.asarray(forced_sel[l], np.int64)
+                else:
+                    S = select_rows(D, p.select_mode, frac=p.select_frac, k=p.select_k,
+                                    thresh=p.select_thresh, floor=p.drift_floor)
+                tr["D"].append(D)
+                tr["sel"].append(S)
+                U_idx = S
+                U_val = self._finish(l, self.Hc[l][S], P[S]) if len(S) else np.zeros((0, m.d_model), F64)
+            else:
+                tr["D"].append(None)
+                tr["sel"].append(np.zeros(0, np.int64))
+        tr["x_act"].append(x.copy())
+        self.logits = self._logits(x)
+        tr["logits"] = self.logits
+        tr["delta"] = self.delta
+        # suffix rows of the final packet (Sec. 4.2 "Suffix Block Commit")
+        self.suffix_rows = np.zeros(0, np.int64)
+        self.suffix_logits = None
+        if refresh and len(U_idx):
+            keep = np.array([i for i, wi_ in enumerate(U_idx) if wi_ >= self.n_pre], np.int64)
+            if len(keep):
+                self.suffix_rows = U_idx[keep]
+                self.suffix_logits = self._logits(U_val[keep])
+        tr["suffix_rows"] = self.suffix_rows
+        tr["suffix_logits"] = self.suffix_logits
+        self.trace = tr
+        self.within = True
+
+    # -- commit (Sec. 4.2; Eq. 2) ---------------------------------------------------
+    def commit(self, steps_used: int, forced=None):
+        m, p = self.m, self.p
+        act = self.act
+        B = len(act)
+        ge = bool(p.flags & FLAG_GE_COMPARE)
+        masked = self.y[act] == m.mask_id
+        yhat, conf = confidence_rows(self.logits, m.mask_id)
+        spb = max(1, p.max_steps // max(1, p.gen_len // p.block))
+        n_masked = int(masked.sum())
+        quota = -(-n_masked // max(1, spb - steps_used)) if n_masked else 0
+        r = commit_rule(conf, yhat, masked, self.delta if self.within else None, self.theta,
+                        within=self.within, tau_s=p.tau_s, alpha=p.alpha, ge=ge,
+                        drift_commit=bool(p.flags & FLAG_DRIFT_COMMIT), quota=quota)
+        if self.within and self.delta is not None and p.hist > 0:
+            self.theta = (self.theta + [np.asarray(self.delta, F64).copy()])[-p.hist:]
+        commit = r["commit"] if forced is None else np.asarray(forced["commit"], bool)
+        info = dict(conf=conf, yhat=yhat, masked=masked, quota=quota, **r)
+        n_new = 0
+        n_eos = 0
+        for j in range(B):
+            if commit[j] and masked[j]:
+                self.y[act[j]] = yhat[j]
+                n_new += 1
+                n_eos += int(yhat[j] == m.eos_id)
+        # suffix commit: eligible rows come from the final packet, confidence decides
+        n_suffix = 0
+        suf_commit = []
+        if self.within and (p.flags & FLAG_SUFFIX_COMMIT) and len(self.suffix_rows):
+            sy, sc = confidence_rows(self.suffix_logits, m.mask_id)
+            for t, wi_ in enumerate(self.suffix_rows):
+                pos = self.win[wi_]
+                ok = (sc[t] >= p.tau_suffix) if ge else (sc[t] > p.tau_suffix)
+                if forced is not None:
+                    ok = int(pos) in forced.get("suffix", ())
+                if self.y[pos] == m.mask_id and ok:
+                    self.y[pos] = sy[t]
+                    n_suffix += 1
+                    n_eos += int(sy[t] == m.eos_id)
+                    suf_commit.append(int(pos))
+            info["suffix_conf"], info["suffix_yhat"] = sc, sy
+        self.cum = (n_new + n_suffix) if not self.within else self.cum + n_new + n_suffix
+        info.update(n_committed=n_new + n_suffix, n_by_conf=int((r["by_conf"] & commit).sum()),
+                    n_by_drift=int((r["by_drift"] & commit).sum()),
+                    n_by_quota=int((r["by_quota"] & commit).sum()), n_suffix=n_suffix,
+                    n_eos=n_eos, suffix_committed=suf_commit,
+                    block_done=not bool((self.y[act] == m.mask_id).any()))
+        return info
+
+
+# --------------------------------------------------------------------------
+# controller (Algorithm 1 outer loops; Sec. 4.1 "Update Schedule")
+# --------------------------------------------------------------------------
+
+class PolestarOracle:
+    """Batch of independent sequences advancing blocks in lock-step."""
+
+    def __init__(self, m, weights, p, prompt, rowwise=False, emulate_bf16=None):
+        self.m, self.p = m, p
+        prompt = np.asarray(prompt).reshape(p.batch, p.prompt_len)
+        self.seqs = [_Seq(m, weights, p, prompt[s], rowwise, emulate_bf16) for s in range(p.batch)]
+        self.b = 0
+        self.need_entry = True
+        self.steps_used = 0
+        self.forwards = 0
+        self.pending = False
+        self.done = False
+        self.generated = 0
+        self.generated_non_eos = 0
+
+    def step(self, forced_sel=None):
+        assert not self.done and not self.pending
+        for si, s in enumerate(self.seqs):
+            if self.need_entry:
+                s.step_entry(self.b)
+            else:
+                s.step_within(None if forced_sel is None else forced_sel[si])
+        kind = self.seqs[0].trace["kind"]
+        self.forwards += 1
+        self.pending = True
+        return kind
+
+    def commit(self, forced=None):
+        assert self.pending
+        infos = [s.commit(self.steps_used, None if forced is None else forced[si])
+                 for si, s in enumerate(self.seqs)]
+        self.pending = False
+        self.steps_used += 1
+        self.need_entry = False
+        for i in infos:
+            self.generated += i["n_committed"]
+            self.generated_non_eos += i["n_committed"] - i["n_eos"]
+        if all(i["block_done"] for i in infos):
+            self.b += 1
+            self.need_entry = True
+            self.steps_used = 0
+            if self.b >= self.p.gen_len // self.p.block:
+                self.done = True
+        return infos
+
+    def decode(self, max_forwards: int = 10 ** 9):
+        while not self.done and self.forwards < max_forwards:
+            self.step()
+            self.commit()
+        return self.tokens()
+
+    def tokens(self) -> np.ndarray:
+        return np.stack([s.y for s in self.seqs])
+
+    @property
+    def tpf(self) -> float:
+        return self.generated_non_eos / max(1, self.forwards)
+
+
+class NoCacheOracle:
+    """Reference decoder of Sec. 3.1 "Setup": a full-sequence forward at every
+    step, no cache reuse, the same commit rule."""
+
+    def __init__(self, m, weights, p, prompt, rowwise=False, emulate_bf16=None):
+        import dataclasses
+        p2 = dataclasses.replace(p, flags=p.flags | FLAG_NOCACHE)
+        self.inner = PolestarOracle(m, weights, p2, prompt, rowwise, emulate_bf16)
+
+    def step(self):
+        o = self.inner
+        assert not o.done and not o.pending
+        for s in o.seqs:
+            entry = o.need_entry
+            prev_A, prev_theta = s.Aprev, s.theta
+            s.step_entry(o.b)          # full-sequence forward (NOCACHE flag)
+            if not entry:
+                # same block: keep the drift history, and delta against the previous step
+                a_now = s.Aprev
+                s.delta = kl_rows(a_now, prev_A)
+                s.theta = prev_theta
+                s.within = True
+                s.trace["kind"] = "within"
+                s.trace["delta"] = s.delta
+        o.forwards += 1
+        o.pending = True
+
+    def commit(self):
+        return self.inner.commit()
+
+    def decode(self):
+        o = self.inner
+        while not o.done:
+            self.step()
+            self.commit()
+        return o.tokens()
+
+    def tokens(self):
+        return self.inner.tokens()
+
+    @property
+    def seqs(self):
+        return self.inner.seqs
+
+
+# --------------------------------------------------------------------------
+# refresh chain on its own (select -> gather -> QKV projection -> scatter)
+# --------------------------------------------------------------------------
+
+def refresh_chain(H, drift, k, wq, wk, wv, norm, eps, theta, n_heads, n_kv_heads, head_dim,
+                  Kc, Vc, emulate_bf16=True):
+    """Top-k rows of ``drift`` -> recompute their K/V from the hidden cache H ->
+    write them into copies of Kc, Vc.  One sequence.  Returns (idx, q, Kc', Vc')."""
+    rnd = bf16_round if emulate_bf16 else _ident
+    idx = select_rows(drift, SELECT_TOPK_COUNT, k=k, floor=0.0)
+    a = rnd(rmsnorm(np.asarray(H, F64)[idx], norm, eps))
+    R = len(idx)
+    q = rnd(rope(linear(a, wq).reshape(R, n_heads, head_dim), idx, theta))
+    kk = rnd(rope(linear(a, wk).reshape(R, n_kv_heads, head_dim), idx, theta))
+    vv = rnd(linear(a, wv).reshape(R, n_kv_heads, head_dim))
+    K2, V2 = np.array(Kc, F64, copy=True), np.array(Vc, F64, copy=True)
+    K2[idx] = kk
+    V2[idx] = vv
+    return idx, q, K2, V2
