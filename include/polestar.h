@@ -1,0 +1,264 @@
+/*
+ * polestar.h -- C ABI of the Polestar denoising hot path for masked-diffusion LLMs
+ * on NVIDIA B200 (sm_100a).
+ *
+ * One library call sequence decodes a batch of sequences:
+ *
+ *     polestar_init   -> block-0 entry forward        (Algorithm 1, block entry)
+ *     loop:  polestar_commit -> polestar_step -> polestar_commit -> ...
+ *
+ * `polestar_step` runs ONE model forward (a block-entry forward or a within-block
+ * step with drift-aware cache refresh); `polestar_commit` applies the confidence /
+ * drift-event commit rule to the logits that forward produced and advances the
+ * controller.  `polestar_init` already runs the first forward, so the first call
+ * after it is `polestar_commit`.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global-memory addresses of the current device,
+ *     "host" pointers are ordinary CPU addresses.  No torch / C++ types cross the ABI.
+ *   - The library allocates NO device memory (except where a function says so):
+ *     weights and one workspace are caller-owned device buffers that must outlive
+ *     the context.  The context itself is a small host object.
+ *   - All work is enqueued on the CUDA stream given at init (a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream).  `polestar_commit`,
+ *     `polestar_tokens` and `polestar_read` synchronise that stream.
+ *   - Every function returns 0 (POLESTAR_OK) or a negative error code and never
+ *     throws or aborts.  Asynchronous CUDA errors surface at the next synchronising
+ *     call as POLESTAR_E_CUDA.
+ *   - Hidden states, logits, drift values and attention log-probabilities are
+ *     float32.  Weights, K/V cache and GEMM operands have the model's dtype.
+ *
+ * Memory layout of the weights (device, model dtype, every matrix [out, in] row-major)
+ *   embed, lm_head  [vocab, d_model]
+ *   wqkv[l]         [(n_heads + 2 n_kv_heads) * head_dim, d_model]: query heads, then key
+ *                   heads, then value heads.  Inside every query and key head the rows are
+ *                   PAIR-INTERLEAVED: packed row 2i is logical row i and packed row 2i+1 is
+ *                   logical row i + head_dim/2 (the two elements rotary embedding rotates
+ *                   together).  Scores q.k do not depend on a common permutation of the head
+ *                   dimension, so the cache simply keeps keys in this order.
+ *   wo[l]           [d_model, n_heads * head_dim]
+ *   w_gate_up[l]    [2 * d_ffn, d_model]: row 2f is gate row f, row 2f+1 is up row f
+ *   w_down[l]       [d_model, d_ffn]
+ *   norm1[l], norm2[l], final_norm   [d_model] float32 gains
+ */
+#ifndef POLESTAR_H
+#define POLESTAR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- error codes --------------------------------------------------------------- */
+#define POLESTAR_OK            0
+#define POLESTAR_E_INVAL      (-1)  /* bad argument / unsupported shape            */
+#define POLESTAR_E_STATE      (-2)  /* call order violated                         */
+#define POLESTAR_E_NOSPACE    (-3)  /* workspace too small                         */
+#define POLESTAR_E_CUDA       (-4)  /* a CUDA call or kernel failed                */
+#define POLESTAR_E_NONFINITE  (-5)  /* NaN / Inf met where a decision was needed   */
+#define POLESTAR_E_TIMEOUT    (-6)  /* a bounded device-side wait ran out          */
+#define POLESTAR_E_DONE       (-7)  /* every block is already decoded              */
+
+/* ---- enumerations --------------------------------------------------------------- */
+#define POLESTAR_F32  0
+#define POLESTAR_BF16 1
+
+/* stale-row selection (Sec. 4.1 "Measuring Drift and Layer-wise KV Updates") */
+#define POLESTAR_SELECT_TOPK_FRAC 0   /* k = floor(select_frac * W + 1/2) largest drifts   */
+#define POLESTAR_SELECT_TOPK_COUNT 1  /* k = select_k                                       */
+#define POLESTAR_SELECT_THRESHOLD 2   /* drift > select_thresh                              */
+#define POLESTAR_SELECT_ALL 3         /* every window row (full refresh)                    */
+#define POLESTAR_SELECT_NONE 4        /* never refresh rows (drift still measured)          */
+
+#define POLESTAR_FLAG_DRIFT_COMMIT  (1u << 0) /* drift-event clause of the commit rule (Sec. 4.2)  */
+#define POLESTAR_FLAG_SUFFIX_COMMIT (1u << 1) /* suffix-block commit from the final packet          */
+#define POLESTAR_FLAG_GE_COMPARE    (1u << 2) /* ">=" as in the text of Sec. 4.2; off: ">" (Alg. 1) */
+#define POLESTAR_FLAG_NOCACHE       (1u << 3) /* every step is a full-sequence forward (baseline)   */
+#define POLESTAR_FLAG_KEEP_HIDDEN   (1u << 4) /* keep per-layer active hidden states for read-back  */
+#define POLESTAR_FLAG_SIMT_GEMM     (1u << 5) /* bf16 models: plain CUDA-core GEMMs (debug aid)     */
+
+#define POLESTAR_STEP_ENTRY_FULL   0
+#define POLESTAR_STEP_ENTRY_WINDOW 1
+#define POLESTAR_STEP_WITHIN       2
+
+#define POLESTAR_MAX_BATCH 64
+
+/* ---- plain-data descriptions ------------------------------------------------------ */
+typedef struct polestar_ctx polestar_ctx;
+
+/* Synthetic mask predictor: pre-norm Transformer, RMSNorm, rotary q/k at absolute
+ * positions, grouped-query bidirectional attention, SwiGLU FFN, untied LM head. */
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    int32_t dtype;                 /* POLESTAR_F32 | POLESTAR_BF16 */
+    float   rms_eps, rope_theta;
+    int32_t mask_id, eos_id;
+} polestar_model;
+
+/* All pointers are device pointers, BORROWED for the context's lifetime.
+ * The six arrays of per-layer pointers are HOST arrays of n_layers device pointers. */
+typedef struct {
+    const void *embed, *lm_head;
+    const float *final_norm;
+    const void *const *wqkv, *const *wo, *const *w_gate_up, *const *w_down;
+    const float *const *norm1, *const *norm2;
+} polestar_weights;
+
+/* Decoding parameters; defaults in comments are the paper's (Sec. 5.1, Appendix D Table
+ * "Default hyperparameters"). */
+typedef struct {
+    int32_t batch, prompt_len, gen_len, block /*32*/, max_steps;
+    int32_t win_prefix_blocks /*2*/, win_suffix_blocks /*1*/, full_entry_period /*2*/;
+    int32_t select_mode /*TOPK_FRAC*/;
+    float   select_frac /*0.25*/;
+    int32_t select_k;
+    float   select_thresh, drift_floor /*0*/;
+    int32_t tau_upd /*3; <0: refresh every step; INT32_MAX: never*/, hist /*5*/;
+    float   tau_s /*0.9*/, alpha /*10*/, tau_suffix /*0.9*/, logit_scale /*1*/;
+    uint32_t flags /*DRIFT_COMMIT|SUFFIX_COMMIT|GE_COMPARE*/;
+} polestar_params;
+
+typedef struct {
+    int32_t kind;            /* POLESTAR_STEP_*                                     */
+    int32_t block_index;
+    int32_t n_refreshing;    /* sequences whose cache is being refreshed this step  */
+    int32_t rows;            /* rows forwarded per sequence (upper bound)           */
+    int64_t forwards;        /* forwards so far, this one included                  */
+} polestar_step_info;
+
+typedef struct {
+    int32_t n_committed, n_by_conf, n_by_drift, n_by_quota, n_suffix, n_eos; /* batch sums */
+    int32_t rows_refreshed;  /* cache rows rewritten by the last step, all layers   */
+    int32_t block_index;     /* block the commit belonged to                        */
+    int32_t block_done;      /* 1: the next step is a block entry                   */
+    int32_t all_done;        /* 1: every block decoded                              */
+    int64_t forwards;        /* forwards so far                                     */
+    int64_t generated, generated_non_eos;  /* running totals (TPF numerator, App. D.1) */
+} polestar_commit_info;
+
+/* ---- the decoding path ------------------------------------------------------------ */
+
+/* Bytes of device workspace `polestar_init` needs for this model and these parameters
+ * (0 if they are invalid).  Pure host arithmetic. */
+size_t polestar_workspace_bytes(const polestar_model *m, const polestar_params *p);
+
+/* Create a context and run the block-0 entry forward (Algorithm 1: initial state,
+ * block entry with a full-sequence forward, Sec. 4.1 "Initialization").
+ *   prompt_ids_host  host, [batch][prompt_len] token ids in [0, vocab), none equal mask_id
+ *   workspace_dev    device, >= polestar_workspace_bytes(), 256-byte aligned, caller-owned;
+ *                    the library zero-fills what it needs
+ *   cuda_stream      cudaStream_t as void*
+ * Errors: E_INVAL (NULLs, unsupported shape, bad ids), E_NOSPACE, E_CUDA. *out is NULL on error. */
+int polestar_init(polestar_ctx **out, const polestar_model *m, const polestar_weights *w,
+                  const polestar_params *p, const int32_t *prompt_ids_host,
+                  void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
+/* One forward (Algorithm 1): a block-entry forward if the previous commit finished a block,
+ * otherwise a within-block step: [patch caches from the packet -> active block over the
+ * patched cache (Eq. 3) -> drift of the window rows (Eq. 4) -> select -> sparse forward of the
+ * selected rows -> packet for the next layer] per layer, then logits and confidences.
+ * Asynchronous.  info_host may be NULL.  Errors: E_STATE (commit pending), E_DONE, E_CUDA. */
+int polestar_step(polestar_ctx *c, polestar_step_info *info_host);
+
+/* Commit rule of Sec. 4.2 on the last forward's logits (confidence >= tau_s, or drift delta
+ * >= alpha (tau_s - c)^2 on within-block steps, quota top-up, suffix rows by confidence),
+ * Eq. 2 token update, controller bookkeeping.  Synchronises.  info_host may be NULL.
+ * Errors: E_STATE (no forward pending), E_NONFINITE, E_TIMEOUT, E_CUDA. */
+int polestar_commit(polestar_ctx *c, polestar_commit_info *info_host);
+
+/* Copy the current token ids to host memory: out_host [batch][prompt_len + gen_len]. */
+int polestar_tokens(polestar_ctx *c, int32_t *out_host);
+
+/* Read-back of internal state for parity checks.  `what`: */
+#define POLESTAR_READ_LOGITS      1  /* float [batch][block][vocab], last forward                */
+#define POLESTAR_READ_CONF        2  /* float [batch][block]                                     */
+#define POLESTAR_READ_YHAT        3  /* int32 [batch][block]                                     */
+#define POLESTAR_READ_DELTA       4  /* float [batch][block] last-layer drift of active rows     */
+#define POLESTAR_READ_DRIFT       5  /* float [batch][W_max] drift of window rows at `layer`     */
+#define POLESTAR_READ_SEL_COUNT   6  /* int32 [batch] rows selected at `layer`                   */
+#define POLESTAR_READ_SEL_IDX     7  /* int32 [batch][W_max] ascending window indices, `layer`   */
+#define POLESTAR_READ_HIDDEN      8  /* float [batch][block][d] input of `layer` (0..n_layers;
+                                        n_layers = final hidden); needs FLAG_KEEP_HIDDEN         */
+#define POLESTAR_READ_KCACHE      9  /* model dtype [batch][N][n_kv*head_dim] (keys interleaved) */
+#define POLESTAR_READ_VCACHE     10  /* model dtype [batch][N][n_kv*head_dim]                    */
+#define POLESTAR_READ_HCACHE     11  /* float [batch][W_max][d] window hidden cache at `layer`   */
+#define POLESTAR_READ_COMMIT     12  /* int32 [batch][block] bit0 commit, bit1 by confidence,
+                                        bit2 by drift, bit3 by quota (last commit)               */
+#define POLESTAR_READ_PPREV      13  /* float [batch][W_max][n_heads][N] stored log attention    */
+#define POLESTAR_READ_SUFFIX     14  /* int32 [batch][W_max] bit0 eligible, bit1 committed       */
+/* Synchronises, copies min(bytes, size of the item) bytes to dst_host.
+ * Errors: E_INVAL (unknown item, bad layer, item not kept). */
+int polestar_read(polestar_ctx *c, int32_t what, int32_t layer, void *dst_host, size_t bytes);
+
+/* Forced decisions, for checking each step's arithmetic on its own when a near-tie would let
+ * two correct implementations diverge.  `what`: */
+#define POLESTAR_FORCE_SELECT 1  /* rows refreshed at `layer` in the next step: idx_host holds, per
+                                    sequence, n ascending window indices ([batch][n])            */
+#define POLESTAR_FORCE_COMMIT 2  /* positions committed by the next commit: idx_host holds, per
+                                    sequence, n absolute positions ([batch][n]; -1 = unused)     */
+#define POLESTAR_FORCE_CLEAR  3  /* drop all forced decisions                                     */
+int polestar_force(polestar_ctx *c, int32_t what, int32_t layer, const int32_t *idx_host, int32_t n);
+
+void polestar_destroy(polestar_ctx *c);
+const char *polestar_strerror(int code);
+
+/* ---- single kernels of the path (unit parity, micro-benchmarks) --------------------- */
+
+/* Drift of attention rows (Eq. 4; Algorithm 1 "ProxyAttn" + "KL"), optionally with the attention
+ * output: for each of R query rows and each head, logp = log softmax_j(q.k_j / sqrt(head_dim))
+ * over all N keys; kl[r][h] = sum_j p_j (logp_j - logp_prev[r][h][j]); logp_prev is then
+ * overwritten with logp; out[r] = sum_j p_j v_j.
+ *   q_dev [R][n_heads*head_dim], k_dev / v_dev [N][n_kv*head_dim] (model dtype; one sequence)
+ *   logp_prev_dev float [R][n_heads][N] in/out (NULL: no KL, nothing stored)
+ *   kl_dev float [R][n_heads] (NULL allowed iff logp_prev_dev NULL), out_dev [R][n_heads*head_dim]
+ *   model dtype (NULL: skipped). */
+int polestar_k_attention(const void *q_dev, const void *k_dev, const void *v_dev,
+                         float *logp_prev_dev, float *kl_dev, void *out_dev,
+                         int32_t R, int32_t N, int32_t n_heads, int32_t n_kv_heads,
+                         int32_t head_dim, int32_t dtype, void *cuda_stream);
+
+/* Squared hidden-state change per row, sum_c (a[r][c] - b[r][c])^2 (Appendix B, Cor. 1's
+ * Delta H): a_dev, b_dev [rows][d] model dtype -> out_dev float [rows]. */
+int polestar_k_hidden_delta(const void *a_dev, const void *b_dev, float *out_dev,
+                            int32_t rows, int32_t d, int32_t dtype, void *cuda_stream);
+
+/* Stale-row selection and compaction (Sec. 4.1 top-k; Algorithm 1 "TopK").  Per sequence s of
+ * `batch`: among the W rows with drift_dev[s][i] > floor choose by `mode` (POLESTAR_SELECT_*;
+ * ties: lower index first) and write their indices ascending to idx_dev[s][0..count), count_dev[s].
+ * W <= 4096. */
+int polestar_k_select(const float *drift_dev, int32_t batch, int32_t W, int32_t mode, int32_t k,
+                      float thresh, float floor_, int32_t *idx_dev, int32_t *count_dev,
+                      void *cuda_stream);
+
+/* Gathered K/V refresh (Sec. 4.1; Algorithm 1 "Patch"): for each sequence s and each
+ * i < count_dev[s], row = idx_dev[s][i]: a = RMSNorm(h_dev[s][row]) * norm; (q,k,v) = a Wqkv^T;
+ * rotary on q,k at position `row`; k,v written to kc_dev[s][row], vc_dev[s][row]; q to
+ * q_out_dev[s][i] (NULL: dropped).  Rows not listed are not touched.
+ *   h_dev [batch][P][d], kc_dev/vc_dev [batch][P][n_kv*head_dim], model dtype
+ *   wqkv_dev as in polestar_weights; max_rows = upper bound of count (<= P)
+ *   scratch_dev: >= polestar_k_refresh_scratch_bytes(...) bytes, 1024-byte aligned. */
+size_t polestar_k_refresh_scratch_bytes(int32_t batch, int32_t max_rows, int32_t d,
+                                        int32_t n_heads, int32_t n_kv_heads, int32_t head_dim);
+int polestar_k_refresh(const void *h_dev, const int32_t *idx_dev, const int32_t *count_dev,
+                       const void *wqkv_dev, const float *norm_dev, void *kc_dev, void *vc_dev,
+                       void *q_out_dev, int32_t batch, int32_t P, int32_t max_rows, int32_t d,
+                       int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float rms_eps,
+                       float rope_theta, int32_t dtype, void *scratch_dev, size_t scratch_bytes,
+                       void *cuda_stream);
+
+/* Confidence of logits rows (Eq. 1; Sec. 2 sampler set): per row, y_hat = argmax over v != mask_id
+ * (lowest id on ties), conf = softmax(logits)[y_hat].  logits_dev float [rows][vocab];
+ * scratch_dev: >= rows * 512 bytes of device memory. */
+int polestar_k_confidence(const float *logits_dev, int32_t rows, int32_t vocab, int32_t mask_id,
+                          int32_t *yhat_dev, float *conf_dev, void *scratch_dev, size_t scratch_bytes,
+                          void *cuda_stream);
+
+/* Number of SMs the library sized its grids for (0 before any context exists). */
+int polestar_sm_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POLESTAR_H */

@@ -1,0 +1,320 @@
+// Bidirectional attention rows with drift for bf16 models, head_dim 128 (Eq. 3, Eq. 4).
+//
+// One CTA = 16 query rows of one head; its 4 warps split the keys in interleaved 32-key
+// tiles, each warp streaming its own K/V tiles through a private cp.async double buffer.
+// Pass 1 gives every row's log-sum-exp (online max/sum per warp, combined across warps);
+// pass 2 recomputes the scores, forms logp = s - lse, p = exp(logp), accumulates
+// KL(p || stored row), overwrites the stored row with logp and accumulates p V.
+// Two passes keep logp exact (no running rescale of the stored rows); the second read of K
+// comes from L2.  Tensor-core path: warp-level mma.sync m16n8k16 (bf16 in, fp32 accumulate).
+#pragma once
+#include "kernels.cuh"
+
+namespace ps {
+
+constexpr int AT_BM = 16;        // query rows per CTA
+constexpr int AT_BN = 32;        // keys per warp tile
+constexpr int AT_WARPS = 4;
+constexpr int AT_DH = 128;
+constexpr int AT_STAGE_BYTES = 2 * AT_BN * AT_DH * 2;            // K tile + V tile
+constexpr int AT_SMEM = AT_WARPS * 2 * AT_STAGE_BYTES + AT_BM * AT_DH * 2 + 1024;
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float* c, const uint32_t* a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
+    const int sz = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// byte offset of 16-byte chunk `ch` of row `row` in a [rows][128] bf16 tile, XOR-swizzled
+__device__ __forceinline__ uint32_t sw_off(int row, int ch) { return (uint32_t)(row * 256 + ((ch ^ (row & 7)) << 4)); }
+
+struct AttnMmaArgs {
+    AttnArgs a;
+    int rows_per_seq;   // forward rows per sequence (stand-alone: n_rows)
+    int tiles_per_seq;
+};
+
+__global__ void __launch_bounds__(AT_WARPS * 32) attention_mma_kernel(AttnMmaArgs g) {
+    extern __shared__ uint8_t at_smem_raw[];
+    __shared__ float red_m[AT_WARPS][AT_BM], red_l[AT_WARPS][AT_BM], red_kl[AT_WARPS][AT_BM];
+    __shared__ float lse_sh[AT_BM];
+    __shared__ float* prev_sh[AT_BM];
+    __shared__ int valid_sh[AT_BM];
+    const AttnArgs& a = g.a;
+    uint8_t* smem = (uint8_t*)(((uintptr_t)at_smem_raw + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int seq = blockIdx.x / g.tiles_per_seq, tile = blockIdx.x - seq * g.tiles_per_seq;
+    const int h = blockIdx.y;
+    const int g_kv = (h * a.n_kv) / a.n_heads;
+    const int dq = a.n_heads * AT_DH, dkv = a.n_kv * AT_DH;
+    const int row0 = seq * g.rows_per_seq + tile * AT_BM;
+    const int n_in_tile = min(AT_BM, g.rows_per_seq - tile * AT_BM);
+
+    uint8_t* q_s = smem + AT_WARPS * 2 * AT_STAGE_BYTES;
+    uint8_t* my_stage = smem + warp * 2 * AT_STAGE_BYTES;
+    const uint32_t q_u32 = (uint32_t)__cvta_generic_to_shared(q_s);
+    const uint32_t st_u32 = (uint32_t)__cvta_generic_to_shared(my_stage);
+
+    // ---- row bookkeeping + Q tile ----------------------------------------------------------
+    int kv_seq = seq;
+    if (threadIdx.x < AT_BM) {
+        const int i = threadIdx.x;
+        float* prev = nullptr;
+        int valid = 0;
+        if (i < n_in_tile) {
+            const int r = row0 + i;
+            if (a.rows) {
+                const Row rw = a.rows[r];
+                if (rw.pos >= 0) {
+                    valid = 1;
+                    if (rw.widx >= 0 && a.pprev) prev = a.pprev + (((size_t)rw.seq * a.W_max + rw.widx) * a.n_heads + h) * a.N;
+                    else if (rw.aidx >= 0 && a.aprev) prev = a.aprev + (((size_t)rw.seq * a.B + rw.aidx) * a.n_heads + h) * a.N;
+                }
+            } else {
+                valid = 1;
+                if (a.pprev) prev = a.pprev + ((size_t)r * a.n_heads + h) * a.N;
+            }
+        }
+        prev_sh[i] = prev;
+        valid_sh[i] = valid;
+    }
+    if (!a.rows) kv_seq = 0;
+    for (int t = threadIdx.x; t < AT_BM * 16; t += blockDim.x) {
+        const int i = t >> 4, ch = t & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (i < n_in_tile) v = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)a.q + (size_t)(row0 + i) * dq + h * AT_DH + ch * 8);
+        *reinterpret_cast<uint4*>(q_s + sw_off(i, ch)) = v;
+    }
+    __syncthreads();
+    // invalid rows may hold uninitialised q: zero them so no NaN/Inf enters the tile's arithmetic
+    for (int t = threadIdx.x; t < AT_BM * 16; t += blockDim.x) {
+        const int i = t >> 4, ch = t & 15;
+        if (!valid_sh[i]) *reinterpret_cast<uint4*>(q_s + sw_off(i, ch)) = make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+
+    uint32_t qf[8][4];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = lane >> 3, r = lane & 7;
+        ldsm_x4(q_u32 + sw_off((i & 1) * 8 + r, 2 * k + (i >> 1)), qf[k][0], qf[k][1], qf[k][2], qf[k][3]);
+    }
+
+    const __nv_bfloat16* Kg = (const __nv_bfloat16*)a.kc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
+    const __nv_bfloat16* Vg = (const __nv_bfloat16*)a.vc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
+    const int n_tiles = (a.N + AT_BN - 1) / AT_BN;
+    const int my_tiles = warp < n_tiles ? (n_tiles - warp + AT_WARPS - 1) / AT_WARPS : 0;
+
+    auto load_tile = [&](int t, int stage, bool with_v) {
+        const int key0 = t * AT_BN;
+        const uint32_t kb = st_u32 + stage * AT_STAGE_BYTES, vb = kb + AT_BN * AT_DH * 2;
+        for (int c = lane; c < AT_BN * 16; c += 32) {
+            const int r = c >> 4, ch = c & 15;
+            const int key = key0 + r;
+            const bool ok = key < a.N;
+            const size_t off = (size_t)(ok ? key : 0) * dkv + ch * 8;
+            cp_async16(kb + sw_off(r, ch), Kg + off, ok);
+            if (with_v) cp_async16(vb + sw_off(r, ch), Vg + off, ok);
+        }
+        cp_async_commit();
+    };
+    // scores of one 32-key tile: s[nt][0..3], nt = 0..3 (8 keys each)
+    auto scores = [&](int stage, float (*s)[4]) {
+        const uint32_t kb = st_u32 + stage * AT_STAGE_BYTES;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+#pragma unroll
+            for (int np = 0; np < 2; ++np) {
+                const int i = lane >> 3, r = lane & 7;
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(kb + sw_off((2 * np + (i >> 1)) * 8 + r, 2 * k + (i & 1)), b0, b1, b2, b3);
+                mma_bf16(s[2 * np], qf[k], b0, b1);
+                mma_bf16(s[2 * np + 1], qf[k], b2, b3);
+            }
+        }
+    };
+
+    const int r_lo = lane >> 2, r_hi = r_lo + 8;
+    const int cpair = (lane & 3) * 2;
+
+    // ---- pass 1: log-sum-exp -----------------------------------------------------------------
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    if (my_tiles > 0) load_tile(warp, 0, false);
+    for (int it = 0; it < my_tiles; ++it) {
+        const int t = warp + it * AT_WARPS;
+        if (it + 1 < my_tiles) { load_tile(t + AT_WARPS, (it + 1) & 1, false); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncwarp();
+        float s[4][4];
+        scores(it & 1, s);
+        float tm_lo = -INFINITY, tm_hi = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int key = t * AT_BN + nt * 8 + cpair + e;
+                const bool ok = key < a.N;
+                s[nt][e] = ok ? s[nt][e] * a.scale : -INFINITY;
+                s[nt][2 + e] = ok ? s[nt][2 + e] * a.scale : -INFINITY;
+                tm_lo = fmaxf(tm_lo, s[nt][e]);
+                tm_hi = fmaxf(tm_hi, s[nt][2 + e]);
+            }
+        }
+        tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 1));
+        tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 2));
+        tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 1));
+        tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 2));
+        const float nm_lo = fmaxf(m_lo, tm_lo), nm_hi = fmaxf(m_hi, tm_hi);
+        float sl = 0.f, sh = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e) { sl += expf(s[nt][e] - nm_lo); sh += expf(s[nt][2 + e] - nm_hi); }
+        }
+        sl += __shfl_xor_sync(0xffffffffu, sl, 1); sl += __shfl_xor_sync(0xffffffffu, sl, 2);
+        sh += __shfl_xor_sync(0xffffffffu, sh, 1); sh += __shfl_xor_sync(0xffffffffu, sh, 2);
+        l_lo = l_lo * expf(m_lo - nm_lo) + sl;
+        l_hi = l_hi * expf(m_hi - nm_hi) + sh;
+        m_lo = nm_lo; m_hi = nm_hi;
+        __syncwarp();
+    }
+    if ((lane & 3) == 0) {
+        red_m[warp][r_lo] = m_lo; red_l[warp][r_lo] = l_lo;
+        red_m[warp][r_hi] = m_hi; red_l[warp][r_hi] = l_hi;
+    }
+    __syncthreads();
+    if (threadIdx.x < AT_BM) {
+        const int i = threadIdx.x;
+        float mx = -INFINITY;
+        for (int w = 0; w < AT_WARPS; ++w) mx = fmaxf(mx, red_m[w][i]);
+        float sum = 0.f;
+        for (int w = 0; w < AT_WARPS; ++w)
+            if (red_l[w][i] > 0.f) sum += red_l[w][i] * expf(red_m[w][i] - mx);
+        lse_sh[i] = mx + logf(sum);
+    }
+    __syncthreads();
+    const float lse_lo = lse_sh[r_lo], lse_hi = lse_sh[r_hi];
+    float* prev_lo = prev_sh[r_lo];
+    float* prev_hi = prev_sh[r_hi];
+
+    // ---- pass 2: logp, KL, stored rows, P V ---------------------------------------------------
+    float o[16][4];
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+    float kl_lo = 0.f, kl_hi = 0.f;
+    if (my_tiles > 0) load_tile(warp, 0, true);
+    for (int it = 0; it < my_tiles; ++it) {
+        const int t = warp + it * AT_WARPS;
+        if (it + 1 < my_tiles) { load_tile(t + AT_WARPS, (it + 1) & 1, true); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncwarp();
+        float s[4][4];
+        scores(it & 1, s);
+        uint32_t pf[2][4];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt) {
+            float p[4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int key = t * AT_BN + nt * 8 + cpair + e;
+                const bool ok = key < a.N;
+                const float lp_lo = s[nt][e] * a.scale - lse_lo, lp_hi = s[nt][2 + e] * a.scale - lse_hi;
+                const float p_lo = ok ? expf(lp_lo) : 0.f, p_hi = ok ? expf(lp_hi) : 0.f;
+                if (ok && prev_lo) { if (a.record_kl) kl_lo += p_lo * (lp_lo - prev_lo[key]); prev_lo[key] = lp_lo; }
+                if (ok && prev_hi) { if (a.record_kl) kl_hi += p_hi * (lp_hi - prev_hi[key]); prev_hi[key] = lp_hi; }
+                p[e] = p_lo; p[2 + e] = p_hi;
+            }
+            pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
+            pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+        }
+        if (a.out) {
+            const uint32_t vb = st_u32 + (it & 1) * AT_STAGE_BYTES + AT_BN * AT_DH * 2;
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    const int i = lane >> 3, r = lane & 7;
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(vb + sw_off(ks * 16 + (i & 1) * 8 + r, 2 * dp + (i >> 1)), b0, b1, b2, b3);
+                    mma_bf16(o[2 * dp], pf[ks], b0, b1);
+                    mma_bf16(o[2 * dp + 1], pf[ks], b2, b3);
+                }
+            }
+        }
+        __syncwarp();
+    }
+    // ---- combine the warps' partial results (fixed order) ---------------------------------------
+    kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 1); kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 2);
+    kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 1); kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 2);
+    if ((lane & 3) == 0) { red_kl[warp][r_lo] = kl_lo; red_kl[warp][r_hi] = kl_hi; }
+    __syncthreads();       // every warp is done with its K/V stages: reuse them for the O partials
+    float* o_s = reinterpret_cast<float*>(smem);     // [warps][16][128] fp32 = 32 KB
+    if (a.out) {
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            const int col = nt * 8 + cpair;
+            float* b0 = o_s + ((size_t)warp * AT_BM + r_lo) * AT_DH + col;
+            float* b1 = o_s + ((size_t)warp * AT_BM + r_hi) * AT_DH + col;
+            b0[0] = o[nt][0]; b0[1] = o[nt][1]; b1[0] = o[nt][2]; b1[1] = o[nt][3];
+        }
+    }
+    __syncthreads();
+    if (a.out) {
+        for (int t = threadIdx.x; t < AT_BM * AT_DH / 2; t += blockDim.x) {
+            const int i = t / (AT_DH / 2), c = (t % (AT_DH / 2)) * 2;
+            if (!valid_sh[i]) continue;
+            float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+            for (int w = 0; w < AT_WARPS; ++w) {
+                v0 += o_s[((size_t)w * AT_BM + i) * AT_DH + c];
+                v1 += o_s[((size_t)w * AT_BM + i) * AT_DH + c + 1];
+            }
+            *reinterpret_cast<__nv_bfloat162*>((__nv_bfloat16*)a.out + (size_t)(row0 + i) * dq + h * AT_DH + c) =
+                __floats2bfloat162_rn(v0, v1);
+        }
+    }
+    if (a.kl && threadIdx.x < AT_BM && valid_sh[threadIdx.x]) {
+        const int i = threadIdx.x;
+        float kl = 0.f;
+        for (int w = 0; w < AT_WARPS; ++w) kl += red_kl[w][i];
+        a.kl[(size_t)(row0 + i) * a.n_heads + h] = (prev_sh[i] && a.record_kl) ? kl : 0.f;
+    }
+}
+
+static int launch_attention_mma(const AttnArgs& a, cudaStream_t st) {
+    AttnMmaArgs g;
+    g.a = a;
+    const int batch = a.batch > 0 ? a.batch : 1;
+    g.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : a.n_rows;
+    g.tiles_per_seq = (g.rows_per_seq + AT_BM - 1) / AT_BM;
+    static bool attr = false;
+    if (!attr) {
+        if (cudaFuncSetAttribute(attention_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM) != cudaSuccess)
+            return -4;
+        attr = true;
+    }
+    dim3 grid(g.tiles_per_seq * batch, a.n_heads);
+    attention_mma_kernel<<<grid, AT_WARPS * 32, AT_SMEM, st>>>(g);
+    return cudaGetLastError() == cudaSuccess ? 0 : -4;
+}
+
+}  // namespace ps

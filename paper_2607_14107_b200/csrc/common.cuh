@@ -1,0 +1,210 @@
+// Shared device-side definitions of the Polestar step kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ps {
+
+// ---- element types ---------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float to_f(T v);
+template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// value a GEMM operand of type T actually carries (identity for float)
+template <typename T> __device__ __forceinline__ float round_to(float v) { return to_f<T>(from_f<T>(v)); }
+
+// ---- rows of one forward -----------------------------------------------------------
+// One descriptor per forwarded row.  pos < 0 marks an unused slot.
+struct Row {
+    int seq;   // sequence in the batch
+    int pos;   // absolute position in the sequence, -1 = unused
+    int widx;  // index in the local window, -1 = not a window row
+    int aidx;  // index in the active block, -1 = not an active row
+};
+
+struct SeqFlags { unsigned char v[64]; };
+
+// Geometry of one forward (Algorithm 1: active block J_b, window Omega_b, entry set E_b).
+struct StepDesc {
+    int kind;          // 0 entry over the whole sequence, 1 entry over window+block, 2 within-block
+    int batch, N, B;
+    int act_start;     // first position of the active block
+    int W, n_pre;      // window rows, of which the first n_pre lie before the block
+    int pre_start;     // first position of the prefix part
+    int suf_start;     // first position of the suffix part
+    int W_max;         // row stride of the per-window buffers
+    int rows_per_seq;  // descriptors per sequence
+    int e0;            // entry steps: first forwarded position
+    int within;        // 1: window rows live in the hidden cache (within-block step)
+    int record_kl;     // 1: drift of recorded rows is measured against the stored rows
+    SeqFlags refresh;  // within-block: which sequences refresh their cache this step
+};
+
+__device__ __forceinline__ int window_pos(const StepDesc& sd, int w) {
+    return w < sd.n_pre ? sd.pre_start + w : sd.suf_start + (w - sd.n_pre);
+}
+__device__ __forceinline__ int window_index(const StepDesc& sd, int pos) {
+    if (pos >= sd.pre_start && pos < sd.pre_start + sd.n_pre) return pos - sd.pre_start;
+    if (pos >= sd.suf_start && pos < sd.suf_start + (sd.W - sd.n_pre)) return sd.n_pre + pos - sd.suf_start;
+    return -1;
+}
+
+// ---- reductions (fixed order => deterministic) --------------------------------------
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+// sum over the whole block; every thread gets the result.  red: >= 33 floats of shared memory.
+__device__ __forceinline__ float block_sum(float v, float* red) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) red[wid] = v;
+    __syncthreads();
+    if (wid == 0) {
+        float t = lane < nw ? red[lane] : 0.f;
+        t = warp_sum(t);
+        if (lane == 0) red[32] = t;
+    }
+    __syncthreads();
+    return red[32];
+}
+__device__ __forceinline__ float block_max(float v, float* red) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_max(v);
+    __syncthreads();
+    if (lane == 0) red[wid] = v;
+    __syncthreads();
+    if (wid == 0) {
+        float t = lane < nw ? red[lane] : -INFINITY;
+        t = warp_max(t);
+        if (lane == 0) red[32] = t;
+    }
+    __syncthreads();
+    return red[32];
+}
+
+// exclusive prefix sum of one int per thread over the block; returns the exclusive value,
+// *total gets the block total.  sc: >= 33 ints of shared memory.
+__device__ __forceinline__ int block_excl_scan(int v, int* sc, int* total) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+    }
+    __syncthreads();
+    if (lane == 31) sc[wid] = inc;
+    __syncthreads();
+    if (wid == 0) {
+        int t = lane < nw ? sc[lane] : 0;
+        int ti = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int u = __shfl_up_sync(0xffffffffu, ti, o);
+            if (lane >= o) ti += u;
+        }
+        if (lane < nw) sc[lane] = ti - t;
+        if (lane == 31) sc[32] = ti;
+    }
+    __syncthreads();
+    int res = inc - v + sc[wid];
+    *total = sc[32];
+    __syncthreads();
+    return res;
+}
+
+// ---- GEMM epilogues -------------------------------------------------------------------
+enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_DOWN = 3, EPI_LOGITS = 4, EPI_QKV_REFRESH = 5 };
+
+// Everything an epilogue may need; unused members are null.
+struct EpiArgs {
+    const Row* rows;          // descriptors of the GEMM's rows (QKV) / of the forward (DOWN)
+    const int* list;          // DOWN: compacted row -> forward row
+    const int* m_count;       // device-side row count (null: use the host bound)
+    const unsigned char* kvflag;  // QKV: write k,v of this row into the cache
+    const float2* rope;       // [N][head_dim/2] (cos, sin)
+    void* q_out;              // QKV: [rows][n_heads*head_dim]
+    void* kc; void* vc;       // cache of this layer [batch][N][n_kv*head_dim]
+    const float* resid;       // RESID / DOWN: residual rows [rows][d]
+    float* out_f32;           // RESID: out rows; DOWN: x rows; LOGITS: logits
+    float* packet;            // DOWN: packet rows [batch][W_max][d]
+    void* out_t;              // SWIGLU: [rows][d_ffn]
+    int N_seq, n_heads, n_kv, head_dim, W_max, within;
+    int ld_out;               // leading dimension of the main output
+    float scale;              // LOGITS
+    // QKV_REFRESH (stand-alone refresh kernel): row r of sequence s = r / max_rows
+    const int* idx; const int* counts; int max_rows; int P;
+};
+
+// One output pair (n even, n+1) of row m.
+template <typename T, int EPI>
+__device__ __forceinline__ void epilogue_pair(const EpiArgs& e, int m, int n, float v0, float v1) {
+    if (EPI == EPI_QKV || EPI == EPI_QKV_REFRESH) {
+        int seq, pos, kvf, qrow;
+        if (EPI == EPI_QKV) {
+            const Row rw = e.rows[m];
+            if (rw.pos < 0) return;
+            seq = rw.seq; pos = rw.pos; kvf = e.kvflag[m]; qrow = m;
+        } else {
+            seq = m / e.max_rows;
+            const int i = m - seq * e.max_rows;
+            if (i >= e.counts[seq]) return;
+            pos = e.idx[seq * e.max_rows + i]; kvf = 1; qrow = m;
+        }
+        const int dq = e.n_heads * e.head_dim, dkv = e.n_kv * e.head_dim;
+        const int Npos = (EPI == EPI_QKV) ? e.N_seq : e.P;
+        if (n < dq + dkv) {
+            const int p = n % e.head_dim;
+            const float2 cs = e.rope[(size_t)pos * (e.head_dim / 2) + (p >> 1)];
+            const float r0 = v0 * cs.x - v1 * cs.y;
+            const float r1 = v1 * cs.x + v0 * cs.y;
+            if (n < dq) {
+                if (e.q_out) {
+                    T* q = (T*)e.q_out + (size_t)qrow * dq + n;
+                    q[0] = from_f<T>(r0); q[1] = from_f<T>(r1);
+                }
+            } else if (kvf) {
+                T* k = (T*)e.kc + ((size_t)seq * Npos + pos) * dkv + (n - dq);
+                k[0] = from_f<T>(r0); k[1] = from_f<T>(r1);
+            }
+        } else if (kvf) {
+            T* v = (T*)e.vc + ((size_t)seq * Npos + pos) * dkv + (n - dq - dkv);
+            v[0] = from_f<T>(v0); v[1] = from_f<T>(v1);
+        }
+    } else if (EPI == EPI_RESID) {
+        const size_t o = (size_t)m * e.ld_out + n;
+        e.out_f32[o] = e.resid[o] + v0;
+        e.out_f32[o + 1] = e.resid[o + 1] + v1;
+    } else if (EPI == EPI_SWIGLU) {
+        const float g = v0 / (1.f + expf(-v0)) * v1;
+        ((T*)e.out_t)[(size_t)m * e.ld_out + (n >> 1)] = from_f<T>(g);
+    } else if (EPI == EPI_DOWN) {
+        const int r = e.list ? e.list[m] : m;
+        const Row rw = e.rows[r];
+        if (rw.pos < 0) return;
+        const size_t o = (size_t)r * e.ld_out + n;
+        const float a0 = e.resid[o] + v0, a1 = e.resid[o + 1] + v1;
+        float* dst = (e.within && rw.widx >= 0)
+                         ? e.packet + ((size_t)rw.seq * e.W_max + rw.widx) * e.ld_out + n
+                         : e.out_f32 + o;
+        dst[0] = a0; dst[1] = a1;
+    } else if (EPI == EPI_LOGITS) {
+        const size_t o = (size_t)m * e.ld_out + n;
+        e.out_f32[o] = v0 * e.scale;
+        e.out_f32[o + 1] = v1 * e.scale;
+    }
+}
+
+}  // namespace ps

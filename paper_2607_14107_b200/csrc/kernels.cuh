@@ -1,0 +1,773 @@
+// CUDA-core kernels of the Polestar step: row table, embedding, RMSNorm staging, a plain
+// tiled GEMM (fp32 models and debugging), attention with drift (fp32 models), select /
+// compaction, confidence and commit.
+#pragma once
+#include "common.cuh"
+
+namespace ps {
+
+// ---------------------------------------------------------------------------------------
+// Row table of one forward (Algorithm 1: E_b at block entry, J_b plus Omega_b within a block)
+// ---------------------------------------------------------------------------------------
+__global__ void build_rows_kernel(StepDesc sd, Row* rows) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int total = sd.batch * sd.rows_per_seq;
+    if (i >= total) return;
+    const int s = i / sd.rows_per_seq, j = i - s * sd.rows_per_seq;
+    Row r;
+    r.seq = s; r.pos = -1; r.widx = -1; r.aidx = -1;
+    if (sd.kind == 2) {
+        if (j < sd.B) {
+            r.pos = sd.act_start + j; r.aidx = j;
+        } else {
+            const int w = j - sd.B;
+            if (w < sd.W && sd.refresh.v[s]) { r.pos = window_pos(sd, w); r.widx = w; }
+        }
+    } else {
+        const int pos = sd.e0 + j;
+        if (pos < sd.N) {
+            r.pos = pos;
+            if (pos >= sd.act_start && pos < sd.act_start + sd.B) r.aidx = pos - sd.act_start;
+            else r.widx = window_index(sd, pos);
+        }
+    }
+    rows[i] = r;
+}
+
+// ---------------------------------------------------------------------------------------
+// Layer-0 inputs: embeddings of forwarded rows; on refresh steps the layer-0 packet holds the
+// embeddings of window positions whose token changed since their cached row was written
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_rows_kernel(StepDesc sd, const Row* rows, const int* y, const T* emb, int d,
+                                  float* x, float* packet, unsigned char* patch0, int* tok_at_h0,
+                                  int* stats) {
+    const int r = blockIdx.x;
+    const Row rw = rows[r];
+    if (rw.pos < 0) return;
+    const int tok = y[rw.seq * sd.N + rw.pos];
+    const T* e = emb + (size_t)tok * d;
+    if (sd.within && rw.widx >= 0) {
+        const int o = rw.seq * sd.W_max + rw.widx;
+        const bool changed = tok_at_h0[o] != tok;
+        if (changed) {
+            float* dst = packet + (size_t)o * d;
+            for (int c = threadIdx.x; c < d; c += blockDim.x) dst[c] = to_f<T>(e[c]);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            patch0[o] = changed ? 1 : 0;
+            tok_at_h0[o] = tok;
+            if (changed) atomicAdd(stats, 1);
+        }
+    } else {
+        float* dst = x + (size_t)r * d;
+        for (int c = threadIdx.x; c < d; c += blockDim.x) dst[c] = to_f<T>(e[c]);
+        if (!sd.within && rw.widx >= 0 && threadIdx.x == 0) tok_at_h0[rw.seq * sd.W_max + rw.widx] = tok;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Patch + RMSNorm + staging of the QKV projection's input rows (Algorithm 1 "Patch")
+//   window rows of a within-block step read the hidden cache (after taking the packet row if
+//   the previous layer selected them); every other row reads the residual stream x.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* hc, const float* packet,
+                                const unsigned char* patch, const float* gain, float eps, int d,
+                                T* a_out, unsigned char* kvflag) {
+    __shared__ float red[33];
+    const int r = blockIdx.x;
+    const Row rw = rows[r];
+    T* a = a_out + (size_t)r * d;
+    if (rw.pos < 0) {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
+        if (threadIdx.x == 0) kvflag[r] = 0;
+        return;
+    }
+    float* xr = x + (size_t)r * d;
+    const float* src = xr;
+    bool kv = true;
+    if (rw.widx >= 0) {
+        const size_t o = (size_t)rw.seq * sd.W_max + rw.widx;
+        float* h = hc + o * d;
+        if (sd.within) {
+            const bool patched = patch[o] != 0;
+            const float* u = packet + o * d;
+            for (int c = threadIdx.x; c < d; c += blockDim.x) {
+                const float v = patched ? u[c] : h[c];
+                if (patched) h[c] = v;
+                xr[c] = v;
+            }
+            kv = patched;
+        } else {
+            for (int c = threadIdx.x; c < d; c += blockDim.x) h[c] = xr[c];
+        }
+        __syncthreads();
+    }
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = src[c]; ss += v * v; }
+    ss = block_sum(ss, red);
+    const float inv = rsqrtf(ss / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(src[c] * inv * gain[c]);
+    if (threadIdx.x == 0) kvflag[r] = kv ? 1 : 0;
+}
+
+// RMSNorm of a compacted list of rows (FFN input, LM-head input).
+//   src row = list ? list[i] : i;  packet_rows: rows flagged as window rows read the packet
+template <typename T>
+__global__ void prep_rows_kernel(const float* x, const int* list, const int* m_count, const float* gain,
+                                 float eps, int d, T* a_out) {
+    __shared__ float red[33];
+    const int i = blockIdx.x;
+    T* a = a_out + (size_t)i * d;
+    if (m_count && i >= *m_count) {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
+        return;
+    }
+    const int r = list ? list[i] : i;
+    const float* src = x + (size_t)r * d;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = src[c]; ss += v * v; }
+    ss = block_sum(ss, red);
+    const float inv = rsqrtf(ss / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(src[c] * inv * gain[c]);
+}
+
+// LM-head input rows: entry i < n_act reads x[act_rows...]; later entries read packet rows.
+struct HeadSrc { int kind; int index; };  // kind 0: x row `index`; 1: packet row `index` (= seq*W_max+w)
+template <typename T>
+__global__ void prep_head_kernel(const float* x, const float* packet, const HeadSrc* src_list,
+                                 const int* m_count, const float* gain, float eps, int d, T* a_out) {
+    __shared__ float red[33];
+    const int i = blockIdx.x;
+    T* a = a_out + (size_t)i * d;
+    if (i >= *m_count) {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
+        return;
+    }
+    const HeadSrc hs = src_list[i];
+    const float* src = (hs.kind ? packet : x) + (size_t)hs.index * d;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = src[c]; ss += v * v; }
+    ss = block_sum(ss, red);
+    const float inv = rsqrtf(ss / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(src[c] * inv * gain[c]);
+}
+
+// Gather + RMSNorm for the stand-alone refresh kernel: row (s, i) <- h[s][idx[s][i]].
+template <typename T>
+__global__ void prep_refresh_kernel(const T* h, const int* idx, const int* counts, int max_rows, int P,
+                                    const float* gain, float eps, int d, T* a_out) {
+    __shared__ float red[33];
+    const int m = blockIdx.x;
+    const int s = m / max_rows, i = m - s * max_rows;
+    T* a = a_out + (size_t)m * d;
+    if (i >= counts[s]) {
+        for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
+        return;
+    }
+    const T* src = h + ((size_t)s * P + idx[s * max_rows + i]) * d;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = to_f<T>(src[c]); ss += v * v; }
+    ss = block_sum(ss, red);
+    const float inv = rsqrtf(ss / (float)d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(to_f<T>(src[c]) * inv * gain[c]);
+}
+
+// ---------------------------------------------------------------------------------------
+// Plain tiled GEMM on CUDA cores: out[m][n] = sum_k A[m][k] W[n][k], fp32 accumulate.
+// 64x64 tile, 16-wide K slices, 256 threads, 4x4 outputs per thread.
+// ---------------------------------------------------------------------------------------
+template <typename T, int EPI>
+__global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ Wt,
+                                                        int M, int Nout, int K, EpiArgs e) {
+    __shared__ float As[16][64 + 4];
+    __shared__ float Ws[16][64 + 4];
+    const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
+    const int Mv = e.m_count ? min(M, *e.m_count) : M;
+    if (m0 >= Mv) return;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int k0 = 0; k0 < K; k0 += 16) {
+        for (int t = threadIdx.x; t < 64 * 16; t += 256) {
+            const int rr = t >> 4, kk = t & 15;
+            const int m = m0 + rr, n = n0 + rr, k = k0 + kk;
+            As[kk][rr] = (m < M && k < K) ? to_f<T>(A[(size_t)m * K + k]) : 0.f;
+            Ws[kk][rr] = (n < Nout && k < K) ? to_f<T>(Wt[(size_t)n * K + k]) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = Ws[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= Mv) continue;
+#pragma unroll
+        for (int j = 0; j < 4; j += 2) {
+            const int n = n0 + tx * 4 + j;
+            if (n + 1 < Nout) epilogue_pair<T, EPI>(e, m, n, acc[i][j], acc[i][j + 1]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Attention rows with drift, CUDA-core version: one warp per (row, head).
+//   logp_j = s_j - logsumexp(s), s_j = q.k_j / sqrt(dh) over all N cache rows (Eq. 3, no mask);
+//   out = sum_j p_j v_j;  recorded rows: kl = sum_j p_j (logp_j - prev_j), prev <- logp (Eq. 4).
+// Dynamic shared memory: warps_per_block * N floats.
+// ---------------------------------------------------------------------------------------
+struct AttnArgs {
+    const Row* rows; int n_rows;
+    const void* q; const void* kc; const void* vc; void* out;
+    float* pprev;    // window rows: [batch][W_max][n_heads][N]   (null: none recorded)
+    float* aprev;    // active rows: [batch][B][n_heads][N]       (null: none recorded)
+    float* kl;       // [n_rows][n_heads]
+    int N, n_heads, n_kv, head_dim, W_max, B, record_kl;
+    int rows_per_seq, batch;   // layout of the forward's rows (stand-alone: n_rows, 1)
+    float scale;
+    // stand-alone form: rows == null, row r belongs to sequence 0 and records into pprev[r]
+};
+
+template <typename T>
+__global__ void attention_simt_kernel(AttnArgs a) {
+    extern __shared__ float sm[];
+    const int wpb = blockDim.x >> 5, wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int r = blockIdx.x * wpb + wid, h = blockIdx.y;
+    if (r >= a.n_rows) return;
+    int seq = 0;
+    float* prev = nullptr;
+    if (a.rows) {
+        const Row rw = a.rows[r];
+        if (rw.pos < 0) return;
+        seq = rw.seq;
+        if (rw.widx >= 0 && a.pprev) prev = a.pprev + (((size_t)seq * a.W_max + rw.widx) * a.n_heads + h) * a.N;
+        else if (rw.aidx >= 0 && a.aprev) prev = a.aprev + (((size_t)seq * a.B + rw.aidx) * a.n_heads + h) * a.N;
+    } else if (a.pprev) {
+        prev = a.pprev + ((size_t)r * a.n_heads + h) * a.N;
+    }
+    float* sc = sm + (size_t)wid * a.N;
+    const int dh = a.head_dim, g = (h * a.n_kv) / a.n_heads;
+    const int dq = a.n_heads * dh, dkv = a.n_kv * dh;
+    const T* q = (const T*)a.q + (size_t)r * dq + h * dh;
+    const T* K = (const T*)a.kc + (size_t)seq * a.N * dkv + g * dh;
+    const T* V = (const T*)a.vc + (size_t)seq * a.N * dkv + g * dh;
+    // scores
+    float mx = -INFINITY;
+    for (int j = lane; j < a.N; j += 32) {
+        const T* kj = K + (size_t)j * dkv;
+        float s = 0.f;
+        for (int c = 0; c < dh; ++c) s = fmaf(to_f<T>(q[c]), to_f<T>(kj[c]), s);
+        s *= a.scale;
+        sc[j] = s;
+        mx = fmaxf(mx, s);
+    }
+    mx = warp_max(mx);
+    float sum = 0.f;
+    for (int j = lane; j < a.N; j += 32) sum += expf(sc[j] - mx);
+    sum = warp_sum(sum);
+    const float lse = mx + logf(sum);
+    float kl = 0.f;
+    for (int j = lane; j < a.N; j += 32) {
+        const float lp = sc[j] - lse;
+        const float p = expf(lp);
+        if (prev) {
+            if (a.record_kl) kl += p * (lp - prev[j]);
+            prev[j] = lp;
+        }
+        sc[j] = round_to<T>(p);
+    }
+    __syncwarp();
+    if (a.kl) {
+        kl = warp_sum(kl);
+        if (lane == 0) a.kl[(size_t)r * a.n_heads + h] = (prev && a.record_kl) ? kl : 0.f;
+    }
+    if (a.out) {
+        T* o = (T*)a.out + (size_t)r * dq + h * dh;
+        for (int c = lane; c < dh; c += 32) {
+            float acc = 0.f;
+            for (int j = 0; j < a.N; ++j) acc = fmaf(sc[j], to_f<T>(V[(size_t)j * dkv + c]), acc);
+            o[c] = from_f<T>(acc);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Squared hidden-state change per row (Appendix B, Cor. 1): one warp per row, 128-bit loads.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void hidden_delta_kernel(const T* __restrict__ a, const T* __restrict__ b, float* out, int rows, int d) {
+    const int wpb = blockDim.x >> 5, wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per = 16 / (int)sizeof(T);
+    for (int r = blockIdx.x * wpb + wid; r < rows; r += gridDim.x * wpb) {
+        const uint4* pa = reinterpret_cast<const uint4*>(a + (size_t)r * d);
+        const uint4* pb = reinterpret_cast<const uint4*>(b + (size_t)r * d);
+        float acc = 0.f;
+        const int nv = d / per;
+        for (int i = lane; i < nv; i += 32) {
+            const uint4 ua = __ldg(pa + i), ub = __ldg(pb + i);
+            const T* ea = reinterpret_cast<const T*>(&ua);
+            const T* eb = reinterpret_cast<const T*>(&ub);
+#pragma unroll
+            for (int t = 0; t < per; ++t) { const float dd = to_f<T>(ea[t]) - to_f<T>(eb[t]); acc = fmaf(dd, dd, acc); }
+        }
+        for (int c = nv * per + lane; c < d; c += 32) {
+            const float dd = to_f<T>(a[(size_t)r * d + c]) - to_f<T>(b[(size_t)r * d + c]);
+            acc = fmaf(dd, dd, acc);
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) out[r] = acc;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Stale-row selection + compaction for one sequence (Sec. 4.1; Algorithm 1 "TopK").
+// Block-wide radix select of the k-th largest drift, ties to the lower index, then a
+// prefix-sum compaction to an ascending index list.  W <= SEL_MAX_W.
+// ---------------------------------------------------------------------------------------
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_ITEMS = 4;
+constexpr int SEL_MAX_W = SEL_THREADS * SEL_ITEMS;
+
+struct SelSmem {
+    int hist[256];
+    int scan[33];
+    unsigned prefix; int kleft; int total;
+};
+
+__device__ __forceinline__ unsigned float_key(float v) {   // order-preserving map to unsigned
+    const unsigned u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// D[i] valid for i < W.  Writes idx_out[0..count) ascending and (optional) flag_out[i] in {0,1}.
+// Returns count (same value in every thread).  Must be called by all SEL_THREADS threads.
+__device__ int select_one(const float* D, int W, int mode, int k, float thresh, float floor_,
+                          int* idx_out, unsigned char* flag_out, SelSmem& s) {
+    const int t = threadIdx.x;
+    unsigned key[SEL_ITEMS];
+    float val[SEL_ITEMS];
+    bool cand[SEL_ITEMS], sel[SEL_ITEMS];
+    // items are blocked: thread t owns indices t*ITEMS .. t*ITEMS+ITEMS-1 (keeps index order in scans)
+#pragma unroll
+    for (int u = 0; u < SEL_ITEMS; ++u) {
+        const int i = t * SEL_ITEMS + u;
+        const float v = i < W ? D[i] : 0.f;
+        cand[u] = (i < W) && (v > floor_);          // NaN compares false: never a candidate
+        val[u] = v;
+        key[u] = float_key(v);
+        sel[u] = false;
+    }
+    int ncand_local = 0;
+#pragma unroll
+    for (int u = 0; u < SEL_ITEMS; ++u) ncand_local += cand[u];
+    int ncand;
+    block_excl_scan(ncand_local, s.scan, &ncand);
+    if (mode == 3) {                                  // ALL: every row
+#pragma unroll
+        for (int u = 0; u < SEL_ITEMS; ++u) sel[u] = (t * SEL_ITEMS + u) < W;
+    } else if (mode == 2) {                           // THRESHOLD
+#pragma unroll
+        for (int u = 0; u < SEL_ITEMS; ++u) sel[u] = cand[u] && (val[u] > thresh);
+    } else if (mode == 4 || k <= 0) {                 // NONE
+    } else if (k >= ncand) {
+#pragma unroll
+        for (int u = 0; u < SEL_ITEMS; ++u) sel[u] = cand[u];
+    } else {
+        // radix select, most significant byte first
+        if (t == 0) { s.prefix = 0u; s.kleft = k; }
+        __syncthreads();
+        for (int pass = 0; pass < 4; ++pass) {
+            const int shift = 24 - 8 * pass;
+            const unsigned himask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+            if (t < 256) s.hist[t] = 0;
+            __syncthreads();
+            const unsigned prefix = s.prefix;
+#pragma unroll
+            for (int u = 0; u < SEL_ITEMS; ++u)
+                if (cand[u] && (key[u] & himask) == prefix) atomicAdd(&s.hist[(key[u] >> shift) & 255u], 1);
+            __syncthreads();
+            if (t == 0) {
+                int left = s.kleft, bsel = 0;
+                for (int bkt = 255; bkt >= 0; --bkt) {
+                    const int c = s.hist[bkt];
+                    if (c >= left) { bsel = bkt; break; }
+                    left -= c;
+                }
+                s.kleft = left;
+                s.prefix = prefix | ((unsigned)bsel << shift);
+            }
+            __syncthreads();
+        }
+        const unsigned kth = s.prefix;     // key of the k-th largest candidate
+        const int need_eq = s.kleft;       // how many rows equal to it are taken (lowest indices)
+        int eq_local = 0;
+#pragma unroll
+        for (int u = 0; u < SEL_ITEMS; ++u) eq_local += (cand[u] && key[u] == kth);
+        int eq_total;
+        int eq_before = block_excl_scan(eq_local, s.scan, &eq_total);
+#pragma unroll
+        for (int u = 0; u < SEL_ITEMS; ++u) {
+            if (!cand[u]) continue;
+            if (key[u] > kth) sel[u] = true;
+            else if (key[u] == kth) { sel[u] = eq_before < need_eq; ++eq_before; }
+        }
+    }
+    int nsel_local = 0;
+#pragma unroll
+    for (int u = 0; u < SEL_ITEMS; ++u) nsel_local += sel[u];
+    int count;
+    int off = block_excl_scan(nsel_local, s.scan, &count);
+#pragma unroll
+    for (int u = 0; u < SEL_ITEMS; ++u) {
+        const int i = t * SEL_ITEMS + u;
+        if (i < W && flag_out) flag_out[i] = sel[u] ? 1 : 0;
+        if (sel[u]) idx_out[off++] = i;
+    }
+    __syncthreads();
+    return count;
+}
+
+__global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* drift, int W, int mode, int k,
+                                                             float thresh, float floor_, int* idx, int* count) {
+    __shared__ SelSmem s;
+    const int b = blockIdx.x;
+    const int c = select_one(drift + (size_t)b * W, W, mode, k, thresh, floor_, idx + (size_t)b * W, nullptr, s);
+    if (threadIdx.x == 0) count[b] = c;
+}
+
+// In-step selection for every refreshing sequence, plus the compacted row list of the sparse
+// forward: all valid non-window rows followed by the selected window rows.
+struct StepSelArgs {
+    const float* kl;            // [rows][n_heads] per-head drift of the forward's rows
+    float* drift;               // [batch][W_max] (output, this layer)
+    int* sel_idx; int* sel_cnt; // this layer: [batch][W_max], [batch]
+    unsigned char* flag_next;   // patch flags of the next layer [batch][W_max]
+    const int* forced_idx; const int* forced_cnt;   // this layer (cnt < 0: not forced)
+    int* list; int* list_count; // compacted rows of the sparse forward
+    int* stats;                 // [0] += refreshed rows
+    int n_heads, mode, k, W_max;
+    float thresh, floor_;
+};
+
+__global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, StepSelArgs a) {
+    __shared__ SelSmem s;
+    __shared__ float dsh[SEL_MAX_W > 1024 ? 1024 : SEL_MAX_W];
+    __shared__ int base;
+    const int t = threadIdx.x;
+    const int nb = sd.batch * sd.B;
+    // active rows first (row id = s*rows_per_seq + j)
+    for (int i = t; i < nb; i += blockDim.x) a.list[i] = (i / sd.B) * sd.rows_per_seq + (i % sd.B);
+    if (t == 0) base = nb;
+    __syncthreads();
+    for (int sq = 0; sq < sd.batch; ++sq) {
+        if (!sd.refresh.v[sq]) {
+            if (t == 0) a.sel_cnt[sq] = 0;
+            continue;
+        }
+        for (int w = t; w < sd.W; w += blockDim.x) {
+            const float* kr = a.kl + (size_t)(sq * sd.rows_per_seq + sd.B + w) * a.n_heads;
+            float acc = 0.f;
+            for (int h = 0; h < a.n_heads; ++h) acc += kr[h];
+            const float dv = acc / (float)a.n_heads;
+            dsh[w] = dv;
+            a.drift[sq * a.W_max + w] = dv;
+        }
+        __syncthreads();
+        int* idx = a.sel_idx + sq * a.W_max;
+        unsigned char* fl = a.flag_next + sq * a.W_max;
+        int cnt;
+        const int fc = a.forced_cnt ? a.forced_cnt[sq] : -1;
+        if (fc >= 0) {
+            for (int w = t; w < sd.W; w += blockDim.x) fl[w] = 0;
+            __syncthreads();
+            for (int i = t; i < fc; i += blockDim.x) { const int w = a.forced_idx[sq * a.W_max + i]; idx[i] = w; fl[w] = 1; }
+            cnt = fc;
+            __syncthreads();
+        } else {
+            cnt = select_one(dsh, sd.W, a.mode, a.k, a.thresh, a.floor_, idx, fl, s);
+        }
+        const int b0 = base;
+        for (int i = t; i < cnt; i += blockDim.x) a.list[b0 + i] = sq * sd.rows_per_seq + sd.B + idx[i];
+        __syncthreads();
+        if (t == 0) { a.sel_cnt[sq] = cnt; base = b0 + cnt; atomicAdd(a.stats, cnt); }
+        __syncthreads();
+    }
+    if (t == 0) *a.list_count = base;
+}
+
+// ---------------------------------------------------------------------------------------
+// LM-head row list: every active row, then (refresh steps with suffix commit) the rows the last
+// layer selected that lie in the suffix window and are still masked (Sec. 4.2 "Suffix Block Commit")
+// ---------------------------------------------------------------------------------------
+__global__ void build_head_list_kernel(StepDesc sd, const int* y, int mask_id, const int* sel_idx,
+                                       const int* sel_cnt, int use_suffix, int act_row0_stride,
+                                       HeadSrc* list, int* count, int* suf_seq, int* suf_w) {
+    // act_row0_stride: forward row of active j in sequence s = s*rows_per_seq + (act offset) + j
+    const int t = threadIdx.x;
+    const int nb = sd.batch * sd.B;
+    const int act_off = sd.kind == 2 ? 0 : (sd.act_start - sd.e0);
+    for (int i = t; i < nb; i += blockDim.x) {
+        HeadSrc h; h.kind = 0; h.index = (i / sd.B) * sd.rows_per_seq + act_off + (i % sd.B);
+        list[i] = h;
+    }
+    __syncthreads();
+    if (t == 0) {
+        int n = nb;
+        if (use_suffix) {
+            for (int s = 0; s < sd.batch; ++s) {
+                if (!sd.refresh.v[s]) continue;
+                const int c = sel_cnt[s];
+                for (int i = 0; i < c; ++i) {
+                    const int w = sel_idx[s * sd.W_max + i];
+                    if (w < sd.n_pre) continue;
+                    const int pos = window_pos(sd, w);
+                    if (y[s * sd.N + pos] != mask_id) continue;
+                    HeadSrc h; h.kind = 1; h.index = s * sd.W_max + w;
+                    list[n] = h; suf_seq[n - nb] = s; suf_w[n - nb] = w;
+                    ++n;
+                }
+            }
+        }
+        *count = n;
+    }
+    (void)act_row0_stride;
+}
+
+// ---------------------------------------------------------------------------------------
+// Confidence of logits rows (Eq. 1 and the confidence of Sec. 2): two stages.
+// ---------------------------------------------------------------------------------------
+struct ConfPart { float mx_all; float sum; float mx_ex; int arg_ex; };
+
+__global__ void conf_partial_kernel(const float* logits, const int* m_count, int rows, int V, int mask_id,
+                                    int chunks, ConfPart* part) {
+    __shared__ float red[33];
+    __shared__ float bv[32];
+    __shared__ int bi[32];
+    const int r = blockIdx.y, ch = blockIdx.x;
+    if (r >= rows || (m_count && r >= *m_count)) return;
+    const int per = ((V + chunks - 1) / chunks + 3) & ~3;
+    const int v0 = ch * per, v1 = min(V, v0 + per);
+    const float* l = logits + (size_t)r * V;
+    float mx = -INFINITY, mxe = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
+        const float x = l[v];
+        mx = fmaxf(mx, x);
+        if (v != mask_id && (x > mxe || (x == mxe && v < arg))) { mxe = x; arg = v; }
+    }
+    const float bmx = block_max(mx, red);
+    float sum = 0.f;
+    for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) sum += expf(l[v] - bmx);
+    sum = block_sum(sum, red);
+    // argmax with lowest id on ties
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, mxe, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, arg, o);
+        if (ov > mxe || (ov == mxe && oi < arg)) { mxe = ov; arg = oi; }
+    }
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    if (lane == 0) { bv[wid] = mxe; bi[wid] = arg; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < nw; ++w)
+            if (bv[w] > mxe || (bv[w] == mxe && bi[w] < arg)) { mxe = bv[w]; arg = bi[w]; }
+        ConfPart p; p.mx_all = bmx; p.sum = (v1 > v0) ? sum : 0.f; p.mx_ex = mxe; p.arg_ex = arg;
+        part[(size_t)r * chunks + ch] = p;
+    }
+}
+
+__global__ void conf_final_kernel(const ConfPart* part, const int* m_count, int rows, int chunks,
+                                  int* yhat, float* conf) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows || (m_count && r >= *m_count)) return;
+    const ConfPart* p = part + (size_t)r * chunks;
+    float mx = -INFINITY, mxe = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int c = 0; c < chunks; ++c) {
+        mx = fmaxf(mx, p[c].mx_all);
+        if (p[c].mx_ex > mxe || (p[c].mx_ex == mxe && p[c].arg_ex < arg)) { mxe = p[c].mx_ex; arg = p[c].arg_ex; }
+    }
+    float sum = 0.f;
+    for (int c = 0; c < chunks; ++c)
+        if (p[c].sum > 0.f) sum += p[c].sum * expf(p[c].mx_all - mx);
+    yhat[r] = arg;
+    conf[r] = expf(mxe - mx) / sum;
+}
+
+// ---------------------------------------------------------------------------------------
+// Commit rule (Sec. 4.2; Algorithm 1 after the layer loop; Eq. 2): one block per sequence.
+// ---------------------------------------------------------------------------------------
+struct CommitArgs {
+    int* y;                      // [batch][N]
+    const float* conf; const int* yhat;   // LM rows: active rows first ([batch*B]), then suffix rows
+    const float* kl;             // per-head drift of the forward's rows (last layer) [rows][n_heads]
+    float* delta_out;            // [batch][B]
+    float* Delta_out; float* taud_out;
+    float* theta; int* theta_cnt;   // [batch][hist][B] ring, [batch] number pushed so far
+    int* commit_flags;           // [batch][B]
+    int* suffix_flags;           // [batch][W_max]
+    const int* head_count; const int* suf_seq; const int* suf_w;
+    const int* forced_pos; int forced_n;      // [batch][forced_n] absolute positions, -1 unused (null: free-running)
+    int* seq_info;               // [batch][8]: committed, by_conf, by_drift, by_quota, suffix, eos, masked_left, nonfinite
+    int n_heads, hist, mask_id, eos_id, act_row_off, steps_used, steps_per_block, use_drift, use_suffix, ge;
+    float tau_s, alpha, tau_suffix;
+};
+
+__global__ void commit_kernel(StepDesc sd, CommitArgs a) {
+    __shared__ float s_conf[256];
+    __shared__ unsigned char s_masked[256], s_flag[256];
+    __shared__ int cnt[8];
+    const int s = blockIdx.x, j = threadIdx.x, B = sd.B;
+    if (j < 8) cnt[j] = 0;
+    __syncthreads();
+    const bool within = sd.record_kl != 0;
+    float c = 0.f, dl = 0.f, Dl = 0.f, td = 0.f;
+    int tok = 0, yh = 0;
+    bool masked = false;
+    int flag = 0;
+    if (j < B) {
+        tok = a.y[s * sd.N + sd.act_start + j];
+        masked = tok == a.mask_id;
+        c = a.conf[s * B + j];
+        yh = a.yhat[s * B + j];
+        if (within) {
+            const float* kr = a.kl + (size_t)(s * sd.rows_per_seq + a.act_row_off + j) * a.n_heads;
+            float acc = 0.f;
+            for (int h = 0; h < a.n_heads; ++h) acc += kr[h];
+            dl = acc / (float)a.n_heads;
+            const int pushed = a.theta_cnt[s];
+            const int nh = min(pushed, a.hist);
+            float mean = 0.f;
+            if (nh > 0) {
+                // oldest to newest, like a running list
+                for (int u = 0; u < nh; ++u) mean += a.theta[((size_t)s * a.hist + ((pushed - nh + u) % a.hist)) * B + j];
+                mean /= (float)nh;
+            }
+            Dl = dl - mean;
+            if (a.hist > 0) a.theta[((size_t)s * a.hist + (pushed % a.hist)) * B + j] = dl;
+        }
+        td = a.alpha * (a.tau_s - c) * (a.tau_s - c);
+        if (masked) {
+            if (!(c == c)) atomicAdd(&cnt[7], 1);
+            const bool c_ok = a.ge ? (c >= a.tau_s) : (c > a.tau_s);
+            const bool d_ok = within && a.use_drift && (a.ge ? (Dl >= td) : (Dl > td));
+            if (c_ok) flag = 1 | 2;
+            else if (d_ok) flag = 1 | 4;
+        }
+        a.delta_out[s * B + j] = dl;
+        a.Delta_out[s * B + j] = Dl;
+        a.taud_out[s * B + j] = td;
+        s_conf[j] = c; s_masked[j] = masked; s_flag[j] = (unsigned char)flag;
+        if (masked) atomicAdd(&cnt[6], 1);
+        if (flag) atomicAdd(&cnt[0], 1);
+    }
+    __syncthreads();
+    if (j == 0 && within && a.hist > 0) a.theta_cnt[s] = a.theta_cnt[s] + 1;
+    const int n_masked = cnt[6];
+    if (a.forced_pos) {
+        if (j < B) {
+            flag = 0;
+            const int pos = sd.act_start + j;
+            for (int u = 0; u < a.forced_n; ++u)
+                if (a.forced_pos[s * a.forced_n + u] == pos) flag = s_flag[j] ? s_flag[j] : (1 | 8);
+            if (!masked) flag = 0;
+        }
+    } else {
+        // quota top-up: the most confident masked rows not yet committed (ties: lowest position)
+        const int denom = max(1, a.steps_per_block - a.steps_used);
+        const int quota = n_masked > 0 ? (n_masked + denom - 1) / denom : 0;
+        const int need = quota - cnt[0];
+        if (need > 0 && j < B && masked && !flag) {
+            int rank = 0;
+            for (int u = 0; u < B; ++u)
+                if (s_masked[u] && !s_flag[u] && (s_conf[u] > c || (s_conf[u] == c && u < j))) ++rank;
+            if (rank < need) flag = 1 | 8;
+        }
+    }
+    __syncthreads();
+    if (j < 6) cnt[j] = 0;
+    __syncthreads();
+    if (j < B) {
+        a.commit_flags[s * B + j] = flag;
+        if (flag & 1) {
+            a.y[s * sd.N + sd.act_start + j] = yh;
+            atomicAdd(&cnt[0], 1);
+            if (flag & 2) atomicAdd(&cnt[1], 1);
+            if (flag & 4) atomicAdd(&cnt[2], 1);
+            if (flag & 8) atomicAdd(&cnt[3], 1);
+            if (yh == a.eos_id) atomicAdd(&cnt[5], 1);
+        }
+    }
+    // suffix rows of the final packet: confidence alone decides
+    for (int w = j; w < sd.W_max; w += blockDim.x) a.suffix_flags[s * sd.W_max + w] = 0;
+    __syncthreads();
+    if (a.use_suffix && within) {
+        const int n_suf = *a.head_count - sd.batch * B;
+        for (int i = j; i < n_suf; i += blockDim.x) {
+            if (a.suf_seq[i] != s) continue;
+            const int w = a.suf_w[i];
+            const int pos = window_pos(sd, w);
+            const float sc = a.conf[sd.batch * B + i];
+            bool ok = a.ge ? (sc >= a.tau_suffix) : (sc > a.tau_suffix);
+            if (a.forced_pos) {
+                ok = false;
+                for (int u = 0; u < a.forced_n; ++u) if (a.forced_pos[s * a.forced_n + u] == pos) ok = true;
+            }
+            int f = 1;
+            if (ok && a.y[s * sd.N + pos] == a.mask_id) {
+                const int t2 = a.yhat[sd.batch * B + i];
+                a.y[s * sd.N + pos] = t2;
+                f |= 2;
+                atomicAdd(&cnt[0], 1); atomicAdd(&cnt[4], 1);
+                if (t2 == a.eos_id) atomicAdd(&cnt[5], 1);
+            }
+            a.suffix_flags[s * sd.W_max + w] = f;
+        }
+    }
+    __syncthreads();
+    if (j == 0) {
+        int* o = a.seq_info + s * 8;
+        o[0] = cnt[0]; o[1] = cnt[1]; o[2] = cnt[2]; o[3] = cnt[3]; o[4] = cnt[4]; o[5] = cnt[5];
+        o[6] = n_masked - (cnt[0] - cnt[4]);
+        o[7] = cnt[7];
+    }
+}
+
+// gather rows of x into a keep buffer: dst[s][j][:] = x[row(s, j)][:]
+__global__ void keep_hidden_kernel(StepDesc sd, const float* x, int act_row_off, int d, float* dst) {
+    const int i = blockIdx.x;
+    const int s = i / sd.B, j = i - s * sd.B;
+    const float* src = x + (size_t)(s * sd.rows_per_seq + act_row_off + j) * d;
+    float* o = dst + (size_t)i * d;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = src[c];
+}
+
+// rotary table: tab[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), computed in double precision
+__global__ void rope_table_kernel(float2* tab, int N, int half, double theta) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= N * half) return;
+    const int pos = i / half, k = i - pos * half;
+    const double inv = pow(theta, -(double)k / (double)half);
+    const double ang = (double)pos * inv;
+    tab[i] = make_float2((float)cos(ang), (float)sin(ang));
+}
+
+}  // namespace ps

@@ -1,0 +1,872 @@
+// Host side of the Polestar C ABI: workspace plan, controller (Algorithm 1's outer loops and
+// the update schedule of Sec. 4.1), kernel sequencing of one forward, read-back.
+#include "../../include/polestar.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <climits>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <new>
+#include <tuple>
+#include <vector>
+
+#include "attn_mma.cuh"
+#include "gemm_tc.cuh"
+#include "kernels.cuh"
+
+using namespace ps;
+
+#define CK(call)                                             \
+    do {                                                     \
+        cudaError_t _e = (call);                             \
+        if (_e != cudaSuccess) { last_cuda_error = _e; return POLESTAR_E_CUDA; } \
+    } while (0)
+
+static thread_local cudaError_t last_cuda_error = cudaSuccess;
+static int g_sm_count = 0;
+
+// ------------------------------------------------------------------------------------------
+// tensor maps (TMA descriptors) through the driver entry point, no libcuda link dependency
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+// bf16 matrix [rows, K] row-major, box = box_rows x 64 elements, 128-byte swizzle
+static bool make_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t K, uint32_t box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {K, rows};
+    cuuint64_t strides[1] = {K * 2};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct MapCache {
+    std::map<std::tuple<const void*, uint64_t, uint64_t, uint32_t>, CUtensorMap> m;
+    const CUtensorMap* get(const void* base, uint64_t rows, uint64_t K, uint32_t box_rows) {
+        auto key = std::make_tuple(base, rows, K, box_rows);
+        auto it = m.find(key);
+        if (it != m.end()) return &it->second;
+        CUtensorMap tm;
+        if (!make_map(&tm, base, rows, K, box_rows)) return nullptr;
+        return &m.emplace(key, tm).first->second;
+    }
+};
+
+// ------------------------------------------------------------------------------------------
+// GEMM dispatch
+// ------------------------------------------------------------------------------------------
+struct GemmWs {
+    float* partial = nullptr; size_t partial_bytes = 0;
+    int* counters = nullptr; int n_counters = 0;
+    int* status = nullptr;
+};
+
+static int env_int(const char* name, int dflt) {
+    const char* s = getenv(name);
+    return s ? atoi(s) : dflt;
+}
+
+template <typename T, int EPI>
+static int launch_gemm_simt(const void* A, const void* W, int M, int N_out, int K, const EpiArgs& e, cudaStream_t st) {
+    if (M <= 0) return POLESTAR_OK;
+    dim3 grid((N_out + 63) / 64, (M + 63) / 64);
+    gemm_simt_kernel<T, EPI><<<grid, 256, 0, st>>>((const T*)A, (const T*)W, M, N_out, K, e);
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
+}
+
+template <int EPI>
+static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a_rows_alloc, const void* W, int M,
+                          int N_out, int K, const EpiArgs& e, cudaStream_t st) {
+    if (M <= 0) return POLESTAR_OK;
+    const int NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    const CUtensorMap* mw = maps.get(W, (uint64_t)N_out, (uint64_t)K, 128);
+    const CUtensorMap* ma = maps.get(A, (uint64_t)a_rows_alloc, (uint64_t)K, (uint32_t)NT);
+    if (!mw || !ma) return POLESTAR_E_CUDA;
+    tc::GemmArgs g;
+    g.M = M; g.N_out = N_out; g.K = K; g.NT = NT;
+    const int tiles_f = N_out / 128, tiles_t = (M + NT - 1) / NT;
+    const int kb = K / 64;
+    const int stage_bytes = 128 * 64 * 2 + NT * 64 * 2;
+    const int smem_budget = env_int("POLESTAR_GEMM_SMEM", 100 * 1024);
+    int stages = std::max(2, std::min(12, smem_budget / stage_bytes));
+    stages = env_int("POLESTAR_GEMM_STAGES", stages);
+    stages = std::max(2, std::min(12, std::min(stages, (220 * 1024) / stage_bytes)));
+    const int target = env_int("POLESTAR_GEMM_TARGET_CTAS", g_sm_count > 0 ? g_sm_count : 148);
+    int splits = std::max(1, (target + tiles_f * tiles_t - 1) / (tiles_f * tiles_t));
+    splits = std::min(splits, std::max(1, kb / 4));
+    splits = std::min(splits, env_int("POLESTAR_GEMM_MAX_SPLITS", 8));
+    while (splits > 1 && ((size_t)splits * tiles_f * tiles_t * NT * 128 * 4 > ws.partial_bytes ||
+                          tiles_f * tiles_t > ws.n_counters))
+        --splits;
+    g.stages = stages; g.splits = splits;
+    g.partial = ws.partial; g.tile_counter = ws.counters; g.status = ws.status;
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    auto kern = tc::gemm_tc_kernel<__nv_bfloat16, EPI>;
+    static size_t smem_set = 0;
+    if (smem > smem_set) {
+        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        smem_set = 225 * 1024;
+    }
+    dim3 grid(tiles_f, tiles_t, splits);
+    kern<<<grid, tc::THREADS, smem, st>>>(*mw, *ma, g, e);
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// context
+// ------------------------------------------------------------------------------------------
+struct Plan {
+    size_t total = 0;
+    size_t take(size_t bytes) {
+        const size_t o = total;
+        total += (bytes + 1023) & ~(size_t)1023;
+        return o;
+    }
+};
+
+struct Buffers {
+    // persistent
+    int* y; float2* rope; char* kc; char* vc; float* hc; float* pprev; float* aprev; float* theta; int* theta_cnt;
+    int* tok_at_h0; float* drift; int* sel_idx; int* sel_cnt; unsigned char* patch; int* forced_idx; int* forced_cnt;
+    int* forced_commit; float* conf; int* yhat; float* delta; float* Delta; float* taud; int* commit_flags;
+    int* suffix_flags; int* seq_info; int* head_count; int* suf_seq; int* suf_w; int* stats; int* status;
+    int* list_count; float* hidden_keep;
+    // scratch
+    Row* rows; unsigned char* kvflag; float* x; float* x1; float* packet; char* a_buf; char* q_buf; char* o_buf;
+    char* g_buf; float* kl; int* list; HeadSrc* head_list; char* a_head; float* logits; ConfPart* conf_part;
+    float* gemm_partial; int* gemm_counters;
+};
+
+static const int CONF_CHUNKS = 32;
+static const int FORCED_COMMIT_MAX = 512;
+static const size_t GEMM_PARTIAL_BYTES = (size_t)64 << 20;
+static const int GEMM_COUNTERS = 8192;
+
+struct polestar_ctx {
+    polestar_model m;
+    polestar_params p;
+    std::vector<const void*> wqkv, wo, wgu, wd;
+    std::vector<const float*> n1, n2;
+    const void *embed, *lm_head;
+    const float* final_norm;
+    cudaStream_t st;
+    char* ws;
+    Buffers b;
+    MapCache maps;
+    GemmWs gws;
+    int es;          // element size of the model dtype
+    int N, B, W_max, n_blocks, M_max, rows_lm;
+    // controller
+    int block = 0;
+    bool need_entry = true, pending = false, done = false;
+    int steps_used = 0;
+    long long forwards = 0, generated = 0, generated_non_eos = 0;
+    std::vector<int> cum;
+    StepDesc last_sd;
+    int last_act_row_off = 0;
+    bool forced_select = false, forced_commit = false;
+    int forced_commit_n = 0;
+    std::vector<int> seq_info_host;
+};
+
+static bool valid_cfg(const polestar_model* m, const polestar_params* p) {
+    if (!m || !p) return false;
+    if (m->n_layers <= 0 || m->d_model <= 0 || m->n_heads <= 0 || m->n_kv_heads <= 0 || m->head_dim <= 0) return false;
+    if (m->n_heads % m->n_kv_heads) return false;
+    if (m->head_dim % 2 || m->head_dim > 256 || m->d_ffn <= 0 || m->vocab < 4 || m->vocab % 2) return false;
+    if (m->dtype != POLESTAR_F32 && m->dtype != POLESTAR_BF16) return false;
+    if (m->mask_id < 0 || m->mask_id >= m->vocab || m->eos_id < 0 || m->eos_id >= m->vocab) return false;
+    if (m->d_model % 8 || (m->n_heads * m->head_dim) % 8 || m->d_ffn % 8) return false;
+    if (p->batch <= 0 || p->batch > POLESTAR_MAX_BATCH) return false;
+    if (p->prompt_len < 0 || p->gen_len <= 0 || p->block <= 0 || p->block > 256) return false;
+    if (p->gen_len % p->block) return false;
+    if (p->max_steps <= 0 || p->win_prefix_blocks < 0 || p->win_suffix_blocks < 0 || p->full_entry_period <= 0) return false;
+    if (p->select_mode < 0 || p->select_mode > 4 || p->hist < 0 || p->hist > 64) return false;
+    const long long N = (long long)p->prompt_len + p->gen_len;
+    if (N > 65536) return false;
+    const long long wmax = std::min<long long>((long long)(p->win_prefix_blocks + p->win_suffix_blocks) * p->block, N - p->block);
+    if (wmax > 1024) return false;
+    return true;
+}
+
+static int window_max(const polestar_params* p) {
+    const long long N = (long long)p->prompt_len + p->gen_len;
+    long long w = std::min<long long>((long long)(p->win_prefix_blocks + p->win_suffix_blocks) * p->block, N - p->block);
+    return (int)std::max<long long>(w, 1);
+}
+
+static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffers* b, char* base) {
+    Plan pl;
+    const size_t es = m->dtype == POLESTAR_BF16 ? 2 : 4;
+    const size_t L = m->n_layers, bs = p->batch, N = (size_t)p->prompt_len + p->gen_len, B = p->block;
+    const size_t d = m->d_model, dq = (size_t)m->n_heads * m->head_dim, dkv = (size_t)m->n_kv_heads * m->head_dim;
+    const size_t F = m->d_ffn, V = m->vocab, nh = m->n_heads;
+    const size_t Wm = window_max(p);
+    const size_t n_suf = std::min<size_t>((size_t)p->win_suffix_blocks * B, Wm);
+    const size_t Mmax = bs * std::max(N, B + Wm);
+    const size_t rows_lm = bs * (B + n_suf);
+#define TAKE(field, type, count)                                  \
+    do {                                                          \
+        const size_t _o = pl.take((size_t)(count) * sizeof(type)); \
+        if (b) b->field = (type*)(base + _o);                     \
+    } while (0)
+    TAKE(y, int, bs * N);
+    TAKE(rope, float2, N * (m->head_dim / 2));
+    TAKE(kc, char, L * bs * N * dkv * es);
+    TAKE(vc, char, L * bs * N * dkv * es);
+    TAKE(hc, float, L * bs * Wm * d);
+    TAKE(pprev, float, L * bs * Wm * nh * N);
+    TAKE(aprev, float, bs * B * nh * N);
+    TAKE(theta, float, bs * std::max<size_t>(1, p->hist) * B);
+    TAKE(theta_cnt, int, bs);
+    TAKE(tok_at_h0, int, bs * Wm);
+    TAKE(drift, float, L * bs * Wm);
+    TAKE(sel_idx, int, L * bs * Wm);
+    TAKE(sel_cnt, int, L * bs);
+    TAKE(patch, unsigned char, (L + 1) * bs * Wm);
+    TAKE(forced_idx, int, L * bs * Wm);
+    TAKE(forced_cnt, int, L * bs);
+    TAKE(forced_commit, int, bs * FORCED_COMMIT_MAX);
+    TAKE(conf, float, rows_lm);
+    TAKE(yhat, int, rows_lm);
+    TAKE(delta, float, bs * B);
+    TAKE(Delta, float, bs * B);
+    TAKE(taud, float, bs * B);
+    TAKE(commit_flags, int, bs * B);
+    TAKE(suffix_flags, int, bs * Wm);
+    TAKE(seq_info, int, bs * 8);
+    TAKE(head_count, int, 1);
+    TAKE(suf_seq, int, bs * Wm);
+    TAKE(suf_w, int, bs * Wm);
+    TAKE(stats, int, 4);
+    TAKE(status, int, 1);
+    TAKE(list_count, int, 1);
+    TAKE(hidden_keep, float, (p->flags & POLESTAR_FLAG_KEEP_HIDDEN) ? (L + 1) * bs * B * d : 1);
+    TAKE(rows, Row, Mmax);
+    TAKE(kvflag, unsigned char, Mmax);
+    TAKE(x, float, Mmax * d);
+    TAKE(x1, float, Mmax * d);
+    TAKE(packet, float, bs * Wm * d);
+    TAKE(a_buf, char, Mmax * d * es);
+    TAKE(q_buf, char, Mmax * dq * es);
+    TAKE(o_buf, char, Mmax * dq * es);
+    TAKE(g_buf, char, Mmax * F * es);
+    TAKE(kl, float, Mmax * nh);
+    TAKE(list, int, Mmax);
+    TAKE(head_list, HeadSrc, rows_lm);
+    TAKE(a_head, char, rows_lm * d * es);
+    TAKE(logits, float, rows_lm * V);
+    TAKE(conf_part, ConfPart, rows_lm * CONF_CHUNKS);
+    TAKE(gemm_partial, float, GEMM_PARTIAL_BYTES / 4);
+    TAKE(gemm_counters, int, GEMM_COUNTERS);
+#undef TAKE
+    return pl.total;
+}
+
+extern "C" size_t polestar_workspace_bytes(const polestar_model* m, const polestar_params* p) {
+    if (!valid_cfg(m, p)) return 0;
+    return make_plan(m, p, nullptr, nullptr);
+}
+
+extern "C" int polestar_sm_count(void) { return g_sm_count; }
+
+extern "C" const char* polestar_strerror(int code) {
+    switch (code) {
+        case POLESTAR_OK: return "ok";
+        case POLESTAR_E_INVAL: return "invalid argument or unsupported shape";
+        case POLESTAR_E_STATE: return "call order violated";
+        case POLESTAR_E_NOSPACE: return "workspace too small";
+        case POLESTAR_E_CUDA: return cudaGetErrorString(last_cuda_error);
+        case POLESTAR_E_NONFINITE: return "non-finite confidence";
+        case POLESTAR_E_TIMEOUT: return "device-side wait timed out";
+        case POLESTAR_E_DONE: return "decoding already finished";
+        default: return "unknown error";
+    }
+}
+
+static int init_device_info() {
+    if (g_sm_count == 0) {
+        int dev = 0;
+        CK(cudaGetDevice(&dev));
+        CK(cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
+    return POLESTAR_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// one forward
+// ------------------------------------------------------------------------------------------
+template <typename T>
+struct Path {
+    static constexpr bool is_bf16 = sizeof(T) == 2;
+
+    template <int EPI>
+    static int gemm(polestar_ctx* c, const void* A, int a_rows_alloc, const void* W, int M, int N_out, int K,
+                    const EpiArgs& e) {
+        if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 128 == 0 &&
+            (EPI != EPI_QKV || c->m.head_dim == 128))
+            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st);
+        return launch_gemm_simt<T, EPI>(A, W, M, N_out, K, e, c->st);
+    }
+
+    static int attention(polestar_ctx* c, const AttnArgs& a) {
+        if (is_bf16 && c->m.head_dim == 128 && !env_int("POLESTAR_ATTN_SIMT", 0))
+            return launch_attention_mma(a, c->st);
+        const int wpb = 4;
+        const size_t smem = (size_t)wpb * a.N * sizeof(float);
+        static size_t set = 0;
+        if (smem > 48 * 1024 && smem > set) {
+            CK(cudaFuncSetAttribute(attention_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            set = smem;
+        }
+        dim3 grid((a.n_rows + wpb - 1) / wpb, a.n_heads);
+        attention_simt_kernel<T><<<grid, wpb * 32, smem, c->st>>>(a);
+        CK(cudaGetLastError());
+        return POLESTAR_OK;
+    }
+
+    static int forward(polestar_ctx* c, const StepDesc& sd, bool any_refresh) {
+        const polestar_model& m = c->m;
+        const polestar_params& p = c->p;
+        Buffers& b = c->b;
+        cudaStream_t st = c->st;
+        const int d = m.d_model, dq = m.n_heads * m.head_dim, dkv = m.n_kv_heads * m.head_dim, F = m.d_ffn;
+        const int L = m.n_layers, bs = p.batch, N = c->N, B = c->B, Wm = c->W_max;
+        const int M = bs * sd.rows_per_seq;
+        const int act_off = sd.kind == 2 ? 0 : (sd.act_start - sd.e0);
+        const size_t es = sizeof(T);
+        const bool within = sd.kind == 2;
+        const bool sparse = within && any_refresh;
+        int rc;
+
+        build_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(sd, b.rows);
+        CK(cudaMemsetAsync(b.stats, 0, 4 * sizeof(int), st));
+        embed_rows_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.y, (const T*)c->embed, d, b.x, b.packet, b.patch,
+                                               b.tok_at_h0, b.stats);
+        CK(cudaGetLastError());
+
+        for (int l = 0; l < L; ++l) {
+            char* kc = b.kc + (size_t)l * bs * N * dkv * es;
+            char* vc = b.vc + (size_t)l * bs * N * dkv * es;
+            float* hc = b.hc + (size_t)l * bs * Wm * d;
+            float* pprev = b.pprev + (size_t)l * bs * Wm * m.n_heads * N;
+            const bool last = l == L - 1;
+            if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN)
+                keep_hidden_kernel<<<bs * B, 256, 0, st>>>(sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d);
+
+            prep_qkv_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
+                                                 c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag);
+            CK(cudaGetLastError());
+
+            EpiArgs e;
+            memset(&e, 0, sizeof(e));
+            e.rows = b.rows; e.kvflag = b.kvflag; e.rope = b.rope; e.q_out = b.q_buf; e.kc = kc; e.vc = vc;
+            e.N_seq = N; e.n_heads = m.n_heads; e.n_kv = m.n_kv_heads; e.head_dim = m.head_dim; e.W_max = Wm;
+            e.within = within; e.ld_out = dq;
+            if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->M_max, c->wqkv[l], M, dq + 2 * dkv, d, e))) return rc;
+
+            AttnArgs a;
+            memset(&a, 0, sizeof(a));
+            a.rows = b.rows; a.n_rows = M; a.q = b.q_buf; a.kc = kc; a.vc = vc; a.out = b.o_buf;
+            a.pprev = (sparse || !within) ? pprev : nullptr;
+            a.aprev = last ? b.aprev : nullptr;
+            a.kl = b.kl; a.N = N; a.n_heads = m.n_heads; a.n_kv = m.n_kv_heads; a.head_dim = m.head_dim;
+            a.W_max = Wm; a.B = B; a.record_kl = sd.record_kl; a.rows_per_seq = sd.rows_per_seq; a.batch = bs;
+            a.scale = 1.0f / sqrtf((float)m.head_dim);
+            if ((rc = attention(c, a))) return rc;
+
+            const int* list = nullptr;
+            const int* m2_count = nullptr;
+            if (sparse) {
+                StepSelArgs s;
+                memset(&s, 0, sizeof(s));
+                s.kl = b.kl; s.drift = b.drift + (size_t)l * bs * Wm; s.sel_idx = b.sel_idx + (size_t)l * bs * Wm;
+                s.sel_cnt = b.sel_cnt + (size_t)l * bs; s.flag_next = b.patch + (size_t)(l + 1) * bs * Wm;
+                s.forced_idx = b.forced_idx + (size_t)l * bs * Wm; s.forced_cnt = b.forced_cnt + (size_t)l * bs;
+                s.list = b.list; s.list_count = b.list_count; s.stats = b.stats; s.n_heads = m.n_heads;
+                s.mode = p.select_mode;
+                s.k = p.select_mode == POLESTAR_SELECT_TOPK_FRAC ? (int)floorf(p.select_frac * (float)sd.W + 0.5f) : p.select_k;
+                s.W_max = Wm; s.thresh = p.select_thresh; s.floor_ = p.drift_floor;
+                step_select_kernel<<<1, SEL_THREADS, 0, st>>>(sd, s);
+                CK(cudaGetLastError());
+                list = b.list; m2_count = b.list_count;
+            }
+
+            memset(&e, 0, sizeof(e));
+            e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
+            if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e))) return rc;
+
+            prep_rows_kernel<T><<<M, 256, 0, st>>>(b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf);
+            CK(cudaGetLastError());
+
+            memset(&e, 0, sizeof(e));
+            e.out_t = b.g_buf; e.ld_out = F; e.m_count = m2_count;
+            if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->M_max, c->wgu[l], M, 2 * F, d, e))) return rc;
+
+            memset(&e, 0, sizeof(e));
+            e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = b.x1; e.out_f32 = b.x; e.packet = b.packet;
+            e.W_max = Wm; e.within = within; e.ld_out = d;
+            if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e))) return rc;
+        }
+        if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN)
+            keep_hidden_kernel<<<bs * B, 256, 0, st>>>(sd, b.x, act_off, d, b.hidden_keep + (size_t)L * bs * B * d);
+
+        // logits of the active rows (+ eligible suffix rows), confidences
+        const int use_suffix = sparse && (p.flags & POLESTAR_FLAG_SUFFIX_COMMIT);
+        build_head_list_kernel<<<1, 256, 0, st>>>(sd, b.y, m.mask_id, b.sel_idx + (size_t)(L - 1) * bs * Wm,
+                                                  b.sel_cnt + (size_t)(L - 1) * bs, use_suffix, 0, b.head_list,
+                                                  b.head_count, b.suf_seq, b.suf_w);
+        CK(cudaGetLastError());
+        const int Mh = use_suffix ? c->rows_lm : bs * B;
+        prep_head_kernel<T><<<Mh, 256, 0, st>>>(b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
+                                               (T*)b.a_head);
+        CK(cudaGetLastError());
+        EpiArgs e;
+        memset(&e, 0, sizeof(e));
+        e.out_f32 = b.logits; e.ld_out = m.vocab; e.scale = p.logit_scale; e.m_count = b.head_count;
+        if ((rc = gemm<EPI_LOGITS>(c, b.a_head, c->rows_lm, c->lm_head, Mh, m.vocab, d, e))) return rc;
+        conf_partial_kernel<<<dim3(CONF_CHUNKS, Mh), 256, 0, st>>>(b.logits, b.head_count, Mh, m.vocab, m.mask_id,
+                                                                  CONF_CHUNKS, b.conf_part);
+        conf_final_kernel<<<(Mh + 127) / 128, 128, 0, st>>>(b.conf_part, b.head_count, Mh, CONF_CHUNKS, b.yhat, b.conf);
+        CK(cudaGetLastError());
+        c->last_act_row_off = act_off;
+        return POLESTAR_OK;
+    }
+};
+
+static StepDesc make_step_desc(polestar_ctx* c, bool* any_refresh) {
+    const polestar_params& p = c->p;
+    StepDesc sd;
+    memset(&sd, 0, sizeof(sd));
+    const int N = c->N, B = c->B;
+    const int start = p.prompt_len + c->block * B, end = start + B;
+    sd.batch = p.batch; sd.N = N; sd.B = B; sd.act_start = start; sd.W_max = c->W_max;
+    sd.pre_start = (int)std::max<long long>(0, (long long)start - (long long)p.win_prefix_blocks * B);
+    sd.n_pre = start - sd.pre_start;
+    sd.suf_start = end;
+    const int n_suf = (int)(std::min<long long>(N, (long long)end + (long long)p.win_suffix_blocks * B) - end);
+    sd.W = sd.n_pre + n_suf;
+    const bool nocache = (p.flags & POLESTAR_FLAG_NOCACHE) != 0;
+    *any_refresh = false;
+    if (c->need_entry || nocache) {
+        const bool full = nocache || (c->block % p.full_entry_period == 0);
+        sd.kind = full ? 0 : 1;
+        sd.e0 = full ? 0 : sd.pre_start;
+        sd.rows_per_seq = full ? N : (sd.n_pre + B + n_suf);
+        sd.within = 0;
+        sd.record_kl = (nocache && !c->need_entry) ? 1 : 0;
+    } else {
+        sd.kind = 2;
+        sd.within = 1;
+        sd.record_kl = 1;
+        for (int s = 0; s < p.batch; ++s) {
+            const bool r = p.tau_upd < 0 || c->cum[s] > p.tau_upd;
+            sd.refresh.v[s] = r ? 1 : 0;
+            if (r) { *any_refresh = true; c->cum[s] = 0; }
+        }
+        sd.rows_per_seq = *any_refresh ? B + sd.W : B;
+    }
+    return sd;
+}
+
+extern "C" int polestar_step(polestar_ctx* c, polestar_step_info* info) {
+    if (!c) return POLESTAR_E_INVAL;
+    if (c->done) return POLESTAR_E_DONE;
+    if (c->pending) return POLESTAR_E_STATE;
+    bool any_refresh = false;
+    StepDesc sd = make_step_desc(c, &any_refresh);
+    int rc = c->m.dtype == POLESTAR_BF16 ? Path<__nv_bfloat16>::forward(c, sd, any_refresh)
+                                         : Path<float>::forward(c, sd, any_refresh);
+    if (rc) return rc;
+    if (c->forced_select) {
+        CK(cudaMemsetAsync(c->b.forced_cnt, 0xFF, (size_t)c->m.n_layers * c->p.batch * sizeof(int), c->st));
+        c->forced_select = false;
+    }
+    c->last_sd = sd;
+    c->pending = true;
+    c->forwards += 1;
+    if (info) {
+        info->kind = sd.kind;
+        info->block_index = c->block;
+        int nr = 0;
+        for (int s = 0; s < c->p.batch; ++s) nr += sd.refresh.v[s];
+        info->n_refreshing = nr;
+        info->rows = sd.rows_per_seq;
+        info->forwards = c->forwards;
+    }
+    return POLESTAR_OK;
+}
+
+extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
+    if (!c) return POLESTAR_E_INVAL;
+    if (!c->pending) return POLESTAR_E_STATE;
+    const polestar_params& p = c->p;
+    const StepDesc& sd = c->last_sd;
+    Buffers& b = c->b;
+    CommitArgs a;
+    memset(&a, 0, sizeof(a));
+    a.y = b.y; a.conf = b.conf; a.yhat = b.yhat;
+    a.kl = b.kl; a.delta_out = b.delta; a.Delta_out = b.Delta; a.taud_out = b.taud;
+    a.theta = b.theta; a.theta_cnt = b.theta_cnt; a.commit_flags = b.commit_flags; a.suffix_flags = b.suffix_flags;
+    a.head_count = b.head_count; a.suf_seq = b.suf_seq; a.suf_w = b.suf_w;
+    a.forced_pos = c->forced_commit ? b.forced_commit : nullptr;
+    a.forced_n = c->forced_commit_n;
+    a.seq_info = b.seq_info;
+    a.n_heads = c->m.n_heads; a.hist = p.hist; a.mask_id = c->m.mask_id; a.eos_id = c->m.eos_id;
+    a.act_row_off = c->last_act_row_off; a.steps_used = c->steps_used;
+    a.steps_per_block = std::max(1, p.max_steps / std::max(1, c->n_blocks));
+    a.use_drift = (p.flags & POLESTAR_FLAG_DRIFT_COMMIT) ? 1 : 0;
+    a.use_suffix = (p.flags & POLESTAR_FLAG_SUFFIX_COMMIT) ? 1 : 0;
+    a.ge = (p.flags & POLESTAR_FLAG_GE_COMPARE) ? 1 : 0;
+    a.tau_s = p.tau_s; a.alpha = p.alpha; a.tau_suffix = p.tau_suffix;
+    const bool entry_like = sd.record_kl == 0;
+    if (entry_like) CK(cudaMemsetAsync(b.theta_cnt, 0, p.batch * sizeof(int), c->st));   // history cleared at block entry
+    commit_kernel<<<p.batch, 256, 0, c->st>>>(sd, a);
+    CK(cudaGetLastError());
+    c->seq_info_host.resize((size_t)p.batch * 8 + 8);
+    CK(cudaMemcpyAsync(c->seq_info_host.data(), b.seq_info, (size_t)p.batch * 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+    CK(cudaMemcpyAsync(c->seq_info_host.data() + p.batch * 8, b.stats, 4 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+    CK(cudaMemcpyAsync(c->seq_info_host.data() + p.batch * 8 + 4, b.status, sizeof(int), cudaMemcpyDeviceToHost, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    c->pending = false;
+    c->forced_commit = false;
+    const int* si = c->seq_info_host.data();
+    polestar_commit_info ci;
+    memset(&ci, 0, sizeof(ci));
+    bool all_block_done = true;
+    int nonfinite = 0;
+    for (int s = 0; s < p.batch; ++s) {
+        const int* o = si + s * 8;
+        ci.n_committed += o[0]; ci.n_by_conf += o[1]; ci.n_by_drift += o[2]; ci.n_by_quota += o[3];
+        ci.n_suffix += o[4]; ci.n_eos += o[5];
+        if (o[6] > 0) all_block_done = false;
+        nonfinite += o[7];
+        if (entry_like && !(p.flags & POLESTAR_FLAG_NOCACHE)) c->cum[s] = o[0];
+        else c->cum[s] += o[0];
+    }
+    ci.rows_refreshed = si[p.batch * 8];
+    const int status = si[p.batch * 8 + 4];
+    ci.block_index = c->block;
+    c->steps_used += 1;
+    c->need_entry = false;
+    c->generated += ci.n_committed;
+    c->generated_non_eos += ci.n_committed - ci.n_eos;
+    if (all_block_done) {
+        c->block += 1;
+        c->need_entry = true;
+        c->steps_used = 0;
+        ci.block_done = 1;
+        if (c->block >= c->n_blocks) { c->done = true; ci.all_done = 1; }
+    }
+    ci.forwards = c->forwards; ci.generated = c->generated; ci.generated_non_eos = c->generated_non_eos;
+    if (info) *info = ci;
+    if (status) return POLESTAR_E_TIMEOUT;
+    if (nonfinite) return POLESTAR_E_NONFINITE;
+    return POLESTAR_OK;
+}
+
+extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const polestar_weights* w,
+                             const polestar_params* p, const int32_t* prompt, void* ws, size_t ws_bytes, void* stream) {
+    if (out) *out = nullptr;
+    if (!out || !m || !w || !p || !ws || (!prompt && p->prompt_len > 0)) return POLESTAR_E_INVAL;
+    if (!valid_cfg(m, p)) return POLESTAR_E_INVAL;
+    if (!w->embed || !w->lm_head || !w->final_norm || !w->wqkv || !w->wo || !w->w_gate_up || !w->w_down || !w->norm1 ||
+        !w->norm2)
+        return POLESTAR_E_INVAL;
+    if (((uintptr_t)ws) & 255) return POLESTAR_E_INVAL;
+    for (int i = 0; i < p->batch * p->prompt_len; ++i)
+        if (prompt[i] < 0 || prompt[i] >= m->vocab || prompt[i] == m->mask_id) return POLESTAR_E_INVAL;
+    const size_t need = make_plan(m, p, nullptr, nullptr);
+    if (ws_bytes < need) return POLESTAR_E_NOSPACE;
+    int rc = init_device_info();
+    if (rc) return rc;
+    polestar_ctx* c = new (std::nothrow) polestar_ctx();
+    if (!c) return POLESTAR_E_INVAL;
+    c->m = *m; c->p = *p;
+    for (int l = 0; l < m->n_layers; ++l) {
+        if (!w->wqkv[l] || !w->wo[l] || !w->w_gate_up[l] || !w->w_down[l] || !w->norm1[l] || !w->norm2[l]) {
+            delete c;
+            return POLESTAR_E_INVAL;
+        }
+        c->wqkv.push_back(w->wqkv[l]); c->wo.push_back(w->wo[l]); c->wgu.push_back(w->w_gate_up[l]);
+        c->wd.push_back(w->w_down[l]); c->n1.push_back(w->norm1[l]); c->n2.push_back(w->norm2[l]);
+    }
+    c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
+    c->st = (cudaStream_t)stream;
+    c->ws = (char*)(((uintptr_t)ws + 1023) & ~(uintptr_t)1023);
+    if ((size_t)(c->ws - (char*)ws) + need > ws_bytes + 1024) { delete c; return POLESTAR_E_NOSPACE; }
+    make_plan(m, p, &c->b, c->ws);
+    c->es = m->dtype == POLESTAR_BF16 ? 2 : 4;
+    c->N = p->prompt_len + p->gen_len; c->B = p->block; c->W_max = window_max(p);
+    c->n_blocks = p->gen_len / p->block;
+    c->M_max = p->batch * std::max(c->N, c->B + c->W_max);
+    c->rows_lm = p->batch * (c->B + std::min(p->win_suffix_blocks * c->B, c->W_max));
+    c->cum.assign(p->batch, 0);
+    c->gws.partial = c->b.gemm_partial; c->gws.partial_bytes = GEMM_PARTIAL_BYTES;
+    c->gws.counters = c->b.gemm_counters; c->gws.n_counters = GEMM_COUNTERS; c->gws.status = c->b.status;
+
+    auto fail = [&](int code) { delete c; return code; };
+    // zero the persistent state (everything in front of the scratch rows)
+    const size_t persist = (size_t)((char*)c->b.rows - c->ws);
+    if (cudaMemsetAsync(c->ws, 0, persist, c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
+    if (cudaMemsetAsync(c->b.forced_cnt, 0xFF, (size_t)m->n_layers * p->batch * sizeof(int), c->st) != cudaSuccess)
+        return fail(POLESTAR_E_CUDA);
+    if (cudaMemsetAsync(c->b.gemm_counters, 0, GEMM_COUNTERS * sizeof(int), c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
+    std::vector<int> y((size_t)p->batch * c->N, m->mask_id);
+    for (int s = 0; s < p->batch; ++s)
+        for (int i = 0; i < p->prompt_len; ++i) y[(size_t)s * c->N + i] = prompt[(size_t)s * p->prompt_len + i];
+    if (cudaMemcpyAsync(c->b.y, y.data(), y.size() * sizeof(int), cudaMemcpyHostToDevice, c->st) != cudaSuccess)
+        return fail(POLESTAR_E_CUDA);
+    const int half = m->head_dim / 2;
+    rope_table_kernel<<<(c->N * half + 255) / 256, 256, 0, c->st>>>(c->b.rope, c->N, half, (double)m->rope_theta);
+    if (cudaStreamSynchronize(c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
+    rc = polestar_step(c, nullptr);
+    if (rc) return fail(rc);
+    *out = c;
+    return POLESTAR_OK;
+}
+
+extern "C" void polestar_destroy(polestar_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->st);
+    delete c;
+}
+
+extern "C" int polestar_tokens(polestar_ctx* c, int32_t* out) {
+    if (!c || !out) return POLESTAR_E_INVAL;
+    CK(cudaMemcpyAsync(out, c->b.y, (size_t)c->p.batch * c->N * sizeof(int), cudaMemcpyDeviceToHost, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    return POLESTAR_OK;
+}
+
+extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void* dst, size_t bytes) {
+    if (!c || !dst) return POLESTAR_E_INVAL;
+    const polestar_model& m = c->m;
+    const size_t bs = c->p.batch, B = c->B, Wm = c->W_max, N = c->N, d = m.d_model, L = m.n_layers;
+    const size_t dkv = (size_t)m.n_kv_heads * m.head_dim;
+    const void* src = nullptr;
+    size_t sz = 0;
+    const bool need_layer = what == POLESTAR_READ_DRIFT || what == POLESTAR_READ_SEL_COUNT || what == POLESTAR_READ_SEL_IDX ||
+                            what == POLESTAR_READ_KCACHE || what == POLESTAR_READ_VCACHE || what == POLESTAR_READ_HCACHE ||
+                            what == POLESTAR_READ_PPREV;
+    if (need_layer && (layer < 0 || layer >= (int)L)) return POLESTAR_E_INVAL;
+    switch (what) {
+        case POLESTAR_READ_LOGITS: src = c->b.logits; sz = bs * B * m.vocab * 4; break;
+        case POLESTAR_READ_CONF: src = c->b.conf; sz = bs * B * 4; break;
+        case POLESTAR_READ_YHAT: src = c->b.yhat; sz = bs * B * 4; break;
+        case POLESTAR_READ_DELTA: src = c->b.delta; sz = bs * B * 4; break;
+        case POLESTAR_READ_DRIFT: src = c->b.drift + layer * bs * Wm; sz = bs * Wm * 4; break;
+        case POLESTAR_READ_SEL_COUNT: src = c->b.sel_cnt + layer * bs; sz = bs * 4; break;
+        case POLESTAR_READ_SEL_IDX: src = c->b.sel_idx + layer * bs * Wm; sz = bs * Wm * 4; break;
+        case POLESTAR_READ_HIDDEN:
+            if (!(c->p.flags & POLESTAR_FLAG_KEEP_HIDDEN) || layer < 0 || layer > (int)L) return POLESTAR_E_INVAL;
+            src = c->b.hidden_keep + layer * bs * B * d; sz = bs * B * d * 4; break;
+        case POLESTAR_READ_KCACHE: src = c->b.kc + layer * bs * N * dkv * c->es; sz = bs * N * dkv * c->es; break;
+        case POLESTAR_READ_VCACHE: src = c->b.vc + layer * bs * N * dkv * c->es; sz = bs * N * dkv * c->es; break;
+        case POLESTAR_READ_HCACHE: src = c->b.hc + layer * bs * Wm * d; sz = bs * Wm * d * 4; break;
+        case POLESTAR_READ_COMMIT: src = c->b.commit_flags; sz = bs * B * 4; break;
+        case POLESTAR_READ_PPREV: src = c->b.pprev + layer * bs * Wm * m.n_heads * N; sz = bs * Wm * m.n_heads * N * 4; break;
+        case POLESTAR_READ_SUFFIX: src = c->b.suffix_flags; sz = bs * Wm * 4; break;
+        default: return POLESTAR_E_INVAL;
+    }
+    CK(cudaMemcpyAsync(dst, src, std::min(sz, bytes), cudaMemcpyDeviceToHost, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    return POLESTAR_OK;
+}
+
+extern "C" int polestar_force(polestar_ctx* c, int32_t what, int32_t layer, const int32_t* idx, int32_t n) {
+    if (!c) return POLESTAR_E_INVAL;
+    const int bs = c->p.batch, Wm = c->W_max, L = c->m.n_layers;
+    if (what == POLESTAR_FORCE_CLEAR) {
+        CK(cudaMemsetAsync(c->b.forced_cnt, 0xFF, (size_t)L * bs * sizeof(int), c->st));
+        c->forced_select = false; c->forced_commit = false;
+        return POLESTAR_OK;
+    }
+    if (n < 0 || (n > 0 && !idx)) return POLESTAR_E_INVAL;
+    if (what == POLESTAR_FORCE_SELECT) {
+        if (layer < 0 || layer >= L || n > Wm) return POLESTAR_E_INVAL;
+        std::vector<int> cnt(bs, 0);
+        for (int s = 0; s < bs; ++s) {
+            int ns = 0;
+            while (ns < n && idx[s * n + ns] >= 0) ++ns;       // trailing -1 entries pad shorter lists
+            for (int i = 0; i < ns; ++i) {
+                const int w = idx[s * n + i];
+                if (w >= Wm || (i > 0 && w <= idx[s * n + i - 1])) return POLESTAR_E_INVAL;
+            }
+            cnt[s] = ns;
+            if (ns) CK(cudaMemcpyAsync(c->b.forced_idx + ((size_t)layer * bs + s) * Wm, idx + (size_t)s * n, ns * sizeof(int),
+                                       cudaMemcpyHostToDevice, c->st));
+        }
+        CK(cudaMemcpyAsync(c->b.forced_cnt + (size_t)layer * bs, cnt.data(), bs * sizeof(int), cudaMemcpyHostToDevice, c->st));
+        CK(cudaStreamSynchronize(c->st));
+        c->forced_select = true;
+        return POLESTAR_OK;
+    }
+    if (what == POLESTAR_FORCE_COMMIT) {
+        if (n > FORCED_COMMIT_MAX) return POLESTAR_E_INVAL;
+        if (n) CK(cudaMemcpyAsync(c->b.forced_commit, idx, (size_t)bs * n * sizeof(int), cudaMemcpyHostToDevice, c->st));
+        CK(cudaStreamSynchronize(c->st));
+        c->forced_commit = true;
+        c->forced_commit_n = n;
+        return POLESTAR_OK;
+    }
+    return POLESTAR_E_INVAL;
+}
+
+// ------------------------------------------------------------------------------------------
+// single kernels
+// ------------------------------------------------------------------------------------------
+extern "C" int polestar_k_attention(const void* q, const void* k, const void* v, float* logp_prev, float* kl, void* out,
+                                    int32_t R, int32_t N, int32_t n_heads, int32_t n_kv, int32_t head_dim, int32_t dtype,
+                                    void* stream) {
+    if (!q || !k || !v || R < 0 || N <= 0 || n_heads <= 0 || n_kv <= 0 || n_heads % n_kv || head_dim <= 0 || head_dim > 256)
+        return POLESTAR_E_INVAL;
+    if (logp_prev && !kl) return POLESTAR_E_INVAL;
+    if (dtype != POLESTAR_F32 && dtype != POLESTAR_BF16) return POLESTAR_E_INVAL;
+    if (R == 0) return POLESTAR_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    AttnArgs a;
+    memset(&a, 0, sizeof(a));
+    a.n_rows = R; a.q = q; a.kc = k; a.vc = v; a.out = out; a.pprev = logp_prev; a.kl = kl; a.N = N;
+    a.n_heads = n_heads; a.n_kv = n_kv; a.head_dim = head_dim; a.record_kl = 1; a.rows_per_seq = R; a.batch = 1;
+    a.scale = 1.0f / sqrtf((float)head_dim);
+    if (dtype == POLESTAR_BF16 && head_dim == 128 && !env_int("POLESTAR_ATTN_SIMT", 0)) return launch_attention_mma(a, st);
+    const int wpb = 4;
+    const size_t smem = (size_t)wpb * N * sizeof(float);
+    if (smem > 200 * 1024) return POLESTAR_E_INVAL;
+    dim3 grid((R + wpb - 1) / wpb, n_heads);
+    if (dtype == POLESTAR_BF16) {
+        CK(cudaFuncSetAttribute(attention_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        attention_simt_kernel<__nv_bfloat16><<<grid, wpb * 32, smem, st>>>(a);
+    } else {
+        CK(cudaFuncSetAttribute(attention_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        attention_simt_kernel<float><<<grid, wpb * 32, smem, st>>>(a);
+    }
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
+}
+
+extern "C" int polestar_k_hidden_delta(const void* a, const void* b, float* out, int32_t rows, int32_t d, int32_t dtype,
+                                       void* stream) {
+    if (!a || !b || !out || rows < 0 || d <= 0) return POLESTAR_E_INVAL;
+    if (dtype != POLESTAR_F32 && dtype != POLESTAR_BF16) return POLESTAR_E_INVAL;
+    const int per = dtype == POLESTAR_BF16 ? 8 : 4;
+    if (d % per || (((uintptr_t)a | (uintptr_t)b) & 15)) return POLESTAR_E_INVAL;
+    if (rows == 0) return POLESTAR_OK;
+    int rc = init_device_info();
+    if (rc) return rc;
+    const int wpb = 8;
+    const int grid = std::min((rows + wpb - 1) / wpb, g_sm_count * 8);
+    if (dtype == POLESTAR_BF16)
+        hidden_delta_kernel<__nv_bfloat16><<<grid, wpb * 32, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, out, rows, d);
+    else
+        hidden_delta_kernel<float><<<grid, wpb * 32, 0, (cudaStream_t)stream>>>((const float*)a, (const float*)b, out, rows, d);
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
+}
+
+extern "C" int polestar_k_select(const float* drift, int32_t batch, int32_t W, int32_t mode, int32_t k, float thresh,
+                                 float floor_, int32_t* idx, int32_t* count, void* stream) {
+    if (!drift || !idx || !count || batch < 0 || W <= 0 || W > SEL_MAX_W || mode < 0 || mode > 4) return POLESTAR_E_INVAL;
+    if (batch == 0) return POLESTAR_OK;
+    select_kernel<<<batch, SEL_THREADS, 0, (cudaStream_t)stream>>>(drift, W, mode, k, thresh, floor_, idx, count);
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
+}
+
+static size_t refresh_layout(int batch, int max_rows, int d, int head_dim, int P, size_t* off_rope, size_t* off_part,
+                             size_t* off_cnt, size_t* off_status) {
+    Plan pl;
+    pl.take((size_t)batch * max_rows * d * 2 + 256 * (size_t)d * 2);   // staged rows (+ one tile of slack)
+    *off_rope = pl.take((size_t)P * (head_dim / 2) * sizeof(float2));
+    *off_part = pl.take(GEMM_PARTIAL_BYTES / 2);
+    *off_cnt = pl.take(GEMM_COUNTERS * sizeof(int));
+    *off_status = pl.take(sizeof(int));
+    return pl.total;
+}
+
+extern "C" size_t polestar_k_refresh_scratch_bytes(int32_t batch, int32_t max_rows, int32_t d, int32_t n_heads,
+                                                   int32_t n_kv, int32_t head_dim) {
+    (void)n_heads; (void)n_kv;
+    if (batch <= 0 || max_rows <= 0 || d <= 0 || head_dim <= 0) return 0;
+    size_t a, b, c, e;
+    return refresh_layout(batch, max_rows, d, head_dim, 65536, &a, &b, &c, &e);
+}
+
+extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32_t* counts, const void* wqkv,
+                                  const float* norm, void* kc, void* vc, void* q_out, int32_t batch, int32_t P,
+                                  int32_t max_rows, int32_t d, int32_t n_heads, int32_t n_kv, int32_t head_dim,
+                                  float rms_eps, float rope_theta, int32_t dtype, void* scratch, size_t scratch_bytes,
+                                  void* stream) {
+    if (!h || !idx || !counts || !wqkv || !norm || !kc || !vc || !scratch) return POLESTAR_E_INVAL;
+    if (batch <= 0 || P <= 0 || P > 65536 || max_rows <= 0 || max_rows > P || d <= 0 || n_heads <= 0 || n_kv <= 0 ||
+        n_heads % n_kv || head_dim <= 0 || head_dim % 2)
+        return POLESTAR_E_INVAL;
+    if (dtype != POLESTAR_BF16) return POLESTAR_E_INVAL;
+    if (((uintptr_t)scratch) & 1023) return POLESTAR_E_INVAL;
+    size_t off_rope, off_part, off_cnt, off_status;
+    const size_t need = refresh_layout(batch, max_rows, d, head_dim, 65536, &off_rope, &off_part, &off_cnt, &off_status);
+    if (scratch_bytes < need) return POLESTAR_E_NOSPACE;
+    int rc = init_device_info();
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* sc = (char*)scratch;
+    __nv_bfloat16* a_buf = (__nv_bfloat16*)sc;
+    float2* rope = (float2*)(sc + off_rope);
+    static MapCache maps;
+    static const void* counters_zeroed_for = nullptr;
+    GemmWs ws;
+    ws.partial = (float*)(sc + off_part); ws.partial_bytes = GEMM_PARTIAL_BYTES / 2;
+    ws.counters = (int*)(sc + off_cnt); ws.n_counters = GEMM_COUNTERS; ws.status = (int*)(sc + off_status);
+    if (counters_zeroed_for != scratch) {
+        CK(cudaMemsetAsync(ws.counters, 0, GEMM_COUNTERS * sizeof(int) + 1024, st));
+        counters_zeroed_for = scratch;
+    }
+    const int half = head_dim / 2;
+    rope_table_kernel<<<(P * half + 255) / 256, 256, 0, st>>>(rope, P, half, (double)rope_theta);
+    const int M = batch * max_rows;
+    prep_refresh_kernel<__nv_bfloat16><<<M, 256, 0, st>>>((const __nv_bfloat16*)h, idx, counts, max_rows, P, norm, rms_eps, d, a_buf);
+    CK(cudaGetLastError());
+    EpiArgs e;
+    memset(&e, 0, sizeof(e));
+    e.rope = rope; e.q_out = q_out; e.kc = kc; e.vc = vc; e.n_heads = n_heads; e.n_kv = n_kv; e.head_dim = head_dim;
+    e.idx = idx; e.counts = counts; e.max_rows = max_rows; e.P = P;
+    const int dq = n_heads * head_dim, dkv = n_kv * head_dim;
+    if (d % 64 == 0 && (dq + 2 * dkv) % 128 == 0 && head_dim == 128 && !env_int("POLESTAR_REFRESH_SIMT", 0))
+        return launch_gemm_tc<EPI_QKV_REFRESH>(maps, ws, a_buf, M, wqkv, M, dq + 2 * dkv, d, e, st);
+    return launch_gemm_simt<__nv_bfloat16, EPI_QKV_REFRESH>(a_buf, wqkv, M, dq + 2 * dkv, d, e, st);
+}
+
+extern "C" int polestar_k_confidence(const float* logits, int32_t rows, int32_t vocab, int32_t mask_id, int32_t* yhat,
+                                     float* conf, void* scratch, size_t scratch_bytes, void* stream) {
+    if (!logits || !yhat || !conf || !scratch || rows < 0 || vocab <= 0) return POLESTAR_E_INVAL;
+    if (scratch_bytes < (size_t)rows * CONF_CHUNKS * sizeof(ConfPart)) return POLESTAR_E_NOSPACE;
+    if (rows == 0) return POLESTAR_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    conf_partial_kernel<<<dim3(CONF_CHUNKS, rows), 256, 0, st>>>(logits, nullptr, rows, vocab, mask_id, CONF_CHUNKS, (ConfPart*)scratch);
+    conf_final_kernel<<<(rows + 127) / 128, 128, 0, st>>>((const ConfPart*)scratch, nullptr, rows, CONF_CHUNKS, yhat, conf);
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
+}

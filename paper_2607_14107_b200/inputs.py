@@ -239,7 +239,7 @@ def torch_dtype(m: ModelCfg):
 
 
 def make_weights(m: ModelCfg, seed: int = 0, device="cpu", std: float = 0.02,
-                 layers: Optional[List[int]] = None) -> Dict:
+                 layers: Optional[List[int]] = None, with_globals: bool = True) -> Dict:
     """Logical weights, every matrix stored [out_features, in_features].
 
     Values are rounded to the model's storage dtype (bf16 models hold
@@ -252,8 +252,10 @@ def make_weights(m: ModelCfg, seed: int = 0, device="cpu", std: float = 0.02,
     def mk(layer, tid, shape):
         return normal_tensor(tensor_key(seed, layer, tid), shape, std, dt, device)
 
-    w = {"embed": mk(-1, T_EMBED, (V, d)), "lm_head": mk(-1, T_LM_HEAD, (V, d)),
-         "final_norm": torch.ones(d, dtype=dt, device=device), "layers": []}
+    w = {"layers": []}
+    if with_globals:
+        w.update({"embed": mk(-1, T_EMBED, (V, d)), "lm_head": mk(-1, T_LM_HEAD, (V, d)),
+                  "final_norm": torch.ones(d, dtype=dt, device=device)})
     for l in (range(m.n_layers) if layers is None else layers):
         w["layers"].append({
             "wq": mk(l, T_WQ, (dq, d)), "wk": mk(l, T_WK, (dkv, d)), "wv": mk(l, T_WV, (dkv, d)),

@@ -1,0 +1,243 @@
+"""Parity of the CUDA decoding path (through the C ABI) with the CPU oracle, step by step."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import polestar_oracle as O
+from paper_2607_14107_b200 import binding as Bd
+from paper_2607_14107_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+TOL = {I.DTYPE_F32: 1e-4, I.DTYPE_BF16: 2e-2}     # abs/rel tolerance on hidden states and logits
+
+
+def close(a, b, tol, what=""):
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    assert a.shape == b.shape, (what, a.shape, b.shape)
+    err = np.abs(a - b) - tol * np.abs(b)
+    assert np.isfinite(a).all(), what
+    assert err.max() <= tol, f"{what}: max abs err {np.abs(a - b).max():.3e} (tol {tol})"
+
+
+def setup(name, **kw):
+    m, p = I.config(name)
+    p = dataclasses.replace(p, flags=p.flags | I.FLAG_KEEP_HIDDEN, **kw)
+    w = I.make_weights(m, seed=0)
+    wn = I.weights_to_numpy(w)
+    prompt = I.make_prompt(m, p)
+    gpu = Bd.Polestar(m, Bd.pack_weights(m, w), p, prompt.numpy())
+    ora = O.PolestarOracle(m, wn, p, prompt.numpy())
+    return m, p, gpu, ora
+
+
+def topk_margin_ok(D, sel, tol):
+    """True if every decision of the top-k cut is farther than tol from the cut value."""
+    D = np.asarray(D, np.float64)
+    if len(sel) == 0 or len(sel) == len(D):
+        return True
+    inside = D[sel].min()
+    outside = np.delete(D, sel)
+    outside = outside[outside > 0].max() if (outside > 0).any() else 0.0
+    cut = 0.5 * (inside + outside)
+    return (inside - outside) > 2 * (tol + tol * abs(cut))
+
+
+def run_forced(name, n_steps, **kw):
+    """The CUDA path replays the oracle's refresh sets and commits; every step's numbers are compared."""
+    m, p, gpu, ora = setup(name, **kw)
+    tol = TOL[m.dtype]
+    L = m.n_layers
+    seen = dict(refresh=0, entry_window=0, within=0)
+    for step in range(n_steps):
+        if ora.done:
+            break
+        ora.step()     # oracle first, so that its refresh sets can be imposed on the CUDA step
+        tr = ora.seqs[0].trace
+        if step > 0:
+            if tr["kind"] == "within" and tr["refresh"]:
+                for l in range(L):
+                    sel = np.full((p.batch, gpu.W_max), -1, np.int32)
+                    for s in range(p.batch):
+                        sl = ora.seqs[s].trace["sel"][l]
+                        sel[s, :len(sl)] = sl
+                    gpu.force_select(l, sel)
+            info = gpu.step()
+            assert {0: "entry_full", 1: "entry_window", 2: "within"}[info.kind] == tr["kind"]
+        for s in range(p.batch):
+            trs = ora.seqs[s].trace
+            for l in range(L + 1):
+                close(gpu.read(Bd.READ_HIDDEN, l)[s], trs["x_act"][l], tol, f"step {step} hidden l{l}")
+            close(gpu.read(Bd.READ_LOGITS)[s], trs["logits"], tol, f"step {step} logits")
+            if trs["kind"] == "within":
+                seen["within"] += 1
+                close(gpu.read(Bd.READ_DELTA)[s], trs["delta"], tol, f"step {step} delta")
+                if trs["refresh"]:
+                    seen["refresh"] += 1
+                    W = len(ora.seqs[s].win)
+                    for l in range(L):
+                        close(gpu.read(Bd.READ_DRIFT, l)[s, :W], trs["D"][l], tol, f"step {step} drift l{l}")
+                        n = gpu.read(Bd.READ_SEL_COUNT, l)[s]
+                        assert list(gpu.read(Bd.READ_SEL_IDX, l)[s, :n]) == list(trs["sel"][l])
+            elif trs["kind"] == "entry_window":
+                seen["entry_window"] += 1
+            for l in range(L):
+                close(gpu.read(Bd.READ_KCACHE, l)[s].reshape(ora.seqs[s].Kc[l].shape), ora.seqs[s].Kc[l], tol,
+                      f"step {step} K l{l}")
+                close(gpu.read(Bd.READ_VCACHE, l)[s].reshape(ora.seqs[s].Vc[l].shape), ora.seqs[s].Vc[l], tol,
+                      f"step {step} V l{l}")
+                W = len(ora.seqs[s].win)
+                close(gpu.read(Bd.READ_HCACHE, l)[s, :W], ora.seqs[s].Hc[l], tol, f"step {step} H l{l}")
+            _, conf = O.confidence_rows(trs["logits"], m.mask_id)
+            close(gpu.read(Bd.READ_CONF)[s], conf, tol, f"step {step} conf")
+        infos = ora.commit()
+        forced = np.full((p.batch, p.block + gpu.W_max), -1, np.int32)
+        for s, i in enumerate(infos):
+            pos = [int(ora.seqs[s].act[j]) for j in np.nonzero(i["commit"] & i["masked"])[0]] + i["suffix_committed"]
+            forced[s, :len(pos)] = pos
+        gpu.force_commit(forced)
+        ci = gpu.commit()
+        assert ci.n_committed == sum(i["n_committed"] for i in infos)
+        assert np.array_equal(gpu.tokens(), ora.tokens()), f"step {step} tokens"
+        assert bool(ci.all_done) == ora.done
+    gpu.destroy()
+    return seen
+
+
+def test_c1_forced_decisions_every_step():
+    seen = run_forced("c1", 40)
+    assert seen["refresh"] > 0 and seen["entry_window"] > 0
+
+
+def test_c1_refresh_every_step_with_scaled_logits():
+    seen = run_forced("c1", 20, tau_upd=-1, logit_scale=25.0, tau_suffix=0.5)
+    assert seen["refresh"] > 3
+
+
+def test_c1b_bf16_tensor_core_path():
+    seen = run_forced("c1b", 16, tau_upd=-1, logit_scale=20.0)
+    assert seen["refresh"] > 3
+
+
+def test_c1b_bf16_simt_gemm_path():
+    run_forced("c1b", 6, tau_upd=-1, flags=I.FLAG_DEFAULT | Bd.FLAG_SIMT_GEMM)
+
+
+def test_c1_batch2_gqa():
+    m, p = I.config("c1")
+    m = dataclasses.replace(m, n_kv_heads=2)
+    p = dataclasses.replace(p, batch=2, flags=p.flags | I.FLAG_KEEP_HIDDEN, tau_upd=1)
+    w = I.make_weights(m, seed=0)
+    prompt = I.make_prompt(m, p)
+    gpu = Bd.Polestar(m, Bd.pack_weights(m, w), p, prompt.numpy())
+    ora = O.PolestarOracle(m, I.weights_to_numpy(w), p, prompt.numpy())
+    gpu.commit(); ora.commit()
+    for step in range(10):
+        gpu.step(); ora.step()
+        for s in range(2):
+            close(gpu.read(Bd.READ_LOGITS)[s], ora.seqs[s].trace["logits"], 1e-4, f"step {step} seq {s}")
+        gpu.commit(); ora.commit()
+        assert np.array_equal(gpu.tokens(), ora.tokens())
+
+
+def test_c1_free_running_matches_oracle():
+    """Both sides take their own decisions; fp32 margins are far above the arithmetic error, so
+    index sets and committed tokens must agree exactly (a low-margin decision ends the check)."""
+    m, p, gpu, ora = setup("c1", logit_scale=25.0, tau_upd=2)
+    tol = TOL[m.dtype]
+    first = True
+    n_steps = 0
+    while not ora.done:
+        ora.step()
+        if not first:
+            gpu.step()
+        first = False
+        tr = ora.seqs[0].trace
+        if tr["kind"] == "within" and tr["refresh"]:
+            W = len(ora.seqs[0].win)
+            for l in range(m.n_layers):
+                D = gpu.read(Bd.READ_DRIFT, l)[0, :W]
+                if not topk_margin_ok(tr["D"][l], tr["sel"][l], tol):
+                    return
+                n = gpu.read(Bd.READ_SEL_COUNT, l)[0]
+                assert list(gpu.read(Bd.READ_SEL_IDX, l)[0, :n]) == list(tr["sel"][l])
+                close(D, tr["D"][l], tol, "drift")
+        info = ora.commit()[0]
+        ci = gpu.commit()
+        conf = info["conf"]
+        near = np.abs(conf - p.tau_s) < 2 * tol
+        near |= np.abs(info["Delta"] - info["tau_d"]) < 2 * tol * (1 + np.abs(info["tau_d"]))
+        if (near & info["masked"]).any():
+            return
+        flags = gpu.read(Bd.READ_COMMIT)[0]
+        if info["n_by_quota"] == 0:
+            assert np.array_equal((flags & 1).astype(bool), info["commit"] & info["masked"])
+            assert np.array_equal(gpu.tokens(), ora.tokens())
+            assert (ci.n_by_conf, ci.n_by_drift, ci.n_suffix) == (info["n_by_conf"], info["n_by_drift"], info["n_suffix"])
+        elif not np.array_equal(gpu.tokens(), ora.tokens()):
+            return      # quota picked between near-equal confidences
+        n_steps += 1
+    assert ora.done and n_steps > 4
+    assert np.array_equal(gpu.tokens(), ora.tokens())
+    assert not (gpu.tokens() == m.mask_id).any()
+
+
+def test_full_refresh_equals_nocache_on_gpu():
+    """select = ALL, window = everything, refresh every step must reproduce the full-recompute
+    decoder of the same library (Sec. 4.1; Sec. 3.1 baseline)."""
+    m, p = I.config("c1")
+    w = I.make_weights(m, seed=0)
+    prompt = I.make_prompt(m, p).numpy()
+    packed = Bd.pack_weights(m, w)
+    pa = dataclasses.replace(p, select_mode=I.SELECT_ALL, tau_upd=-1, win_prefix_blocks=8, win_suffix_blocks=8,
+                             flags=(I.FLAG_DEFAULT | I.FLAG_KEEP_HIDDEN) & ~I.FLAG_SUFFIX_COMMIT, logit_scale=25.0)
+    pb = dataclasses.replace(pa, flags=pa.flags | I.FLAG_NOCACHE)
+    a, b = Bd.Polestar(m, packed, pa, prompt), Bd.Polestar(m, packed, pb, prompt)
+    first = True
+    while True:
+        if not first:
+            a.step(); b.step()
+        first = False
+        for l in range(m.n_layers + 1):
+            close(a.read(Bd.READ_HIDDEN, l), b.read(Bd.READ_HIDDEN, l), 1e-4, f"hidden l{l}")
+        close(a.read(Bd.READ_LOGITS), b.read(Bd.READ_LOGITS), 1e-4, "logits")
+        ia, ib = a.commit(), b.commit()
+        assert np.array_equal(a.tokens(), b.tokens())
+        if ia.all_done:
+            break
+    assert ib.all_done and ia.forwards == ib.forwards
+
+
+def test_zero_drift_refreshes_nothing_on_gpu():
+    m, p, gpu, ora = setup("c1", tau_upd=-1)
+    gpu.force_commit(np.full((1, 4), -1, np.int32))       # commit nothing at entry
+    gpu.commit()
+    K0 = [gpu.read(Bd.READ_KCACHE, l).copy() for l in range(m.n_layers)]
+    info = gpu.step()
+    assert info.kind == 2 and info.n_refreshing == 1
+    for l in range(m.n_layers):
+        assert gpu.read(Bd.READ_SEL_COUNT, l)[0] == 0
+        assert np.abs(gpu.read(Bd.READ_DRIFT, l)).max() < 1e-5
+        assert np.array_equal(gpu.read(Bd.READ_KCACHE, l), K0[l])
+    assert np.abs(gpu.read(Bd.READ_DELTA)).max() < 1e-5
+
+
+def test_call_order_errors():
+    m, p, gpu, ora = setup("c1")
+    with pytest.raises(Bd.PolestarError) as e:
+        gpu.step()                                        # commit pending after init
+    assert e.value.code == Bd.E_STATE
+    gpu.commit()
+    with pytest.raises(Bd.PolestarError) as e:
+        gpu.commit()
+    assert e.value.code == Bd.E_STATE
+    while True:
+        gpu.step()
+        if gpu.commit().all_done:
+            break
+    with pytest.raises(Bd.PolestarError) as e:
+        gpu.step()
+    assert e.value.code == Bd.E_DONE
+    assert not (gpu.tokens() == m.mask_id).any()

@@ -1,0 +1,180 @@
+"""Each CUDA kernel of the path against the matching oracle function, through the C ABI."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import polestar_oracle as O
+from paper_2607_14107_b200 import binding as Bd
+from paper_2607_14107_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+def bf16_np(t):
+    return t.detach().to("cpu", torch.float32).numpy().astype(np.float64)
+
+
+def rnd(shape, key, std=1.0, dtype=torch.float32):
+    return I.normal_tensor(I.tensor_key(77, -1, key), shape, std, dtype, "cpu")
+
+
+# ------------------------------------------------------------------ attention + drift (a1, a5)
+@pytest.mark.parametrize("dtype,R,N,nh,nkv,dh", [
+    (torch.float32, 5, 37, 4, 4, 64),          # ragged everything
+    (torch.float32, 33, 128, 4, 2, 64),
+    (torch.bfloat16, 16, 512, 4, 4, 128),      # one tile
+    (torch.bfloat16, 37, 200, 4, 2, 128),      # ragged rows and keys, GQA
+    (torch.bfloat16, 128, 512, 2, 2, 128),     # window + block rows of the 8B shape
+    (torch.bfloat16, 3, 31, 2, 1, 128),        # fewer keys than one warp tile
+])
+def test_attention_drift_matches_oracle(dtype, R, N, nh, nkv, dh):
+    q = rnd((R, nh * dh), 1, 1.0, dtype).cuda()
+    k = rnd((N, nkv * dh), 2, 1.0, dtype).cuda()
+    v = rnd((N, nkv * dh), 3, 1.0, dtype).cuda()
+    prev_s = rnd((R, nh, N), 4, 1.0).double()
+    prev = (prev_s - torch.logsumexp(prev_s, -1, keepdim=True)).float()
+    prev_dev = prev.clone().cuda()
+    kl = torch.full((R, nh), -1.0, device="cuda")
+    out = torch.zeros((R, nh * dh), dtype=dtype, device="cuda")
+    Bd.polestar_k_attention(q, k, v, prev_dev, kl, out, nh, nkv, dh)
+    torch.cuda.synchronize()
+    qn, kn, vn = bf16_np(q).reshape(R, nh, dh), bf16_np(k).reshape(N, nkv, dh), bf16_np(v).reshape(N, nkv, dh)
+    logp = O.attn_logp_rows(qn, kn)
+    tol = 1e-4 if dtype == torch.float32 else 2e-2
+    rp = O.bf16_round if dtype == torch.bfloat16 else (lambda x: x)
+    ref_out = O.attn_out_rows(logp, vn, rp)
+    ref_kl = np.sum(np.exp(logp) * (logp - prev.double().numpy()), -1)
+    assert np.allclose(prev_dev.cpu().numpy(), logp, atol=2e-4, rtol=1e-5)       # stored rows = new log-probs
+    assert np.allclose(kl.cpu().numpy(), ref_kl, atol=1e-3 * max(1.0, np.abs(ref_kl).max()), rtol=1e-3)
+    assert np.allclose(bf16_np(out), ref_out, atol=tol, rtol=tol)
+    # Eq. 4 invariants: drift against the rows just stored is zero, and KL >= 0
+    kl2 = torch.full((R, nh), -1.0, device="cuda")
+    Bd.polestar_k_attention(q, k, v, prev_dev, kl2, None, nh, nkv, dh)
+    torch.cuda.synchronize()
+    assert np.abs(kl2.cpu().numpy()).max() < 1e-5
+    assert (kl.cpu().numpy() > -1e-4).all()
+    # Pinsker bound of Appendix B, Prop. 2 with the current value rows
+    M = np.linalg.norm(vn, axis=-1).max()
+    p_old = np.exp(prev.double().numpy())
+    for h in range(nh):
+        g = (h * nkv) // nh
+        d_out = np.linalg.norm((np.exp(logp[:, h]) - p_old[:, h]) @ vn[:, g], axis=-1)
+        assert (d_out <= M * np.sqrt(2 * np.maximum(kl.cpu().numpy()[:, h], 0)) + 1e-3).all()
+
+
+def test_attention_without_recording():
+    R, N, nh, dh = 20, 96, 2, 128
+    q = rnd((R, nh * dh), 1, 1.0, torch.bfloat16).cuda()
+    k = rnd((N, nh * dh), 2, 1.0, torch.bfloat16).cuda()
+    v = rnd((N, nh * dh), 3, 1.0, torch.bfloat16).cuda()
+    out = torch.zeros((R, nh * dh), dtype=torch.bfloat16, device="cuda")
+    Bd.polestar_k_attention(q, k, v, None, None, out, nh, nh, dh)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        q.float().view(R, nh, dh).permute(1, 0, 2)[None], k.float().view(N, nh, dh).permute(1, 0, 2)[None],
+        v.float().view(N, nh, dh).permute(1, 0, 2)[None])[0].permute(1, 0, 2).reshape(R, nh * dh)
+    assert torch.allclose(out.float(), ref, atol=2e-2, rtol=2e-2)
+
+
+# ------------------------------------------------------------------ hidden delta (a1b)
+@pytest.mark.parametrize("dtype,rows,d", [(torch.bfloat16, 4096, 4096), (torch.float32, 77, 256), (torch.bfloat16, 1, 8)])
+def test_hidden_delta(dtype, rows, d):
+    a = rnd((rows, d), 5, 1.0, dtype).cuda()
+    b = a.clone()
+    b[::3] += rnd((rows, d), 6, 0.5, dtype).cuda()[::3]
+    out = torch.empty(rows, device="cuda")
+    Bd.polestar_k_hidden_delta(a, b, out)
+    ref = ((a.double() - b.double()) ** 2).sum(-1)
+    assert torch.allclose(out.double(), ref, rtol=1e-4, atol=1e-6)
+    assert (out[1::3] == 0).all()                       # Cor. 1: unchanged rows give exactly zero
+
+
+# ------------------------------------------------------------------ select + compaction (a2)
+@pytest.mark.parametrize("W,batch", [(96, 1), (64, 3), (192, 8), (4096, 2), (1, 1), (1000, 1)])
+def test_select_matches_bruteforce(W, batch):
+    g = torch.Generator().manual_seed(W * 31 + batch)
+    z = torch.randn(batch, W, generator=g)
+    drift = torch.exp(z)
+    drift[:, ::7] = 0.0                                  # zero-drift rows are never candidates
+    if W > 8:
+        drift[:, 5] = drift[:, 3]                        # ties: lower index first
+    dd = drift.cuda()
+    idx = torch.full((batch, W), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    for mode, k, th in [(I.SELECT_TOPK_COUNT, max(1, W // 4), 0.0), (I.SELECT_TOPK_COUNT, W, 0.0),
+                        (I.SELECT_TOPK_COUNT, 1, 0.0), (I.SELECT_THRESHOLD, 0, 1.0), (I.SELECT_ALL, 0, 0.0),
+                        (I.SELECT_NONE, 0, 0.0), (I.SELECT_TOPK_COUNT, max(1, W // 100), 0.0)]:
+        Bd.polestar_k_select(dd, mode, k, th, 0.0, idx, cnt)
+        torch.cuda.synchronize()
+        for s in range(batch):
+            ref = O.select_rows(drift[s].numpy(), mode, k=k, thresh=th, floor=0.0)
+            n = int(cnt[s])
+            assert n == len(ref), (mode, k, s)
+            assert idx[s, :n].cpu().tolist() == ref.tolist()
+
+
+def test_select_zero_drift_and_nan():
+    d = torch.zeros(2, 96, device="cuda")
+    d[1, 10] = float("nan")
+    idx = torch.zeros((2, 96), dtype=torch.int32, device="cuda")
+    cnt = torch.full((2,), -1, dtype=torch.int32, device="cuda")
+    Bd.polestar_k_select(d, I.SELECT_TOPK_COUNT, 24, 0.0, 0.0, idx, cnt)
+    assert cnt.cpu().tolist() == [0, 0]
+
+
+# ------------------------------------------------------------------ gathered refresh (a3 + a4)
+@pytest.mark.parametrize("P,d,nh,nkv,k,batch", [(256, 256, 2, 2, 37, 1), (512, 512, 4, 1, 128, 2), (300, 256, 2, 2, 300, 1)])
+def test_refresh_chain_matches_oracle(P, d, nh, nkv, k, batch):
+    dh = 128
+    h, drift = I.make_refresh_inputs(batch, P, d)
+    m = I.ModelCfg(1, d, nh, nkv, dh, 2 * d, 1024, I.DTYPE_BF16, 1e-5, 500000.0)
+    w = I.make_weights(m, seed=5)
+    packed = Bd.pack_weights(m, w)
+    kc0 = rnd((batch, P, nkv * dh), 8, 1.0, torch.bfloat16)
+    vc0 = rnd((batch, P, nkv * dh), 9, 1.0, torch.bfloat16)
+    kc, vc = kc0.clone().cuda(), vc0.clone().cuda()
+    idx = torch.zeros((batch, k), dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(batch, dtype=torch.int32, device="cuda")
+    full_idx = torch.zeros((batch, P), dtype=torch.int32, device="cuda")
+    Bd.polestar_k_select(drift.cuda(), I.SELECT_TOPK_COUNT, k, 0.0, 0.0, full_idx, cnt)
+    idx.copy_(full_idx[:, :k])
+    q_out = torch.zeros((batch, k, nh * dh), dtype=torch.bfloat16, device="cuda")
+    scratch = torch.empty(Bd.polestar_k_refresh_scratch_bytes(batch, k, d, nh, nkv, dh) + 1024, dtype=torch.uint8, device="cuda")
+    off = (-scratch.data_ptr()) % 1024
+    Bd.polestar_k_refresh(h.cuda(), idx, cnt, packed["wqkv"][0], packed["norm1"][0], kc, vc, q_out, k, nh, nkv, dh,
+                          m.rms_eps, m.rope_theta, scratch[off:])
+    torch.cuda.synchronize()
+    wl = I.weights_to_numpy(w)["layers"][0]
+    inv = np.argsort(Bd.rope_interleave_index(dh).numpy())
+    for s in range(batch):
+        ridx, q_ref, K_ref, V_ref = O.refresh_chain(bf16_np(h[s]), drift[s].numpy(), k, wl["wq"], wl["wk"], wl["wv"],
+                                                    np.ones(d), m.rms_eps, m.rope_theta, nh, nkv, dh,
+                                                    bf16_np(kc0[s]).reshape(P, nkv, dh), bf16_np(vc0[s]).reshape(P, nkv, dh))
+        assert idx[s, :int(cnt[s])].cpu().tolist() == ridx.tolist()
+        Kg = bf16_np(kc[s]).reshape(P, nkv, dh)
+        Vg = bf16_np(vc[s]).reshape(P, nkv, dh)
+        Kg_log = Kg[..., inv]
+        assert np.allclose(Kg_log[ridx], K_ref[ridx], atol=2e-2, rtol=2e-2)
+        assert np.allclose(Vg[ridx], V_ref[ridx], atol=2e-2, rtol=2e-2)
+        qg = bf16_np(q_out[s]).reshape(k, nh, dh)[..., inv]
+        assert np.allclose(qg[:len(ridx)], q_ref, atol=2e-2, rtol=2e-2)
+        rest = np.setdiff1d(np.arange(P), ridx)          # rows not selected keep their bits
+        assert torch.equal(kc[s].cpu()[rest], kc0[s][rest]) and torch.equal(vc[s].cpu()[rest], vc0[s][rest])
+
+
+# ------------------------------------------------------------------ confidence (a6, first half)
+@pytest.mark.parametrize("rows,V", [(32, 126464), (7, 1024), (1, 50)])
+def test_confidence_matches_oracle(rows, V):
+    logits = rnd((rows, V), 11, 3.0)
+    mask_id = V - 1
+    logits[0, mask_id] = 50.0                            # [MASK] must never be predicted
+    if rows > 1:
+        logits[1, 3] = logits[1, 9] = 40.0               # tie: lowest id
+    yhat = torch.zeros(rows, dtype=torch.int32, device="cuda")
+    conf = torch.zeros(rows, device="cuda")
+    scratch = torch.empty(rows * 512, dtype=torch.uint8, device="cuda")
+    Bd.polestar_k_confidence(logits.cuda(), mask_id, yhat, conf, scratch)
+    ry, rc = O.confidence_rows(logits.numpy(), mask_id)
+    assert yhat.cpu().tolist() == ry.tolist()
+    assert np.allclose(conf.cpu().numpy(), rc, rtol=1e-4, atol=1e-7)

@@ -1,0 +1,115 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every declared symbol,
+sizes workspaces sensibly and rejects bad arguments before touching the device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+from paper_2607_14107_b200 import binding as Bd
+from paper_2607_14107_b200 import build as build_mod
+from paper_2607_14107_b200 import inputs as I
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_mod.build()
+    return Bd.load()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "polestar.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(polestar_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = declared_symbols()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(Bd.EXPORTS) == names
+
+
+def test_workspace_bytes(lib):
+    for name, lo, hi in [("c1", 1e6, 5e8), ("c2", 1e8, 5e9), ("c3", 5e8, 2e10), ("c4", 1e10, 6e10)]:
+        m, p = I.config(name)
+        n = Bd.polestar_workspace_bytes(m, p)
+        assert lo < n < hi, (name, n)
+    m, p = I.config("c1")
+    p.gen_len = 65                      # not a multiple of the block
+    assert Bd.polestar_workspace_bytes(m, p) == 0
+    m, p = I.config("c1")
+    m.n_heads = 3                       # not a multiple of the kv heads
+    assert Bd.polestar_workspace_bytes(m, p) == 0
+
+
+def test_init_rejects_bad_arguments_before_using_the_device(lib):
+    m, p = I.config("c1")
+    cm, cp = Bd.c_model(m), Bd.c_params(p)
+    ctx = C.c_void_p(123)
+    assert lib.polestar_init(C.byref(ctx), C.byref(cm), None, C.byref(cp), None, None, 0, None) == Bd.E_INVAL
+    assert ctx.value is None
+    assert lib.polestar_init(None, C.byref(cm), None, C.byref(cp), None, None, 0, None) == Bd.E_INVAL
+    assert lib.polestar_step(None, None) == Bd.E_INVAL
+    assert lib.polestar_commit(None, None) == Bd.E_INVAL
+    assert lib.polestar_tokens(None, None) == Bd.E_INVAL
+    lib.polestar_destroy(None)
+
+
+def test_kernel_entry_points_validate(lib):
+    assert lib.polestar_k_select(None, 1, 96, 0, 1, 0.0, 0.0, None, None, None) == Bd.E_INVAL
+    assert lib.polestar_k_attention(None, None, None, None, None, None, 1, 1, 1, 1, 64, 0, None) == Bd.E_INVAL
+    assert lib.polestar_k_hidden_delta(None, None, None, 1, 8, 0, None) == Bd.E_INVAL
+    assert lib.polestar_k_refresh_scratch_bytes(0, 1, 1, 1, 1, 1) == 0
+    assert lib.polestar_k_refresh_scratch_bytes(1, 128, 4096, 32, 32, 128) > 128 * 4096 * 2
+
+
+def test_strerror(lib):
+    assert lib.polestar_strerror(0) == b"ok"
+    for code in range(-7, 0):
+        if code != Bd.E_CUDA:
+            assert len(lib.polestar_strerror(code)) > 3
+
+
+def test_binding_refuses_to_run_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    m, p = I.config("c1")
+    with pytest.raises(Bd.PolestarError):
+        Bd.Polestar(m, {}, p, [[0] * p.prompt_len])
+
+
+def test_pack_weights_layout():
+    import torch
+    m = I.ModelCfg(1, 16, 2, 1, 8, 24, 32)
+    w = I.make_weights(m)
+    pk = Bd.pack_weights(m, w, device="cpu")
+    l = w["layers"][0]
+    qkv = pk["wqkv"][0]
+    assert qkv.shape == (2 * 8 + 2 * 8, 16)
+    # head 1 of q: packed row 2i = logical row i, 2i+1 = logical row i + 4
+    assert torch.equal(qkv[8 + 0], l["wq"][8 + 0]) and torch.equal(qkv[8 + 1], l["wq"][8 + 4])
+    assert torch.equal(qkv[8 + 6], l["wq"][8 + 3]) and torch.equal(qkv[8 + 7], l["wq"][8 + 7])
+    assert torch.equal(qkv[16 + 1], l["wk"][4]) and torch.equal(qkv[24:], l["wv"])
+    gu = pk["w_gate_up"][0]
+    assert torch.equal(gu[0], l["wg"][0]) and torch.equal(gu[1], l["wu"][0]) and torch.equal(gu[47], l["wu"][23])
+    # interleaving is a permutation of the head dimension: q.k is unchanged
+    x = torch.randn(16)
+    qa, ka = l["wq"][:8] @ x, l["wk"] @ x
+    qb, kb = qkv[:8] @ x, qkv[16:24] @ x
+    assert torch.allclose(qa @ ka, qb @ kb, atol=1e-6)
+
+
+def test_generator_is_device_independent_and_sliceable():
+    import torch
+    key = I.tensor_key(0, 3, I.T_WO)
+    a = I.normal_tensor(key, (64, 33), 0.02)
+    b = I.normal_range(key, 64 * 33 - 100, 100, 0.02)
+    assert torch.equal(a.flatten()[-100:], b)
+    assert abs(a.std().item() - 0.02) < 2e-3 and abs(a.mean().item()) < 2e-3
+    ids = I.make_prompt(*I.config("c2"))
+    assert ids.shape == (1, 256) and int(ids.max()) < 126463 and int(ids.min()) >= 0
