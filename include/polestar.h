@@ -78,6 +78,22 @@ extern "C" {
 #define POLESTAR_FLAG_NOCACHE       (1u << 3) /* every step is a full-sequence forward (baseline)   */
 #define POLESTAR_FLAG_KEEP_HIDDEN   (1u << 4) /* keep per-layer active hidden states for read-back  */
 #define POLESTAR_FLAG_SIMT_GEMM     (1u << 5) /* bf16 models: plain CUDA-core GEMMs (debug aid)     */
+#define POLESTAR_FLAG_PROMPT_DEVICE (1u << 6) /* polestar_init: prompt ids are a DEVICE array       */
+#define POLESTAR_FLAG_PROFILE       (1u << 7) /* bracket kernel families with CUDA events           */
+
+/* kernel families reported by polestar_profile */
+#define POLESTAR_PROF_GEMM_QKV     0
+#define POLESTAR_PROF_GEMM_O       1
+#define POLESTAR_PROF_GEMM_GATE_UP 2
+#define POLESTAR_PROF_GEMM_DOWN    3
+#define POLESTAR_PROF_GEMM_LM_HEAD 4
+#define POLESTAR_PROF_ATTENTION    5
+#define POLESTAR_PROF_STAGE        6  /* row table, embedding, RMSNorm staging */
+#define POLESTAR_PROF_SELECT       7
+#define POLESTAR_PROF_CONFIDENCE   8
+#define POLESTAR_PROF_COMMIT       9
+#define POLESTAR_PROF_MISC        10
+#define POLESTAR_PROF_FAMILIES    11
 
 #define POLESTAR_STEP_ENTRY_FULL   0
 #define POLESTAR_STEP_ENTRY_WINDOW 1
@@ -136,6 +152,7 @@ typedef struct {
     int32_t all_done;        /* 1: every block decoded                              */
     int64_t forwards;        /* forwards so far                                     */
     int64_t generated, generated_non_eos;  /* running totals (TPF numerator, App. D.1) */
+    int64_t launches;        /* kernels launched by this context so far             */
 } polestar_commit_info;
 
 /* ---- the decoding path ------------------------------------------------------------ */
@@ -147,6 +164,8 @@ size_t polestar_workspace_bytes(const polestar_model *m, const polestar_params *
 /* Create a context and run the block-0 entry forward (Algorithm 1: initial state,
  * block entry with a full-sequence forward, Sec. 4.1 "Initialization").
  *   prompt_ids_host  host, [batch][prompt_len] token ids in [0, vocab), none equal mask_id
+ *                    (with POLESTAR_FLAG_PROMPT_DEVICE: a device array of the same shape, not
+ *                    validated; out-of-range ids are clamped)
  *   workspace_dev    device, >= polestar_workspace_bytes(), 256-byte aligned, caller-owned;
  *                    the library zero-fills what it needs
  *   cuda_stream      cudaStream_t as void*
@@ -200,6 +219,12 @@ int polestar_read(polestar_ctx *c, int32_t what, int32_t layer, void *dst_host, 
                                     sequence, n absolute positions ([batch][n]; -1 = unused)     */
 #define POLESTAR_FORCE_CLEAR  3  /* drop all forced decisions                                     */
 int polestar_force(polestar_ctx *c, int32_t what, int32_t layer, const int32_t *idx_host, int32_t n);
+
+/* Per-family device time of the forwards so far (context created with POLESTAR_FLAG_PROFILE;
+ * harvested at every polestar_commit).  out_host: double [POLESTAR_PROF_FAMILIES][4] =
+ * {launch groups, milliseconds, algorithmic bytes, flops}.  reset != 0 clears the totals.
+ * The paper has no counterpart (its Appendix D breakdown figure is the closest). */
+int polestar_profile(polestar_ctx *c, double *out_host, int32_t reset);
 
 void polestar_destroy(polestar_ctx *c);
 const char *polestar_strerror(int code);

@@ -23,11 +23,13 @@ OK, E_INVAL, E_STATE, E_NOSPACE, E_CUDA, E_NONFINITE, E_TIMEOUT, E_DONE = 0, -1,
 READ_LOGITS, READ_CONF, READ_YHAT, READ_DELTA, READ_DRIFT, READ_SEL_COUNT, READ_SEL_IDX = 1, 2, 3, 4, 5, 6, 7
 READ_HIDDEN, READ_KCACHE, READ_VCACHE, READ_HCACHE, READ_COMMIT, READ_PPREV, READ_SUFFIX = 8, 9, 10, 11, 12, 13, 14
 FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR = 1, 2, 3
-FLAG_SIMT_GEMM = 1 << 5
+FLAG_SIMT_GEMM, FLAG_PROMPT_DEVICE, FLAG_PROFILE = 1 << 5, 1 << 6, 1 << 7
+PROF_FAMILIES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head", "attention", "stage", "select",
+                 "confidence", "commit", "misc"]
 
 EXPORTS = [
     "polestar_workspace_bytes", "polestar_init", "polestar_step", "polestar_commit", "polestar_tokens",
-    "polestar_read", "polestar_force", "polestar_destroy", "polestar_strerror",
+    "polestar_read", "polestar_force", "polestar_profile", "polestar_destroy", "polestar_strerror",
     "polestar_k_attention", "polestar_k_hidden_delta", "polestar_k_select",
     "polestar_k_refresh_scratch_bytes", "polestar_k_refresh", "polestar_k_confidence", "polestar_sm_count",
 ]
@@ -69,7 +71,8 @@ class CStepInfo(C.Structure):
 class CCommitInfo(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_committed", "n_by_conf", "n_by_drift", "n_by_quota", "n_suffix", "n_eos",
                                          "rows_refreshed", "block_index", "block_done", "all_done")] + \
-               [("forwards", C.c_int64), ("generated", C.c_int64), ("generated_non_eos", C.c_int64)]
+               [("forwards", C.c_int64), ("generated", C.c_int64), ("generated_non_eos", C.c_int64),
+                ("launches", C.c_int64)]
 
 
 _lib = None
@@ -99,6 +102,8 @@ def load():
     lib.polestar_read.argtypes = [vp, i32, i32, vp, sz]
     lib.polestar_force.restype = C.c_int
     lib.polestar_force.argtypes = [vp, i32, i32, C.POINTER(i32), i32]
+    lib.polestar_profile.restype = C.c_int
+    lib.polestar_profile.argtypes = [vp, C.POINTER(C.c_double), i32]
     lib.polestar_destroy.restype = None
     lib.polestar_destroy.argtypes = [vp]
     lib.polestar_strerror.restype = C.c_char_p
@@ -234,11 +239,16 @@ class Polestar:
         self._arrays = [arr(packed[k]) for k in ("wqkv", "wo", "w_gate_up", "w_down", "norm1", "norm2")]
         cw = CWeights(packed["embed"].data_ptr(), packed["lm_head"].data_ptr(), packed["final_norm"].data_ptr(),
                       *self._arrays)
-        prompt = np.ascontiguousarray(np.asarray(prompt, dtype=np.int32).reshape(p.batch, p.prompt_len))
+        if p.flags & FLAG_PROMPT_DEVICE:
+            self._prompt = prompt.to(device="cuda", dtype=torch.int32).contiguous()
+            prompt_ptr = C.cast(C.c_void_p(self._prompt.data_ptr()), C.POINTER(C.c_int32))
+        else:
+            self._prompt = np.ascontiguousarray(np.asarray(prompt, dtype=np.int32).reshape(p.batch, p.prompt_len))
+            prompt_ptr = self._prompt.ctypes.data_as(C.POINTER(C.c_int32))
         self.ctx = C.c_void_p()
         base = (self.workspace.data_ptr() + 255) & ~255
         _check(lib.polestar_init(C.byref(self.ctx), C.byref(cm), C.byref(cw), C.byref(cp),
-                                 prompt.ctypes.data_as(C.POINTER(C.c_int32)), C.c_void_p(base),
+                                 prompt_ptr, C.c_void_p(base),
                                  need + 1024 - (base - self.workspace.data_ptr()), C.c_void_p(_stream())))
         self.done = False
 
@@ -287,6 +297,12 @@ class Polestar:
             inv = np.argsort(rope_interleave_index(m.head_dim).numpy())
             out = out.reshape(bs, N, m.n_kv_heads, m.head_dim)[..., inv].reshape(bs, N, dkv)
         return out
+
+    def profile(self, reset: bool = False) -> Dict:
+        out = (C.c_double * (len(PROF_FAMILIES) * 4))()
+        _check(load().polestar_profile(self.ctx, out, 1 if reset else 0))
+        return {f: dict(calls=out[4 * i], ms=out[4 * i + 1], bytes=out[4 * i + 2], flops=out[4 * i + 3])
+                for i, f in enumerate(PROF_FAMILIES)}
 
     def force_select(self, layer: int, idx) -> None:
         idx = np.ascontiguousarray(np.asarray(idx, np.int32).reshape(self.p.batch, -1))

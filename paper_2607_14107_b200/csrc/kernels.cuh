@@ -649,10 +649,7 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
         c = a.conf[s * B + j];
         yh = a.yhat[s * B + j];
         if (within) {
-            const float* kr = a.kl + (size_t)(s * sd.rows_per_seq + a.act_row_off + j) * a.n_heads;
-            float acc = 0.f;
-            for (int h = 0; h < a.n_heads; ++h) acc += kr[h];
-            dl = acc / (float)a.n_heads;
+            dl = a.delta_out[s * B + j];      // written by delta_kernel at the end of the forward
             const int pushed = a.theta_cnt[s];
             const int nh = min(pushed, a.hist);
             float mean = 0.f;
@@ -751,6 +748,20 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
     }
 }
 
+// Last-layer drift of the active rows (Algorithm 1, delta): mean over heads of the per-head KL.
+__global__ void delta_kernel(StepDesc sd, const float* kl, int act_row_off, int n_heads, float* delta) {
+    const int s = blockIdx.x, j = threadIdx.x;
+    if (j >= sd.B) return;
+    float dl = 0.f;
+    if (sd.record_kl) {
+        const float* kr = kl + (size_t)(s * sd.rows_per_seq + act_row_off + j) * n_heads;
+        float acc = 0.f;
+        for (int h = 0; h < n_heads; ++h) acc += kr[h];
+        dl = acc / (float)n_heads;
+    }
+    delta[s * sd.B + j] = dl;
+}
+
 // gather rows of x into a keep buffer: dst[s][j][:] = x[row(s, j)][:]
 __global__ void keep_hidden_kernel(StepDesc sd, const float* x, int act_row_off, int d, float* dst) {
     const int i = blockIdx.x;
@@ -758,6 +769,20 @@ __global__ void keep_hidden_kernel(StepDesc sd, const float* x, int act_row_off,
     const float* src = x + (size_t)(s * sd.rows_per_seq + act_row_off + j) * d;
     float* o = dst + (size_t)i * d;
     for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = src[c];
+}
+
+// y = [prompt ; MASK ...] from a prompt that already lives on the device (ids clamped to the vocabulary)
+__global__ void init_tokens_kernel(int* y, const int* prompt, int batch, int prompt_len, int N, int mask_id, int vocab) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= batch * N) return;
+    const int s = i / N, pos = i - s * N;
+    int t = mask_id;
+    if (pos < prompt_len) {
+        t = prompt[s * prompt_len + pos];
+        t = t < 0 ? 0 : (t >= vocab ? vocab - 1 : t);
+        if (t == mask_id) t = (mask_id + 1) % vocab;
+    }
+    y[i] = t;
 }
 
 // rotary table: tab[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), computed in double precision

@@ -189,6 +189,38 @@ struct polestar_ctx {
     bool forced_select = false, forced_commit = false;
     int forced_commit_n = 0;
     std::vector<int> seq_info_host;
+    // launch accounting and optional per-family device timing (POLESTAR_FLAG_PROFILE)
+    long long launches = 0;
+    struct ProfRec { int fam; size_t ev; double bytes, flops; };
+    std::vector<cudaEvent_t> prof_ev;
+    std::vector<ProfRec> prof_recs;
+    size_t prof_used = 0;
+    double prof_acc[POLESTAR_PROF_FAMILIES][4] = {};
+};
+
+// Scope of one kernel family inside a forward: counts launches, and with FLAG_PROFILE brackets the
+// launches with CUDA events that polestar_commit turns into per-family device times.
+struct Scope {
+    polestar_ctx* c;
+    bool on;
+    size_t ev = 0;
+    Scope(polestar_ctx* c_, int fam, double bytes, double flops, int n_launches) : c(c_) {
+        c->launches += n_launches;
+        on = (c->p.flags & POLESTAR_FLAG_PROFILE) != 0;
+        if (!on) return;
+        while (c->prof_ev.size() < c->prof_used + 2) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { on = false; return; }
+            c->prof_ev.push_back(e);
+        }
+        ev = c->prof_used;
+        c->prof_used += 2;
+        cudaEventRecord(c->prof_ev[ev], c->st);
+        c->prof_recs.push_back({fam, ev, bytes, flops});
+    }
+    ~Scope() {
+        if (on) cudaEventRecord(c->prof_ev[ev + 1], c->st);
+    }
 };
 
 static bool valid_cfg(const polestar_model* m, const polestar_params* p) {
@@ -361,11 +393,19 @@ struct Path {
         const bool sparse = within && any_refresh;
         int rc;
 
-        build_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(sd, b.rows);
-        CK(cudaMemsetAsync(b.stats, 0, 4 * sizeof(int), st));
-        embed_rows_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.y, (const T*)c->embed, d, b.x, b.packet, b.patch,
-                                               b.tok_at_h0, b.stats);
-        CK(cudaGetLastError());
+        const double esd = (double)es;
+        const double Mlive = sparse ? (double)bs * (B + std::min(sd.W, (int)(p.select_mode == POLESTAR_SELECT_TOPK_FRAC
+                                                       ? floorf(p.select_frac * (float)sd.W + 0.5f)
+                                                       : (p.select_mode == POLESTAR_SELECT_TOPK_COUNT ? p.select_k : sd.W))))
+                                    : (double)M;
+        {
+            Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (esd + 4), 0, 2);
+            build_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(sd, b.rows);
+            CK(cudaMemsetAsync(b.stats, 0, 4 * sizeof(int), st));
+            embed_rows_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.y, (const T*)c->embed, d, b.x, b.packet, b.patch,
+                                                   b.tok_at_h0, b.stats);
+            CK(cudaGetLastError());
+        }
 
         for (int l = 0; l < L; ++l) {
             char* kc = b.kc + (size_t)l * bs * N * dkv * es;
@@ -373,33 +413,46 @@ struct Path {
             float* hc = b.hc + (size_t)l * bs * Wm * d;
             float* pprev = b.pprev + (size_t)l * bs * Wm * m.n_heads * N;
             const bool last = l == L - 1;
-            if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN)
+            if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
+                Scope sc(c, POLESTAR_PROF_MISC, 0, 0, 1);
                 keep_hidden_kernel<<<bs * B, 256, 0, st>>>(sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d);
-
-            prep_qkv_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
-                                                 c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag);
-            CK(cudaGetLastError());
-
+            }
+            {
+                Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
+                prep_qkv_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
+                                                     c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag);
+                CK(cudaGetLastError());
+            }
             EpiArgs e;
-            memset(&e, 0, sizeof(e));
-            e.rows = b.rows; e.kvflag = b.kvflag; e.rope = b.rope; e.q_out = b.q_buf; e.kc = kc; e.vc = vc;
-            e.N_seq = N; e.n_heads = m.n_heads; e.n_kv = m.n_kv_heads; e.head_dim = m.head_dim; e.W_max = Wm;
-            e.within = within; e.ld_out = dq;
-            if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->M_max, c->wqkv[l], M, dq + 2 * dkv, d, e))) return rc;
-
-            AttnArgs a;
-            memset(&a, 0, sizeof(a));
-            a.rows = b.rows; a.n_rows = M; a.q = b.q_buf; a.kc = kc; a.vc = vc; a.out = b.o_buf;
-            a.pprev = (sparse || !within) ? pprev : nullptr;
-            a.aprev = last ? b.aprev : nullptr;
-            a.kl = b.kl; a.N = N; a.n_heads = m.n_heads; a.n_kv = m.n_kv_heads; a.head_dim = m.head_dim;
-            a.W_max = Wm; a.B = B; a.record_kl = sd.record_kl; a.rows_per_seq = sd.rows_per_seq; a.batch = bs;
-            a.scale = 1.0f / sqrtf((float)m.head_dim);
-            if ((rc = attention(c, a))) return rc;
-
+            {
+                const double nq = dq + 2 * dkv;
+                Scope sc(c, POLESTAR_PROF_GEMM_QKV, (nq * d + (double)M * d + (double)M * nq) * esd, 2.0 * M * nq * d, 1);
+                memset(&e, 0, sizeof(e));
+                e.rows = b.rows; e.kvflag = b.kvflag; e.rope = b.rope; e.q_out = b.q_buf; e.kc = kc; e.vc = vc;
+                e.N_seq = N; e.n_heads = m.n_heads; e.n_kv = m.n_kv_heads; e.head_dim = m.head_dim; e.W_max = Wm;
+                e.within = within; e.ld_out = dq;
+                if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->M_max, c->wqkv[l], M, dq + 2 * dkv, d, e))) return rc;
+            }
+            {
+                const bool rec_w = sparse || !within;
+                const double rec_rows = (rec_w ? (double)bs * sd.W : 0.0) + (last ? (double)bs * B : 0.0);
+                Scope sc(c, POLESTAR_PROF_ATTENTION,
+                         2.0 * bs * N * dkv * esd + 2.0 * M * dq * esd + (sd.record_kl ? 2.0 : 1.0) * rec_rows * m.n_heads * N * 4,
+                         4.0 * M * (double)N * dq, 1);
+                AttnArgs a;
+                memset(&a, 0, sizeof(a));
+                a.rows = b.rows; a.n_rows = M; a.q = b.q_buf; a.kc = kc; a.vc = vc; a.out = b.o_buf;
+                a.pprev = rec_w ? pprev : nullptr;
+                a.aprev = last ? b.aprev : nullptr;
+                a.kl = b.kl; a.N = N; a.n_heads = m.n_heads; a.n_kv = m.n_kv_heads; a.head_dim = m.head_dim;
+                a.W_max = Wm; a.B = B; a.record_kl = sd.record_kl; a.rows_per_seq = sd.rows_per_seq; a.batch = bs;
+                a.scale = 1.0f / sqrtf((float)m.head_dim);
+                if ((rc = attention(c, a))) return rc;
+            }
             const int* list = nullptr;
             const int* m2_count = nullptr;
             if (sparse) {
+                Scope sc(c, POLESTAR_PROF_SELECT, (double)bs * sd.W * (m.n_heads * 4 + 8), 0, 1);
                 StepSelArgs s;
                 memset(&s, 0, sizeof(s));
                 s.kl = b.kl; s.drift = b.drift + (size_t)l * bs * Wm; s.sel_idx = b.sel_idx + (size_t)l * bs * Wm;
@@ -413,44 +466,64 @@ struct Path {
                 CK(cudaGetLastError());
                 list = b.list; m2_count = b.list_count;
             }
-
-            memset(&e, 0, sizeof(e));
-            e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
-            if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e))) return rc;
-
-            prep_rows_kernel<T><<<M, 256, 0, st>>>(b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf);
-            CK(cudaGetLastError());
-
-            memset(&e, 0, sizeof(e));
-            e.out_t = b.g_buf; e.ld_out = F; e.m_count = m2_count;
-            if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->M_max, c->wgu[l], M, 2 * F, d, e))) return rc;
-
-            memset(&e, 0, sizeof(e));
-            e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = b.x1; e.out_f32 = b.x; e.packet = b.packet;
-            e.W_max = Wm; e.within = within; e.ld_out = d;
-            if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e))) return rc;
+            {
+                Scope sc(c, POLESTAR_PROF_GEMM_O, (double)d * dq * esd + (double)M * dq * esd + 2.0 * M * d * 4, 2.0 * M * d * (double)dq, 1);
+                memset(&e, 0, sizeof(e));
+                e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
+                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e))) return rc;
+            }
+            {
+                Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
+                prep_rows_kernel<T><<<M, 256, 0, st>>>(b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf);
+                CK(cudaGetLastError());
+            }
+            {
+                Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, (2.0 * F * d + Mlive * d + Mlive * F) * esd, 4.0 * Mlive * F * (double)d, 1);
+                memset(&e, 0, sizeof(e));
+                e.out_t = b.g_buf; e.ld_out = F; e.m_count = m2_count;
+                if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->M_max, c->wgu[l], M, 2 * F, d, e))) return rc;
+            }
+            {
+                Scope sc(c, POLESTAR_PROF_GEMM_DOWN, ((double)F * d + Mlive * F) * esd + 2.0 * Mlive * d * 4, 2.0 * Mlive * F * (double)d, 1);
+                memset(&e, 0, sizeof(e));
+                e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = b.x1; e.out_f32 = b.x; e.packet = b.packet;
+                e.W_max = Wm; e.within = within; e.ld_out = d;
+                if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e))) return rc;
+            }
         }
-        if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN)
+        if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
+            Scope sc(c, POLESTAR_PROF_MISC, 0, 0, 1);
             keep_hidden_kernel<<<bs * B, 256, 0, st>>>(sd, b.x, act_off, d, b.hidden_keep + (size_t)L * bs * B * d);
+        }
 
         // logits of the active rows (+ eligible suffix rows), confidences
         const int use_suffix = sparse && (p.flags & POLESTAR_FLAG_SUFFIX_COMMIT);
-        build_head_list_kernel<<<1, 256, 0, st>>>(sd, b.y, m.mask_id, b.sel_idx + (size_t)(L - 1) * bs * Wm,
-                                                  b.sel_cnt + (size_t)(L - 1) * bs, use_suffix, 0, b.head_list,
-                                                  b.head_count, b.suf_seq, b.suf_w);
-        CK(cudaGetLastError());
         const int Mh = use_suffix ? c->rows_lm : bs * B;
-        prep_head_kernel<T><<<Mh, 256, 0, st>>>(b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
-                                               (T*)b.a_head);
-        CK(cudaGetLastError());
-        EpiArgs e;
-        memset(&e, 0, sizeof(e));
-        e.out_f32 = b.logits; e.ld_out = m.vocab; e.scale = p.logit_scale; e.m_count = b.head_count;
-        if ((rc = gemm<EPI_LOGITS>(c, b.a_head, c->rows_lm, c->lm_head, Mh, m.vocab, d, e))) return rc;
-        conf_partial_kernel<<<dim3(CONF_CHUNKS, Mh), 256, 0, st>>>(b.logits, b.head_count, Mh, m.vocab, m.mask_id,
-                                                                  CONF_CHUNKS, b.conf_part);
-        conf_final_kernel<<<(Mh + 127) / 128, 128, 0, st>>>(b.conf_part, b.head_count, Mh, CONF_CHUNKS, b.yhat, b.conf);
-        CK(cudaGetLastError());
+        {
+            Scope sc(c, POLESTAR_PROF_STAGE, (double)bs * B * d * (4 + esd), 0, 2);
+            build_head_list_kernel<<<1, 256, 0, st>>>(sd, b.y, m.mask_id, b.sel_idx + (size_t)(L - 1) * bs * Wm,
+                                                      b.sel_cnt + (size_t)(L - 1) * bs, use_suffix, 0, b.head_list,
+                                                      b.head_count, b.suf_seq, b.suf_w);
+            prep_head_kernel<T><<<Mh, 256, 0, st>>>(b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
+                                                   (T*)b.a_head);
+            CK(cudaGetLastError());
+        }
+        {
+            Scope sc(c, POLESTAR_PROF_GEMM_LM_HEAD, ((double)m.vocab * d + (double)bs * B * d) * esd + (double)bs * B * m.vocab * 4,
+                     2.0 * bs * B * (double)m.vocab * d, 1);
+            EpiArgs e;
+            memset(&e, 0, sizeof(e));
+            e.out_f32 = b.logits; e.ld_out = m.vocab; e.scale = p.logit_scale; e.m_count = b.head_count;
+            if ((rc = gemm<EPI_LOGITS>(c, b.a_head, c->rows_lm, c->lm_head, Mh, m.vocab, d, e))) return rc;
+        }
+        {
+            Scope sc(c, POLESTAR_PROF_CONFIDENCE, (double)bs * B * m.vocab * 4, 0, 3);
+            conf_partial_kernel<<<dim3(CONF_CHUNKS, Mh), 256, 0, st>>>(b.logits, b.head_count, Mh, m.vocab, m.mask_id,
+                                                                      CONF_CHUNKS, b.conf_part);
+            conf_final_kernel<<<(Mh + 127) / 128, 128, 0, st>>>(b.conf_part, b.head_count, Mh, CONF_CHUNKS, b.yhat, b.conf);
+            delta_kernel<<<bs, 256, 0, st>>>(sd, b.kl, act_off, m.n_heads, b.delta);
+            CK(cudaGetLastError());
+        }
         c->last_act_row_off = act_off;
         return POLESTAR_OK;
     }
@@ -543,13 +616,25 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     a.tau_s = p.tau_s; a.alpha = p.alpha; a.tau_suffix = p.tau_suffix;
     const bool entry_like = sd.record_kl == 0;
     if (entry_like) CK(cudaMemsetAsync(b.theta_cnt, 0, p.batch * sizeof(int), c->st));   // history cleared at block entry
-    commit_kernel<<<p.batch, 256, 0, c->st>>>(sd, a);
-    CK(cudaGetLastError());
+    {
+        Scope sc(c, POLESTAR_PROF_COMMIT, (double)p.batch * c->B * 16, 0, 1);
+        commit_kernel<<<p.batch, 256, 0, c->st>>>(sd, a);
+        CK(cudaGetLastError());
+    }
     c->seq_info_host.resize((size_t)p.batch * 8 + 8);
     CK(cudaMemcpyAsync(c->seq_info_host.data(), b.seq_info, (size_t)p.batch * 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
     CK(cudaMemcpyAsync(c->seq_info_host.data() + p.batch * 8, b.stats, 4 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
     CK(cudaMemcpyAsync(c->seq_info_host.data() + p.batch * 8 + 4, b.status, sizeof(int), cudaMemcpyDeviceToHost, c->st));
     CK(cudaStreamSynchronize(c->st));
+    for (const auto& r : c->prof_recs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->prof_ev[r.ev], c->prof_ev[r.ev + 1]) == cudaSuccess) {
+            c->prof_acc[r.fam][0] += 1; c->prof_acc[r.fam][1] += ms;
+            c->prof_acc[r.fam][2] += r.bytes; c->prof_acc[r.fam][3] += r.flops;
+        }
+    }
+    c->prof_recs.clear();
+    c->prof_used = 0;
     c->pending = false;
     c->forced_commit = false;
     const int* si = c->seq_info_host.data();
@@ -581,6 +666,7 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
         if (c->block >= c->n_blocks) { c->done = true; ci.all_done = 1; }
     }
     ci.forwards = c->forwards; ci.generated = c->generated; ci.generated_non_eos = c->generated_non_eos;
+    ci.launches = c->launches;
     if (info) *info = ci;
     if (status) return POLESTAR_E_TIMEOUT;
     if (nonfinite) return POLESTAR_E_NONFINITE;
@@ -596,8 +682,10 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
         !w->norm2)
         return POLESTAR_E_INVAL;
     if (((uintptr_t)ws) & 255) return POLESTAR_E_INVAL;
-    for (int i = 0; i < p->batch * p->prompt_len; ++i)
-        if (prompt[i] < 0 || prompt[i] >= m->vocab || prompt[i] == m->mask_id) return POLESTAR_E_INVAL;
+    const bool prompt_dev = (p->flags & POLESTAR_FLAG_PROMPT_DEVICE) != 0;
+    if (!prompt_dev)
+        for (int i = 0; i < p->batch * p->prompt_len; ++i)
+            if (prompt[i] < 0 || prompt[i] >= m->vocab || prompt[i] == m->mask_id) return POLESTAR_E_INVAL;
     const size_t need = make_plan(m, p, nullptr, nullptr);
     if (ws_bytes < need) return POLESTAR_E_NOSPACE;
     int rc = init_device_info();
@@ -634,11 +722,16 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     if (cudaMemsetAsync(c->b.forced_cnt, 0xFF, (size_t)m->n_layers * p->batch * sizeof(int), c->st) != cudaSuccess)
         return fail(POLESTAR_E_CUDA);
     if (cudaMemsetAsync(c->b.gemm_counters, 0, GEMM_COUNTERS * sizeof(int), c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
-    std::vector<int> y((size_t)p->batch * c->N, m->mask_id);
-    for (int s = 0; s < p->batch; ++s)
-        for (int i = 0; i < p->prompt_len; ++i) y[(size_t)s * c->N + i] = prompt[(size_t)s * p->prompt_len + i];
-    if (cudaMemcpyAsync(c->b.y, y.data(), y.size() * sizeof(int), cudaMemcpyHostToDevice, c->st) != cudaSuccess)
-        return fail(POLESTAR_E_CUDA);
+    if (prompt_dev) {
+        init_tokens_kernel<<<(p->batch * c->N + 255) / 256, 256, 0, c->st>>>(c->b.y, prompt, p->batch, p->prompt_len, c->N,
+                                                                            m->mask_id, m->vocab);
+    } else {
+        std::vector<int> y((size_t)p->batch * c->N, m->mask_id);
+        for (int s = 0; s < p->batch; ++s)
+            for (int i = 0; i < p->prompt_len; ++i) y[(size_t)s * c->N + i] = prompt[(size_t)s * p->prompt_len + i];
+        if (cudaMemcpyAsync(c->b.y, y.data(), y.size() * sizeof(int), cudaMemcpyHostToDevice, c->st) != cudaSuccess)
+            return fail(POLESTAR_E_CUDA);
+    }
     const int half = m->head_dim / 2;
     rope_table_kernel<<<(c->N * half + 255) / 256, 256, 0, c->st>>>(c->b.rope, c->N, half, (double)m->rope_theta);
     if (cudaStreamSynchronize(c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
@@ -651,7 +744,15 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
 extern "C" void polestar_destroy(polestar_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->st);
+    for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     delete c;
+}
+
+extern "C" int polestar_profile(polestar_ctx* c, double* out, int32_t reset) {
+    if (!c || !out) return POLESTAR_E_INVAL;
+    memcpy(out, c->prof_acc, sizeof(c->prof_acc));
+    if (reset) memset(c->prof_acc, 0, sizeof(c->prof_acc));
+    return POLESTAR_OK;
 }
 
 extern "C" int polestar_tokens(polestar_ctx* c, int32_t* out) {
@@ -836,14 +937,11 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     __nv_bfloat16* a_buf = (__nv_bfloat16*)sc;
     float2* rope = (float2*)(sc + off_rope);
     static MapCache maps;
-    static const void* counters_zeroed_for = nullptr;
     GemmWs ws;
     ws.partial = (float*)(sc + off_part); ws.partial_bytes = GEMM_PARTIAL_BYTES / 2;
     ws.counters = (int*)(sc + off_cnt); ws.n_counters = GEMM_COUNTERS; ws.status = (int*)(sc + off_status);
-    if (counters_zeroed_for != scratch) {
-        CK(cudaMemsetAsync(ws.counters, 0, GEMM_COUNTERS * sizeof(int) + 1024, st));
-        counters_zeroed_for = scratch;
-    }
+    // the scratch is caller memory with unknown contents: the split-K tile counters must start at zero
+    CK(cudaMemsetAsync(ws.counters, 0, GEMM_COUNTERS * sizeof(int) + 1024, st));
     const int half = head_dim / 2;
     rope_table_kernel<<<(P * half + 255) / 256, 256, 0, st>>>(rope, P, half, (double)rope_theta);
     const int M = batch * max_rows;

@@ -24,7 +24,8 @@ def close(a, b, tol, what=""):
 
 def setup(name, **kw):
     m, p = I.config(name)
-    p = dataclasses.replace(p, flags=p.flags | I.FLAG_KEEP_HIDDEN, **kw)
+    kw["flags"] = kw.get("flags", p.flags) | I.FLAG_KEEP_HIDDEN
+    p = dataclasses.replace(p, **kw)
     w = I.make_weights(m, seed=0)
     wn = I.weights_to_numpy(w)
     prompt = I.make_prompt(m, p)
@@ -70,7 +71,8 @@ def run_forced(name, n_steps, **kw):
             trs = ora.seqs[s].trace
             for l in range(L + 1):
                 close(gpu.read(Bd.READ_HIDDEN, l)[s], trs["x_act"][l], tol, f"step {step} hidden l{l}")
-            close(gpu.read(Bd.READ_LOGITS)[s], trs["logits"], tol, f"step {step} logits")
+            # logits are multiplied by logit_scale, and so is their absolute error
+            close(gpu.read(Bd.READ_LOGITS)[s] / p.logit_scale, trs["logits"] / p.logit_scale, tol, f"step {step} logits")
             if trs["kind"] == "within":
                 seen["within"] += 1
                 close(gpu.read(Bd.READ_DELTA)[s], trs["delta"], tol, f"step {step} delta")
@@ -112,13 +114,13 @@ def test_c1_forced_decisions_every_step():
 
 
 def test_c1_refresh_every_step_with_scaled_logits():
-    seen = run_forced("c1", 20, tau_upd=-1, logit_scale=25.0, tau_suffix=0.5)
-    assert seen["refresh"] > 3
+    seen = run_forced("c1", 20, tau_upd=-1, logit_scale=12.0, tau_suffix=0.5)
+    assert seen["refresh"] > 10
 
 
 def test_c1b_bf16_tensor_core_path():
-    seen = run_forced("c1b", 16, tau_upd=-1, logit_scale=20.0)
-    assert seen["refresh"] > 3
+    seen = run_forced("c1b", 16, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["refresh"] > 5
 
 
 def test_c1b_bf16_simt_gemm_path():
@@ -133,6 +135,7 @@ def test_c1_batch2_gqa():
     prompt = I.make_prompt(m, p)
     gpu = Bd.Polestar(m, Bd.pack_weights(m, w), p, prompt.numpy())
     ora = O.PolestarOracle(m, I.weights_to_numpy(w), p, prompt.numpy())
+    ora.step()
     gpu.commit(); ora.commit()
     for step in range(10):
         gpu.step(); ora.step()
@@ -145,7 +148,7 @@ def test_c1_batch2_gqa():
 def test_c1_free_running_matches_oracle():
     """Both sides take their own decisions; fp32 margins are far above the arithmetic error, so
     index sets and committed tokens must agree exactly (a low-margin decision ends the check)."""
-    m, p, gpu, ora = setup("c1", logit_scale=25.0, tau_upd=2)
+    m, p, gpu, ora = setup("c1", logit_scale=12.0, tau_upd=2)
     tol = TOL[m.dtype]
     first = True
     n_steps = 0
