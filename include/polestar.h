@@ -40,6 +40,13 @@
  *   w_gate_up[l]    [2 * d_ffn, d_model]: row 2f is gate row f, row 2f+1 is up row f
  *   w_down[l]       [d_model, d_ffn]
  *   norm1[l], norm2[l], final_norm   [d_model] float32 gains
+ *
+ *   TILE-MAJOR storage: a bf16 GEMM weight (wqkv, wo, w_gate_up, w_down, lm_head) whose
+ *   out-features are a multiple of 256 and in-features a multiple of 64 is stored as contiguous
+ *   [256][64] blocks, block (o / 256, i / 64) at block index (o / 256) * (in / 64) + i / 64 and
+ *   element (o % 256, i % 64) inside it; the row order above applies to the index o.  Every
+ *   other matrix (fp32 models, odd shapes, the embedding table) is plain row-major.  Streaming
+ *   kernels then read each weight block as one sequential 32 KB burst.
  */
 #ifndef POLESTAR_H
 #define POLESTAR_H
@@ -218,6 +225,9 @@ int polestar_read(polestar_ctx *c, int32_t what, int32_t layer, void *dst_host, 
 #define POLESTAR_FORCE_COMMIT 2  /* positions committed by the next commit: idx_host holds, per
                                     sequence, n absolute positions ([batch][n]; -1 = unused)     */
 #define POLESTAR_FORCE_CLEAR  3  /* drop all forced decisions                                     */
+#define POLESTAR_FORCE_TOKENS 4  /* after FORCE_COMMIT with the same n: token ids written at those
+                                    positions ([batch][n]) instead of the library's own argmax (two
+                                    near-equal logits may rank differently in another arithmetic)  */
 int polestar_force(polestar_ctx *c, int32_t what, int32_t layer, const int32_t *idx_host, int32_t n);
 
 /* Per-family device time of the forwards so far (context created with POLESTAR_FLAG_PROFILE;

@@ -22,7 +22,7 @@ OK, E_INVAL, E_STATE, E_NOSPACE, E_CUDA, E_NONFINITE, E_TIMEOUT, E_DONE = 0, -1,
 
 READ_LOGITS, READ_CONF, READ_YHAT, READ_DELTA, READ_DRIFT, READ_SEL_COUNT, READ_SEL_IDX = 1, 2, 3, 4, 5, 6, 7
 READ_HIDDEN, READ_KCACHE, READ_VCACHE, READ_HCACHE, READ_COMMIT, READ_PPREV, READ_SUFFIX = 8, 9, 10, 11, 12, 13, 14
-FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR = 1, 2, 3
+FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR, FORCE_TOKENS = 1, 2, 3, 4
 FLAG_SIMT_GEMM, FLAG_PROMPT_DEVICE, FLAG_PROFILE = 1 << 5, 1 << 6, 1 << 7
 PROF_FAMILIES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head", "attention", "stage", "select",
                  "confidence", "commit", "misc"]
@@ -169,6 +169,24 @@ def rope_interleave_index(head_dim: int) -> torch.Tensor:
     return idx
 
 
+TILE_ROWS = 256   # out-features per weight block of the tile-major layout
+
+
+def tile_major(w: torch.Tensor) -> torch.Tensor:
+    """[out, in] -> contiguous [256][64] blocks (bf16, out % 256 == 0, in % 64 == 0); else unchanged."""
+    o, i = w.shape
+    if w.dtype != torch.bfloat16 or o % TILE_ROWS or i % 64:
+        return w.contiguous()
+    return w.view(o // TILE_ROWS, TILE_ROWS, i // 64, 64).permute(0, 2, 1, 3).contiguous().view(o, i)
+
+
+def untile(w: torch.Tensor) -> torch.Tensor:
+    o, i = w.shape
+    if w.dtype != torch.bfloat16 or o % TILE_ROWS or i % 64:
+        return w
+    return w.view(o // TILE_ROWS, i // 64, TILE_ROWS, 64).permute(0, 2, 1, 3).contiguous().view(o, i)
+
+
 def pack_weights(m: I.ModelCfg, w: Dict, device="cuda", consume: bool = False) -> Dict:
     """Logical weights (inputs.make_weights) -> the library's device layout."""
     dev = torch.device(device)
@@ -181,18 +199,18 @@ def pack_weights(m: I.ModelCfg, w: Dict, device="cuda", consume: bool = False) -
 
     out = {"wqkv": [], "wo": [], "w_gate_up": [], "w_down": [], "norm1": [], "norm2": []}
     if "embed" in w:
-        out.update({"embed": w["embed"].to(dev, dt).contiguous(), "lm_head": w["lm_head"].to(dev, dt).contiguous(),
+        out.update({"embed": w["embed"].to(dev, dt).contiguous(), "lm_head": tile_major(w["lm_head"].to(dev, dt)),
                     "final_norm": w["final_norm"].to(dev, torch.float32).contiguous()})
     layers = w["layers"]
     for i in range(len(layers)):
         l = layers[i]
         q = heads_perm(l["wq"].to(dev, dt), m.n_heads)
         k = heads_perm(l["wk"].to(dev, dt), m.n_kv_heads)
-        out["wqkv"].append(torch.cat([q, k, l["wv"].to(dev, dt)], 0).contiguous())
-        out["wo"].append(l["wo"].to(dev, dt).contiguous())
-        out["w_gate_up"].append(torch.stack([l["wg"].to(dev, dt), l["wu"].to(dev, dt)], 1)
-                                .reshape(2 * m.d_ffn, m.d_model).contiguous())
-        out["w_down"].append(l["wd"].to(dev, dt).contiguous())
+        out["wqkv"].append(tile_major(torch.cat([q, k, l["wv"].to(dev, dt)], 0)))
+        out["wo"].append(tile_major(l["wo"].to(dev, dt)))
+        out["w_gate_up"].append(tile_major(torch.stack([l["wg"].to(dev, dt), l["wu"].to(dev, dt)], 1)
+                                           .reshape(2 * m.d_ffn, m.d_model)))
+        out["w_down"].append(tile_major(l["wd"].to(dev, dt)))
         out["norm1"].append(l["norm1"].to(dev, torch.float32).contiguous())
         out["norm2"].append(l["norm2"].to(dev, torch.float32).contiguous())
         if consume:
@@ -309,10 +327,14 @@ class Polestar:
         _check(load().polestar_force(self.ctx, FORCE_SELECT, layer, idx.ctypes.data_as(C.POINTER(C.c_int32)),
                                      idx.shape[1]))
 
-    def force_commit(self, positions) -> None:
+    def force_commit(self, positions, tokens=None) -> None:
         pos = np.ascontiguousarray(np.asarray(positions, np.int32).reshape(self.p.batch, -1))
         _check(load().polestar_force(self.ctx, FORCE_COMMIT, 0, pos.ctypes.data_as(C.POINTER(C.c_int32)),
                                      pos.shape[1]))
+        if tokens is not None:
+            tok = np.ascontiguousarray(np.asarray(tokens, np.int32).reshape(self.p.batch, -1))
+            _check(load().polestar_force(self.ctx, FORCE_TOKENS, 0, tok.ctypes.data_as(C.POINTER(C.c_int32)),
+                                         tok.shape[1]))
 
     def force_clear(self) -> None:
         _check(load().polestar_force(self.ctx, FORCE_CLEAR, 0, None, 0))

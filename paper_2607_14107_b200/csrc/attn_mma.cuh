@@ -52,6 +52,8 @@ struct AttnMmaArgs {
 };
 
 __global__ void __launch_bounds__(AT_WARPS * 32) attention_mma_kernel(AttnMmaArgs g) {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ uint8_t at_smem_raw[];
     __shared__ float red_m[AT_WARPS][AT_BM], red_l[AT_WARPS][AT_BM], red_kl[AT_WARPS][AT_BM];
     __shared__ float lse_sh[AT_BM];
@@ -300,21 +302,330 @@ __global__ void __launch_bounds__(AT_WARPS * 32) attention_mma_kernel(AttnMmaArg
     }
 }
 
-static int launch_attention_mma(const AttnArgs& a, cudaStream_t st) {
+// ------------------------------------------------------------------------------------------
+// Single-pass variant for N <= NW * TPW * 32 keys: every warp keeps the scores of its (at most
+// TPW) key tiles in registers, so K is read once.  Loads of a warp form one sequence
+// K_0 .. K_{n-1}, V_0 .. V_{n-1} through a private two-slot ring; the V tiles stream in while
+// the warps exchange their row maxima / sums.  Stored rows are read before they are rewritten,
+// a tile at a time, with all loads of the tile issued together.
+// ------------------------------------------------------------------------------------------
+constexpr int SP_SLOT_BYTES = AT_BN * AT_DH * 2;     // one K or V tile: 8 KB
+
+template <int NW, int TPW>
+__global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
+    pdl_trigger();
+    pdl_wait();
+    extern __shared__ uint8_t at_smem_raw[];
+    __shared__ float red_m[NW][AT_BM], red_l[NW][AT_BM], red_kl[NW][AT_BM];
+    __shared__ float lse_sh[AT_BM];
+    __shared__ float* prev_sh[AT_BM];
+    __shared__ int valid_sh[AT_BM];
+    const AttnArgs& a = g.a;
+    uint8_t* smem = (uint8_t*)(((uintptr_t)at_smem_raw + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int seq = blockIdx.x / g.tiles_per_seq, tile = blockIdx.x - seq * g.tiles_per_seq;
+    const int h = blockIdx.y;
+    const int g_kv = (h * a.n_kv) / a.n_heads;
+    const int dq = a.n_heads * AT_DH, dkv = a.n_kv * AT_DH;
+    const int row0 = seq * g.rows_per_seq + tile * AT_BM;
+    const int n_in_tile = min(AT_BM, g.rows_per_seq - tile * AT_BM);
+
+    uint8_t* q_s = smem + NW * 2 * SP_SLOT_BYTES;
+    const uint32_t q_u32 = (uint32_t)__cvta_generic_to_shared(q_s);
+    const uint32_t ring = (uint32_t)__cvta_generic_to_shared(smem + warp * 2 * SP_SLOT_BYTES);
+
+    const int kv_seq = a.rows ? seq : 0;
+    const __nv_bfloat16* Kg = (const __nv_bfloat16*)a.kc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
+    const __nv_bfloat16* Vg = (const __nv_bfloat16*)a.vc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
+    const int n_tiles = (a.N + AT_BN - 1) / AT_BN;
+    const int my_tiles = warp < n_tiles ? min(TPW, (n_tiles - warp + NW - 1) / NW) : 0;
+    const int n_loads = a.out ? 2 * my_tiles : my_tiles;
+
+    auto issue = [&](int j) {      // load j of this warp's sequence into slot j & 1
+        const bool is_v = j >= my_tiles;
+        const int t = warp + (is_v ? j - my_tiles : j) * NW;
+        const __nv_bfloat16* src = is_v ? Vg : Kg;
+        const uint32_t dst = ring + (j & 1) * SP_SLOT_BYTES;
+        const int key0 = t * AT_BN;
+#pragma unroll 4
+        for (int c = lane; c < AT_BN * 16; c += 32) {
+            const int r = c >> 4, ch = c & 15;
+            const int key = key0 + r;
+            const bool ok = key < a.N;
+            cp_async16(dst + sw_off(r, ch), src + (size_t)(ok ? key : 0) * dkv + ch * 8, ok);
+        }
+        cp_async_commit();
+    };
+    if (n_loads > 0) issue(0);
+    if (n_loads > 1) issue(1);
+
+    // ---- row bookkeeping + Q tile (overlaps the first K loads) -------------------------------
+    if (threadIdx.x < AT_BM) {
+        const int i = threadIdx.x;
+        float* prev = nullptr;
+        int valid = 0;
+        if (i < n_in_tile) {
+            const int r = row0 + i;
+            if (a.rows) {
+                const Row rw = a.rows[r];
+                if (rw.pos >= 0) {
+                    valid = 1;
+                    if (rw.widx >= 0 && a.pprev) prev = a.pprev + (((size_t)rw.seq * a.W_max + rw.widx) * a.n_heads + h) * a.N;
+                    else if (rw.aidx >= 0 && a.aprev) prev = a.aprev + (((size_t)rw.seq * a.B + rw.aidx) * a.n_heads + h) * a.N;
+                }
+            } else {
+                valid = 1;
+                if (a.pprev) prev = a.pprev + ((size_t)r * a.n_heads + h) * a.N;
+            }
+        }
+        prev_sh[i] = prev;
+        valid_sh[i] = valid;
+    }
+    __syncthreads();
+    for (int t = threadIdx.x; t < AT_BM * 16; t += blockDim.x) {
+        const int i = t >> 4, ch = t & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (valid_sh[i]) v = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)a.q + (size_t)(row0 + i) * dq + h * AT_DH + ch * 8);
+        *reinterpret_cast<uint4*>(q_s + sw_off(i, ch)) = v;
+    }
+    __syncthreads();
+    uint32_t qf[8][4];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = lane >> 3, r = lane & 7;
+        ldsm_x4(q_u32 + sw_off((i & 1) * 8 + r, 2 * k + (i >> 1)), qf[k][0], qf[k][1], qf[k][2], qf[k][3]);
+    }
+
+    const int r_lo = lane >> 2, r_hi = r_lo + 8;
+    const int cpair = (lane & 3) * 2;
+
+    // ---- scores of my tiles, kept in registers ---------------------------------------------------
+    float s[TPW][4][4];
+    float m_lo = -INFINITY, m_hi = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < TPW; ++i) {
+        if (i < my_tiles) {
+            if (i + 1 < n_loads) cp_async_wait<1>(); else cp_async_wait<0>();
+            __syncwarp();
+            const uint32_t kb = ring + (i & 1) * SP_SLOT_BYTES;
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) { s[i][nt][0] = s[i][nt][1] = s[i][nt][2] = s[i][nt][3] = 0.f; }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+#pragma unroll
+                for (int np = 0; np < 2; ++np) {
+                    const int ii = lane >> 3, r = lane & 7;
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4(kb + sw_off((2 * np + (ii >> 1)) * 8 + r, 2 * k + (ii & 1)), b0, b1, b2, b3);
+                    mma_bf16(s[i][2 * np], qf[k], b0, b1);
+                    mma_bf16(s[i][2 * np + 1], qf[k], b2, b3);
+                }
+            }
+            __syncwarp();
+            if (i + 2 < n_loads) issue(i + 2);
+            const int t = warp + i * NW;
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool ok = t * AT_BN + nt * 8 + cpair + e < a.N;
+                    s[i][nt][e] = ok ? s[i][nt][e] * a.scale : -INFINITY;
+                    s[i][nt][2 + e] = ok ? s[i][nt][2 + e] * a.scale : -INFINITY;
+                    m_lo = fmaxf(m_lo, s[i][nt][e]);
+                    m_hi = fmaxf(m_hi, s[i][nt][2 + e]);
+                }
+            }
+        }
+    }
+    m_lo = fmaxf(m_lo, __shfl_xor_sync(0xffffffffu, m_lo, 1));
+    m_lo = fmaxf(m_lo, __shfl_xor_sync(0xffffffffu, m_lo, 2));
+    m_hi = fmaxf(m_hi, __shfl_xor_sync(0xffffffffu, m_hi, 1));
+    m_hi = fmaxf(m_hi, __shfl_xor_sync(0xffffffffu, m_hi, 2));
+    float l_lo = 0.f, l_hi = 0.f;
+#pragma unroll
+    for (int i = 0; i < TPW; ++i) {
+        if (i < my_tiles) {
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) { l_lo += expf(s[i][nt][e] - m_lo); l_hi += expf(s[i][nt][2 + e] - m_hi); }
+        }
+    }
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    if ((lane & 3) == 0) {
+        red_m[warp][r_lo] = m_lo; red_l[warp][r_lo] = my_tiles ? l_lo : 0.f;
+        red_m[warp][r_hi] = m_hi; red_l[warp][r_hi] = my_tiles ? l_hi : 0.f;
+    }
+    __syncthreads();
+    if (threadIdx.x < AT_BM) {
+        const int i = threadIdx.x;
+        float mx = -INFINITY;
+        for (int w = 0; w < NW; ++w) mx = fmaxf(mx, red_m[w][i]);
+        float sum = 0.f;
+        for (int w = 0; w < NW; ++w)
+            if (red_l[w][i] > 0.f) sum += red_l[w][i] * expf(red_m[w][i] - mx);
+        lse_sh[i] = mx + logf(sum);
+    }
+    __syncthreads();
+    const float lse_lo = lse_sh[r_lo], lse_hi = lse_sh[r_hi];
+    float* prev_lo = prev_sh[r_lo];
+    float* prev_hi = prev_sh[r_hi];
+    const bool vec = (a.N & 1) == 0;
+
+    // ---- logp, KL, stored rows, P V ----------------------------------------------------------------
+    float o[16][4];
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+    float kl_lo = 0.f, kl_hi = 0.f;
+#pragma unroll
+    for (int i = 0; i < TPW; ++i) {
+        if (i < my_tiles) {
+            const int t = warp + i * NW;
+            // stored rows of this tile: all loads first
+            float pv_lo[4][2], pv_hi[4][2];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int key = t * AT_BN + nt * 8 + cpair;
+                pv_lo[nt][0] = pv_lo[nt][1] = pv_hi[nt][0] = pv_hi[nt][1] = 0.f;
+                if (a.record_kl) {
+                    if (vec) {
+                        if (prev_lo && key < a.N) { const float2 v = *reinterpret_cast<const float2*>(prev_lo + key); pv_lo[nt][0] = v.x; pv_lo[nt][1] = v.y; }
+                        if (prev_hi && key < a.N) { const float2 v = *reinterpret_cast<const float2*>(prev_hi + key); pv_hi[nt][0] = v.x; pv_hi[nt][1] = v.y; }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            if (prev_lo && key + e < a.N) pv_lo[nt][e] = prev_lo[key + e];
+                            if (prev_hi && key + e < a.N) pv_hi[nt][e] = prev_hi[key + e];
+                        }
+                    }
+                }
+            }
+            uint32_t pf[2][4];
+            float lp_lo[4][2], lp_hi[4][2];
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                float p[4];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool ok = t * AT_BN + nt * 8 + cpair + e < a.N;
+                    lp_lo[nt][e] = s[i][nt][e] - lse_lo; lp_hi[nt][e] = s[i][nt][2 + e] - lse_hi;
+                    const float p_lo = ok ? expf(lp_lo[nt][e]) : 0.f, p_hi = ok ? expf(lp_hi[nt][e]) : 0.f;
+                    if (ok && a.record_kl) {
+                        if (prev_lo) kl_lo += p_lo * (lp_lo[nt][e] - pv_lo[nt][e]);
+                        if (prev_hi) kl_hi += p_hi * (lp_hi[nt][e] - pv_hi[nt][e]);
+                    }
+                    p[e] = p_lo; p[2 + e] = p_hi;
+                }
+                pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
+                pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+            }
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int key = t * AT_BN + nt * 8 + cpair;
+                if (vec) {
+                    if (prev_lo && key < a.N) *reinterpret_cast<float2*>(prev_lo + key) = make_float2(lp_lo[nt][0], lp_lo[nt][1]);
+                    if (prev_hi && key < a.N) *reinterpret_cast<float2*>(prev_hi + key) = make_float2(lp_hi[nt][0], lp_hi[nt][1]);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        if (prev_lo && key + e < a.N) prev_lo[key + e] = lp_lo[nt][e];
+                        if (prev_hi && key + e < a.N) prev_hi[key + e] = lp_hi[nt][e];
+                    }
+                }
+            }
+            if (a.out) {
+                const int j = my_tiles + i;
+                if (j + 1 < n_loads) cp_async_wait<1>(); else cp_async_wait<0>();
+                __syncwarp();
+                const uint32_t vb = ring + (j & 1) * SP_SLOT_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < 2; ++ks) {
+#pragma unroll
+                    for (int dp = 0; dp < 8; ++dp) {
+                        const int ii = lane >> 3, r = lane & 7;
+                        uint32_t b0, b1, b2, b3;
+                        ldsm_x4_t(vb + sw_off(ks * 16 + (ii & 1) * 8 + r, 2 * dp + (ii >> 1)), b0, b1, b2, b3);
+                        mma_bf16(o[2 * dp], pf[ks], b0, b1);
+                        mma_bf16(o[2 * dp + 1], pf[ks], b2, b3);
+                    }
+                }
+                __syncwarp();
+                if (j + 2 < n_loads) issue(j + 2);
+            }
+        }
+    }
+    // ---- combine the warps' partial results (fixed order) ---------------------------------------
+    kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 1); kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 2);
+    kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 1); kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 2);
+    if ((lane & 3) == 0) { red_kl[warp][r_lo] = kl_lo; red_kl[warp][r_hi] = kl_hi; }
+    __syncthreads();       // every warp is done with its ring: reuse it for the O partials
+    float* o_s = reinterpret_cast<float*>(smem);     // [NW][16][128] fp32 = NW * 8 KB <= ring size
+    if (a.out) {
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            const int col = nt * 8 + cpair;
+            *reinterpret_cast<float2*>(o_s + ((size_t)warp * AT_BM + r_lo) * AT_DH + col) = make_float2(o[nt][0], o[nt][1]);
+            *reinterpret_cast<float2*>(o_s + ((size_t)warp * AT_BM + r_hi) * AT_DH + col) = make_float2(o[nt][2], o[nt][3]);
+        }
+    }
+    __syncthreads();
+    if (a.out) {
+        for (int t = threadIdx.x; t < AT_BM * AT_DH / 2; t += blockDim.x) {
+            const int i = t / (AT_DH / 2), c = (t % (AT_DH / 2)) * 2;
+            if (!valid_sh[i]) continue;
+            float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+            for (int w = 0; w < NW; ++w) {
+                const float2 v = *reinterpret_cast<const float2*>(o_s + ((size_t)w * AT_BM + i) * AT_DH + c);
+                v0 += v.x; v1 += v.y;
+            }
+            *reinterpret_cast<__nv_bfloat162*>((__nv_bfloat16*)a.out + (size_t)(row0 + i) * dq + h * AT_DH + c) =
+                __floats2bfloat162_rn(v0, v1);
+        }
+    }
+    if (a.kl && threadIdx.x < AT_BM && valid_sh[threadIdx.x]) {
+        const int i = threadIdx.x;
+        float kl = 0.f;
+        for (int w = 0; w < NW; ++w) kl += red_kl[w][i];
+        a.kl[(size_t)(row0 + i) * a.n_heads + h] = (prev_sh[i] && a.record_kl) ? kl : 0.f;
+    }
+}
+
+template <int NW, int TPW>
+static int launch_attention_sp(const AttnMmaArgs& g, dim3 grid, cudaStream_t st) {
+    constexpr int smem = NW * 2 * SP_SLOT_BYTES + AT_BM * AT_DH * 2 + 1024;
+    static bool attr = false;
+    if (!attr) {
+        if (cudaFuncSetAttribute(attention_sp_kernel<NW, TPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+            return -4;
+        attr = true;
+    }
+    return launch_k(attention_sp_kernel<NW, TPW>, grid, dim3(NW * 32), smem, st, g) == cudaSuccess ? 0 : -4;
+}
+
+static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count = 148) {
     AttnMmaArgs g;
     g.a = a;
     const int batch = a.batch > 0 ? a.batch : 1;
     g.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : a.n_rows;
     g.tiles_per_seq = (g.rows_per_seq + AT_BM - 1) / AT_BM;
+    dim3 grid(g.tiles_per_seq * batch, a.n_heads);
+    const long long ctas = (long long)grid.x * grid.y;
+    const char* force = getenv("POLESTAR_ATTN_KERNEL");
+    const int mode = force ? atoi(force) : 0;      // 0 auto, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>
+    if (mode != 1) {
+        if ((mode == 2 || (mode == 0 && ctas <= 2LL * sm_count)) && a.N <= 8 * 2 * AT_BN) return launch_attention_sp<8, 2>(g, grid, st);
+        if ((mode == 3 || mode == 0) && a.N <= 4 * 4 * AT_BN) return launch_attention_sp<4, 4>(g, grid, st);
+        if ((mode == 4 || mode == 0) && a.N <= 8 * 4 * AT_BN) return launch_attention_sp<8, 4>(g, grid, st);
+    }
     static bool attr = false;
     if (!attr) {
         if (cudaFuncSetAttribute(attention_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM) != cudaSuccess)
             return -4;
         attr = true;
     }
-    dim3 grid(g.tiles_per_seq * batch, a.n_heads);
-    attention_mma_kernel<<<grid, AT_WARPS * 32, AT_SMEM, st>>>(g);
-    return cudaGetLastError() == cudaSuccess ? 0 : -4;
+    return launch_k(attention_mma_kernel, grid, dim3(AT_WARPS * 32), AT_SMEM, st, g) == cudaSuccess ? 0 : -4;
 }
 
 }  // namespace ps

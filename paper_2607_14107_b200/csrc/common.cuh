@@ -14,8 +14,24 @@ template <typename T> __device__ __forceinline__ T from_f(float v);
 template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// two adjacent elements (even index) in one store
+template <typename T> __device__ __forceinline__ void store_pair(T* p, float a, float b);
+template <> __device__ __forceinline__ void store_pair<float>(float* p, float a, float b) {
+    *reinterpret_cast<float2*>(p) = make_float2(a, b);
+}
+template <> __device__ __forceinline__ void store_pair<__nv_bfloat16>(__nv_bfloat16* p, float a, float b) {
+    *reinterpret_cast<__nv_bfloat162*>(p) = __floats2bfloat162_rn(a, b);
+}
+
 // value a GEMM operand of type T actually carries (identity for float)
 template <typename T> __device__ __forceinline__ float round_to(float v) { return to_f<T>(from_f<T>(v)); }
+
+// ---- programmatic dependent launch -------------------------------------------------------
+// Kernels of a forward are launched back to back with programmatic stream serialization: a
+// kernel may start while its predecessor drains, and calls pdl_wait() before it touches anything
+// the predecessor produced (the instructions are no-ops for ordinary launches).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---- rows of one forward -----------------------------------------------------------
 // One descriptor per forwarded row.  pos < 0 marks an unused slot.
@@ -154,57 +170,67 @@ __device__ __forceinline__ void epilogue_pair(const EpiArgs& e, int m, int n, fl
     if (EPI == EPI_QKV || EPI == EPI_QKV_REFRESH) {
         int seq, pos, kvf, qrow;
         if (EPI == EPI_QKV) {
-            const Row rw = e.rows[m];
-            if (rw.pos < 0) return;
-            seq = rw.seq; pos = rw.pos; kvf = e.kvflag[m]; qrow = m;
+            const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + m);   // {seq, pos, widx, aidx}
+            if (rw.y < 0) return;
+            seq = rw.x; pos = rw.y; kvf = __ldg(e.kvflag + m); qrow = m;
         } else {
             seq = m / e.max_rows;
             const int i = m - seq * e.max_rows;
-            if (i >= e.counts[seq]) return;
-            pos = e.idx[seq * e.max_rows + i]; kvf = 1; qrow = m;
+            if (i >= __ldg(e.counts + seq)) return;
+            pos = __ldg(e.idx + seq * e.max_rows + i); kvf = 1; qrow = m;
         }
         const int dq = e.n_heads * e.head_dim, dkv = e.n_kv * e.head_dim;
         const int Npos = (EPI == EPI_QKV) ? e.N_seq : e.P;
         if (n < dq + dkv) {
             const int p = n % e.head_dim;
-            const float2 cs = e.rope[(size_t)pos * (e.head_dim / 2) + (p >> 1)];
+            const float2 cs = __ldg(e.rope + (size_t)pos * (e.head_dim / 2) + (p >> 1));
             const float r0 = v0 * cs.x - v1 * cs.y;
             const float r1 = v1 * cs.x + v0 * cs.y;
             if (n < dq) {
                 if (e.q_out) {
-                    T* q = (T*)e.q_out + (size_t)qrow * dq + n;
-                    q[0] = from_f<T>(r0); q[1] = from_f<T>(r1);
+                    store_pair<T>((T*)e.q_out + (size_t)qrow * dq + n, r0, r1);
                 }
             } else if (kvf) {
-                T* k = (T*)e.kc + ((size_t)seq * Npos + pos) * dkv + (n - dq);
-                k[0] = from_f<T>(r0); k[1] = from_f<T>(r1);
+                store_pair<T>((T*)e.kc + ((size_t)seq * Npos + pos) * dkv + (n - dq), r0, r1);
             }
         } else if (kvf) {
-            T* v = (T*)e.vc + ((size_t)seq * Npos + pos) * dkv + (n - dq - dkv);
-            v[0] = from_f<T>(v0); v[1] = from_f<T>(v1);
+            store_pair<T>((T*)e.vc + ((size_t)seq * Npos + pos) * dkv + (n - dq - dkv), v0, v1);
         }
     } else if (EPI == EPI_RESID) {
         const size_t o = (size_t)m * e.ld_out + n;
-        e.out_f32[o] = e.resid[o] + v0;
-        e.out_f32[o + 1] = e.resid[o + 1] + v1;
+        const float2 r = __ldg(reinterpret_cast<const float2*>(e.resid + o));
+        *reinterpret_cast<float2*>(e.out_f32 + o) = make_float2(r.x + v0, r.y + v1);
     } else if (EPI == EPI_SWIGLU) {
         const float g = v0 / (1.f + expf(-v0)) * v1;
         ((T*)e.out_t)[(size_t)m * e.ld_out + (n >> 1)] = from_f<T>(g);
     } else if (EPI == EPI_DOWN) {
-        const int r = e.list ? e.list[m] : m;
-        const Row rw = e.rows[r];
-        if (rw.pos < 0) return;
+        const int r = e.list ? __ldg(e.list + m) : m;
+        const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + r);       // {seq, pos, widx, aidx}
+        if (rw.y < 0) return;
         const size_t o = (size_t)r * e.ld_out + n;
-        const float a0 = e.resid[o] + v0, a1 = e.resid[o + 1] + v1;
-        float* dst = (e.within && rw.widx >= 0)
-                         ? e.packet + ((size_t)rw.seq * e.W_max + rw.widx) * e.ld_out + n
+        const float2 rs = __ldg(reinterpret_cast<const float2*>(e.resid + o));
+        float* dst = (e.within && rw.z >= 0)
+                         ? e.packet + ((size_t)rw.x * e.W_max + rw.z) * e.ld_out + n
                          : e.out_f32 + o;
-        dst[0] = a0; dst[1] = a1;
+        *reinterpret_cast<float2*>(dst) = make_float2(rs.x + v0, rs.y + v1);
     } else if (EPI == EPI_LOGITS) {
         const size_t o = (size_t)m * e.ld_out + n;
-        e.out_f32[o] = v0 * e.scale;
-        e.out_f32[o + 1] = v1 * e.scale;
+        *reinterpret_cast<float2*>(e.out_f32 + o) = make_float2(v0 * e.scale, v1 * e.scale);
     }
+}
+
+// ---- host: launch with programmatic stream serialization -----------------------------------
+inline bool g_use_pdl = true;
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = g_use_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
 }
 
 }  // namespace ps

@@ -1,22 +1,32 @@
-// Skinny-M bf16 GEMM on 5th-generation tensor cores (tcgen05 + TMEM, operands staged by TMA).
+// Weight-streaming bf16 GEMM on 5th-generation tensor cores (tcgen05 + TMEM, operands staged by TMA).
 //
 //   out[m][n] = sum_k A[m][k] * W[n][k]      A: activations [M, K], W: weights [N_out, K]
 //
-// The decoding step multiplies a few dozen to a few hundred rows by every weight matrix, so
-// the kernel is bound by streaming W from HBM.  The operands are therefore swapped: the
-// weight tile (128 output features x 64 k) is the 128-row "A" operand of the MMA and the
-// activation tile (NT tokens x 64 k, NT = 16..256) is the "B" operand.  The accumulator in
-// tensor memory holds D^T: lane = output feature, column = token.  A small activation tile
-// keeps shared memory for a deep pipeline of weight tiles, and no MMA rows are wasted on
-// padding when only 32 rows are live.
+// The decoding step multiplies a few dozen to a few hundred rows by every weight matrix, so the
+// kernel is bound by streaming W from HBM.  Design points, each taken from a measurement:
 //
-// grid = (N_out / 128, ceil(M / NT), splits).  With splits > 1 every CTA writes its fp32
-// partial tile to a workspace and the last CTA to arrive (per output tile) adds the partials in
-// split order and runs the epilogue, which keeps results deterministic.
+//  * W is stored TILE-MAJOR: the 256 x 64 block (feature tile f, k block kb) is one contiguous
+//    32 KB chunk at chunk index f * (K / 64) + kb, so a weight TMA is one sequential burst.
+//  * One MMA instruction takes a few hundred cycles however small its N is, so the instruction
+//    shape is made as large as it gets: M = 128 tokens x N = 256 features x K = 16.  With the
+//    features on the small side of the instruction the tensor pipe, not HBM, was the limit
+//    (~4 TB/s).  Rows beyond the live tokens are out-of-bounds rows of the activation tensor
+//    map: TMA fills them with zeros without reading memory.
+//  * Stream-K: a persistent grid of one CTA per SM splits the work units -- (output tile,
+//    k block) pairs, ordered so that the token tiles of one feature tile are adjacent (their
+//    weights are then L2 hits) -- into equal contiguous ranges.  Every SM streams the same number
+//    of bytes whatever the matrix shape and the pipeline fills once per launch.  A range is a
+//    sequence of segments (one per output tile touched).  A segment that covers its tile's
+//    whole K runs the epilogue straight from tensor memory; partial segments go to a workspace
+//    slot, and the last CTA to arrive at the tile adds the slots in ascending-k order
+//    (deterministic) and runs the epilogue.
+//  * Programmatic dependent launch: weight tiles of the first pipeline stages are requested
+//    before griddepcontrol.wait, i.e. while the previous kernel of the stream still drains;
+//    activations, residuals and every global write come after it.
 //
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (one TMEM lane quarter each).  Every mbarrier wait is bounded; on
-// time-out the CTA raises a status word, stops issuing work and leaves in an orderly way.
+// warps 2..5 = epilogue (TMEM lane quarter warp % 4 = 32 tokens each).  Every mbarrier wait is
+// bounded; on time-out the CTA raises a status word, stops issuing work and leaves in order.
 #pragma once
 #include <cuda.h>
 
@@ -25,10 +35,15 @@
 namespace ps {
 namespace tc {
 
-constexpr int BLOCK_F = 128;   // output features per CTA (UMMA M)
+constexpr int BLOCK_T = 128;   // tokens per tile (UMMA M)
+constexpr int BLOCK_F = 256;   // output features per tile (UMMA N)
 constexpr int BLOCK_K = 64;    // bf16 elements per k block = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int THREADS = 192;
+constexpr int MAX_STAGES = 8;
+constexpr uint32_t A_BYTES = BLOCK_T * BLOCK_K * 2;   // 16 KB
+constexpr uint32_t W_BYTES = BLOCK_F * BLOCK_K * 2;   // 32 KB
+constexpr uint32_t STAGE_BYTES = A_BYTES + W_BYTES;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // ~2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -38,6 +53,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -81,6 +99,7 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// 16 consecutive accumulator columns of this thread's TMEM lane
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
     uint32_t r[16];
     asm volatile(
@@ -106,53 +125,56 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     d |= (uint64_t)2 << 61;
     return d;
 }
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
-__host__ __device__ inline uint32_t instr_desc_bf16(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BLOCK_F >> 4) << 24);
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N.
+__host__ __device__ inline uint32_t instr_desc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-struct GemmArgs {
-    int M;          // rows of A that may be live (host bound)
-    int N_out, K;
-    int NT;         // tokens per tile: 16, 32, 64, 128 or 256
-    int stages;
-    int splits;
-    float* partial;     // [splits][tiles_f][tiles_t][NT][128] fp32 (splits > 1)
+struct SkArgs {
+    int M, N_out, K, stages;
+    int tiles_f, tiles_t;
+    float* partial;     // [2 * gridDim.x][BLOCK_T][BLOCK_F] fp32
     int* tile_counter;  // [tiles_f * tiles_t], zero before launch, zero again after
     int* status;        // set to 1 on a wait time-out
 };
 
+// first unit of CTA c when U units are split over G CTAs
+__device__ __forceinline__ long long sk_begin(long long U, int G, int c) { return (U * c) / G; }
+__device__ __forceinline__ int sk_owner(long long U, int G, long long u) {
+    int c = (int)((u * G) / U);
+    while (c > 0 && sk_begin(U, G, c) > u) --c;
+    while (c + 1 < G && sk_begin(U, G, c + 1) <= u) ++c;
+    return c;
+}
+
 template <typename T, int EPI>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
-               GemmArgs g, EpiArgs e) {
+gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
+               SkArgs g, EpiArgs e) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * 12 + 1];
+    __shared__ uint64_t bars[2 * MAX_STAGES + 2];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
     __shared__ int last_sh;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile_f = blockIdx.x, tile_t = blockIdx.y, split = blockIdx.z;
-    const int t0 = tile_t * g.NT;
-    const int Mv = e.m_count ? min(g.M, *e.m_count) : g.M;
-    if (t0 >= Mv) return;     // whole tile beyond the live rows (uniform over the CTA)
-
+    const int G = gridDim.x, cta = blockIdx.x;
     const int kb_total = g.K / BLOCK_K;
-    const int kb_begin = (int)(((long long)kb_total * split) / g.splits);
-    const int kb_end = (int)(((long long)kb_total * (split + 1)) / g.splits);
-    const int n_kb = kb_end - kb_begin;
+    const long long U = (long long)g.tiles_f * g.tiles_t * kb_total;
+    const long long u_begin = sk_begin(U, G, cta), u_end = sk_begin(U, G, cta + 1);
+    const int n_units = (int)(u_end - u_begin);
+    // tile index = tile_f * tiles_t + tile_t : token tiles of one feature tile are neighbours
 
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const uint32_t w_bytes = BLOCK_F * BLOCK_K * 2, a_bytes = (uint32_t)g.NT * BLOCK_K * 2;
-    const uint32_t stage_bytes = w_bytes + a_bytes;
     const uint32_t smem_base = smem_u32(smem);
-    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[12]), accum_bar = smem_u32(&bars[24]);
-    const uint32_t ncols = g.NT < 32 ? 32u : (uint32_t)g.NT;
+    const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[MAX_STAGES]);
+    const uint32_t accum_full = smem_u32(&bars[2 * MAX_STAGES]), accum_empty = smem_u32(&bars[2 * MAX_STAGES + 1]);
+    constexpr uint32_t ncols = BLOCK_F;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        mbar_init(accum_bar, 1);
+        mbar_init(accum_full, 1);
+        mbar_init(accum_empty, 4);      // one arrival per epilogue warp
         abort_sh = 0;
         last_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -162,100 +184,180 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_trigger();
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int i = 0; i < n_kb; ++i) {
+            // weights do not depend on the previous kernel: request the first stages right away
+            const int pre = min(g.stages, n_units);
+            for (int i = 0; i < pre; ++i) {
+                const long long u = u_begin + i;
+                const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
+                mbar_expect_tx(full0 + 8 * i, STAGE_BYTES);
+                tma_load_2d(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
+                            ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
+            }
+            pdl_wait();
+            for (int i = 0; i < pre; ++i) {
+                const long long u = u_begin + i;
+                const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
+                tma_load_2d(smem_base + i * STAGE_BYTES, &map_a, full0 + 8 * i, kb * BLOCK_K, (tile % g.tiles_t) * BLOCK_T);
+            }
+            for (int i = pre; i < n_units; ++i) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
-                const uint32_t dst = smem_base + s * stage_bytes;
-                mbar_expect_tx(full0 + 8 * s, stage_bytes);
-                tma_load_2d(dst, &map_w, full0 + 8 * s, (kb_begin + i) * BLOCK_K, tile_f * BLOCK_F);
-                tma_load_2d(dst + w_bytes, &map_a, full0 + 8 * s, (kb_begin + i) * BLOCK_K, t0);
+                const long long u = u_begin + i;
+                const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
+                const uint32_t dst = smem_base + s * STAGE_BYTES;
+                mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+                tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
+                tma_load_2d(dst, &map_a, full0 + 8 * s, kb * BLOCK_K, (tile % g.tiles_t) * BLOCK_T);
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(g.NT);
-            bool ok = true;
-            for (int i = 0; i < n_kb && ok; ++i) {
+            const uint32_t idesc = instr_desc_bf16(BLOCK_T, BLOCK_F);
+            int seg = 0;
+            bool seg_start = true;
+            for (int i = 0; i < n_units; ++i) {
+                const long long u = u_begin + i;
+                const int kb = (int)(u % kb_total);
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
-                ok = mbar_wait(full0 + 8 * s, ph, abort_flag);
-                if (!ok) break;
+                if (seg_start && seg > 0) {
+                    // the epilogue must have drained the accumulator of the previous segment
+                    if (!mbar_wait(accum_empty, (uint32_t)(seg - 1) & 1u, abort_flag)) break;
+                    tc_fence_after();
+                }
+                if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t wa = smem_base + s * stage_bytes;
-                const uint64_t dw = smem_desc_sw128(wa), da = smem_desc_sw128(wa + w_bytes);
+                const uint32_t sa = smem_base + s * STAGE_BYTES;
+                const uint64_t da = smem_desc_sw128(sa), dw = smem_desc_sw128(sa + A_BYTES);
 #pragma unroll
                 for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                    umma_bf16(tmem_base, dw + (uint64_t)(k * 2), da + (uint64_t)(k * 2), idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    umma_bf16(tmem_base, da + (uint64_t)(k * 2), dw + (uint64_t)(k * 2), idesc, (!seg_start || k > 0) ? 1u : 0u);
                 umma_commit(empty0 + 8 * s);
+                seg_start = false;
+                if (kb == kb_total - 1 || i == n_units - 1) {
+                    umma_commit(accum_full);
+                    ++seg;
+                    seg_start = true;
+                }
             }
-            umma_commit(accum_bar);     // arrives once every MMA issued so far has finished
         }
     } else {
-        // ---- epilogue warps: quarter q of the TMEM lanes = features 32q .. 32q+31 of the tile
+        // ---- epilogue warps: TMEM lane = token, column = feature ------------------------------------
+        pdl_wait();
         const int q = warp & 3;
-        const int f_local = q * 32 + lane;
-        const int n = tile_f * BLOCK_F + f_local;
-        const bool got = mbar_wait(accum_bar, 0, abort_flag);
-        tc_fence_after();
-        if (got) {
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
-            const int nt_live = min(g.NT, Mv - t0);
-            if (g.splits == 1) {
-                for (int c0 = 0; c0 < nt_live; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + (uint32_t)c0, v);
+        const int t_local = q * 32 + lane;
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
+        int seg = 0;
+        long long u = u_begin;
+        while (u < u_end) {
+            const int tile = (int)(u / kb_total);
+            const int k0 = (int)(u - (long long)tile * kb_total);
+            const long long tile_end = (long long)(tile + 1) * kb_total;
+            const long long seg_end = tile_end < u_end ? tile_end : u_end;
+            const int k1 = (int)(seg_end - (long long)tile * kb_total);
+            const int tile_f = tile / g.tiles_t, tile_t = tile % g.tiles_t;
+            const int m = tile_t * BLOCK_T + t_local;
+            const int n0 = tile_f * BLOCK_F;
+            const bool live = m < Mv;
+            const bool warp_live = tile_t * BLOCK_T + q * 32 < Mv;      // any live token in this warp's quarter
+            const bool whole = (k0 == 0 && k1 == kb_total);
+            if (!mbar_wait(accum_full, (uint32_t)seg & 1u, abort_flag)) break;
+            tc_fence_after();
+            if (whole) {
+                if (warp_live) {
+                    for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(taddr + (uint32_t)c0, v);
+                        if (live) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float partner = __shfl_xor_sync(0xffffffffu, v[c], 1);
-                        const int m = t0 + c0 + c;
-                        if (!(lane & 1) && m < Mv && n < g.N_out) epilogue_pair<T, EPI>(e, m, n, v[c], partner);
+                            for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, m, n0 + c0 + c, v[c], v[c + 1]);
+                        }
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(accum_empty);
             } else {
-                float* part = g.partial + ((((size_t)split * gridDim.x + tile_f) * gridDim.y + tile_t) * g.NT) * BLOCK_F;
-                for (int c0 = 0; c0 < nt_live; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(taddr + (uint32_t)c0, v);
+                const int which = (k0 == 0) ? 1 : 0;     // slot 0: my range starts inside this tile
+                float* part = g.partial + ((size_t)(2 * cta + which) * BLOCK_T + t_local) * BLOCK_F;
+                if (warp_live) {
+                    for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(taddr + (uint32_t)c0, v);
+                        if (live) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) part[(size_t)(c0 + c) * BLOCK_F + f_local] = v[c];
+                            for (int c = 0; c < 16; c += 4)
+                                *reinterpret_cast<float4*>(part + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                        }
+                    }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(accum_empty);
                 __threadfence();
-            }
-        }
-    }
-
-    if (g.splits > 1) {
-        // last CTA of this output tile sums the partials (fixed order) and runs the epilogue
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const int prev = atomicAdd(&g.tile_counter[tile_f * gridDim.y + tile_t], 1);
-            last_sh = (prev == g.splits - 1);
-        }
-        __syncthreads();
-        if (last_sh && warp >= 2 && !abort_sh) {
-            __threadfence();
-            const int q = warp & 3;
-            const int f_local = q * 32 + lane;
-            const int n = tile_f * BLOCK_F + f_local;
-            const int nt_live = min(g.NT, Mv - t0);
-            for (int c = 0; c < nt_live; ++c) {
-                float acc = 0.f;
-                for (int sp = 0; sp < g.splits; ++sp) {
-                    const float* part = g.partial + ((((size_t)sp * gridDim.x + tile_f) * gridDim.y + tile_t) * g.NT) * BLOCK_F;
-                    acc += __ldcg(part + (size_t)c * BLOCK_F + f_local);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int c_lo = sk_owner(U, G, (long long)tile * kb_total), c_hi = sk_owner(U, G, tile_end - 1);
+                if (threadIdx.x == 64) {
+                    const int prev = atomicAdd(&g.tile_counter[tile], 1);
+                    last_sh = (prev == c_hi - c_lo);
+                    if (last_sh) g.tile_counter[tile] = 0;
                 }
-                const float partner = __shfl_xor_sync(0xffffffffu, acc, 1);
-                const int m = t0 + c;
-                if (!(lane & 1) && n < g.N_out) epilogue_pair<T, EPI>(e, m, n, acc, partner);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (last_sh) {
+                    // The partial tiles sit in global memory, so the fix-up is not tied to TMEM lanes:
+                    // (token, 16-feature chunk) items are spread over all 128 epilogue threads, and the
+                    // loads of four segments are issued together before they are added in k order.
+                    __threadfence();
+                    const int nseg = c_hi - c_lo + 1;
+                    const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
+                    for (int item = (int)threadIdx.x - 64; item < n_live * (BLOCK_F / 16); item += 128) {
+                        const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16;
+                        float acc[16];
+#pragma unroll
+                        for (int x = 0; x < 16; ++x) acc[x] = 0.f;
+                        for (int sg0 = 0; sg0 < nseg; sg0 += 4) {
+                            float4 tv[4][4];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int cc = c_lo + sg0 + j;
+                                if (sg0 + j < nseg) {
+                                    // a CTA whose range starts inside the tile wrote slot 0, otherwise slot 1
+                                    const int wsl = (sk_begin(U, G, cc) > (long long)tile * kb_total) ? 0 : 1;
+                                    const float4* ps = reinterpret_cast<const float4*>(
+                                        g.partial + ((size_t)(2 * cc + wsl) * BLOCK_T + tl) * BLOCK_F + c0);
+#pragma unroll
+                                    for (int x = 0; x < 4; ++x) tv[j][x] = __ldcg(ps + x);
+                                } else {
+#pragma unroll
+                                    for (int x = 0; x < 4; ++x) tv[j][x] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                }
+                            }
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                                for (int x = 0; x < 4; ++x) {
+                                    acc[4 * x] += tv[j][x].x; acc[4 * x + 1] += tv[j][x].y;
+                                    acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
+                                }
+                        }
+                        const int mm = tile_t * BLOCK_T + tl;
+#pragma unroll
+                        for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, mm, n0 + c0 + c, acc[c], acc[c + 1]);
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");     // last_sh is reused by the next segment
             }
+            ++seg;
+            u = seg_end;
         }
-        if (last_sh && threadIdx.x == 0) g.tile_counter[tile_f * gridDim.y + tile_t] = 0;
     }
 
     tc_fence_before();

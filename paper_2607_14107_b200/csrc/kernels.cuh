@@ -10,6 +10,8 @@ namespace ps {
 // Row table of one forward (Algorithm 1: E_b at block entry, J_b plus Omega_b within a block)
 // ---------------------------------------------------------------------------------------
 __global__ void build_rows_kernel(StepDesc sd, Row* rows) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int total = sd.batch * sd.rows_per_seq;
     if (i >= total) return;
@@ -42,6 +44,8 @@ template <typename T>
 __global__ void embed_rows_kernel(StepDesc sd, const Row* rows, const int* y, const T* emb, int d,
                                   float* x, float* packet, unsigned char* patch0, int* tok_at_h0,
                                   int* stats) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x;
     const Row rw = rows[r];
     if (rw.pos < 0) return;
@@ -76,6 +80,8 @@ template <typename T>
 __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* hc, const float* packet,
                                 const unsigned char* patch, const float* gain, float eps, int d,
                                 T* a_out, unsigned char* kvflag) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[33];
     const int r = blockIdx.x;
     const Row rw = rows[r];
@@ -118,6 +124,8 @@ __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* h
 template <typename T>
 __global__ void prep_rows_kernel(const float* x, const int* list, const int* m_count, const float* gain,
                                  float eps, int d, T* a_out) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[33];
     const int i = blockIdx.x;
     T* a = a_out + (size_t)i * d;
@@ -139,6 +147,8 @@ struct HeadSrc { int kind; int index; };  // kind 0: x row `index`; 1: packet ro
 template <typename T>
 __global__ void prep_head_kernel(const float* x, const float* packet, const HeadSrc* src_list,
                                  const int* m_count, const float* gain, float eps, int d, T* a_out) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[33];
     const int i = blockIdx.x;
     T* a = a_out + (size_t)i * d;
@@ -159,6 +169,8 @@ __global__ void prep_head_kernel(const float* x, const float* packet, const Head
 template <typename T>
 __global__ void prep_refresh_kernel(const T* h, const int* idx, const int* counts, int max_rows, int P,
                                     const float* gain, float eps, int d, T* a_out) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[33];
     const int m = blockIdx.x;
     const int s = m / max_rows, i = m - s * max_rows;
@@ -181,7 +193,9 @@ __global__ void prep_refresh_kernel(const T* h, const int* idx, const int* count
 // ---------------------------------------------------------------------------------------
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ Wt,
-                                                        int M, int Nout, int K, EpiArgs e) {
+                                                        int M, int Nout, int K, int w_tiled, EpiArgs e) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float As[16][64 + 4];
     __shared__ float Ws[16][64 + 4];
     const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
@@ -198,7 +212,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A,
             const int rr = t >> 4, kk = t & 15;
             const int m = m0 + rr, n = n0 + rr, k = k0 + kk;
             As[kk][rr] = (m < M && k < K) ? to_f<T>(A[(size_t)m * K + k]) : 0.f;
-            Ws[kk][rr] = (n < Nout && k < K) ? to_f<T>(Wt[(size_t)n * K + k]) : 0.f;
+            // tile-major weights: block (n / 256, k / 64) is a contiguous [256][64] chunk
+            const size_t wi = w_tiled ? ((size_t)((n >> 8) * (K >> 6) + (k >> 6)) << 14) + ((n & 255) << 6) + (k & 63)
+                                      : (size_t)n * K + k;
+            Ws[kk][rr] = (n < Nout && k < K) ? to_f<T>(Wt[wi]) : 0.f;
         }
         __syncthreads();
 #pragma unroll
@@ -247,6 +264,8 @@ struct AttnArgs {
 
 template <typename T>
 __global__ void attention_simt_kernel(AttnArgs a) {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ float sm[];
     const int wpb = blockDim.x >> 5, wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * wpb + wid, h = blockIdx.y;
@@ -313,6 +332,8 @@ __global__ void attention_simt_kernel(AttnArgs a) {
 // ---------------------------------------------------------------------------------------
 template <typename T>
 __global__ void hidden_delta_kernel(const T* __restrict__ a, const T* __restrict__ b, float* out, int rows, int d) {
+    pdl_trigger();
+    pdl_wait();
     const int wpb = blockDim.x >> 5, wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per = 16 / (int)sizeof(T);
     for (int r = blockIdx.x * wpb + wid; r < rows; r += gridDim.x * wpb) {
@@ -446,6 +467,8 @@ __device__ int select_one(const float* D, int W, int mode, int k, float thresh, 
 
 __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* drift, int W, int mode, int k,
                                                              float thresh, float floor_, int* idx, int* count) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ SelSmem s;
     const int b = blockIdx.x;
     const int c = select_one(drift + (size_t)b * W, W, mode, k, thresh, floor_, idx + (size_t)b * W, nullptr, s);
@@ -467,6 +490,8 @@ struct StepSelArgs {
 };
 
 __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, StepSelArgs a) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ SelSmem s;
     __shared__ float dsh[SEL_MAX_W > 1024 ? 1024 : SEL_MAX_W];
     __shared__ int base;
@@ -519,6 +544,8 @@ __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, S
 __global__ void build_head_list_kernel(StepDesc sd, const int* y, int mask_id, const int* sel_idx,
                                        const int* sel_cnt, int use_suffix, int act_row0_stride,
                                        HeadSrc* list, int* count, int* suf_seq, int* suf_w) {
+    pdl_trigger();
+    pdl_wait();
     // act_row0_stride: forward row of active j in sequence s = s*rows_per_seq + (act offset) + j
     const int t = threadIdx.x;
     const int nb = sd.batch * sd.B;
@@ -557,6 +584,8 @@ struct ConfPart { float mx_all; float sum; float mx_ex; int arg_ex; };
 
 __global__ void conf_partial_kernel(const float* logits, const int* m_count, int rows, int V, int mask_id,
                                     int chunks, ConfPart* part) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[33];
     __shared__ float bv[32];
     __shared__ int bi[32];
@@ -596,6 +625,8 @@ __global__ void conf_partial_kernel(const float* logits, const int* m_count, int
 
 __global__ void conf_final_kernel(const ConfPart* part, const int* m_count, int rows, int chunks,
                                   int* yhat, float* conf) {
+    pdl_trigger();
+    pdl_wait();
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= rows || (m_count && r >= *m_count)) return;
     const ConfPart* p = part + (size_t)r * chunks;
@@ -626,12 +657,15 @@ struct CommitArgs {
     int* suffix_flags;           // [batch][W_max]
     const int* head_count; const int* suf_seq; const int* suf_w;
     const int* forced_pos; int forced_n;      // [batch][forced_n] absolute positions, -1 unused (null: free-running)
+    const int* forced_tok;                    // optional tokens written at the forced positions (null: own prediction)
     int* seq_info;               // [batch][8]: committed, by_conf, by_drift, by_quota, suffix, eos, masked_left, nonfinite
     int n_heads, hist, mask_id, eos_id, act_row_off, steps_used, steps_per_block, use_drift, use_suffix, ge;
     float tau_s, alpha, tau_suffix;
 };
 
 __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float s_conf[256];
     __shared__ unsigned char s_masked[256], s_flag[256];
     __shared__ int cnt[8];
@@ -684,7 +718,10 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
             flag = 0;
             const int pos = sd.act_start + j;
             for (int u = 0; u < a.forced_n; ++u)
-                if (a.forced_pos[s * a.forced_n + u] == pos) flag = s_flag[j] ? s_flag[j] : (1 | 8);
+                if (a.forced_pos[s * a.forced_n + u] == pos) {
+                    flag = s_flag[j] ? s_flag[j] : (1 | 8);
+                    if (a.forced_tok) yh = a.forced_tok[s * a.forced_n + u];
+                }
             if (!masked) flag = 0;
         }
     } else {
@@ -724,13 +761,14 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
             const int pos = window_pos(sd, w);
             const float sc = a.conf[sd.batch * B + i];
             bool ok = a.ge ? (sc >= a.tau_suffix) : (sc > a.tau_suffix);
+            int t2 = a.yhat[sd.batch * B + i];
             if (a.forced_pos) {
                 ok = false;
-                for (int u = 0; u < a.forced_n; ++u) if (a.forced_pos[s * a.forced_n + u] == pos) ok = true;
+                for (int u = 0; u < a.forced_n; ++u)
+                    if (a.forced_pos[s * a.forced_n + u] == pos) { ok = true; if (a.forced_tok) t2 = a.forced_tok[s * a.forced_n + u]; }
             }
             int f = 1;
             if (ok && a.y[s * sd.N + pos] == a.mask_id) {
-                const int t2 = a.yhat[sd.batch * B + i];
                 a.y[s * sd.N + pos] = t2;
                 f |= 2;
                 atomicAdd(&cnt[0], 1); atomicAdd(&cnt[4], 1);
@@ -750,6 +788,8 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
 
 // Last-layer drift of the active rows (Algorithm 1, delta): mean over heads of the per-head KL.
 __global__ void delta_kernel(StepDesc sd, const float* kl, int act_row_off, int n_heads, float* delta) {
+    pdl_trigger();
+    pdl_wait();
     const int s = blockIdx.x, j = threadIdx.x;
     if (j >= sd.B) return;
     float dl = 0.f;
@@ -764,6 +804,8 @@ __global__ void delta_kernel(StepDesc sd, const float* kl, int act_row_off, int 
 
 // gather rows of x into a keep buffer: dst[s][j][:] = x[row(s, j)][:]
 __global__ void keep_hidden_kernel(StepDesc sd, const float* x, int act_row_off, int d, float* dst) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x;
     const int s = i / sd.B, j = i - s * sd.B;
     const float* src = x + (size_t)(s * sd.rows_per_seq + act_row_off + j) * d;
@@ -773,6 +815,8 @@ __global__ void keep_hidden_kernel(StepDesc sd, const float* x, int act_row_off,
 
 // y = [prompt ; MASK ...] from a prompt that already lives on the device (ids clamped to the vocabulary)
 __global__ void init_tokens_kernel(int* y, const int* prompt, int batch, int prompt_len, int N, int mask_id, int vocab) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= batch * N) return;
     const int s = i / N, pos = i - s * N;
@@ -787,6 +831,8 @@ __global__ void init_tokens_kernel(int* y, const int* prompt, int batch, int pro
 
 // rotary table: tab[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), computed in double precision
 __global__ void rope_table_kernel(float2* tab, int N, int half, double theta) {
+    pdl_trigger();
+    pdl_wait();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N * half) return;
     const int pos = i / half, k = i - pos * half;

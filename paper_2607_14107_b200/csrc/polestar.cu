@@ -30,6 +30,13 @@ using namespace ps;
 static thread_local cudaError_t last_cuda_error = cudaSuccess;
 static int g_sm_count = 0;
 
+static int env_int(const char* name, int dflt) {
+    const char* s = getenv(name);
+    return s ? atoi(s) : dflt;
+}
+
+
+
 // ------------------------------------------------------------------------------------------
 // tensor maps (TMA descriptors) through the driver entry point, no libcuda link dependency
 // ------------------------------------------------------------------------------------------
@@ -56,7 +63,7 @@ static bool make_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t
     cuuint32_t box[2] = {64, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, (CUtensorMapL2promotion)env_int("POLESTAR_TMA_L2PROMO", CU_TENSOR_MAP_L2_PROMOTION_L2_128B),
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -81,16 +88,15 @@ struct GemmWs {
     int* status = nullptr;
 };
 
-static int env_int(const char* name, int dflt) {
-    const char* s = getenv(name);
-    return s ? atoi(s) : dflt;
-}
+// bf16 matrices with out % 256 == 0 and in % 64 == 0 are stored tile-major (see polestar.h)
+static bool weight_is_tiled(int dtype, int n_out, int k) { return dtype == POLESTAR_BF16 && n_out % 256 == 0 && k % 64 == 0; }
 
 template <typename T, int EPI>
 static int launch_gemm_simt(const void* A, const void* W, int M, int N_out, int K, const EpiArgs& e, cudaStream_t st) {
     if (M <= 0) return POLESTAR_OK;
     dim3 grid((N_out + 63) / 64, (M + 63) / 64);
-    gemm_simt_kernel<T, EPI><<<grid, 256, 0, st>>>((const T*)A, (const T*)W, M, N_out, K, e);
+    const int w_tiled = weight_is_tiled(sizeof(T) == 2 ? POLESTAR_BF16 : POLESTAR_F32, N_out, K) ? 1 : 0;
+    gemm_simt_kernel<T, EPI><<<grid, 256, 0, st>>>((const T*)A, (const T*)W, M, N_out, K, w_tiled, e);
     CK(cudaGetLastError());
     return POLESTAR_OK;
 }
@@ -99,38 +105,31 @@ template <int EPI>
 static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a_rows_alloc, const void* W, int M,
                           int N_out, int K, const EpiArgs& e, cudaStream_t st) {
     if (M <= 0) return POLESTAR_OK;
-    const int NT = M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-    const CUtensorMap* mw = maps.get(W, (uint64_t)N_out, (uint64_t)K, 128);
-    const CUtensorMap* ma = maps.get(A, (uint64_t)a_rows_alloc, (uint64_t)K, (uint32_t)NT);
+    (void)a_rows_alloc;
+    // weights: tile-major [chunks * 256][64]; activations: exactly M rows, so that the rows of a token tile
+    // beyond M are out of bounds and arrive as zeros without being read
+    const CUtensorMap* mw = maps.get(W, (uint64_t)N_out * (uint64_t)(K / 64), 64, tc::BLOCK_F);
+    const CUtensorMap* ma = maps.get(A, (uint64_t)M, (uint64_t)K, tc::BLOCK_T);
     if (!mw || !ma) return POLESTAR_E_CUDA;
-    tc::GemmArgs g;
-    g.M = M; g.N_out = N_out; g.K = K; g.NT = NT;
-    const int tiles_f = N_out / 128, tiles_t = (M + NT - 1) / NT;
+    const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + tc::BLOCK_T - 1) / tc::BLOCK_T;
     const int kb = K / 64;
-    const int stage_bytes = 128 * 64 * 2 + NT * 64 * 2;
-    const int smem_budget = env_int("POLESTAR_GEMM_SMEM", 100 * 1024);
-    int stages = std::max(2, std::min(12, smem_budget / stage_bytes));
-    stages = env_int("POLESTAR_GEMM_STAGES", stages);
-    stages = std::max(2, std::min(12, std::min(stages, (220 * 1024) / stage_bytes)));
-    const int target = env_int("POLESTAR_GEMM_TARGET_CTAS", g_sm_count > 0 ? g_sm_count : 148);
-    int splits = std::max(1, (target + tiles_f * tiles_t - 1) / (tiles_f * tiles_t));
-    splits = std::min(splits, std::max(1, kb / 4));
-    splits = std::min(splits, env_int("POLESTAR_GEMM_MAX_SPLITS", 8));
-    while (splits > 1 && ((size_t)splits * tiles_f * tiles_t * NT * 128 * 4 > ws.partial_bytes ||
-                          tiles_f * tiles_t > ws.n_counters))
-        --splits;
-    g.stages = stages; g.splits = splits;
+    const int sms = g_sm_count > 0 ? g_sm_count : 148;
+    const long long U = (long long)tiles_f * tiles_t * kb;
+    long long G = std::min<long long>((long long)sms, U);
+    while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 > ws.partial_bytes)) --G;
+    if (tiles_f * tiles_t > ws.n_counters) return POLESTAR_E_INVAL;
+    tc::SkArgs g;
+    g.M = M; g.N_out = N_out; g.K = K; g.tiles_f = tiles_f; g.tiles_t = tiles_t;
+    g.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", 4)));
     g.partial = ws.partial; g.tile_counter = ws.counters; g.status = ws.status;
-    const size_t smem = (size_t)stages * stage_bytes + 1024;
-    auto kern = tc::gemm_tc_kernel<__nv_bfloat16, EPI>;
-    static size_t smem_set = 0;
-    if (smem > smem_set) {
+    const size_t smem = (size_t)g.stages * tc::STAGE_BYTES + 1024;
+    auto kern = tc::gemm_sk_kernel<__nv_bfloat16, EPI>;
+    static bool attr = false;
+    if (!attr) {
         CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-        smem_set = 225 * 1024;
+        attr = true;
     }
-    dim3 grid(tiles_f, tiles_t, splits);
-    kern<<<grid, tc::THREADS, smem, st>>>(*mw, *ma, g, e);
-    CK(cudaGetLastError());
+    CK(launch_k(kern, dim3((unsigned)G), dim3(tc::THREADS), smem, st, *mw, *ma, g, e));
     return POLESTAR_OK;
 }
 
@@ -150,7 +149,7 @@ struct Buffers {
     // persistent
     int* y; float2* rope; char* kc; char* vc; float* hc; float* pprev; float* aprev; float* theta; int* theta_cnt;
     int* tok_at_h0; float* drift; int* sel_idx; int* sel_cnt; unsigned char* patch; int* forced_idx; int* forced_cnt;
-    int* forced_commit; float* conf; int* yhat; float* delta; float* Delta; float* taud; int* commit_flags;
+    int* forced_commit; int* forced_tok; float* conf; int* yhat; float* delta; float* Delta; float* taud; int* commit_flags;
     int* suffix_flags; int* seq_info; int* head_count; int* suf_seq; int* suf_w; int* stats; int* status;
     int* list_count; float* hidden_keep;
     // scratch
@@ -161,7 +160,7 @@ struct Buffers {
 
 static const int CONF_CHUNKS = 32;
 static const int FORCED_COMMIT_MAX = 512;
-static const size_t GEMM_PARTIAL_BYTES = (size_t)64 << 20;
+static const size_t GEMM_PARTIAL_BYTES = (size_t)40 << 20;   // 2 slots x 148 CTAs x 128 x 256 fp32
 static const int GEMM_COUNTERS = 8192;
 
 struct polestar_ctx {
@@ -186,7 +185,7 @@ struct polestar_ctx {
     std::vector<int> cum;
     StepDesc last_sd;
     int last_act_row_off = 0;
-    bool forced_select = false, forced_commit = false;
+    bool forced_select = false, forced_commit = false, forced_tokens = false;
     int forced_commit_n = 0;
     std::vector<int> seq_info_host;
     // launch accounting and optional per-family device timing (POLESTAR_FLAG_PROFILE)
@@ -281,6 +280,7 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(forced_idx, int, L * bs * Wm);
     TAKE(forced_cnt, int, L * bs);
     TAKE(forced_commit, int, bs * FORCED_COMMIT_MAX);
+    TAKE(forced_tok, int, bs * FORCED_COMMIT_MAX);
     TAKE(conf, float, rows_lm);
     TAKE(yhat, int, rows_lm);
     TAKE(delta, float, bs * B);
@@ -357,8 +357,7 @@ struct Path {
     template <int EPI>
     static int gemm(polestar_ctx* c, const void* A, int a_rows_alloc, const void* W, int M, int N_out, int K,
                     const EpiArgs& e) {
-        if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 128 == 0 &&
-            (EPI != EPI_QKV || c->m.head_dim == 128))
+        if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 256 == 0)
             return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st);
         return launch_gemm_simt<T, EPI>(A, W, M, N_out, K, e, c->st);
     }
@@ -374,7 +373,7 @@ struct Path {
             set = smem;
         }
         dim3 grid((a.n_rows + wpb - 1) / wpb, a.n_heads);
-        attention_simt_kernel<T><<<grid, wpb * 32, smem, c->st>>>(a);
+        CK(launch_k(attention_simt_kernel<T>, dim3(grid), dim3(wpb * 32), smem, c->st, a));
         CK(cudaGetLastError());
         return POLESTAR_OK;
     }
@@ -400,10 +399,10 @@ struct Path {
                                     : (double)M;
         {
             Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (esd + 4), 0, 2);
-            build_rows_kernel<<<(M + 255) / 256, 256, 0, st>>>(sd, b.rows);
+            CK(launch_k(build_rows_kernel, dim3((M + 255) / 256), dim3(256), 0, st, sd, b.rows));
             CK(cudaMemsetAsync(b.stats, 0, 4 * sizeof(int), st));
-            embed_rows_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.y, (const T*)c->embed, d, b.x, b.packet, b.patch,
-                                                   b.tok_at_h0, b.stats);
+            CK(launch_k(embed_rows_kernel<T>, dim3(M), dim3(256), 0, st, sd, b.rows, b.y, (const T*)c->embed, d, b.x, b.packet, b.patch,
+                                                   b.tok_at_h0, b.stats));
             CK(cudaGetLastError());
         }
 
@@ -415,12 +414,12 @@ struct Path {
             const bool last = l == L - 1;
             if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
                 Scope sc(c, POLESTAR_PROF_MISC, 0, 0, 1);
-                keep_hidden_kernel<<<bs * B, 256, 0, st>>>(sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d);
+                CK(launch_k(keep_hidden_kernel, dim3(bs * B), dim3(256), 0, st, sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d));
             }
             {
                 Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
-                prep_qkv_kernel<T><<<M, 256, 0, st>>>(sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
-                                                     c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag);
+                CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(256), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
+                                                     c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag));
                 CK(cudaGetLastError());
             }
             EpiArgs e;
@@ -462,7 +461,7 @@ struct Path {
                 s.mode = p.select_mode;
                 s.k = p.select_mode == POLESTAR_SELECT_TOPK_FRAC ? (int)floorf(p.select_frac * (float)sd.W + 0.5f) : p.select_k;
                 s.W_max = Wm; s.thresh = p.select_thresh; s.floor_ = p.drift_floor;
-                step_select_kernel<<<1, SEL_THREADS, 0, st>>>(sd, s);
+                CK(launch_k(step_select_kernel, dim3(1), dim3(SEL_THREADS), 0, st, sd, s));
                 CK(cudaGetLastError());
                 list = b.list; m2_count = b.list_count;
             }
@@ -474,7 +473,7 @@ struct Path {
             }
             {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
-                prep_rows_kernel<T><<<M, 256, 0, st>>>(b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf);
+                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(256), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
                 CK(cudaGetLastError());
             }
             {
@@ -493,7 +492,7 @@ struct Path {
         }
         if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
             Scope sc(c, POLESTAR_PROF_MISC, 0, 0, 1);
-            keep_hidden_kernel<<<bs * B, 256, 0, st>>>(sd, b.x, act_off, d, b.hidden_keep + (size_t)L * bs * B * d);
+            CK(launch_k(keep_hidden_kernel, dim3(bs * B), dim3(256), 0, st, sd, b.x, act_off, d, b.hidden_keep + (size_t)L * bs * B * d));
         }
 
         // logits of the active rows (+ eligible suffix rows), confidences
@@ -501,11 +500,11 @@ struct Path {
         const int Mh = use_suffix ? c->rows_lm : bs * B;
         {
             Scope sc(c, POLESTAR_PROF_STAGE, (double)bs * B * d * (4 + esd), 0, 2);
-            build_head_list_kernel<<<1, 256, 0, st>>>(sd, b.y, m.mask_id, b.sel_idx + (size_t)(L - 1) * bs * Wm,
+            CK(launch_k(build_head_list_kernel, dim3(1), dim3(256), 0, st, sd, b.y, m.mask_id, b.sel_idx + (size_t)(L - 1) * bs * Wm,
                                                       b.sel_cnt + (size_t)(L - 1) * bs, use_suffix, 0, b.head_list,
-                                                      b.head_count, b.suf_seq, b.suf_w);
-            prep_head_kernel<T><<<Mh, 256, 0, st>>>(b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
-                                                   (T*)b.a_head);
+                                                      b.head_count, b.suf_seq, b.suf_w));
+            CK(launch_k(prep_head_kernel<T>, dim3(Mh), dim3(256), 0, st, b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
+                                                   (T*)b.a_head));
             CK(cudaGetLastError());
         }
         {
@@ -518,10 +517,10 @@ struct Path {
         }
         {
             Scope sc(c, POLESTAR_PROF_CONFIDENCE, (double)bs * B * m.vocab * 4, 0, 3);
-            conf_partial_kernel<<<dim3(CONF_CHUNKS, Mh), 256, 0, st>>>(b.logits, b.head_count, Mh, m.vocab, m.mask_id,
-                                                                      CONF_CHUNKS, b.conf_part);
-            conf_final_kernel<<<(Mh + 127) / 128, 128, 0, st>>>(b.conf_part, b.head_count, Mh, CONF_CHUNKS, b.yhat, b.conf);
-            delta_kernel<<<bs, 256, 0, st>>>(sd, b.kl, act_off, m.n_heads, b.delta);
+            CK(launch_k(conf_partial_kernel, dim3(CONF_CHUNKS, Mh), dim3(256), 0, st, b.logits, b.head_count, Mh, m.vocab, m.mask_id,
+                                                                      CONF_CHUNKS, b.conf_part));
+            CK(launch_k(conf_final_kernel, dim3((Mh + 127) / 128), dim3(128), 0, st, b.conf_part, b.head_count, Mh, CONF_CHUNKS, b.yhat, b.conf));
+            CK(launch_k(delta_kernel, dim3(bs), dim3(256), 0, st, sd, b.kl, act_off, m.n_heads, b.delta));
             CK(cudaGetLastError());
         }
         c->last_act_row_off = act_off;
@@ -606,6 +605,7 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     a.head_count = b.head_count; a.suf_seq = b.suf_seq; a.suf_w = b.suf_w;
     a.forced_pos = c->forced_commit ? b.forced_commit : nullptr;
     a.forced_n = c->forced_commit_n;
+    a.forced_tok = (c->forced_commit && c->forced_tokens) ? b.forced_tok : nullptr;
     a.seq_info = b.seq_info;
     a.n_heads = c->m.n_heads; a.hist = p.hist; a.mask_id = c->m.mask_id; a.eos_id = c->m.eos_id;
     a.act_row_off = c->last_act_row_off; a.steps_used = c->steps_used;
@@ -618,7 +618,7 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     if (entry_like) CK(cudaMemsetAsync(b.theta_cnt, 0, p.batch * sizeof(int), c->st));   // history cleared at block entry
     {
         Scope sc(c, POLESTAR_PROF_COMMIT, (double)p.batch * c->B * 16, 0, 1);
-        commit_kernel<<<p.batch, 256, 0, c->st>>>(sd, a);
+        CK(launch_k(commit_kernel, dim3(p.batch), dim3(256), 0, c->st, sd, a));
         CK(cudaGetLastError());
     }
     c->seq_info_host.resize((size_t)p.batch * 8 + 8);
@@ -637,6 +637,7 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     c->prof_used = 0;
     c->pending = false;
     c->forced_commit = false;
+    c->forced_tokens = false;
     const int* si = c->seq_info_host.data();
     polestar_commit_info ci;
     memset(&ci, 0, sizeof(ci));
@@ -690,6 +691,7 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     if (ws_bytes < need) return POLESTAR_E_NOSPACE;
     int rc = init_device_info();
     if (rc) return rc;
+    g_use_pdl = env_int("POLESTAR_PDL", 1) != 0;
     polestar_ctx* c = new (std::nothrow) polestar_ctx();
     if (!c) return POLESTAR_E_INVAL;
     c->m = *m; c->p = *p;
@@ -830,7 +832,15 @@ extern "C" int polestar_force(polestar_ctx* c, int32_t what, int32_t layer, cons
         if (n) CK(cudaMemcpyAsync(c->b.forced_commit, idx, (size_t)bs * n * sizeof(int), cudaMemcpyHostToDevice, c->st));
         CK(cudaStreamSynchronize(c->st));
         c->forced_commit = true;
+        c->forced_tokens = false;
         c->forced_commit_n = n;
+        return POLESTAR_OK;
+    }
+    if (what == POLESTAR_FORCE_TOKENS) {
+        if (!c->forced_commit || n != c->forced_commit_n) return POLESTAR_E_STATE;
+        if (n) CK(cudaMemcpyAsync(c->b.forced_tok, idx, (size_t)bs * n * sizeof(int), cudaMemcpyHostToDevice, c->st));
+        CK(cudaStreamSynchronize(c->st));
+        c->forced_tokens = true;
         return POLESTAR_OK;
     }
     return POLESTAR_E_INVAL;
@@ -902,7 +912,7 @@ static size_t refresh_layout(int batch, int max_rows, int d, int head_dim, int P
     Plan pl;
     pl.take((size_t)batch * max_rows * d * 2 + 256 * (size_t)d * 2);   // staged rows (+ one tile of slack)
     *off_rope = pl.take((size_t)P * (head_dim / 2) * sizeof(float2));
-    *off_part = pl.take(GEMM_PARTIAL_BYTES / 2);
+    *off_part = pl.take(GEMM_PARTIAL_BYTES);
     *off_cnt = pl.take(GEMM_COUNTERS * sizeof(int));
     *off_status = pl.take(sizeof(int));
     return pl.total;
@@ -938,7 +948,7 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     float2* rope = (float2*)(sc + off_rope);
     static MapCache maps;
     GemmWs ws;
-    ws.partial = (float*)(sc + off_part); ws.partial_bytes = GEMM_PARTIAL_BYTES / 2;
+    ws.partial = (float*)(sc + off_part); ws.partial_bytes = GEMM_PARTIAL_BYTES;
     ws.counters = (int*)(sc + off_cnt); ws.n_counters = GEMM_COUNTERS; ws.status = (int*)(sc + off_status);
     // the scratch is caller memory with unknown contents: the split-K tile counters must start at zero
     CK(cudaMemsetAsync(ws.counters, 0, GEMM_COUNTERS * sizeof(int) + 1024, st));
@@ -952,7 +962,7 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     e.rope = rope; e.q_out = q_out; e.kc = kc; e.vc = vc; e.n_heads = n_heads; e.n_kv = n_kv; e.head_dim = head_dim;
     e.idx = idx; e.counts = counts; e.max_rows = max_rows; e.P = P;
     const int dq = n_heads * head_dim, dkv = n_kv * head_dim;
-    if (d % 64 == 0 && (dq + 2 * dkv) % 128 == 0 && head_dim == 128 && !env_int("POLESTAR_REFRESH_SIMT", 0))
+    if (d % 64 == 0 && (dq + 2 * dkv) % 256 == 0 && !env_int("POLESTAR_REFRESH_SIMT", 0))
         return launch_gemm_tc<EPI_QKV_REFRESH>(maps, ws, a_buf, M, wqkv, M, dq + 2 * dkv, d, e, st);
     return launch_gemm_simt<__nv_bfloat16, EPI_QKV_REFRESH>(a_buf, wqkv, M, dq + 2 * dkv, d, e, st);
 }

@@ -96,10 +96,19 @@ def run_forced(name, n_steps, **kw):
             close(gpu.read(Bd.READ_CONF)[s], conf, tol, f"step {step} conf")
         infos = ora.commit()
         forced = np.full((p.batch, p.block + gpu.W_max), -1, np.int32)
+        ftok = np.zeros_like(forced)
+        yh_gpu = gpu.read(Bd.READ_YHAT)
         for s, i in enumerate(infos):
-            pos = [int(ora.seqs[s].act[j]) for j in np.nonzero(i["commit"] & i["masked"])[0]] + i["suffix_committed"]
+            rows = np.nonzero(i["commit"] & i["masked"])[0]
+            pos = [int(ora.seqs[s].act[j]) for j in rows] + i["suffix_committed"]
             forced[s, :len(pos)] = pos
-        gpu.force_commit(forced)
+            ftok[s, :len(pos)] = ora.tokens()[s, pos]
+            # the CUDA path's own argmax may differ only where the oracle's two best logits nearly tie
+            lg = ora.seqs[s].trace["logits"]
+            for j in rows:
+                if yh_gpu[s, j] != i["yhat"][j]:
+                    assert abs(lg[j, yh_gpu[s, j]] - lg[j, i["yhat"][j]]) <= 2 * tol * max(1.0, p.logit_scale)
+        gpu.force_commit(forced, ftok)
         ci = gpu.commit()
         assert ci.n_committed == sum(i["n_committed"] for i in infos)
         assert np.array_equal(gpu.tokens(), ora.tokens()), f"step {step} tokens"

@@ -102,6 +102,14 @@ def test_pack_weights_layout():
     qa, ka = l["wq"][:8] @ x, l["wk"] @ x
     qb, kb = qkv[:8] @ x, qkv[16:24] @ x
     assert torch.allclose(qa @ ka, qb @ kb, atol=1e-6)
+    # tile-major storage of bf16 GEMM weights: block (o / 128, i / 64) is contiguous
+    wt = torch.arange(512 * 128, dtype=torch.float32).view(512, 128).to(torch.bfloat16)
+    tm = Bd.tile_major(wt)
+    assert torch.equal(tm.flatten()[:64], wt[0, :64]) and torch.equal(tm.flatten()[64:128], wt[1, :64])
+    assert torch.equal(tm.flatten()[256 * 64:256 * 64 + 64], wt[0, 64:128])
+    assert torch.equal(tm.flatten()[2 * 256 * 64:2 * 256 * 64 + 64], wt[256, :64])
+    assert torch.equal(Bd.untile(tm), wt)
+    assert torch.equal(Bd.tile_major(wt.float()), wt.float())          # fp32 stays row-major
 
 
 def test_generator_is_device_independent_and_sliceable():
