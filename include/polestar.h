@@ -290,6 +290,22 @@ int polestar_k_confidence(const float *logits_dev, int32_t rows, int32_t vocab, 
                           int32_t *yhat_dev, float *conf_dev, void *scratch_dev, size_t scratch_bytes,
                           void *cuda_stream);
 
+/* Same result as polestar_k_confidence for callers that cannot provide or allocate device scratch
+ * (a server whose memory pool owns every byte of the GPU, a loop that must not hit cudaMalloc's
+ * device-wide synchronisation, a plug-in interface that passes inputs and outputs only).  The
+ * partial results live in a 512 KB array that is part of the library image on every GPU using it.
+ * The paper has no counterpart: this is a packaging variant of the confidence kernel.
+ *   - rows <= POLESTAR_NOALLOC_MAX_ROWS, otherwise POLESTAR_E_NOSPACE (use polestar_k_confidence).
+ *   - Calls no allocation routine.  The first call on each device looks up the array's device
+ *     address (cudaGetSymbolAddress, with the caller's current device); make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array: calls that may overlap on the GPU (different
+ *     streams without ordering) race on it and must be serialised by the caller.  Nothing in the
+ *     array has to be cleared between calls; it simply keeps the last call's partial results. */
+#define POLESTAR_NOALLOC_MAX_ROWS 1024
+int polestar_k_confidence_noalloc(const float *logits_dev, int32_t rows, int32_t vocab, int32_t mask_id,
+                                  int32_t *yhat_dev, float *conf_dev, void *cuda_stream);
+
 /* Number of SMs the library sized its grids for (0 before any context exists). */
 int polestar_sm_count(void);
 

@@ -31,7 +31,8 @@ EXPORTS = [
     "polestar_workspace_bytes", "polestar_init", "polestar_step", "polestar_commit", "polestar_tokens",
     "polestar_read", "polestar_force", "polestar_profile", "polestar_destroy", "polestar_strerror",
     "polestar_k_attention", "polestar_k_hidden_delta", "polestar_k_select",
-    "polestar_k_refresh_scratch_bytes", "polestar_k_refresh", "polestar_k_confidence", "polestar_sm_count",
+    "polestar_k_refresh_scratch_bytes", "polestar_k_refresh", "polestar_k_confidence",
+    "polestar_k_confidence_noalloc", "polestar_sm_count",
 ]
 
 
@@ -121,6 +122,8 @@ def load():
                                        i32, vp, sz, vp]
     lib.polestar_k_confidence.restype = C.c_int
     lib.polestar_k_confidence.argtypes = [vp, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.polestar_k_confidence_noalloc.restype = C.c_int
+    lib.polestar_k_confidence_noalloc.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     lib.polestar_sm_count.restype = C.c_int
     lib.polestar_sm_count.argtypes = []
     _lib = lib
@@ -397,3 +400,14 @@ def polestar_k_confidence(logits, mask_id, yhat, conf, scratch):
     rows, V = logits.shape
     _check(load().polestar_k_confidence(_ptr(logits), rows, V, mask_id, _ptr(yhat), _ptr(conf), _ptr(scratch),
                                         scratch.numel() * scratch.element_size(), C.c_void_p(_stream())))
+
+
+NOALLOC_MAX_ROWS = 1024
+
+
+def polestar_k_confidence_noalloc(logits, mask_id, yhat, conf):
+    """Confidence of logits rows using the library's built-in scratch (no allocation, rows <= 1024).
+    For callers that cannot hand over scratch memory; concurrent calls on one device must be serialised."""
+    rows, V = logits.shape
+    _check(load().polestar_k_confidence_noalloc(_ptr(logits), rows, V, mask_id, _ptr(yhat), _ptr(conf),
+                                                C.c_void_p(_stream())))

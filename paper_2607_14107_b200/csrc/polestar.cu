@@ -978,3 +978,48 @@ extern "C" int polestar_k_confidence(const float* logits, int32_t rows, int32_t 
     CK(cudaGetLastError());
     return POLESTAR_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// Confidence without any caller-provided or allocated scratch
+// ------------------------------------------------------------------------------------------
+// Some callers have no way to obtain device scratch at call time: a serving process that handed
+// its whole memory budget to a KV-cache pool at start-up, a latency-critical loop in which
+// cudaMalloc's implicit device synchronisation is not acceptable, or a plug-in that is only
+// given input and output buffers.  For them the per-chunk partial results of the confidence
+// kernel live in a fixed array inside the library image (every GPU that loads the library
+// carries these 512 KB until the process exits).
+static __device__ __align__(256) ConfPart g_conf_scratch[POLESTAR_NOALLOC_MAX_ROWS * CONF_CHUNKS];
+
+// On the host, `g_conf_scratch` is only a handle of the symbol, not a device address: the real
+// address differs per device and has to be looked up once per device with that device current.
+static ConfPart* conf_scratch_ptr(int* err) {
+    static ConfPart* ptrs[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= 64) { last_cuda_error = e; *err = POLESTAR_E_CUDA; return nullptr; }
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_conf_scratch);
+        if (e != cudaSuccess || !p) { last_cuda_error = e; *err = POLESTAR_E_CUDA; return nullptr; }
+        ptrs[dev] = (ConfPart*)p;
+    }
+    *err = POLESTAR_OK;
+    return ptrs[dev];
+}
+
+extern "C" int polestar_k_confidence_noalloc(const float* logits, int32_t rows, int32_t vocab, int32_t mask_id,
+                                             int32_t* yhat, float* conf, void* stream) {
+    if (!logits || !yhat || !conf || rows < 0 || vocab <= 0) return POLESTAR_E_INVAL;
+    if (rows > POLESTAR_NOALLOC_MAX_ROWS) return POLESTAR_E_NOSPACE;    // beyond the built-in scratch: use polestar_k_confidence
+    if (rows == 0) return POLESTAR_OK;
+    int err = POLESTAR_OK;
+    ConfPart* scratch = conf_scratch_ptr(&err);
+    if (!scratch) return err;
+    cudaStream_t st = (cudaStream_t)stream;
+    // every partial the second kernel reads is written by the first one in this call, so nothing of the
+    // previous call's contents has to be cleared
+    conf_partial_kernel<<<dim3(CONF_CHUNKS, rows), 256, 0, st>>>(logits, nullptr, rows, vocab, mask_id, CONF_CHUNKS, scratch);
+    conf_final_kernel<<<(rows + 127) / 128, 128, 0, st>>>(scratch, nullptr, rows, CONF_CHUNKS, yhat, conf);
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
+}
