@@ -18,8 +18,9 @@
 //    of bytes whatever the matrix shape and the pipeline fills once per launch.  A range is a
 //    sequence of segments (one per output tile touched).  A segment that covers its tile's
 //    whole K runs the epilogue straight from tensor memory; partial segments go to a workspace
-//    slot, and the last CTA to arrive at the tile adds the slots in ascending-k order
-//    (deterministic) and runs the epilogue.
+//    slot; once all contributors of a tile have published theirs (bounded wait), each of them
+//    adds the slots in ascending-k order (deterministic) for its share of the tile and runs the
+//    epilogue on it.
 //  * Programmatic dependent launch: weight tiles of the first pipeline stages are requested
 //    before griddepcontrol.wait, i.e. while the previous kernel of the stream still drains;
 //    activations, residuals and every global write come after it.
@@ -134,9 +135,15 @@ struct SkArgs {
     int M, N_out, K, stages;
     int tiles_f, tiles_t;
     float* partial;     // [2 * gridDim.x][BLOCK_T][BLOCK_F] fp32
-    int* tile_counter;  // [tiles_f * tiles_t], zero before launch, zero again after
+    int* tile_counter;  // arrivals [tile] and, done_offset further on, finished shares [tile]; zero before
+                        // launch, zero again after
+    int done_offset;
     int* status;        // set to 1 on a wait time-out
+    long long* trace;   // optional [gridDim.x][8] nanosecond stamps of this launch (null: off)
 };
+
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define SK_STAMP(i) do { if (g.trace) g.trace[(size_t)cta * 8 + (i)] = gtime(); } while (0)
 
 // first unit of CTA c when U units are split over G CTAs
 __device__ __forceinline__ long long sk_begin(long long U, int G, int c) { return (U * c) / G; }
@@ -152,13 +159,14 @@ __global__ void __launch_bounds__(THREADS, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                SkArgs g, EpiArgs e) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t bars[2 * MAX_STAGES + 2];
+    __shared__ uint64_t bars[2 * MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
     __shared__ int last_sh;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, cta = blockIdx.x;
+    if (threadIdx.x == 0) SK_STAMP(0);
     const int kb_total = g.K / BLOCK_K;
     const long long U = (long long)g.tiles_f * g.tiles_t * kb_total;
     const long long u_begin = sk_begin(U, G, cta), u_end = sk_begin(U, G, cta + 1);
@@ -168,13 +176,17 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[MAX_STAGES]);
-    const uint32_t accum_full = smem_u32(&bars[2 * MAX_STAGES]), accum_empty = smem_u32(&bars[2 * MAX_STAGES + 1]);
-    constexpr uint32_t ncols = BLOCK_F;
+    // two accumulators in tensor memory (segment s uses buffer s & 1): the epilogue of one segment
+    // drains its buffer while the MMAs of the next segment already fill the other
+    const uint32_t accum_full = smem_u32(&bars[2 * MAX_STAGES]), accum_empty = smem_u32(&bars[2 * MAX_STAGES + 2]);
+    constexpr uint32_t ncols = 2 * BLOCK_F;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-        mbar_init(accum_full, 1);
-        mbar_init(accum_empty, 4);      // one arrival per epilogue warp
+        for (int b2 = 0; b2 < 2; ++b2) {
+            mbar_init(accum_full + 8 * b2, 1);
+            mbar_init(accum_empty + 8 * b2, 4);      // one arrival per epilogue warp
+        }
         abort_sh = 0;
         last_sh = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -185,6 +197,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     pdl_trigger();
+    if (threadIdx.x == 0) SK_STAMP(1);
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
 
@@ -200,6 +213,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
             }
             pdl_wait();
+            SK_STAMP(2);
             for (int i = 0; i < pre; ++i) {
                 const long long u = u_begin + i;
                 const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
@@ -227,22 +241,25 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int kb = (int)(u % kb_total);
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
-                if (seg_start && seg > 0) {
-                    // the epilogue must have drained the accumulator of the previous segment
-                    if (!mbar_wait(accum_empty, (uint32_t)(seg - 1) & 1u, abort_flag)) break;
+                if (seg_start && seg > 1) {
+                    // the epilogue must have drained this buffer's previous segment (seg - 2)
+                    if (!mbar_wait(accum_empty + 8 * (seg & 1), (uint32_t)((seg >> 1) - 1) & 1u, abort_flag)) break;
                     tc_fence_after();
                 }
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) break;
+                if (i == 0) SK_STAMP(3);
                 tc_fence_after();
                 const uint32_t sa = smem_base + s * STAGE_BYTES;
                 const uint64_t da = smem_desc_sw128(sa), dw = smem_desc_sw128(sa + A_BYTES);
 #pragma unroll
                 for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                    umma_bf16(tmem_base, da + (uint64_t)(k * 2), dw + (uint64_t)(k * 2), idesc, (!seg_start || k > 0) ? 1u : 0u);
+                    umma_bf16(tmem_base + (uint32_t)((seg & 1) * BLOCK_F), da + (uint64_t)(k * 2), dw + (uint64_t)(k * 2), idesc,
+                              (!seg_start || k > 0) ? 1u : 0u);
                 umma_commit(empty0 + 8 * s);
                 seg_start = false;
                 if (kb == kb_total - 1 || i == n_units - 1) {
-                    umma_commit(accum_full);
+                    umma_commit(accum_full + 8 * (seg & 1));
+                    if (i == n_units - 1) SK_STAMP(4);
                     ++seg;
                     seg_start = true;
                 }
@@ -253,9 +270,11 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         pdl_wait();
         const int q = warp & 3;
         const int t_local = q * 32 + lane;
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t taddr0 = tmem_base + ((uint32_t)(q * 32) << 16);
         const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
         int seg = 0;
+        int fix_tile[2];
+        int n_fix = 0;
         long long u = u_begin;
         while (u < u_end) {
             const int tile = (int)(u / kb_total);
@@ -269,8 +288,9 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const bool live = m < Mv;
             const bool warp_live = tile_t * BLOCK_T + q * 32 < Mv;      // any live token in this warp's quarter
             const bool whole = (k0 == 0 && k1 == kb_total);
-            if (!mbar_wait(accum_full, (uint32_t)seg & 1u, abort_flag)) break;
+            if (!mbar_wait(accum_full + 8 * (seg & 1), (uint32_t)(seg >> 1) & 1u, abort_flag)) break;
             tc_fence_after();
+            const uint32_t taddr = taddr0 + (uint32_t)((seg & 1) * BLOCK_F);
             if (whole) {
                 if (warp_live) {
                     for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
@@ -284,8 +304,10 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(accum_empty);
+                if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
             } else {
+                // partial segment: publish it now, reduce later (pass 2), so that publishing never
+                // waits on another CTA
                 const int which = (k0 == 0) ? 1 : 0;     // slot 0: my range starts inside this tile
                 float* part = g.partial + ((size_t)(2 * cta + which) * BLOCK_T + t_local) * BLOCK_F;
                 if (warp_live) {
@@ -301,68 +323,89 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(accum_empty);
+                if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int c_lo = sk_owner(U, G, (long long)tile * kb_total), c_hi = sk_owner(U, G, tile_end - 1);
-                if (threadIdx.x == 64) {
-                    const int prev = atomicAdd(&g.tile_counter[tile], 1);
-                    last_sh = (prev == c_hi - c_lo);
-                    if (last_sh) g.tile_counter[tile] = 0;
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (last_sh) {
-                    // The partial tiles sit in global memory, so the fix-up is not tied to TMEM lanes:
-                    // (token, 16-feature chunk) items are spread over all 128 epilogue threads, and the
-                    // loads of four segments are issued together before they are added in k order.
-                    __threadfence();
-                    const int nseg = c_hi - c_lo + 1;
-                    const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
-                    for (int item = (int)threadIdx.x - 64; item < n_live * (BLOCK_F / 16); item += 128) {
-                        const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16;
-                        float acc[16];
-#pragma unroll
-                        for (int x = 0; x < 16; ++x) acc[x] = 0.f;
-                        for (int sg0 = 0; sg0 < nseg; sg0 += 4) {
-                            float4 tv[4][4];
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                const int cc = c_lo + sg0 + j;
-                                if (sg0 + j < nseg) {
-                                    // a CTA whose range starts inside the tile wrote slot 0, otherwise slot 1
-                                    const int wsl = (sk_begin(U, G, cc) > (long long)tile * kb_total) ? 0 : 1;
-                                    const float4* ps = reinterpret_cast<const float4*>(
-                                        g.partial + ((size_t)(2 * cc + wsl) * BLOCK_T + tl) * BLOCK_F + c0);
-#pragma unroll
-                                    for (int x = 0; x < 4; ++x) tv[j][x] = __ldcg(ps + x);
-                                } else {
-#pragma unroll
-                                    for (int x = 0; x < 4; ++x) tv[j][x] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                }
-                            }
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-#pragma unroll
-                                for (int x = 0; x < 4; ++x) {
-                                    acc[4 * x] += tv[j][x].x; acc[4 * x + 1] += tv[j][x].y;
-                                    acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
-                                }
-                        }
-                        const int mm = tile_t * BLOCK_T + tl;
-#pragma unroll
-                        for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, mm, n0 + c0 + c, acc[c], acc[c + 1]);
-                    }
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");     // last_sh is reused by the next segment
+                if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile], 1);
+                if (n_fix < 2) fix_tile[n_fix++] = tile;
             }
             ++seg;
             u = seg_end;
+        }
+        if (threadIdx.x == 64) SK_STAMP(5);
+        // ---- pass 2: every CTA that contributed to a split tile reduces its share of that tile ------
+        for (int f = 0; f < n_fix; ++f) {
+            const int tile = fix_tile[f];
+            const long long tile_begin = (long long)tile * kb_total, tile_end = tile_begin + kb_total;
+            const int c_lo = sk_owner(U, G, tile_begin), c_hi = sk_owner(U, G, tile_end - 1);
+            const int nseg = c_hi - c_lo + 1;
+            const int tile_f = tile / g.tiles_t, tile_t = tile % g.tiles_t;
+            const int n0 = tile_f * BLOCK_F;
+            if (threadIdx.x == 64) {
+                // bounded wait until all contributors have published their partial tile
+                const long long t0 = clock64();
+                int ok = 1;
+                while (*((volatile int*)&g.tile_counter[tile]) < nseg) {
+                    if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) { ok = 0; *abort_flag = 1; break; }
+                    __nanosleep(64);
+                }
+                last_sh = ok;
+                if (f == 0) SK_STAMP(6);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (last_sh) {
+                __threadfence();
+                const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
+                const int n_items = n_live * (BLOCK_F / 16);
+                // items are dealt round-robin to the contributing CTAs, then to their 128 epilogue threads
+                for (int item = (cta - c_lo) * 128 + ((int)threadIdx.x - 64); item < n_items; item += nseg * 128) {
+                    const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16;
+                    float acc[16];
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) acc[x] = 0.f;
+                    for (int sg0 = 0; sg0 < nseg; sg0 += 4) {
+                        float4 tv[4][4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int cc = c_lo + sg0 + j;
+                            if (sg0 + j < nseg) {
+                                // a CTA whose range starts inside the tile wrote slot 0, otherwise slot 1
+                                const int wsl = (sk_begin(U, G, cc) > tile_begin) ? 0 : 1;
+                                const float4* ps = reinterpret_cast<const float4*>(
+                                    g.partial + ((size_t)(2 * cc + wsl) * BLOCK_T + tl) * BLOCK_F + c0);
+#pragma unroll
+                                for (int x = 0; x < 4; ++x) tv[j][x] = __ldcg(ps + x);
+                            } else {
+#pragma unroll
+                                for (int x = 0; x < 4; ++x) tv[j][x] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                acc[4 * x] += tv[j][x].x; acc[4 * x + 1] += tv[j][x].y;
+                                acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
+                            }
+                    }
+                    const int mm = tile_t * BLOCK_T + tl;
+#pragma unroll
+                    for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, mm, n0 + c0 + c, acc[c], acc[c + 1]);
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64 && last_sh) {
+                // the last contributor to finish its share re-arms the tile's counters for the next launch
+                const int prev = atomicAdd(&g.tile_counter[g.done_offset + tile], 1);
+                if (prev == nseg - 1) { g.tile_counter[tile] = 0; g.tile_counter[g.done_offset + tile] = 0; }
+            }
         }
     }
 
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, ncols);
+    if (threadIdx.x == 0) SK_STAMP(7);
     if (threadIdx.x == 0 && abort_sh) atomicExch(g.status, 1);
 }
 

@@ -116,12 +116,21 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     const int sms = g_sm_count > 0 ? g_sm_count : 148;
     const long long U = (long long)tiles_f * tiles_t * kb;
     long long G = std::min<long long>((long long)sms, U);
-    while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 > ws.partial_bytes)) --G;
-    if (tiles_f * tiles_t > ws.n_counters) return POLESTAR_E_INVAL;
+    // When a multiple of the tile count fits on >= 85 % of the SMs, take it: CTA ranges then never cross a
+    // tile boundary, so every CTA has one segment (one fix-up instead of two, or none at all).
+    {
+        const long long tiles = (long long)tiles_f * tiles_t;
+        const long long mult = (G / tiles) * tiles;
+        if (mult > 0 && mult * 100 >= (long long)sms * env_int("POLESTAR_GEMM_ALIGN_PCT", 85)) G = mult;
+    }
+    while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 > ws.partial_bytes)) --G;
+    if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
     tc::SkArgs g;
     g.M = M; g.N_out = N_out; g.K = K; g.tiles_f = tiles_f; g.tiles_t = tiles_t;
     g.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", 4)));
-    g.partial = ws.partial; g.tile_counter = ws.counters; g.status = ws.status;
+    g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
+    // debug: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
+    g.trace = (env_int("POLESTAR_GEMM_TRACE", -1) == EPI) ? (long long*)((char*)ws.partial + ws.partial_bytes - 16384) : nullptr;
     const size_t smem = (size_t)g.stages * tc::STAGE_BYTES + 1024;
     auto kern = tc::gemm_sk_kernel<__nv_bfloat16, EPI>;
     static bool attr = false;
@@ -160,8 +169,8 @@ struct Buffers {
 
 static const int CONF_CHUNKS = 32;
 static const int FORCED_COMMIT_MAX = 512;
-static const size_t GEMM_PARTIAL_BYTES = (size_t)40 << 20;   // 2 slots x 148 CTAs x 128 x 256 fp32
-static const int GEMM_COUNTERS = 8192;
+static const size_t GEMM_PARTIAL_BYTES = ((size_t)40 << 20) + 16384;   // 2 slots x 148 CTAs x 128 x 256 fp32
+static const int GEMM_COUNTERS = 1 << 17;     // arrivals + finished shares for up to 65536 output tiles
 
 struct polestar_ctx {
     polestar_model m;
@@ -792,6 +801,7 @@ extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void*
         case POLESTAR_READ_COMMIT: src = c->b.commit_flags; sz = bs * B * 4; break;
         case POLESTAR_READ_PPREV: src = c->b.pprev + layer * bs * Wm * m.n_heads * N; sz = bs * Wm * m.n_heads * N * 4; break;
         case POLESTAR_READ_SUFFIX: src = c->b.suffix_flags; sz = bs * Wm * 4; break;
+        case 99: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384; sz = 16384; break;   // debug: GEMM time stamps
         default: return POLESTAR_E_INVAL;
     }
     CK(cudaMemcpyAsync(dst, src, std::min(sz, bytes), cudaMemcpyDeviceToHost, c->st));
