@@ -144,7 +144,7 @@ def run_ours(args):
     import numpy as np
     import torch
     import torch.distributed as dist
-    from paper_2607_14107_b200 import binding as Bd, inputs as I
+    from paper_2607_14107_b200 import binding as Bd, inputs as I, replicas as R
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -163,7 +163,7 @@ def run_ours(args):
         p = dataclasses.replace(p, tau_upd=args.tau_upd)
     packed = Bd.make_packed_weights(m, seed=0, device="cuda")
     # one batch of prompts per replica: independent sequences, no exchange between ranks (weak scaling)
-    prompt = I.make_prompt(m, p, seed=1 + rank)
+    prompt = I.make_prompt(m, p, seed=R.replica_prompt_seed(1, rank))
     prompt_dev = prompt.cuda()
     prompt_pinned = prompt.pin_memory()
     out_pinned = torch.empty((p.batch, p.seq_len), dtype=torch.int32).pin_memory()
@@ -223,18 +223,12 @@ def run_ours(args):
         prof = dec.profile()
         dec.destroy()
 
-    t = torch.tensor([ms, ms2], dtype=torch.float64, device="cuda")
-    tot = torch.tensor([gen, gen2, fwd, launches], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM)
-    ms, ms2 = t.tolist()
-    gen, gen2, fwd, launches = tot.tolist()
+    (ms, ms2), (gen, gen2, fwd, launches) = R.aggregate([ms, ms2], [gen, gen2, fwd, launches], device="cuda")
 
     if rank == 0:
         hbm, tf, which = measured_peaks()
         out = {
-            "metric": METRIC, "value": gen / (ms / 1e3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": R.whole_job_rate(gen, ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if m.dtype == I.DTYPE_BF16 else "f32", "data": "synthetic",
             "config": {"workload": f"{args.config}: LLaDA-8B shape, batch {p.batch}, prompt {p.prompt_len} + gen {p.gen_len}, "
