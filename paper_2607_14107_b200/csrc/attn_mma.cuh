@@ -45,6 +45,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // byte offset of 16-byte chunk `ch` of row `row` in a [rows][128] bf16 tile, XOR-swizzled
 __device__ __forceinline__ uint32_t sw_off(int row, int ch) { return (uint32_t)(row * 256 + ((ch ^ (row & 7)) << 4)); }
 
+// 2^x by the special-function unit (relative error ~2^-22); scores are kept in the log2 domain so that
+// every probability costs one multiply-add and one ex2
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr float LN2 = 0.6931471805599453f;
+
 struct AttnMmaArgs {
     AttnArgs a;
     int rows_per_seq;   // forward rows per sequence (stand-alone: n_rows)
@@ -52,8 +62,7 @@ struct AttnMmaArgs {
 };
 
 __global__ void __launch_bounds__(AT_WARPS * 32) attention_mma_kernel(AttnMmaArgs g) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(7);   // __launch_bounds__
     extern __shared__ uint8_t at_smem_raw[];
     __shared__ float red_m[AT_WARPS][AT_BM], red_l[AT_WARPS][AT_BM], red_kl[AT_WARPS][AT_BM];
     __shared__ float lse_sh[AT_BM];
@@ -313,8 +322,7 @@ constexpr int SP_SLOT_BYTES = AT_BN * AT_DH * 2;     // one K or V tile: 8 KB
 
 template <int NW, int TPW>
 __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(7);   // __launch_bounds__
     extern __shared__ uint8_t at_smem_raw[];
     __shared__ float red_m[NW][AT_BM], red_l[NW][AT_BM], red_kl[NW][AT_BM];
     __shared__ float lse_sh[AT_BM];
@@ -359,7 +367,15 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
     if (n_loads > 0) issue(0);
     if (n_loads > 1) issue(1);
 
-    // ---- row bookkeeping + Q tile (overlaps the first K loads) -------------------------------
+    // ---- row bookkeeping + Q tile (overlap the first K loads; neither waits for the other) ----------
+    // Rows without a valid descriptor may hold stale q values: they only ever affect their own row of
+    // the tile, which is never written.
+    for (int t = threadIdx.x; t < AT_BM * 16; t += blockDim.x) {
+        const int i = t >> 4, ch = t & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (i < n_in_tile) v = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)a.q + (size_t)(row0 + i) * dq + h * AT_DH + ch * 8);
+        *reinterpret_cast<uint4*>(q_s + sw_off(i, ch)) = v;
+    }
     if (threadIdx.x < AT_BM) {
         const int i = threadIdx.x;
         float* prev = nullptr;
@@ -382,13 +398,6 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
         valid_sh[i] = valid;
     }
     __syncthreads();
-    for (int t = threadIdx.x; t < AT_BM * 16; t += blockDim.x) {
-        const int i = t >> 4, ch = t & 15;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (valid_sh[i]) v = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)a.q + (size_t)(row0 + i) * dq + h * AT_DH + ch * 8);
-        *reinterpret_cast<uint4*>(q_s + sw_off(i, ch)) = v;
-    }
-    __syncthreads();
     uint32_t qf[8][4];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
@@ -400,6 +409,7 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
     const int cpair = (lane & 3) * 2;
 
     // ---- scores of my tiles, kept in registers ---------------------------------------------------
+    const float scale2 = a.scale * LOG2E;
     float s[TPW][4][4];
     float m_lo = -INFINITY, m_hi = -INFINITY;
 #pragma unroll
@@ -429,8 +439,8 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const bool ok = t * AT_BN + nt * 8 + cpair + e < a.N;
-                    s[i][nt][e] = ok ? s[i][nt][e] * a.scale : -INFINITY;
-                    s[i][nt][2 + e] = ok ? s[i][nt][2 + e] * a.scale : -INFINITY;
+                    s[i][nt][e] = ok ? s[i][nt][e] * scale2 : -INFINITY;          // log2 domain
+                    s[i][nt][2 + e] = ok ? s[i][nt][2 + e] * scale2 : -INFINITY;
                     m_lo = fmaxf(m_lo, s[i][nt][e]);
                     m_hi = fmaxf(m_hi, s[i][nt][2 + e]);
                 }
@@ -448,7 +458,7 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt)
 #pragma unroll
-                for (int e = 0; e < 2; ++e) { l_lo += expf(s[i][nt][e] - m_lo); l_hi += expf(s[i][nt][2 + e] - m_hi); }
+                for (int e = 0; e < 2; ++e) { l_lo += fast_exp2(s[i][nt][e] - m_lo); l_hi += fast_exp2(s[i][nt][2 + e] - m_hi); }
         }
     }
     l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
@@ -464,8 +474,8 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
         for (int w = 0; w < NW; ++w) mx = fmaxf(mx, red_m[w][i]);
         float sum = 0.f;
         for (int w = 0; w < NW; ++w)
-            if (red_l[w][i] > 0.f) sum += red_l[w][i] * expf(red_m[w][i] - mx);
-        lse_sh[i] = mx + logf(sum);
+            if (red_l[w][i] > 0.f) sum += red_l[w][i] * fast_exp2(red_m[w][i] - mx);
+        lse_sh[i] = mx + log2f(sum);            // log2 domain
     }
     __syncthreads();
     const float lse_lo = lse_sh[r_lo], lse_hi = lse_sh[r_hi];
@@ -509,8 +519,9 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const bool ok = t * AT_BN + nt * 8 + cpair + e < a.N;
-                    lp_lo[nt][e] = s[i][nt][e] - lse_lo; lp_hi[nt][e] = s[i][nt][2 + e] - lse_hi;
-                    const float p_lo = ok ? expf(lp_lo[nt][e]) : 0.f, p_hi = ok ? expf(lp_hi[nt][e]) : 0.f;
+                    const float d_lo = s[i][nt][e] - lse_lo, d_hi = s[i][nt][2 + e] - lse_hi;
+                    const float p_lo = ok ? fast_exp2(d_lo) : 0.f, p_hi = ok ? fast_exp2(d_hi) : 0.f;
+                    lp_lo[nt][e] = d_lo * LN2; lp_hi[nt][e] = d_hi * LN2;       // natural-log probabilities
                     if (ok && a.record_kl) {
                         if (prev_lo) kl_lo += p_lo * (lp_lo[nt][e] - pv_lo[nt][e]);
                         if (prev_hi) kl_hi += p_hi * (lp_hi[nt][e] - pv_hi[nt][e]);

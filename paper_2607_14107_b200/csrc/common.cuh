@@ -33,6 +33,23 @@ template <typename T> __device__ __forceinline__ float round_to(float v) { retur
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// ---- optional kernel timeline (debugging aid) ---------------------------------------------
+// When a trace buffer is installed, block 0 of every kernel records (kernel id, nanosecond time) once
+// its dependencies are resolved; consecutive stamps give each kernel's real cost inside the pipeline.
+__device__ long long* g_trace_buf = nullptr;   // [0] = next slot, then pairs (id, time)
+__device__ __forceinline__ void trace_stamp(int id, int thread = 0) {
+    long long* t = g_trace_buf;
+    if (t && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == thread) {
+        const unsigned long long slot = atomicAdd((unsigned long long*)t, 1ULL);
+        if (slot < 4000) {
+            long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            t[1 + 2 * slot] = id; t[2 + 2 * slot] = now;
+        }
+    }
+}
+#define KERNEL_PROLOGUE(id) do { pdl_trigger(); pdl_wait(); trace_stamp(id); } while (0)
+
 // ---- rows of one forward -----------------------------------------------------------
 // One descriptor per forwarded row.  pos < 0 marks an unused slot.
 struct Row {

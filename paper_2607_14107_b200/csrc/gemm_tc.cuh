@@ -140,6 +140,10 @@ struct SkArgs {
     int done_offset;
     int* status;        // set to 1 on a wait time-out
     long long* trace;   // optional [gridDim.x][8] nanosecond stamps of this launch (null: off)
+    // L2 prefetch of weights that later GEMMs of the stream will read: while this kernel's epilogue and
+    // fix-up run, HBM would otherwise idle.  Entry j: tile-major weight base, that GEMM's unit count and grid,
+    // and the slice [first, first + count) of every CTA's unit range to prefetch (count 0: unused).
+    struct Prefetch { const char* w; long long U; int G; int first, count; } pf[2];
 };
 
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
@@ -230,6 +234,19 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
                 tma_load_2d(dst, &map_a, full0 + 8 * s, kb * BLOCK_K, (tile % g.tiles_t) * BLOCK_T);
             }
+            // all of this CTA's loads are requested: start pulling the next GEMMs' weights into L2
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                if (g.pf[j].count > 0 && cta < g.pf[j].G) {
+                    const long long nb = sk_begin(g.pf[j].U, g.pf[j].G, cta) + g.pf[j].first;
+                    const long long ne = sk_begin(g.pf[j].U, g.pf[j].G, cta + 1);
+                    const int n = (int)max(0LL, min((long long)g.pf[j].count, ne - nb));
+                    for (int i = 0; i < n; ++i) {
+                        const char* src = g.pf[j].w + (size_t)(nb + i) * W_BYTES;
+                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(W_BYTES) : "memory");
+                    }
+                }
+            }
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -268,6 +285,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     } else {
         // ---- epilogue warps: TMEM lane = token, column = feature ------------------------------------
         pdl_wait();
+        trace_stamp(100 + EPI, 64);
         const int q = warp & 3;
         const int t_local = q * 32 + lane;
         const uint32_t taddr0 = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -406,6 +424,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, ncols);
     if (threadIdx.x == 0) SK_STAMP(7);
+    trace_stamp(200 + EPI, 0);
     if (threadIdx.x == 0 && abort_sh) atomicExch(g.status, 1);
 }
 

@@ -10,8 +10,7 @@ namespace ps {
 // Row table of one forward (Algorithm 1: E_b at block entry, J_b plus Omega_b within a block)
 // ---------------------------------------------------------------------------------------
 __global__ void build_rows_kernel(StepDesc sd, Row* rows) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(1);   // build_rows_kernel
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     const int total = sd.batch * sd.rows_per_seq;
     if (i >= total) return;
@@ -44,8 +43,7 @@ template <typename T>
 __global__ void embed_rows_kernel(StepDesc sd, const Row* rows, const int* y, const T* emb, int d,
                                   float* x, float* packet, unsigned char* patch0, int* tok_at_h0,
                                   int* stats) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(2);   // embed_rows_kernel
     const int r = blockIdx.x;
     const Row rw = rows[r];
     if (rw.pos < 0) return;
@@ -72,6 +70,59 @@ __global__ void embed_rows_kernel(StepDesc sd, const Row* rows, const int* y, co
 }
 
 // ---------------------------------------------------------------------------------------
+// One row of RMSNorm + staging, held in registers: every thread owns up to NORM_VPT float4 chunks,
+// so the row is read once (all loads in flight together), reduced, scaled and stored.
+// Requires d % 4 == 0 and d <= 4 * NORM_VPT * blockDim.x.
+// ---------------------------------------------------------------------------------------
+constexpr int NORM_THREADS = 512;
+constexpr int NORM_VPT = 8;
+template <typename T>
+__device__ __forceinline__ void store4(T* p, float a, float b, float c, float d4);
+template <>
+__device__ __forceinline__ void store4<float>(float* p, float a, float b, float c, float d4) {
+    *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d4);
+}
+template <>
+__device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16* p, float a, float b, float c, float d4) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d4);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&lo);
+    u.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = u;
+}
+// src row -> a_out row (normed, times gain); optional copies of the raw row to up to two fp32 destinations
+template <typename T>
+__device__ __forceinline__ void norm_row(const float* __restrict__ src, const float* __restrict__ gain, float eps, int d,
+                                         T* a_out, float* copy0, float* copy1, float* red) {
+    const int n4 = d >> 2;
+    float4 v[NORM_VPT];
+    float ss = 0.f;
+#pragma unroll
+    for (int u = 0; u < NORM_VPT; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        v[u] = c4 < n4 ? __ldcg(reinterpret_cast<const float4*>(src) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < NORM_VPT; ++u) ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
+    ss = block_sum(ss, red);
+    const float inv = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+    for (int u = 0; u < NORM_VPT; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        if (c4 < n4) {
+            const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + c4);
+            store4<T>(a_out + 4 * c4, v[u].x * inv * g.x, v[u].y * inv * g.y, v[u].z * inv * g.z, v[u].w * inv * g.w);
+            if (copy0) reinterpret_cast<float4*>(copy0)[c4] = v[u];
+            if (copy1) reinterpret_cast<float4*>(copy1)[c4] = v[u];
+        }
+    }
+}
+template <typename T>
+__device__ __forceinline__ void zero_row(T* a, int d) {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
+}
+
+// ---------------------------------------------------------------------------------------
 // Patch + RMSNorm + staging of the QKV projection's input rows (Algorithm 1 "Patch")
 //   window rows of a within-block step read the hidden cache (after taking the packet row if
 //   the previous layer selected them); every other row reads the residual stream x.
@@ -80,42 +131,33 @@ template <typename T>
 __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* hc, const float* packet,
                                 const unsigned char* patch, const float* gain, float eps, int d,
                                 T* a_out, unsigned char* kvflag) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(3);   // prep_qkv_kernel
     __shared__ float red[33];
     const int r = blockIdx.x;
     const Row rw = rows[r];
     T* a = a_out + (size_t)r * d;
     if (rw.pos < 0) {
-        for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
+        zero_row<T>(a, d);
         if (threadIdx.x == 0) kvflag[r] = 0;
         return;
     }
     float* xr = x + (size_t)r * d;
-    const float* src = xr;
     bool kv = true;
     if (rw.widx >= 0) {
         const size_t o = (size_t)rw.seq * sd.W_max + rw.widx;
         float* h = hc + o * d;
         if (sd.within) {
+            // window row of a within-block step: the packet row if the previous layer selected it
+            // (then it also replaces the cached hidden row), else the cached hidden row
             const bool patched = patch[o] != 0;
-            const float* u = packet + o * d;
-            for (int c = threadIdx.x; c < d; c += blockDim.x) {
-                const float v = patched ? u[c] : h[c];
-                if (patched) h[c] = v;
-                xr[c] = v;
-            }
             kv = patched;
+            norm_row<T>(patched ? packet + o * d : h, gain, eps, d, a, xr, patched ? h : nullptr, red);
         } else {
-            for (int c = threadIdx.x; c < d; c += blockDim.x) h[c] = xr[c];
+            norm_row<T>(xr, gain, eps, d, a, h, nullptr, red);      // block entry: record the hidden row
         }
-        __syncthreads();
+    } else {
+        norm_row<T>(xr, gain, eps, d, a, nullptr, nullptr, red);
     }
-    float ss = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = src[c]; ss += v * v; }
-    ss = block_sum(ss, red);
-    const float inv = rsqrtf(ss / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(src[c] * inv * gain[c]);
     if (threadIdx.x == 0) kvflag[r] = kv ? 1 : 0;
 }
 
@@ -124,8 +166,7 @@ __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* h
 template <typename T>
 __global__ void prep_rows_kernel(const float* x, const int* list, const int* m_count, const float* gain,
                                  float eps, int d, T* a_out) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(4);   // prep_rows_kernel
     __shared__ float red[33];
     const int i = blockIdx.x;
     T* a = a_out + (size_t)i * d;
@@ -134,12 +175,7 @@ __global__ void prep_rows_kernel(const float* x, const int* list, const int* m_c
         return;
     }
     const int r = list ? list[i] : i;
-    const float* src = x + (size_t)r * d;
-    float ss = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = src[c]; ss += v * v; }
-    ss = block_sum(ss, red);
-    const float inv = rsqrtf(ss / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(src[c] * inv * gain[c]);
+    norm_row<T>(x + (size_t)r * d, gain, eps, d, a, nullptr, nullptr, red);
 }
 
 // LM-head input rows: entry i < n_act reads x[act_rows...]; later entries read packet rows.
@@ -147,8 +183,7 @@ struct HeadSrc { int kind; int index; };  // kind 0: x row `index`; 1: packet ro
 template <typename T>
 __global__ void prep_head_kernel(const float* x, const float* packet, const HeadSrc* src_list,
                                  const int* m_count, const float* gain, float eps, int d, T* a_out) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(5);   // prep_head_kernel
     __shared__ float red[33];
     const int i = blockIdx.x;
     T* a = a_out + (size_t)i * d;
@@ -157,20 +192,14 @@ __global__ void prep_head_kernel(const float* x, const float* packet, const Head
         return;
     }
     const HeadSrc hs = src_list[i];
-    const float* src = (hs.kind ? packet : x) + (size_t)hs.index * d;
-    float ss = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) { const float v = src[c]; ss += v * v; }
-    ss = block_sum(ss, red);
-    const float inv = rsqrtf(ss / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(src[c] * inv * gain[c]);
+    norm_row<T>((hs.kind ? packet : x) + (size_t)hs.index * d, gain, eps, d, a, nullptr, nullptr, red);
 }
 
 // Gather + RMSNorm for the stand-alone refresh kernel: row (s, i) <- h[s][idx[s][i]].
 template <typename T>
 __global__ void prep_refresh_kernel(const T* h, const int* idx, const int* counts, int max_rows, int P,
                                     const float* gain, float eps, int d, T* a_out) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(6);   // prep_refresh_kernel
     __shared__ float red[33];
     const int m = blockIdx.x;
     const int s = m / max_rows, i = m - s * max_rows;
@@ -194,8 +223,7 @@ __global__ void prep_refresh_kernel(const T* h, const int* idx, const int* count
 template <typename T, int EPI>
 __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ Wt,
                                                         int M, int Nout, int K, int w_tiled, EpiArgs e) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(7);   // __launch_bounds__
     __shared__ float As[16][64 + 4];
     __shared__ float Ws[16][64 + 4];
     const int m0 = blockIdx.y * 64, n0 = blockIdx.x * 64;
@@ -264,8 +292,7 @@ struct AttnArgs {
 
 template <typename T>
 __global__ void attention_simt_kernel(AttnArgs a) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(8);   // attention_simt_kernel
     extern __shared__ float sm[];
     const int wpb = blockDim.x >> 5, wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int r = blockIdx.x * wpb + wid, h = blockIdx.y;
@@ -332,8 +359,7 @@ __global__ void attention_simt_kernel(AttnArgs a) {
 // ---------------------------------------------------------------------------------------
 template <typename T>
 __global__ void hidden_delta_kernel(const T* __restrict__ a, const T* __restrict__ b, float* out, int rows, int d) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(9);   // hidden_delta_kernel
     const int wpb = blockDim.x >> 5, wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per = 16 / (int)sizeof(T);
     for (int r = blockIdx.x * wpb + wid; r < rows; r += gridDim.x * wpb) {
@@ -465,13 +491,45 @@ __device__ int select_one(const float* D, int W, int mode, int k, float thresh, 
     return count;
 }
 
+// Small windows (W <= SEL_SMALL_W, the in-step case: W = 3B): rank counting, two barriers.
+// Thread i owns row i; rank = number of candidates ahead of it in (drift descending, index ascending) order.
+constexpr int SEL_SMALL_W = 256;
+__device__ int select_small(const float* D, int W, int mode, int k, float thresh, float floor_,
+                            int* idx_out, unsigned char* flag_out, int* sel_sh /* [SEL_SMALL_W] */) {
+    const int i = threadIdx.x;
+    const float v = i < W ? D[i] : 0.f;
+    const bool cand = i < W && v > floor_;
+    bool sel = false;
+    if (mode == 3) sel = i < W;
+    else if (mode == 2) sel = cand && v > thresh;
+    else if (mode != 4 && k > 0 && cand) {
+        int rank = 0;
+        for (int j = 0; j < W; ++j) {
+            const float dj = D[j];
+            rank += (dj > floor_ && (dj > v || (dj == v && j < i))) ? 1 : 0;
+        }
+        sel = rank < k;
+    }
+    if (i < SEL_SMALL_W) sel_sh[i] = sel ? 1 : 0;
+    __syncthreads();
+    int pos = 0, total = 0;
+    for (int j = 0; j < W; ++j) { const int f = sel_sh[j]; total += f; pos += (j < i) ? f : 0; }
+    if (i < W) {
+        if (flag_out) flag_out[i] = sel ? 1 : 0;
+        if (sel) idx_out[pos] = i;
+    }
+    __syncthreads();
+    return total;
+}
+
 __global__ void __launch_bounds__(SEL_THREADS) select_kernel(const float* drift, int W, int mode, int k,
                                                              float thresh, float floor_, int* idx, int* count) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(7);   // __launch_bounds__
     __shared__ SelSmem s;
     const int b = blockIdx.x;
-    const int c = select_one(drift + (size_t)b * W, W, mode, k, thresh, floor_, idx + (size_t)b * W, nullptr, s);
+    __shared__ int sel_sh[SEL_SMALL_W];
+    const int c = W <= SEL_SMALL_W ? select_small(drift + (size_t)b * W, W, mode, k, thresh, floor_, idx + (size_t)b * W, nullptr, sel_sh)
+                                   : select_one(drift + (size_t)b * W, W, mode, k, thresh, floor_, idx + (size_t)b * W, nullptr, s);
     if (threadIdx.x == 0) count[b] = c;
 }
 
@@ -490,10 +548,10 @@ struct StepSelArgs {
 };
 
 __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, StepSelArgs a) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(7);   // __launch_bounds__
     __shared__ SelSmem s;
     __shared__ float dsh[SEL_MAX_W > 1024 ? 1024 : SEL_MAX_W];
+    __shared__ int sel_sh[SEL_SMALL_W];
     __shared__ int base;
     const int t = threadIdx.x;
     const int nb = sd.batch * sd.B;
@@ -526,7 +584,8 @@ __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, S
             cnt = fc;
             __syncthreads();
         } else {
-            cnt = select_one(dsh, sd.W, a.mode, a.k, a.thresh, a.floor_, idx, fl, s);
+            cnt = sd.W <= SEL_SMALL_W ? select_small(dsh, sd.W, a.mode, a.k, a.thresh, a.floor_, idx, fl, sel_sh)
+                                      : select_one(dsh, sd.W, a.mode, a.k, a.thresh, a.floor_, idx, fl, s);
         }
         const int b0 = base;
         for (int i = t; i < cnt; i += blockDim.x) a.list[b0 + i] = sq * sd.rows_per_seq + sd.B + idx[i];
@@ -544,8 +603,7 @@ __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, S
 __global__ void build_head_list_kernel(StepDesc sd, const int* y, int mask_id, const int* sel_idx,
                                        const int* sel_cnt, int use_suffix, int act_row0_stride,
                                        HeadSrc* list, int* count, int* suf_seq, int* suf_w) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(10);   // build_head_list_kernel
     // act_row0_stride: forward row of active j in sequence s = s*rows_per_seq + (act offset) + j
     const int t = threadIdx.x;
     const int nb = sd.batch * sd.B;
@@ -584,8 +642,7 @@ struct ConfPart { float mx_all; float sum; float mx_ex; int arg_ex; };
 
 __global__ void conf_partial_kernel(const float* logits, const int* m_count, int rows, int V, int mask_id,
                                     int chunks, ConfPart* part) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(11);   // conf_partial_kernel
     __shared__ float red[33];
     __shared__ float bv[32];
     __shared__ int bi[32];
@@ -625,8 +682,7 @@ __global__ void conf_partial_kernel(const float* logits, const int* m_count, int
 
 __global__ void conf_final_kernel(const ConfPart* part, const int* m_count, int rows, int chunks,
                                   int* yhat, float* conf) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(12);   // conf_final_kernel
     const int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r >= rows || (m_count && r >= *m_count)) return;
     const ConfPart* p = part + (size_t)r * chunks;
@@ -664,8 +720,7 @@ struct CommitArgs {
 };
 
 __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(13);   // commit_kernel
     __shared__ float s_conf[256];
     __shared__ unsigned char s_masked[256], s_flag[256];
     __shared__ int cnt[8];
@@ -788,8 +843,7 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
 
 // Last-layer drift of the active rows (Algorithm 1, delta): mean over heads of the per-head KL.
 __global__ void delta_kernel(StepDesc sd, const float* kl, int act_row_off, int n_heads, float* delta) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(14);   // delta_kernel
     const int s = blockIdx.x, j = threadIdx.x;
     if (j >= sd.B) return;
     float dl = 0.f;
@@ -804,8 +858,7 @@ __global__ void delta_kernel(StepDesc sd, const float* kl, int act_row_off, int 
 
 // gather rows of x into a keep buffer: dst[s][j][:] = x[row(s, j)][:]
 __global__ void keep_hidden_kernel(StepDesc sd, const float* x, int act_row_off, int d, float* dst) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(15);   // keep_hidden_kernel
     const int i = blockIdx.x;
     const int s = i / sd.B, j = i - s * sd.B;
     const float* src = x + (size_t)(s * sd.rows_per_seq + act_row_off + j) * d;
@@ -815,8 +868,7 @@ __global__ void keep_hidden_kernel(StepDesc sd, const float* x, int act_row_off,
 
 // y = [prompt ; MASK ...] from a prompt that already lives on the device (ids clamped to the vocabulary)
 __global__ void init_tokens_kernel(int* y, const int* prompt, int batch, int prompt_len, int N, int mask_id, int vocab) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(16);   // init_tokens_kernel
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= batch * N) return;
     const int s = i / N, pos = i - s * N;
@@ -831,8 +883,7 @@ __global__ void init_tokens_kernel(int* y, const int* prompt, int batch, int pro
 
 // rotary table: tab[pos][i] = (cos, sin)(pos * theta^(-2i/dh)), computed in double precision
 __global__ void rope_table_kernel(float2* tab, int N, int half, double theta) {
-    pdl_trigger();
-    pdl_wait();
+    KERNEL_PROLOGUE(17);   // rope_table_kernel
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N * half) return;
     const int pos = i / half, k = i - pos * half;

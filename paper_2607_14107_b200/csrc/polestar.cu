@@ -101,9 +101,24 @@ static int launch_gemm_simt(const void* A, const void* W, int M, int N_out, int 
     return POLESTAR_OK;
 }
 
+// Weights a later GEMM of the same forward will stream (for L2 prefetch during this GEMM's tail).
+struct NextW { const void* w = nullptr; int N_out = 0, K = 0, M = 0, first = 0, count = 0; };
+
+// stream-K grid of a GEMM with M rows: G CTAs over U units
+static void sk_grid(int M, int N_out, int K, long long* U, long long* G) {
+    const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + tc::BLOCK_T - 1) / tc::BLOCK_T;
+    const int sms = g_sm_count > 0 ? g_sm_count : 148;
+    *U = (long long)tiles_f * tiles_t * (K / 64);
+    long long g = std::min<long long>((long long)sms, *U);
+    const long long tiles = (long long)tiles_f * tiles_t;
+    const long long mult = (g / tiles) * tiles;
+    if (mult > 0 && mult * 100 >= (long long)sms * env_int("POLESTAR_GEMM_ALIGN_PCT", 85)) g = mult;
+    *G = g;
+}
+
 template <int EPI>
 static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a_rows_alloc, const void* W, int M,
-                          int N_out, int K, const EpiArgs& e, cudaStream_t st) {
+                          int N_out, int K, const EpiArgs& e, cudaStream_t st, const NextW* next = nullptr) {
     if (M <= 0) return POLESTAR_OK;
     (void)a_rows_alloc;
     // weights: tile-major [chunks * 256][64]; activations: exactly M rows, so that the rows of a token tile
@@ -114,22 +129,27 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + tc::BLOCK_T - 1) / tc::BLOCK_T;
     const int kb = K / 64;
     const int sms = g_sm_count > 0 ? g_sm_count : 148;
-    const long long U = (long long)tiles_f * tiles_t * kb;
-    long long G = std::min<long long>((long long)sms, U);
-    // When a multiple of the tile count fits on >= 85 % of the SMs, take it: CTA ranges then never cross a
-    // tile boundary, so every CTA has one segment (one fix-up instead of two, or none at all).
-    {
-        const long long tiles = (long long)tiles_f * tiles_t;
-        const long long mult = (G / tiles) * tiles;
-        if (mult > 0 && mult * 100 >= (long long)sms * env_int("POLESTAR_GEMM_ALIGN_PCT", 85)) G = mult;
-    }
-    while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 > ws.partial_bytes)) --G;
+    // When a multiple of the tile count fits on >= 85 % of the SMs, the grid takes it: CTA ranges then never
+    // cross a tile boundary, so every CTA has one segment (one fix-up instead of two, or none at all).
+    long long U, G;
+    sk_grid(M, N_out, K, &U, &G);
+    (void)sms; (void)kb;
+    while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
     if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
     tc::SkArgs g;
     g.M = M; g.N_out = N_out; g.K = K; g.tiles_f = tiles_f; g.tiles_t = tiles_t;
     g.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", 4)));
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
     // debug: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
+    memset(g.pf, 0, sizeof(g.pf));
+    for (int j = 0; next && j < 2; ++j) {
+        if (!next[j].w || next[j].count <= 0 || next[j].M > tc::BLOCK_T) continue;      // only weight-bound successors
+        if (next[j].N_out % tc::BLOCK_F || next[j].K % 64) continue;
+        long long nU, nG;
+        sk_grid(next[j].M, next[j].N_out, next[j].K, &nU, &nG);
+        g.pf[j].w = (const char*)next[j].w; g.pf[j].U = nU; g.pf[j].G = (int)nG;
+        g.pf[j].first = next[j].first; g.pf[j].count = next[j].count;
+    }
     g.trace = (env_int("POLESTAR_GEMM_TRACE", -1) == EPI) ? (long long*)((char*)ws.partial + ws.partial_bytes - 16384) : nullptr;
     const size_t smem = (size_t)g.stages * tc::STAGE_BYTES + 1024;
     auto kern = tc::gemm_sk_kernel<__nv_bfloat16, EPI>;
@@ -169,7 +189,7 @@ struct Buffers {
 
 static const int CONF_CHUNKS = 32;
 static const int FORCED_COMMIT_MAX = 512;
-static const size_t GEMM_PARTIAL_BYTES = ((size_t)40 << 20) + 16384;   // 2 slots x 148 CTAs x 128 x 256 fp32
+static const size_t GEMM_PARTIAL_BYTES = ((size_t)40 << 20) + 16384 + 65536;   // 2 slots x 148 CTAs x 128 x 256 fp32
 static const int GEMM_COUNTERS = 1 << 17;     // arrivals + finished shares for up to 65536 output tiles
 
 struct polestar_ctx {
@@ -239,6 +259,7 @@ static bool valid_cfg(const polestar_model* m, const polestar_params* p) {
     if (m->dtype != POLESTAR_F32 && m->dtype != POLESTAR_BF16) return false;
     if (m->mask_id < 0 || m->mask_id >= m->vocab || m->eos_id < 0 || m->eos_id >= m->vocab) return false;
     if (m->d_model % 8 || (m->n_heads * m->head_dim) % 8 || m->d_ffn % 8) return false;
+    if (m->d_model > 4 * NORM_VPT * NORM_THREADS) return false;
     if (p->batch <= 0 || p->batch > POLESTAR_MAX_BATCH) return false;
     if (p->prompt_len < 0 || p->gen_len <= 0 || p->block <= 0 || p->block > 256) return false;
     if (p->gen_len % p->block) return false;
@@ -365,9 +386,9 @@ struct Path {
 
     template <int EPI>
     static int gemm(polestar_ctx* c, const void* A, int a_rows_alloc, const void* W, int M, int N_out, int K,
-                    const EpiArgs& e) {
+                    const EpiArgs& e, const NextW* next = nullptr) {
         if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 256 == 0)
-            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st);
+            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st, next);
         return launch_gemm_simt<T, EPI>(A, W, M, N_out, K, e, c->st);
     }
 
@@ -402,6 +423,10 @@ struct Path {
         int rc;
 
         const double esd = (double)es;
+        // 32 KB weight units per CTA that a GEMM asks L2 to fetch for its successors while its own tail runs.
+        // Off by default: measured on B200 it slows the decode by 5-12 % (the prefetch burst queues in front
+        // of the latency-critical partial-tile exchange of the GEMM's own tail).
+        const int pf_units = env_int("POLESTAR_PREFETCH_UNITS", 0), pf_units2 = env_int("POLESTAR_PREFETCH_UNITS2", 0);
         const double Mlive = sparse ? (double)bs * (B + std::min(sd.W, (int)(p.select_mode == POLESTAR_SELECT_TOPK_FRAC
                                                        ? floorf(p.select_frac * (float)sd.W + 0.5f)
                                                        : (p.select_mode == POLESTAR_SELECT_TOPK_COUNT ? p.select_k : sd.W))))
@@ -427,7 +452,7 @@ struct Path {
             }
             {
                 Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
-                CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(256), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
+                CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
                                                      c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag));
                 CK(cudaGetLastError());
             }
@@ -439,7 +464,10 @@ struct Path {
                 e.rows = b.rows; e.kvflag = b.kvflag; e.rope = b.rope; e.q_out = b.q_buf; e.kc = kc; e.vc = vc;
                 e.N_seq = N; e.n_heads = m.n_heads; e.n_kv = m.n_kv_heads; e.head_dim = m.head_dim; e.W_max = Wm;
                 e.within = within; e.ld_out = dq;
-                if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->M_max, c->wqkv[l], M, dq + 2 * dkv, d, e))) return rc;
+                NextW nx[2];
+                nx[0].w = c->wo[l]; nx[0].N_out = d; nx[0].K = dq; nx[0].M = M; nx[0].count = pf_units;
+                nx[1].w = c->wgu[l]; nx[1].N_out = 2 * F; nx[1].K = d; nx[1].M = M; nx[1].count = pf_units2;
+                if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->M_max, c->wqkv[l], M, dq + 2 * dkv, d, e, nx))) return rc;
             }
             {
                 const bool rec_w = sparse || !within;
@@ -478,25 +506,33 @@ struct Path {
                 Scope sc(c, POLESTAR_PROF_GEMM_O, (double)d * dq * esd + (double)M * dq * esd + 2.0 * M * d * 4, 2.0 * M * d * (double)dq, 1);
                 memset(&e, 0, sizeof(e));
                 e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
-                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e))) return rc;
+                NextW nx[2];
+                nx[0].w = c->wgu[l]; nx[0].N_out = 2 * F; nx[0].K = d; nx[0].M = M; nx[0].first = pf_units2; nx[0].count = pf_units;
+                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e, nx))) return rc;
             }
             {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
-                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(256), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
+                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
                 CK(cudaGetLastError());
             }
             {
                 Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, (2.0 * F * d + Mlive * d + Mlive * F) * esd, 4.0 * Mlive * F * (double)d, 1);
                 memset(&e, 0, sizeof(e));
                 e.out_t = b.g_buf; e.ld_out = F; e.m_count = m2_count;
-                if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->M_max, c->wgu[l], M, 2 * F, d, e))) return rc;
+                NextW nx[2];
+                nx[0].w = c->wd[l]; nx[0].N_out = d; nx[0].K = F; nx[0].M = M; nx[0].count = pf_units;
+                if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->M_max, c->wgu[l], M, 2 * F, d, e, nx))) return rc;
             }
             {
                 Scope sc(c, POLESTAR_PROF_GEMM_DOWN, ((double)F * d + Mlive * F) * esd + 2.0 * Mlive * d * 4, 2.0 * Mlive * F * (double)d, 1);
                 memset(&e, 0, sizeof(e));
                 e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = b.x1; e.out_f32 = b.x; e.packet = b.packet;
                 e.W_max = Wm; e.within = within; e.ld_out = d;
-                if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e))) return rc;
+                NextW nx[2];
+                if (l + 1 < L) { nx[0].w = c->wqkv[l + 1]; nx[0].N_out = dq + 2 * dkv; nx[0].K = d; nx[0].M = M; }
+                else { nx[0].w = c->lm_head; nx[0].N_out = m.vocab; nx[0].K = d; nx[0].M = bs * B; }
+                nx[0].count = pf_units;
+                if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e, nx))) return rc;
             }
         }
         if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
@@ -512,7 +548,7 @@ struct Path {
             CK(launch_k(build_head_list_kernel, dim3(1), dim3(256), 0, st, sd, b.y, m.mask_id, b.sel_idx + (size_t)(L - 1) * bs * Wm,
                                                       b.sel_cnt + (size_t)(L - 1) * bs, use_suffix, 0, b.head_list,
                                                       b.head_count, b.suf_seq, b.suf_w));
-            CK(launch_k(prep_head_kernel<T>, dim3(Mh), dim3(256), 0, st, b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
+            CK(launch_k(prep_head_kernel<T>, dim3(Mh), dim3(NORM_THREADS), 0, st, b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
                                                    (T*)b.a_head));
             CK(cudaGetLastError());
         }
@@ -746,6 +782,11 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     const int half = m->head_dim / 2;
     rope_table_kernel<<<(c->N * half + 255) / 256, 256, 0, c->st>>>(c->b.rope, c->N, half, (double)m->rope_theta);
     if (cudaStreamSynchronize(c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
+    if (env_int("POLESTAR_KERNEL_TRACE", 0)) {
+        long long* tb = (long long*)((char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384 - 65536);
+        cudaMemsetAsync(tb, 0, 65536, c->st);
+        cudaMemcpyToSymbolAsync(g_trace_buf, &tb, sizeof(tb), 0, cudaMemcpyHostToDevice, c->st);
+    }
     rc = polestar_step(c, nullptr);
     if (rc) return fail(rc);
     *out = c;
@@ -801,6 +842,7 @@ extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void*
         case POLESTAR_READ_COMMIT: src = c->b.commit_flags; sz = bs * B * 4; break;
         case POLESTAR_READ_PPREV: src = c->b.pprev + layer * bs * Wm * m.n_heads * N; sz = bs * Wm * m.n_heads * N * 4; break;
         case POLESTAR_READ_SUFFIX: src = c->b.suffix_flags; sz = bs * Wm * 4; break;
+        case 98: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384 - 65536; sz = 65536; break;   // debug: kernel timeline
         case 99: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384; sz = 16384; break;   // debug: GEMM time stamps
         default: return POLESTAR_E_INVAL;
     }

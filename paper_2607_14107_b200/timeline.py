@@ -1,0 +1,61 @@
+"""Kernel timeline of real forwards (debugging / profiling aid).
+
+With POLESTAR_KERNEL_TRACE=1 the library records, for every kernel of a forward, the time at which
+block 0 had its dependencies resolved (and, for the GEMM, when its CTA 0 finished).  Consecutive
+stamps give what each kernel really costs inside the pipeline, launch gaps included -- something
+neither CUDA events (too coarse) nor ncu (serialised, idle clocks) show.
+
+    python -m paper_2607_14107_b200.timeline [--config c2] [--forwards 6]
+"""
+from __future__ import annotations
+
+import argparse
+import collections
+import ctypes as C
+import os
+
+import numpy as np
+
+NAMES = {1: "build_rows", 2: "embed", 3: "prep_qkv", 4: "prep_rows", 5: "prep_head", 7: "attention/select",
+         10: "head_list", 11: "conf_partial", 12: "conf_final", 13: "commit", 14: "delta", 15: "keep_hidden",
+         100: "gemm_qkv", 101: "gemm_o", 102: "gemm_gate_up", 103: "gemm_down", 104: "gemm_lm_head",
+         200: "gemm_qkv:cta0_done", 201: "gemm_o:cta0_done", 202: "gemm_gate_up:cta0_done",
+         203: "gemm_down:cta0_done", 204: "gemm_lm_head:cta0_done"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", default="c2")
+    ap.add_argument("--forwards", type=int, default=6)
+    a = ap.parse_args()
+    os.environ["POLESTAR_KERNEL_TRACE"] = "1"
+    import torch
+    from . import binding as Bd, inputs as I
+    m, p = I.config(a.config)
+    dec = Bd.Polestar(m, Bd.make_packed_weights(m), p, I.make_prompt(m, p).numpy())
+    dec.commit()
+    for _ in range(a.forwards):
+        dec.step()
+        dec.commit()
+    torch.cuda.synchronize()
+    out = np.zeros(8192, np.int64)
+    Bd._check(Bd.load().polestar_read(dec.ctx, 98, 0, out.ctypes.data_as(C.c_void_p), 65536))
+    n = min(int(out[0]), 4000)
+    ids, ts = out[1:1 + 2 * n:2], out[2:2 + 2 * n:2].astype(np.float64) / 1000.0
+    order = np.argsort(ts, kind="stable")
+    ids, ts = ids[order], ts[order]
+    starts = [i for i in range(n) if ids[i] == 1]
+    for f in range(1, len(starts) - 1):
+        lo, hi = starts[f], starts[f + 1]
+        agg = collections.OrderedDict()
+        for i in range(lo, hi):
+            x = agg.setdefault(NAMES.get(int(ids[i]), str(int(ids[i]))), [0, 0.0])
+            x[0] += 1
+            x[1] += ts[i + 1] - ts[i]
+        print(f"forward {f}: {ts[hi] - ts[lo]:.0f} us, {hi - lo} stamps")
+        for k, v in agg.items():
+            print(f"    {k:24s} x{v[0]:3d}  avg {v[1] / v[0]:7.1f} us  total {v[1]:8.0f} us")
+
+
+if __name__ == "__main__":
+    main()
