@@ -238,9 +238,20 @@ __global__ void __launch_bounds__(AT_WARPS * 32) attention_mma_kernel(AttnMmaArg
         if (it + 1 < my_tiles) { load_tile(t + AT_WARPS, (it + 1) & 1, true); cp_async_wait<1>(); }
         else cp_async_wait<0>();
         __syncwarp();
+        // stored rows of this tile first: all loads are issued together, before any of the stores below
+        float pv_lo[4][2], pv_hi[4][2];
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int key = t * AT_BN + nt * 8 + cpair + e;
+                pv_lo[nt][e] = (a.record_kl && prev_lo && key < a.N) ? prev_lo[key] : 0.f;
+                pv_hi[nt][e] = (a.record_kl && prev_hi && key < a.N) ? prev_hi[key] : 0.f;
+            }
         float s[4][4];
         scores(it & 1, s);
         uint32_t pf[2][4];
+        float lp_lo[4][2], lp_hi[4][2];
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
             float p[4];
@@ -248,15 +259,25 @@ __global__ void __launch_bounds__(AT_WARPS * 32) attention_mma_kernel(AttnMmaArg
             for (int e = 0; e < 2; ++e) {
                 const int key = t * AT_BN + nt * 8 + cpair + e;
                 const bool ok = key < a.N;
-                const float lp_lo = s[nt][e] * a.scale - lse_lo, lp_hi = s[nt][2 + e] * a.scale - lse_hi;
-                const float p_lo = ok ? expf(lp_lo) : 0.f, p_hi = ok ? expf(lp_hi) : 0.f;
-                if (ok && prev_lo) { if (a.record_kl) kl_lo += p_lo * (lp_lo - prev_lo[key]); prev_lo[key] = lp_lo; }
-                if (ok && prev_hi) { if (a.record_kl) kl_hi += p_hi * (lp_hi - prev_hi[key]); prev_hi[key] = lp_hi; }
+                lp_lo[nt][e] = s[nt][e] * a.scale - lse_lo; lp_hi[nt][e] = s[nt][2 + e] * a.scale - lse_hi;
+                const float p_lo = ok ? fast_exp2(lp_lo[nt][e] * LOG2E) : 0.f, p_hi = ok ? fast_exp2(lp_hi[nt][e] * LOG2E) : 0.f;
+                if (ok && a.record_kl) {
+                    if (prev_lo) kl_lo += p_lo * (lp_lo[nt][e] - pv_lo[nt][e]);
+                    if (prev_hi) kl_hi += p_hi * (lp_hi[nt][e] - pv_hi[nt][e]);
+                }
                 p[e] = p_lo; p[2 + e] = p_hi;
             }
             pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
             pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
         }
+#pragma unroll
+        for (int nt = 0; nt < 4; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int key = t * AT_BN + nt * 8 + cpair + e;
+                if (prev_lo && key < a.N) prev_lo[key] = lp_lo[nt][e];
+                if (prev_hi && key < a.N) prev_hi[key] = lp_hi[nt][e];
+            }
         if (a.out) {
             const uint32_t vb = st_u32 + (it & 1) * AT_STAGE_BYTES + AT_BN * AT_DH * 2;
 #pragma unroll

@@ -131,6 +131,22 @@ __host__ __device__ inline uint32_t instr_desc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+constexpr int PSTRIDE = BLOCK_F + 4;     // floats per token row of a partial tile in shared memory (conflict-free float4 rows)
+
 struct SkArgs {
     int M, N_out, K, stages;
     int tiles_f, tiles_t;
@@ -139,6 +155,8 @@ struct SkArgs {
                         // launch, zero again after
     int done_offset;
     int* status;        // set to 1 on a wait time-out
+    int cluster_n;      // > 0: launched in clusters of cluster_n CTAs = the contributors of one output tile;
+                        // partial tiles are then exchanged through distributed shared memory, not global memory
     long long* trace;   // optional [gridDim.x][8] nanosecond stamps of this launch (null: off)
     // L2 prefetch of weights that later GEMMs of the stream will read: while this kernel's epilogue and
     // fix-up run, HBM would otherwise idle.  Entry j: tile-major weight base, that GEMM's unit count and grid,
@@ -323,6 +341,24 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
+            } else if (g.cluster_n > 0) {
+                // cluster path: the partial tile goes to this CTA's shared memory (the operand ring is idle once
+                // the last MMA has completed); the cluster adds the tiles up after the barrier further down
+                float* prow = reinterpret_cast<float*>(smem) + (size_t)t_local * PSTRIDE;
+                if (warp_live) {
+                    for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
+                        float v[16];
+                        tmem_ld16(taddr + (uint32_t)c0, v);
+                        if (live) {
+#pragma unroll
+                            for (int c = 0; c < 16; c += 4)
+                                *reinterpret_cast<float4*>(prow + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
             } else {
                 // partial segment: publish it now, reduce later (pass 2), so that publishing never
                 // waits on another CTA
@@ -418,6 +454,54 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (prev == nseg - 1) { g.tile_counter[tile] = 0; g.tile_counter[g.done_offset + tile] = 0; }
             }
         }
+    }
+
+    if (g.cluster_n > 0) {
+        // Every CTA of the cluster worked on the same output tile (consecutive k ranges, rank = k order).  All
+        // threads meet at the cluster barrier; then each CTA adds up its share of the tile, reading the other
+        // CTAs' partial tiles through distributed shared memory in rank order (deterministic), and runs the epilogue.
+        cluster_sync_all();
+        if (warp >= 2 && !abort_sh) {
+            const int tile = (int)(u_begin / kb_total);
+            const int tile_f = tile / g.tiles_t, tile_t = tile % g.tiles_t;
+            const int n0 = tile_f * BLOCK_F;
+            const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
+            const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
+            const int n_items = n_live * (BLOCK_F / 16);
+            const int rank = cta % g.cluster_n;
+            for (int item = rank * 128 + ((int)threadIdx.x - 64); item < n_items; item += g.cluster_n * 128) {
+                const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16;
+                const uint32_t local = smem_base + (uint32_t)((tl * PSTRIDE + c0) * 4);
+                float acc[16];
+#pragma unroll
+                for (int x = 0; x < 16; ++x) acc[x] = 0.f;
+                for (int r0 = 0; r0 < g.cluster_n; r0 += 4) {
+                    float4 tv[4][4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (r0 + j < g.cluster_n) {
+                            const uint32_t ra = dsmem_addr(local, (uint32_t)(r0 + j));
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) tv[j][x] = ld_dsmem_f4(ra + 16 * x);
+                        } else {
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) tv[j][x] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) {
+                            acc[4 * x] += tv[j][x].x; acc[4 * x + 1] += tv[j][x].y;
+                            acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
+                        }
+                }
+                const int mm = tile_t * BLOCK_T + tl;
+#pragma unroll
+                for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, mm, n0 + c0 + c, acc[c], acc[c + 1]);
+            }
+        }
+        cluster_sync_all();       // nobody leaves while its partial tile may still be read
     }
 
     tc_fence_before();

@@ -112,7 +112,14 @@ static void sk_grid(int M, int N_out, int K, long long* U, long long* G) {
     long long g = std::min<long long>((long long)sms, *U);
     const long long tiles = (long long)tiles_f * tiles_t;
     const long long mult = (g / tiles) * tiles;
-    if (mult > 0 && mult * 100 >= (long long)sms * env_int("POLESTAR_GEMM_ALIGN_PCT", 85)) g = mult;
+    const int pct = env_int("POLESTAR_GEMM_ALIGN_PCT", 85);
+    if (mult > 0 && mult * 100 >= (long long)sms * pct) g = mult;
+    else if (tiles % 2 == 0 && env_int("POLESTAR_GEMM_HALF_ALIGN", 1)) {
+        // next best: a multiple of half the tile count, so that CTA ranges cross a tile boundary only in every
+        // third (fifth, ...) CTA instead of in nearly all of them
+        const long long half = tiles / 2, mult2 = (g / half) * half;
+        if (mult2 > 0 && mult2 * 100 >= (long long)sms * pct) g = mult2;
+    }
     *G = g;
 }
 
@@ -133,13 +140,29 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     // cross a tile boundary, so every CTA has one segment (one fix-up instead of two, or none at all).
     long long U, G;
     sk_grid(M, N_out, K, &U, &G);
-    (void)sms; (void)kb;
+    (void)kb;
+    // Cluster path: when the output tiles can be split over n <= 8 CTAs each with n * tiles covering >= 85 % of
+    // the SMs, the n contributors of a tile form a thread-block cluster and add their partial tiles up through
+    // distributed shared memory (no global round trips, no waiting on a counter).
+    int cluster_n = 0;
+    {
+        const long long tiles = (long long)tiles_f * tiles_t;
+        const long long n = std::min<long long>(8, sms / tiles);
+        // Off by default: on B200 at most 45 clusters of 3 / 15 clusters of 8 CTAs with this much shared memory
+        // are co-resident (GPC sizes), fewer than the 48 / 16 the 8B shapes need, so the grid ran in two waves.
+        if (env_int("POLESTAR_GEMM_CLUSTER", 0) && n >= 2 && tiles * n * 100 >= (long long)sms * 85 &&
+            (size_t)tc::BLOCK_T * tc::PSTRIDE * 4 <= (size_t)4 * tc::STAGE_BYTES) {
+            cluster_n = (int)n;
+            G = tiles * n;
+        }
+    }
     while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
     if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
     tc::SkArgs g;
     g.M = M; g.N_out = N_out; g.K = K; g.tiles_f = tiles_f; g.tiles_t = tiles_t;
     g.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", 4)));
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
+    g.cluster_n = cluster_n;
     // debug: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
     memset(g.pf, 0, sizeof(g.pf));
     for (int j = 0; next && j < 2; ++j) {
@@ -158,7 +181,8 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
         CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr = true;
     }
-    CK(launch_k(kern, dim3((unsigned)G), dim3(tc::THREADS), smem, st, *mw, *ma, g, e));
+    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e));
+    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::THREADS), smem, st, *mw, *ma, g, e));
     return POLESTAR_OK;
 }
 
