@@ -624,6 +624,230 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Many-rows variant (block-entry forwards, long sequences, batches): one CTA = 64 query rows of one
+// head, 4 warps x 16 rows; every 64-key K/V tile is staged once per CTA in shared memory (cp.async,
+// two stages) and used by all four warps, so K/V are re-read once per 64 rows instead of once per
+// 16.  Each warp keeps its rows' running max / sum (pass 1) and output accumulator (pass 2) in
+// registers; no cross-warp reduction is needed.
+// ------------------------------------------------------------------------------------------
+constexpr int BG_BM = 64, BG_BN = 64, BG_WARPS = 4;
+constexpr int BG_TILE_BYTES = BG_BN * AT_DH * 2;                  // 16 KB
+constexpr int BG_SMEM = BG_BM * AT_DH * 2 + 2 * 2 * BG_TILE_BYTES + 1024;
+
+__global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArgs g) {
+    KERNEL_PROLOGUE(7);
+    extern __shared__ uint8_t at_smem_raw[];
+    __shared__ float* prev_sh[BG_BM];
+    __shared__ int valid_sh[BG_BM];
+    const AttnArgs& a = g.a;
+    uint8_t* smem = (uint8_t*)(((uintptr_t)at_smem_raw + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int seq = blockIdx.x / g.tiles_per_seq, tile = blockIdx.x - seq * g.tiles_per_seq;   // 64-row tiles here
+    const int h = blockIdx.y;
+    const int g_kv = (h * a.n_kv) / a.n_heads;
+    const int dq = a.n_heads * AT_DH, dkv = a.n_kv * AT_DH;
+    const int row0 = seq * g.rows_per_seq + tile * BG_BM;
+    const int n_in_tile = min(BG_BM, g.rows_per_seq - tile * BG_BM);
+    uint8_t* q_s = smem;
+    const uint32_t q_u32 = (uint32_t)__cvta_generic_to_shared(q_s);
+    const uint32_t st_u32 = q_u32 + BG_BM * AT_DH * 2;
+    const int kv_seq = a.rows ? seq : 0;
+    const __nv_bfloat16* Kg = (const __nv_bfloat16*)a.kc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
+    const __nv_bfloat16* Vg = (const __nv_bfloat16*)a.vc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
+    const int n_tiles = (a.N + BG_BN - 1) / BG_BN;
+
+    auto load_tile = [&](int t, int stage, bool with_v) {
+        const int key0 = t * BG_BN;
+        const uint32_t kb = st_u32 + stage * 2 * BG_TILE_BYTES, vb = kb + BG_TILE_BYTES;
+        for (int c = threadIdx.x; c < BG_BN * 16; c += BG_WARPS * 32) {
+            const int r = c >> 4, ch = c & 15;
+            const int key = key0 + r;
+            const bool ok = key < a.N;
+            const size_t off = (size_t)(ok ? key : 0) * dkv + ch * 8;
+            cp_async16(kb + sw_off(r, ch), Kg + off, ok);
+            if (with_v) cp_async16(vb + sw_off(r, ch), Vg + off, ok);
+        }
+        cp_async_commit();
+    };
+    load_tile(0, 0, false);
+    for (int t = threadIdx.x; t < BG_BM * 16; t += blockDim.x) {
+        const int i = t >> 4, ch = t & 15;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (i < n_in_tile) v = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)a.q + (size_t)(row0 + i) * dq + h * AT_DH + ch * 8);
+        *reinterpret_cast<uint4*>(q_s + sw_off(i, ch)) = v;
+    }
+    if (threadIdx.x < BG_BM) {
+        const int i = threadIdx.x;
+        float* prev = nullptr;
+        int valid = 0;
+        if (i < n_in_tile) {
+            const int r = row0 + i;
+            if (a.rows) {
+                const Row rw = a.rows[r];
+                if (rw.pos >= 0) {
+                    valid = 1;
+                    if (rw.widx >= 0 && a.pprev) prev = a.pprev + (((size_t)rw.seq * a.W_max + rw.widx) * a.n_heads + h) * a.N;
+                    else if (rw.aidx >= 0 && a.aprev) prev = a.aprev + (((size_t)rw.seq * a.B + rw.aidx) * a.n_heads + h) * a.N;
+                }
+            } else {
+                valid = 1;
+                if (a.pprev) prev = a.pprev + ((size_t)r * a.n_heads + h) * a.N;
+            }
+        }
+        prev_sh[i] = prev;
+        valid_sh[i] = valid;
+    }
+    __syncthreads();
+    uint32_t qf[8][4];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const int i = lane >> 3, r = lane & 7;
+        ldsm_x4(q_u32 + sw_off(warp * 16 + (i & 1) * 8 + r, 2 * k + (i >> 1)), qf[k][0], qf[k][1], qf[k][2], qf[k][3]);
+    }
+    const int r_lo = warp * 16 + (lane >> 2), r_hi = r_lo + 8;
+    const int cpair = (lane & 3) * 2;
+    const float scale2 = a.scale * LOG2E;
+
+    auto scores = [&](int stage, float (*s)[4]) {     // s[8][4]: 16 rows x 64 keys per warp, log2 domain, masked
+        const uint32_t kb = st_u32 + stage * 2 * BG_TILE_BYTES;
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                const int i = lane >> 3, r = lane & 7;
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(kb + sw_off((2 * np + (i >> 1)) * 8 + r, 2 * k + (i & 1)), b0, b1, b2, b3);
+                mma_bf16(s[2 * np], qf[k], b0, b1);
+                mma_bf16(s[2 * np + 1], qf[k], b2, b3);
+            }
+        }
+    };
+
+    // ---- pass 1: running max and sum (log2 domain) ---------------------------------------------------
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+    for (int t = 0; t < n_tiles; ++t) {
+        if (t + 1 < n_tiles) { load_tile(t + 1, (t + 1) & 1, false); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncthreads();
+        float s[8][4];
+        scores(t & 1, s);
+        float tm_lo = -INFINITY, tm_hi = -INFINITY;
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const bool ok = t * BG_BN + nt * 8 + cpair + e < a.N;
+                s[nt][e] = ok ? s[nt][e] * scale2 : -INFINITY;
+                s[nt][2 + e] = ok ? s[nt][2 + e] * scale2 : -INFINITY;
+                tm_lo = fmaxf(tm_lo, s[nt][e]); tm_hi = fmaxf(tm_hi, s[nt][2 + e]);
+            }
+        tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 1)); tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 2));
+        tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 1)); tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 2));
+        const float nm_lo = fmaxf(m_lo, tm_lo), nm_hi = fmaxf(m_hi, tm_hi);
+        float sl = 0.f, sh = 0.f;
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) { sl += fast_exp2(s[nt][e] - nm_lo); sh += fast_exp2(s[nt][2 + e] - nm_hi); }
+        l_lo = l_lo * fast_exp2(m_lo - nm_lo) + sl;
+        l_hi = l_hi * fast_exp2(m_hi - nm_hi) + sh;
+        m_lo = nm_lo; m_hi = nm_hi;
+        __syncthreads();
+    }
+    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+    const float lse_lo = m_lo + log2f(l_lo), lse_hi = m_hi + log2f(l_hi);
+    float* prev_lo = prev_sh[r_lo];
+    float* prev_hi = prev_sh[r_hi];
+
+    // ---- pass 2: logp, KL, stored rows, P V --------------------------------------------------------------
+    float o[16][4];
+#pragma unroll
+    for (int nt = 0; nt < 16; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+    float kl_lo = 0.f, kl_hi = 0.f;
+    load_tile(0, 0, true);
+    for (int t = 0; t < n_tiles; ++t) {
+        if (t + 1 < n_tiles) { load_tile(t + 1, (t + 1) & 1, true); cp_async_wait<1>(); }
+        else cp_async_wait<0>();
+        __syncthreads();
+        float s[8][4];
+        scores(t & 1, s);
+        uint32_t pf[4][4];
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {            // two halves of 4 key groups keep the register count down
+            float pv_lo[4][2], pv_hi[4][2], lp_lo[4][2], lp_hi[4][2];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
+                    pv_lo[u][e] = (a.record_kl && prev_lo && key < a.N) ? prev_lo[key] : 0.f;
+                    pv_hi[u][e] = (a.record_kl && prev_hi && key < a.N) ? prev_hi[key] : 0.f;
+                }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int nt = hf * 4 + u;
+                float p[4];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const bool ok = t * BG_BN + nt * 8 + cpair + e < a.N;
+                    const float d_lo = s[nt][e] * scale2 - lse_lo, d_hi = s[nt][2 + e] * scale2 - lse_hi;
+                    const float p_lo = ok ? fast_exp2(d_lo) : 0.f, p_hi = ok ? fast_exp2(d_hi) : 0.f;
+                    lp_lo[u][e] = d_lo * LN2; lp_hi[u][e] = d_hi * LN2;
+                    if (ok && a.record_kl) {
+                        if (prev_lo) kl_lo += p_lo * (lp_lo[u][e] - pv_lo[u][e]);
+                        if (prev_hi) kl_hi += p_hi * (lp_hi[u][e] - pv_hi[u][e]);
+                    }
+                    p[e] = p_lo; p[2 + e] = p_hi;
+                }
+                pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
+                pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
+                    if (prev_lo && key < a.N) prev_lo[key] = lp_lo[u][e];
+                    if (prev_hi && key < a.N) prev_hi[key] = lp_hi[u][e];
+                }
+        }
+        if (a.out) {
+            const uint32_t vb = st_u32 + (t & 1) * 2 * BG_TILE_BYTES + BG_TILE_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+                for (int dp = 0; dp < 8; ++dp) {
+                    const int i = lane >> 3, r = lane & 7;
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(vb + sw_off(ks * 16 + (i & 1) * 8 + r, 2 * dp + (i >> 1)), b0, b1, b2, b3);
+                    mma_bf16(o[2 * dp], pf[ks], b0, b1);
+                    mma_bf16(o[2 * dp + 1], pf[ks], b2, b3);
+                }
+            }
+        }
+        __syncthreads();
+    }
+    kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 1); kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 2);
+    kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 1); kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 2);
+    const bool v_lo = valid_sh[r_lo] != 0, v_hi = valid_sh[r_hi] != 0;
+    if (a.out) {
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+            const int col = h * AT_DH + nt * 8 + cpair;
+            if (v_lo) *reinterpret_cast<__nv_bfloat162*>((__nv_bfloat16*)a.out + (size_t)(row0 + r_lo) * dq + col) = __floats2bfloat162_rn(o[nt][0], o[nt][1]);
+            if (v_hi) *reinterpret_cast<__nv_bfloat162*>((__nv_bfloat16*)a.out + (size_t)(row0 + r_hi) * dq + col) = __floats2bfloat162_rn(o[nt][2], o[nt][3]);
+        }
+    }
+    if (a.kl && (lane & 3) == 0) {
+        if (v_lo) a.kl[(size_t)(row0 + r_lo) * a.n_heads + h] = (prev_lo && a.record_kl) ? kl_lo : 0.f;
+        if (v_hi) a.kl[(size_t)(row0 + r_hi) * a.n_heads + h] = (prev_hi && a.record_kl) ? kl_hi : 0.f;
+    }
+}
+
 template <int NW, int TPW>
 static int launch_attention_sp(const AttnMmaArgs& g, dim3 grid, cudaStream_t st) {
     constexpr int smem = NW * 2 * SP_SLOT_BYTES + AT_BM * AT_DH * 2 + 1024;
@@ -645,7 +869,19 @@ static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count
     dim3 grid(g.tiles_per_seq * batch, a.n_heads);
     const long long ctas = (long long)grid.x * grid.y;
     const char* force = getenv("POLESTAR_ATTN_KERNEL");
-    const int mode = force ? atoi(force) : 0;      // 0 auto, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>
+    const int mode = force ? atoi(force) : 0;      // 0 auto, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>, 5 many-rows
+    // many rows per head (entry forwards, long sequences): share each K/V tile among 64 rows
+    if (mode == 5 || (mode == 0 && (a.N > 8 * 4 * AT_BN || ctas >= 8LL * sm_count) && g.rows_per_seq >= 48)) {
+        AttnMmaArgs gb = g;
+        gb.tiles_per_seq = (g.rows_per_seq + BG_BM - 1) / BG_BM;
+        static bool attr_b = false;
+        if (!attr_b) {
+            if (cudaFuncSetAttribute(attention_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BG_SMEM) != cudaSuccess)
+                return -4;
+            attr_b = true;
+        }
+        return launch_k(attention_big_kernel, dim3(gb.tiles_per_seq * batch, a.n_heads), dim3(BG_WARPS * 32), BG_SMEM, st, gb) == cudaSuccess ? 0 : -4;
+    }
     if (mode != 1) {
         if ((mode == 2 || (mode == 0 && ctas <= 2LL * sm_count)) && a.N <= 8 * 2 * AT_BN) return launch_attention_sp<8, 2>(g, grid, st);
         if ((mode == 3 || mode == 0) && a.N <= 4 * 4 * AT_BN) return launch_attention_sp<4, 4>(g, grid, st);

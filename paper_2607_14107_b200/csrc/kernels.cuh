@@ -651,16 +651,36 @@ __global__ void conf_partial_kernel(const float* logits, const int* m_count, int
     const int per = ((V + chunks - 1) / chunks + 3) & ~3;
     const int v0 = ch * per, v1 = min(V, v0 + per);
     const float* l = logits + (size_t)r * V;
-    float mx = -INFINITY, mxe = -INFINITY;
+    // one pass: every thread keeps a running (max, sum of exp relative to that max) and its best
+    // non-[MASK] candidate; 128-bit loads when the row is 16-byte aligned
+    float mx = -INFINITY, sum = 0.f, mxe = -INFINITY;
     int arg = 0x7fffffff;
-    for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
-        const float x = l[v];
-        mx = fmaxf(mx, x);
-        if (v != mask_id && (x > mxe || (x == mxe && v < arg))) { mxe = x; arg = v; }
+    if ((V & 3) == 0) {
+        const float4* l4 = reinterpret_cast<const float4*>(l);
+        for (int v4 = (v0 >> 2) + threadIdx.x; v4 < (v1 >> 2); v4 += blockDim.x) {
+            const float4 x = __ldg(l4 + v4);
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+            const float m4 = fmaxf(fmaxf(x.x, x.y), fmaxf(x.z, x.w));
+            const float nm = fmaxf(mx, m4);
+            sum = sum * expf(mx - nm) + expf(x.x - nm) + expf(x.y - nm) + expf(x.z - nm) + expf(x.w - nm);
+            mx = nm;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int v = 4 * v4 + u;
+                if (v != mask_id && (xs[u] > mxe || (xs[u] == mxe && v < arg))) { mxe = xs[u]; arg = v; }
+            }
+        }
+    } else {
+        for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) {
+            const float x = l[v];
+            const float nm = fmaxf(mx, x);
+            sum = sum * expf(mx - nm) + expf(x - nm);
+            mx = nm;
+            if (v != mask_id && (x > mxe || (x == mxe && v < arg))) { mxe = x; arg = v; }
+        }
     }
     const float bmx = block_max(mx, red);
-    float sum = 0.f;
-    for (int v = v0 + threadIdx.x; v < v1; v += blockDim.x) sum += expf(l[v] - bmx);
+    sum = (mx == -INFINITY) ? 0.f : sum * expf(mx - bmx);
     sum = block_sum(sum, red);
     // argmax with lowest id on ties
 #pragma unroll
