@@ -871,7 +871,8 @@ static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count
     const char* force = getenv("POLESTAR_ATTN_KERNEL");
     const int mode = force ? atoi(force) : 0;      // 0 auto, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>, 5 many-rows
     // many rows per head (entry forwards, long sequences): share each K/V tile among 64 rows
-    if (mode == 5 || (mode == 0 && (a.N > 8 * 4 * AT_BN || ctas >= 8LL * sm_count) && g.rows_per_seq >= 48)) {
+    const long long big_ctas = (long long)((g.rows_per_seq + BG_BM - 1) / BG_BM) * batch * a.n_heads;
+    if (mode == 5 || (mode == 0 && (a.N > 8 * 4 * AT_BN || ctas >= 4LL * sm_count) && g.rows_per_seq >= 48 && big_ctas >= sm_count)) {
         AttnMmaArgs gb = g;
         gb.tiles_per_seq = (g.rows_per_seq + BG_BM - 1) / BG_BM;
         static bool attr_b = false;

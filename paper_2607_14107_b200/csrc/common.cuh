@@ -236,6 +236,25 @@ __device__ __forceinline__ void epilogue_pair(const EpiArgs& e, int m, int n, fl
     }
 }
 
+// Prefetch into L1 what epilogue_pair will read for the 16 outputs n .. n+15 of row m (row descriptor,
+// RoPE entries, residual values), so that the epilogue after a wait starts on cache hits.
+__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+template <typename T, int EPI>
+__device__ __forceinline__ void epilogue_prefetch(const EpiArgs& e, int m, int n) {
+    if (EPI == EPI_QKV) {
+        const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + m);
+        prefetch_l1(e.kvflag + m);
+        if (rw.y >= 0 && n < (e.n_heads + e.n_kv) * e.head_dim)
+            prefetch_l1(e.rope + (size_t)rw.y * (e.head_dim / 2) + ((n % e.head_dim) >> 1));
+    } else if (EPI == EPI_RESID) {
+        prefetch_l1(e.resid + (size_t)m * e.ld_out + n);
+    } else if (EPI == EPI_DOWN) {
+        const int r = e.list ? __ldg(e.list + m) : m;
+        prefetch_l1(reinterpret_cast<const int4*>(e.rows) + r);
+        prefetch_l1(e.resid + (size_t)r * e.ld_out + n);
+    }
+}
+
 // ---- host: launch with programmatic stream serialization -----------------------------------
 inline bool g_use_pdl = true;
 template <typename... KArgs, typename... Args>

@@ -84,6 +84,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+// same with an L2 eviction policy: weights that are streamed once carry evict_first, so that they do not
+// push activations, partial tiles, the K/V cache and instruction lines out of L2
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "l"(policy)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -113,6 +126,17 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// the same load without the wait: several may be in flight before one tmem_ld_wait(); the registers may only
+// be consumed by memory operations placed after the wait (its "memory" clobber orders them)
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 
@@ -155,6 +179,7 @@ struct SkArgs {
                         // launch, zero again after
     int done_offset;
     int* status;        // set to 1 on a wait time-out
+    int w_stream;       // 1: every weight byte is read once by this launch: load it with the evict_first L2 policy
     int cluster_n;      // > 0: launched in clusters of cluster_n CTAs = the contributors of one output tile;
                         // partial tiles are then exchanged through distributed shared memory, not global memory
     long long* trace;   // optional [gridDim.x][8] nanosecond stamps of this launch (null: off)
@@ -165,7 +190,7 @@ struct SkArgs {
 };
 
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define SK_STAMP(i) do { if (g.trace) g.trace[(size_t)cta * 8 + (i)] = gtime(); } while (0)
+#define SK_STAMP(i) do { if (g.trace) g.trace[(size_t)cta * 12 + (i)] = gtime(); } while (0)
 
 // first unit of CTA c when U units are split over G CTAs
 __device__ __forceinline__ long long sk_begin(long long U, int G, int c) { return (U * c) / G; }
@@ -174,6 +199,21 @@ __device__ __forceinline__ int sk_owner(long long U, int G, long long u) {
     while (c > 0 && sk_begin(U, G, c) > u) --c;
     while (c + 1 < G && sk_begin(U, G, c + 1) <= u) ++c;
     return c;
+}
+
+// Number of partial tile segments in CTA c's unit range (0, 1 or 2): what it has to publish and then help reduce.
+__device__ __forceinline__ int sk_partial_segments(long long U, int G, int c, int kb_total) {
+    const long long b = sk_begin(U, G, c), e = sk_begin(U, G, c + 1);
+    if (e <= b) return 0;
+    const long long tb = b / kb_total, te = (e - 1) / kb_total;
+    const bool head_cut = b != tb * kb_total, tail_cut = e != (te + 1) * kb_total;
+    if (tb == te) return (head_cut || tail_cut) ? 1 : 0;
+    return (head_cut ? 1 : 0) + (tail_cut ? 1 : 0);
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
 template <typename T, int EPI>
@@ -227,12 +267,15 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (lane == 0) {
             // weights do not depend on the previous kernel: request the first stages right away
             const int pre = min(g.stages, n_units);
+            const uint64_t pol = l2_policy_evict_first();
             for (int i = 0; i < pre; ++i) {
                 const long long u = u_begin + i;
                 const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
                 mbar_expect_tx(full0 + 8 * i, STAGE_BYTES);
-                tma_load_2d(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
-                            ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
+                if (g.w_stream) tma_load_2d_hint(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
+                                                 ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F, pol);
+                else tma_load_2d(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
+                                 ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
             }
             pdl_wait();
             SK_STAMP(2);
@@ -249,7 +292,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
                 const uint32_t dst = smem_base + s * STAGE_BYTES;
                 mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
-                tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
+                if (g.w_stream) tma_load_2d_hint(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F, pol);
+                else tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
                 tma_load_2d(dst, &map_a, full0 + 8 * s, kb * BLOCK_K, (tile % g.tiles_t) * BLOCK_T);
             }
             // all of this CTA's loads are requested: start pulling the next GEMMs' weights into L2
@@ -309,8 +353,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const uint32_t taddr0 = tmem_base + ((uint32_t)(q * 32) << 16);
         const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
         int seg = 0;
-        int fix_tile[2];
-        int n_fix = 0;
         long long u = u_begin;
         while (u < u_end) {
             const int tile = (int)(u / kb_total);
@@ -365,13 +407,18 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int which = (k0 == 0) ? 1 : 0;     // slot 0: my range starts inside this tile
                 float* part = g.partial + ((size_t)(2 * cta + which) * BLOCK_T + t_local) * BLOCK_F;
                 if (warp_live) {
-                    for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
-                        float v[16];
-                        tmem_ld16(taddr + (uint32_t)c0, v);
+                    // 64 columns per round trip to TMEM (four loads in flight, one wait)
+                    for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
+                        uint32_t r[4][16];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * j), r[j]);
+                        tmem_ld_wait();
                         if (live) {
 #pragma unroll
-                            for (int c = 0; c < 16; c += 4)
-                                *reinterpret_cast<float4*>(part + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+                            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                                for (int c = 0; c < 16; c += 4)
+                                    *reinterpret_cast<uint4*>(part + c0 + 16 * j + c) = make_uint4(r[j][c], r[j][c + 1], r[j][c + 2], r[j][c + 3]);
                         }
                     }
                 }
@@ -381,38 +428,85 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile], 1);
-                if (n_fix < 2) fix_tile[n_fix++] = tile;
             }
             ++seg;
             u = seg_end;
         }
         if (threadIdx.x == 64) SK_STAMP(5);
-        // ---- pass 2: every CTA that contributed to a split tile reduces its share of that tile ------
-        for (int f = 0; f < n_fix; ++f) {
-            const int tile = fix_tile[f];
-            const long long tile_begin = (long long)tile * kb_total, tile_end = tile_begin + kb_total;
-            const int c_lo = sk_owner(U, G, tile_begin), c_hi = sk_owner(U, G, tile_end - 1);
-            const int nseg = c_hi - c_lo + 1;
-            const int tile_f = tile / g.tiles_t, tile_t = tile % g.tiles_t;
-            const int n0 = tile_f * BLOCK_F;
+    }
+
+    // ---- pass 2 (all six warps): every CTA that contributed to split tiles reduces its share of them ------
+    // The partial tiles of this CTA's unit range follow from the range alone: its first tile if the range starts
+    // inside it or ends before its end, and its last tile (when different) if the range ends inside it.
+    if (g.cluster_n == 0 && n_units > 0) {
+        __syncwarp();
+        pdl_wait();
+        const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
+        const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;
+        const bool head_cut = u_begin != tb * kb_total, tail_cut = u_end != (te + 1) * kb_total;
+        int fix_tile[2];
+        int n_fix = 0;
+        if (tb == te) { if (head_cut || tail_cut) fix_tile[n_fix++] = (int)tb; }
+        else {
+            if (head_cut) fix_tile[n_fix++] = (int)tb;
+            if (tail_cut) fix_tile[n_fix++] = (int)te;
+        }
+        if (n_fix > 0) {
+            // The items (one row x 16 columns each) of a tile are dealt to its contributors in contiguous shares.
+            // A CTA that contributes to two tiles takes half a share of each, so that every CTA reduces about
+            // the same number of items; inside the CTA the items of both tiles form one list for its 192 threads.
+            int f_lo[2] = {0, 0}, f_n[2] = {0, 0}, f_clo[2] = {0, 0}, f_nseg[2] = {1, 1};
+#pragma unroll
+            for (int f = 0; f < 2; ++f) {
+                if (f < n_fix) {
+                    const int tile = fix_tile[f];
+                    const long long tile_begin = (long long)tile * kb_total, tile_end = tile_begin + kb_total;
+                    const int c_lo = sk_owner(U, G, tile_begin), c_hi = sk_owner(U, G, tile_end - 1);
+                    const int nseg = c_hi - c_lo + 1;
+                    const int tile_t = tile % g.tiles_t;
+                    const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
+                    const int n_items = n_live * (BLOCK_F / 16);
+                    const int w_lo = sk_partial_segments(U, G, c_lo, kb_total) == 2 ? 1 : 2;
+                    const int w_hi = (nseg > 1 && sk_partial_segments(U, G, c_hi, kb_total) == 2) ? 1 : 2;
+                    const int w_all = (nseg == 1) ? w_lo : w_lo + w_hi + 2 * (nseg - 2);
+                    const int before = (cta == c_lo) ? 0 : w_lo + 2 * (cta - c_lo - 1);
+                    const int mine = (cta == c_lo) ? w_lo : (cta == c_hi ? w_hi : 2);
+                    f_lo[f] = (int)(((long long)n_items * before) / w_all);
+                    f_n[f] = (int)(((long long)n_items * (before + mine)) / w_all) - f_lo[f];
+                    f_clo[f] = c_lo;
+                    f_nseg[f] = nseg;
+                }
+            }
+            const int total = f_n[0] + f_n[1];
+            if ((int)threadIdx.x < total) {
+                // pull what the epilogue of this thread's first item reads into L1 while the tiles are still arriving
+                const int f = (int)threadIdx.x < f_n[0] ? 0 : 1;
+                const int item = f_lo[f] + (int)threadIdx.x - (f ? f_n[0] : 0);
+                const int tile = fix_tile[f];
+                epilogue_prefetch<T, EPI>(e, (tile % g.tiles_t) * BLOCK_T + item / (BLOCK_F / 16),
+                                          (tile / g.tiles_t) * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
+            }
             if (threadIdx.x == 64) {
-                // bounded wait until all contributors have published their partial tile
+                // bounded wait until all contributors have published their partial tiles
                 const long long t0 = clock64();
                 int ok = 1;
-                while (*((volatile int*)&g.tile_counter[tile]) < nseg) {
-                    if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) { ok = 0; *abort_flag = 1; break; }
-                    __nanosleep(64);
+                for (int f = 0; f < n_fix && ok; ++f) {
+                    while (ld_acquire_gpu(&g.tile_counter[fix_tile[f]]) < f_nseg[f]) {
+                        if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) { ok = 0; *abort_flag = 1; break; }
+                        __nanosleep(64);
+                    }
                 }
                 last_sh = ok;
-                if (f == 0) SK_STAMP(6);
+                SK_STAMP(6);
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            __syncthreads();
             if (last_sh) {
-                __threadfence();
-                const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
-                const int n_items = n_live * (BLOCK_F / 16);
-                // items are dealt round-robin to the contributing CTAs, then to their 128 epilogue threads
-                for (int item = (cta - c_lo) * 128 + ((int)threadIdx.x - 64); item < n_items; item += nseg * 128) {
+                for (int i = (int)threadIdx.x; i < total; i += THREADS) {
+                    const int f = i < f_n[0] ? 0 : 1;
+                    const int item = f_lo[f] + i - (f ? f_n[0] : 0);
+                    const int tile = fix_tile[f];
+                    const long long tile_begin = (long long)tile * kb_total;
+                    const int c_lo = f_clo[f], nseg = f_nseg[f];
                     const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16;
                     float acc[16];
 #pragma unroll
@@ -442,16 +536,21 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
                             }
                     }
-                    const int mm = tile_t * BLOCK_T + tl;
+                    const int mm = (tile % g.tiles_t) * BLOCK_T + tl;
+                    const int n0 = (tile / g.tiles_t) * BLOCK_F;
 #pragma unroll
                     for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, mm, n0 + c0 + c, acc[c], acc[c + 1]);
                 }
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) SK_STAMP(8);
+            __syncthreads();
             if (threadIdx.x == 64 && last_sh) {
                 // the last contributor to finish its share re-arms the tile's counters for the next launch
-                const int prev = atomicAdd(&g.tile_counter[g.done_offset + tile], 1);
-                if (prev == nseg - 1) { g.tile_counter[tile] = 0; g.tile_counter[g.done_offset + tile] = 0; }
+                for (int f = 0; f < n_fix; ++f) {
+                    const int tile = fix_tile[f];
+                    const int prev = atomicAdd(&g.tile_counter[g.done_offset + tile], 1);
+                    if (prev == f_nseg[f] - 1) { g.tile_counter[tile] = 0; g.tile_counter[g.done_offset + tile] = 0; }
+                }
             }
         }
     }

@@ -163,6 +163,7 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     g.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", 4)));
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
     g.cluster_n = cluster_n;
+    g.w_stream = (g.tiles_t == 1 && env_int("POLESTAR_GEMM_EVICT_FIRST", 1)) ? 1 : 0;
     // debug: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
     memset(g.pf, 0, sizeof(g.pf));
     for (int j = 0; next && j < 2; ++j) {

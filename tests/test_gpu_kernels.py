@@ -30,6 +30,23 @@ def rnd(shape, key, std=1.0, dtype=torch.float32):
     (torch.bfloat16, 3, 31, 2, 1, 128),        # fewer keys than one warp tile
 ])
 def test_attention_drift_matches_oracle(dtype, R, N, nh, nkv, dh):
+    check_attention(dtype, R, N, nh, nkv, dh)
+
+
+@pytest.mark.parametrize("variant,R,N,nh,nkv", [
+    (1, 37, 200, 4, 2),            # two-pass kernel, ragged
+    (1, 40, 1100, 2, 1),           # two-pass kernel beyond the single-pass key limit
+    (2, 37, 200, 4, 2), (3, 37, 200, 4, 2), (4, 37, 1000, 2, 1),     # single-pass variants
+    (5, 150, 1100, 2, 1),          # 64-row tiles: three row tiles (last ragged), 18 key tiles (last ragged)
+    (5, 5, 37, 2, 2),              # 64-row tiles, fewer rows and keys than one tile
+    (0, 200, 2048, 8, 8),          # automatic choice at a long sequence
+])
+def test_attention_kernel_variants(monkeypatch, variant, R, N, nh, nkv):
+    monkeypatch.setenv("POLESTAR_ATTN_KERNEL", str(variant))
+    check_attention(torch.bfloat16, R, N, nh, nkv, 128)
+
+
+def check_attention(dtype, R, N, nh, nkv, dh):
     q = rnd((R, nh * dh), 1, 1.0, dtype).cuda()
     k = rnd((N, nkv * dh), 2, 1.0, dtype).cuda()
     v = rnd((N, nkv * dh), 3, 1.0, dtype).cuda()
