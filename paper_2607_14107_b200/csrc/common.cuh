@@ -199,7 +199,8 @@ __device__ __forceinline__ void epilogue_pair(const EpiArgs& e, int m, int n, fl
         const int dq = e.n_heads * e.head_dim, dkv = e.n_kv * e.head_dim;
         const int Npos = (EPI == EPI_QKV) ? e.N_seq : e.P;
         if (n < dq + dkv) {
-            const int p = n % e.head_dim;
+            const int hd1 = e.head_dim - 1;
+            const int p = (e.head_dim & hd1) ? n % e.head_dim : (n & hd1);      // power-of-two head sizes: no division
             const float2 cs = __ldg(e.rope + (size_t)pos * (e.head_dim / 2) + (p >> 1));
             const float r0 = v0 * cs.x - v1 * cs.y;
             const float r1 = v1 * cs.x + v0 * cs.y;

@@ -40,7 +40,10 @@ constexpr int BLOCK_T = 128;   // tokens per tile (UMMA M)
 constexpr int BLOCK_F = 256;   // output features per tile (UMMA N)
 constexpr int BLOCK_K = 64;    // bf16 elements per k block = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr int THREADS = 192;
+constexpr int THREADS = 192;          // producer warp, MMA warp, four epilogue warps
+// Launched block size: the warps beyond the six role warps sleep at a barrier until the fix-up pass, where the
+// reduction of partial tiles is pure memory latency and more threads in flight mean fewer rounds.
+constexpr int FIX_THREADS = 512;
 constexpr int MAX_STAGES = 8;
 constexpr uint32_t A_BYTES = BLOCK_T * BLOCK_K * 2;   // 16 KB
 constexpr uint32_t W_BYTES = BLOCK_F * BLOCK_K * 2;   // 32 KB
@@ -217,7 +220,7 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
 }
 
 template <typename T, int EPI>
-__global__ void __launch_bounds__(THREADS, 1)
+__global__ void __launch_bounds__(FIX_THREADS, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                SkArgs g, EpiArgs e) {
     extern __shared__ uint8_t smem_raw[];
@@ -225,6 +228,9 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
     __shared__ int last_sh;
+    __shared__ int fx_par[2][6];          // per partial tile of this CTA: tile, c_lo, nseg, before, mine, w_all
+    __shared__ int fx_n;
+    __shared__ volatile int fx_ready;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, cta = blockIdx.x;
@@ -251,6 +257,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         }
         abort_sh = 0;
         last_sh = 0;
+        fx_ready = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -263,14 +270,51 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
 
+    if (threadIdx.x == THREADS) {
+        // An idle thread works out, while the main loop runs, which partial tiles this CTA will help reduce and
+        // which share of their items is its own (64-bit divisions that must not sit on the tail's critical path).
+        // The partial tiles of the CTA's unit range follow from the range alone: its first tile if the range
+        // starts inside it or ends before its end, and its last tile (when different) if the range ends inside it.
+        // A tile's items (one row x 16 columns each) are dealt to its contributors in contiguous shares; a CTA that
+        // contributes to two tiles takes half a share of each, so that every CTA reduces about as many items.
+        int n_fix = 0;
+        if (g.cluster_n == 0 && n_units > 0) {
+            const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;
+            const bool head_cut = u_begin != tb * kb_total, tail_cut = u_end != (te + 1) * kb_total;
+            int fix_tile[2] = {0, 0};
+            if (tb == te) { if (head_cut || tail_cut) fix_tile[n_fix++] = (int)tb; }
+            else {
+                if (head_cut) fix_tile[n_fix++] = (int)tb;
+                if (tail_cut) fix_tile[n_fix++] = (int)te;
+            }
+            for (int f = 0; f < n_fix; ++f) {
+                const int tile = fix_tile[f];
+                const long long tile_begin = (long long)tile * kb_total, tile_end = tile_begin + kb_total;
+                const int c_lo = sk_owner(U, G, tile_begin), c_hi = sk_owner(U, G, tile_end - 1);
+                const int nseg = c_hi - c_lo + 1;
+                const int w_lo = sk_partial_segments(U, G, c_lo, kb_total) == 2 ? 1 : 2;
+                const int w_hi = (nseg > 1 && sk_partial_segments(U, G, c_hi, kb_total) == 2) ? 1 : 2;
+                fx_par[f][0] = tile; fx_par[f][1] = c_lo; fx_par[f][2] = nseg;
+                fx_par[f][3] = (cta == c_lo) ? 0 : w_lo + 2 * (cta - c_lo - 1);
+                fx_par[f][4] = (cta == c_lo) ? w_lo : (cta == c_hi ? w_hi : 2);
+                fx_par[f][5] = (nseg == 1) ? w_lo : w_lo + w_hi + 2 * (nseg - 2);
+            }
+        }
+        fx_n = n_fix;
+        __threadfence_block();
+        fx_ready = 1;
+    }
+
     if (warp == 0) {
         if (lane == 0) {
             // weights do not depend on the previous kernel: request the first stages right away
             const int pre = min(g.stages, n_units);
             const uint64_t pol = l2_policy_evict_first();
-            for (int i = 0; i < pre; ++i) {
-                const long long u = u_begin + i;
-                const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
+            // (tile, kb) of a unit are advanced incrementally: no 64-bit division per unit on this thread
+            const int tile0 = (int)(u_begin / kb_total), kb0 = (int)(u_begin - (long long)tile0 * kb_total);
+            int tile = tile0, kb = kb0;
+            auto advance = [&](int& t, int& k) { if (++k == kb_total) { k = 0; ++t; } };
+            for (int i = 0; i < pre; ++i, advance(tile, kb)) {
                 mbar_expect_tx(full0 + 8 * i, STAGE_BYTES);
                 if (g.w_stream) tma_load_2d_hint(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
                                                  ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F, pol);
@@ -279,17 +323,15 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
             pdl_wait();
             SK_STAMP(2);
-            for (int i = 0; i < pre; ++i) {
-                const long long u = u_begin + i;
-                const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
-                tma_load_2d(smem_base + i * STAGE_BYTES, &map_a, full0 + 8 * i, kb * BLOCK_K, (tile % g.tiles_t) * BLOCK_T);
+            {
+                int ta = tile0, ka = kb0;
+                for (int i = 0; i < pre; ++i, advance(ta, ka))
+                    tma_load_2d(smem_base + i * STAGE_BYTES, &map_a, full0 + 8 * i, ka * BLOCK_K, (ta % g.tiles_t) * BLOCK_T);
             }
-            for (int i = pre; i < n_units; ++i) {
+            for (int i = pre; i < n_units; ++i, advance(tile, kb)) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
-                const long long u = u_begin + i;
-                const int tile = (int)(u / kb_total), kb = (int)(u - (long long)tile * kb_total);
                 const uint32_t dst = smem_base + s * STAGE_BYTES;
                 mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
                 if (g.w_stream) tma_load_2d_hint(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F, pol);
@@ -315,9 +357,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const uint32_t idesc = instr_desc_bf16(BLOCK_T, BLOCK_F);
             int seg = 0;
             bool seg_start = true;
-            for (int i = 0; i < n_units; ++i) {
-                const long long u = u_begin + i;
-                const int kb = (int)(u % kb_total);
+            int kb = (int)(u_begin % kb_total);
+            for (int i = 0; i < n_units; ++i, kb = (kb + 1 == kb_total) ? 0 : kb + 1) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (seg_start && seg > 1) {
@@ -344,7 +385,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
             }
         }
-    } else {
+    } else if (warp < 6) {
         // ---- epilogue warps: TMEM lane = token, column = feature ------------------------------------
         pdl_wait();
         trace_stamp(100 + EPI, 64);
@@ -435,46 +476,30 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (threadIdx.x == 64) SK_STAMP(5);
     }
 
-    // ---- pass 2 (all six warps): every CTA that contributed to split tiles reduces its share of them ------
-    // The partial tiles of this CTA's unit range follow from the range alone: its first tile if the range starts
-    // inside it or ends before its end, and its last tile (when different) if the range ends inside it.
+    // ---- pass 2 (all warps): every CTA that contributed to split tiles reduces its share of them ------------
     if (g.cluster_n == 0 && n_units > 0) {
         __syncwarp();
         pdl_wait();
         const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
-        const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;
-        const bool head_cut = u_begin != tb * kb_total, tail_cut = u_end != (te + 1) * kb_total;
-        int fix_tile[2];
-        int n_fix = 0;
-        if (tb == te) { if (head_cut || tail_cut) fix_tile[n_fix++] = (int)tb; }
-        else {
-            if (head_cut) fix_tile[n_fix++] = (int)tb;
-            if (tail_cut) fix_tile[n_fix++] = (int)te;
+        {
+            const long long t0 = clock64();
+            while (!fx_ready) { if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; break; } }
+            __threadfence_block();
         }
+        const int n_fix = fx_ready ? fx_n : 0;
         if (n_fix > 0) {
-            // The items (one row x 16 columns each) of a tile are dealt to its contributors in contiguous shares.
-            // A CTA that contributes to two tiles takes half a share of each, so that every CTA reduces about
-            // the same number of items; inside the CTA the items of both tiles form one list for its 192 threads.
-            int f_lo[2] = {0, 0}, f_n[2] = {0, 0}, f_clo[2] = {0, 0}, f_nseg[2] = {1, 1};
+            // inside the CTA the items of both tiles form one list for all its threads
+            int fix_tile[2] = {0, 0}, f_lo[2] = {0, 0}, f_n[2] = {0, 0}, f_clo[2] = {0, 0}, f_nseg[2] = {1, 1};
 #pragma unroll
             for (int f = 0; f < 2; ++f) {
                 if (f < n_fix) {
-                    const int tile = fix_tile[f];
-                    const long long tile_begin = (long long)tile * kb_total, tile_end = tile_begin + kb_total;
-                    const int c_lo = sk_owner(U, G, tile_begin), c_hi = sk_owner(U, G, tile_end - 1);
-                    const int nseg = c_hi - c_lo + 1;
-                    const int tile_t = tile % g.tiles_t;
+                    fix_tile[f] = fx_par[f][0]; f_clo[f] = fx_par[f][1]; f_nseg[f] = fx_par[f][2];
+                    const int before = fx_par[f][3], mine = fx_par[f][4], w_all = fx_par[f][5];
+                    const int tile_t = fix_tile[f] % g.tiles_t;
                     const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
                     const int n_items = n_live * (BLOCK_F / 16);
-                    const int w_lo = sk_partial_segments(U, G, c_lo, kb_total) == 2 ? 1 : 2;
-                    const int w_hi = (nseg > 1 && sk_partial_segments(U, G, c_hi, kb_total) == 2) ? 1 : 2;
-                    const int w_all = (nseg == 1) ? w_lo : w_lo + w_hi + 2 * (nseg - 2);
-                    const int before = (cta == c_lo) ? 0 : w_lo + 2 * (cta - c_lo - 1);
-                    const int mine = (cta == c_lo) ? w_lo : (cta == c_hi ? w_hi : 2);
-                    f_lo[f] = (int)(((long long)n_items * before) / w_all);
-                    f_n[f] = (int)(((long long)n_items * (before + mine)) / w_all) - f_lo[f];
-                    f_clo[f] = c_lo;
-                    f_nseg[f] = nseg;
+                    f_lo[f] = (n_items * before) / w_all;
+                    f_n[f] = (n_items * (before + mine)) / w_all - f_lo[f];
                 }
             }
             const int total = f_n[0] + f_n[1];
@@ -501,11 +526,10 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
             __syncthreads();
             if (last_sh) {
-                for (int i = (int)threadIdx.x; i < total; i += THREADS) {
+                for (int i = (int)threadIdx.x; i < total; i += FIX_THREADS) {
                     const int f = i < f_n[0] ? 0 : 1;
                     const int item = f_lo[f] + i - (f ? f_n[0] : 0);
                     const int tile = fix_tile[f];
-                    const long long tile_begin = (long long)tile * kb_total;
                     const int c_lo = f_clo[f], nseg = f_nseg[f];
                     const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16;
                     float acc[16];
@@ -518,7 +542,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             const int cc = c_lo + sg0 + j;
                             if (sg0 + j < nseg) {
                                 // a CTA whose range starts inside the tile wrote slot 0, otherwise slot 1
-                                const int wsl = (sk_begin(U, G, cc) > tile_begin) ? 0 : 1;
+                                // (only the tile's first contributor can start at or before the tile's first unit)
+                                const int wsl = (cc == c_lo) ? 1 : 0;
                                 const float4* ps = reinterpret_cast<const float4*>(
                                     g.partial + ((size_t)(2 * cc + wsl) * BLOCK_T + tl) * BLOCK_F + c0);
 #pragma unroll
@@ -560,7 +585,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // threads meet at the cluster barrier; then each CTA adds up its share of the tile, reading the other
         // CTAs' partial tiles through distributed shared memory in rank order (deterministic), and runs the epilogue.
         cluster_sync_all();
-        if (warp >= 2 && !abort_sh) {
+        if (warp >= 2 && warp < 6 && !abort_sh) {
             const int tile = (int)(u_begin / kb_total);
             const int tile_f = tile / g.tiles_t, tile_t = tile % g.tiles_t;
             const int n0 = tile_f * BLOCK_F;

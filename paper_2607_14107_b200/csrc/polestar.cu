@@ -182,8 +182,8 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
         CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr = true;
     }
-    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e));
-    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::THREADS), smem, st, *mw, *ma, g, e));
+    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e));
+    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e));
     return POLESTAR_OK;
 }
 
