@@ -181,6 +181,24 @@ struct EpiArgs {
     const int* idx; const int* counts; int max_rows; int P;
 };
 
+// Row-wise work appended to a GEMM whose output rows are the input of the next normalisation: once every CTA
+// of the grid has stored its outputs (a counter all CTAs add to), the CTAs share out the rows and stage the
+// next GEMM's operand, which saves a kernel boundary per normalisation.
+//   kind 1: RMSNorm of the finished rows (FFN input);  kind 2: patch + RMSNorm + staging of the next layer's
+//   QKV input (Algorithm 1 "Patch").  kind 0: nothing.
+struct PostArgs {
+    int kind, n_rows, d;
+    float eps;
+    const float* gain;
+    void* a_out;
+    float* x;                                  // rows written by this GEMM (kind 1: source; kind 2: residual stream)
+    const int* list; const int* m_count;       // kind 1
+    const Row* rows; float* hc; const float* packet; const unsigned char* patch; unsigned char* kvflag;   // kind 2
+    StepDesc sd;                               // kind 2
+    unsigned* counter;                         // never reset: `expect` is the running total after this launch
+    unsigned expect;
+};
+
 // One output pair (n even, n+1) of row m.
 template <typename T, int EPI>
 __device__ __forceinline__ void epilogue_pair(const EpiArgs& e, int m, int n, float v0, float v1) {

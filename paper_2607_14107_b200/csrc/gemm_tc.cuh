@@ -32,6 +32,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "kernels.cuh"
 
 namespace ps {
 namespace tc {
@@ -222,7 +223,7 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
 template <typename T, int EPI>
 __global__ void __launch_bounds__(FIX_THREADS, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
-               SkArgs g, EpiArgs e) {
+               SkArgs g, EpiArgs e, PostArgs post) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_sh;
@@ -631,6 +632,36 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, ncols);
+    if constexpr (EPI == EPI_RESID || EPI == EPI_DOWN) {
+        if (post.kind != 0) {
+            // Every output store of this CTA is issued (barrier above).  Add to the grid's counter, wait until
+            // all CTAs have done so (all are resident: the grid has at most one CTA per SM), then share out the rows.
+            __shared__ float post_red[33];
+            __shared__ int post_ok;
+            if (threadIdx.x == 0) { __threadfence(); atomicAdd(post.counter, 1u); }
+            if (cta < post.n_rows) {
+                if (threadIdx.x == 0) {
+                    const long long t0 = clock64();
+                    int ok = 1;
+                    while ((int)((unsigned)ld_acquire_gpu(reinterpret_cast<const int*>(post.counter)) - post.expect) < 0) {
+                        if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) { ok = 0; *abort_flag = 1; break; }
+                        __nanosleep(32);
+                    }
+                    post_ok = ok;
+                }
+                __syncthreads();
+                if (post_ok) {
+                    for (int r = cta; r < post.n_rows; r += G) {
+                        if (post.kind == 1)
+                            prep_rows_row<T>(r, post.x, post.list, post.m_count, post.gain, post.eps, post.d, (T*)post.a_out, post_red);
+                        else
+                            prep_qkv_row<T>(post.sd, r, post.rows, post.x, post.hc, post.packet, post.patch, post.gain, post.eps,
+                                            post.d, (T*)post.a_out, post.kvflag, post_red);
+                    }
+                }
+            }
+        }
+    }
     if (threadIdx.x == 0) SK_STAMP(7);
     trace_stamp(200 + EPI, 0);
     if (threadIdx.x == 0 && abort_sh) atomicExch(g.status, 1);

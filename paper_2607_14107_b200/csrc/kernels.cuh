@@ -128,12 +128,9 @@ __device__ __forceinline__ void zero_row(T* a, int d) {
 //   the previous layer selected them); every other row reads the residual stream x.
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* hc, const float* packet,
-                                const unsigned char* patch, const float* gain, float eps, int d,
-                                T* a_out, unsigned char* kvflag) {
-    KERNEL_PROLOGUE(3);   // prep_qkv_kernel
-    __shared__ float red[33];
-    const int r = blockIdx.x;
+__device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Row* rows, float* x, float* hc, const float* packet,
+                                             const unsigned char* patch, const float* gain, float eps, int d,
+                                             T* a_out, unsigned char* kvflag, float* red) {
     const Row rw = rows[r];
     T* a = a_out + (size_t)r * d;
     if (rw.pos < 0) {
@@ -160,15 +157,20 @@ __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* h
     }
     if (threadIdx.x == 0) kvflag[r] = kv ? 1 : 0;
 }
+template <typename T>
+__global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* hc, const float* packet,
+                                const unsigned char* patch, const float* gain, float eps, int d,
+                                T* a_out, unsigned char* kvflag) {
+    KERNEL_PROLOGUE(3);   // prep_qkv_kernel
+    __shared__ float red[33];
+    prep_qkv_row<T>(sd, blockIdx.x, rows, x, hc, packet, patch, gain, eps, d, a_out, kvflag, red);
+}
 
 // RMSNorm of a compacted list of rows (FFN input, LM-head input).
 //   src row = list ? list[i] : i;  packet_rows: rows flagged as window rows read the packet
 template <typename T>
-__global__ void prep_rows_kernel(const float* x, const int* list, const int* m_count, const float* gain,
-                                 float eps, int d, T* a_out) {
-    KERNEL_PROLOGUE(4);   // prep_rows_kernel
-    __shared__ float red[33];
-    const int i = blockIdx.x;
+__device__ __forceinline__ void prep_rows_row(int i, const float* x, const int* list, const int* m_count, const float* gain,
+                                              float eps, int d, T* a_out, float* red) {
     T* a = a_out + (size_t)i * d;
     if (m_count && i >= *m_count) {
         for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
@@ -176,6 +178,13 @@ __global__ void prep_rows_kernel(const float* x, const int* list, const int* m_c
     }
     const int r = list ? list[i] : i;
     norm_row<T>(x + (size_t)r * d, gain, eps, d, a, nullptr, nullptr, red);
+}
+template <typename T>
+__global__ void prep_rows_kernel(const float* x, const int* list, const int* m_count, const float* gain,
+                                 float eps, int d, T* a_out) {
+    KERNEL_PROLOGUE(4);   // prep_rows_kernel
+    __shared__ float red[33];
+    prep_rows_row<T>(blockIdx.x, x, list, m_count, gain, eps, d, a_out, red);
 }
 
 // LM-head input rows: entry i < n_act reads x[act_rows...]; later entries read packet rows.

@@ -86,6 +86,8 @@ struct GemmWs {
     float* partial = nullptr; size_t partial_bytes = 0;
     int* counters = nullptr; int n_counters = 0;
     int* status = nullptr;
+    unsigned* post_counter = nullptr;      // grid-wide arrival counter of GEMMs with appended row work (never reset)
+    mutable unsigned post_total = 0;       // its value once every launch so far has completed
 };
 
 // bf16 matrices with out % 256 == 0 and in % 64 == 0 are stored tile-major (see polestar.h)
@@ -125,7 +127,8 @@ static void sk_grid(int M, int N_out, int K, long long* U, long long* G) {
 
 template <int EPI>
 static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a_rows_alloc, const void* W, int M,
-                          int N_out, int K, const EpiArgs& e, cudaStream_t st, const NextW* next = nullptr) {
+                          int N_out, int K, const EpiArgs& e, cudaStream_t st, const NextW* next = nullptr,
+                          const PostArgs* post = nullptr) {
     if (M <= 0) return POLESTAR_OK;
     (void)a_rows_alloc;
     // weights: tile-major [chunks * 256][64]; activations: exactly M rows, so that the rows of a token tile
@@ -182,8 +185,16 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
         CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr = true;
     }
-    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e));
-    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e));
+    PostArgs pa;
+    memset(&pa, 0, sizeof(pa));
+    if (post && post->kind && ws.post_counter) {
+        pa = *post;
+        pa.counter = ws.post_counter;
+        ws.post_total += (unsigned)G;
+        pa.expect = ws.post_total;
+    }
+    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e, pa));
+    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e, pa));
     return POLESTAR_OK;
 }
 
@@ -411,9 +422,15 @@ struct Path {
 
     template <int EPI>
     static int gemm(polestar_ctx* c, const void* A, int a_rows_alloc, const void* W, int M, int N_out, int K,
-                    const EpiArgs& e, const NextW* next = nullptr) {
-        if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 256 == 0)
-            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st, next);
+                    const EpiArgs& e, const NextW* next = nullptr, const PostArgs* post = nullptr, bool* fused = nullptr) {
+        if (fused) *fused = false;
+        if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 256 == 0) {
+            const bool fuse = post && post->kind && c->gws.post_counter && post->d <= 4 * NORM_VPT * tc::FIX_THREADS &&
+                              env_int("POLESTAR_FUSE_PREP", 0);      // measured on B200: no faster than the separate kernel
+                                                                     // (grid-wide counter round trip = kernel boundary)
+            if (fused) *fused = fuse;
+            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st, next, fuse ? post : nullptr);
+        }
         return launch_gemm_simt<T, EPI>(A, W, M, N_out, K, e, c->st);
     }
 
@@ -465,6 +482,7 @@ struct Path {
             CK(cudaGetLastError());
         }
 
+        bool qkv_staged = false, ffn_staged = false;
         for (int l = 0; l < L; ++l) {
             char* kc = b.kc + (size_t)l * bs * N * dkv * es;
             char* vc = b.vc + (size_t)l * bs * N * dkv * es;
@@ -475,12 +493,13 @@ struct Path {
                 Scope sc(c, POLESTAR_PROF_MISC, 0, 0, 1);
                 CK(launch_k(keep_hidden_kernel, dim3(bs * B), dim3(256), 0, st, sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d));
             }
-            {
+            if (!qkv_staged) {      // (layers after the first: done in the tail of the previous layer's down projection)
                 Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
                 CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
                                                      c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag));
                 CK(cudaGetLastError());
             }
+            qkv_staged = false;
             EpiArgs e;
             {
                 const double nq = dq + 2 * dkv;
@@ -533,9 +552,13 @@ struct Path {
                 e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
                 NextW nx[2];
                 nx[0].w = c->wgu[l]; nx[0].N_out = 2 * F; nx[0].K = d; nx[0].M = M; nx[0].first = pf_units2; nx[0].count = pf_units;
-                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e, nx))) return rc;
+                PostArgs po;
+                memset(&po, 0, sizeof(po));
+                po.kind = 1; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n2[l]; po.a_out = b.a_buf;
+                po.x = b.x1; po.list = list; po.m_count = m2_count;
+                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e, nx, &po, &ffn_staged))) return rc;
             }
-            {
+            if (!ffn_staged) {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
                 CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
                 CK(cudaGetLastError());
@@ -557,7 +580,14 @@ struct Path {
                 if (l + 1 < L) { nx[0].w = c->wqkv[l + 1]; nx[0].N_out = dq + 2 * dkv; nx[0].K = d; nx[0].M = M; }
                 else { nx[0].w = c->lm_head; nx[0].N_out = m.vocab; nx[0].K = d; nx[0].M = bs * B; }
                 nx[0].count = pf_units;
-                if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e, nx))) return rc;
+                PostArgs po;
+                memset(&po, 0, sizeof(po));
+                if (l + 1 < L) {
+                    po.kind = 2; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n1[l + 1]; po.a_out = b.a_buf;
+                    po.x = b.x; po.rows = b.rows; po.hc = b.hc + (size_t)(l + 1) * bs * Wm * d; po.packet = b.packet;
+                    po.patch = b.patch + (size_t)(l + 1) * bs * Wm; po.kvflag = b.kvflag; po.sd = sd;
+                }
+                if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e, nx, &po, &qkv_staged))) return rc;
             }
         }
         if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
@@ -785,7 +815,8 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     c->rows_lm = p->batch * (c->B + std::min(p->win_suffix_blocks * c->B, c->W_max));
     c->cum.assign(p->batch, 0);
     c->gws.partial = c->b.gemm_partial; c->gws.partial_bytes = GEMM_PARTIAL_BYTES;
-    c->gws.counters = c->b.gemm_counters; c->gws.n_counters = GEMM_COUNTERS; c->gws.status = c->b.status;
+    c->gws.counters = c->b.gemm_counters; c->gws.n_counters = GEMM_COUNTERS - 2; c->gws.status = c->b.status;
+    c->gws.post_counter = reinterpret_cast<unsigned*>(c->b.gemm_counters + GEMM_COUNTERS - 1); c->gws.post_total = 0;
 
     auto fail = [&](int code) { delete c; return code; };
     // zero the persistent state (everything in front of the scratch rows)

@@ -132,6 +132,13 @@ def test_c1b_bf16_tensor_core_path():
     assert seen["refresh"] > 5
 
 
+def test_c1b_bf16_norm_staging_inside_the_gemm_tail(monkeypatch):
+    # opt-in variant: the RMSNorm staging of the next GEMM's input runs in the tail of the producing GEMM
+    monkeypatch.setenv("POLESTAR_FUSE_PREP", "1")
+    seen = run_forced("c1b", 10, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["refresh"] > 3
+
+
 def test_c1b_bf16_simt_gemm_path():
     run_forced("c1b", 6, tau_upd=-1, flags=I.FLAG_DEFAULT | Bd.FLAG_SIMT_GEMM)
 
