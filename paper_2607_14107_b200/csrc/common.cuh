@@ -255,6 +255,110 @@ __device__ __forceinline__ void epilogue_pair(const EpiArgs& e, int m, int n, fl
     }
 }
 
+// 16 consecutive values to dst (16-byte aligned)
+template <typename T> __device__ __forceinline__ void store16(T* dst, const float* v);
+template <> __device__ __forceinline__ void store16<float>(float* dst, const float* v) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+}
+template <> __device__ __forceinline__ void store16<__nv_bfloat16>(__nv_bfloat16* dst, const float* v) {
+    uint32_t w[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+}
+template <typename T> __device__ __forceinline__ void store8(T* dst, const float* v);
+template <> __device__ __forceinline__ void store8<float>(float* dst, const float* v) {
+    reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+template <> __device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16* dst, const float* v) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// The 16 outputs n .. n+15 (n % 16 == 0) of row m: the same arithmetic as epilogue_pair on each pair, with the
+// row descriptor read once and all loads and stores 16 bytes wide.  Requires head_dim % 16 == 0 and leading
+// dimensions that keep 16-column groups 16-byte aligned (true for every matrix the tensor-core path accepts).
+template <typename T, int EPI>
+__device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int n, const float* v) {
+    if (EPI == EPI_QKV || EPI == EPI_QKV_REFRESH) {
+        int seq, pos, kvf;
+        if (EPI == EPI_QKV) {
+            const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + m);   // {seq, pos, widx, aidx}
+            if (rw.y < 0) return;
+            seq = rw.x; pos = rw.y; kvf = __ldg(e.kvflag + m);
+        } else {
+            seq = m / e.max_rows;
+            const int i = m - seq * e.max_rows;
+            if (i >= __ldg(e.counts + seq)) return;
+            pos = __ldg(e.idx + seq * e.max_rows + i); kvf = 1;
+        }
+        const int dq = e.n_heads * e.head_dim, dkv = e.n_kv * e.head_dim;
+        const int Npos = (EPI == EPI_QKV) ? e.N_seq : e.P;
+        if (n < dq + dkv) {
+            if (n < dq ? e.q_out == nullptr : !kvf) return;
+            const int hd1 = e.head_dim - 1;
+            const int p = (e.head_dim & hd1) ? n % e.head_dim : (n & hd1);
+            const float4* cs = reinterpret_cast<const float4*>(e.rope + (size_t)pos * (e.head_dim / 2) + (p >> 1));
+            float r[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float4 c = __ldg(cs + i);          // (cos, sin) of two pairs
+                r[4 * i] = v[4 * i] * c.x - v[4 * i + 1] * c.y;
+                r[4 * i + 1] = v[4 * i + 1] * c.x + v[4 * i] * c.y;
+                r[4 * i + 2] = v[4 * i + 2] * c.z - v[4 * i + 3] * c.w;
+                r[4 * i + 3] = v[4 * i + 3] * c.z + v[4 * i + 2] * c.w;
+            }
+            if (n < dq) store16<T>((T*)e.q_out + (size_t)m * dq + n, r);
+            else store16<T>((T*)e.kc + ((size_t)seq * Npos + pos) * dkv + (n - dq), r);
+        } else if (kvf) {
+            store16<T>((T*)e.vc + ((size_t)seq * Npos + pos) * dkv + (n - dq - dkv), v);
+        }
+    } else if (EPI == EPI_RESID) {
+        const size_t o = (size_t)m * e.ld_out + n;
+        float r[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 c = __ldg(reinterpret_cast<const float4*>(e.resid + o) + i);
+            r[4 * i] = c.x + v[4 * i]; r[4 * i + 1] = c.y + v[4 * i + 1]; r[4 * i + 2] = c.z + v[4 * i + 2]; r[4 * i + 3] = c.w + v[4 * i + 3];
+        }
+        store16<float>(e.out_f32 + o, r);
+    } else if (EPI == EPI_SWIGLU) {
+        float gl[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) gl[i] = v[2 * i] / (1.f + expf(-v[2 * i])) * v[2 * i + 1];
+        store8<T>((T*)e.out_t + (size_t)m * e.ld_out + (n >> 1), gl);
+    } else if (EPI == EPI_DOWN) {
+        const int r0 = e.list ? __ldg(e.list + m) : m;
+        const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + r0);       // {seq, pos, widx, aidx}
+        if (rw.y < 0) return;
+        const size_t o = (size_t)r0 * e.ld_out + n;
+        float r[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 c = __ldg(reinterpret_cast<const float4*>(e.resid + o) + i);
+            r[4 * i] = c.x + v[4 * i]; r[4 * i + 1] = c.y + v[4 * i + 1]; r[4 * i + 2] = c.z + v[4 * i + 2]; r[4 * i + 3] = c.w + v[4 * i + 3];
+        }
+        float* dst = (e.within && rw.z >= 0) ? e.packet + ((size_t)rw.x * e.W_max + rw.z) * e.ld_out + n : e.out_f32 + o;
+        store16<float>(dst, r);
+    } else if (EPI == EPI_LOGITS) {
+        float r[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r[i] = v[i] * e.scale;
+        store16<float>(e.out_f32 + (size_t)m * e.ld_out + n, r);
+    }
+}
+
 // Prefetch into L1 what epilogue_pair will read for the 16 outputs n .. n+15 of row m (row descriptor,
 // RoPE entries, residual values), so that the epilogue after a wait starts on cache hits.
 __device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }

@@ -417,8 +417,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         float v[16];
                         tmem_ld16(taddr + (uint32_t)c0, v);
                         if (live) {
-#pragma unroll
-                            for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, m, n0 + c0 + c, v[c], v[c + 1]);
+                            epilogue16<T, EPI>(e, m, n0 + c0, v);
                         }
                     }
                 }
@@ -564,8 +563,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                     const int mm = (tile % g.tiles_t) * BLOCK_T + tl;
                     const int n0 = (tile / g.tiles_t) * BLOCK_F;
-#pragma unroll
-                    for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, mm, n0 + c0 + c, acc[c], acc[c + 1]);
+                    epilogue16<T, EPI>(e, mm, n0 + c0, acc);
                 }
             }
             if (threadIdx.x == 64) SK_STAMP(8);
@@ -622,8 +620,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                         }
                 }
                 const int mm = tile_t * BLOCK_T + tl;
-#pragma unroll
-                for (int c = 0; c < 16; c += 2) epilogue_pair<T, EPI>(e, mm, n0 + c0 + c, acc[c], acc[c + 1]);
+                epilogue16<T, EPI>(e, mm, n0 + c0, acc);
             }
         }
         cluster_sync_all();       // nobody leaves while its partial tile may still be read
