@@ -341,7 +341,10 @@ __global__ void __launch_bounds__(AT_WARPS * 32) attention_mma_kernel(AttnMmaArg
 // ------------------------------------------------------------------------------------------
 constexpr int SP_SLOT_BYTES = AT_BN * AT_DH * 2;     // one K or V tile: 8 KB
 
-template <int NW, int TPW>
+// CL = 2: the keys of one (row tile, head) are split over a cluster of two CTAs (few rows: more SMs pull K/V,
+// and each warp's K and V tile are all in flight from the start).  The two CTAs exchange their rows'
+// (max, sum), partial KL and partial outputs through distributed shared memory; rank 0 writes the results.
+template <int NW, int TPW, int CL>
 __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
     KERNEL_PROLOGUE(7);   // __launch_bounds__
     extern __shared__ uint8_t at_smem_raw[];
@@ -349,10 +352,14 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
     __shared__ float lse_sh[AT_BM];
     __shared__ float* prev_sh[AT_BM];
     __shared__ int valid_sh[AT_BM];
+    __shared__ float2 cl_ml[AT_BM];       // CL = 2: this CTA's (max, sum) per row
+    __shared__ float cl_kl[AT_BM];
     const AttnArgs& a = g.a;
     uint8_t* smem = (uint8_t*)(((uintptr_t)at_smem_raw + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int seq = blockIdx.x / g.tiles_per_seq, tile = blockIdx.x - seq * g.tiles_per_seq;
+    const int rank = CL > 1 ? (int)cluster_rank() : 0;
+    const int bx = CL > 1 ? blockIdx.x / CL : blockIdx.x;
+    const int seq = bx / g.tiles_per_seq, tile = bx - seq * g.tiles_per_seq;
     const int h = blockIdx.y;
     const int g_kv = (h * a.n_kv) / a.n_heads;
     const int dq = a.n_heads * AT_DH, dkv = a.n_kv * AT_DH;
@@ -367,12 +374,15 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
     const __nv_bfloat16* Kg = (const __nv_bfloat16*)a.kc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
     const __nv_bfloat16* Vg = (const __nv_bfloat16*)a.vc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
     const int n_tiles = (a.N + AT_BN - 1) / AT_BN;
-    const int my_tiles = warp < n_tiles ? min(TPW, (n_tiles - warp + NW - 1) / NW) : 0;
+    // key tile of (warp, i): warp + (i * CL + rank) * NW
+    int my_tiles = 0;
+#pragma unroll
+    for (int i = 0; i < TPW; ++i) my_tiles += (warp + (i * CL + rank) * NW < n_tiles) ? 1 : 0;
     const int n_loads = a.out ? 2 * my_tiles : my_tiles;
 
     auto issue = [&](int j) {      // load j of this warp's sequence into slot j & 1
         const bool is_v = j >= my_tiles;
-        const int t = warp + (is_v ? j - my_tiles : j) * NW;
+        const int t = warp + ((is_v ? j - my_tiles : j) * CL + rank) * NW;
         const __nv_bfloat16* src = is_v ? Vg : Kg;
         const uint32_t dst = ring + (j & 1) * SP_SLOT_BYTES;
         const int key0 = t * AT_BN;
@@ -454,7 +464,7 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
             }
             __syncwarp();
             if (i + 2 < n_loads) issue(i + 2);
-            const int t = warp + i * NW;
+            const int t = warp + (i * CL + rank) * NW;
 #pragma unroll
             for (int nt = 0; nt < 4; ++nt) {
 #pragma unroll
@@ -496,7 +506,22 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
         float sum = 0.f;
         for (int w = 0; w < NW; ++w)
             if (red_l[w][i] > 0.f) sum += red_l[w][i] * fast_exp2(red_m[w][i] - mx);
-        lse_sh[i] = mx + log2f(sum);            // log2 domain
+        if (CL > 1) cl_ml[i] = make_float2(mx, sum);
+        else lse_sh[i] = mx + log2f(sum);       // log2 domain
+    }
+    if (CL > 1) {
+        cluster_sync_all();
+        if (threadIdx.x < AT_BM) {
+            // both CTAs combine the two halves in rank order, so both get the same value
+            const int i = threadIdx.x;
+            const uint32_t mine = (uint32_t)__cvta_generic_to_shared(&cl_ml[i]);
+            const float2 h0 = ld_dsmem_f2(dsmem_addr(mine, 0)), h1 = ld_dsmem_f2(dsmem_addr(mine, 1));
+            const float mx = fmaxf(h0.x, h1.x);
+            float sum = 0.f;
+            if (h0.y > 0.f) sum += h0.y * fast_exp2(h0.x - mx);
+            if (h1.y > 0.f) sum += h1.y * fast_exp2(h1.x - mx);
+            lse_sh[i] = mx + log2f(sum);
+        }
     }
     __syncthreads();
     const float lse_lo = lse_sh[r_lo], lse_hi = lse_sh[r_hi];
@@ -512,7 +537,7 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
 #pragma unroll
     for (int i = 0; i < TPW; ++i) {
         if (i < my_tiles) {
-            const int t = warp + i * NW;
+            const int t = warp + (i * CL + rank) * NW;
             // stored rows of this tile: all loads first
             float pv_lo[4][2], pv_hi[4][2];
 #pragma unroll
@@ -602,6 +627,50 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
         }
     }
     __syncthreads();
+    float* o_red = reinterpret_cast<float*>(smem + NW * 2 * SP_SLOT_BYTES + AT_BM * AT_DH * 2);   // CL = 2: [16][128] fp32
+    if (CL > 1) {
+        // each CTA adds up its warps; rank 0 then adds the two CTAs (rank order) and writes
+        if (a.out) {
+            for (int t = threadIdx.x; t < AT_BM * AT_DH / 2; t += blockDim.x) {
+                const int i = t / (AT_DH / 2), c = (t % (AT_DH / 2)) * 2;
+                float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+                for (int w = 0; w < NW; ++w) {
+                    const float2 v = *reinterpret_cast<const float2*>(o_s + ((size_t)w * AT_BM + i) * AT_DH + c);
+                    v0 += v.x; v1 += v.y;
+                }
+                *reinterpret_cast<float2*>(o_red + i * AT_DH + c) = make_float2(v0, v1);
+            }
+        }
+        if (threadIdx.x < AT_BM) {
+            float kl = 0.f;
+            for (int w = 0; w < NW; ++w) kl += red_kl[w][threadIdx.x];
+            cl_kl[threadIdx.x] = kl;
+        }
+        cluster_sync_all();
+        if (rank == 0) {
+            if (a.out) {
+                const uint32_t peer = dsmem_addr((uint32_t)__cvta_generic_to_shared(o_red), 1);
+                for (int t = threadIdx.x; t < AT_BM * AT_DH / 2; t += blockDim.x) {
+                    const int i = t / (AT_DH / 2), c = (t % (AT_DH / 2)) * 2;
+                    if (!valid_sh[i]) continue;
+                    const float2 v0 = *reinterpret_cast<const float2*>(o_red + i * AT_DH + c);
+                    const float2 v1 = ld_dsmem_f2(peer + (uint32_t)((i * AT_DH + c) * 4));
+                    *reinterpret_cast<__nv_bfloat162*>((__nv_bfloat16*)a.out + (size_t)(row0 + i) * dq + h * AT_DH + c) =
+                        __floats2bfloat162_rn(v0.x + v1.x, v0.y + v1.y);
+                }
+            }
+            if (a.kl && threadIdx.x < AT_BM && valid_sh[threadIdx.x]) {
+                const int i = threadIdx.x;
+                float other;
+                asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(other)
+                             : "r"(dsmem_addr((uint32_t)__cvta_generic_to_shared(&cl_kl[i]), 1)) : "memory");
+                a.kl[(size_t)(row0 + i) * a.n_heads + h] = (prev_sh[i] && a.record_kl) ? cl_kl[i] + other : 0.f;
+            }
+        }
+        cluster_sync_all();       // rank 1 stays until rank 0 has read its shared memory
+        return;
+    }
     if (a.out) {
         for (int t = threadIdx.x; t < AT_BM * AT_DH / 2; t += blockDim.x) {
             const int i = t / (AT_DH / 2), c = (t % (AT_DH / 2)) * 2;
@@ -848,16 +917,20 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
     }
 }
 
-template <int NW, int TPW>
+template <int NW, int TPW, int CL = 1>
 static int launch_attention_sp(const AttnMmaArgs& g, dim3 grid, cudaStream_t st) {
-    constexpr int smem = NW * 2 * SP_SLOT_BYTES + AT_BM * AT_DH * 2 + 1024;
+    constexpr int smem = NW * 2 * SP_SLOT_BYTES + AT_BM * AT_DH * 2 + (CL > 1 ? AT_BM * AT_DH * 4 : 0) + 1024;
     static bool attr = false;
     if (!attr) {
-        if (cudaFuncSetAttribute(attention_sp_kernel<NW, TPW>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(attention_sp_kernel<NW, TPW, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return -4;
         attr = true;
     }
-    return launch_k(attention_sp_kernel<NW, TPW>, grid, dim3(NW * 32), smem, st, g) == cudaSuccess ? 0 : -4;
+    if (CL > 1) {
+        grid.x *= CL;
+        return launch_k_cluster(attention_sp_kernel<NW, TPW, CL>, grid, dim3(NW * 32), smem, st, (unsigned)CL, g) == cudaSuccess ? 0 : -4;
+    }
+    return launch_k(attention_sp_kernel<NW, TPW, CL>, grid, dim3(NW * 32), smem, st, g) == cudaSuccess ? 0 : -4;
 }
 
 static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count = 148) {
@@ -869,7 +942,7 @@ static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count
     dim3 grid(g.tiles_per_seq * batch, a.n_heads);
     const long long ctas = (long long)grid.x * grid.y;
     const char* force = getenv("POLESTAR_ATTN_KERNEL");
-    const int mode = force ? atoi(force) : 0;      // 0 auto, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>, 5 many-rows
+    const int mode = force ? atoi(force) : 0;      // 0 auto, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>, 5 many-rows, 6 / 7 key split over two CTAs
     // many rows per head (entry forwards, long sequences): share each K/V tile among 64 rows
     const long long big_ctas = (long long)((g.rows_per_seq + BG_BM - 1) / BG_BM) * batch * a.n_heads;
     if (mode == 5 || (mode == 0 && (a.N > 8 * 4 * AT_BN || ctas >= 4LL * sm_count) && g.rows_per_seq >= 48 && big_ctas >= sm_count)) {
@@ -884,6 +957,9 @@ static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count
         return launch_k(attention_big_kernel, dim3(gb.tiles_per_seq * batch, a.n_heads), dim3(BG_WARPS * 32), BG_SMEM, st, gb) == cudaSuccess ? 0 : -4;
     }
     if (mode != 1) {
+        // few rows: split the keys of every (row tile, head) over a cluster of two CTAs
+        if ((mode == 6 || (mode == 0 && 2 * ctas <= sm_count)) && a.N <= 2 * 8 * AT_BN) return launch_attention_sp<8, 1, 2>(g, grid, st);
+        if ((mode == 7 || (mode == 0 && 2 * ctas <= sm_count)) && a.N <= 2 * 8 * 2 * AT_BN) return launch_attention_sp<8, 2, 2>(g, grid, st);
         if ((mode == 2 || (mode == 0 && ctas <= 2LL * sm_count)) && a.N <= 8 * 2 * AT_BN) return launch_attention_sp<8, 2>(g, grid, st);
         if ((mode == 3 || mode == 0) && a.N <= 4 * 4 * AT_BN) return launch_attention_sp<4, 4>(g, grid, st);
         if ((mode == 4 || mode == 0) && a.N <= 8 * 4 * AT_BN) return launch_attention_sp<8, 4>(g, grid, st);

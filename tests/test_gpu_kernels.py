@@ -40,6 +40,9 @@ def test_attention_drift_matches_oracle(dtype, R, N, nh, nkv, dh):
     (5, 150, 1100, 2, 1),          # 64-row tiles: three row tiles (last ragged), 18 key tiles (last ragged)
     (5, 5, 37, 2, 2),              # 64-row tiles, fewer rows and keys than one tile
     (0, 200, 2048, 8, 8),          # automatic choice at a long sequence
+    (6, 32, 512, 4, 4), (6, 21, 300, 4, 2), (6, 5, 37, 2, 2),        # keys split over a cluster of two CTAs
+    (7, 32, 1000, 2, 1), (7, 16, 512, 2, 2),
+    (0, 32, 512, 2, 2),            # automatic choice for one block of rows
 ])
 def test_attention_kernel_variants(monkeypatch, variant, R, N, nh, nkv):
     monkeypatch.setenv("POLESTAR_ATTN_KERNEL", str(variant))
