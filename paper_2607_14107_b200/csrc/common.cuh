@@ -385,6 +385,24 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int n, const
     }
 }
 
+// Four outputs n .. n+3 (n % 4 == 0) of row m for the two residual epilogues (same arithmetic as epilogue16).
+template <typename T, int EPI>
+__device__ __forceinline__ void epilogue4(const EpiArgs& e, int m, int n, float4 v) {
+    if (EPI == EPI_RESID) {
+        const size_t o = (size_t)m * e.ld_out + n;
+        const float4 c = __ldg(reinterpret_cast<const float4*>(e.resid + o));
+        *reinterpret_cast<float4*>(e.out_f32 + o) = make_float4(c.x + v.x, c.y + v.y, c.z + v.z, c.w + v.w);
+    } else if (EPI == EPI_DOWN) {
+        const int r0 = e.list ? __ldg(e.list + m) : m;
+        const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + r0);       // {seq, pos, widx, aidx}
+        if (rw.y < 0) return;
+        const size_t o = (size_t)r0 * e.ld_out + n;
+        const float4 c = __ldg(reinterpret_cast<const float4*>(e.resid + o));
+        float* dst = (e.within && rw.z >= 0) ? e.packet + ((size_t)rw.x * e.W_max + rw.z) * e.ld_out + n : e.out_f32 + o;
+        *reinterpret_cast<float4*>(dst) = make_float4(c.x + v.x, c.y + v.y, c.z + v.z, c.w + v.w);
+    }
+}
+
 // Prefetch into L1 what epilogue_pair will read for the 16 outputs n .. n+15 of row m (row descriptor,
 // RoPE entries, residual values), so that the epilogue after a wait starts on cache hits.
 __device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }

@@ -511,7 +511,34 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 SK_STAMP(6);
             }
             __syncthreads();
-            if (last_sh) {
+            if ((EPI == EPI_RESID || EPI == EPI_DOWN) && last_sh && max(f_nseg[0], f_nseg[1]) > 4) {
+                // Many contributors per tile (few output tiles): four threads share an item, each owning four
+                // columns, so that one float4 per contributor is in flight for all contributors at once (one
+                // round trip to L2 instead of one per group of four contributors).  Same summation order.
+                for (int i4 = (int)threadIdx.x; i4 < 4 * total; i4 += FIX_THREADS) {
+                    const int i = i4 >> 2;
+                    const int f = i < f_n[0] ? 0 : 1;
+                    const int item = f_lo[f] + i - (f ? f_n[0] : 0);
+                    const int tile = fix_tile[f];
+                    const int c_lo = f_clo[f], nseg = f_nseg[f];
+                    const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16 + (i4 & 3) * 4;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int sg0 = 0; sg0 < nseg; sg0 += 16) {
+                        float4 tv[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int cc = c_lo + sg0 + j;
+                            const int wsl = (cc == c_lo) ? 1 : 0;
+                            tv[j] = (sg0 + j < nseg)
+                                        ? __ldcg(reinterpret_cast<const float4*>(g.partial + ((size_t)(2 * cc + wsl) * BLOCK_T + tl) * BLOCK_F + c0))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { acc.x += tv[j].x; acc.y += tv[j].y; acc.z += tv[j].z; acc.w += tv[j].w; }
+                    }
+                    epilogue4<T, EPI>(e, (tile % g.tiles_t) * BLOCK_T + tl, (tile / g.tiles_t) * BLOCK_F + c0, acc);
+                }
+            } else if (last_sh) {
                 for (int i = (int)threadIdx.x; i < total; i += FIX_THREADS) {
                     const int f = i < f_n[0] ? 0 : 1;
                     const int item = f_lo[f] + i - (f ? f_n[0] : 0);
