@@ -257,6 +257,28 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
 
+    if (threadIdx.x == THREADS + 32 && (g.pf[0].count > 0 || g.pf[1].count > 0) && n_units > 0) {
+        // Optional L2 prefetch of the weights later GEMMs will stream, by an otherwise idle thread, once this CTA's
+        // last accumulator is complete (its own stream has ended, so the prefetch competes with nothing of ours).
+        const int n_seg = (int)((u_end - 1) / kb_total - u_begin / kb_total) + 1;
+        const int last = n_seg - 1;
+        if (mbar_wait(accum_full + 8 * (last & 1), (uint32_t)(last >> 1) & 1u, abort_flag)) {
+            uint64_t pol_keep;
+            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                if (g.pf[j].count > 0 && cta < g.pf[j].G) {
+                    const long long nb = sk_begin(g.pf[j].U, g.pf[j].G, cta) + g.pf[j].first;
+                    const long long ne = sk_begin(g.pf[j].U, g.pf[j].G, cta + 1);
+                    const int n = (int)max(0LL, min((long long)g.pf[j].count, ne - nb));
+                    for (int i = 0; i < n; ++i) {
+                        const char* src = g.pf[j].w + (size_t)(nb + i) * W_BYTES;
+                        asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src), "r"(W_BYTES), "l"(pol_keep) : "memory");
+                    }
+                }
+            }
+        }
+    }
     if (threadIdx.x == THREADS) {
         // An idle thread works out, while the main loop runs, which partial tiles this CTA will help reduce and
         // which share of their items is its own (64-bit divisions that must not sit on the tail's critical path).
@@ -324,19 +346,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (g.w_stream) tma_load_2d_hint(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F, pol);
                 else tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
                 tma_load_2d(dst, &map_a, full0 + 8 * s, kb * BLOCK_K, (tile % g.tiles_t) * BLOCK_T);
-            }
-            // all of this CTA's loads are requested: start pulling the next GEMMs' weights into L2
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                if (g.pf[j].count > 0 && cta < g.pf[j].G) {
-                    const long long nb = sk_begin(g.pf[j].U, g.pf[j].G, cta) + g.pf[j].first;
-                    const long long ne = sk_begin(g.pf[j].U, g.pf[j].G, cta + 1);
-                    const int n = (int)max(0LL, min((long long)g.pf[j].count, ne - nb));
-                    for (int i = 0; i < n; ++i) {
-                        const char* src = g.pf[j].w + (size_t)(nb + i) * W_BYTES;
-                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(W_BYTES) : "memory");
-                    }
-                }
             }
         }
     } else if (warp == 1) {

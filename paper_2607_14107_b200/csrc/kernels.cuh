@@ -556,23 +556,19 @@ struct StepSelArgs {
     float thresh, floor_;
 };
 
+// One CTA per sequence; the CTA that finishes last (arrival counter a.stats[3], left at zero again) builds the
+// compacted row list from all sequences' selections.
 __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, StepSelArgs a) {
     KERNEL_PROLOGUE(7);   // __launch_bounds__
     __shared__ SelSmem s;
     __shared__ float dsh[SEL_MAX_W > 1024 ? 1024 : SEL_MAX_W];
     __shared__ int sel_sh[SEL_SMALL_W];
-    __shared__ int base;
+    __shared__ int offs[65];
+    __shared__ int last_sh;
     const int t = threadIdx.x;
-    const int nb = sd.batch * sd.B;
-    // active rows first (row id = s*rows_per_seq + j)
-    for (int i = t; i < nb; i += blockDim.x) a.list[i] = (i / sd.B) * sd.rows_per_seq + (i % sd.B);
-    if (t == 0) base = nb;
-    __syncthreads();
-    for (int sq = 0; sq < sd.batch; ++sq) {
-        if (!sd.refresh.v[sq]) {
-            if (t == 0) a.sel_cnt[sq] = 0;
-            continue;
-        }
+    const int sq = blockIdx.x;
+    int cnt = 0;
+    if (sd.refresh.v[sq]) {
         for (int w = t; w < sd.W; w += blockDim.x) {
             const float* kr = a.kl + (size_t)(sq * sd.rows_per_seq + sd.B + w) * a.n_heads;
             float acc = 0.f;
@@ -584,25 +580,47 @@ __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, S
         __syncthreads();
         int* idx = a.sel_idx + sq * a.W_max;
         unsigned char* fl = a.flag_next + sq * a.W_max;
-        int cnt;
         const int fc = a.forced_cnt ? a.forced_cnt[sq] : -1;
         if (fc >= 0) {
             for (int w = t; w < sd.W; w += blockDim.x) fl[w] = 0;
             __syncthreads();
             for (int i = t; i < fc; i += blockDim.x) { const int w = a.forced_idx[sq * a.W_max + i]; idx[i] = w; fl[w] = 1; }
             cnt = fc;
-            __syncthreads();
         } else {
             cnt = sd.W <= SEL_SMALL_W ? select_small(dsh, sd.W, a.mode, a.k, a.thresh, a.floor_, idx, fl, sel_sh)
                                       : select_one(dsh, sd.W, a.mode, a.k, a.thresh, a.floor_, idx, fl, s);
         }
-        const int b0 = base;
-        for (int i = t; i < cnt; i += blockDim.x) a.list[b0 + i] = sq * sd.rows_per_seq + sd.B + idx[i];
-        __syncthreads();
-        if (t == 0) { a.sel_cnt[sq] = cnt; base = b0 + cnt; atomicAdd(a.stats, cnt); }
-        __syncthreads();
     }
-    if (t == 0) *a.list_count = base;
+    __syncthreads();
+    if (t == 0) {
+        a.sel_cnt[sq] = cnt;
+        int last = 1;
+        if (sd.batch > 1) {
+            __threadfence();
+            last = atomicAdd(a.stats + 3, 1) == sd.batch - 1;
+            __threadfence();
+        }
+        last_sh = last;
+    }
+    __syncthreads();
+    if (!last_sh) return;
+    // compacted row list of the sparse forward: all active rows (row id = s*rows_per_seq + j), then the selected
+    // window rows sequence by sequence
+    const int nb = sd.batch * sd.B;
+    if (t == 0) {
+        int base = nb;
+        for (int q = 0; q < sd.batch; ++q) { offs[q] = base; base += __ldcg(a.sel_cnt + q); }
+        offs[sd.batch] = base;
+        *a.list_count = base;
+        atomicAdd(a.stats, base - nb);
+        a.stats[3] = 0;
+    }
+    for (int i = t; i < nb; i += blockDim.x) a.list[i] = (i / sd.B) * sd.rows_per_seq + (i % sd.B);
+    __syncthreads();
+    for (int q = 0; q < sd.batch; ++q) {
+        const int b0 = offs[q], n = offs[q + 1] - b0;
+        for (int i = t; i < n; i += blockDim.x) a.list[b0 + i] = q * sd.rows_per_seq + sd.B + __ldcg(a.sel_idx + q * a.W_max + i);
+    }
 }
 
 // ---------------------------------------------------------------------------------------

@@ -542,7 +542,7 @@ struct Path {
                 s.mode = p.select_mode;
                 s.k = p.select_mode == POLESTAR_SELECT_TOPK_FRAC ? (int)floorf(p.select_frac * (float)sd.W + 0.5f) : p.select_k;
                 s.W_max = Wm; s.thresh = p.select_thresh; s.floor_ = p.drift_floor;
-                CK(launch_k(step_select_kernel, dim3(1), dim3(SEL_THREADS), 0, st, sd, s));
+                CK(launch_k(step_select_kernel, dim3(bs), dim3(SEL_THREADS), 0, st, sd, s));
                 CK(cudaGetLastError());
                 list = b.list; m2_count = b.list_count;
             }

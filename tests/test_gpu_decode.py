@@ -139,6 +139,15 @@ def test_c1b_bf16_norm_staging_inside_the_gemm_tail(monkeypatch):
     assert seen["refresh"] > 3
 
 
+@pytest.mark.parametrize("variant", ["0", "5"])
+def test_c1b_long_ragged_sequence(monkeypatch, variant):
+    # N = 1100 + 64 > 1024 keys: the two-pass attention kernel (automatic choice) and the 64-row-tile kernel
+    # (forced) inside the decoding loop; the prompt length is not a multiple of the block size
+    monkeypatch.setenv("POLESTAR_ATTN_KERNEL", variant)
+    seen = run_forced("c1b", 5, prompt_len=1100, gen_len=64, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["refresh"] >= 2
+
+
 def test_c1b_bf16_simt_gemm_path():
     run_forced("c1b", 6, tau_upd=-1, flags=I.FLAG_DEFAULT | Bd.FLAG_SIMT_GEMM)
 
