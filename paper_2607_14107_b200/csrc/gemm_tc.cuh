@@ -191,6 +191,21 @@ __device__ __forceinline__ int sk_owner(long long U, int G, long long u) {
     return c;
 }
 
+// Tile id -> (feature tile, token tile).  Ids run over chunks of RASTER_T token tiles: inside a chunk the token
+// tile varies fastest, then the feature tile.  The G tiles that the CTAs work on at the same time (consecutive
+// ids) then cover a compact block of the output, about sqrt(G) feature tiles x RASTER_T token tiles, so that
+// every operand tile fetched into L2 is used by many CTAs while it is there.
+constexpr int RASTER_T = 16;
+__device__ __forceinline__ void tile_ft(int tile, int tiles_f, int tiles_t, int& f, int& t) {
+    if (tiles_t <= RASTER_T) { f = tile / tiles_t; t = tile - f * tiles_t; return; }
+    const int per_chunk = tiles_f * RASTER_T;
+    const int chunk = tile / per_chunk;
+    const int local = tile - chunk * per_chunk;
+    const int tc = min(RASTER_T, tiles_t - chunk * RASTER_T);
+    f = local / tc;
+    t = chunk * RASTER_T + (local - f * tc);
+}
+
 // Number of partial tile segments in CTA c's unit range (0, 1 or 2): what it has to publish and then help reduce.
 __device__ __forceinline__ int sk_partial_segments(long long U, int G, int c, int kb_total) {
     const long long b = sk_begin(U, G, c), e = sk_begin(U, G, c + 1);
@@ -215,7 +230,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __shared__ uint32_t tmem_base_sh;
     __shared__ int abort_sh;
     __shared__ int last_sh;
-    __shared__ int fx_par[2][6];          // per partial tile of this CTA: tile, c_lo, nseg, before, mine, w_all
+    __shared__ int fx_par[2][8];          // per partial tile of this CTA: tile, c_lo, nseg, before, mine, w_all, tile_f, tile_t
     __shared__ int fx_n;
     __shared__ volatile int fx_ready;
 
@@ -223,10 +238,18 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int G = gridDim.x, cta = blockIdx.x;
     if (threadIdx.x == 0) SK_STAMP(0);
     const int kb_total = g.K / BLOCK_K;
-    const long long U = (long long)g.tiles_f * g.tiles_t * kb_total;
+    // Schedule: with more tiles than CTAs, CTA c first takes the whole tiles c, c + G, c + 2G, ... (`dp` of them:
+    // at any time the grid works on G consecutive tile ids, see tile_ft), and the last G + (tiles mod G) tiles
+    // (all tiles, when there are fewer than G) are split stream-K: units (tile, k block) in contiguous ranges
+    // [u_begin, u_end) per CTA, whose partial tiles are reduced in the fix-up pass.  U, u_begin, u_end and the
+    // arithmetic derived from them count units of this stream-K part; its tiles have ids tile_base + u / kb_total.
+    const int tiles_all = g.tiles_f * g.tiles_t;
+    const int dp = (g.cluster_n > 0 || tiles_all < G) ? 0 : (tiles_all % G == 0 ? tiles_all / G : tiles_all / G - 1);
+    const int tile_base = dp * G;
+    const long long U = (long long)(tiles_all - tile_base) * kb_total;
     const long long u_begin = sk_begin(U, G, cta), u_end = sk_begin(U, G, cta + 1);
-    const int n_units = (int)(u_end - u_begin);
-    // tile index = tile_f * tiles_t + tile_t : token tiles of one feature tile are neighbours
+    const int n_tail = (int)(u_end - u_begin);
+    const int n_units = dp * kb_total + n_tail;
 
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
@@ -260,7 +283,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     if (threadIdx.x == THREADS + 32 && (g.pf[0].count > 0 || g.pf[1].count > 0) && n_units > 0) {
         // Optional L2 prefetch of the weights later GEMMs will stream, by an otherwise idle thread, once this CTA's
         // last accumulator is complete (its own stream has ended, so the prefetch competes with nothing of ours).
-        const int n_seg = (int)((u_end - 1) / kb_total - u_begin / kb_total) + 1;
+        const int n_seg = dp + (n_tail > 0 ? (int)((u_end - 1) / kb_total - u_begin / kb_total) + 1 : 0);
         const int last = n_seg - 1;
         if (mbar_wait(accum_full + 8 * (last & 1), (uint32_t)(last >> 1) & 1u, abort_flag)) {
             uint64_t pol_keep;
@@ -287,8 +310,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // A tile's items (one row x 16 columns each) are dealt to its contributors in contiguous shares; a CTA that
         // contributes to two tiles takes half a share of each, so that every CTA reduces about as many items.
         int n_fix = 0;
-        if (g.cluster_n == 0 && n_units > 0) {
-            const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;
+        if (g.cluster_n == 0 && n_tail > 0) {
+            const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;       // (stream-K part's own numbering)
             const bool head_cut = u_begin != tb * kb_total, tail_cut = u_end != (te + 1) * kb_total;
             int fix_tile[2] = {0, 0};
             if (tb == te) { if (head_cut || tail_cut) fix_tile[n_fix++] = (int)tb; }
@@ -303,10 +326,11 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int nseg = c_hi - c_lo + 1;
                 const int w_lo = sk_partial_segments(U, G, c_lo, kb_total) == 2 ? 1 : 2;
                 const int w_hi = (nseg > 1 && sk_partial_segments(U, G, c_hi, kb_total) == 2) ? 1 : 2;
-                fx_par[f][0] = tile; fx_par[f][1] = c_lo; fx_par[f][2] = nseg;
+                fx_par[f][0] = tile_base + tile; fx_par[f][1] = c_lo; fx_par[f][2] = nseg;
                 fx_par[f][3] = (cta == c_lo) ? 0 : w_lo + 2 * (cta - c_lo - 1);
                 fx_par[f][4] = (cta == c_lo) ? w_lo : (cta == c_hi ? w_hi : 2);
                 fx_par[f][5] = (nseg == 1) ? w_lo : w_lo + w_hi + 2 * (nseg - 2);
+                tile_ft(tile_base + tile, g.tiles_f, g.tiles_t, fx_par[f][6], fx_par[f][7]);
             }
         }
         fx_n = n_fix;
@@ -319,33 +343,49 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             // weights do not depend on the previous kernel: request the first stages right away
             const int pre = min(g.stages, n_units);
             const uint64_t pol = l2_policy_evict_first();
-            // (tile, kb) of a unit are advanced incrementally: no 64-bit division per unit on this thread
-            const int tile0 = (int)(u_begin / kb_total), kb0 = (int)(u_begin - (long long)tile0 * kb_total);
-            int tile = tile0, kb = kb0;
-            auto advance = [&](int& t, int& k) { if (++k == kb_total) { k = 0; ++t; } };
-            for (int i = 0; i < pre; ++i, advance(tile, kb)) {
+            // (tile, k block) of a unit are advanced incrementally: no 64-bit division per unit on this thread
+            const int tail_tile0 = (int)(u_begin / kb_total), tail_kb0 = (int)(u_begin - (long long)tail_tile0 * kb_total);
+            struct It { int j, tile, kb, f, t; };
+            auto start = [&]() {
+                It it;
+                it.j = 0;
+                if (dp > 0) { it.tile = cta; it.kb = 0; } else { it.tile = tile_base + tail_tile0; it.kb = tail_kb0; }
+                tile_ft(it.tile, g.tiles_f, g.tiles_t, it.f, it.t);
+                return it;
+            };
+            auto advance = [&](It& it) {
+                if (++it.kb == kb_total) {
+                    it.kb = 0;
+                    ++it.j;
+                    if (it.j < dp) it.tile = it.j * G + cta;
+                    else if (it.j == dp && dp > 0) { it.tile = tile_base + tail_tile0; it.kb = tail_kb0; }
+                    else ++it.tile;
+                    tile_ft(it.tile, g.tiles_f, g.tiles_t, it.f, it.t);
+                }
+            };
+            It iw = start();
+            for (int i = 0; i < pre; ++i, advance(iw)) {
                 mbar_expect_tx(full0 + 8 * i, STAGE_BYTES);
                 if (g.w_stream) tma_load_2d_hint(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
-                                                 ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F, pol);
-                else tma_load_2d(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
-                                 ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
+                                                 (iw.f * kb_total + iw.kb) * BLOCK_F, pol);
+                else tma_load_2d(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0, (iw.f * kb_total + iw.kb) * BLOCK_F);
             }
             pdl_wait();
             SK_STAMP(2);
             {
-                int ta = tile0, ka = kb0;
-                for (int i = 0; i < pre; ++i, advance(ta, ka))
-                    tma_load_2d(smem_base + i * STAGE_BYTES, &map_a, full0 + 8 * i, ka * BLOCK_K, (ta % g.tiles_t) * BLOCK_T);
+                It ia = start();
+                for (int i = 0; i < pre; ++i, advance(ia))
+                    tma_load_2d(smem_base + i * STAGE_BYTES, &map_a, full0 + 8 * i, ia.kb * BLOCK_K, ia.t * BLOCK_T);
             }
-            for (int i = pre; i < n_units; ++i, advance(tile, kb)) {
+            for (int i = pre; i < n_units; ++i, advance(iw)) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
                 const uint32_t dst = smem_base + s * STAGE_BYTES;
                 mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
-                if (g.w_stream) tma_load_2d_hint(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F, pol);
-                else tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, ((tile / g.tiles_t) * kb_total + kb) * BLOCK_F);
-                tma_load_2d(dst, &map_a, full0 + 8 * s, kb * BLOCK_K, (tile % g.tiles_t) * BLOCK_T);
+                if (g.w_stream) tma_load_2d_hint(dst + A_BYTES, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F, pol);
+                else tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F);
+                tma_load_2d(dst, &map_a, full0 + 8 * s, iw.kb * BLOCK_K, iw.t * BLOCK_T);
             }
         }
     } else if (warp == 1) {
@@ -353,8 +393,10 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const uint32_t idesc = instr_desc_bf16(BLOCK_T, BLOCK_F);
             int seg = 0;
             bool seg_start = true;
-            int kb = (int)(u_begin % kb_total);
-            for (int i = 0; i < n_units; ++i, kb = (kb + 1 == kb_total) ? 0 : kb + 1) {
+            const int tail_kb0 = (int)(u_begin % kb_total);
+            const int dp_units = dp * kb_total;
+            int kb = dp > 0 ? 0 : tail_kb0;
+            for (int i = 0; i < n_units; ++i, kb = (i == dp_units) ? tail_kb0 : ((kb + 1 == kb_total) ? 0 : kb + 1)) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (seg_start && seg > 1) {
@@ -391,13 +433,21 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
         int seg = 0;
         long long u = u_begin;
-        while (u < u_end) {
-            const int tile = (int)(u / kb_total);
-            const int k0 = (int)(u - (long long)tile * kb_total);
-            const long long tile_end = (long long)(tile + 1) * kb_total;
-            const long long seg_end = tile_end < u_end ? tile_end : u_end;
-            const int k1 = (int)(seg_end - (long long)tile * kb_total);
-            const int tile_f = tile / g.tiles_t, tile_t = tile % g.tiles_t;
+        for (int sgi = 0;; ++sgi) {
+            int tile, k0, k1;
+            if (sgi < dp) { tile = sgi * G + cta; k0 = 0; k1 = kb_total; }       // whole tiles first
+            else {
+                if (u >= u_end) break;
+                const int lt = (int)(u / kb_total);
+                k0 = (int)(u - (long long)lt * kb_total);
+                const long long tile_end = (long long)(lt + 1) * kb_total;
+                const long long seg_end = tile_end < u_end ? tile_end : u_end;
+                k1 = (int)(seg_end - (long long)lt * kb_total);
+                tile = tile_base + lt;
+                u = seg_end;
+            }
+            int tile_f, tile_t;
+            tile_ft(tile, g.tiles_f, g.tiles_t, tile_f, tile_t);
             const int m = tile_t * BLOCK_T + t_local;
             const int n0 = tile_f * BLOCK_F;
             const bool live = m < Mv;
@@ -466,7 +516,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile], 1);
             }
             ++seg;
-            u = seg_end;
         }
         if (threadIdx.x == 64) SK_STAMP(5);
     }
@@ -485,12 +534,14 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (n_fix > 0) {
             // inside the CTA the items of both tiles form one list for all its threads
             int fix_tile[2] = {0, 0}, f_lo[2] = {0, 0}, f_n[2] = {0, 0}, f_clo[2] = {0, 0}, f_nseg[2] = {1, 1};
+            int f_tf[2] = {0, 0}, f_tt[2] = {0, 0};
 #pragma unroll
             for (int f = 0; f < 2; ++f) {
                 if (f < n_fix) {
                     fix_tile[f] = fx_par[f][0]; f_clo[f] = fx_par[f][1]; f_nseg[f] = fx_par[f][2];
                     const int before = fx_par[f][3], mine = fx_par[f][4], w_all = fx_par[f][5];
-                    const int tile_t = fix_tile[f] % g.tiles_t;
+                    f_tf[f] = fx_par[f][6]; f_tt[f] = fx_par[f][7];
+                    const int tile_t = f_tt[f];
                     const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
                     const int n_items = n_live * (BLOCK_F / 16);
                     f_lo[f] = (n_items * before) / w_all;
@@ -503,8 +554,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int f = (int)threadIdx.x < f_n[0] ? 0 : 1;
                 const int item = f_lo[f] + (int)threadIdx.x - (f ? f_n[0] : 0);
                 const int tile = fix_tile[f];
-                epilogue_prefetch<T, EPI>(e, (tile % g.tiles_t) * BLOCK_T + item / (BLOCK_F / 16),
-                                          (tile / g.tiles_t) * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
+                epilogue_prefetch<T, EPI>(e, f_tt[f] * BLOCK_T + item / (BLOCK_F / 16), f_tf[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
             }
             if (threadIdx.x == 64) {
                 // bounded wait until all contributors have published their partial tiles
@@ -545,7 +595,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                         for (int j = 0; j < 16; ++j) { acc.x += tv[j].x; acc.y += tv[j].y; acc.z += tv[j].z; acc.w += tv[j].w; }
                     }
-                    epilogue4<T, EPI>(e, (tile % g.tiles_t) * BLOCK_T + tl, (tile / g.tiles_t) * BLOCK_F + c0, acc);
+                    epilogue4<T, EPI>(e, f_tt[f] * BLOCK_T + tl, f_tf[f] * BLOCK_F + c0, acc);
                 }
             } else if (last_sh) {
                 for (int i = (int)threadIdx.x; i < total; i += FIX_THREADS) {
@@ -583,8 +633,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
                             }
                     }
-                    const int mm = (tile % g.tiles_t) * BLOCK_T + tl;
-                    const int n0 = (tile / g.tiles_t) * BLOCK_F;
+                    const int mm = f_tt[f] * BLOCK_T + tl;
+                    const int n0 = f_tf[f] * BLOCK_F;
                     epilogue16<T, EPI>(e, mm, n0 + c0, acc);
                 }
             }
@@ -608,7 +658,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         cluster_sync_all();
         if (warp >= 2 && warp < 6 && !abort_sh) {
             const int tile = (int)(u_begin / kb_total);
-            const int tile_f = tile / g.tiles_t, tile_t = tile % g.tiles_t;
+            int tile_f, tile_t;
+            tile_ft(tile, g.tiles_f, g.tiles_t, tile_f, tile_t);
             const int n0 = tile_f * BLOCK_F;
             const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
             const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));

@@ -144,7 +144,11 @@ def test_select_zero_drift_and_nan():
 
 
 # ------------------------------------------------------------------ gathered refresh (a3 + a4)
-@pytest.mark.parametrize("P,d,nh,nkv,k,batch", [(256, 256, 2, 2, 37, 1), (512, 512, 4, 1, 128, 2), (300, 256, 2, 2, 300, 1)])
+@pytest.mark.parametrize("P,d,nh,nkv,k,batch", [
+    (256, 256, 2, 2, 37, 1), (512, 512, 4, 1, 128, 2), (300, 256, 2, 2, 300, 1),
+    (3400, 256, 2, 2, 3300, 4),       # 13200 rows: 312 output tiles > SM count (whole tiles round-robin + stream-K tail)
+    (2000, 256, 2, 2, 1700, 2),       # 3400 rows: 27 token tiles (two raster chunks), fewer tiles than SMs
+])
 def test_refresh_chain_matches_oracle(P, d, nh, nkv, k, batch):
     dh = 128
     h, drift = I.make_refresh_inputs(batch, P, d)
