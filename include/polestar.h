@@ -240,6 +240,12 @@ void polestar_destroy(polestar_ctx *c);
 const char *polestar_strerror(int code);
 
 /* ---- single kernels of the path (unit parity, micro-benchmarks) --------------------- */
+/* All pointers are device pointers owned by the caller; the calls are asynchronous on `cuda_stream`.
+ * Return POLESTAR_OK or a negative code (POLESTAR_E_INVAL for null pointers, negative sizes,
+ * unsupported shapes or misaligned buffers; POLESTAR_E_CUDA for a failed launch).  A call with zero
+ * rows (R, rows, batch or W = 0) is a valid no-op: it returns POLESTAR_OK, touches nothing (select with
+ * W = 0 writes zero counts) and accepts null row pointers. */
+
 
 /* Drift of attention rows (Eq. 4; Algorithm 1 "ProxyAttn" + "KL"), optionally with the attention
  * output: for each of R query rows and each head, logp = log softmax_j(q.k_j / sqrt(head_dim))

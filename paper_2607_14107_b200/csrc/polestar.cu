@@ -960,11 +960,12 @@ extern "C" int polestar_force(polestar_ctx* c, int32_t what, int32_t layer, cons
 extern "C" int polestar_k_attention(const void* q, const void* k, const void* v, float* logp_prev, float* kl, void* out,
                                     int32_t R, int32_t N, int32_t n_heads, int32_t n_kv, int32_t head_dim, int32_t dtype,
                                     void* stream) {
-    if (!q || !k || !v || R < 0 || N <= 0 || n_heads <= 0 || n_kv <= 0 || n_heads % n_kv || head_dim <= 0 || head_dim > 256)
+    if (R < 0 || N <= 0 || n_heads <= 0 || n_kv <= 0 || n_heads % n_kv || head_dim <= 0 || head_dim > 256)
         return POLESTAR_E_INVAL;
-    if (logp_prev && !kl) return POLESTAR_E_INVAL;
     if (dtype != POLESTAR_F32 && dtype != POLESTAR_BF16) return POLESTAR_E_INVAL;
-    if (R == 0) return POLESTAR_OK;
+    if (R == 0) return POLESTAR_OK;              // no rows: nothing to do (the row pointers may be null)
+    if (!q || !k || !v) return POLESTAR_E_INVAL;
+    if (logp_prev && !kl) return POLESTAR_E_INVAL;
     cudaStream_t st = (cudaStream_t)stream;
     AttnArgs a;
     memset(&a, 0, sizeof(a));
@@ -989,8 +990,10 @@ extern "C" int polestar_k_attention(const void* q, const void* k, const void* v,
 
 extern "C" int polestar_k_hidden_delta(const void* a, const void* b, float* out, int32_t rows, int32_t d, int32_t dtype,
                                        void* stream) {
-    if (!a || !b || !out || rows < 0 || d <= 0) return POLESTAR_E_INVAL;
+    if (rows < 0 || d <= 0) return POLESTAR_E_INVAL;
     if (dtype != POLESTAR_F32 && dtype != POLESTAR_BF16) return POLESTAR_E_INVAL;
+    if (rows == 0) return POLESTAR_OK;           // no rows: nothing to do (the pointers may be null)
+    if (!a || !b || !out) return POLESTAR_E_INVAL;
     const int per = dtype == POLESTAR_BF16 ? 8 : 4;
     if (d % per || (((uintptr_t)a | (uintptr_t)b) & 15)) return POLESTAR_E_INVAL;
     if (rows == 0) return POLESTAR_OK;
@@ -1008,8 +1011,14 @@ extern "C" int polestar_k_hidden_delta(const void* a, const void* b, float* out,
 
 extern "C" int polestar_k_select(const float* drift, int32_t batch, int32_t W, int32_t mode, int32_t k, float thresh,
                                  float floor_, int32_t* idx, int32_t* count, void* stream) {
-    if (!drift || !idx || !count || batch < 0 || W <= 0 || W > SEL_MAX_W || mode < 0 || mode > 4) return POLESTAR_E_INVAL;
+    if (batch < 0 || W < 0 || W > SEL_MAX_W || mode < 0 || mode > 4) return POLESTAR_E_INVAL;
     if (batch == 0) return POLESTAR_OK;
+    if (!count) return POLESTAR_E_INVAL;
+    if (W == 0) {                                 // no candidates: every count is zero (drift and idx may be null)
+        CK(cudaMemsetAsync(count, 0, (size_t)batch * sizeof(int32_t), (cudaStream_t)stream));
+        return POLESTAR_OK;
+    }
+    if (!drift || !idx) return POLESTAR_E_INVAL;
     select_kernel<<<batch, SEL_THREADS, 0, (cudaStream_t)stream>>>(drift, W, mode, k, thresh, floor_, idx, count);
     CK(cudaGetLastError());
     return POLESTAR_OK;
@@ -1077,7 +1086,9 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
 
 extern "C" int polestar_k_confidence(const float* logits, int32_t rows, int32_t vocab, int32_t mask_id, int32_t* yhat,
                                      float* conf, void* scratch, size_t scratch_bytes, void* stream) {
-    if (!logits || !yhat || !conf || !scratch || rows < 0 || vocab <= 0) return POLESTAR_E_INVAL;
+    if (rows < 0 || vocab <= 0) return POLESTAR_E_INVAL;
+    if (rows == 0) return POLESTAR_OK;           // no rows: nothing to do (the pointers may be null)
+    if (!logits || !yhat || !conf || !scratch) return POLESTAR_E_INVAL;
     if (scratch_bytes < (size_t)rows * CONF_CHUNKS * sizeof(ConfPart)) return POLESTAR_E_NOSPACE;
     if (rows == 0) return POLESTAR_OK;
     cudaStream_t st = (cudaStream_t)stream;

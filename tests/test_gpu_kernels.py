@@ -202,3 +202,43 @@ def test_confidence_matches_oracle(rows, V):
     ry, rc = O.confidence_rows(logits.numpy(), mask_id)
     assert yhat.cpu().tolist() == ry.tolist()
     assert np.allclose(conf.cpu().numpy(), rc, rtol=1e-4, atol=1e-7)
+
+
+# ------------------------------------------------------------------ empty inputs
+def test_empty_inputs_are_noops():
+    dev = "cuda"
+    cnt = torch.full((2,), -7, dtype=torch.int32, device=dev)
+    Bd.polestar_k_select(torch.zeros((2, 0), device=dev), I.SELECT_TOPK_COUNT, 3, 0.0, 0.0,
+                         torch.zeros((2, 0), dtype=torch.int32, device=dev), cnt)
+    assert cnt.tolist() == [0, 0]
+    drift = torch.rand(2, 100, device=dev)
+    idx = torch.full((2, 100), -7, dtype=torch.int32, device=dev)
+    Bd.polestar_k_select(drift, I.SELECT_TOPK_COUNT, 0, 0.0, 0.0, idx, cnt)          # budget 0
+    assert cnt.tolist() == [0, 0]
+    e = torch.zeros((0, 256), dtype=torch.bfloat16, device=dev)
+    Bd.polestar_k_hidden_delta(e, e, torch.zeros(0, device=dev))
+    Bd.polestar_k_confidence(torch.zeros((0, 1024), device=dev), 1023, torch.zeros(0, dtype=torch.int32, device=dev),
+                             torch.zeros(0, device=dev), torch.empty(4096, dtype=torch.uint8, device=dev))
+    k = torch.zeros((10, 256), dtype=torch.bfloat16, device=dev)
+    Bd.polestar_k_attention(e, k, k, None, None, torch.zeros((0, 256), dtype=torch.bfloat16, device=dev), 2, 2, 128)
+    with pytest.raises(Bd.PolestarError):                                             # no keys: softmax over nothing
+        Bd.polestar_k_attention(torch.zeros((4, 256), dtype=torch.bfloat16, device=dev), e, e, None, None,
+                                torch.zeros((4, 256), dtype=torch.bfloat16, device=dev), 2, 2, 128)
+    torch.cuda.synchronize()
+
+
+def test_refresh_with_zero_selected_rows_touches_nothing():
+    P, d, nh, nkv, dh, batch, k = 256, 256, 2, 2, 128, 2, 16
+    m = I.ModelCfg(1, d, nh, nkv, dh, 2 * d, 1024, I.DTYPE_BF16, 1e-5, 500000.0)
+    packed = Bd.pack_weights(m, I.make_weights(m, seed=5))
+    h, _ = I.make_refresh_inputs(batch, P, d)
+    kc0 = rnd((batch, P, nkv * dh), 8, 1.0, torch.bfloat16)
+    kc, vc = kc0.clone().cuda(), kc0.clone().cuda()
+    idx = torch.zeros((batch, k), dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(batch, dtype=torch.int32, device="cuda")                        # nothing selected
+    scratch = torch.empty(Bd.polestar_k_refresh_scratch_bytes(batch, k, d, nh, nkv, dh) + 1024, dtype=torch.uint8, device="cuda")
+    off = (-scratch.data_ptr()) % 1024
+    Bd.polestar_k_refresh(h.cuda(), idx, cnt, packed["wqkv"][0], packed["norm1"][0], kc, vc, None, k, nh, nkv, dh,
+                          m.rms_eps, m.rope_theta, scratch[off:])
+    torch.cuda.synchronize()
+    assert torch.equal(kc.cpu(), kc0) and torch.equal(vc.cpu(), kc0)
