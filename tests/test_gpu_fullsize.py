@@ -187,3 +187,26 @@ def test_c2_full_depth_default_mode_invariants(c2_full):
         prev = cur.copy()
     assert n_refresh >= 3
     gpu.destroy()
+
+
+def test_c2_full_depth_decode_is_bitwise_reproducible(c2_full):
+    # split tiles are reduced in a fixed order and no kernel uses floating-point atomics: two runs of the same
+    # decode give the same bits (also a guard against races in the partial-tile exchange)
+    m, p, packed = c2_full
+    prompt = I.make_prompt(m, p).numpy()
+    p = dataclasses.replace(p, max_steps=64, logit_scale=30.0, tau_upd=-1)
+    runs = []
+    for _ in range(2):
+        gpu = Bd.Polestar(m, packed, p, prompt)
+        trace = []
+        for step in range(6):
+            if step:
+                gpu.step()
+            trace.append((gpu.read(Bd.READ_LOGITS).copy(), gpu.read(Bd.READ_CONF).copy(), gpu.read(Bd.READ_DELTA).copy()))
+            gpu.commit()
+            trace.append((gpu.tokens().copy(),))
+        runs.append(trace)
+        gpu.destroy()
+    for a, b in zip(*runs):
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
