@@ -240,11 +240,13 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int kb_total = g.K / BLOCK_K;
     // Schedule: with more tiles than CTAs, CTA c first takes the whole tiles c, c + G, c + 2G, ... (`dp` of them:
     // at any time the grid works on G consecutive tile ids, see tile_ft), and the last G + (tiles mod G) tiles
-    // (all tiles, when there are fewer than G) are split stream-K: units (tile, k block) in contiguous ranges
+    // (or just the tiles mod G; all tiles, when there are fewer than G) are split stream-K: units (tile, k block) in contiguous ranges
     // [u_begin, u_end) per CTA, whose partial tiles are reduced in the fix-up pass.  U, u_begin, u_end and the
     // arithmetic derived from them count units of this stream-K part; its tiles have ids tile_base + u / kb_total.
     const int tiles_all = g.tiles_f * g.tiles_t;
-    const int dp = (g.cluster_n > 0 || tiles_all < G) ? 0 : (tiles_all % G == 0 ? tiles_all / G : tiles_all / G - 1);
+    // (the stream-K part is the remainder r = tiles mod G when that leaves at most ~8 CTAs per tile, else G + r tiles)
+    const int rem = tiles_all % G;
+    const int dp = (g.cluster_n > 0 || tiles_all < G) ? 0 : ((rem == 0 || rem * 8 >= G) ? tiles_all / G : tiles_all / G - 1);
     const int tile_base = dp * G;
     const long long U = (long long)(tiles_all - tile_base) * kb_total;
     const long long u_begin = sk_begin(U, G, cta), u_end = sk_begin(U, G, cta + 1);
