@@ -700,10 +700,21 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
 // 16.  Each warp keeps its rows' running max / sum (pass 1) and output accumulator (pass 2) in
 // registers; no cross-warp reduction is needed.
 // ------------------------------------------------------------------------------------------
-constexpr int BG_BM = 64, BG_BN = 64, BG_WARPS = 4;
-constexpr int BG_TILE_BYTES = BG_BN * AT_DH * 2;                  // 16 KB
-constexpr int BG_SMEM = BG_BM * AT_DH * 2 + 2 * 2 * BG_TILE_BYTES + 1024;
+constexpr int BG_BM = 64, BG_BN = 64, BG_WARPS = 4, BG_STAGES = 3;
+constexpr int BG_TILE_BYTES = BG_BN * AT_DH * 2;                  // 16 KB: one K or V tile
+constexpr int BG_SMEM = BG_STAGES * 2 * BG_TILE_BYTES + 1024;     // 97 KB: two CTAs per SM
 
+__device__ __forceinline__ void cp_async_wait_pending(int n) {    // at most n groups still in flight
+    if (n <= 0) cp_async_wait<0>();
+    else if (n == 1) cp_async_wait<1>();
+    else cp_async_wait<2>();
+}
+
+// K/V tiles go through a three-stage cp.async ring (two tiles ahead of the one being used); the Q tile
+// borrows the third stage until its fragments are in registers.  When no row of the launch records
+// attention rows (no stored rows, no KL) the kernel makes ONE pass with a running maximum: the output
+// accumulator is rescaled when the maximum grows and divided by the row sum at the end, so K is read
+// once.  Otherwise two passes (exact log-probabilities need the final row sum before anything is stored).
 __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArgs g) {
     KERNEL_PROLOGUE(7);
     extern __shared__ uint8_t at_smem_raw[];
@@ -718,17 +729,19 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
     const int dq = a.n_heads * AT_DH, dkv = a.n_kv * AT_DH;
     const int row0 = seq * g.rows_per_seq + tile * BG_BM;
     const int n_in_tile = min(BG_BM, g.rows_per_seq - tile * BG_BM);
-    uint8_t* q_s = smem;
+    const uint32_t st_u32 = (uint32_t)__cvta_generic_to_shared(smem);
+    uint8_t* q_s = smem + (BG_STAGES - 1) * 2 * BG_TILE_BYTES;       // borrowed: the last stage's K slot
     const uint32_t q_u32 = (uint32_t)__cvta_generic_to_shared(q_s);
-    const uint32_t st_u32 = q_u32 + BG_BM * AT_DH * 2;
     const int kv_seq = a.rows ? seq : 0;
     const __nv_bfloat16* Kg = (const __nv_bfloat16*)a.kc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
     const __nv_bfloat16* Vg = (const __nv_bfloat16*)a.vc + (size_t)kv_seq * a.N * dkv + g_kv * AT_DH;
     const int n_tiles = (a.N + BG_BN - 1) / BG_BN;
+    const bool record = (a.pprev != nullptr) || (a.aprev != nullptr);
+    const bool single = !record;
 
-    auto load_tile = [&](int t, int stage, bool with_v) {
+    auto load_tile = [&](int t, bool with_v) {
         const int key0 = t * BG_BN;
-        const uint32_t kb = st_u32 + stage * 2 * BG_TILE_BYTES, vb = kb + BG_TILE_BYTES;
+        const uint32_t kb = st_u32 + (t % BG_STAGES) * 2 * BG_TILE_BYTES, vb = kb + BG_TILE_BYTES;
         for (int c = threadIdx.x; c < BG_BN * 16; c += BG_WARPS * 32) {
             const int r = c >> 4, ch = c & 15;
             const int key = key0 + r;
@@ -739,7 +752,10 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
         }
         cp_async_commit();
     };
-    load_tile(0, 0, false);
+    // first pass of the ring: tiles 0 and 1 now, tile 2 once Q has left its stage
+    const bool v_first = single && a.out != nullptr;
+    load_tile(0, v_first);
+    if (n_tiles > 1) load_tile(1, v_first);
     for (int t = threadIdx.x; t < BG_BM * 16; t += blockDim.x) {
         const int i = t >> 4, ch = t & 15;
         uint4 v = make_uint4(0, 0, 0, 0);
@@ -774,12 +790,14 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
         const int i = lane >> 3, r = lane & 7;
         ldsm_x4(q_u32 + sw_off(warp * 16 + (i & 1) * 8 + r, 2 * k + (i >> 1)), qf[k][0], qf[k][1], qf[k][2], qf[k][3]);
     }
+    __syncthreads();                                    // Q is in registers: its stage joins the ring
+    if (n_tiles > 2) load_tile(2, v_first);
     const int r_lo = warp * 16 + (lane >> 2), r_hi = r_lo + 8;
     const int cpair = (lane & 3) * 2;
     const float scale2 = a.scale * LOG2E;
 
-    auto scores = [&](int stage, float (*s)[4]) {     // s[8][4]: 16 rows x 64 keys per warp, log2 domain, masked
-        const uint32_t kb = st_u32 + stage * 2 * BG_TILE_BYTES;
+    auto scores = [&](int t, float (*s)[4]) {     // s[8][4]: 16 rows x 64 keys per warp, raw q.k
+        const uint32_t kb = st_u32 + (t % BG_STAGES) * 2 * BG_TILE_BYTES;
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) { s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f; }
 #pragma unroll
@@ -794,111 +812,167 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
             }
         }
     };
-
-    // ---- pass 1: running max and sum (log2 domain) ---------------------------------------------------
-    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
-    for (int t = 0; t < n_tiles; ++t) {
-        if (t + 1 < n_tiles) { load_tile(t + 1, (t + 1) & 1, false); cp_async_wait<1>(); }
-        else cp_async_wait<0>();
-        __syncthreads();
-        float s[8][4];
-        scores(t & 1, s);
-        float tm_lo = -INFINITY, tm_hi = -INFINITY;
+    auto pv = [&](int t, const uint32_t (*pf)[4], float (*o)[4]) {      // o += P V for the 64 keys of tile t
+        const uint32_t vb = st_u32 + (t % BG_STAGES) * 2 * BG_TILE_BYTES + BG_TILE_BYTES;
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
+        for (int ks = 0; ks < 4; ++ks) {
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const bool ok = t * BG_BN + nt * 8 + cpair + e < a.N;
-                s[nt][e] = ok ? s[nt][e] * scale2 : -INFINITY;
-                s[nt][2 + e] = ok ? s[nt][2 + e] * scale2 : -INFINITY;
-                tm_lo = fmaxf(tm_lo, s[nt][e]); tm_hi = fmaxf(tm_hi, s[nt][2 + e]);
+            for (int dp = 0; dp < 8; ++dp) {
+                const int i = lane >> 3, r = lane & 7;
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(vb + sw_off(ks * 16 + (i & 1) * 8 + r, 2 * dp + (i >> 1)), b0, b1, b2, b3);
+                mma_bf16(o[2 * dp], pf[ks], b0, b1);
+                mma_bf16(o[2 * dp + 1], pf[ks], b2, b3);
             }
-        tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 1)); tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 2));
-        tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 1)); tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 2));
-        const float nm_lo = fmaxf(m_lo, tm_lo), nm_hi = fmaxf(m_hi, tm_hi);
-        float sl = 0.f, sh = 0.f;
-#pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) { sl += fast_exp2(s[nt][e] - nm_lo); sh += fast_exp2(s[nt][2 + e] - nm_hi); }
-        l_lo = l_lo * fast_exp2(m_lo - nm_lo) + sl;
-        l_hi = l_hi * fast_exp2(m_hi - nm_hi) + sh;
-        m_lo = nm_lo; m_hi = nm_hi;
+        }
+    };
+    // one step of the ring: request tile t + 2 (its stage was released at the end of step t - 1), wait for tile t
+    auto ring_step = [&](int t, bool with_v) {
+        if (t >= 1 && t + 2 < n_tiles) load_tile(t + 2, with_v);
+        cp_async_wait_pending(min(2, n_tiles - 1 - t));
         __syncthreads();
-    }
-    l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
-    l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-    const float lse_lo = m_lo + log2f(l_lo), lse_hi = m_hi + log2f(l_hi);
-    float* prev_lo = prev_sh[r_lo];
-    float* prev_hi = prev_sh[r_hi];
+    };
 
-    // ---- pass 2: logp, KL, stored rows, P V --------------------------------------------------------------
     float o[16][4];
 #pragma unroll
     for (int nt = 0; nt < 16; ++nt) { o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f; }
+    float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
     float kl_lo = 0.f, kl_hi = 0.f;
-    load_tile(0, 0, true);
-    for (int t = 0; t < n_tiles; ++t) {
-        if (t + 1 < n_tiles) { load_tile(t + 1, (t + 1) & 1, true); cp_async_wait<1>(); }
-        else cp_async_wait<0>();
-        __syncthreads();
-        float s[8][4];
-        scores(t & 1, s);
-        uint32_t pf[4][4];
+    float* prev_lo = prev_sh[r_lo];
+    float* prev_hi = prev_sh[r_hi];
+
+    if (single) {
+        // ---- one pass: running maximum, rescaled accumulator ---------------------------------------------
+        for (int t = 0; t < n_tiles; ++t) {
+            ring_step(t, a.out != nullptr);
+            float s[8][4];
+            scores(t, s);
+            float tm_lo = -INFINITY, tm_hi = -INFINITY;
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {            // two halves of 4 key groups keep the register count down
-            float pv_lo[4][2], pv_hi[4][2], lp_lo[4][2], lp_hi[4][2];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
-                    pv_lo[u][e] = (a.record_kl && prev_lo && key < a.N) ? prev_lo[key] : 0.f;
-                    pv_hi[u][e] = (a.record_kl && prev_hi && key < a.N) ? prev_hi[key] : 0.f;
-                }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int nt = hf * 4 + u;
-                float p[4];
+            for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
                     const bool ok = t * BG_BN + nt * 8 + cpair + e < a.N;
-                    const float d_lo = s[nt][e] * scale2 - lse_lo, d_hi = s[nt][2 + e] * scale2 - lse_hi;
-                    const float p_lo = ok ? fast_exp2(d_lo) : 0.f, p_hi = ok ? fast_exp2(d_hi) : 0.f;
-                    lp_lo[u][e] = d_lo * LN2; lp_hi[u][e] = d_hi * LN2;
-                    if (ok && a.record_kl) {
-                        if (prev_lo) kl_lo += p_lo * (lp_lo[u][e] - pv_lo[u][e]);
-                        if (prev_hi) kl_hi += p_hi * (lp_hi[u][e] - pv_hi[u][e]);
-                    }
-                    p[e] = p_lo; p[2 + e] = p_hi;
+                    s[nt][e] = ok ? s[nt][e] * scale2 : -INFINITY;
+                    s[nt][2 + e] = ok ? s[nt][2 + e] * scale2 : -INFINITY;
+                    tm_lo = fmaxf(tm_lo, s[nt][e]); tm_hi = fmaxf(tm_hi, s[nt][2 + e]);
+                }
+            tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 1)); tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 2));
+            tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 1)); tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 2));
+            const float nm_lo = fmaxf(m_lo, tm_lo), nm_hi = fmaxf(m_hi, tm_hi);
+            const float al_lo = fast_exp2(m_lo - nm_lo), al_hi = fast_exp2(m_hi - nm_hi);
+            uint32_t pf[4][4];
+            float sl = 0.f, sh = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt) {
+                float p[4];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    p[e] = fast_exp2(s[nt][e] - nm_lo); p[2 + e] = fast_exp2(s[nt][2 + e] - nm_hi);
+                    sl += p[e]; sh += p[2 + e];
                 }
                 pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
                 pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
             }
+            l_lo = l_lo * al_lo + sl; l_hi = l_hi * al_hi + sh;
+            m_lo = nm_lo; m_hi = nm_hi;
+            if (a.out) {
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+                for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= al_lo; o[nt][1] *= al_lo; o[nt][2] *= al_hi; o[nt][3] *= al_hi; }
+                pv(t, pf, o);
+            }
+            __syncthreads();
+        }
+        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+        const float il_lo = 1.f / l_lo, il_hi = 1.f / l_hi;
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) { o[nt][0] *= il_lo; o[nt][1] *= il_lo; o[nt][2] *= il_hi; o[nt][3] *= il_hi; }
+    } else {
+        // ---- pass 1: running max and sum (log2 domain) ---------------------------------------------------
+        for (int t = 0; t < n_tiles; ++t) {
+            ring_step(t, false);
+            float s[8][4];
+            scores(t, s);
+            float tm_lo = -INFINITY, tm_hi = -INFINITY;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
-                    if (prev_lo && key < a.N) prev_lo[key] = lp_lo[u][e];
-                    if (prev_hi && key < a.N) prev_hi[key] = lp_hi[u][e];
+                    const bool ok = t * BG_BN + nt * 8 + cpair + e < a.N;
+                    s[nt][e] = ok ? s[nt][e] * scale2 : -INFINITY;
+                    s[nt][2 + e] = ok ? s[nt][2 + e] * scale2 : -INFINITY;
+                    tm_lo = fmaxf(tm_lo, s[nt][e]); tm_hi = fmaxf(tm_hi, s[nt][2 + e]);
                 }
+            tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 1)); tm_lo = fmaxf(tm_lo, __shfl_xor_sync(0xffffffffu, tm_lo, 2));
+            tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 1)); tm_hi = fmaxf(tm_hi, __shfl_xor_sync(0xffffffffu, tm_hi, 2));
+            const float nm_lo = fmaxf(m_lo, tm_lo), nm_hi = fmaxf(m_hi, tm_hi);
+            float sl = 0.f, sh = 0.f;
+#pragma unroll
+            for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) { sl += fast_exp2(s[nt][e] - nm_lo); sh += fast_exp2(s[nt][2 + e] - nm_hi); }
+            l_lo = l_lo * fast_exp2(m_lo - nm_lo) + sl;
+            l_hi = l_hi * fast_exp2(m_hi - nm_hi) + sh;
+            m_lo = nm_lo; m_hi = nm_hi;
+            __syncthreads();
         }
-        if (a.out) {
-            const uint32_t vb = st_u32 + (t & 1) * 2 * BG_TILE_BYTES + BG_TILE_BYTES;
+        l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+        l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+        const float lse_lo = m_lo + log2f(l_lo), lse_hi = m_hi + log2f(l_hi);
+
+        // ---- pass 2: logp, KL, stored rows, P V ----------------------------------------------------------
+        const bool with_v = a.out != nullptr;
+        load_tile(0, with_v);
+        if (n_tiles > 1) load_tile(1, with_v);
+        if (n_tiles > 2) load_tile(2, with_v);
+        for (int t = 0; t < n_tiles; ++t) {
+            ring_step(t, with_v);
+            float s[8][4];
+            scores(t, s);
+            uint32_t pf[4][4];
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
+            for (int hf = 0; hf < 2; ++hf) {            // two halves of 4 key groups keep the register count down
+                float pv_lo[4][2], pv_hi[4][2], lp_lo[4][2], lp_hi[4][2];
 #pragma unroll
-                for (int dp = 0; dp < 8; ++dp) {
-                    const int i = lane >> 3, r = lane & 7;
-                    uint32_t b0, b1, b2, b3;
-                    ldsm_x4_t(vb + sw_off(ks * 16 + (i & 1) * 8 + r, 2 * dp + (i >> 1)), b0, b1, b2, b3);
-                    mma_bf16(o[2 * dp], pf[ks], b0, b1);
-                    mma_bf16(o[2 * dp + 1], pf[ks], b2, b3);
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
+                        pv_lo[u][e] = (a.record_kl && prev_lo && key < a.N) ? prev_lo[key] : 0.f;
+                        pv_hi[u][e] = (a.record_kl && prev_hi && key < a.N) ? prev_hi[key] : 0.f;
+                    }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int nt = hf * 4 + u;
+                    float p[4];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const bool ok = t * BG_BN + nt * 8 + cpair + e < a.N;
+                        const float d_lo = s[nt][e] * scale2 - lse_lo, d_hi = s[nt][2 + e] * scale2 - lse_hi;
+                        const float p_lo = ok ? fast_exp2(d_lo) : 0.f, p_hi = ok ? fast_exp2(d_hi) : 0.f;
+                        lp_lo[u][e] = d_lo * LN2; lp_hi[u][e] = d_hi * LN2;
+                        if (ok && a.record_kl) {
+                            if (prev_lo) kl_lo += p_lo * (lp_lo[u][e] - pv_lo[u][e]);
+                            if (prev_hi) kl_hi += p_hi * (lp_hi[u][e] - pv_hi[u][e]);
+                        }
+                        p[e] = p_lo; p[2 + e] = p_hi;
+                    }
+                    pf[nt >> 1][(nt & 1) * 2 + 0] = pack_bf16(p[0], p[1]);
+                    pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
                 }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
+                        if (prev_lo && key < a.N) prev_lo[key] = lp_lo[u][e];
+                        if (prev_hi && key < a.N) prev_hi[key] = lp_hi[u][e];
+                    }
             }
+            if (a.out) pv(t, pf, o);
+            __syncthreads();
         }
-        __syncthreads();
     }
     kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 1); kl_lo += __shfl_xor_sync(0xffffffffu, kl_lo, 2);
     kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 1); kl_hi += __shfl_xor_sync(0xffffffffu, kl_hi, 2);

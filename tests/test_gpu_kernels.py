@@ -97,6 +97,23 @@ def test_attention_without_recording():
     assert torch.allclose(out.float(), ref, atol=2e-2, rtol=2e-2)
 
 
+@pytest.mark.parametrize("variant,R,N,nh,nkv", [(5, 150, 1100, 2, 1), (5, 64, 2048, 4, 4), (5, 5, 37, 2, 2), (0, 300, 2048, 8, 2)])
+def test_attention_many_rows_single_pass(monkeypatch, variant, R, N, nh, nkv):
+    # without stored rows the 64-row-tile kernel makes one pass with a running maximum (probabilities are rounded
+    # to bf16 before the final normalisation): same tolerance against the oracle
+    monkeypatch.setenv("POLESTAR_ATTN_KERNEL", str(variant))
+    dh = 128
+    q = rnd((R, nh * dh), 1, 1.0, torch.bfloat16).cuda()
+    k = rnd((N, nkv * dh), 2, 1.0, torch.bfloat16).cuda()
+    v = rnd((N, nkv * dh), 3, 1.0, torch.bfloat16).cuda()
+    out = torch.zeros((R, nh * dh), dtype=torch.bfloat16, device="cuda")
+    Bd.polestar_k_attention(q, k, v, None, None, out, nh, nkv, dh)
+    torch.cuda.synchronize()
+    qn, kn, vn = bf16_np(q).reshape(R, nh, dh), bf16_np(k).reshape(N, nkv, dh), bf16_np(v).reshape(N, nkv, dh)
+    ref = O.attn_out_rows(O.attn_logp_rows(qn, kn), vn, O.bf16_round)
+    assert np.allclose(bf16_np(out), ref, atol=2e-2, rtol=2e-2)
+
+
 # ------------------------------------------------------------------ hidden delta (a1b)
 @pytest.mark.parametrize("dtype,rows,d", [(torch.bfloat16, 4096, 4096), (torch.float32, 77, 256), (torch.bfloat16, 1, 8)])
 def test_hidden_delta(dtype, rows, d):
