@@ -1034,7 +1034,8 @@ static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count
         // few rows: split the keys of every (row tile, head) over a cluster of two CTAs
         if ((mode == 6 || (mode == 0 && 2 * ctas <= sm_count)) && a.N <= 2 * 8 * AT_BN) return launch_attention_sp<8, 1, 2>(g, grid, st);
         if ((mode == 7 || (mode == 0 && 2 * ctas <= sm_count)) && a.N <= 2 * 8 * 2 * AT_BN) return launch_attention_sp<8, 2, 2>(g, grid, st);
-        if ((mode == 2 || (mode == 0 && ctas <= 2LL * sm_count)) && a.N <= 8 * 2 * AT_BN) return launch_attention_sp<8, 2>(g, grid, st);
+        // (one CTA of <8,2> per SM: beyond one wave the smaller <4,4> CTAs, three per SM, finish sooner)
+        if ((mode == 2 || (mode == 0 && ctas <= sm_count)) && a.N <= 8 * 2 * AT_BN) return launch_attention_sp<8, 2>(g, grid, st);
         if ((mode == 3 || mode == 0) && a.N <= 4 * 4 * AT_BN) return launch_attention_sp<4, 4>(g, grid, st);
         if ((mode == 4 || mode == 0) && a.N <= 8 * 4 * AT_BN) return launch_attention_sp<8, 4>(g, grid, st);
     }
