@@ -569,13 +569,23 @@ __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, S
     const int sq = blockIdx.x;
     int cnt = 0;
     if (sd.refresh.v[sq]) {
-        for (int w = t; w < sd.W; w += blockDim.x) {
-            const float* kr = a.kl + (size_t)(sq * sd.rows_per_seq + sd.B + w) * a.n_heads;
+        // head mean of the per-head drift (Eq. 4): eight lanes per row, all loads of a row in flight at once;
+        // the partial sums are combined in a fixed order
+        for (int w0 = 0; w0 < sd.W; w0 += blockDim.x / 8) {
+            const int w = w0 + (t >> 3), part = t & 7;
             float acc = 0.f;
-            for (int h = 0; h < a.n_heads; ++h) acc += kr[h];
-            const float dv = acc / (float)a.n_heads;
-            dsh[w] = dv;
-            a.drift[sq * a.W_max + w] = dv;
+            if (w < sd.W) {
+                const float* kr = a.kl + (size_t)(sq * sd.rows_per_seq + sd.B + w) * a.n_heads;
+                for (int h = part; h < a.n_heads; h += 8) acc += __ldg(kr + h);
+            }
+            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+            if (w < sd.W && part == 0) {
+                const float dv = acc / (float)a.n_heads;
+                dsh[w] = dv;
+                a.drift[sq * a.W_max + w] = dv;
+            }
         }
         __syncthreads();
         int* idx = a.sel_idx + sq * a.W_max;
