@@ -949,4 +949,18 @@ __global__ void rope_table_kernel(float2* tab, int N, int half, double theta) {
     tab[i] = make_float2((float)cos(ang), (float)sin(ang));
 }
 
+// the same entries for the listed positions only: row i < counts[s] of sequence s fills tab[idx[s][i]]
+__global__ void rope_rows_kernel(float2* tab, const int* idx, const int* counts, int max_rows, int n_rows, int half, double theta) {
+    KERNEL_PROLOGUE(17);   // rope_rows_kernel
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_rows * half) return;
+    const int m = i / half, k = i - m * half;
+    const int s = m / max_rows, r = m - s * max_rows;
+    if (r >= counts[s]) return;
+    const int pos = idx[s * max_rows + r];
+    const double inv = pow(theta, -(double)k / (double)half);
+    const double ang = (double)pos * inv;
+    tab[(size_t)pos * half + k] = make_float2((float)cos(ang), (float)sin(ang));
+}
+
 }  // namespace ps

@@ -1066,19 +1066,26 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     static MapCache maps;
     GemmWs ws;
     ws.partial = (float*)(sc + off_part); ws.partial_bytes = GEMM_PARTIAL_BYTES;
-    ws.counters = (int*)(sc + off_cnt); ws.n_counters = GEMM_COUNTERS; ws.status = (int*)(sc + off_status);
-    // the scratch is caller memory with unknown contents: the split-K tile counters must start at zero
-    CK(cudaMemsetAsync(ws.counters, 0, GEMM_COUNTERS * sizeof(int) + 1024, st));
-    const int half = head_dim / 2;
-    rope_table_kernel<<<(P * half + 255) / 256, 256, 0, st>>>(rope, P, half, (double)rope_theta);
     const int M = batch * max_rows;
-    prep_refresh_kernel<__nv_bfloat16><<<M, 256, 0, st>>>((const __nv_bfloat16*)h, idx, counts, max_rows, P, norm, rms_eps, d, a_buf);
+    const int dq = n_heads * head_dim, dkv = n_kv * head_dim;
+    // The scratch is caller memory with unknown contents: the split-K tile counters must start at zero.  Only the
+    // counters of this GEMM's output tiles (arrivals, then finished shares) are used, so only those are cleared.
+    const long long tiles = (long long)((dq + 2 * dkv + tc::BLOCK_F - 1) / tc::BLOCK_F) * ((M + tc::BLOCK_T - 1) / tc::BLOCK_T);
+    const int n_cnt = (int)std::min<long long>(GEMM_COUNTERS, 2 * (tiles + 1));
+    ws.counters = (int*)(sc + off_cnt); ws.n_counters = n_cnt; ws.status = (int*)(sc + off_status);
+    CK(cudaMemsetAsync(ws.counters, 0, (size_t)n_cnt * sizeof(int), st));
+    const int half = head_dim / 2;
+    // launched back to back with programmatic stream serialization: each kernel starts while its predecessor drains
+    // rotary entries: of the selected positions only when these are fewer than the whole table
+    if (M < P) CK(launch_k(rope_rows_kernel, dim3((M * half + 255) / 256), dim3(256), 0, st, rope, idx, counts, max_rows, M, half, (double)rope_theta));
+    else CK(launch_k(rope_table_kernel, dim3((P * half + 255) / 256), dim3(256), 0, st, rope, P, half, (double)rope_theta));
+    CK(launch_k(prep_refresh_kernel<__nv_bfloat16>, dim3(M), dim3(256), 0, st, (const __nv_bfloat16*)h, idx, counts, max_rows, P, norm,
+                rms_eps, d, a_buf));
     CK(cudaGetLastError());
     EpiArgs e;
     memset(&e, 0, sizeof(e));
     e.rope = rope; e.q_out = q_out; e.kc = kc; e.vc = vc; e.n_heads = n_heads; e.n_kv = n_kv; e.head_dim = head_dim;
     e.idx = idx; e.counts = counts; e.max_rows = max_rows; e.P = P;
-    const int dq = n_heads * head_dim, dkv = n_kv * head_dim;
     if (d % 64 == 0 && (dq + 2 * dkv) % 256 == 0 && !env_int("POLESTAR_REFRESH_SIMT", 0))
         return launch_gemm_tc<EPI_QKV_REFRESH>(maps, ws, a_buf, M, wqkv, M, dq + 2 * dkv, d, e, st);
     return launch_gemm_simt<__nv_bfloat16, EPI_QKV_REFRESH>(a_buf, wqkv, M, dq + 2 * dkv, d, e, st);
