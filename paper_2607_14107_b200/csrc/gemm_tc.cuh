@@ -7,27 +7,38 @@
 //
 //  * W is stored TILE-MAJOR: the 256 x 64 block (feature tile f, k block kb) is one contiguous
 //    32 KB chunk at chunk index f * (K / 64) + kb, so a weight TMA is one sequential burst.
-//  * One MMA instruction takes a few hundred cycles however small its N is, so the instruction
-//    shape is made as large as it gets: M = 128 tokens x N = 256 features x K = 16.  With the
-//    features on the small side of the instruction the tensor pipe, not HBM, was the limit
-//    (~4 TB/s).  Rows beyond the live tokens are out-of-bounds rows of the activation tensor
-//    map: TMA fills them with zeros without reading memory.
-//  * Stream-K: a persistent grid of one CTA per SM splits the work units -- (output tile,
-//    k block) pairs, ordered so that the token tiles of one feature tile are adjacent (their
-//    weights are then L2 hits) -- into equal contiguous ranges.  Every SM streams the same number
-//    of bytes whatever the matrix shape and the pipeline fills once per launch.  A range is a
-//    sequence of segments (one per output tile touched).  A segment that covers its tile's
-//    whole K runs the epilogue straight from tensor memory; partial segments go to a workspace
-//    slot; once all contributors of a tile have published theirs (bounded wait), each of them
-//    adds the slots in ascending-k order (deterministic) for its share of the tile and runs the
-//    epilogue on it.
+//    These loads carry the evict_first L2 policy when every weight byte is used once per launch
+//    (a single token tile): a weight stream with the default policy pushed activations, partial tiles,
+//    the K/V cache and instruction lines out of L2 (14 % of the decode time).
+//  * One 128 x 256 x 16 MMA consumes 8 KB of weights and the tensor pipe issues one every ~150 ns at
+//    the rate HBM delivers them, so the instruction shape is made as large as it gets: M = 128 tokens
+//    x N = 256 features.  With the features on the small side of the instruction the tensor pipe, not
+//    HBM, was the limit (~4 TB/s).  Rows beyond the live tokens are out-of-bounds rows of the
+//    activation tensor map: TMA fills them with zeros without reading memory.
+//  * Schedule.  Tile ids are rasterised (tile_ft) so that consecutive ids form a compact block of the
+//    output.  With more tiles than CTAs, CTA c first takes the whole tiles c, c + G, ...: the grid
+//    works on G consecutive ids at a time and operand tiles are shared through L2.  The remaining
+//    tiles -- all of them in the decoding step, where there are fewer tiles than SMs -- are split
+//    stream-K: the (tile, k block) units are dealt in equal contiguous ranges, so every SM streams the
+//    same number of bytes whatever the matrix shape.  A range is a sequence of segments (one per
+//    output tile touched).  A segment that covers its tile's whole K runs the epilogue straight from
+//    tensor memory (two accumulators: the next segment's MMAs overlap it); a partial segment is
+//    published to a workspace slot.
+//  * Reduction of split tiles (one pass at the end, all 16 warps): once the contributors of a CTA's
+//    partial tiles have published (arrival counters, bounded wait), the CTA adds the slots in
+//    ascending-k order (deterministic, no floating-point atomics) for its share of the items
+//    (one row x 16 columns; four columns when a tile has many contributors) and runs the epilogue.
+//    Shares are balanced (a CTA with two partial tiles takes half a share of each); all of this
+//    arithmetic (64-bit divisions) is done by an idle thread while the main loop runs.
 //  * Programmatic dependent launch: weight tiles of the first pipeline stages are requested
 //    before griddepcontrol.wait, i.e. while the previous kernel of the stream still drains;
 //    activations, residuals and every global write come after it.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
-// warps 2..5 = epilogue (TMEM lane quarter warp % 4 = 32 tokens each).  Every mbarrier wait is
-// bounded; on time-out the CTA raises a status word, stops issuing work and leaves in order.
+// Warp roles (512 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = epilogue (TMEM lane quarter warp % 4 = 32 tokens each), warps 6..15 only take part in
+// the reduction (its loads are pure L2 latency: more threads, fewer rounds).  Every mbarrier wait and
+// every wait on a counter is bounded; on time-out the CTA raises a status word, stops issuing work and
+// leaves in order.
 #pragma once
 #include <cuda.h>
 
