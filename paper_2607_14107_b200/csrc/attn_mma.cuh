@@ -1,8 +1,12 @@
 // Bidirectional attention rows with drift for bf16 models, head_dim 128 (Eq. 3, Eq. 4).
 //
-// One CTA = 16 query rows of one head; its 4 warps split the keys in interleaved 32-key
-// tiles, each warp streaming its own K/V tiles through a private cp.async double buffer.
-// Pass 1 gives every row's log-sum-exp (online max/sum per warp, combined across warps);
+// Three kernels share the tile helpers below; launch_attention_mma picks one from the row and key counts:
+//   attention_sp_kernel   16 query rows x 1 head per CTA, keys split over the warps, scores kept in registers
+//                         (N <= 1024): K is read once.  With a single block of rows the keys of a (row tile, head)
+//                         are further split over a cluster of two CTAs.
+//   attention_mma_kernel  the same tiling for N > 1024 with few rows: two passes over K (below).
+//   attention_big_kernel  64 query rows x 1 head per CTA for entry forwards, batches and long sequences.
+// The two-pass form: pass 1 gives every row's log-sum-exp (online max/sum per warp, combined across warps);
 // pass 2 recomputes the scores, forms logp = s - lse, p = exp(logp), accumulates
 // KL(p || stored row), overwrites the stored row with logp and accumulates p V.
 // Two passes keep logp exact (no running rescale of the stored rows); the second read of K
@@ -695,10 +699,10 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
 
 // ------------------------------------------------------------------------------------------
 // Many-rows variant (block-entry forwards, long sequences, batches): one CTA = 64 query rows of one
-// head, 4 warps x 16 rows; every 64-key K/V tile is staged once per CTA in shared memory (cp.async,
-// two stages) and used by all four warps, so K/V are re-read once per 64 rows instead of once per
-// 16.  Each warp keeps its rows' running max / sum (pass 1) and output accumulator (pass 2) in
-// registers; no cross-warp reduction is needed.
+// head, 4 warps x 16 rows; every 64-key K/V tile is staged once per CTA in shared memory (cp.async
+// ring) and used by all four warps, so K/V are re-read once per 64 rows instead of once per
+// 16.  Each warp keeps its rows' running max / sum and output accumulator in registers; no cross-warp
+// reduction is needed.
 // ------------------------------------------------------------------------------------------
 constexpr int BG_BM = 64, BG_BN = 64, BG_WARPS = 4, BG_STAGES = 3;
 constexpr int BG_TILE_BYTES = BG_BN * AT_DH * 2;                  // 16 KB: one K or V tile
