@@ -232,10 +232,18 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
     return v;
 }
 
+// Stale-row selection of the step (Sec. 4.1) riding on the O projection: eight of the warps of CTA 0 that are
+// idle until the reduction pass do it while the weights stream (batch of one sequence, small window).
+struct SelFuse {
+    int on;
+    StepDesc sd;
+    StepSelArgs a;
+};
+
 template <typename T, int EPI>
 __global__ void __launch_bounds__(FIX_THREADS, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
-               SkArgs g, EpiArgs e, PostArgs post) {
+               SkArgs g, EpiArgs e, PostArgs post, SelFuse sf) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t bars[2 * MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_sh;
@@ -349,6 +357,16 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         fx_n = n_fix;
         __threadfence_block();
         fx_ready = 1;
+    }
+
+    if constexpr (EPI == EPI_RESID) {
+        if (sf.on && cta == 0 && warp >= 6 && warp < 14) {
+            __shared__ float sel_dsh[SEL_SMALL_W];
+            __shared__ int sel_flags[SEL_SMALL_W];
+            __syncwarp();
+            pdl_wait();                                  // the per-head drift comes from the attention kernel
+            step_select_inline(sf.sd, sf.a, (int)threadIdx.x - THREADS, 256, 2, sel_dsh, sel_flags);
+        }
     }
 
     if (warp == 0) {

@@ -503,9 +503,15 @@ __device__ int select_one(const float* D, int W, int mode, int k, float thresh, 
 // Small windows (W <= SEL_SMALL_W, the in-step case: W = 3B): rank counting, two barriers.
 // Thread i owns row i; rank = number of candidates ahead of it in (drift descending, index ascending) order.
 constexpr int SEL_SMALL_W = 256;
+// `i` = index of the calling thread among the participating threads (at least W of them); bar < 0: they are the
+// whole block (__syncthreads), else they synchronise on named barrier `bar` with `nthr` threads.
+__device__ __forceinline__ void sel_sync(int bar, int nthr) {
+    if (bar < 0) __syncthreads();
+    else asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(nthr) : "memory");
+}
 __device__ int select_small(const float* D, int W, int mode, int k, float thresh, float floor_,
-                            int* idx_out, unsigned char* flag_out, int* sel_sh /* [SEL_SMALL_W] */) {
-    const int i = threadIdx.x;
+                            int* idx_out, unsigned char* flag_out, int* sel_sh /* [SEL_SMALL_W] */,
+                            int i = threadIdx.x, int bar = -1, int nthr = 0) {
     const float v = i < W ? D[i] : 0.f;
     const bool cand = i < W && v > floor_;
     bool sel = false;
@@ -520,14 +526,14 @@ __device__ int select_small(const float* D, int W, int mode, int k, float thresh
         sel = rank < k;
     }
     if (i < SEL_SMALL_W) sel_sh[i] = sel ? 1 : 0;
-    __syncthreads();
+    sel_sync(bar, nthr);
     int pos = 0, total = 0;
     for (int j = 0; j < W; ++j) { const int f = sel_sh[j]; total += f; pos += (j < i) ? f : 0; }
     if (i < W) {
         if (flag_out) flag_out[i] = sel ? 1 : 0;
         if (sel) idx_out[pos] = i;
     }
-    __syncthreads();
+    sel_sync(bar, nthr);
     return total;
 }
 
@@ -555,6 +561,53 @@ struct StepSelArgs {
     int n_heads, mode, k, W_max;
     float thresh, floor_;
 };
+
+// The same work for a batch of one sequence with a window of at most SEL_SMALL_W rows, done by `nthr` >= W threads
+// (t = 0 .. nthr-1) of a kernel that is busy otherwise: they synchronise on named barrier `bar` only.  Used by
+// the O projection, whose idle warps select the stale rows while the weights stream.
+__device__ __forceinline__ void step_select_inline(const StepDesc& sd, const StepSelArgs& a, int t, int nthr, int bar,
+                                                   float* dsh /* [SEL_SMALL_W] */, int* sel_sh /* [SEL_SMALL_W] */) {
+    int cnt = 0;
+    int* idx = a.sel_idx;
+    if (sd.refresh.v[0]) {
+        for (int w0 = 0; w0 < sd.W; w0 += nthr / 8) {
+            const int w = w0 + (t >> 3), part = t & 7;
+            float acc = 0.f;
+            if (w < sd.W) {
+                const float* kr = a.kl + (size_t)(sd.B + w) * a.n_heads;
+                for (int h = part; h < a.n_heads; h += 8) acc += __ldcg(kr + h);
+            }
+            acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+            acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+            if (w < sd.W && part == 0) {
+                const float dv = acc / (float)a.n_heads;
+                dsh[w] = dv;
+                a.drift[w] = dv;
+            }
+        }
+        sel_sync(bar, nthr);
+        unsigned char* fl = a.flag_next;
+        const int fc = a.forced_cnt ? a.forced_cnt[0] : -1;
+        if (fc >= 0) {
+            for (int w = t; w < sd.W; w += nthr) fl[w] = 0;
+            sel_sync(bar, nthr);
+            for (int i = t; i < fc; i += nthr) { const int w = a.forced_idx[i]; idx[i] = w; fl[w] = 1; }
+            cnt = fc;
+            sel_sync(bar, nthr);
+        } else {
+            cnt = select_small(dsh, sd.W, a.mode, a.k, a.thresh, a.floor_, idx, fl, sel_sh, t, bar, nthr);
+        }
+    }
+    // compacted row list of the sparse forward: the active rows, then the selected window rows
+    for (int i = t; i < sd.B; i += nthr) a.list[i] = i;
+    for (int i = t; i < cnt; i += nthr) a.list[sd.B + i] = sd.B + idx[i];
+    if (t == 0) {
+        a.sel_cnt[0] = cnt;
+        *a.list_count = sd.B + cnt;
+        atomicAdd(a.stats, cnt);
+    }
+}
 
 // One CTA per sequence; the CTA that finishes last (arrival counter a.stats[3], left at zero again) builds the
 // compacted row list from all sequences' selections.

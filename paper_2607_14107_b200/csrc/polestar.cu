@@ -128,7 +128,7 @@ static void sk_grid(int M, int N_out, int K, long long* U, long long* G) {
 template <int EPI>
 static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a_rows_alloc, const void* W, int M,
                           int N_out, int K, const EpiArgs& e, cudaStream_t st, const NextW* next = nullptr,
-                          const PostArgs* post = nullptr) {
+                          const PostArgs* post = nullptr, const tc::SelFuse* sel = nullptr) {
     if (M <= 0) return POLESTAR_OK;
     (void)a_rows_alloc;
     // weights: tile-major [chunks * 256][64]; activations: exactly M rows, so that the rows of a token tile
@@ -182,7 +182,8 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     auto kern = tc::gemm_sk_kernel<__nv_bfloat16, EPI>;
     static bool attr = false;
     if (!attr) {
-        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        // (four stages of 48 KB + alignment slack; static shared memory comes on top of it)
+        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (int)tc::STAGE_BYTES + 1024));
         attr = true;
     }
     PostArgs pa;
@@ -193,8 +194,10 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
         ws.post_total += (unsigned)G;
         pa.expect = ws.post_total;
     }
-    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e, pa));
-    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e, pa));
+    tc::SelFuse sfz;
+    if (sel) sfz = *sel; else memset(&sfz, 0, sizeof(sfz));
+    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e, pa, sfz));
+    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e, pa, sfz));
     return POLESTAR_OK;
 }
 
@@ -422,14 +425,15 @@ struct Path {
 
     template <int EPI>
     static int gemm(polestar_ctx* c, const void* A, int a_rows_alloc, const void* W, int M, int N_out, int K,
-                    const EpiArgs& e, const NextW* next = nullptr, const PostArgs* post = nullptr, bool* fused = nullptr) {
+                    const EpiArgs& e, const NextW* next = nullptr, const PostArgs* post = nullptr, bool* fused = nullptr,
+                    const tc::SelFuse* sel = nullptr) {
         if (fused) *fused = false;
         if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 256 == 0) {
             const bool fuse = post && post->kind && c->gws.post_counter && post->d <= 4 * NORM_VPT * tc::FIX_THREADS &&
                               env_int("POLESTAR_FUSE_PREP", 0);      // measured on B200: no faster than the separate kernel
                                                                      // (grid-wide counter round trip = kernel boundary)
             if (fused) *fused = fuse;
-            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st, next, fuse ? post : nullptr);
+            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st, next, fuse ? post : nullptr, sel);
         }
         return launch_gemm_simt<T, EPI>(A, W, M, N_out, K, e, c->st);
     }
@@ -531,8 +535,14 @@ struct Path {
             }
             const int* list = nullptr;
             const int* m2_count = nullptr;
+            // One sequence with a small window on the tensor-core path: the selection rides on the O projection
+            // (idle warps of its first CTA), off the critical path; otherwise it is a kernel of its own.
+            const bool sel_in_gemm = sparse && bs == 1 && sd.W <= SEL_SMALL_W && is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) &&
+                                     dq % 64 == 0 && d % 256 == 0 && env_int("POLESTAR_FUSE_SELECT", 1);
+            tc::SelFuse sf;
+            memset(&sf, 0, sizeof(sf));
             if (sparse) {
-                Scope sc(c, POLESTAR_PROF_SELECT, (double)bs * sd.W * (m.n_heads * 4 + 8), 0, 1);
+                Scope sc(c, POLESTAR_PROF_SELECT, (double)bs * sd.W * (m.n_heads * 4 + 8), 0, sel_in_gemm ? 0 : 1);
                 StepSelArgs s;
                 memset(&s, 0, sizeof(s));
                 s.kl = b.kl; s.drift = b.drift + (size_t)l * bs * Wm; s.sel_idx = b.sel_idx + (size_t)l * bs * Wm;
@@ -542,8 +552,11 @@ struct Path {
                 s.mode = p.select_mode;
                 s.k = p.select_mode == POLESTAR_SELECT_TOPK_FRAC ? (int)floorf(p.select_frac * (float)sd.W + 0.5f) : p.select_k;
                 s.W_max = Wm; s.thresh = p.select_thresh; s.floor_ = p.drift_floor;
-                CK(launch_k(step_select_kernel, dim3(bs), dim3(SEL_THREADS), 0, st, sd, s));
-                CK(cudaGetLastError());
+                if (sel_in_gemm) { sf.on = 1; sf.sd = sd; sf.a = s; }
+                else {
+                    CK(launch_k(step_select_kernel, dim3(bs), dim3(SEL_THREADS), 0, st, sd, s));
+                    CK(cudaGetLastError());
+                }
                 list = b.list; m2_count = b.list_count;
             }
             {
@@ -556,7 +569,7 @@ struct Path {
                 memset(&po, 0, sizeof(po));
                 po.kind = 1; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n2[l]; po.a_out = b.a_buf;
                 po.x = b.x1; po.list = list; po.m_count = m2_count;
-                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e, nx, &po, &ffn_staged))) return rc;
+                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e, nx, &po, &ffn_staged, sf.on ? &sf : nullptr))) return rc;
             }
             if (!ffn_staged) {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
