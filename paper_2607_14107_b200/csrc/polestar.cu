@@ -17,6 +17,7 @@
 
 #include "attn_mma.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_chain.cuh"
 #include "kernels.cuh"
 
 using namespace ps;
@@ -88,6 +89,8 @@ struct GemmWs {
     int* status = nullptr;
     unsigned* post_counter = nullptr;      // grid-wide arrival counter of GEMMs with appended row work (never reset)
     mutable unsigned post_total = 0;       // its value once every launch so far has completed
+    unsigned* chain_counter = nullptr;     // the same for chained launches
+    mutable unsigned chain_total = 0;
 };
 
 // bf16 matrices with out % 256 == 0 and in % 64 == 0 are stored tile-major (see polestar.h)
@@ -229,6 +232,65 @@ struct Buffers {
 static const int CONF_CHUNKS = 32;
 static const int FORCED_COMMIT_MAX = 512;
 static const size_t GEMM_PARTIAL_BYTES = ((size_t)40 << 20) + 16384 + 65536;   // 2 slots x 148 CTAs x 128 x 256 fp32
+// One projection of a chained launch (gemm_chain.cuh): A [M, K] x W [N_out, K]^T with epilogue `epi`.
+struct ChainSpec {
+    const void* A; const void* W;
+    int N_out, K, epi, norm_after;
+    EpiArgs e;
+    PostArgs post;
+};
+// Launches the projections as one persistent kernel when the chain applies (M <= 128 rows, tile-major weights,
+// the same stream-K grid for all of them); otherwise *applies = false and nothing is launched.
+template <typename T>
+static int launch_gemm_chain(MapCache& maps, const GemmWs& ws, const ChainSpec* sp, int n, int M, cudaStream_t st,
+                             const tc::SelFuse* sel, bool* applies) {
+    *applies = false;
+    if (n < 2 || n > tc::CHAIN_MAX || M <= 0 || M > tc::BLOCK_T || !ws.chain_counter) return POLESTAR_OK;
+    long long G0 = 0;
+    for (int i = 0; i < n; ++i) {
+        if (sp[i].N_out % tc::BLOCK_F || sp[i].K % 64) return POLESTAR_OK;
+        long long U, G;
+        sk_grid(M, sp[i].N_out, sp[i].K, &U, &G);
+        if (i == 0) G0 = G;
+        if (G != G0 || sp[i].N_out / tc::BLOCK_F > G) return POLESTAR_OK;
+    }
+    if ((size_t)2 * G0 * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes) return POLESTAR_OK;
+    tc::ChainMaps cm;
+    tc::ChainArgs ca;
+    memset(&ca, 0, sizeof(ca));
+    int n_bar = 0;
+    for (int i = 0; i < n; ++i) {
+        const CUtensorMap* mw = maps.get(sp[i].W, (uint64_t)sp[i].N_out * (uint64_t)(sp[i].K / 64), 64, tc::BLOCK_F);
+        const CUtensorMap* ma = maps.get(sp[i].A, (uint64_t)M, (uint64_t)sp[i].K, tc::BLOCK_T);
+        if (!mw || !ma) return POLESTAR_E_CUDA;
+        cm.w[i] = *mw; cm.a[i] = *ma;
+        tc::ChainProb& P = ca.p[i];
+        P.M = M; P.N_out = sp[i].N_out; P.K = sp[i].K; P.tiles_f = sp[i].N_out / tc::BLOCK_F;
+        P.epi = sp[i].epi; P.norm_after = (i + 1 < n) ? sp[i].norm_after : 0;
+        P.e = sp[i].e; P.post = sp[i].post;
+        if (i + 1 < n) n_bar += 1 + P.norm_after;
+    }
+    for (int i = n; i < tc::CHAIN_MAX; ++i) { cm.w[i] = cm.w[0]; cm.a[i] = cm.a[0]; }
+    ca.n = n;
+    ca.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", 4)));
+    ca.partial = ws.partial; ca.tile_counter = ws.counters; ca.done_offset = ws.n_counters / 2; ca.status = ws.status;
+    ca.bar_counter = ws.chain_counter;
+    ca.bar_base = ws.chain_total;
+    ws.chain_total += (unsigned)(n_bar * G0);
+    tc::SelFuse sfz;
+    if (sel) sfz = *sel; else memset(&sfz, 0, sizeof(sfz));
+    const size_t smem = (size_t)ca.stages * tc::STAGE_BYTES + 1024;
+    auto kern = tc::gemm_chain_kernel<T>;
+    static bool attr = false;
+    if (!attr) {
+        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (int)tc::STAGE_BYTES + 1024));
+        attr = true;
+    }
+    CK(launch_k(kern, dim3((unsigned)G0), dim3(tc::FIX_THREADS), smem, st, cm, ca, sfz));
+    *applies = true;
+    return POLESTAR_OK;
+}
+
 static const int GEMM_COUNTERS = 1 << 17;     // arrivals + finished shares for up to 65536 output tiles
 
 struct polestar_ctx {
@@ -559,6 +621,26 @@ struct Path {
                 }
                 list = b.list; m2_count = b.list_count;
             }
+            // O projection -> RMSNorm -> gate/up -> down as one persistent kernel when the step is small enough
+            bool chained = false;
+            if (is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && M <= tc::BLOCK_T && env_int("POLESTAR_CHAIN", 1)) {
+                ChainSpec sp[3];
+                memset(sp, 0, sizeof(sp));
+                sp[0].A = b.o_buf; sp[0].W = c->wo[l]; sp[0].N_out = d; sp[0].K = dq; sp[0].epi = EPI_RESID; sp[0].norm_after = 1;
+                sp[0].e.resid = b.x; sp[0].e.out_f32 = b.x1; sp[0].e.ld_out = d;
+                sp[0].post.kind = 1; sp[0].post.n_rows = M; sp[0].post.d = d; sp[0].post.eps = m.rms_eps; sp[0].post.gain = c->n2[l];
+                sp[0].post.a_out = b.a_buf; sp[0].post.x = b.x1; sp[0].post.list = list; sp[0].post.m_count = m2_count;
+                sp[1].A = b.a_buf; sp[1].W = c->wgu[l]; sp[1].N_out = 2 * F; sp[1].K = d; sp[1].epi = EPI_SWIGLU;
+                sp[1].e.out_t = b.g_buf; sp[1].e.ld_out = F; sp[1].e.m_count = m2_count;
+                sp[2].A = b.g_buf; sp[2].W = c->wd[l]; sp[2].N_out = d; sp[2].K = F; sp[2].epi = EPI_DOWN;
+                sp[2].e.rows = b.rows; sp[2].e.list = list; sp[2].e.m_count = m2_count; sp[2].e.resid = b.x1; sp[2].e.out_f32 = b.x;
+                sp[2].e.packet = b.packet; sp[2].e.W_max = Wm; sp[2].e.within = within; sp[2].e.ld_out = d;
+                const double by = ((double)d * dq + 3.0 * F * d) * esd, fl = 2.0 * M * d * (double)dq + 6.0 * Mlive * F * (double)d;
+                Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, by, fl, 0);
+                if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, 3, M, st, sf.on ? &sf : nullptr, &chained))) return rc;
+                if (chained) c->launches += 1;
+            }
+            if (!chained) {
             {
                 Scope sc(c, POLESTAR_PROF_GEMM_O, (double)d * dq * esd + (double)M * dq * esd + 2.0 * M * d * 4, 2.0 * M * d * (double)dq, 1);
                 memset(&e, 0, sizeof(e));
@@ -601,6 +683,7 @@ struct Path {
                     po.patch = b.patch + (size_t)(l + 1) * bs * Wm; po.kvflag = b.kvflag; po.sd = sd;
                 }
                 if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e, nx, &po, &qkv_staged))) return rc;
+            }
             }
         }
         if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
@@ -828,8 +911,10 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     c->rows_lm = p->batch * (c->B + std::min(p->win_suffix_blocks * c->B, c->W_max));
     c->cum.assign(p->batch, 0);
     c->gws.partial = c->b.gemm_partial; c->gws.partial_bytes = GEMM_PARTIAL_BYTES;
-    c->gws.counters = c->b.gemm_counters; c->gws.n_counters = GEMM_COUNTERS - 2; c->gws.status = c->b.status;
+    // the last 512 words of the counter array hold the grid-wide counters, the rest the per-tile counters
+    c->gws.counters = c->b.gemm_counters; c->gws.n_counters = GEMM_COUNTERS - 512; c->gws.status = c->b.status;
     c->gws.post_counter = reinterpret_cast<unsigned*>(c->b.gemm_counters + GEMM_COUNTERS - 1); c->gws.post_total = 0;
+    c->gws.chain_counter = reinterpret_cast<unsigned*>(c->b.gemm_counters + GEMM_COUNTERS - 512); c->gws.chain_total = 0;
 
     auto fail = [&](int code) { delete c; return code; };
     // zero the persistent state (everything in front of the scratch rows)
