@@ -210,3 +210,30 @@ def test_c2_full_depth_decode_is_bitwise_reproducible(c2_full):
     for a, b in zip(*runs):
         for x, y in zip(a, b):
             assert np.array_equal(x, y)
+
+
+def test_c2_chained_projections_equal_separate_launches(monkeypatch):
+    # the persistent O -> RMSNorm -> gate/up -> down kernel does the arithmetic of the four separate launches in the
+    # same order: same bits (2 layers at full widths, an entry forward, plain and refresh steps)
+    m, p = I.config("c2")
+    m = I.reduced_depth(m, 2)
+    p = dataclasses.replace(p, max_steps=64, logit_scale=30.0, flags=p.flags | I.FLAG_KEEP_HIDDEN)
+    packed = Bd.make_packed_weights(m, seed=0, device="cuda")
+    prompt = I.make_prompt(m, p).numpy()
+    runs = []
+    for chain in ("1", "0"):
+        monkeypatch.setenv("POLESTAR_CHAIN", chain)
+        gpu = Bd.Polestar(m, packed, p, prompt)
+        trace = []
+        for step in range(8):
+            if step:
+                gpu.step()
+            trace.append((gpu.read(Bd.READ_LOGITS).copy(), gpu.read(Bd.READ_HIDDEN, m.n_layers).copy(),
+                          gpu.read(Bd.READ_KCACHE, 1).copy(), gpu.read(Bd.READ_HCACHE, 1).copy()))
+            gpu.commit()
+            trace.append((gpu.tokens().copy(),))
+        runs.append(trace)
+        gpu.destroy()
+    for a, b in zip(*runs):
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
