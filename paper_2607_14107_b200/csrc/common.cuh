@@ -205,7 +205,30 @@ struct EpiArgs {
     float scale;              // LOGITS
     // QKV_REFRESH (stand-alone refresh kernel): row r of sequence s = r / max_rows
     const int* idx; const int* counts; int max_rows; int P;
+    // RMSNorm folded into two GEMMs (steps whose rows all come straight from the previous GEMM): the producing
+    // epilogue (RESID / DOWN) also stores a = x * gain in the model dtype and adds the row's sum of squares to
+    // fold_ss (64-bit fixed point, 2^16: integer additions commute, so the sum is reproducible); the consuming
+    // epilogue (SWIGLU / QKV) multiplies its rows by rsqrt(ss / d + eps), which commutes with the matrix product.
+    void* fold_a; const float* fold_gain; long long* fold_ss;
+    const long long* in_ss; float in_eps; int in_d;
 };
+
+constexpr float FOLD_SCALE = 65536.f;
+// Adds `partial` (sum of squares of some columns of row `row`) to ss[row].  The lanes of the warp that hold the same
+// row are added up first, in lane order, and one lane issues the integer atomic.
+__device__ __forceinline__ void fold_ss_add(long long* ss, int row, float partial) {
+    const unsigned act = __activemask();
+    const unsigned grp = __match_any_sync(act, row);
+    float sum = 0.f;
+    for (unsigned rest = grp; rest; rest &= rest - 1) sum += __shfl_sync(grp, partial, __ffs(rest) - 1);
+    if ((int)(threadIdx.x & 31) == __ffs(grp) - 1)
+        atomicAdd(reinterpret_cast<unsigned long long*>(ss + row), (unsigned long long)__float2ll_rn(sum * FOLD_SCALE));
+}
+__device__ __forceinline__ float fold_inv(const EpiArgs& e, int m) {
+    // (final before the consuming GEMM's first load; read through L1 so that epilogue_prefetch can have it waiting)
+    const float ss = (float)e.in_ss[m] * (1.f / FOLD_SCALE);
+    return rsqrtf(ss / (float)e.in_d + e.in_eps);
+}
 
 // Row-wise work appended to a GEMM whose output rows are the input of the next normalisation: once every CTA
 // of the grid has stored its outputs (a counter all CTAs add to), the CTAs share out the rows and stage the
@@ -312,6 +335,29 @@ template <> __device__ __forceinline__ void store8<__nv_bfloat16>(__nv_bfloat16*
     reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// producing side of the folded RMSNorm: a = x * gain for 16 (4) finished values of row `row`, and their squares
+template <typename T>
+__device__ __forceinline__ void fold_store16(const EpiArgs& e, int row, size_t o, int n, const float* r) {
+    float a16[16];
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float4 g = __ldg(reinterpret_cast<const float4*>(e.fold_gain + n) + i);
+        a16[4 * i] = r[4 * i] * g.x; a16[4 * i + 1] = r[4 * i + 1] * g.y; a16[4 * i + 2] = r[4 * i + 2] * g.z; a16[4 * i + 3] = r[4 * i + 3] * g.w;
+        ss += r[4 * i] * r[4 * i] + r[4 * i + 1] * r[4 * i + 1] + r[4 * i + 2] * r[4 * i + 2] + r[4 * i + 3] * r[4 * i + 3];
+    }
+    store16<T>((T*)e.fold_a + o, a16);
+    fold_ss_add(e.fold_ss, row, ss);
+}
+template <typename T>
+__device__ __forceinline__ void fold_store4(const EpiArgs& e, int row, size_t o, int n, float4 r) {
+    const float4 g = __ldg(reinterpret_cast<const float4*>(e.fold_gain + n));
+    T* dst = (T*)e.fold_a + o;
+    store_pair<T>(dst, r.x * g.x, r.y * g.y);
+    store_pair<T>(dst + 2, r.z * g.z, r.w * g.w);
+    fold_ss_add(e.fold_ss, row, r.x * r.x + r.y * r.y + r.z * r.z + r.w * r.w);
+}
+
 // The 16 outputs n .. n+15 (n % 16 == 0) of row m: the same arithmetic as epilogue_pair on each pair, with the
 // row descriptor read once and all loads and stores 16 bytes wide.  Requires head_dim % 16 == 0 and leading
 // dimensions that keep 16-column groups 16-byte aligned (true for every matrix the tensor-core path accepts).
@@ -331,6 +377,13 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int n, const
         }
         const int dq = e.n_heads * e.head_dim, dkv = e.n_kv * e.head_dim;
         const int Npos = (EPI == EPI_QKV) ? e.N_seq : e.P;
+        float vs[16];
+        {
+            const float inv = (EPI == EPI_QKV && e.in_ss) ? fold_inv(e, m) : 1.f;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) vs[i] = v[i] * inv;
+        }
+        v = vs;
         if (n < dq + dkv) {
             if (n < dq ? e.q_out == nullptr : !kvf) return;
             const int hd1 = e.head_dim - 1;
@@ -359,10 +412,15 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int n, const
             r[4 * i] = c.x + v[4 * i]; r[4 * i + 1] = c.y + v[4 * i + 1]; r[4 * i + 2] = c.z + v[4 * i + 2]; r[4 * i + 3] = c.w + v[4 * i + 3];
         }
         store16<float>(e.out_f32 + o, r);
+        if (e.fold_a) fold_store16<T>(e, m, o, n, r);
     } else if (EPI == EPI_SWIGLU) {
+        const float inv = e.in_ss ? fold_inv(e, m) : 1.f;
         float gl[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) gl[i] = v[2 * i] / (1.f + expf(-v[2 * i])) * v[2 * i + 1];
+        for (int i = 0; i < 8; ++i) {
+            const float ga = v[2 * i] * inv, up = v[2 * i + 1] * inv;
+            gl[i] = ga / (1.f + expf(-ga)) * up;
+        }
         store8<T>((T*)e.out_t + (size_t)m * e.ld_out + (n >> 1), gl);
     } else if (EPI == EPI_DOWN) {
         const int r0 = e.list ? __ldg(e.list + m) : m;
@@ -377,6 +435,7 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int n, const
         }
         float* dst = (e.within && rw.z >= 0) ? e.packet + ((size_t)rw.x * e.W_max + rw.z) * e.ld_out + n : e.out_f32 + o;
         store16<float>(dst, r);
+        if (e.fold_a && !(e.within && rw.z >= 0)) fold_store16<T>(e, r0, o, n, r);
     } else if (EPI == EPI_LOGITS) {
         float r[16];
 #pragma unroll
@@ -391,7 +450,9 @@ __device__ __forceinline__ void epilogue4(const EpiArgs& e, int m, int n, float4
     if (EPI == EPI_RESID) {
         const size_t o = (size_t)m * e.ld_out + n;
         const float4 c = __ldg(reinterpret_cast<const float4*>(e.resid + o));
-        *reinterpret_cast<float4*>(e.out_f32 + o) = make_float4(c.x + v.x, c.y + v.y, c.z + v.z, c.w + v.w);
+        const float4 r = make_float4(c.x + v.x, c.y + v.y, c.z + v.z, c.w + v.w);
+        *reinterpret_cast<float4*>(e.out_f32 + o) = r;
+        if (e.fold_a) fold_store4<T>(e, m, o, n, r);
     } else if (EPI == EPI_DOWN) {
         const int r0 = e.list ? __ldg(e.list + m) : m;
         const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + r0);       // {seq, pos, widx, aidx}
@@ -399,7 +460,9 @@ __device__ __forceinline__ void epilogue4(const EpiArgs& e, int m, int n, float4
         const size_t o = (size_t)r0 * e.ld_out + n;
         const float4 c = __ldg(reinterpret_cast<const float4*>(e.resid + o));
         float* dst = (e.within && rw.z >= 0) ? e.packet + ((size_t)rw.x * e.W_max + rw.z) * e.ld_out + n : e.out_f32 + o;
-        *reinterpret_cast<float4*>(dst) = make_float4(c.x + v.x, c.y + v.y, c.z + v.z, c.w + v.w);
+        const float4 r = make_float4(c.x + v.x, c.y + v.y, c.z + v.z, c.w + v.w);
+        *reinterpret_cast<float4*>(dst) = r;
+        if (e.fold_a && !(e.within && rw.z >= 0)) fold_store4<T>(e, r0, o, n, r);
     }
 }
 
@@ -411,14 +474,19 @@ __device__ __forceinline__ void epilogue_prefetch(const EpiArgs& e, int m, int n
     if (EPI == EPI_QKV) {
         const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + m);
         prefetch_l1(e.kvflag + m);
+        if (e.in_ss) prefetch_l1(e.in_ss + m);
         if (rw.y >= 0 && n < (e.n_heads + e.n_kv) * e.head_dim)
             prefetch_l1(e.rope + (size_t)rw.y * (e.head_dim / 2) + ((n % e.head_dim) >> 1));
     } else if (EPI == EPI_RESID) {
         prefetch_l1(e.resid + (size_t)m * e.ld_out + n);
+        if (e.fold_a) prefetch_l1(e.fold_gain + n);
     } else if (EPI == EPI_DOWN) {
         const int r = e.list ? __ldg(e.list + m) : m;
         prefetch_l1(reinterpret_cast<const int4*>(e.rows) + r);
         prefetch_l1(e.resid + (size_t)r * e.ld_out + n);
+        if (e.fold_a) prefetch_l1(e.fold_gain + n);
+    } else if (EPI == EPI_SWIGLU) {
+        if (e.in_ss) prefetch_l1(e.in_ss + m);
     }
 }
 

@@ -353,6 +353,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     const int item = f_lo[f] + (int)threadIdx.x - (f ? f_n[0] : 0);
                     if (P.epi == EPI_RESID) epilogue_prefetch<T, EPI_RESID>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
                     else if (P.epi == EPI_DOWN) epilogue_prefetch<T, EPI_DOWN>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
+                    else epilogue_prefetch<T, EPI_SWIGLU>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
                 }
                 if (threadIdx.x == 64) {
                     const long long t0 = clock64();

@@ -225,7 +225,7 @@ struct Buffers {
     int* list_count; float* hidden_keep;
     // scratch
     Row* rows; unsigned char* kvflag; float* x; float* x1; float* packet; char* a_buf; char* q_buf; char* o_buf;
-    char* g_buf; float* kl; int* list; HeadSrc* head_list; char* a_head; float* logits; ConfPart* conf_part;
+    char* g_buf; float* kl; int* list; long long* fold_ss; HeadSrc* head_list; char* a_head; float* logits; ConfPart* conf_part;
     float* gemm_partial; int* gemm_counters;
 };
 
@@ -438,6 +438,7 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(g_buf, char, Mmax * F * es);
     TAKE(kl, float, Mmax * nh);
     TAKE(list, int, Mmax);
+    TAKE(fold_ss, long long, (size_t)2 * L * Mmax);
     TAKE(head_list, HeadSrc, rows_lm);
     TAKE(a_head, char, rows_lm * d * es);
     TAKE(logits, float, rows_lm * V);
@@ -548,6 +549,12 @@ struct Path {
             CK(cudaGetLastError());
         }
 
+        // Steps whose rows all come straight from the previous projection (within-block steps without refresh): the two
+        // RMSNorms of a layer are folded into the projections around them (EpiArgs::fold_*), no staging kernels.
+        const bool fold = within && !sparse && is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && d % 256 == 0 && dq % 64 == 0 &&
+                          F % 64 == 0 && (dq + 2 * dkv) % 256 == 0 && (2 * F) % 256 == 0 && env_int("POLESTAR_FOLD_NORM", 0);
+        const size_t Mm = (size_t)c->M_max;
+        if (fold) CK(cudaMemsetAsync(b.fold_ss, 0, (size_t)2 * L * Mm * sizeof(long long), st));
         bool qkv_staged = false, ffn_staged = false;
         for (int l = 0; l < L; ++l) {
             char* kc = b.kc + (size_t)l * bs * N * dkv * es;
@@ -559,6 +566,7 @@ struct Path {
                 Scope sc(c, POLESTAR_PROF_MISC, 0, 0, 1);
                 CK(launch_k(keep_hidden_kernel, dim3(bs * B), dim3(256), 0, st, sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d));
             }
+            if (fold && l > 0) qkv_staged = true;      // the previous down projection stored x * gain and the sums of squares
             if (!qkv_staged) {      // (layers after the first: done in the tail of the previous layer's down projection)
                 Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
                 CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
@@ -574,6 +582,7 @@ struct Path {
                 e.rows = b.rows; e.kvflag = b.kvflag; e.rope = b.rope; e.q_out = b.q_buf; e.kc = kc; e.vc = vc;
                 e.N_seq = N; e.n_heads = m.n_heads; e.n_kv = m.n_kv_heads; e.head_dim = m.head_dim; e.W_max = Wm;
                 e.within = within; e.ld_out = dq;
+                if (fold && l > 0) { e.in_ss = b.fold_ss + (size_t)(2 * l) * Mm; e.in_eps = m.rms_eps; e.in_d = d; }
                 NextW nx[2];
                 nx[0].w = c->wo[l]; nx[0].N_out = d; nx[0].K = dq; nx[0].M = M; nx[0].count = pf_units;
                 nx[1].w = c->wgu[l]; nx[1].N_out = 2 * F; nx[1].K = d; nx[1].M = M; nx[1].count = pf_units2;
@@ -635,6 +644,14 @@ struct Path {
                 sp[2].A = b.g_buf; sp[2].W = c->wd[l]; sp[2].N_out = d; sp[2].K = F; sp[2].epi = EPI_DOWN;
                 sp[2].e.rows = b.rows; sp[2].e.list = list; sp[2].e.m_count = m2_count; sp[2].e.resid = b.x1; sp[2].e.out_f32 = b.x;
                 sp[2].e.packet = b.packet; sp[2].e.W_max = Wm; sp[2].e.within = within; sp[2].e.ld_out = d;
+                if (fold) {
+                    sp[0].norm_after = 0;
+                    sp[0].e.fold_a = b.a_buf; sp[0].e.fold_gain = c->n2[l]; sp[0].e.fold_ss = b.fold_ss + (size_t)(2 * l + 1) * Mm;
+                    sp[1].e.in_ss = sp[0].e.fold_ss; sp[1].e.in_eps = m.rms_eps; sp[1].e.in_d = d;
+                    if (l + 1 < L) {
+                        sp[2].e.fold_a = b.a_buf; sp[2].e.fold_gain = c->n1[l + 1]; sp[2].e.fold_ss = b.fold_ss + (size_t)(2 * l + 2) * Mm;
+                    }
+                }
                 const double by = ((double)d * dq + 3.0 * F * d) * esd, fl = 2.0 * M * d * (double)dq + 6.0 * Mlive * F * (double)d;
                 Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, by, fl, 0);
                 if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, 3, M, st, sf.on ? &sf : nullptr, &chained))) return rc;
@@ -645,6 +662,7 @@ struct Path {
                 Scope sc(c, POLESTAR_PROF_GEMM_O, (double)d * dq * esd + (double)M * dq * esd + 2.0 * M * d * 4, 2.0 * M * d * (double)dq, 1);
                 memset(&e, 0, sizeof(e));
                 e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
+                if (fold) { e.fold_a = b.a_buf; e.fold_gain = c->n2[l]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 1) * Mm; }
                 NextW nx[2];
                 nx[0].w = c->wgu[l]; nx[0].N_out = 2 * F; nx[0].K = d; nx[0].M = M; nx[0].first = pf_units2; nx[0].count = pf_units;
                 PostArgs po;
@@ -653,6 +671,7 @@ struct Path {
                 po.x = b.x1; po.list = list; po.m_count = m2_count;
                 if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e, nx, &po, &ffn_staged, sf.on ? &sf : nullptr))) return rc;
             }
+            if (fold) ffn_staged = true;
             if (!ffn_staged) {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
                 CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
@@ -662,6 +681,7 @@ struct Path {
                 Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, (2.0 * F * d + Mlive * d + Mlive * F) * esd, 4.0 * Mlive * F * (double)d, 1);
                 memset(&e, 0, sizeof(e));
                 e.out_t = b.g_buf; e.ld_out = F; e.m_count = m2_count;
+                if (fold) { e.in_ss = b.fold_ss + (size_t)(2 * l + 1) * Mm; e.in_eps = m.rms_eps; e.in_d = d; }
                 NextW nx[2];
                 nx[0].w = c->wd[l]; nx[0].N_out = d; nx[0].K = F; nx[0].M = M; nx[0].count = pf_units;
                 if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->M_max, c->wgu[l], M, 2 * F, d, e, nx))) return rc;
@@ -671,6 +691,7 @@ struct Path {
                 memset(&e, 0, sizeof(e));
                 e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = b.x1; e.out_f32 = b.x; e.packet = b.packet;
                 e.W_max = Wm; e.within = within; e.ld_out = d;
+                if (fold && l + 1 < L) { e.fold_a = b.a_buf; e.fold_gain = c->n1[l + 1]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 2) * Mm; }
                 NextW nx[2];
                 if (l + 1 < L) { nx[0].w = c->wqkv[l + 1]; nx[0].N_out = dq + 2 * dkv; nx[0].K = d; nx[0].M = M; }
                 else { nx[0].w = c->lm_head; nx[0].N_out = m.vocab; nx[0].K = d; nx[0].M = bs * B; }

@@ -148,6 +148,21 @@ def test_c1b_long_ragged_sequence(monkeypatch, variant):
     assert seen["refresh"] >= 2
 
 
+def test_c1b_bf16_rmsnorm_folded_into_the_projections(monkeypatch):
+    # opt-in variant for steps without refresh: the producing projection stores x * gain and the row's sum of squares,
+    # the consuming projection scales its rows (bf16 rounding before instead of after the normalisation)
+    monkeypatch.setenv("POLESTAR_FOLD_NORM", "1")
+    seen = run_forced("c1b", 12, tau_upd=3, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["within"] > seen["refresh"]
+
+
+def test_c1b_bf16_separate_launches(monkeypatch):
+    # the projections of a layer as separate launches instead of one chained kernel
+    monkeypatch.setenv("POLESTAR_CHAIN", "0")
+    seen = run_forced("c1b", 10, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["refresh"] > 3
+
+
 def test_c1b_bf16_simt_gemm_path():
     run_forced("c1b", 6, tau_upd=-1, flags=I.FLAG_DEFAULT | Bd.FLAG_SIMT_GEMM)
 
