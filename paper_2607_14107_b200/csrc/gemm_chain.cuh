@@ -1,5 +1,5 @@
 // A chain of weight-streaming GEMMs of one decoding step in ONE persistent kernel (O projection -> RMSNorm ->
-// gate/up -> down).  Each of these projections multiplies at most 128 rows by its weights, so every one of them is
+// gate/up -> down -> patch + RMSNorm -> the next layer's QKV projection).  Each of these projections multiplies at most 128 rows by its weights, so every one of them is
 // a stream-K launch of gemm_sk_kernel whose weight stream takes 4-27 us and whose drain, partial-tile exchange and
 // kernel boundary take another ~10 us.  Chained, the boundary becomes a grid-wide counter, and while one
 // projection drains and reduces, the TMA producer already fills the operand ring with the next projection's
@@ -18,12 +18,13 @@
 namespace ps {
 namespace tc {
 
-constexpr int CHAIN_MAX = 3;
+constexpr int CHAIN_MAX = 4;
 
 struct ChainProb {
     int M, N_out, K, tiles_f;     // one token tile; tiles_f = N_out / 256 output tiles
-    int epi;                      // EPI_RESID, EPI_SWIGLU or EPI_DOWN
-    int norm_after;               // 1: RMSNorm staging of this projection's output rows (post) before the next one
+    int epi;                      // EPI_RESID, EPI_SWIGLU, EPI_DOWN or EPI_QKV
+    int norm_after;               // row staging between this projection and the next (post): 1 RMSNorm of the output
+                                  // rows, 2 patch + RMSNorm of the next layer's QKV input (Algorithm 1 "Patch")
     EpiArgs e;
     PostArgs post;
 };
@@ -46,7 +47,8 @@ template <typename T>
 __device__ __forceinline__ void epi16_dyn(int kind, const EpiArgs& e, int m, int n, const float* v) {
     if (kind == EPI_RESID) epilogue16<T, EPI_RESID>(e, m, n, v);
     else if (kind == EPI_SWIGLU) epilogue16<T, EPI_SWIGLU>(e, m, n, v);
-    else epilogue16<T, EPI_DOWN>(e, m, n, v);
+    else if (kind == EPI_DOWN) epilogue16<T, EPI_DOWN>(e, m, n, v);
+    else epilogue16<T, EPI_QKV>(e, m, n, v);
 }
 template <typename T>
 __device__ __forceinline__ void epi4_dyn(int kind, const EpiArgs& e, int m, int n, float4 v) {
@@ -353,7 +355,8 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     const int item = f_lo[f] + (int)threadIdx.x - (f ? f_n[0] : 0);
                     if (P.epi == EPI_RESID) epilogue_prefetch<T, EPI_RESID>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
                     else if (P.epi == EPI_DOWN) epilogue_prefetch<T, EPI_DOWN>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
-                    else epilogue_prefetch<T, EPI_SWIGLU>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
+                    else if (P.epi == EPI_SWIGLU) epilogue_prefetch<T, EPI_SWIGLU>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
+                    else epilogue_prefetch<T, EPI_QKV>(P.e, item / (BLOCK_F / 16), fix_tile[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
                 }
                 if (threadIdx.x == 64) {
                     const long long t0 = clock64();
@@ -367,7 +370,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     last_sh = ok;
                 }
                 __syncthreads();
-                if (P.epi != EPI_SWIGLU && last_sh && max(f_nseg[0], f_nseg[1]) > 4) {
+                if ((P.epi == EPI_RESID || P.epi == EPI_DOWN) && last_sh && max(f_nseg[0], f_nseg[1]) > 4) {
                     for (int i4 = (int)threadIdx.x; i4 < 4 * total; i4 += FIX_THREADS) {
                         const int i = i4 >> 2;
                         const int f = i < f_n[0] ? 0 : 1;
@@ -457,8 +460,13 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             if (threadIdx.x == 0) post_ok = grid_counter_wait(ca.bar_counter, ca.bar_base + bar_k * (unsigned)G, abort_flag) ? 1 : 0;
             __syncthreads();
             if (post_ok) {
-                for (int r = cta; r < P.post.n_rows; r += G)
-                    prep_rows_row<T>(r, P.post.x, P.post.list, P.post.m_count, P.post.gain, P.post.eps, P.post.d, (T*)P.post.a_out, post_red);
+                for (int r = cta; r < P.post.n_rows; r += G) {
+                    if (P.norm_after == 1)
+                        prep_rows_row<T>(r, P.post.x, P.post.list, P.post.m_count, P.post.gain, P.post.eps, P.post.d, (T*)P.post.a_out, post_red);
+                    else
+                        prep_qkv_row<T>(P.post.sd, r, P.post.rows, P.post.x, P.post.hc, P.post.packet, P.post.patch, P.post.gain,
+                                        P.post.eps, P.post.d, (T*)P.post.a_out, P.post.kvflag, post_red);
+                }
             }
             arrive();
         }

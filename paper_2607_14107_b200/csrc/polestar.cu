@@ -266,9 +266,9 @@ static int launch_gemm_chain(MapCache& maps, const GemmWs& ws, const ChainSpec* 
         cm.w[i] = *mw; cm.a[i] = *ma;
         tc::ChainProb& P = ca.p[i];
         P.M = M; P.N_out = sp[i].N_out; P.K = sp[i].K; P.tiles_f = sp[i].N_out / tc::BLOCK_F;
-        P.epi = sp[i].epi; P.norm_after = (i + 1 < n) ? sp[i].norm_after : 0;
+        P.epi = sp[i].epi; P.norm_after = (i + 1 < n) ? sp[i].norm_after : 0;      // 0 none, 1 RMSNorm rows, 2 QKV input staging
         P.e = sp[i].e; P.post = sp[i].post;
-        if (i + 1 < n) n_bar += 1 + P.norm_after;
+        if (i + 1 < n) n_bar += 1 + (P.norm_after ? 1 : 0);
     }
     for (int i = n; i < tc::CHAIN_MAX; ++i) { cm.w[i] = cm.w[0]; cm.a[i] = cm.a[0]; }
     ca.n = n;
@@ -556,6 +556,7 @@ struct Path {
         const size_t Mm = (size_t)c->M_max;
         if (fold) CK(cudaMemsetAsync(b.fold_ss, 0, (size_t)2 * L * Mm * sizeof(long long), st));
         bool qkv_staged = false, ffn_staged = false;
+        bool qkv_done = false;      // this layer's QKV projection ran at the end of the previous layer's chained kernel
         for (int l = 0; l < L; ++l) {
             char* kc = b.kc + (size_t)l * bs * N * dkv * es;
             char* vc = b.vc + (size_t)l * bs * N * dkv * es;
@@ -567,7 +568,7 @@ struct Path {
                 CK(launch_k(keep_hidden_kernel, dim3(bs * B), dim3(256), 0, st, sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d));
             }
             if (fold && l > 0) qkv_staged = true;      // the previous down projection stored x * gain and the sums of squares
-            if (!qkv_staged) {      // (layers after the first: done in the tail of the previous layer's down projection)
+            if (!qkv_done && !qkv_staged) {      // (else: staged by the previous layer's down projection or chained kernel)
                 Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
                 CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
                                                      c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag));
@@ -575,7 +576,7 @@ struct Path {
             }
             qkv_staged = false;
             EpiArgs e;
-            {
+            if (!qkv_done) {
                 const double nq = dq + 2 * dkv;
                 Scope sc(c, POLESTAR_PROF_GEMM_QKV, (nq * d + (double)M * d + (double)M * nq) * esd, 2.0 * M * nq * d, 1);
                 memset(&e, 0, sizeof(e));
@@ -588,6 +589,7 @@ struct Path {
                 nx[1].w = c->wgu[l]; nx[1].N_out = 2 * F; nx[1].K = d; nx[1].M = M; nx[1].count = pf_units2;
                 if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->M_max, c->wqkv[l], M, dq + 2 * dkv, d, e, nx))) return rc;
             }
+            qkv_done = false;
             {
                 const bool rec_w = sparse || !within;
                 const double rec_rows = (rec_w ? (double)bs * sd.W : 0.0) + (last ? (double)bs * B : 0.0);
@@ -633,7 +635,7 @@ struct Path {
             // O projection -> RMSNorm -> gate/up -> down as one persistent kernel when the step is small enough
             bool chained = false;
             if (is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && M <= tc::BLOCK_T && env_int("POLESTAR_CHAIN", 1)) {
-                ChainSpec sp[3];
+                ChainSpec sp[4];
                 memset(sp, 0, sizeof(sp));
                 sp[0].A = b.o_buf; sp[0].W = c->wo[l]; sp[0].N_out = d; sp[0].K = dq; sp[0].epi = EPI_RESID; sp[0].norm_after = 1;
                 sp[0].e.resid = b.x; sp[0].e.out_f32 = b.x1; sp[0].e.ld_out = d;
@@ -653,9 +655,35 @@ struct Path {
                     }
                 }
                 const double by = ((double)d * dq + 3.0 * F * d) * esd, fl = 2.0 * M * d * (double)dq + 6.0 * Mlive * F * (double)d;
-                Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, by, fl, 0);
-                if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, 3, M, st, sf.on ? &sf : nullptr, &chained))) return rc;
-                if (chained) c->launches += 1;
+                // ... and, behind it, the next layer's input staging and QKV projection
+                int n_chain = 3;
+                double by4 = 0, fl4 = 0;
+                // (off by default: measured 1 % slower than launching that projection on its own)
+                if (l + 1 < L && !fold && env_int("POLESTAR_CHAIN_QKV", 0)) {
+                    n_chain = 4;
+                    sp[2].norm_after = 2;
+                    PostArgs& po = sp[2].post;
+                    po.kind = 2; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n1[l + 1]; po.a_out = b.a_buf;
+                    po.x = b.x; po.rows = b.rows; po.hc = b.hc + (size_t)(l + 1) * bs * Wm * d; po.packet = b.packet;
+                    po.patch = b.patch + (size_t)(l + 1) * bs * Wm; po.kvflag = b.kvflag; po.sd = sd;
+                    sp[3].A = b.a_buf; sp[3].W = c->wqkv[l + 1]; sp[3].N_out = dq + 2 * dkv; sp[3].K = d; sp[3].epi = EPI_QKV;
+                    EpiArgs& eq = sp[3].e;
+                    eq.rows = b.rows; eq.kvflag = b.kvflag; eq.rope = b.rope; eq.q_out = b.q_buf;
+                    eq.kc = b.kc + (size_t)(l + 1) * bs * N * dkv * es; eq.vc = b.vc + (size_t)(l + 1) * bs * N * dkv * es;
+                    eq.N_seq = N; eq.n_heads = m.n_heads; eq.n_kv = m.n_kv_heads; eq.head_dim = m.head_dim; eq.W_max = Wm;
+                    eq.within = within; eq.ld_out = dq;
+                    by4 = (double)(dq + 2 * dkv) * d * esd; fl4 = 2.0 * M * (double)(dq + 2 * dkv) * d;
+                }
+                {
+                    Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, by + (n_chain == 4 ? by4 : 0), fl + (n_chain == 4 ? fl4 : 0), 0);
+                    if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, n_chain, M, st, sf.on ? &sf : nullptr, &chained))) return rc;
+                    if (!chained && n_chain == 4) {
+                        n_chain = 3;
+                        sp[2].norm_after = 0;
+                        if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, 3, M, st, sf.on ? &sf : nullptr, &chained))) return rc;
+                    }
+                }
+                if (chained) { c->launches += 1; qkv_done = (n_chain == 4); }
             }
             if (!chained) {
             {

@@ -156,6 +156,13 @@ def test_c1b_bf16_rmsnorm_folded_into_the_projections(monkeypatch):
     assert seen["within"] > seen["refresh"]
 
 
+def test_c1b_bf16_chain_through_the_next_qkv_projection(monkeypatch):
+    # opt-in: the chained kernel also stages and runs the next layer's QKV projection
+    monkeypatch.setenv("POLESTAR_CHAIN_QKV", "1")
+    seen = run_forced("c1b", 10, tau_upd=3, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["within"] > 0 and seen["refresh"] > 0
+
+
 def test_c1b_bf16_separate_launches(monkeypatch):
     # the projections of a layer as separate launches instead of one chained kernel
     monkeypatch.setenv("POLESTAR_CHAIN", "0")
