@@ -262,7 +262,7 @@ def run_ours(args):
                                "traffic": TRAFFIC_OVER_ALGORITHMIC * g_b / max(g_calls, 1),
                                "algorithmic_bytes_per_launch": g_b / max(g_calls, 1),
                                "peak_source": which + " (copy bandwidth)",
-                               "kernel": "gemm_sk_kernel (the five projections of a forward, one template)",
+                               "kernel": "gemm_sk_kernel / gemm_chain_kernel (the five projections of a forward: one stream-K tcgen05 design)",
                                "launches": g_calls, "avg_launch_us": 1e3 * g_ms / max(g_calls, 1),
                                "avg_launch_us_in_pipeline": 1e3 * g_ms_timed / max(g_calls, 1),
                                "frac_in_pipeline": ach_pipe / hbm,
