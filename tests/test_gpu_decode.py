@@ -174,6 +174,15 @@ def test_c1b_bf16_simt_gemm_path():
     run_forced("c1b", 6, tau_upd=-1, flags=I.FLAG_DEFAULT | Bd.FLAG_SIMT_GEMM)
 
 
+@pytest.mark.parametrize("batch,prompt_len,gen_len,block", [(3, 50, 48, 16), (5, 33, 64, 32), (2, 100, 24, 8)])
+def test_c1b_odd_shapes(batch, prompt_len, gen_len, block):
+    # bf16 tensor-core path with batches, prompt lengths and block sizes that leave ragged row counts everywhere
+    # (48 / 160 / 16 rows in the chained projections, window rows of several sequences in the sparse forward)
+    seen = run_forced("c1b", 8, batch=batch, prompt_len=prompt_len, gen_len=gen_len, block=block, max_steps=gen_len // 2,
+                      tau_upd=1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["within"] > 0
+
+
 def test_c1_batch2_gqa():
     m, p = I.config("c1")
     m = dataclasses.replace(m, n_kv_heads=2)
