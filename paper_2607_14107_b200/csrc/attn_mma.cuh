@@ -927,6 +927,7 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
 
         // ---- pass 2: logp, KL, stored rows, P V ----------------------------------------------------------
         const bool with_v = a.out != nullptr;
+        const bool vec = (a.N & 1) == 0;
         load_tile(0, with_v);
         if (n_tiles > 1) load_tile(1, with_v);
         if (n_tiles > 2) load_tile(2, with_v);
@@ -939,13 +940,22 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
             for (int hf = 0; hf < 2; ++hf) {            // two halves of 4 key groups keep the register count down
                 float pv_lo[4][2], pv_hi[4][2], lp_lo[4][2], lp_hi[4][2];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
+                for (int u = 0; u < 4; ++u) {
+                    const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair;
+                    pv_lo[u][0] = pv_lo[u][1] = pv_hi[u][0] = pv_hi[u][1] = 0.f;
+                    if (a.record_kl) {
+                        if (vec) {        // even N: the two keys of a thread are one 8-byte access
+                            if (prev_lo && key < a.N) { const float2 v = *reinterpret_cast<const float2*>(prev_lo + key); pv_lo[u][0] = v.x; pv_lo[u][1] = v.y; }
+                            if (prev_hi && key < a.N) { const float2 v = *reinterpret_cast<const float2*>(prev_hi + key); pv_hi[u][0] = v.x; pv_hi[u][1] = v.y; }
+                        } else {
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
-                        pv_lo[u][e] = (a.record_kl && prev_lo && key < a.N) ? prev_lo[key] : 0.f;
-                        pv_hi[u][e] = (a.record_kl && prev_hi && key < a.N) ? prev_hi[key] : 0.f;
+                            for (int e = 0; e < 2; ++e) {
+                                if (prev_lo && key + e < a.N) pv_lo[u][e] = prev_lo[key + e];
+                                if (prev_hi && key + e < a.N) pv_hi[u][e] = prev_hi[key + e];
+                            }
+                        }
                     }
+                }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const int nt = hf * 4 + u;
@@ -966,13 +976,19 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
                     pf[nt >> 1][(nt & 1) * 2 + 1] = pack_bf16(p[2], p[3]);
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
+                for (int u = 0; u < 4; ++u) {
+                    const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair;
+                    if (vec) {
+                        if (prev_lo && key < a.N) *reinterpret_cast<float2*>(prev_lo + key) = make_float2(lp_lo[u][0], lp_lo[u][1]);
+                        if (prev_hi && key < a.N) *reinterpret_cast<float2*>(prev_hi + key) = make_float2(lp_hi[u][0], lp_hi[u][1]);
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int key = t * BG_BN + (hf * 4 + u) * 8 + cpair + e;
-                        if (prev_lo && key < a.N) prev_lo[key] = lp_lo[u][e];
-                        if (prev_hi && key < a.N) prev_hi[key] = lp_hi[u][e];
+                        for (int e = 0; e < 2; ++e) {
+                            if (prev_lo && key + e < a.N) prev_lo[key + e] = lp_lo[u][e];
+                            if (prev_hi && key + e < a.N) prev_hi[key + e] = lp_hi[u][e];
+                        }
                     }
+                }
             }
             if (a.out) pv(t, pf, o);
             __syncthreads();
