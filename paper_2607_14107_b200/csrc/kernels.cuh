@@ -824,7 +824,9 @@ struct CommitArgs {
     const int* head_count; const int* suf_seq; const int* suf_w;
     const int* forced_pos; int forced_n;      // [batch][forced_n] absolute positions, -1 unused (null: free-running)
     const int* forced_tok;                    // optional tokens written at the forced positions (null: own prediction)
-    int* seq_info;               // [batch][8]: committed, by_conf, by_drift, by_quota, suffix, eos, masked_left, nonfinite
+    int* seq_info;               // [batch][8]: committed, by_conf, by_drift, by_quota, suffix, eos, masked_left, nonfinite;
+                                 // then 8 more words: the step's counters (stats[0..3]) and the GEMM status word
+    const int* stats; const int* status; int batch;
     int n_heads, hist, mask_id, eos_id, act_row_off, steps_used, steps_per_block, use_drift, use_suffix, ge;
     float tau_s, alpha, tau_suffix;
 };
@@ -948,6 +950,11 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
         o[0] = cnt[0]; o[1] = cnt[1]; o[2] = cnt[2]; o[3] = cnt[3]; o[4] = cnt[4]; o[5] = cnt[5];
         o[6] = n_masked - (cnt[0] - cnt[4]);
         o[7] = cnt[7];
+        if (s == 0) {        // one record for the host: a single copy brings everything the controller reads
+            int* t = a.seq_info + a.batch * 8;
+            t[0] = a.stats[0]; t[1] = a.stats[1]; t[2] = a.stats[2]; t[3] = a.stats[3];
+            t[4] = *a.status;
+        }
     }
 }
 

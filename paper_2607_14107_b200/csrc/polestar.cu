@@ -317,7 +317,7 @@ struct polestar_ctx {
     int last_act_row_off = 0;
     bool forced_select = false, forced_commit = false, forced_tokens = false;
     int forced_commit_n = 0;
-    std::vector<int> seq_info_host;
+    int* seq_info_host = nullptr;          // pinned: bs * 8 + 8 words
     // launch accounting and optional per-family device timing (POLESTAR_FLAG_PROFILE)
     long long launches = 0;
     struct ProfRec { int fam; size_t ev; double bytes, flops; };
@@ -419,7 +419,7 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(taud, float, bs * B);
     TAKE(commit_flags, int, bs * B);
     TAKE(suffix_flags, int, bs * Wm);
-    TAKE(seq_info, int, bs * 8);
+    TAKE(seq_info, int, bs * 8 + 8);
     TAKE(head_count, int, 1);
     TAKE(suf_seq, int, bs * Wm);
     TAKE(suf_w, int, bs * Wm);
@@ -851,7 +851,7 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     a.forced_pos = c->forced_commit ? b.forced_commit : nullptr;
     a.forced_n = c->forced_commit_n;
     a.forced_tok = (c->forced_commit && c->forced_tokens) ? b.forced_tok : nullptr;
-    a.seq_info = b.seq_info;
+    a.seq_info = b.seq_info; a.stats = b.stats; a.status = b.status; a.batch = p.batch;
     a.n_heads = c->m.n_heads; a.hist = p.hist; a.mask_id = c->m.mask_id; a.eos_id = c->m.eos_id;
     a.act_row_off = c->last_act_row_off; a.steps_used = c->steps_used;
     a.steps_per_block = std::max(1, p.max_steps / std::max(1, c->n_blocks));
@@ -866,10 +866,9 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
         CK(launch_k(commit_kernel, dim3(p.batch), dim3(256), 0, c->st, sd, a));
         CK(cudaGetLastError());
     }
-    c->seq_info_host.resize((size_t)p.batch * 8 + 8);
-    CK(cudaMemcpyAsync(c->seq_info_host.data(), b.seq_info, (size_t)p.batch * 8 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
-    CK(cudaMemcpyAsync(c->seq_info_host.data() + p.batch * 8, b.stats, 4 * sizeof(int), cudaMemcpyDeviceToHost, c->st));
-    CK(cudaMemcpyAsync(c->seq_info_host.data() + p.batch * 8 + 4, b.status, sizeof(int), cudaMemcpyDeviceToHost, c->st));
+    if (!c->seq_info_host && cudaHostAlloc((void**)&c->seq_info_host, ((size_t)p.batch * 8 + 8) * sizeof(int), cudaHostAllocDefault) != cudaSuccess)
+        return POLESTAR_E_CUDA;
+    CK(cudaMemcpyAsync(c->seq_info_host, b.seq_info, ((size_t)p.batch * 8 + 8) * sizeof(int), cudaMemcpyDeviceToHost, c->st));
     CK(cudaStreamSynchronize(c->st));
     for (const auto& r : c->prof_recs) {
         float ms = 0.f;
@@ -883,7 +882,7 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     c->pending = false;
     c->forced_commit = false;
     c->forced_tokens = false;
-    const int* si = c->seq_info_host.data();
+    const int* si = c->seq_info_host;
     polestar_commit_info ci;
     memset(&ci, 0, sizeof(ci));
     bool all_block_done = true;
@@ -1000,6 +999,7 @@ extern "C" void polestar_destroy(polestar_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->st);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+    if (c->seq_info_host) cudaFreeHost(c->seq_info_host);
     delete c;
 }
 
