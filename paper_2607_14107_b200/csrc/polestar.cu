@@ -166,9 +166,9 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
     tc::SkArgs g;
     g.M = M; g.N_out = N_out; g.K = K; g.tiles_f = tiles_f; g.tiles_t = tiles_t;
-    // Three stages (145 KB) for the weight-bound steps: the stream needs no more in flight, and the small kernels between
-    // the GEMMs (staging, attention) then fit next to a GEMM block, so that they are resident and past their prologue
-    // when the GEMM ends (measured +2 % tokens/s).  Four stages when operands come from L2 (several token tiles).
+    // Three stages (145 KB) for the weight-bound steps: measured +2 % tokens/s over four (the HBM stream needs no more in
+    // flight, and less shared memory per block leaves room for the next kernel's blocks to become resident early); two
+    // stages are 4 % slower.  Four stages when operands come from L2 (several token tiles).
     g.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", tiles_t == 1 ? 3 : 4)));
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
     g.cluster_n = cluster_n;
