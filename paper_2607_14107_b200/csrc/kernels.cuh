@@ -101,6 +101,8 @@ __device__ __forceinline__ void norm_row(const float* __restrict__ src, const fl
     for (int u = 0; u < NORM_VPT; ++u) {
         const int c4 = threadIdx.x + u * blockDim.x;
         v[u] = c4 < n4 ? __ldcg(reinterpret_cast<const float4*>(src) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        // the gains are needed only after the reduction: have them in L1 by then
+        if (c4 < n4) asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const float4*>(gain) + c4));
     }
 #pragma unroll
     for (int u = 0; u < NORM_VPT; ++u) ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
