@@ -183,7 +183,9 @@ struct SkArgs {
     int w_stream;       // 1: every weight byte is read once by this launch: load it with the evict_first L2 policy
     int cluster_n;      // > 0: launched in clusters of cluster_n CTAs = the contributors of one output tile;
                         // partial tiles are then exchanged through distributed shared memory, not global memory
-    long long* trace;   // optional [gridDim.x][8] nanosecond stamps of this launch (null: off)
+    long long* trace;   // optional [gridDim.x][12] nanosecond stamps of this launch (null: off): 0 start, 1 set-up done,
+                        // 2 dependencies resolved, 3 first stage full, 4 last MMA issued, 5 partial tiles published,
+                        // 6 other contributors arrived, 8 share reduced, 7 end
     // L2 prefetch of weights that later GEMMs of the stream will read: while this kernel's epilogue and
     // fix-up run, HBM would otherwise idle.  Entry j: tile-major weight base, that GEMM's unit count and grid,
     // and the slice [first, first + count) of every CTA's unit range to prefetch (count 0: unused).
