@@ -7,8 +7,8 @@
 // 4 us per layer less than three launches plus the RMSNorm kernel (the grid-wide counter costs about what a
 // kernel boundary costs; the gain is the ring filled ahead and one launch instead of four).
 //
-// Restrictions (the decoding regime): one token tile per projection (M <= 128), no more output tiles than CTAs,
-// the same grid for every projection of the chain.  Everything else -- tile-major weights with the evict_first
+// Restrictions (the decoding regime): one token tile per projection (M <= 128), no more output tiles than CTAs.
+// Every projection keeps the stream-K grid it would have alone (ChainProb::G); the launch has the largest of them.  Everything else -- tile-major weights with the evict_first
 // policy, tcgen05 128 x 256 x 16 MMAs into two TMEM accumulators, published partial tiles reduced in ascending-k
 // order by all 16 warps -- is as in gemm_tc.cuh, whose helpers this file uses.  All CTAs of the grid are resident
 // (at most one per SM), so the grid-wide counters cannot deadlock; their waits are bounded all the same.
@@ -22,6 +22,8 @@ constexpr int CHAIN_MAX = 4;
 
 struct ChainProb {
     int M, N_out, K, tiles_f;     // one token tile; tiles_f = N_out / 256 output tiles
+    int G;                        // CTAs that work on this projection (the first G of the grid; the rest only take part
+                                  // in the grid-wide counters and the row staging)
     int epi;                      // EPI_RESID, EPI_SWIGLU, EPI_DOWN or EPI_QKV
     int norm_after;               // row staging between this projection and the next (post): 1 RMSNorm of the output
                                   // rows, 2 patch + RMSNorm of the next layer's QKV input (Algorithm 1 "Patch")
@@ -120,8 +122,9 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
     auto range = [&](int p, int& kb_total, long long& U, long long& u_begin, long long& u_end) {
         kb_total = ca.p[p].K / BLOCK_K;
         U = (long long)ca.p[p].tiles_f * kb_total;
-        u_begin = sk_begin(U, G, cta);
-        u_end = sk_begin(U, G, cta + 1);
+        const int Gp = ca.p[p].G;
+        u_begin = cta < Gp ? sk_begin(U, Gp, cta) : 0;
+        u_end = cta < Gp ? sk_begin(U, Gp, cta + 1) : 0;
     };
 
     if (threadIdx.x == THREADS) {
@@ -129,6 +132,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
         for (int p = 0; p < ca.n; ++p) {
             int kb_total; long long U, u_begin, u_end;
             range(p, kb_total, U, u_begin, u_end);
+            const int Gp = ca.p[p].G;
             int n_fix = 0;
             if (u_end > u_begin) {
                 const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;
@@ -142,10 +146,10 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 for (int f = 0; f < n_fix; ++f) {
                     const int tile = fix_tile[f];
                     const long long tile_begin = (long long)tile * kb_total, tile_end = tile_begin + kb_total;
-                    const int c_lo = sk_owner(U, G, tile_begin), c_hi = sk_owner(U, G, tile_end - 1);
+                    const int c_lo = sk_owner(U, Gp, tile_begin), c_hi = sk_owner(U, Gp, tile_end - 1);
                     const int nseg = c_hi - c_lo + 1;
-                    const int w_lo = sk_partial_segments(U, G, c_lo, kb_total) == 2 ? 1 : 2;
-                    const int w_hi = (nseg > 1 && sk_partial_segments(U, G, c_hi, kb_total) == 2) ? 1 : 2;
+                    const int w_lo = sk_partial_segments(U, Gp, c_lo, kb_total) == 2 ? 1 : 2;
+                    const int w_hi = (nseg > 1 && sk_partial_segments(U, Gp, c_hi, kb_total) == 2) ? 1 : 2;
                     fx_par[p][f][0] = tile; fx_par[p][f][1] = c_lo; fx_par[p][f][2] = nseg;
                     fx_par[p][f][3] = (cta == c_lo) ? 0 : w_lo + 2 * (cta - c_lo - 1);
                     fx_par[p][f][4] = (cta == c_lo) ? w_lo : (cta == c_hi ? w_hi : 2);

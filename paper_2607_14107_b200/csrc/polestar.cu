@@ -242,20 +242,20 @@ struct ChainSpec {
     EpiArgs e;
     PostArgs post;
 };
-// Launches the projections as one persistent kernel when the chain applies (M <= 128 rows, tile-major weights,
-// the same stream-K grid for all of them); otherwise *applies = false and nothing is launched.
+// Launches the projections as one persistent kernel when the chain applies (M <= 128 rows, tile-major weights);
+// otherwise *applies = false and nothing is launched.
 template <typename T>
 static int launch_gemm_chain(MapCache& maps, const GemmWs& ws, const ChainSpec* sp, int n, int M, cudaStream_t st,
                              const tc::SelFuse* sel, bool* applies) {
     *applies = false;
     if (n < 2 || n > tc::CHAIN_MAX || M <= 0 || M > tc::BLOCK_T || !ws.chain_counter) return POLESTAR_OK;
-    long long G0 = 0;
+    long long G0 = 0, Gp[tc::CHAIN_MAX];
     for (int i = 0; i < n; ++i) {
         if (sp[i].N_out % tc::BLOCK_F || sp[i].K % 64) return POLESTAR_OK;
-        long long U, G;
-        sk_grid(M, sp[i].N_out, sp[i].K, &U, &G);
-        if (i == 0) G0 = G;
-        if (G != G0 || sp[i].N_out / tc::BLOCK_F > G) return POLESTAR_OK;
+        long long U;
+        sk_grid(M, sp[i].N_out, sp[i].K, &U, &Gp[i]);
+        if (sp[i].N_out / tc::BLOCK_F > Gp[i]) return POLESTAR_OK;
+        G0 = std::max(G0, Gp[i]);
     }
     if ((size_t)2 * G0 * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes) return POLESTAR_OK;
     tc::ChainMaps cm;
@@ -268,7 +268,7 @@ static int launch_gemm_chain(MapCache& maps, const GemmWs& ws, const ChainSpec* 
         if (!mw || !ma) return POLESTAR_E_CUDA;
         cm.w[i] = *mw; cm.a[i] = *ma;
         tc::ChainProb& P = ca.p[i];
-        P.M = M; P.N_out = sp[i].N_out; P.K = sp[i].K; P.tiles_f = sp[i].N_out / tc::BLOCK_F;
+        P.M = M; P.N_out = sp[i].N_out; P.K = sp[i].K; P.tiles_f = sp[i].N_out / tc::BLOCK_F; P.G = (int)Gp[i];
         P.epi = sp[i].epi; P.norm_after = (i + 1 < n) ? sp[i].norm_after : 0;      // 0 none, 1 RMSNorm rows, 2 QKV input staging
         P.e = sp[i].e; P.post = sp[i].post;
         if (i + 1 < n) n_bar += 1 + (P.norm_after ? 1 : 0);
