@@ -27,6 +27,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c2")
     ap.add_argument("--forwards", type=int, default=6)
+    ap.add_argument("--entry", action="store_true", help="also print forward 0, the block-entry forward of the first block")
     a = ap.parse_args()
     os.environ["POLESTAR_KERNEL_TRACE"] = "1"
     import torch
@@ -45,7 +46,7 @@ def main():
     order = np.argsort(ts, kind="stable")
     ids, ts = ids[order], ts[order]
     starts = [i for i in range(n) if ids[i] == 1]
-    for f in range(1, len(starts) - 1):
+    for f in range(0 if a.entry else 1, len(starts) - 1):
         lo, hi = starts[f], starts[f + 1]
         agg = collections.OrderedDict()
         for i in range(lo, hi):
