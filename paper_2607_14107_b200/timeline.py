@@ -27,12 +27,16 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", default="c2")
     ap.add_argument("--forwards", type=int, default=6)
+    ap.add_argument("--max-steps", type=int, default=0, help="override the step budget (fewer steps: more tokens per step, blocks turn over sooner)")
     ap.add_argument("--entry", action="store_true", help="also print forward 0, the block-entry forward of the first block")
     a = ap.parse_args()
     os.environ["POLESTAR_KERNEL_TRACE"] = "1"
     import torch
     from . import binding as Bd, inputs as I
     m, p = I.config(a.config)
+    if a.max_steps:
+        import dataclasses
+        p = dataclasses.replace(p, max_steps=a.max_steps)
     dec = Bd.Polestar(m, Bd.make_packed_weights(m), p, I.make_prompt(m, p).numpy())
     dec.commit()
     for _ in range(a.forwards):
