@@ -65,7 +65,8 @@ extern "C" {
 #define POLESTAR_E_NOSPACE    (-3)  /* workspace too small                         */
 #define POLESTAR_E_CUDA       (-4)  /* a CUDA call or kernel failed                */
 #define POLESTAR_E_NONFINITE  (-5)  /* NaN / Inf met where a decision was needed   */
-#define POLESTAR_E_TIMEOUT    (-6)  /* a bounded device-side wait ran out          */
+#define POLESTAR_E_TIMEOUT    (-6)  /* a bounded device-side wait ran out; the context
+                                       is unusable afterwards (later calls: E_STATE)  */
 #define POLESTAR_E_DONE       (-7)  /* every block is already decoded              */
 
 /* ---- enumerations --------------------------------------------------------------- */
@@ -165,7 +166,7 @@ typedef struct {
 /* ---- the decoding path ------------------------------------------------------------ */
 
 /* Bytes of device workspace `polestar_init` needs for this model and these parameters
- * (0 if they are invalid).  Pure host arithmetic. */
+ * (0 if they are invalid), valid for any 256-byte aligned base address.  Pure host arithmetic. */
 size_t polestar_workspace_bytes(const polestar_model *m, const polestar_params *p);
 
 /* Create a context and run the block-0 entry forward (Algorithm 1: initial state,
@@ -176,6 +177,8 @@ size_t polestar_workspace_bytes(const polestar_model *m, const polestar_params *
  *   workspace_dev    device, >= polestar_workspace_bytes(), 256-byte aligned, caller-owned;
  *                    the library zero-fills what it needs
  *   cuda_stream      cudaStream_t as void*
+ * The POLESTAR_* environment switches are read here, once, into the context (and become the switches of the
+ * stand-alone kernel calls below); nothing reads the environment on the launch path.
  * Errors: E_INVAL (NULLs, unsupported shape, bad ids), E_NOSPACE, E_CUDA. *out is NULL on error. */
 int polestar_init(polestar_ctx **out, const polestar_model *m, const polestar_weights *w,
                   const polestar_params *p, const int32_t *prompt_ids_host,
@@ -191,7 +194,9 @@ int polestar_step(polestar_ctx *c, polestar_step_info *info_host);
 /* Commit rule of Sec. 4.2 on the last forward's logits (confidence >= tau_s, or drift delta
  * >= alpha (tau_s - c)^2 on within-block steps, quota top-up, suffix rows by confidence),
  * Eq. 2 token update, controller bookkeeping.  Synchronises.  info_host may be NULL.
- * Errors: E_STATE (no forward pending), E_NONFINITE, E_TIMEOUT, E_CUDA. */
+ * Errors: E_STATE (no forward pending, or the context failed earlier), E_NONFINITE, E_CUDA, and E_TIMEOUT
+ * when a kernel of the forward gave up a bounded wait: its outputs may be partial and its counters are out of
+ * step, so the context is dead from then on (every later step / commit returns E_STATE; destroy it). */
 int polestar_commit(polestar_ctx *c, polestar_commit_info *info_host);
 
 /* Copy the current token ids to host memory: out_host [batch][prompt_len + gen_len]. */
@@ -213,7 +218,19 @@ int polestar_tokens(polestar_ctx *c, int32_t *out_host);
 #define POLESTAR_READ_COMMIT     12  /* int32 [batch][block] bit0 commit, bit1 by confidence,
                                         bit2 by drift, bit3 by quota (last commit)               */
 #define POLESTAR_READ_PPREV      13  /* float [batch][W_max][n_heads][N] stored log attention    */
-#define POLESTAR_READ_SUFFIX     14  /* int32 [batch][W_max] bit0 eligible, bit1 committed       */
+#define POLESTAR_READ_SUFFIX     14  /* int32 [batch][W_max] bit0 eligible, bit1 committed, bit2 the
+                                        rule's own decision (confidence >= tau_suffix)           */
+/* Quantities of the last commit (Sec. 4.2 "Current Block Commit"; Algorithm 1 after the layer loop): */
+#define POLESTAR_READ_DRIFT_DELTA 15 /* float [batch][block] Delta = delta - mean(Theta)          */
+#define POLESTAR_READ_TAU_D      16  /* float [batch][block] alpha (tau_s - c)^2                  */
+#define POLESTAR_READ_THETA      17  /* float [batch][max(1,hist)][block] drift history ring: the
+                                        vector pushed as number n (0-based) sits in slot n % hist */
+#define POLESTAR_READ_THETA_COUNT 18 /* int32 [batch] vectors pushed since the block was entered  */
+#define POLESTAR_READ_OWN_COMMIT 19  /* int32 [batch][block] the rule's own decision (bits as in
+                                        READ_COMMIT), also when a forced decision replaced it    */
+/* Libraries built with -DPOLESTAR_TRACE only (time stamps, see csrc/common.cuh): */
+#define POLESTAR_READ_TRACE_KERNELS 98 /* int64 [8192]: next slot, then (kernel id, ns) pairs      */
+#define POLESTAR_READ_TRACE_GEMM 99  /* int64 [CTAs][12] stamps of the traced GEMM kind            */
 /* Synchronises, copies min(bytes, size of the item) bytes to dst_host.
  * Errors: E_INVAL (unknown item, bad layer, item not kept). */
 int polestar_read(polestar_ctx *c, int32_t what, int32_t layer, void *dst_host, size_t bytes);
@@ -238,6 +255,10 @@ int polestar_profile(polestar_ctx *c, double *out_host, int32_t reset);
 
 void polestar_destroy(polestar_ctx *c);
 const char *polestar_strerror(int code);
+
+/* Re-read the POLESTAR_* environment switches for the stand-alone kernel calls below (contexts keep the
+ * values they read at polestar_init).  The paper has no counterpart. */
+int polestar_reload_env(void);
 
 /* ---- single kernels of the path (unit parity, micro-benchmarks) --------------------- */
 /* All pointers are device pointers owned by the caller; the calls are asynchronous on `cuda_stream`.
@@ -288,10 +309,15 @@ int polestar_k_refresh(const void *h_dev, const int32_t *idx_dev, const int32_t 
                        int32_t n_heads, int32_t n_kv_heads, int32_t head_dim, float rms_eps,
                        float rope_theta, int32_t dtype, void *scratch_dev, size_t scratch_bytes,
                        void *cuda_stream);
+/* Outcome of the last polestar_k_refresh on this scratch (same batch, max_rows, d, head_dim): synchronises the
+ * stream; POLESTAR_OK, or POLESTAR_E_TIMEOUT if a bounded device-side wait of its projection gave up (the cache
+ * rows of that call are then incomplete). */
+int polestar_k_refresh_status(const void *scratch_dev, size_t scratch_bytes, int32_t batch, int32_t max_rows,
+                              int32_t d, int32_t head_dim, void *cuda_stream);
 
 /* Confidence of logits rows (Eq. 1; Sec. 2 sampler set): per row, y_hat = argmax over v != mask_id
- * (lowest id on ties), conf = softmax(logits)[y_hat].  logits_dev float [rows][vocab];
- * scratch_dev: >= rows * 512 bytes of device memory. */
+ * (lowest id on ties), conf = softmax(logits)[y_hat].  logits_dev float [rows][vocab], 16-byte aligned
+ * when vocab % 4 == 0 (E_INVAL otherwise); scratch_dev: >= rows * 512 bytes of device memory. */
 int polestar_k_confidence(const float *logits_dev, int32_t rows, int32_t vocab, int32_t mask_id,
                           int32_t *yhat_dev, float *conf_dev, void *scratch_dev, size_t scratch_bytes,
                           void *cuda_stream);
@@ -312,7 +338,7 @@ int polestar_k_confidence(const float *logits_dev, int32_t rows, int32_t vocab, 
 int polestar_k_confidence_noalloc(const float *logits_dev, int32_t rows, int32_t vocab, int32_t mask_id,
                                   int32_t *yhat_dev, float *conf_dev, void *cuda_stream);
 
-/* Number of SMs the library sized its grids for (0 before any context exists). */
+/* Number of SMs of the device the library last sized grids for (0 before any call that launches kernels). */
 int polestar_sm_count(void);
 
 #ifdef __cplusplus

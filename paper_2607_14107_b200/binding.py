@@ -16,12 +16,15 @@ import torch
 from . import inputs as I
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libpolestar.so")
+# POLESTAR_LIB selects another build of the same library (e.g. the time-stamping build of `build.py --trace`)
+LIB_PATH = os.environ.get("POLESTAR_LIB") or os.path.join(_HERE, "libpolestar.so")
 
 OK, E_INVAL, E_STATE, E_NOSPACE, E_CUDA, E_NONFINITE, E_TIMEOUT, E_DONE = 0, -1, -2, -3, -4, -5, -6, -7
 
 READ_LOGITS, READ_CONF, READ_YHAT, READ_DELTA, READ_DRIFT, READ_SEL_COUNT, READ_SEL_IDX = 1, 2, 3, 4, 5, 6, 7
 READ_HIDDEN, READ_KCACHE, READ_VCACHE, READ_HCACHE, READ_COMMIT, READ_PPREV, READ_SUFFIX = 8, 9, 10, 11, 12, 13, 14
+READ_DRIFT_DELTA, READ_TAU_D, READ_THETA, READ_THETA_COUNT, READ_OWN_COMMIT = 15, 16, 17, 18, 19
+READ_TRACE_KERNELS, READ_TRACE_GEMM = 98, 99
 FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR, FORCE_TOKENS = 1, 2, 3, 4
 FLAG_SIMT_GEMM, FLAG_PROMPT_DEVICE, FLAG_PROFILE = 1 << 5, 1 << 6, 1 << 7
 PROF_FAMILIES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head", "attention", "stage", "select",
@@ -30,6 +33,7 @@ PROF_FAMILIES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_hea
 EXPORTS = [
     "polestar_workspace_bytes", "polestar_init", "polestar_step", "polestar_commit", "polestar_tokens",
     "polestar_read", "polestar_force", "polestar_profile", "polestar_destroy", "polestar_strerror",
+    "polestar_reload_env", "polestar_k_refresh_status",
     "polestar_k_attention", "polestar_k_hidden_delta", "polestar_k_select",
     "polestar_k_refresh_scratch_bytes", "polestar_k_refresh", "polestar_k_confidence",
     "polestar_k_confidence_noalloc", "polestar_sm_count",
@@ -126,6 +130,10 @@ def load():
     lib.polestar_k_confidence_noalloc.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     lib.polestar_sm_count.restype = C.c_int
     lib.polestar_sm_count.argtypes = []
+    lib.polestar_reload_env.restype = C.c_int
+    lib.polestar_reload_env.argtypes = []
+    lib.polestar_k_refresh_status.restype = C.c_int
+    lib.polestar_k_refresh_status.argtypes = [vp, sz, i32, i32, i32, i32, vp]
     _lib = lib
     return lib
 
@@ -254,7 +262,7 @@ class Polestar:
         need = int(lib.polestar_workspace_bytes(C.byref(cm), C.byref(cp)))
         if need == 0:
             raise PolestarError(E_INVAL, "invalid model / parameters")
-        self.workspace = torch.empty(need + 1024, dtype=torch.uint8, device="cuda")
+        self.workspace = torch.empty(need, dtype=torch.uint8, device="cuda")       # torch allocations are 512-byte aligned
         L = m.n_layers
         arr = lambda ts: (C.c_void_p * L)(*[t.data_ptr() for t in ts])
         self._arrays = [arr(packed[k]) for k in ("wqkv", "wo", "w_gate_up", "w_down", "norm1", "norm2")]
@@ -267,10 +275,8 @@ class Polestar:
             self._prompt = np.ascontiguousarray(np.asarray(prompt, dtype=np.int32).reshape(p.batch, p.prompt_len))
             prompt_ptr = self._prompt.ctypes.data_as(C.POINTER(C.c_int32))
         self.ctx = C.c_void_p()
-        base = (self.workspace.data_ptr() + 255) & ~255
         _check(lib.polestar_init(C.byref(self.ctx), C.byref(cm), C.byref(cw), C.byref(cp),
-                                 prompt_ptr, C.c_void_p(base),
-                                 need + 1024 - (base - self.workspace.data_ptr()), C.c_void_p(_stream())))
+                                 prompt_ptr, C.c_void_p(self.workspace.data_ptr()), need, C.c_void_p(_stream())))
         self.done = False
 
     def step(self) -> CStepInfo:
@@ -308,7 +314,11 @@ class Polestar:
                   READ_SEL_IDX: ((bs, Wm), np.int32), READ_HIDDEN: ((bs, B, m.d_model), np.float32),
                   READ_KCACHE: ((bs, N, dkv), el), READ_VCACHE: ((bs, N, dkv), el),
                   READ_HCACHE: ((bs, Wm, m.d_model), np.float32), READ_COMMIT: ((bs, B), np.int32),
-                  READ_PPREV: ((bs, Wm, m.n_heads, N), np.float32), READ_SUFFIX: ((bs, Wm), np.int32)}
+                  READ_PPREV: ((bs, Wm, m.n_heads, N), np.float32), READ_SUFFIX: ((bs, Wm), np.int32),
+                  READ_DRIFT_DELTA: ((bs, B), np.float32), READ_TAU_D: ((bs, B), np.float32),
+                  READ_THETA: ((bs, max(1, p.hist), B), np.float32), READ_THETA_COUNT: ((bs,), np.int32),
+                  READ_OWN_COMMIT: ((bs, B), np.int32),
+                  READ_TRACE_KERNELS: ((8192,), np.int64), READ_TRACE_GEMM: ((2048,), np.int64)}
         shape, dt = shapes[what]
         out = np.empty(shape, dt)
         _check(load().polestar_read(self.ctx, what, layer, out.ctypes.data_as(C.c_void_p), out.nbytes))
@@ -394,6 +404,16 @@ def polestar_k_refresh(h, idx, counts, wqkv, norm, kc, vc, q_out, max_rows, n_he
                                      _ptr(q_out), batch, P, max_rows, d, n_heads, n_kv_heads, head_dim, rms_eps,
                                      rope_theta, _dtype_code(h), _ptr(scratch), scratch.numel() * scratch.element_size(),
                                      C.c_void_p(_stream())))
+
+
+def polestar_reload_env() -> None:
+    """Make the stand-alone kernel calls re-read the POLESTAR_* environment switches."""
+    _check(load().polestar_reload_env())
+
+
+def polestar_k_refresh_status(scratch, batch, max_rows, d, head_dim) -> int:
+    return int(load().polestar_k_refresh_status(_ptr(scratch), scratch.numel() * scratch.element_size(), batch,
+                                                max_rows, d, head_dim, C.c_void_p(_stream())))
 
 
 def polestar_k_confidence(logits, mask_id, yhat, conf, scratch):

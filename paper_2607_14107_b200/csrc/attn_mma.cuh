@@ -1012,22 +1012,35 @@ __global__ void __launch_bounds__(BG_WARPS * 32) attention_big_kernel(AttnMmaArg
 }
 
 template <int NW, int TPW, int CL = 1>
-static int launch_attention_sp(const AttnMmaArgs& g, dim3 grid, cudaStream_t st) {
-    constexpr int smem = NW * 2 * SP_SLOT_BYTES + AT_BM * AT_DH * 2 + (CL > 1 ? AT_BM * AT_DH * 4 : 0) + 1024;
-    static bool attr = false;
-    if (!attr) {
-        if (cudaFuncSetAttribute(attention_sp_kernel<NW, TPW, CL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
-            return -4;
-        attr = true;
-    }
+constexpr int sp_smem_bytes() { return NW * 2 * SP_SLOT_BYTES + AT_BM * AT_DH * 2 + (CL > 1 ? AT_BM * AT_DH * 4 : 0) + 1024; }
+
+template <int NW, int TPW, int CL = 1>
+static cudaError_t launch_attention_sp(const AttnMmaArgs& g, dim3 grid, cudaStream_t st) {
+    constexpr int smem = sp_smem_bytes<NW, TPW, CL>();
     if (CL > 1) {
         grid.x *= CL;
-        return launch_k_cluster(attention_sp_kernel<NW, TPW, CL>, grid, dim3(NW * 32), smem, st, (unsigned)CL, g) == cudaSuccess ? 0 : -4;
+        return launch_k_cluster(attention_sp_kernel<NW, TPW, CL>, grid, dim3(NW * 32), smem, st, (unsigned)CL, g);
     }
-    return launch_k(attention_sp_kernel<NW, TPW, CL>, grid, dim3(NW * 32), smem, st, g) == cudaSuccess ? 0 : -4;
+    return launch_k(attention_sp_kernel<NW, TPW, CL>, grid, dim3(NW * 32), smem, st, g);
 }
 
-static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count = 148) {
+// Dynamic shared-memory limits of the kernels above; once per device, before their first launch there.
+static cudaError_t attention_mma_set_attributes() {
+    cudaError_t e;
+#define PS_ATTR(kern, bytes) if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e
+    PS_ATTR((attention_sp_kernel<8, 1, 2>), (sp_smem_bytes<8, 1, 2>()));
+    PS_ATTR((attention_sp_kernel<8, 2, 2>), (sp_smem_bytes<8, 2, 2>()));
+    PS_ATTR((attention_sp_kernel<8, 2, 1>), (sp_smem_bytes<8, 2, 1>()));
+    PS_ATTR((attention_sp_kernel<4, 4, 1>), (sp_smem_bytes<4, 4, 1>()));
+    PS_ATTR((attention_sp_kernel<8, 4, 1>), (sp_smem_bytes<8, 4, 1>()));
+    PS_ATTR(attention_big_kernel, BG_SMEM);
+    PS_ATTR(attention_mma_kernel, AT_SMEM);
+#undef PS_ATTR
+    return cudaSuccess;
+}
+
+// mode: 0 automatic, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>, 5 many-rows, 6 / 7 key split over two CTAs
+static cudaError_t launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count, int mode) {
     AttnMmaArgs g;
     g.a = a;
     const int batch = a.batch > 0 ? a.batch : 1;
@@ -1035,20 +1048,12 @@ static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count
     g.tiles_per_seq = (g.rows_per_seq + AT_BM - 1) / AT_BM;
     dim3 grid(g.tiles_per_seq * batch, a.n_heads);
     const long long ctas = (long long)grid.x * grid.y;
-    const char* force = getenv("POLESTAR_ATTN_KERNEL");
-    const int mode = force ? atoi(force) : 0;      // 0 auto, 1 two-pass, 2 <8,2>, 3 <4,4>, 4 <8,4>, 5 many-rows, 6 / 7 key split over two CTAs
     // many rows per head (entry forwards, long sequences): share each K/V tile among 64 rows
     const long long big_ctas = (long long)((g.rows_per_seq + BG_BM - 1) / BG_BM) * batch * a.n_heads;
     if (mode == 5 || (mode == 0 && (a.N > 8 * 4 * AT_BN || ctas >= 4LL * sm_count) && g.rows_per_seq >= 48 && big_ctas >= sm_count)) {
         AttnMmaArgs gb = g;
         gb.tiles_per_seq = (g.rows_per_seq + BG_BM - 1) / BG_BM;
-        static bool attr_b = false;
-        if (!attr_b) {
-            if (cudaFuncSetAttribute(attention_big_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, BG_SMEM) != cudaSuccess)
-                return -4;
-            attr_b = true;
-        }
-        return launch_k(attention_big_kernel, dim3(gb.tiles_per_seq * batch, a.n_heads), dim3(BG_WARPS * 32), BG_SMEM, st, gb) == cudaSuccess ? 0 : -4;
+        return launch_k(attention_big_kernel, dim3(gb.tiles_per_seq * batch, a.n_heads), dim3(BG_WARPS * 32), BG_SMEM, st, gb);
     }
     if (mode != 1) {
         // few rows: split the keys of every (row tile, head) over a cluster of two CTAs
@@ -1059,13 +1064,7 @@ static int launch_attention_mma(const AttnArgs& a, cudaStream_t st, int sm_count
         if ((mode == 3 || mode == 0) && a.N <= 4 * 4 * AT_BN) return launch_attention_sp<4, 4>(g, grid, st);
         if ((mode == 4 || mode == 0) && a.N <= 8 * 4 * AT_BN) return launch_attention_sp<8, 4>(g, grid, st);
     }
-    static bool attr = false;
-    if (!attr) {
-        if (cudaFuncSetAttribute(attention_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, AT_SMEM) != cudaSuccess)
-            return -4;
-        attr = true;
-    }
-    return launch_k(attention_mma_kernel, grid, dim3(AT_WARPS * 32), AT_SMEM, st, g) == cudaSuccess ? 0 : -4;
+    return launch_k(attention_mma_kernel, grid, dim3(AT_WARPS * 32), AT_SMEM, st, g);
 }
 
 }  // namespace ps

@@ -59,9 +59,11 @@ __device__ __forceinline__ uint32_t cluster_rank() {
     return r;
 }
 
-// ---- optional kernel timeline (debugging aid) ---------------------------------------------
-// When a trace buffer is installed, block 0 of every kernel records (kernel id, nanosecond time) once
-// its dependencies are resolved; consecutive stamps give each kernel's real cost inside the pipeline.
+// ---- optional kernel timeline (POLESTAR_TRACE builds only) ----------------------------------
+// In a library built with -DPOLESTAR_TRACE, block 0 of every kernel records (kernel id, nanosecond time) once
+// its dependencies are resolved; consecutive stamps give each kernel's real cost inside the pipeline.  The
+// default build compiles none of this.
+#ifdef POLESTAR_TRACE
 __device__ long long* g_trace_buf = nullptr;   // [0] = next slot, then pairs (id, time)
 __device__ __forceinline__ void trace_stamp(int id, int thread = 0) {
     long long* t = g_trace_buf;
@@ -74,6 +76,9 @@ __device__ __forceinline__ void trace_stamp(int id, int thread = 0) {
         }
     }
 }
+#else
+__device__ __forceinline__ void trace_stamp(int, int = 0) {}
+#endif
 #define KERNEL_PROLOGUE(id) do { pdl_trigger(); pdl_wait(); trace_stamp(id); } while (0)
 
 // ---- rows of one forward -----------------------------------------------------------

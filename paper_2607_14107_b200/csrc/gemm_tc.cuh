@@ -170,8 +170,6 @@ __host__ __device__ inline uint32_t instr_desc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-constexpr int PSTRIDE = BLOCK_F + 4;     // floats per token row of a partial tile in shared memory (conflict-free float4 rows)
-
 struct SkArgs {
     int M, N_out, K, stages;
     int tiles_f, tiles_t;
@@ -181,19 +179,17 @@ struct SkArgs {
     int done_offset;
     int* status;        // set to 1 on a wait time-out
     int w_stream;       // 1: every weight byte is read once by this launch: load it with the evict_first L2 policy
-    int cluster_n;      // > 0: launched in clusters of cluster_n CTAs = the contributors of one output tile;
-                        // partial tiles are then exchanged through distributed shared memory, not global memory
-    long long* trace;   // optional [gridDim.x][12] nanosecond stamps of this launch (null: off): 0 start, 1 set-up done,
-                        // 2 dependencies resolved, 3 first stage full, 4 last MMA issued, 5 partial tiles published,
-                        // 6 other contributors arrived, 8 share reduced, 7 end
-    // L2 prefetch of weights that later GEMMs of the stream will read: while this kernel's epilogue and
-    // fix-up run, HBM would otherwise idle.  Entry j: tile-major weight base, that GEMM's unit count and grid,
-    // and the slice [first, first + count) of every CTA's unit range to prefetch (count 0: unused).
-    struct Prefetch { const char* w; long long U; int G; int first, count; } pf[2];
+    long long* trace;   // POLESTAR_TRACE builds: [gridDim.x][12] nanosecond stamps of this launch (null: off): 0 start,
+                        // 1 set-up done, 2 dependencies resolved, 3 first stage full, 4 last MMA issued, 5 partial tiles
+                        // published, 6 other contributors arrived, 8 share reduced, 7 end
 };
 
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#ifdef POLESTAR_TRACE
 #define SK_STAMP(i) do { if (g.trace) g.trace[(size_t)cta * 12 + (i)] = gtime(); } while (0)
+#else
+#define SK_STAMP(i) do { } while (0)
+#endif
 
 // first unit of CTA c when U units are split over G CTAs
 __device__ __forceinline__ long long sk_begin(long long U, int G, int c) { return (U * c) / G; }
@@ -267,7 +263,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const int tiles_all = g.tiles_f * g.tiles_t;
     // (the stream-K part is the remainder r = tiles mod G when that leaves at most ~8 CTAs per tile, else G + r tiles)
     const int rem = tiles_all % G;
-    const int dp = (g.cluster_n > 0 || tiles_all < G) ? 0 : ((rem == 0 || rem * 8 >= G) ? tiles_all / G : tiles_all / G - 1);
+    const int dp = (tiles_all < G) ? 0 : ((rem == 0 || rem * 8 >= G) ? tiles_all / G : tiles_all / G - 1);
     const int tile_base = dp * G;
     const long long U = (long long)(tiles_all - tile_base) * kb_total;
     const long long u_begin = sk_begin(U, G, cta), u_end = sk_begin(U, G, cta + 1);
@@ -303,28 +299,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     const uint32_t tmem_base = tmem_base_sh;
     volatile int* abort_flag = &abort_sh;
 
-    if (threadIdx.x == THREADS + 32 && (g.pf[0].count > 0 || g.pf[1].count > 0) && n_units > 0) {
-        // Optional L2 prefetch of the weights later GEMMs will stream, by an otherwise idle thread, once this CTA's
-        // last accumulator is complete (its own stream has ended, so the prefetch competes with nothing of ours).
-        const int n_seg = dp + (n_tail > 0 ? (int)((u_end - 1) / kb_total - u_begin / kb_total) + 1 : 0);
-        const int last = n_seg - 1;
-        if (mbar_wait(accum_full + 8 * (last & 1), (uint32_t)(last >> 1) & 1u, abort_flag)) {
-            uint64_t pol_keep;
-            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-#pragma unroll
-            for (int j = 0; j < 2; ++j) {
-                if (g.pf[j].count > 0 && cta < g.pf[j].G) {
-                    const long long nb = sk_begin(g.pf[j].U, g.pf[j].G, cta) + g.pf[j].first;
-                    const long long ne = sk_begin(g.pf[j].U, g.pf[j].G, cta + 1);
-                    const int n = (int)max(0LL, min((long long)g.pf[j].count, ne - nb));
-                    for (int i = 0; i < n; ++i) {
-                        const char* src = g.pf[j].w + (size_t)(nb + i) * W_BYTES;
-                        asm volatile("cp.async.bulk.prefetch.L2.global.L2::cache_hint [%0], %1, %2;" ::"l"(src), "r"(W_BYTES), "l"(pol_keep) : "memory");
-                    }
-                }
-            }
-        }
-    }
     if (threadIdx.x == THREADS) {
         // An idle thread works out, while the main loop runs, which partial tiles this CTA will help reduce and
         // which share of their items is its own (64-bit divisions that must not sit on the tail's critical path).
@@ -333,7 +307,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // A tile's items (one row x 16 columns each) are dealt to its contributors in contiguous shares; a CTA that
         // contributes to two tiles takes half a share of each, so that every CTA reduces about as many items.
         int n_fix = 0;
-        if (g.cluster_n == 0 && n_tail > 0) {
+        if (n_tail > 0) {
             const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;       // (stream-K part's own numbering)
             const bool head_cut = u_begin != tb * kb_total, tail_cut = u_end != (te + 1) * kb_total;
             int fix_tile[2] = {0, 0};
@@ -502,24 +476,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
-            } else if (g.cluster_n > 0) {
-                // cluster path: the partial tile goes to this CTA's shared memory (the operand ring is idle once
-                // the last MMA has completed); the cluster adds the tiles up after the barrier further down
-                float* prow = reinterpret_cast<float*>(smem) + (size_t)t_local * PSTRIDE;
-                if (warp_live) {
-                    for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
-                        float v[16];
-                        tmem_ld16(taddr + (uint32_t)c0, v);
-                        if (live) {
-#pragma unroll
-                            for (int c = 0; c < 16; c += 4)
-                                *reinterpret_cast<float4*>(prow + c0 + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
-                        }
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
             } else {
                 // partial segment: publish it now, reduce later (pass 2), so that publishing never
                 // waits on another CTA
@@ -554,7 +510,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
 
     // ---- pass 2 (all warps): every CTA that contributed to split tiles reduces its share of them ------------
-    if (g.cluster_n == 0 && n_units > 0) {
+    if (n_units > 0) {
         __syncwarp();
         pdl_wait();
         const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
@@ -682,54 +638,6 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
             }
         }
-    }
-
-    if (g.cluster_n > 0) {
-        // Every CTA of the cluster worked on the same output tile (consecutive k ranges, rank = k order).  All
-        // threads meet at the cluster barrier; then each CTA adds up its share of the tile, reading the other
-        // CTAs' partial tiles through distributed shared memory in rank order (deterministic), and runs the epilogue.
-        cluster_sync_all();
-        if (warp >= 2 && warp < 6 && !abort_sh) {
-            const int tile = (int)(u_begin / kb_total);
-            int tile_f, tile_t;
-            tile_ft(tile, g.tiles_f, g.tiles_t, tile_f, tile_t);
-            const int n0 = tile_f * BLOCK_F;
-            const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
-            const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
-            const int n_items = n_live * (BLOCK_F / 16);
-            const int rank = cta % g.cluster_n;
-            for (int item = rank * 128 + ((int)threadIdx.x - 64); item < n_items; item += g.cluster_n * 128) {
-                const int tl = item / (BLOCK_F / 16), c0 = (item % (BLOCK_F / 16)) * 16;
-                const uint32_t local = smem_base + (uint32_t)((tl * PSTRIDE + c0) * 4);
-                float acc[16];
-#pragma unroll
-                for (int x = 0; x < 16; ++x) acc[x] = 0.f;
-                for (int r0 = 0; r0 < g.cluster_n; r0 += 4) {
-                    float4 tv[4][4];
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (r0 + j < g.cluster_n) {
-                            const uint32_t ra = dsmem_addr(local, (uint32_t)(r0 + j));
-#pragma unroll
-                            for (int x = 0; x < 4; ++x) tv[j][x] = ld_dsmem_f4(ra + 16 * x);
-                        } else {
-#pragma unroll
-                            for (int x = 0; x < 4; ++x) tv[j][x] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-#pragma unroll
-                        for (int x = 0; x < 4; ++x) {
-                            acc[4 * x] += tv[j][x].x; acc[4 * x + 1] += tv[j][x].y;
-                            acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
-                        }
-                }
-                const int mm = tile_t * BLOCK_T + tl;
-                epilogue16<T, EPI>(e, mm, n0 + c0, acc);
-            }
-        }
-        cluster_sync_all();       // nobody leaves while its partial tile may still be read
     }
 
     tc_fence_before();

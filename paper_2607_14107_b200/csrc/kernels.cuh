@@ -822,6 +822,7 @@ struct CommitArgs {
     float* Delta_out; float* taud_out;
     float* theta; int* theta_cnt;   // [batch][hist][B] ring, [batch] number pushed so far
     int* commit_flags;           // [batch][B]
+    int* own_flags;              // [batch][B]: the rule's own decision, before a forced decision replaces it
     int* suffix_flags;           // [batch][W_max]
     const int* head_count; const int* suf_seq; const int* suf_w;
     const int* forced_pos; int forced_n;      // [batch][forced_n] absolute positions, -1 unused (null: free-running)
@@ -882,18 +883,7 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
     __syncthreads();
     if (j == 0 && within && a.hist > 0) a.theta_cnt[s] = a.theta_cnt[s] + 1;
     const int n_masked = cnt[6];
-    if (a.forced_pos) {
-        if (j < B) {
-            flag = 0;
-            const int pos = sd.act_start + j;
-            for (int u = 0; u < a.forced_n; ++u)
-                if (a.forced_pos[s * a.forced_n + u] == pos) {
-                    flag = s_flag[j] ? s_flag[j] : (1 | 8);
-                    if (a.forced_tok) yh = a.forced_tok[s * a.forced_n + u];
-                }
-            if (!masked) flag = 0;
-        }
-    } else {
+    {
         // quota top-up: the most confident masked rows not yet committed (ties: lowest position)
         const int denom = max(1, a.steps_per_block - a.steps_used);
         const int quota = n_masked > 0 ? (n_masked + denom - 1) / denom : 0;
@@ -903,6 +893,21 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
             for (int u = 0; u < B; ++u)
                 if (s_masked[u] && !s_flag[u] && (s_conf[u] > c || (s_conf[u] == c && u < j))) ++rank;
             if (rank < need) flag = 1 | 8;
+        }
+    }
+    if (j < B) a.own_flags[s * B + j] = flag;
+    if (a.forced_pos) {
+        // a forced decision replaces the rule's own (kept in own_flags); the label of a row the rule also chose stays
+        if (j < B) {
+            const int own = flag;
+            flag = 0;
+            const int pos = sd.act_start + j;
+            for (int u = 0; u < a.forced_n; ++u)
+                if (a.forced_pos[s * a.forced_n + u] == pos) {
+                    flag = own ? own : (1 | 8);
+                    if (a.forced_tok) yh = a.forced_tok[s * a.forced_n + u];
+                }
+            if (!masked) flag = 0;
         }
     }
     __syncthreads();
@@ -931,12 +936,12 @@ __global__ void commit_kernel(StepDesc sd, CommitArgs a) {
             const float sc = a.conf[sd.batch * B + i];
             bool ok = a.ge ? (sc >= a.tau_suffix) : (sc > a.tau_suffix);
             int t2 = a.yhat[sd.batch * B + i];
+            int f = 1 | (ok ? 4 : 0);          // bit 2: the rule's own decision for this eligible row
             if (a.forced_pos) {
                 ok = false;
                 for (int u = 0; u < a.forced_n; ++u)
                     if (a.forced_pos[s * a.forced_n + u] == pos) { ok = true; if (a.forced_tok) t2 = a.forced_tok[s * a.forced_n + u]; }
             }
-            int f = 1;
             if (ok && a.y[s * sd.N + pos] == a.mask_id) {
                 a.y[s * sd.N + pos] = t2;
                 f |= 2;

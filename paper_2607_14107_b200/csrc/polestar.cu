@@ -10,7 +10,9 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <map>
+#include <mutex>
 #include <new>
 #include <tuple>
 #include <vector>
@@ -29,14 +31,88 @@ using namespace ps;
     } while (0)
 
 static thread_local cudaError_t last_cuda_error = cudaSuccess;
-static int g_sm_count = 0;
 
+// ------------------------------------------------------------------------------------------
+// environment switches: read by polestar_init (into the context) and by polestar_reload_env,
+// never on the launch path
+// ------------------------------------------------------------------------------------------
+struct Switches {
+    int pdl = 1;             // POLESTAR_PDL: programmatic dependent launch between the kernels of a forward
+    int evict_first = 1;     // POLESTAR_GEMM_EVICT_FIRST: weight TMA loads carry the evict_first L2 policy
+    int fuse_select = 1;     // POLESTAR_FUSE_SELECT: batch-1 selection inside the O projection
+    int chain = 1;           // POLESTAR_CHAIN: O -> norm -> gate/up -> down as one persistent launch
+    int stages = 0;          // POLESTAR_GEMM_STAGES: operand ring depth (0 = 3 for one token tile, else 4)
+    int align_pct = 85;      // POLESTAR_GEMM_ALIGN_PCT
+    int half_align = 1;      // POLESTAR_GEMM_HALF_ALIGN
+    int attn_kernel = 0;     // POLESTAR_ATTN_KERNEL: 0 automatic, else force a kernel variant
+    int attn_simt = 0;       // POLESTAR_ATTN_SIMT: CUDA-core attention for bf16 models (debugging)
+    int refresh_simt = 0;    // POLESTAR_REFRESH_SIMT
+    int fuse_prep = 0;       // POLESTAR_FUSE_PREP (measured negative result, kept with its test)
+    int fold_norm = 0;       // POLESTAR_FOLD_NORM (same)
+    int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
+    int l2promo = (int)CU_TENSOR_MAP_L2_PROMOTION_L2_128B;   // POLESTAR_TMA_L2PROMO
+    int gemm_trace = -1;     // POLESTAR_GEMM_TRACE (POLESTAR_TRACE builds)
+    int kernel_trace = 0;    // POLESTAR_KERNEL_TRACE (POLESTAR_TRACE builds)
+};
 static int env_int(const char* name, int dflt) {
     const char* s = getenv(name);
     return s ? atoi(s) : dflt;
 }
+static Switches read_switches() {
+    Switches w;
+    w.pdl = env_int("POLESTAR_PDL", w.pdl);
+    w.evict_first = env_int("POLESTAR_GEMM_EVICT_FIRST", w.evict_first);
+    w.fuse_select = env_int("POLESTAR_FUSE_SELECT", w.fuse_select);
+    w.chain = env_int("POLESTAR_CHAIN", w.chain);
+    w.stages = env_int("POLESTAR_GEMM_STAGES", w.stages);
+    w.align_pct = env_int("POLESTAR_GEMM_ALIGN_PCT", w.align_pct);
+    w.half_align = env_int("POLESTAR_GEMM_HALF_ALIGN", w.half_align);
+    w.attn_kernel = env_int("POLESTAR_ATTN_KERNEL", w.attn_kernel);
+    w.attn_simt = env_int("POLESTAR_ATTN_SIMT", w.attn_simt);
+    w.refresh_simt = env_int("POLESTAR_REFRESH_SIMT", w.refresh_simt);
+    w.fuse_prep = env_int("POLESTAR_FUSE_PREP", w.fuse_prep);
+    w.fold_norm = env_int("POLESTAR_FOLD_NORM", w.fold_norm);
+    w.chain_qkv = env_int("POLESTAR_CHAIN_QKV", w.chain_qkv);
+    w.l2promo = env_int("POLESTAR_TMA_L2PROMO", w.l2promo);
+    w.gemm_trace = env_int("POLESTAR_GEMM_TRACE", w.gemm_trace);
+    w.kernel_trace = env_int("POLESTAR_KERNEL_TRACE", w.kernel_trace);
+    return w;
+}
+static std::mutex g_mu;                 // guards g_sw and g_dev
+static Switches g_sw;                   // switches of the stand-alone kernel calls
+static bool g_sw_loaded = false;
+static Switches stand_alone_switches() {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (!g_sw_loaded) { g_sw = read_switches(); g_sw_loaded = true; }
+    return g_sw;
+}
 
+// ------------------------------------------------------------------------------------------
+// per-device facts: SM count, dynamic shared-memory attributes of the kernels, built-in scratch
+// ------------------------------------------------------------------------------------------
+struct DevInfo { bool ready = false; int sm_count = 0; };
+static const int MAX_DEVICES = 64;
+static DevInfo g_dev[MAX_DEVICES];
+static int g_last_sm_count = 0;
 
+static cudaError_t set_kernel_attributes();
+// Facts of the CURRENT device; the first call on a device queries it and raises the shared-memory limits of
+// every kernel that needs more than the default there (function attributes are per device).
+static int device_info(DevInfo* out) {
+    int dev = 0;
+    CK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return POLESTAR_E_INVAL;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DevInfo& di = g_dev[dev];
+    if (!di.ready) {
+        CK(cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev));
+        CK(set_kernel_attributes());
+        di.ready = true;
+    }
+    g_last_sm_count = di.sm_count;
+    *out = di;
+    return POLESTAR_OK;
+}
 
 // ------------------------------------------------------------------------------------------
 // tensor maps (TMA descriptors) through the driver entry point, no libcuda link dependency
@@ -45,18 +121,21 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn get_encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    static std::atomic<EncodeTiledFn> fn{nullptr};
+    EncodeTiledFn f = fn.load();
+    if (!f) {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
+            qres == cudaDriverEntryPointSuccess) {
+            f = (EncodeTiledFn)p;
+            fn.store(f);
+        }
     }
-    return fn;
+    return f;
 }
 // bf16 matrix [rows, K] row-major, box = box_rows x 64 elements, 128-byte swizzle
-static bool make_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t K, uint32_t box_rows) {
+static bool make_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t K, uint32_t box_rows, int l2promo) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {K, rows};
@@ -64,18 +143,21 @@ static bool make_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t
     cuuint32_t box[2] = {64, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, (CUtensorMapL2promotion)env_int("POLESTAR_TMA_L2PROMO", CU_TENSOR_MAP_L2_PROMOTION_L2_128B),
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, (CUtensorMapL2promotion)l2promo,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor maps of one context (its weights and staging buffers at the handful of row counts a decode uses);
+// owned by the context, so it is bounded by the context's buffers and needs no lock.
 struct MapCache {
     std::map<std::tuple<const void*, uint64_t, uint64_t, uint32_t>, CUtensorMap> m;
+    int l2promo = (int)CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
     const CUtensorMap* get(const void* base, uint64_t rows, uint64_t K, uint32_t box_rows) {
         auto key = std::make_tuple(base, rows, K, box_rows);
         auto it = m.find(key);
         if (it != m.end()) return &it->second;
         CUtensorMap tm;
-        if (!make_map(&tm, base, rows, K, box_rows)) return nullptr;
+        if (!make_map(&tm, base, rows, K, box_rows, l2promo)) return nullptr;
         return &m.emplace(key, tm).first->second;
     }
 };
@@ -91,6 +173,8 @@ struct GemmWs {
     mutable unsigned post_total = 0;       // its value once every launch so far has completed
     unsigned* chain_counter = nullptr;     // the same for chained launches
     mutable unsigned chain_total = 0;
+    int sms = 148;                         // SMs of the device the launches go to
+    Switches sw;
 };
 
 // bf16 matrices with out % 256 == 0 and in % 64 == 0 are stored tile-major (see polestar.h)
@@ -106,20 +190,17 @@ static int launch_gemm_simt(const void* A, const void* W, int M, int N_out, int 
     return POLESTAR_OK;
 }
 
-// Weights a later GEMM of the same forward will stream (for L2 prefetch during this GEMM's tail).
-struct NextW { const void* w = nullptr; int N_out = 0, K = 0, M = 0, first = 0, count = 0; };
-
 // stream-K grid of a GEMM with M rows: G CTAs over U units
-static void sk_grid(int M, int N_out, int K, long long* U, long long* G) {
+static void sk_grid(const GemmWs& ws, int M, int N_out, int K, long long* U, long long* G) {
     const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + tc::BLOCK_T - 1) / tc::BLOCK_T;
-    const int sms = g_sm_count > 0 ? g_sm_count : 148;
+    const int sms = ws.sms;
     *U = (long long)tiles_f * tiles_t * (K / 64);
     long long g = std::min<long long>((long long)sms, *U);
     const long long tiles = (long long)tiles_f * tiles_t;
     const long long mult = (g / tiles) * tiles;
-    const int pct = env_int("POLESTAR_GEMM_ALIGN_PCT", 85);
+    const int pct = ws.sw.align_pct;
     if (mult > 0 && mult * 100 >= (long long)sms * pct) g = mult;
-    else if (tiles % 2 == 0 && env_int("POLESTAR_GEMM_HALF_ALIGN", 1)) {
+    else if (tiles % 2 == 0 && ws.sw.half_align) {
         // next best: a multiple of half the tile count, so that CTA ranges cross a tile boundary only in every
         // third (fifth, ...) CTA instead of in nearly all of them
         const long long half = tiles / 2, mult2 = (g / half) * half;
@@ -129,39 +210,20 @@ static void sk_grid(int M, int N_out, int K, long long* U, long long* G) {
 }
 
 template <int EPI>
-static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a_rows_alloc, const void* W, int M,
-                          int N_out, int K, const EpiArgs& e, cudaStream_t st, const NextW* next = nullptr,
+static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const void* W, int M,
+                          int N_out, int K, const EpiArgs& e, cudaStream_t st,
                           const PostArgs* post = nullptr, const tc::SelFuse* sel = nullptr) {
     if (M <= 0) return POLESTAR_OK;
-    (void)a_rows_alloc;
     // weights: tile-major [chunks * 256][64]; activations: exactly M rows, so that the rows of a token tile
     // beyond M are out of bounds and arrive as zeros without being read
     const CUtensorMap* mw = maps.get(W, (uint64_t)N_out * (uint64_t)(K / 64), 64, tc::BLOCK_F);
     const CUtensorMap* ma = maps.get(A, (uint64_t)M, (uint64_t)K, tc::BLOCK_T);
     if (!mw || !ma) return POLESTAR_E_CUDA;
     const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + tc::BLOCK_T - 1) / tc::BLOCK_T;
-    const int kb = K / 64;
-    const int sms = g_sm_count > 0 ? g_sm_count : 148;
     // When a multiple of the tile count fits on >= 85 % of the SMs, the grid takes it: CTA ranges then never
     // cross a tile boundary, so every CTA has one segment (one fix-up instead of two, or none at all).
     long long U, G;
-    sk_grid(M, N_out, K, &U, &G);
-    (void)kb;
-    // Cluster path: when the output tiles can be split over n <= 8 CTAs each with n * tiles covering >= 85 % of
-    // the SMs, the n contributors of a tile form a thread-block cluster and add their partial tiles up through
-    // distributed shared memory (no global round trips, no waiting on a counter).
-    int cluster_n = 0;
-    {
-        const long long tiles = (long long)tiles_f * tiles_t;
-        const long long n = std::min<long long>(8, sms / tiles);
-        // Off by default: on B200 at most 45 clusters of 3 / 15 clusters of 8 CTAs with this much shared memory
-        // are co-resident (GPC sizes), fewer than the 48 / 16 the 8B shapes need, so the grid ran in two waves.
-        if (env_int("POLESTAR_GEMM_CLUSTER", 0) && n >= 2 && tiles * n * 100 >= (long long)sms * 85 &&
-            (size_t)tc::BLOCK_T * tc::PSTRIDE * 4 <= (size_t)4 * tc::STAGE_BYTES) {
-            cluster_n = (int)n;
-            G = tiles * n;
-        }
-    }
+    sk_grid(ws, M, N_out, K, &U, &G);
     while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
     if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
     tc::SkArgs g;
@@ -169,29 +231,13 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     // Three stages (145 KB) for the weight-bound steps: measured +2 % tokens/s over four (the HBM stream needs no more in
     // flight, and less shared memory per block leaves room for the next kernel's blocks to become resident early); two
     // stages are 4 % slower.  Four stages when operands come from L2 (several token tiles).
-    g.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", tiles_t == 1 ? 3 : 4)));
+    g.stages = std::max(2, std::min(4, ws.sw.stages > 0 ? ws.sw.stages : (tiles_t == 1 ? 3 : 4)));
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
-    g.cluster_n = cluster_n;
-    g.w_stream = (g.tiles_t == 1 && env_int("POLESTAR_GEMM_EVICT_FIRST", 1)) ? 1 : 0;
-    // debug: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
-    memset(g.pf, 0, sizeof(g.pf));
-    for (int j = 0; next && j < 2; ++j) {
-        if (!next[j].w || next[j].count <= 0 || next[j].M > tc::BLOCK_T) continue;      // only weight-bound successors
-        if (next[j].N_out % tc::BLOCK_F || next[j].K % 64) continue;
-        long long nU, nG;
-        sk_grid(next[j].M, next[j].N_out, next[j].K, &nU, &nG);
-        g.pf[j].w = (const char*)next[j].w; g.pf[j].U = nU; g.pf[j].G = (int)nG;
-        g.pf[j].first = next[j].first; g.pf[j].count = next[j].count;
-    }
-    g.trace = (env_int("POLESTAR_GEMM_TRACE", -1) == EPI) ? (long long*)((char*)ws.partial + ws.partial_bytes - 16384) : nullptr;
+    g.w_stream = (g.tiles_t == 1 && ws.sw.evict_first) ? 1 : 0;
+    // POLESTAR_TRACE builds: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
+    g.trace = (ws.sw.gemm_trace == EPI) ? (long long*)((char*)ws.partial + ws.partial_bytes - 16384) : nullptr;
     const size_t smem = (size_t)g.stages * tc::STAGE_BYTES + 1024;
     auto kern = tc::gemm_sk_kernel<__nv_bfloat16, EPI>;
-    static bool attr = false;
-    if (!attr) {
-        // (four stages of 48 KB + alignment slack; static shared memory comes on top of it)
-        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (int)tc::STAGE_BYTES + 1024));
-        attr = true;
-    }
     PostArgs pa;
     memset(&pa, 0, sizeof(pa));
     if (post && post->kind && ws.post_counter) {
@@ -202,8 +248,7 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, int a
     }
     tc::SelFuse sfz;
     if (sel) sfz = *sel; else memset(&sfz, 0, sizeof(sfz));
-    if (cluster_n > 0) CK(launch_k_cluster(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, (unsigned)cluster_n, *mw, *ma, g, e, pa, sfz));
-    else CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e, pa, sfz));
+    CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e, pa, sfz));
     return POLESTAR_OK;
 }
 
@@ -224,7 +269,7 @@ struct Buffers {
     int* y; float2* rope; char* kc; char* vc; float* hc; float* pprev; float* aprev; float* theta; int* theta_cnt;
     int* tok_at_h0; float* drift; int* sel_idx; int* sel_cnt; unsigned char* patch; int* forced_idx; int* forced_cnt;
     int* forced_commit; int* forced_tok; float* conf; int* yhat; float* delta; float* Delta; float* taud; int* commit_flags;
-    int* suffix_flags; int* seq_info; int* head_count; int* suf_seq; int* suf_w; int* stats; int* status;
+    int* own_flags; int* suffix_flags; int* seq_info; int* head_count; int* suf_seq; int* suf_w; int* stats; int* status;
     int* list_count; float* hidden_keep;
     // scratch
     Row* rows; unsigned char* kvflag; float* x; float* x1; float* packet; char* a_buf; char* q_buf; char* o_buf;
@@ -253,7 +298,7 @@ static int launch_gemm_chain(MapCache& maps, const GemmWs& ws, const ChainSpec* 
     for (int i = 0; i < n; ++i) {
         if (sp[i].N_out % tc::BLOCK_F || sp[i].K % 64) return POLESTAR_OK;
         long long U;
-        sk_grid(M, sp[i].N_out, sp[i].K, &U, &Gp[i]);
+        sk_grid(ws, M, sp[i].N_out, sp[i].K, &U, &Gp[i]);
         if (sp[i].N_out / tc::BLOCK_F > Gp[i]) return POLESTAR_OK;
         G0 = std::max(G0, Gp[i]);
     }
@@ -275,7 +320,7 @@ static int launch_gemm_chain(MapCache& maps, const GemmWs& ws, const ChainSpec* 
     }
     for (int i = n; i < tc::CHAIN_MAX; ++i) { cm.w[i] = cm.w[0]; cm.a[i] = cm.a[0]; }
     ca.n = n;
-    ca.stages = std::max(2, std::min(4, env_int("POLESTAR_GEMM_STAGES", 3)));
+    ca.stages = std::max(2, std::min(4, ws.sw.stages > 0 ? ws.sw.stages : 3));
     ca.partial = ws.partial; ca.tile_counter = ws.counters; ca.done_offset = ws.n_counters / 2; ca.status = ws.status;
     ca.bar_counter = ws.chain_counter;
     ca.bar_base = ws.chain_total;
@@ -283,13 +328,7 @@ static int launch_gemm_chain(MapCache& maps, const GemmWs& ws, const ChainSpec* 
     tc::SelFuse sfz;
     if (sel) sfz = *sel; else memset(&sfz, 0, sizeof(sfz));
     const size_t smem = (size_t)ca.stages * tc::STAGE_BYTES + 1024;
-    auto kern = tc::gemm_chain_kernel<T>;
-    static bool attr = false;
-    if (!attr) {
-        CK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 4 * (int)tc::STAGE_BYTES + 1024));
-        attr = true;
-    }
-    CK(launch_k(kern, dim3((unsigned)G0), dim3(tc::FIX_THREADS), smem, st, cm, ca, sfz));
+    CK(launch_k(tc::gemm_chain_kernel<T>, dim3((unsigned)G0), dim3(tc::FIX_THREADS), smem, st, cm, ca, sfz));
     *applies = true;
     return POLESTAR_OK;
 }
@@ -309,10 +348,15 @@ struct polestar_ctx {
     MapCache maps;
     GemmWs gws;
     int es;          // element size of the model dtype
+    int device = 0;  // CUDA device the context was created on
+    int sms = 148;
+    Switches sw;
     int N, B, W_max, n_blocks, M_max, rows_lm;
     // controller
     int block = 0;
     bool need_entry = true, pending = false, done = false;
+    bool trace_installed = false;
+    bool failed = false;     // a device-side wait timed out: counters and caches are in an unknown state
     int steps_used = 0;
     long long forwards = 0, generated = 0, generated_non_eos = 0;
     std::vector<int> cum;
@@ -421,6 +465,7 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(Delta, float, bs * B);
     TAKE(taud, float, bs * B);
     TAKE(commit_flags, int, bs * B);
+    TAKE(own_flags, int, bs * B);
     TAKE(suffix_flags, int, bs * Wm);
     TAKE(seq_info, int, bs * 8 + 8);
     TAKE(head_count, int, 1);
@@ -454,10 +499,22 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
 
 extern "C" size_t polestar_workspace_bytes(const polestar_model* m, const polestar_params* p) {
     if (!valid_cfg(m, p)) return 0;
-    return make_plan(m, p, nullptr, nullptr);
+    // the plan is laid out from a 1024-byte boundary inside the caller's buffer: a 256-byte aligned base can lose 768 bytes
+    return make_plan(m, p, nullptr, nullptr) + 1024;
 }
 
-extern "C" int polestar_sm_count(void) { return g_sm_count; }
+extern "C" int polestar_sm_count(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_last_sm_count;
+}
+
+extern "C" int polestar_reload_env(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_sw = read_switches();
+    g_sw_loaded = true;
+    g_use_pdl = g_sw.pdl != 0;
+    return POLESTAR_OK;
+}
 
 extern "C" const char* polestar_strerror(int code) {
     switch (code) {
@@ -473,13 +530,22 @@ extern "C" const char* polestar_strerror(int code) {
     }
 }
 
-static int init_device_info() {
-    if (g_sm_count == 0) {
-        int dev = 0;
-        CK(cudaGetDevice(&dev));
-        CK(cudaDeviceGetAttribute(&g_sm_count, cudaDevAttrMultiProcessorCount, dev));
-    }
-    return POLESTAR_OK;
+static const size_t SIMT_ATTN_SMEM_MAX = 200 * 1024;
+static cudaError_t set_kernel_attributes() {
+    cudaError_t e;
+    const int gemm_smem = 4 * (int)tc::STAGE_BYTES + 1024;    // four stages of 48 KB + alignment slack
+#define PS_ATTR(kern, bytes) if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_RESID>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_SWIGLU>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_DOWN>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_LOGITS>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV_REFRESH>), gemm_smem);
+    PS_ATTR(tc::gemm_chain_kernel<__nv_bfloat16>, gemm_smem);
+    PS_ATTR(attention_simt_kernel<float>, (int)SIMT_ATTN_SMEM_MAX);
+    PS_ATTR(attention_simt_kernel<__nv_bfloat16>, (int)SIMT_ATTN_SMEM_MAX);
+#undef PS_ATTR
+    return attention_mma_set_attributes();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -490,30 +556,28 @@ struct Path {
     static constexpr bool is_bf16 = sizeof(T) == 2;
 
     template <int EPI>
-    static int gemm(polestar_ctx* c, const void* A, int a_rows_alloc, const void* W, int M, int N_out, int K,
-                    const EpiArgs& e, const NextW* next = nullptr, const PostArgs* post = nullptr, bool* fused = nullptr,
+    static int gemm(polestar_ctx* c, const void* A, const void* W, int M, int N_out, int K,
+                    const EpiArgs& e, const PostArgs* post = nullptr, bool* fused = nullptr,
                     const tc::SelFuse* sel = nullptr) {
         if (fused) *fused = false;
         if (is_bf16 && !(c->p.flags & POLESTAR_FLAG_SIMT_GEMM) && K % 64 == 0 && N_out % 256 == 0) {
             const bool fuse = post && post->kind && c->gws.post_counter && post->d <= 4 * NORM_VPT * tc::FIX_THREADS &&
-                              env_int("POLESTAR_FUSE_PREP", 0);      // measured on B200: no faster than the separate kernel
-                                                                     // (grid-wide counter round trip = kernel boundary)
+                              c->sw.fuse_prep;      // measured on B200: no faster than the separate kernel
+                                                    // (grid-wide counter round trip = kernel boundary)
             if (fused) *fused = fuse;
-            return launch_gemm_tc<EPI>(c->maps, c->gws, A, a_rows_alloc, W, M, N_out, K, e, c->st, next, fuse ? post : nullptr, sel);
+            return launch_gemm_tc<EPI>(c->maps, c->gws, A, W, M, N_out, K, e, c->st, fuse ? post : nullptr, sel);
         }
         return launch_gemm_simt<T, EPI>(A, W, M, N_out, K, e, c->st);
     }
 
     static int attention(polestar_ctx* c, const AttnArgs& a) {
-        if (is_bf16 && c->m.head_dim == 128 && !env_int("POLESTAR_ATTN_SIMT", 0))
-            return launch_attention_mma(a, c->st);
+        if (is_bf16 && c->m.head_dim == 128 && !c->sw.attn_simt) {
+            CK(launch_attention_mma(a, c->st, c->sms, c->sw.attn_kernel));
+            return POLESTAR_OK;
+        }
         const int wpb = 4;
         const size_t smem = (size_t)wpb * a.N * sizeof(float);
-        static size_t set = 0;
-        if (smem > 48 * 1024 && smem > set) {
-            CK(cudaFuncSetAttribute(attention_simt_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            set = smem;
-        }
+        if (smem > SIMT_ATTN_SMEM_MAX) return POLESTAR_E_INVAL;
         dim3 grid((a.n_rows + wpb - 1) / wpb, a.n_heads);
         CK(launch_k(attention_simt_kernel<T>, dim3(grid), dim3(wpb * 32), smem, c->st, a));
         CK(cudaGetLastError());
@@ -535,10 +599,6 @@ struct Path {
         int rc;
 
         const double esd = (double)es;
-        // 32 KB weight units per CTA that a GEMM asks L2 to fetch for its successors while its own tail runs.
-        // Off by default: measured on B200 it slows the decode by 5-12 % (the prefetch burst queues in front
-        // of the latency-critical partial-tile exchange of the GEMM's own tail).
-        const int pf_units = env_int("POLESTAR_PREFETCH_UNITS", 0), pf_units2 = env_int("POLESTAR_PREFETCH_UNITS2", 0);
         const double Mlive = sparse ? (double)bs * (B + std::min(sd.W, (int)(p.select_mode == POLESTAR_SELECT_TOPK_FRAC
                                                        ? floorf(p.select_frac * (float)sd.W + 0.5f)
                                                        : (p.select_mode == POLESTAR_SELECT_TOPK_COUNT ? p.select_k : sd.W))))
@@ -555,7 +615,7 @@ struct Path {
         // Steps whose rows all come straight from the previous projection (within-block steps without refresh): the two
         // RMSNorms of a layer are folded into the projections around them (EpiArgs::fold_*), no staging kernels.
         const bool fold = within && !sparse && is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && d % 256 == 0 && dq % 64 == 0 &&
-                          F % 64 == 0 && (dq + 2 * dkv) % 256 == 0 && (2 * F) % 256 == 0 && env_int("POLESTAR_FOLD_NORM", 0);
+                          F % 64 == 0 && (dq + 2 * dkv) % 256 == 0 && (2 * F) % 256 == 0 && c->sw.fold_norm;
         const size_t Mm = (size_t)c->M_max;
         if (fold) CK(cudaMemsetAsync(b.fold_ss, 0, (size_t)2 * L * Mm * sizeof(long long), st));
         bool qkv_staged = false, ffn_staged = false;
@@ -587,10 +647,7 @@ struct Path {
                 e.N_seq = N; e.n_heads = m.n_heads; e.n_kv = m.n_kv_heads; e.head_dim = m.head_dim; e.W_max = Wm;
                 e.within = within; e.ld_out = dq;
                 if (fold && l > 0) { e.in_ss = b.fold_ss + (size_t)(2 * l) * Mm; e.in_eps = m.rms_eps; e.in_d = d; }
-                NextW nx[2];
-                nx[0].w = c->wo[l]; nx[0].N_out = d; nx[0].K = dq; nx[0].M = M; nx[0].count = pf_units;
-                nx[1].w = c->wgu[l]; nx[1].N_out = 2 * F; nx[1].K = d; nx[1].M = M; nx[1].count = pf_units2;
-                if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->M_max, c->wqkv[l], M, dq + 2 * dkv, d, e, nx))) return rc;
+                if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->wqkv[l], M, dq + 2 * dkv, d, e))) return rc;
             }
             qkv_done = false;
             {
@@ -614,7 +671,7 @@ struct Path {
             // One sequence with a small window on the tensor-core path: the selection rides on the O projection
             // (idle warps of its first CTA), off the critical path; otherwise it is a kernel of its own.
             const bool sel_in_gemm = sparse && bs == 1 && sd.W <= SEL_SMALL_W && is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) &&
-                                     dq % 64 == 0 && d % 256 == 0 && env_int("POLESTAR_FUSE_SELECT", 1);
+                                     dq % 64 == 0 && d % 256 == 0 && c->sw.fuse_select;
             tc::SelFuse sf;
             memset(&sf, 0, sizeof(sf));
             if (sparse) {
@@ -637,7 +694,7 @@ struct Path {
             }
             // O projection -> RMSNorm -> gate/up -> down as one persistent kernel when the step is small enough
             bool chained = false;
-            if (is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && M <= tc::BLOCK_T && env_int("POLESTAR_CHAIN", 1)) {
+            if (is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && M <= tc::BLOCK_T && c->sw.chain) {
                 ChainSpec sp[4];
                 memset(sp, 0, sizeof(sp));
                 sp[0].A = b.o_buf; sp[0].W = c->wo[l]; sp[0].N_out = d; sp[0].K = dq; sp[0].epi = EPI_RESID; sp[0].norm_after = 1;
@@ -662,7 +719,7 @@ struct Path {
                 int n_chain = 3;
                 double by4 = 0, fl4 = 0;
                 // (off by default: measured 1 % slower than launching that projection on its own)
-                if (l + 1 < L && !fold && env_int("POLESTAR_CHAIN_QKV", 0)) {
+                if (l + 1 < L && !fold && c->sw.chain_qkv) {
                     n_chain = 4;
                     sp[2].norm_after = 2;
                     PostArgs& po = sp[2].post;
@@ -694,13 +751,11 @@ struct Path {
                 memset(&e, 0, sizeof(e));
                 e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
                 if (fold) { e.fold_a = b.a_buf; e.fold_gain = c->n2[l]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 1) * Mm; }
-                NextW nx[2];
-                nx[0].w = c->wgu[l]; nx[0].N_out = 2 * F; nx[0].K = d; nx[0].M = M; nx[0].first = pf_units2; nx[0].count = pf_units;
                 PostArgs po;
                 memset(&po, 0, sizeof(po));
                 po.kind = 1; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n2[l]; po.a_out = b.a_buf;
                 po.x = b.x1; po.list = list; po.m_count = m2_count;
-                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->M_max, c->wo[l], M, d, dq, e, nx, &po, &ffn_staged, sf.on ? &sf : nullptr))) return rc;
+                if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->wo[l], M, d, dq, e, &po, &ffn_staged, sf.on ? &sf : nullptr))) return rc;
             }
             if (fold) ffn_staged = true;
             if (!ffn_staged) {
@@ -713,9 +768,7 @@ struct Path {
                 memset(&e, 0, sizeof(e));
                 e.out_t = b.g_buf; e.ld_out = F; e.m_count = m2_count;
                 if (fold) { e.in_ss = b.fold_ss + (size_t)(2 * l + 1) * Mm; e.in_eps = m.rms_eps; e.in_d = d; }
-                NextW nx[2];
-                nx[0].w = c->wd[l]; nx[0].N_out = d; nx[0].K = F; nx[0].M = M; nx[0].count = pf_units;
-                if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->M_max, c->wgu[l], M, 2 * F, d, e, nx))) return rc;
+                if ((rc = gemm<EPI_SWIGLU>(c, b.a_buf, c->wgu[l], M, 2 * F, d, e))) return rc;
             }
             {
                 Scope sc(c, POLESTAR_PROF_GEMM_DOWN, ((double)F * d + Mlive * F) * esd + 2.0 * Mlive * d * 4, 2.0 * Mlive * F * (double)d, 1);
@@ -723,10 +776,6 @@ struct Path {
                 e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = b.x1; e.out_f32 = b.x; e.packet = b.packet;
                 e.W_max = Wm; e.within = within; e.ld_out = d;
                 if (fold && l + 1 < L) { e.fold_a = b.a_buf; e.fold_gain = c->n1[l + 1]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 2) * Mm; }
-                NextW nx[2];
-                if (l + 1 < L) { nx[0].w = c->wqkv[l + 1]; nx[0].N_out = dq + 2 * dkv; nx[0].K = d; nx[0].M = M; }
-                else { nx[0].w = c->lm_head; nx[0].N_out = m.vocab; nx[0].K = d; nx[0].M = bs * B; }
-                nx[0].count = pf_units;
                 PostArgs po;
                 memset(&po, 0, sizeof(po));
                 if (l + 1 < L) {
@@ -734,7 +783,7 @@ struct Path {
                     po.x = b.x; po.rows = b.rows; po.hc = b.hc + (size_t)(l + 1) * bs * Wm * d; po.packet = b.packet;
                     po.patch = b.patch + (size_t)(l + 1) * bs * Wm; po.kvflag = b.kvflag; po.sd = sd;
                 }
-                if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->M_max, c->wd[l], M, d, F, e, nx, &po, &qkv_staged))) return rc;
+                if ((rc = gemm<EPI_DOWN>(c, b.g_buf, c->wd[l], M, d, F, e, &po, &qkv_staged))) return rc;
             }
             }
         }
@@ -761,7 +810,7 @@ struct Path {
             EpiArgs e;
             memset(&e, 0, sizeof(e));
             e.out_f32 = b.logits; e.ld_out = m.vocab; e.scale = p.logit_scale; e.m_count = b.head_count;
-            if ((rc = gemm<EPI_LOGITS>(c, b.a_head, c->rows_lm, c->lm_head, Mh, m.vocab, d, e))) return rc;
+            if ((rc = gemm<EPI_LOGITS>(c, b.a_head, c->lm_head, Mh, m.vocab, d, e))) return rc;
         }
         {
             Scope sc(c, POLESTAR_PROF_CONFIDENCE, (double)bs * B * m.vocab * 4, 0, 3);
@@ -813,6 +862,7 @@ static StepDesc make_step_desc(polestar_ctx* c, bool* any_refresh) {
 
 extern "C" int polestar_step(polestar_ctx* c, polestar_step_info* info) {
     if (!c) return POLESTAR_E_INVAL;
+    if (c->failed) return POLESTAR_E_STATE;
     if (c->done) return POLESTAR_E_DONE;
     if (c->pending) return POLESTAR_E_STATE;
     bool any_refresh = false;
@@ -841,7 +891,7 @@ extern "C" int polestar_step(polestar_ctx* c, polestar_step_info* info) {
 
 extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     if (!c) return POLESTAR_E_INVAL;
-    if (!c->pending) return POLESTAR_E_STATE;
+    if (c->failed || !c->pending) return POLESTAR_E_STATE;
     const polestar_params& p = c->p;
     const StepDesc& sd = c->last_sd;
     Buffers& b = c->b;
@@ -849,7 +899,8 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     memset(&a, 0, sizeof(a));
     a.y = b.y; a.conf = b.conf; a.yhat = b.yhat;
     a.kl = b.kl; a.delta_out = b.delta; a.Delta_out = b.Delta; a.taud_out = b.taud;
-    a.theta = b.theta; a.theta_cnt = b.theta_cnt; a.commit_flags = b.commit_flags; a.suffix_flags = b.suffix_flags;
+    a.theta = b.theta; a.theta_cnt = b.theta_cnt; a.commit_flags = b.commit_flags; a.own_flags = b.own_flags;
+    a.suffix_flags = b.suffix_flags;
     a.head_count = b.head_count; a.suf_seq = b.suf_seq; a.suf_w = b.suf_w;
     a.forced_pos = c->forced_commit ? b.forced_commit : nullptr;
     a.forced_n = c->forced_commit_n;
@@ -916,7 +967,12 @@ extern "C" int polestar_commit(polestar_ctx* c, polestar_commit_info* info) {
     ci.forwards = c->forwards; ci.generated = c->generated; ci.generated_non_eos = c->generated_non_eos;
     ci.launches = c->launches;
     if (info) *info = ci;
-    if (status) return POLESTAR_E_TIMEOUT;
+    if (status) {
+        // a bounded device-side wait gave up: tile and grid counters no longer match the host's bookkeeping and
+        // outputs may be partial, so the context refuses further work
+        c->failed = true;
+        return POLESTAR_E_TIMEOUT;
+    }
     if (nonfinite) return POLESTAR_E_NONFINITE;
     return POLESTAR_OK;
 }
@@ -935,13 +991,23 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
         for (int i = 0; i < p->batch * p->prompt_len; ++i)
             if (prompt[i] < 0 || prompt[i] >= m->vocab || prompt[i] == m->mask_id) return POLESTAR_E_INVAL;
     const size_t need = make_plan(m, p, nullptr, nullptr);
-    if (ws_bytes < need) return POLESTAR_E_NOSPACE;
-    int rc = init_device_info();
+    char* ws_aligned = (char*)(((uintptr_t)ws + 1023) & ~(uintptr_t)1023);
+    if ((size_t)(ws_aligned - (char*)ws) + need > ws_bytes) return POLESTAR_E_NOSPACE;
+    DevInfo di;
+    int rc = device_info(&di);
     if (rc) return rc;
-    g_use_pdl = env_int("POLESTAR_PDL", 1) != 0;
     polestar_ctx* c = new (std::nothrow) polestar_ctx();
     if (!c) return POLESTAR_E_INVAL;
     c->m = *m; c->p = *p;
+    c->sw = read_switches();
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_sw = c->sw; g_sw_loaded = true;
+        g_use_pdl = c->sw.pdl != 0;
+    }
+    c->sms = di.sm_count;
+    c->maps.l2promo = c->sw.l2promo;
+    cudaGetDevice(&c->device);
     for (int l = 0; l < m->n_layers; ++l) {
         if (!w->wqkv[l] || !w->wo[l] || !w->w_gate_up[l] || !w->w_down[l] || !w->norm1[l] || !w->norm2[l]) {
             delete c;
@@ -952,8 +1018,7 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     }
     c->embed = w->embed; c->lm_head = w->lm_head; c->final_norm = w->final_norm;
     c->st = (cudaStream_t)stream;
-    c->ws = (char*)(((uintptr_t)ws + 1023) & ~(uintptr_t)1023);
-    if ((size_t)(c->ws - (char*)ws) + need > ws_bytes + 1024) { delete c; return POLESTAR_E_NOSPACE; }
+    c->ws = ws_aligned;
     make_plan(m, p, &c->b, c->ws);
     c->es = m->dtype == POLESTAR_BF16 ? 2 : 4;
     c->N = p->prompt_len + p->gen_len; c->B = p->block; c->W_max = window_max(p);
@@ -966,6 +1031,7 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     c->gws.counters = c->b.gemm_counters; c->gws.n_counters = GEMM_COUNTERS - 512; c->gws.status = c->b.status;
     c->gws.post_counter = reinterpret_cast<unsigned*>(c->b.gemm_counters + GEMM_COUNTERS - 1); c->gws.post_total = 0;
     c->gws.chain_counter = reinterpret_cast<unsigned*>(c->b.gemm_counters + GEMM_COUNTERS - 512); c->gws.chain_total = 0;
+    c->gws.sms = c->sms; c->gws.sw = c->sw;
 
     auto fail = [&](int code) { delete c; return code; };
     // zero the persistent state (everything in front of the scratch rows)
@@ -987,11 +1053,14 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     const int half = m->head_dim / 2;
     rope_table_kernel<<<(c->N * half + 255) / 256, 256, 0, c->st>>>(c->b.rope, c->N, half, (double)m->rope_theta);
     if (cudaStreamSynchronize(c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
-    if (env_int("POLESTAR_KERNEL_TRACE", 0)) {
+#ifdef POLESTAR_TRACE
+    if (c->sw.kernel_trace) {
         long long* tb = (long long*)((char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384 - 65536);
         cudaMemsetAsync(tb, 0, 65536, c->st);
         cudaMemcpyToSymbolAsync(g_trace_buf, &tb, sizeof(tb), 0, cudaMemcpyHostToDevice, c->st);
+        c->trace_installed = true;
     }
+#endif
     rc = polestar_step(c, nullptr);
     if (rc) return fail(rc);
     *out = c;
@@ -1001,6 +1070,12 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
 extern "C" void polestar_destroy(polestar_ctx* c) {
     if (!c) return;
     cudaStreamSynchronize(c->st);
+#ifdef POLESTAR_TRACE
+    if (c->trace_installed) {        // the stamps must not outlive the workspace they are written to
+        long long* none = nullptr;
+        cudaMemcpyToSymbol(g_trace_buf, &none, sizeof(none));
+    }
+#endif
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     if (c->seq_info_host) cudaFreeHost(c->seq_info_host);
     delete c;
@@ -1048,8 +1123,15 @@ extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void*
         case POLESTAR_READ_COMMIT: src = c->b.commit_flags; sz = bs * B * 4; break;
         case POLESTAR_READ_PPREV: src = c->b.pprev + layer * bs * Wm * m.n_heads * N; sz = bs * Wm * m.n_heads * N * 4; break;
         case POLESTAR_READ_SUFFIX: src = c->b.suffix_flags; sz = bs * Wm * 4; break;
-        case 98: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384 - 65536; sz = 65536; break;   // debug: kernel timeline
-        case 99: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384; sz = 16384; break;   // debug: GEMM time stamps
+        case POLESTAR_READ_DRIFT_DELTA: src = c->b.Delta; sz = bs * B * 4; break;
+        case POLESTAR_READ_TAU_D: src = c->b.taud; sz = bs * B * 4; break;
+        case POLESTAR_READ_THETA: src = c->b.theta; sz = bs * std::max<size_t>(1, c->p.hist) * B * 4; break;
+        case POLESTAR_READ_THETA_COUNT: src = c->b.theta_cnt; sz = bs * 4; break;
+        case POLESTAR_READ_OWN_COMMIT: src = c->b.own_flags; sz = bs * B * 4; break;
+#ifdef POLESTAR_TRACE
+        case POLESTAR_READ_TRACE_KERNELS: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384 - 65536; sz = 65536; break;
+        case POLESTAR_READ_TRACE_GEMM: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384; sz = 16384; break;
+#endif
         default: return POLESTAR_E_INVAL;
     }
     CK(cudaMemcpyAsync(dst, src, std::min(sz, bytes), cudaMemcpyDeviceToHost, c->st));
@@ -1122,18 +1204,20 @@ extern "C" int polestar_k_attention(const void* q, const void* k, const void* v,
     a.n_rows = R; a.q = q; a.kc = k; a.vc = v; a.out = out; a.pprev = logp_prev; a.kl = kl; a.N = N;
     a.n_heads = n_heads; a.n_kv = n_kv; a.head_dim = head_dim; a.record_kl = 1; a.rows_per_seq = R; a.batch = 1;
     a.scale = 1.0f / sqrtf((float)head_dim);
-    if (dtype == POLESTAR_BF16 && head_dim == 128 && !env_int("POLESTAR_ATTN_SIMT", 0)) return launch_attention_mma(a, st);
+    DevInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    const Switches sw = stand_alone_switches();
+    if (dtype == POLESTAR_BF16 && head_dim == 128 && !sw.attn_simt) {
+        CK(launch_attention_mma(a, st, di.sm_count, sw.attn_kernel));
+        return POLESTAR_OK;
+    }
     const int wpb = 4;
     const size_t smem = (size_t)wpb * N * sizeof(float);
-    if (smem > 200 * 1024) return POLESTAR_E_INVAL;
+    if (smem > SIMT_ATTN_SMEM_MAX) return POLESTAR_E_INVAL;
     dim3 grid((R + wpb - 1) / wpb, n_heads);
-    if (dtype == POLESTAR_BF16) {
-        CK(cudaFuncSetAttribute(attention_simt_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        attention_simt_kernel<__nv_bfloat16><<<grid, wpb * 32, smem, st>>>(a);
-    } else {
-        CK(cudaFuncSetAttribute(attention_simt_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        attention_simt_kernel<float><<<grid, wpb * 32, smem, st>>>(a);
-    }
+    if (dtype == POLESTAR_BF16) attention_simt_kernel<__nv_bfloat16><<<grid, wpb * 32, smem, st>>>(a);
+    else attention_simt_kernel<float><<<grid, wpb * 32, smem, st>>>(a);
     CK(cudaGetLastError());
     return POLESTAR_OK;
 }
@@ -1146,11 +1230,11 @@ extern "C" int polestar_k_hidden_delta(const void* a, const void* b, float* out,
     if (!a || !b || !out) return POLESTAR_E_INVAL;
     const int per = dtype == POLESTAR_BF16 ? 8 : 4;
     if (d % per || (((uintptr_t)a | (uintptr_t)b) & 15)) return POLESTAR_E_INVAL;
-    if (rows == 0) return POLESTAR_OK;
-    int rc = init_device_info();
+    DevInfo di;
+    int rc = device_info(&di);
     if (rc) return rc;
     const int wpb = 8;
-    const int grid = std::min((rows + wpb - 1) / wpb, g_sm_count * 8);
+    const int grid = std::min((rows + wpb - 1) / wpb, di.sm_count * 8);
     if (dtype == POLESTAR_BF16)
         hidden_delta_kernel<__nv_bfloat16><<<grid, wpb * 32, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, out, rows, d);
     else
@@ -1207,14 +1291,17 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     size_t off_rope, off_part, off_cnt, off_status;
     const size_t need = refresh_layout(batch, max_rows, d, head_dim, 65536, &off_rope, &off_part, &off_cnt, &off_status);
     if (scratch_bytes < need) return POLESTAR_E_NOSPACE;
-    int rc = init_device_info();
+    DevInfo di;
+    int rc = device_info(&di);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     char* sc = (char*)scratch;
     __nv_bfloat16* a_buf = (__nv_bfloat16*)sc;
     float2* rope = (float2*)(sc + off_rope);
-    static MapCache maps;
+    MapCache maps;                     // the two tensor maps of this call (built per call: no shared state)
     GemmWs ws;
+    ws.sms = di.sm_count; ws.sw = stand_alone_switches();
+    maps.l2promo = ws.sw.l2promo;
     ws.partial = (float*)(sc + off_part); ws.partial_bytes = GEMM_PARTIAL_BYTES;
     const int M = batch * max_rows;
     const int dq = n_heads * head_dim, dkv = n_kv * head_dim;
@@ -1224,6 +1311,7 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     const int n_cnt = (int)std::min<long long>(GEMM_COUNTERS, 2 * (tiles + 1));
     ws.counters = (int*)(sc + off_cnt); ws.n_counters = n_cnt; ws.status = (int*)(sc + off_status);
     CK(cudaMemsetAsync(ws.counters, 0, (size_t)n_cnt * sizeof(int), st));
+    CK(cudaMemsetAsync(ws.status, 0, sizeof(int), st));       // read back by polestar_k_refresh_status
     const int half = head_dim / 2;
     // launched back to back with programmatic stream serialization: each kernel starts while its predecessor drains
     // rotary entries: of the selected positions only when these are fewer than the whole table
@@ -1236,9 +1324,27 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     memset(&e, 0, sizeof(e));
     e.rope = rope; e.q_out = q_out; e.kc = kc; e.vc = vc; e.n_heads = n_heads; e.n_kv = n_kv; e.head_dim = head_dim;
     e.idx = idx; e.counts = counts; e.max_rows = max_rows; e.P = P;
-    if (d % 64 == 0 && (dq + 2 * dkv) % 256 == 0 && !env_int("POLESTAR_REFRESH_SIMT", 0))
-        return launch_gemm_tc<EPI_QKV_REFRESH>(maps, ws, a_buf, M, wqkv, M, dq + 2 * dkv, d, e, st);
+    if (d % 64 == 0 && (dq + 2 * dkv) % 256 == 0 && !ws.sw.refresh_simt)
+        return launch_gemm_tc<EPI_QKV_REFRESH>(maps, ws, a_buf, wqkv, M, dq + 2 * dkv, d, e, st);
     return launch_gemm_simt<__nv_bfloat16, EPI_QKV_REFRESH>(a_buf, wqkv, M, dq + 2 * dkv, d, e, st);
+}
+
+extern "C" int polestar_k_refresh_status(const void* scratch, size_t scratch_bytes, int32_t batch, int32_t max_rows,
+                                         int32_t d, int32_t head_dim, void* stream) {
+    if (!scratch || batch <= 0 || max_rows <= 0 || d <= 0 || head_dim <= 0) return POLESTAR_E_INVAL;
+    size_t off_rope, off_part, off_cnt, off_status;
+    const size_t need = refresh_layout(batch, max_rows, d, head_dim, 65536, &off_rope, &off_part, &off_cnt, &off_status);
+    if (scratch_bytes < need) return POLESTAR_E_NOSPACE;
+    int status = 0;
+    CK(cudaMemcpyAsync(&status, (const char*)scratch + off_status, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    return status ? POLESTAR_E_TIMEOUT : POLESTAR_OK;
+}
+
+// The confidence kernel reads rows with 16-byte loads when the vocabulary is a multiple of four: the base must
+// then be 16-byte aligned (rows follow at multiples of 16 bytes); otherwise 4-byte alignment is enough.
+static bool conf_logits_aligned(const float* logits, int vocab) {
+    return (((uintptr_t)logits) & ((vocab & 3) == 0 ? 15 : 3)) == 0;
 }
 
 extern "C" int polestar_k_confidence(const float* logits, int32_t rows, int32_t vocab, int32_t mask_id, int32_t* yhat,
@@ -1246,8 +1352,8 @@ extern "C" int polestar_k_confidence(const float* logits, int32_t rows, int32_t 
     if (rows < 0 || vocab <= 0) return POLESTAR_E_INVAL;
     if (rows == 0) return POLESTAR_OK;           // no rows: nothing to do (the pointers may be null)
     if (!logits || !yhat || !conf || !scratch) return POLESTAR_E_INVAL;
+    if (!conf_logits_aligned(logits, vocab)) return POLESTAR_E_INVAL;
     if (scratch_bytes < (size_t)rows * CONF_CHUNKS * sizeof(ConfPart)) return POLESTAR_E_NOSPACE;
-    if (rows == 0) return POLESTAR_OK;
     cudaStream_t st = (cudaStream_t)stream;
     conf_partial_kernel<<<dim3(CONF_CHUNKS, rows), 256, 0, st>>>(logits, nullptr, rows, vocab, mask_id, CONF_CHUNKS, (ConfPart*)scratch);
     conf_final_kernel<<<(rows + 127) / 128, 128, 0, st>>>((const ConfPart*)scratch, nullptr, rows, CONF_CHUNKS, yhat, conf);
@@ -1285,9 +1391,11 @@ static ConfPart* conf_scratch_ptr(int* err) {
 
 extern "C" int polestar_k_confidence_noalloc(const float* logits, int32_t rows, int32_t vocab, int32_t mask_id,
                                              int32_t* yhat, float* conf, void* stream) {
-    if (!logits || !yhat || !conf || rows < 0 || vocab <= 0) return POLESTAR_E_INVAL;
+    if (rows < 0 || vocab <= 0) return POLESTAR_E_INVAL;
+    if (rows == 0) return POLESTAR_OK;           // no rows: nothing to do (the pointers may be null)
+    if (!logits || !yhat || !conf) return POLESTAR_E_INVAL;
+    if (!conf_logits_aligned(logits, vocab)) return POLESTAR_E_INVAL;
     if (rows > POLESTAR_NOALLOC_MAX_ROWS) return POLESTAR_E_NOSPACE;    // beyond the built-in scratch: use polestar_k_confidence
-    if (rows == 0) return POLESTAR_OK;
     int err = POLESTAR_OK;
     ConfPart* scratch = conf_scratch_ptr(&err);
     if (!scratch) return err;

@@ -228,8 +228,8 @@ def uniform_ids(key: int, count: int, modulus: int, device="cpu") -> torch.Tenso
 # --------------------------------------------------------------------------
 
 # tensor ids inside a layer (layer = -1 for the global tensors)
-T_WQ, T_WK, T_WV, T_WO, T_WG, T_WU, T_WD = range(7)
-T_EMBED, T_LM_HEAD = 16, 17
+T_WQ, T_WK, T_WV, T_WO, T_WG, T_WU, T_WD, T_NORM1, T_NORM2 = range(9)
+T_EMBED, T_LM_HEAD, T_FINAL_NORM = 16, 17, 18
 T_PROMPT = 32
 T_HCACHE, T_DRIFT = 48, 49
 
@@ -239,12 +239,16 @@ def torch_dtype(m: ModelCfg):
 
 
 def make_weights(m: ModelCfg, seed: int = 0, device="cpu", std: float = 0.02,
-                 layers: Optional[List[int]] = None, with_globals: bool = True) -> Dict:
+                 layers: Optional[List[int]] = None, with_globals: bool = True,
+                 gain_std: float = 0.1) -> Dict:
     """Logical weights, every matrix stored [out_features, in_features].
 
     Values are rounded to the model's storage dtype (bf16 models hold
-    bf16-representable numbers).  RMSNorm gains are one.  ``layers`` limits
-    generation to a subset of layers (same values as in the full model).
+    bf16-representable numbers).  RMSNorm gains are 1 + gain_std * normal, one
+    stream per norm (two per layer and the final one), so that a swapped or
+    dropped gain changes the result; ``gain_std = 0`` gives unit gains.
+    ``layers`` limits generation to a subset of layers (same values as in the
+    full model).
     """
     dt = torch_dtype(m)
     d, dq, dkv, F, V = m.d_model, m.d_q, m.d_kv, m.d_ffn, m.vocab
@@ -252,17 +256,20 @@ def make_weights(m: ModelCfg, seed: int = 0, device="cpu", std: float = 0.02,
     def mk(layer, tid, shape):
         return normal_tensor(tensor_key(seed, layer, tid), shape, std, dt, device)
 
+    def gain(layer, tid):
+        g = normal_tensor(tensor_key(seed, layer, tid), (d,), gain_std, torch.float32, device)
+        return (1.0 + g).to(dt)
+
     w = {"layers": []}
     if with_globals:
         w.update({"embed": mk(-1, T_EMBED, (V, d)), "lm_head": mk(-1, T_LM_HEAD, (V, d)),
-                  "final_norm": torch.ones(d, dtype=dt, device=device)})
+                  "final_norm": gain(-1, T_FINAL_NORM)})
     for l in (range(m.n_layers) if layers is None else layers):
         w["layers"].append({
             "wq": mk(l, T_WQ, (dq, d)), "wk": mk(l, T_WK, (dkv, d)), "wv": mk(l, T_WV, (dkv, d)),
             "wo": mk(l, T_WO, (d, dq)), "wg": mk(l, T_WG, (F, d)), "wu": mk(l, T_WU, (F, d)),
             "wd": mk(l, T_WD, (d, F)),
-            "norm1": torch.ones(d, dtype=dt, device=device),
-            "norm2": torch.ones(d, dtype=dt, device=device),
+            "norm1": gain(l, T_NORM1), "norm2": gain(l, T_NORM2),
         })
     return w
 

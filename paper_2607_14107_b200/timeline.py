@@ -1,6 +1,7 @@
 """Kernel timeline of real forwards (debugging / profiling aid).
 
-With POLESTAR_KERNEL_TRACE=1 the library records, for every kernel of a forward, the time at which
+A library built with -DPOLESTAR_TRACE (`python -m paper_2607_14107_b200.build --trace`, built here on
+demand) and run with POLESTAR_KERNEL_TRACE=1 records, for every kernel of a forward, the time at which
 block 0 had its dependencies resolved (and, for the GEMM, when its CTA 0 finished).  Consecutive
 stamps give what each kernel really costs inside the pipeline, launch gaps included -- something
 neither CUDA events (too coarse) nor ncu (serialised, idle clocks) show.
@@ -31,6 +32,8 @@ def main():
     ap.add_argument("--entry", action="store_true", help="also print forward 0, the block-entry forward of the first block")
     a = ap.parse_args()
     os.environ["POLESTAR_KERNEL_TRACE"] = "1"
+    from . import build as Bu
+    os.environ["POLESTAR_LIB"] = Bu.build(trace=True)
     import torch
     from . import binding as Bd, inputs as I
     m, p = I.config(a.config)
@@ -44,7 +47,7 @@ def main():
         dec.commit()
     torch.cuda.synchronize()
     out = np.zeros(8192, np.int64)
-    Bd._check(Bd.load().polestar_read(dec.ctx, 98, 0, out.ctypes.data_as(C.c_void_p), 65536))
+    Bd._check(Bd.load().polestar_read(dec.ctx, Bd.READ_TRACE_KERNELS, 0, out.ctypes.data_as(C.c_void_p), 65536))
     n = min(int(out[0]), 4000)
     ids, ts = out[1:1 + 2 * n:2], out[2:2 + 2 * n:2].astype(np.float64) / 1000.0
     order = np.argsort(ts, kind="stable")

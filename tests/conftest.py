@@ -24,3 +24,15 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _fresh_env_switches(request):
+    """The library reads its POLESTAR_* switches once (at polestar_init / polestar_reload_env): after a GPU test
+    that changed the environment, make the stand-alone kernel calls of later tests see the restored values.
+    (Set up before `monkeypatch`, hence torn down after it has restored the environment.)"""
+    yield
+    if "gpu" in request.keywords:
+        from paper_2607_14107_b200 import binding as Bd
+        if Bd._lib is not None:
+            Bd.polestar_reload_env()

@@ -9,6 +9,7 @@ The oracle cannot run 32 layers of this width in reasonable time, so
     full-recompute decode (Sec. 4.1 / Sec. 3.1), plus the invariants of drift, selection and commit.
 """
 import dataclasses
+import re
 
 import numpy as np
 import pytest
@@ -18,11 +19,24 @@ from oracle import polestar_oracle as O
 from paper_2607_14107_b200 import binding as Bd
 from paper_2607_14107_b200 import inputs as I
 
+from parity import check_commit_quantities, new_stats, outside_fraction
+
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
+# Largest share of elements of any compared tensor that may fall outside the plain abs/rel 2e-2 rule (they are
+# inside the RMS-scaled rule of close()); the measured shares are printed at the end of the module (-s).
+OUTSIDE_MAX = 5e-2
+OUTSIDE = {}
 
 
-def close(a, b, tol, what="", scale=1.0, depth=1):
+@pytest.fixture(scope="module", autouse=True)
+def _report_outside_fraction():
+    yield
+    worst = sorted(OUTSIDE.items(), key=lambda kv: -kv[1])[:8]
+    print("\nshare of elements outside the plain abs/rel 2e-2 rule (worst tensors):", worst)
+
+
+def close(a, b, tol, what="", scale=1.0, depth=1, bound=OUTSIDE_MAX):
     """|a - b| <= tol * sqrt(depth) * (s + |b|), s = max(1, rms(b)).
 
     At these widths hidden states have an RMS of ~2 (14 after 32 layers) and dot products run over
@@ -35,10 +49,16 @@ def close(a, b, tol, what="", scale=1.0, depth=1):
     assert np.isfinite(a).all(), what
     s = max(1.0, float(np.sqrt(np.mean(b * b)))) if b.size else 1.0
     err = np.abs(a - b) - tol * np.abs(b)
-    assert err.max() <= tol * s, f"{what}: max abs err {np.abs(a - b).max():.3e} (tol {tol}, scale {s:.2f})"
+    assert err.max(initial=0.0) <= tol * s, f"{what}: max abs err {np.abs(a - b).max():.3e} (tol {tol}, scale {s:.2f})"
+    # what the scaled tolerance hides: the share of elements outside the plain rule |a - b| <= 2e-2 (1 + |b|)
+    frac = outside_fraction(a, b, TOL)
+    key = re.sub(r"(step|seq) \d+ ?", "", what)
+    OUTSIDE[key] = max(frac, OUTSIDE.get(key, 0.0))
+    if bound is not None:       # (None: the 32-layer self-consistency check, where the share is only reported)
+        assert frac <= bound, f"{what}: {frac:.2e} of the elements outside the plain abs/rel {TOL} rule"
 
 
-def forced_commit(gpu, ora, infos, p):
+def forced_commit(gpu, ora, infos, p, m=None, y_before=None, stats=None):
     forced = np.full((p.batch, p.block + gpu.W_max), -1, np.int32)
     ftok = np.zeros_like(forced)
     for s, i in enumerate(infos):
@@ -46,7 +66,10 @@ def forced_commit(gpu, ora, infos, p):
         forced[s, :len(pos)] = pos
         ftok[s, :len(pos)] = ora.tokens()[s, pos]
     gpu.force_commit(forced, ftok)
-    return gpu.commit()
+    ci = gpu.commit()
+    if stats is not None:
+        check_commit_quantities(gpu, ora, infos, y_before, p, m, TOL, stats)
+    return ci
 
 
 def compare_step(gpu, ora, m, p, step):
@@ -82,8 +105,11 @@ def run_reduced_depth(m, p, n_within):
     ora = O.PolestarOracle(m, wn, p, prompt)
     ora.step()
     compare_step(gpu, ora, m, p, 0)
+    kinds = [ora.seqs[0].trace["kind"]]
+    stats = new_stats()
     for step in range(1, n_within + 1):
-        forced_commit(gpu, ora, ora.commit(), p)
+        y_before = ora.tokens().copy()
+        forced_commit(gpu, ora, ora.commit(), p, m, y_before, stats)
         assert np.array_equal(gpu.tokens(), ora.tokens())
         ora.step()
         tr = ora.seqs[0].trace
@@ -96,7 +122,9 @@ def run_reduced_depth(m, p, n_within):
                 gpu.force_select(l, sel)
         gpu.step()
         compare_step(gpu, ora, m, p, step)
+        kinds.append(tr["kind"] + ("_refresh" if tr["kind"] == "within" and tr["refresh"] else ""))
     gpu.destroy()
+    return kinds
 
 
 def test_c2_shape_reduced_depth_matches_oracle():
@@ -107,12 +135,26 @@ def test_c2_shape_reduced_depth_matches_oracle():
 
 
 def test_c3_widths_gqa_batch_matches_oracle():
-    # Dream-7B widths (28 query heads on 4 kv heads, d 3584, FFN 18944, vocab 152064), batch 2, short sequences
+    # Dream-7B widths (28 query heads on 4 kv heads, d 3584, FFN 18944, vocab 152064), batch 4 as in the
+    # workload, short sequences
     m, _ = I.config("c3")
     m = I.reduced_depth(m, 1)
-    p = I.Params(batch=2, prompt_len=64, gen_len=64, block=32, max_steps=64, tau_upd=-1,
+    p = I.Params(batch=4, prompt_len=64, gen_len=64, block=32, max_steps=64, tau_upd=-1,
                  flags=I.FLAG_DEFAULT | I.FLAG_KEEP_HIDDEN)
     run_reduced_depth(m, p, n_within=2)
+
+
+def test_c4_shape_reduced_depth_matches_oracle():
+    # The long-generation workload's shape at depth 1: LLaDA-8B widths and vocabulary, 1024 + 1024 positions,
+    # block 64 (window 192), batch 2.  With 3 steps per block and tau_upd = 25 the first forwards are: a
+    # full-sequence entry (2048 rows per sequence: multi-token-tile GEMMs, the 64-row attention kernel with
+    # recorded rows), a plain step, a refresh step (192 window rows per sequence through drift, select and the
+    # sparse forward) and the window entry of the next block.
+    m, p = I.config("c4")
+    m = I.reduced_depth(m, 1)
+    p = dataclasses.replace(p, batch=2, max_steps=48, tau_upd=25, flags=p.flags | I.FLAG_KEEP_HIDDEN)
+    kinds = run_reduced_depth(m, p, n_within=3)
+    assert kinds == ["entry_full", "within", "within_refresh", "entry_window"], kinds
 
 
 @pytest.fixture(scope="module")
@@ -134,8 +176,9 @@ def test_c2_full_depth_full_refresh_equals_nocache(c2_full):
             a.step(); b.step()
         ha, hb = a.read(Bd.READ_HIDDEN, m.n_layers), b.read(Bd.READ_HIDDEN, m.n_layers)
         close(a.read(Bd.READ_HIDDEN, 1), b.read(Bd.READ_HIDDEN, 1), TOL, f"step {step} hidden after layer 0")
-        close(ha, hb, TOL, f"step {step} final hidden", depth=m.n_layers)
-        close(a.read(Bd.READ_LOGITS), b.read(Bd.READ_LOGITS), TOL, f"step {step} logits", depth=m.n_layers)
+        close(ha, hb, TOL, f"step {step} final hidden (32 layers, self-consistency)", depth=m.n_layers, bound=None)
+        close(a.read(Bd.READ_LOGITS), b.read(Bd.READ_LOGITS), TOL, f"step {step} logits (32 layers, self-consistency)",
+              depth=m.n_layers, bound=None)
         if step:
             close(a.read(Bd.READ_DELTA), b.read(Bd.READ_DELTA), TOL, f"step {step} delta", depth=m.n_layers)
         # keep the two decoders on one trajectory: b commits what a commits

@@ -46,6 +46,7 @@ def test_attention_drift_matches_oracle(dtype, R, N, nh, nkv, dh):
 ])
 def test_attention_kernel_variants(monkeypatch, variant, R, N, nh, nkv):
     monkeypatch.setenv("POLESTAR_ATTN_KERNEL", str(variant))
+    Bd.polestar_reload_env()           # the stand-alone calls read the switches once, not per launch
     check_attention(torch.bfloat16, R, N, nh, nkv, 128)
 
 
@@ -102,6 +103,7 @@ def test_attention_many_rows_single_pass(monkeypatch, variant, R, N, nh, nkv):
     # without stored rows the 64-row-tile kernel makes one pass with a running maximum (probabilities are rounded
     # to bf16 before the final normalisation): same tolerance against the oracle
     monkeypatch.setenv("POLESTAR_ATTN_KERNEL", str(variant))
+    Bd.polestar_reload_env()           # the stand-alone calls read the switches once, not per launch
     dh = 128
     q = rnd((R, nh * dh), 1, 1.0, torch.bfloat16).cuda()
     k = rnd((N, nkv * dh), 2, 1.0, torch.bfloat16).cuda()
@@ -165,15 +167,20 @@ def test_select_zero_drift_and_nan():
     (256, 256, 2, 2, 37, 1), (512, 512, 4, 1, 128, 2), (300, 256, 2, 2, 300, 1),
     (3400, 256, 2, 2, 3300, 4),       # 13200 rows: 312 output tiles > SM count (whole tiles round-robin + stream-K tail)
     (2000, 256, 2, 2, 1700, 2),       # 3400 rows: 27 token tiles (two raster chunks), fewer tiles than SMs
+    # the refresh micro-benchmark's own shape (LLaDA-8B layer: d 4096 = 64 k-blocks, 32 x 128 heads, 4096 positions)
+    (4096, 4096, 32, 32, 41, 1), (4096, 4096, 32, 32, 1024, 1), (4096, 4096, 32, 32, 410, 8),
 ])
 def test_refresh_chain_matches_oracle(P, d, nh, nkv, k, batch):
     dh = 128
-    h, drift = I.make_refresh_inputs(batch, P, d)
-    m = I.ModelCfg(1, d, nh, nkv, dh, 2 * d, 1024, I.DTYPE_BF16, 1e-5, 500000.0)
-    w = I.make_weights(m, seed=5)
+    big = d >= 2048
+    dev = "cuda" if big else "cpu"                      # large inputs are generated on the device (same values)
+    h, drift = I.make_refresh_inputs(batch, P, d, device=dev)
+    drift = drift.cpu()
+    m = I.ModelCfg(1, d, nh, nkv, dh, 256 if big else 2 * d, 1024, I.DTYPE_BF16, 1e-5, 500000.0)
+    w = I.make_weights(m, seed=5, device=dev)
     packed = Bd.pack_weights(m, w)
-    kc0 = rnd((batch, P, nkv * dh), 8, 1.0, torch.bfloat16)
-    vc0 = rnd((batch, P, nkv * dh), 9, 1.0, torch.bfloat16)
+    kc0 = I.normal_tensor(I.tensor_key(77, -1, 8), (batch, P, nkv * dh), 1.0, torch.bfloat16, dev)
+    vc0 = I.normal_tensor(I.tensor_key(77, -1, 9), (batch, P, nkv * dh), 1.0, torch.bfloat16, dev)
     kc, vc = kc0.clone().cuda(), vc0.clone().cuda()
     idx = torch.zeros((batch, k), dtype=torch.int32, device="cuda")
     cnt = torch.zeros(batch, dtype=torch.int32, device="cuda")
@@ -185,23 +192,25 @@ def test_refresh_chain_matches_oracle(P, d, nh, nkv, k, batch):
     off = (-scratch.data_ptr()) % 1024
     Bd.polestar_k_refresh(h.cuda(), idx, cnt, packed["wqkv"][0], packed["norm1"][0], kc, vc, q_out, k, nh, nkv, dh,
                           m.rms_eps, m.rope_theta, scratch[off:])
-    torch.cuda.synchronize()
-    wl = I.weights_to_numpy(w)["layers"][0]
+    assert Bd.polestar_k_refresh_status(scratch[off:], batch, k, d, dh) == Bd.OK      # synchronises
+    assert cnt.cpu().tolist() == [k] * batch
+    wl = {n: t.detach().to("cpu", torch.float32).numpy() for n, t in w["layers"][0].items() if n in ("wq", "wk", "wv", "norm1")}
     inv = np.argsort(Bd.rope_interleave_index(dh).numpy())
+    kc_h, vc_h, kc0_h, vc0_h = kc.cpu(), vc.cpu(), kc0.cpu(), vc0.cpu()
     for s in range(batch):
         ridx, q_ref, K_ref, V_ref = O.refresh_chain(bf16_np(h[s]), drift[s].numpy(), k, wl["wq"], wl["wk"], wl["wv"],
-                                                    np.ones(d), m.rms_eps, m.rope_theta, nh, nkv, dh,
-                                                    bf16_np(kc0[s]).reshape(P, nkv, dh), bf16_np(vc0[s]).reshape(P, nkv, dh))
+                                                    wl["norm1"], m.rms_eps, m.rope_theta, nh, nkv, dh,
+                                                    bf16_np(kc0_h[s]).reshape(P, nkv, dh), bf16_np(vc0_h[s]).reshape(P, nkv, dh))
         assert idx[s, :int(cnt[s])].cpu().tolist() == ridx.tolist()
-        Kg = bf16_np(kc[s]).reshape(P, nkv, dh)
-        Vg = bf16_np(vc[s]).reshape(P, nkv, dh)
+        Kg = bf16_np(kc_h[s]).reshape(P, nkv, dh)
+        Vg = bf16_np(vc_h[s]).reshape(P, nkv, dh)
         Kg_log = Kg[..., inv]
         assert np.allclose(Kg_log[ridx], K_ref[ridx], atol=2e-2, rtol=2e-2)
         assert np.allclose(Vg[ridx], V_ref[ridx], atol=2e-2, rtol=2e-2)
         qg = bf16_np(q_out[s]).reshape(k, nh, dh)[..., inv]
         assert np.allclose(qg[:len(ridx)], q_ref, atol=2e-2, rtol=2e-2)
         rest = np.setdiff1d(np.arange(P), ridx)          # rows not selected keep their bits
-        assert torch.equal(kc[s].cpu()[rest], kc0[s][rest]) and torch.equal(vc[s].cpu()[rest], vc0[s][rest])
+        assert torch.equal(kc_h[s][rest], kc0_h[s][rest]) and torch.equal(vc_h[s][rest], vc0_h[s][rest])
 
 
 # ------------------------------------------------------------------ confidence (a6, first half)

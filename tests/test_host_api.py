@@ -59,6 +59,41 @@ def test_init_rejects_bad_arguments_before_using_the_device(lib):
     lib.polestar_destroy(None)
 
 
+def test_init_charges_the_alignment_loss_to_the_callers_buffer(lib):
+    # the plan starts at the next 1024-byte boundary: a buffer that is too small once those bytes are lost must be
+    # refused (E_NOSPACE) before anything is written; polestar_workspace_bytes() itself suffices for any
+    # 256-byte aligned base.  Fake pointers: the checks run before the device or any pointer is touched.
+    m, p = I.config("c1")
+    cm, cp = Bd.c_model(m), Bd.c_params(p)
+    need = lib.polestar_workspace_bytes(C.byref(cm), C.byref(cp))
+    L = m.n_layers
+    fake = (C.c_void_p * L)(*([0x1000] * L))
+    cw = Bd.CWeights(0x1000, 0x1000, 0x1000, fake, fake, fake, fake, fake, fake)
+    prompt = (C.c_int32 * (p.batch * p.prompt_len))(*([1] * (p.batch * p.prompt_len)))
+    ctx = C.c_void_p()
+    base = 0x7000000100                 # 256 mod 1024: 768 bytes are lost to the alignment
+    assert base % 1024 == 256
+    assert lib.polestar_init(C.byref(ctx), C.byref(cm), C.byref(cw), C.byref(cp), prompt, C.c_void_p(base),
+                             need - 1024 + 767, None) == Bd.E_NOSPACE
+    assert lib.polestar_init(C.byref(ctx), C.byref(cm), C.byref(cw), C.byref(cp), prompt, C.c_void_p(base + 0x300),
+                             need - 1025, None) == Bd.E_NOSPACE
+    assert lib.polestar_init(C.byref(ctx), C.byref(cm), C.byref(cw), C.byref(cp), prompt, C.c_void_p(base + 1),
+                             need, None) == Bd.E_INVAL         # not 256-byte aligned
+    assert ctx.value is None
+
+
+def test_confidence_entry_points_check_alignment_and_empty_input(lib):
+    ok = C.c_void_p(0x7000001000)
+    # vocabulary a multiple of four: rows are read with 16-byte loads, the base must be 16-byte aligned
+    for fn, extra in ((lib.polestar_k_confidence, (ok, 1 << 20, None)), (lib.polestar_k_confidence_noalloc, (None,))):
+        assert fn(C.c_void_p(0x7000001004), 2, 1024, 1023, ok, ok, *extra) == Bd.E_INVAL
+        assert fn(None, 2, 1024, 1023, ok, ok, *extra) == Bd.E_INVAL
+        assert fn(None, 0, 1024, 1023, None, None, *extra) == Bd.OK          # no rows: a no-op, null pointers allowed
+        assert fn(ok, -1, 1024, 1023, ok, ok, *extra) == Bd.E_INVAL
+    assert lib.polestar_k_confidence_noalloc(ok, Bd.NOALLOC_MAX_ROWS + 1, 1024, 1023, ok, ok, None) == Bd.E_NOSPACE
+    assert lib.polestar_reload_env() == Bd.OK
+
+
 def test_kernel_entry_points_validate(lib):
     assert lib.polestar_k_select(None, 1, 96, 0, 1, 0.0, 0.0, None, None, None) == Bd.E_INVAL
     assert lib.polestar_k_attention(None, None, None, None, None, None, 1, 1, 1, 1, 64, 0, None) == Bd.E_INVAL

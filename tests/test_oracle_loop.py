@@ -197,7 +197,7 @@ def test_commit_branches_fire_with_scaled_logits():
 def test_suffix_commit_goes_through_layer0_packet():
     # a suffix token committed early changes that position's embedding; the next refresh step
     # must carry it into the cache (otherwise full refresh could not equal no-cache decoding)
-    m, p, w, prompt = tiny(logit_scale=3.0, tau_upd=-1, select_mode=I.SELECT_ALL, tau_suffix=0.7)
+    m, p, w, prompt = tiny(logit_scale=3.0, tau_upd=-1, select_mode=I.SELECT_ALL, tau_suffix=0.7, max_steps=24)
     a = O.PolestarOracle(m, w, p, prompt)
     seen = False
     while not a.done and not seen:

@@ -342,3 +342,37 @@ def test_refresh_delta_bounded_by_projection_norm():
     sig = np.linalg.norm(np.concatenate([wk, wv], 0), 2)
     assert (lhs <= sig * np.linalg.norm(a1 - a0, axis=-1) + 1e-12).all()
     assert lhs[3] == 0.0
+
+
+def test_refresh_chain_rows_equal_full_recompute():
+    # Sec. 4.1 "Measuring Drift and Layer-wise KV Updates": a refreshed K/V row is what a full recompute of the
+    # same hidden row gives; rows that were not selected keep their old contents.  The full recompute here is
+    # written with an independent rotary formula (complex rotation at the row's absolute position) and with
+    # per-row matrix-vector products, so a wrong position, a wrong gain or a scatter to the wrong row shows.
+    P, d, nh, nkv, dh, k = 23, 32, 4, 2, 8, 7
+    H = rng.standard_normal((P, d))
+    drift = np.exp(rng.standard_normal(P))
+    drift[5] = 0.0                                       # never a candidate
+    wq, wk, wv = (rng.standard_normal((n * dh, d)) for n in (nh, nkv, nkv))
+    gain = 1.0 + 0.3 * rng.standard_normal(d)
+    theta = 500.0
+    Kc, Vc = rng.standard_normal((P, nkv, dh)), rng.standard_normal((P, nkv, dh))
+    idx, q, K2, V2 = O.refresh_chain(H, drift, k, wq, wk, wv, gain, 1e-5, theta, nh, nkv, dh, Kc, Vc, emulate_bf16=False)
+    assert idx.tolist() == sorted(np.argsort(-drift, kind="stable")[:k].tolist())       # brute-force top-k, ascending
+    half = dh // 2
+    inv = theta ** (-2.0 * np.arange(half) / dh)
+
+    def rot(x, pos):        # half-split pairs (i, i + dh/2) rotated by pos * theta^(-2i/dh)
+        z = (x[..., :half] + 1j * x[..., half:]) * np.exp(1j * pos * inv)
+        return np.concatenate([z.real, z.imag], -1)
+    for t, r in enumerate(idx):
+        a = H[r] / np.sqrt(np.mean(H[r] ** 2) + 1e-5) * gain
+        assert np.allclose(K2[r], rot((wk @ a).reshape(nkv, dh), r), rtol=1e-12, atol=1e-12)
+        assert np.allclose(V2[r], (wv @ a).reshape(nkv, dh), rtol=1e-12, atol=1e-12)
+        assert np.allclose(q[t], rot((wq @ a).reshape(nh, dh), r), rtol=1e-12, atol=1e-12)
+    rest = np.setdiff1d(np.arange(P), idx)
+    assert np.array_equal(K2[rest], Kc[rest]) and np.array_equal(V2[rest], Vc[rest])
+    assert 5 not in idx
+    # unchanged hidden row => unchanged K/V (Cor. 1 with dH = 0): refreshing twice changes nothing
+    _, _, K3, V3 = O.refresh_chain(H, drift, k, wq, wk, wv, gain, 1e-5, theta, nh, nkv, dh, K2, V2, emulate_bf16=False)
+    assert np.array_equal(K3, K2) and np.array_equal(V3, V2)
