@@ -217,7 +217,8 @@ int polestar_tokens(polestar_ctx *c, int32_t *out_host);
 #define POLESTAR_READ_HCACHE     11  /* float [batch][W_max][d] window hidden cache at `layer`   */
 #define POLESTAR_READ_COMMIT     12  /* int32 [batch][block] bit0 commit, bit1 by confidence,
                                         bit2 by drift, bit3 by quota (last commit)               */
-#define POLESTAR_READ_PPREV      13  /* float [batch][W_max][n_heads][N] stored log attention    */
+#define POLESTAR_READ_PPREV      13  /* float [batch][W_max][n_heads][N] stored log attention
+                                        (log-probabilities, put together from the stored pair)   */
 #define POLESTAR_READ_SUFFIX     14  /* int32 [batch][W_max] bit0 eligible, bit1 committed, bit2 the
                                         rule's own decision (confidence >= tau_suffix)           */
 /* Quantities of the last commit (Sec. 4.2 "Current Block Commit"; Algorithm 1 after the layer loop): */
@@ -270,14 +271,20 @@ int polestar_reload_env(void);
 
 /* Drift of attention rows (Eq. 4; Algorithm 1 "ProxyAttn" + "KL"), optionally with the attention
  * output: for each of R query rows and each head, logp = log softmax_j(q.k_j / sqrt(head_dim))
- * over all N keys; kl[r][h] = sum_j p_j (logp_j - logp_prev[r][h][j]); logp_prev is then
- * overwritten with logp; out[r] = sum_j p_j v_j.
+ * over all N keys; kl[r][h] = sum_j p_j (logp_j - logp_prev_j); the stored row is then replaced
+ * by the new one; out[r] = sum_j p_j v_j.
+ * A stored row is a pair: row_prev_dev[r][h][:] and lse_prev_dev[r][h] with
+ *     log-probability_j = row_prev[r][h][j] - lse_prev[r][h]
+ * (callers that hold plain log-probabilities pass them with lse = 0).  On return the pair describes the
+ * new distribution in the same way; which split the library chooses (scaled scores and their log-sum-exp,
+ * or log-probabilities and 0) depends on the kernel that ran, so always subtract.
  *   q_dev [R][n_heads*head_dim], k_dev / v_dev [N][n_kv*head_dim] (model dtype; one sequence)
- *   logp_prev_dev float [R][n_heads][N] in/out (NULL: no KL, nothing stored)
- *   kl_dev float [R][n_heads] (NULL allowed iff logp_prev_dev NULL), out_dev [R][n_heads*head_dim]
+ *   row_prev_dev float [R][n_heads][N], lse_prev_dev float [R][n_heads], both in/out (both NULL: no KL,
+ *   nothing stored)
+ *   kl_dev float [R][n_heads] (NULL allowed iff row_prev_dev NULL), out_dev [R][n_heads*head_dim]
  *   model dtype (NULL: skipped). */
 int polestar_k_attention(const void *q_dev, const void *k_dev, const void *v_dev,
-                         float *logp_prev_dev, float *kl_dev, void *out_dev,
+                         float *row_prev_dev, float *lse_prev_dev, float *kl_dev, void *out_dev,
                          int32_t R, int32_t N, int32_t n_heads, int32_t n_kv_heads,
                          int32_t head_dim, int32_t dtype, void *cuda_stream);
 

@@ -114,7 +114,7 @@ def load():
     lib.polestar_strerror.restype = C.c_char_p
     lib.polestar_strerror.argtypes = [C.c_int]
     lib.polestar_k_attention.restype = C.c_int
-    lib.polestar_k_attention.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    lib.polestar_k_attention.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
     lib.polestar_k_hidden_delta.restype = C.c_int
     lib.polestar_k_hidden_delta.argtypes = [vp, vp, vp, i32, i32, i32, vp]
     lib.polestar_k_select.restype = C.c_int
@@ -376,9 +376,10 @@ def _dtype_code(t: torch.Tensor) -> int:
     raise PolestarError(E_INVAL, f"unsupported dtype {t.dtype}")
 
 
-def polestar_k_attention(q, k, v, logp_prev, kl, out, n_heads, n_kv_heads, head_dim):
+def polestar_k_attention(q, k, v, row_prev, lse_prev, kl, out, n_heads, n_kv_heads, head_dim):
+    """Stored rows are pairs (row_prev, lse_prev) with log-probability = row_prev - lse_prev[..., None]."""
     R, N = q.shape[0], k.shape[0]
-    _check(load().polestar_k_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(logp_prev), _ptr(kl), _ptr(out), R, N,
+    _check(load().polestar_k_attention(_ptr(q), _ptr(k), _ptr(v), _ptr(row_prev), _ptr(lse_prev), _ptr(kl), _ptr(out), R, N,
                                        n_heads, n_kv_heads, head_dim, _dtype_code(q), C.c_void_p(_stream())))
 
 

@@ -292,8 +292,12 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const T* __restrict__ A,
 struct AttnArgs {
     const Row* rows; int n_rows;
     const void* q; const void* kc; const void* vc; void* out;
+    // Stored attention rows: a row and one float per row such that log-probability = row - lse.  The tensor-core
+    // kernel keeps scaled scores and their log-sum-exp; the other kernels keep log-probabilities and leave lse at 0.
     float* pprev;    // window rows: [batch][W_max][n_heads][N]   (null: none recorded)
     float* aprev;    // active rows: [batch][B][n_heads][N]       (null: none recorded)
+    float* pprev_lse;   // [batch][W_max][n_heads]
+    float* aprev_lse;   // [batch][B][n_heads]
     float* kl;       // [n_rows][n_heads]
     int N, n_heads, n_kv, head_dim, W_max, B, record_kl;
     int rows_per_seq, batch;   // layout of the forward's rows (stand-alone: n_rows, 1)

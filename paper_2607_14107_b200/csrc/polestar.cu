@@ -19,6 +19,7 @@
 
 #include "attn_mma.cuh"
 #include "gemm_tc.cuh"
+#include "attn_tc.cuh"
 #include "gemm_chain.cuh"
 #include "kernels.cuh"
 
@@ -149,9 +150,32 @@ static bool make_map(CUtensorMap* out, const void* base, uint64_t rows, uint64_t
 
 // Tensor maps of one context (its weights and staging buffers at the handful of row counts a decode uses);
 // owned by the context, so it is bounded by the context's buffers and needs no lock.
+// bf16 tensor [batch][rows][width] (row-major), box = 1 x 128 rows x 64 elements, 128-byte swizzle: rows beyond
+// `rows` are out of bounds per batch entry and arrive as zeros
+static bool make_map3(CUtensorMap* out, const void* base, uint64_t batch, uint64_t rows, uint64_t width, int l2promo) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {width, rows, batch};
+    cuuint64_t strides[2] = {width * 2, rows * width * 2};
+    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, (CUtensorMapL2promotion)l2promo,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct MapCache {
     std::map<std::tuple<const void*, uint64_t, uint64_t, uint32_t>, CUtensorMap> m;
     int l2promo = (int)CU_TENSOR_MAP_L2_PROMOTION_L2_128B;
+    // [batch][rows][width] tensors (K / V caches): keyed with box_rows = 0x80000000 | batch
+    const CUtensorMap* get3(const void* base, uint64_t batch, uint64_t rows, uint64_t width) {
+        auto key = std::make_tuple(base, rows, width, (uint32_t)(0x80000000u | (uint32_t)batch));
+        auto it = m.find(key);
+        if (it != m.end()) return &it->second;
+        CUtensorMap tm;
+        if (!make_map3(&tm, base, batch, rows, width, l2promo)) return nullptr;
+        return &m.emplace(key, tm).first->second;
+    }
     const CUtensorMap* get(const void* base, uint64_t rows, uint64_t K, uint32_t box_rows) {
         auto key = std::make_tuple(base, rows, K, box_rows);
         auto it = m.find(key);
@@ -252,6 +276,36 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     return POLESTAR_OK;
 }
 
+// Attention + drift on tensor cores (attn_tc.cuh): bf16, head_dim 128, at most atc::MAX_N keys.
+static bool attention_tc_applies(const AttnArgs& a) {
+    return a.head_dim == atc::DH && a.N <= atc::MAX_N && a.N > 0 && (a.n_heads * a.head_dim) % 64 == 0 &&
+           (a.n_kv * a.head_dim) % 64 == 0;
+}
+static int launch_attention_tc(MapCache& maps, const AttnArgs& a, cudaStream_t st, int* status) {
+    if (a.n_rows <= 0) return POLESTAR_OK;
+    atc::Args g;
+    memset(&g, 0, sizeof(g));
+    g.a = a;
+    const int batch = a.batch > 0 ? a.batch : 1;
+    g.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : a.n_rows;
+    g.tiles_per_seq = (g.rows_per_seq + atc::ROWS - 1) / atc::ROWS;
+    const int tiles_k = (a.N + atc::KEYS - 1) / atc::KEYS;
+    g.kt = tiles_k > atc::MAX_CL ? 2 : 1;
+    g.cl = (tiles_k + g.kt - 1) / g.kt;
+    g.status = status;
+    const int dq = a.n_heads * a.head_dim, dkv = a.n_kv * a.head_dim;
+    const int kv_batch = a.rows ? batch : 1;
+    const CUtensorMap* mq = maps.get(a.q, (uint64_t)a.n_rows, (uint64_t)dq, atc::ROWS);
+    const CUtensorMap* mk = maps.get3(a.kc, (uint64_t)kv_batch, (uint64_t)a.N, (uint64_t)dkv);
+    const CUtensorMap* mv = maps.get3(a.vc, (uint64_t)kv_batch, (uint64_t)a.N, (uint64_t)dkv);
+    if (!mq || !mk || !mv) return POLESTAR_E_CUDA;
+    dim3 grid((unsigned)(g.cl * g.tiles_per_seq * batch), (unsigned)a.n_heads);
+    const size_t smem = atc::smem_bytes(g.kt);
+    if (g.cl > 1) CK(launch_k_cluster(atc::attention_tc_kernel, grid, dim3(atc::THREADS), smem, st, (unsigned)g.cl, *mq, *mk, *mv, g));
+    else CK(launch_k(atc::attention_tc_kernel, grid, dim3(atc::THREADS), smem, st, *mq, *mk, *mv, g));
+    return POLESTAR_OK;
+}
+
 // ------------------------------------------------------------------------------------------
 // context
 // ------------------------------------------------------------------------------------------
@@ -266,7 +320,8 @@ struct Plan {
 
 struct Buffers {
     // persistent
-    int* y; float2* rope; char* kc; char* vc; float* hc; float* pprev; float* aprev; float* theta; int* theta_cnt;
+    int* y; float2* rope; char* kc; char* vc; float* hc; float* pprev; float* aprev; float* pprev_lse; float* aprev_lse;
+    float* theta; int* theta_cnt;
     int* tok_at_h0; float* drift; int* sel_idx; int* sel_cnt; unsigned char* patch; int* forced_idx; int* forced_cnt;
     int* forced_commit; int* forced_tok; float* conf; int* yhat; float* delta; float* Delta; float* taud; int* commit_flags;
     int* own_flags; int* suffix_flags; int* seq_info; int* head_count; int* suf_seq; int* suf_w; int* stats; int* status;
@@ -448,6 +503,8 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(hc, float, L * bs * Wm * d);
     TAKE(pprev, float, L * bs * Wm * nh * N);
     TAKE(aprev, float, bs * B * nh * N);
+    TAKE(pprev_lse, float, L * bs * Wm * nh);
+    TAKE(aprev_lse, float, bs * B * nh);
     TAKE(theta, float, bs * std::max<size_t>(1, p->hist) * B);
     TAKE(theta_cnt, int, bs);
     TAKE(tok_at_h0, int, bs * Wm);
@@ -542,6 +599,7 @@ static cudaError_t set_kernel_attributes() {
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_LOGITS>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV_REFRESH>), gemm_smem);
     PS_ATTR(tc::gemm_chain_kernel<__nv_bfloat16>, gemm_smem);
+    PS_ATTR(atc::attention_tc_kernel, (int)atc::smem_bytes(atc::MAX_KT));
     PS_ATTR(attention_simt_kernel<float>, (int)SIMT_ATTN_SMEM_MAX);
     PS_ATTR(attention_simt_kernel<__nv_bfloat16>, (int)SIMT_ATTN_SMEM_MAX);
 #undef PS_ATTR
@@ -572,6 +630,10 @@ struct Path {
 
     static int attention(polestar_ctx* c, const AttnArgs& a) {
         if (is_bf16 && c->m.head_dim == 128 && !c->sw.attn_simt) {
+            // one kernel family per context (decided by the shape alone): the families keep stored rows in
+            // different forms (scores + log-sum-exp / log-probabilities)
+            if ((c->sw.attn_kernel == 0 || c->sw.attn_kernel == 8) && attention_tc_applies(a))
+                return launch_attention_tc(c->maps, a, c->st, c->b.status);
             CK(launch_attention_mma(a, c->st, c->sms, c->sw.attn_kernel));
             return POLESTAR_OK;
         }
@@ -661,6 +723,8 @@ struct Path {
                 a.rows = b.rows; a.n_rows = M; a.q = b.q_buf; a.kc = kc; a.vc = vc; a.out = b.o_buf;
                 a.pprev = rec_w ? pprev : nullptr;
                 a.aprev = last ? b.aprev : nullptr;
+                a.pprev_lse = b.pprev_lse + (size_t)l * bs * Wm * m.n_heads;
+                a.aprev_lse = b.aprev_lse;
                 a.kl = b.kl; a.N = N; a.n_heads = m.n_heads; a.n_kv = m.n_kv_heads; a.head_dim = m.head_dim;
                 a.W_max = Wm; a.B = B; a.record_kl = sd.record_kl; a.rows_per_seq = sd.rows_per_seq; a.batch = bs;
                 a.scale = 1.0f / sqrtf((float)m.head_dim);
@@ -1121,7 +1185,18 @@ extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void*
         case POLESTAR_READ_VCACHE: src = c->b.vc + layer * bs * N * dkv * c->es; sz = bs * N * dkv * c->es; break;
         case POLESTAR_READ_HCACHE: src = c->b.hc + layer * bs * Wm * d; sz = bs * Wm * d * 4; break;
         case POLESTAR_READ_COMMIT: src = c->b.commit_flags; sz = bs * B * 4; break;
-        case POLESTAR_READ_PPREV: src = c->b.pprev + layer * bs * Wm * m.n_heads * N; sz = bs * Wm * m.n_heads * N * 4; break;
+        case POLESTAR_READ_PPREV: {
+            // stored as (row, lse) with log-probability = row - lse: put together on the host
+            const size_t n_rows = bs * Wm * m.n_heads;
+            std::vector<float> rows(n_rows * N), lse(n_rows);
+            CK(cudaMemcpyAsync(rows.data(), c->b.pprev + layer * n_rows * N, rows.size() * 4, cudaMemcpyDeviceToHost, c->st));
+            CK(cudaMemcpyAsync(lse.data(), c->b.pprev_lse + layer * n_rows, lse.size() * 4, cudaMemcpyDeviceToHost, c->st));
+            CK(cudaStreamSynchronize(c->st));
+            const size_t n_out = std::min(rows.size(), bytes / 4);
+            float* o = (float*)dst;
+            for (size_t i = 0; i < n_out; ++i) o[i] = rows[i] - lse[i / N];
+            return POLESTAR_OK;
+        }
         case POLESTAR_READ_SUFFIX: src = c->b.suffix_flags; sz = bs * Wm * 4; break;
         case POLESTAR_READ_DRIFT_DELTA: src = c->b.Delta; sz = bs * B * 4; break;
         case POLESTAR_READ_TAU_D: src = c->b.taud; sz = bs * B * 4; break;
@@ -1189,19 +1264,19 @@ extern "C" int polestar_force(polestar_ctx* c, int32_t what, int32_t layer, cons
 // ------------------------------------------------------------------------------------------
 // single kernels
 // ------------------------------------------------------------------------------------------
-extern "C" int polestar_k_attention(const void* q, const void* k, const void* v, float* logp_prev, float* kl, void* out,
-                                    int32_t R, int32_t N, int32_t n_heads, int32_t n_kv, int32_t head_dim, int32_t dtype,
-                                    void* stream) {
+extern "C" int polestar_k_attention(const void* q, const void* k, const void* v, float* logp_prev, float* lse_prev,
+                                    float* kl, void* out, int32_t R, int32_t N, int32_t n_heads, int32_t n_kv,
+                                    int32_t head_dim, int32_t dtype, void* stream) {
     if (R < 0 || N <= 0 || n_heads <= 0 || n_kv <= 0 || n_heads % n_kv || head_dim <= 0 || head_dim > 256)
         return POLESTAR_E_INVAL;
     if (dtype != POLESTAR_F32 && dtype != POLESTAR_BF16) return POLESTAR_E_INVAL;
     if (R == 0) return POLESTAR_OK;              // no rows: nothing to do (the row pointers may be null)
     if (!q || !k || !v) return POLESTAR_E_INVAL;
-    if (logp_prev && !kl) return POLESTAR_E_INVAL;
+    if (logp_prev && (!kl || !lse_prev)) return POLESTAR_E_INVAL;
     cudaStream_t st = (cudaStream_t)stream;
     AttnArgs a;
     memset(&a, 0, sizeof(a));
-    a.n_rows = R; a.q = q; a.kc = k; a.vc = v; a.out = out; a.pprev = logp_prev; a.kl = kl; a.N = N;
+    a.n_rows = R; a.q = q; a.kc = k; a.vc = v; a.out = out; a.pprev = logp_prev; a.pprev_lse = lse_prev; a.kl = kl; a.N = N;
     a.n_heads = n_heads; a.n_kv = n_kv; a.head_dim = head_dim; a.record_kl = 1; a.rows_per_seq = R; a.batch = 1;
     a.scale = 1.0f / sqrtf((float)head_dim);
     DevInfo di;
@@ -1209,6 +1284,12 @@ extern "C" int polestar_k_attention(const void* q, const void* k, const void* v,
     if (rc) return rc;
     const Switches sw = stand_alone_switches();
     if (dtype == POLESTAR_BF16 && head_dim == 128 && !sw.attn_simt) {
+        if ((sw.attn_kernel == 0 || sw.attn_kernel == 8) && attention_tc_applies(a) &&
+            !((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v)) & 15)) {
+            MapCache maps;                 // the three tensor maps of this call
+            maps.l2promo = sw.l2promo;
+            return launch_attention_tc(maps, a, st, nullptr);
+        }
         CK(launch_attention_mma(a, st, di.sm_count, sw.attn_kernel));
         return POLESTAR_OK;
     }

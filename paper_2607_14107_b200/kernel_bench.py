@@ -136,13 +136,14 @@ def bench_drift(quick):
         k = [I.normal_tensor(I.tensor_key(5, c, 2), (N, nh * dh), 1.0, torch.bfloat16, "cuda") for c in range(n_copy)]
         v = [I.normal_tensor(I.tensor_key(5, c, 3), (N, nh * dh), 1.0, torch.bfloat16, "cuda") for c in range(n_copy)]
         prev = [torch.full((R, nh, N), -math.log(N), device="cuda") for _ in range(n_copy)]
+        lse = [torch.zeros((R, nh), device="cuda") for _ in range(n_copy)]
         kl = torch.empty((R, nh), device="cuda")
         out = torch.empty((R, nh * dh), dtype=torch.bfloat16, device="cuda")
-        us = timed(lambda i: Bd.polestar_k_attention(q[i % n_copy], k[i % n_copy], v[i % n_copy], prev[i % n_copy], kl, out,
+        us = timed(lambda i: Bd.polestar_k_attention(q[i % n_copy], k[i % n_copy], v[i % n_copy], prev[i % n_copy], lse[i % n_copy], kl, out,
                                                      nh, nh, dh), 48)
         by = 2 * N * nh * dh * 2 + 2 * R * nh * N * 4 + 2 * R * nh * dh * 2
         emit("drift+attention rows", us, by, 4.0 * R * N * nh * dh, {"shape": name, "rows": R, "keys": N})
-        us = timed(lambda i: Bd.polestar_k_attention(q[i % n_copy], k[i % n_copy], v[i % n_copy], None, None, out,
+        us = timed(lambda i: Bd.polestar_k_attention(q[i % n_copy], k[i % n_copy], v[i % n_copy], None, None, None, out,
                                                      nh, nh, dh), 48)
         emit("attention rows (no drift)", us, 2 * N * nh * dh * 2 + 2 * R * nh * dh * 2, 4.0 * R * N * nh * dh,
              {"shape": name, "rows": R, "keys": N})

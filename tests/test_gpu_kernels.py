@@ -43,6 +43,15 @@ def test_attention_drift_matches_oracle(dtype, R, N, nh, nkv, dh):
     (6, 32, 512, 4, 4), (6, 21, 300, 4, 2), (6, 5, 37, 2, 2),        # keys split over a cluster of two CTAs
     (7, 32, 1000, 2, 1), (7, 16, 512, 2, 2),
     (0, 32, 512, 2, 2),            # automatic choice for one block of rows
+    # tensor-core kernel (tcgen05, S and O in tensor memory, key ranges over a cluster)
+    (8, 128, 512, 2, 2),           # one full row tile, four key ranges
+    (8, 32, 512, 4, 4),            # a block of active rows
+    (8, 5, 37, 2, 2),              # fewer rows and keys than one tile, no cluster
+    (8, 37, 200, 4, 2),            # ragged rows and keys, GQA, two key ranges
+    (8, 150, 1100, 2, 1),          # two row tiles, two S tiles per CTA, five key ranges (last one a single ragged tile)
+    (8, 200, 2048, 8, 8),          # the long-sequence shape: 2 x 8 key tiles
+    (8, 130, 1024, 2, 2),          # eight key ranges of one tile
+    (8, 64, 402, 2, 1),            # key count not a multiple of four (scalar access to the stored rows)
 ])
 def test_attention_kernel_variants(monkeypatch, variant, R, N, nh, nkv):
     monkeypatch.setenv("POLESTAR_ATTN_KERNEL", str(variant))
@@ -57,9 +66,10 @@ def check_attention(dtype, R, N, nh, nkv, dh):
     prev_s = rnd((R, nh, N), 4, 1.0).double()
     prev = (prev_s - torch.logsumexp(prev_s, -1, keepdim=True)).float()
     prev_dev = prev.clone().cuda()
+    lse_dev = torch.zeros((R, nh), device="cuda")          # stored pair (row, lse): log-probability = row - lse
     kl = torch.full((R, nh), -1.0, device="cuda")
     out = torch.zeros((R, nh * dh), dtype=dtype, device="cuda")
-    Bd.polestar_k_attention(q, k, v, prev_dev, kl, out, nh, nkv, dh)
+    Bd.polestar_k_attention(q, k, v, prev_dev, lse_dev, kl, out, nh, nkv, dh)
     torch.cuda.synchronize()
     qn, kn, vn = bf16_np(q).reshape(R, nh, dh), bf16_np(k).reshape(N, nkv, dh), bf16_np(v).reshape(N, nkv, dh)
     logp = O.attn_logp_rows(qn, kn)
@@ -67,14 +77,17 @@ def check_attention(dtype, R, N, nh, nkv, dh):
     rp = O.bf16_round if dtype == torch.bfloat16 else (lambda x: x)
     ref_out = O.attn_out_rows(logp, vn, rp)
     ref_kl = np.sum(np.exp(logp) * (logp - prev.double().numpy()), -1)
-    assert np.allclose(prev_dev.cpu().numpy(), logp, atol=2e-4, rtol=1e-5)       # stored rows = new log-probs
+    stored = prev_dev.cpu().double().numpy() - lse_dev.cpu().double().numpy()[..., None]
+    assert np.allclose(stored, logp, atol=2e-4, rtol=1e-5)       # stored rows = new log-probs
     assert np.allclose(kl.cpu().numpy(), ref_kl, atol=1e-3 * max(1.0, np.abs(ref_kl).max()), rtol=1e-3)
     assert np.allclose(bf16_np(out), ref_out, atol=tol, rtol=tol)
     # Eq. 4 invariants: drift against the rows just stored is zero, and KL >= 0
     kl2 = torch.full((R, nh), -1.0, device="cuda")
-    Bd.polestar_k_attention(q, k, v, prev_dev, kl2, None, nh, nkv, dh)
+    Bd.polestar_k_attention(q, k, v, prev_dev, lse_dev, kl2, None, nh, nkv, dh)
     torch.cuda.synchronize()
     assert np.abs(kl2.cpu().numpy()).max() < 1e-5
+    if dtype == torch.bfloat16:
+        assert (kl2 == 0).all()            # unchanged rows: exactly zero drift (same bits in, same bits out)
     assert (kl.cpu().numpy() > -1e-4).all()
     # Pinsker bound of Appendix B, Prop. 2 with the current value rows
     M = np.linalg.norm(vn, axis=-1).max()
@@ -91,7 +104,7 @@ def test_attention_without_recording():
     k = rnd((N, nh * dh), 2, 1.0, torch.bfloat16).cuda()
     v = rnd((N, nh * dh), 3, 1.0, torch.bfloat16).cuda()
     out = torch.zeros((R, nh * dh), dtype=torch.bfloat16, device="cuda")
-    Bd.polestar_k_attention(q, k, v, None, None, out, nh, nh, dh)
+    Bd.polestar_k_attention(q, k, v, None, None, None, out, nh, nh, dh)
     ref = torch.nn.functional.scaled_dot_product_attention(
         q.float().view(R, nh, dh).permute(1, 0, 2)[None], k.float().view(N, nh, dh).permute(1, 0, 2)[None],
         v.float().view(N, nh, dh).permute(1, 0, 2)[None])[0].permute(1, 0, 2).reshape(R, nh * dh)
@@ -109,7 +122,7 @@ def test_attention_many_rows_single_pass(monkeypatch, variant, R, N, nh, nkv):
     k = rnd((N, nkv * dh), 2, 1.0, torch.bfloat16).cuda()
     v = rnd((N, nkv * dh), 3, 1.0, torch.bfloat16).cuda()
     out = torch.zeros((R, nh * dh), dtype=torch.bfloat16, device="cuda")
-    Bd.polestar_k_attention(q, k, v, None, None, out, nh, nkv, dh)
+    Bd.polestar_k_attention(q, k, v, None, None, None, out, nh, nkv, dh)
     torch.cuda.synchronize()
     qn, kn, vn = bf16_np(q).reshape(R, nh, dh), bf16_np(k).reshape(N, nkv, dh), bf16_np(v).reshape(N, nkv, dh)
     ref = O.attn_out_rows(O.attn_logp_rows(qn, kn), vn, O.bf16_round)
@@ -246,9 +259,9 @@ def test_empty_inputs_are_noops():
     Bd.polestar_k_confidence(torch.zeros((0, 1024), device=dev), 1023, torch.zeros(0, dtype=torch.int32, device=dev),
                              torch.zeros(0, device=dev), torch.empty(4096, dtype=torch.uint8, device=dev))
     k = torch.zeros((10, 256), dtype=torch.bfloat16, device=dev)
-    Bd.polestar_k_attention(e, k, k, None, None, torch.zeros((0, 256), dtype=torch.bfloat16, device=dev), 2, 2, 128)
+    Bd.polestar_k_attention(e, k, k, None, None, None, torch.zeros((0, 256), dtype=torch.bfloat16, device=dev), 2, 2, 128)
     with pytest.raises(Bd.PolestarError):                                             # no keys: softmax over nothing
-        Bd.polestar_k_attention(torch.zeros((4, 256), dtype=torch.bfloat16, device=dev), e, e, None, None,
+        Bd.polestar_k_attention(torch.zeros((4, 256), dtype=torch.bfloat16, device=dev), e, e, None, None, None,
                                 torch.zeros((4, 256), dtype=torch.bfloat16, device=dev), 2, 2, 128)
     torch.cuda.synchronize()
 
