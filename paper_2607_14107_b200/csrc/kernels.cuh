@@ -302,6 +302,8 @@ struct AttnArgs {
     int N, n_heads, n_kv, head_dim, W_max, B, record_kl;
     int rows_per_seq, batch;   // layout of the forward's rows (stand-alone: n_rows, 1)
     float scale;
+    int dirty_lo, dirty_hi;    // key positions [lo, hi) of every sequence that the kernel running just before may have
+                               // written; all other K/V rows were complete before this forward was launched
     // stand-alone form: rows == null, row r belongs to sequence 0 and records into pprev[r]
 };
 

@@ -301,8 +301,8 @@ static int launch_attention_tc(MapCache& maps, const AttnArgs& a, cudaStream_t s
     if (!mq || !mk || !mv) return POLESTAR_E_CUDA;
     dim3 grid((unsigned)(g.cl * g.tiles_per_seq * batch), (unsigned)a.n_heads);
     const size_t smem = atc::smem_bytes(g.kt);
-    if (g.cl > 1) CK(launch_k_cluster(atc::attention_tc_kernel, grid, dim3(atc::THREADS), smem, st, (unsigned)g.cl, *mq, *mk, *mv, g));
-    else CK(launch_k(atc::attention_tc_kernel, grid, dim3(atc::THREADS), smem, st, *mq, *mk, *mv, g));
+    // (always a cluster launch, also for a single key range: the kernel addresses its own CTA through the cluster window)
+    CK(launch_k_cluster(atc::attention_tc_kernel, grid, dim3(atc::THREADS), smem, st, (unsigned)g.cl, *mq, *mk, *mv, g));
     return POLESTAR_OK;
 }
 
@@ -632,7 +632,13 @@ struct Path {
         if (is_bf16 && c->m.head_dim == 128 && !c->sw.attn_simt) {
             // one kernel family per context (decided by the shape alone): the families keep stored rows in
             // different forms (scores + log-sum-exp / log-probabilities)
-            if ((c->sw.attn_kernel == 0 || c->sw.attn_kernel == 8) && attention_tc_applies(a))
+            // Launches that record or compare stored rows all go to the tensor-core kernel.  A launch that touches
+            // no stored row (the layers below the last one of a step without refresh) may take either family: for a
+            // single block of rows the warp-level kernel's shorter dependency chain wins (11 us against 16 us per
+            // layer at the 8B shape), everywhere else the tensor-core kernel does.
+            const bool records = a.pprev != nullptr || a.aprev != nullptr;
+            const bool few_rows = !records && a.rows_per_seq <= 64 && a.N <= 1024 && c->sw.attn_kernel == 0;
+            if ((c->sw.attn_kernel == 0 || c->sw.attn_kernel == 8) && attention_tc_applies(a) && !few_rows)
                 return launch_attention_tc(c->maps, a, c->st, c->b.status);
             CK(launch_attention_mma(a, c->st, c->sms, c->sw.attn_kernel));
             return POLESTAR_OK;
@@ -728,6 +734,13 @@ struct Path {
                 a.kl = b.kl; a.N = N; a.n_heads = m.n_heads; a.n_kv = m.n_kv_heads; a.head_dim = m.head_dim;
                 a.W_max = Wm; a.B = B; a.record_kl = sd.record_kl; a.rows_per_seq = sd.rows_per_seq; a.batch = bs;
                 a.scale = 1.0f / sqrtf((float)m.head_dim);
+                // positions whose K/V this layer's QKV projection writes: the forwarded rows of an entry step; the
+                // active block and, on refresh steps, the patched window rows of a within-block step
+                if (!within) { a.dirty_lo = sd.e0; a.dirty_hi = sd.e0 + sd.rows_per_seq; }
+                else {
+                    a.dirty_lo = sparse ? std::min(sd.act_start, sd.pre_start) : sd.act_start;
+                    a.dirty_hi = sparse ? std::max(sd.act_start + B, sd.suf_start + (sd.W - sd.n_pre)) : sd.act_start + B;
+                }
                 if ((rc = attention(c, a))) return rc;
             }
             const int* list = nullptr;
@@ -1279,6 +1292,7 @@ extern "C" int polestar_k_attention(const void* q, const void* k, const void* v,
     a.n_rows = R; a.q = q; a.kc = k; a.vc = v; a.out = out; a.pprev = logp_prev; a.pprev_lse = lse_prev; a.kl = kl; a.N = N;
     a.n_heads = n_heads; a.n_kv = n_kv; a.head_dim = head_dim; a.record_kl = 1; a.rows_per_seq = R; a.batch = 1;
     a.scale = 1.0f / sqrtf((float)head_dim);
+    a.dirty_lo = 0; a.dirty_hi = N;              // a stand-alone call knows nothing about who wrote K / V: wait for everything
     DevInfo di;
     int rc = device_info(&di);
     if (rc) return rc;

@@ -21,7 +21,8 @@ NAMES = {1: "build_rows", 2: "embed", 3: "prep_qkv", 4: "prep_rows", 5: "prep_he
          10: "head_list", 11: "conf_partial", 12: "conf_final", 13: "commit", 14: "delta", 15: "keep_hidden",
          100: "gemm_qkv", 101: "gemm_o", 102: "gemm_gate_up", 103: "gemm_down", 104: "gemm_lm_head",
          200: "gemm_qkv:cta0_done", 201: "gemm_o:cta0_done", 202: "gemm_gate_up:cta0_done",
-         203: "gemm_down:cta0_done", 204: "gemm_lm_head:cta0_done"}
+         203: "gemm_down:cta0_done", 204: "gemm_lm_head:cta0_done",
+         311: "attn:end"}
 
 
 def main():
@@ -29,6 +30,7 @@ def main():
     ap.add_argument("--config", default="c2")
     ap.add_argument("--forwards", type=int, default=6)
     ap.add_argument("--max-steps", type=int, default=0, help="override the step budget (fewer steps: more tokens per step, blocks turn over sooner)")
+    ap.add_argument("--attn-cycles", action="store_true", help="print the cycle counters of the last attention launch")
     ap.add_argument("--entry", action="store_true", help="also print forward 0, the block-entry forward of the first block")
     a = ap.parse_args()
     os.environ["POLESTAR_KERNEL_TRACE"] = "1"
@@ -48,6 +50,12 @@ def main():
     torch.cuda.synchronize()
     out = np.zeros(8192, np.int64)
     Bd._check(Bd.load().polestar_read(dec.ctx, Bd.READ_TRACE_KERNELS, 0, out.ctypes.data_as(C.c_void_p), 65536))
+    if a.attn_cycles:
+        # cycle counters of the last attention launch (attn_tc.cuh dbg_clock): per thread, relative to its point 0
+        for name, base in (("epilogue rows 64..", 0), ("epilogue rows 0..", 20), ("producer", 40), ("mma", 50)):
+            v = out[8100 + base:8100 + base + 20]
+            t0 = min(x for x in out[8100:8160] if x > 0)
+            print(f"  {name:20s}", [int(x - t0) if x > 0 else None for x in v])
     n = min(int(out[0]), 4000)
     ids, ts = out[1:1 + 2 * n:2], out[2:2 + 2 * n:2].astype(np.float64) / 1000.0
     order = np.argsort(ts, kind="stable")
