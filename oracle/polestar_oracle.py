@@ -35,7 +35,12 @@ the design notes of the repository):
   * committed suffix tokens reach the cache as a layer-0 packet at the next
     refresh step;
   * only rows with drift above ``drift_floor`` are top-k candidates, so zero
-    drift refreshes nothing; mode ALL takes every window row.
+    drift refreshes nothing; mode ALL takes every window row;
+  * centroid proxies (mode CLUSTER_TOPK; Sec. 4.1 "Cluster and Quantize Hidden
+    States", "Measuring Drift and Layer-wise KV Updates"): a deterministic
+    spherical K-means (see ``spherical_kmeans``), proxies = member means at the
+    rounded mean position, incremental centroid update, drift per cluster, the
+    member rows of the top-k clusters are refreshed.
 
 Synthetic model (the paper fixes none of it): pre-norm Transformer without
 attention mask, RMSNorm, half-split RoPE on q and k at absolute positions,
@@ -56,7 +61,7 @@ import numpy as np
 
 F64 = np.float64
 
-SELECT_TOPK_FRAC, SELECT_TOPK_COUNT, SELECT_THRESHOLD, SELECT_ALL, SELECT_NONE = range(5)
+SELECT_TOPK_FRAC, SELECT_TOPK_COUNT, SELECT_THRESHOLD, SELECT_ALL, SELECT_NONE, SELECT_CLUSTER_TOPK = range(6)
 FLAG_DRIFT_COMMIT, FLAG_SUFFIX_COMMIT, FLAG_GE_COMPARE, FLAG_NOCACHE = 1, 2, 4, 8
 
 
@@ -197,6 +202,61 @@ def select_rows(D: np.ndarray, mode: int, *, frac: float = 0.25, k: int = 0,
     return np.array(sorted(cand[:max(kk, 0)]), np.int64)
 
 
+def spherical_kmeans(H: np.ndarray, K: int, iters: int) -> np.ndarray:
+    """Cluster labels of the rows of H by spherical K-means (Sec. 4.1 "Cluster and Quantize
+    Hidden States"): rows are compared by cosine similarity.
+
+    The paper fixes neither the initialisation, the number of iterations nor the handling of
+    empty clusters; the reading taken here is deterministic:
+      * with no more rows than clusters every row is its own cluster (also when rows coincide);
+        otherwise centre j starts at the unit vector of row floor((j + 1/2) * W / K) (evenly
+        spaced rows of the window);
+      * `iters` Lloyd iterations: every row goes to the centre with the largest cosine
+        (lowest cluster id on ties), then every centre becomes the normalised sum of its
+        members' unit vectors; a cluster without members keeps its centre;
+      * the labels of the last assignment are returned.
+    """
+    H = np.asarray(H, F64)
+    W = H.shape[0]
+    if W == 0:
+        return np.zeros(0, np.int64)
+    if W <= int(K):
+        return np.arange(W, dtype=np.int64)      # no more rows than clusters: every row is its own cluster
+    Ke = max(1, int(K))
+    U = H / np.maximum(np.linalg.norm(H, axis=1, keepdims=True), 1e-300)
+    C = np.stack([U[int(math.floor((j + 0.5) * W / Ke))] for j in range(Ke)])
+    labels = np.zeros(W, np.int64)
+    for _ in range(max(1, int(iters))):
+        sims = U @ C.T                                   # [W, Ke] cosines
+        labels = np.argmax(sims, axis=1)                 # first maximum: lowest cluster id on ties
+        for j in range(Ke):
+            mem = np.nonzero(labels == j)[0]
+            if len(mem):
+                v = U[mem].sum(axis=0)
+                n = np.linalg.norm(v)
+                if n > 0:
+                    C[j] = v / n
+    return labels.astype(np.int64)
+
+
+def cluster_proxies(H: np.ndarray, positions: np.ndarray, labels: np.ndarray, K: int):
+    """Proxy rows of the clusters: the mean of the members' hidden states (member scale, so that a
+    cluster of one row is that row) and a rotary position, the rounded mean of the members'
+    positions.  Returns (Z [K, d], pos [K], counts [K]); clusters without members get zeros."""
+    H = np.asarray(H, F64)
+    d = H.shape[1]
+    Z = np.zeros((K, d), F64)
+    pos = np.zeros(K, np.int64)
+    cnt = np.zeros(K, np.int64)
+    for j in range(K):
+        mem = np.nonzero(labels == j)[0]
+        cnt[j] = len(mem)
+        if len(mem):
+            Z[j] = H[mem].mean(axis=0)
+            pos[j] = int(math.floor(np.mean(np.asarray(positions, F64)[mem]) + 0.5))
+    return Z, pos, cnt
+
+
 def confidence_rows(logits: np.ndarray, mask_id: int):
     """Eq. 1 and the confidence of Sec. 2: y_hat = argmax over v != [MASK] (lowest id
     on ties), c = softmax(logits over the whole vocabulary)[y_hat]."""
@@ -301,6 +361,12 @@ class _Seq:
         self.Vc = [np.zeros((self.N, m.n_kv_heads, m.head_dim), F64) for _ in range(L)]
         self.Hc: List[Optional[np.ndarray]] = [None] * L
         self.Pprev: List[Optional[np.ndarray]] = [None] * L
+        # centroid proxies (select_mode CLUSTER_TOPK): per layer the labels of the window rows, the proxy rows
+        # (member means), their rotary positions and member counts
+        self.labels: List[Optional[np.ndarray]] = [None] * L
+        self.Z: List[Optional[np.ndarray]] = [None] * L
+        self.zpos: List[Optional[np.ndarray]] = [None] * L
+        self.zcnt: List[Optional[np.ndarray]] = [None] * L
         self.Aprev = None
         self.theta: List[np.ndarray] = []
         self.tok_at_h0 = None
@@ -360,10 +426,22 @@ class _Seq:
             self.Kc[l][rows] = k
             self.Vc[l][rows] = v
             logp = attn_logp_rows(q, self.Kc[l], self.rowwise)
-            self.Pprev[l] = logp[wi].copy()
+            if p.select_mode == SELECT_CLUSTER_TOPK:
+                # Algorithm 1 block entry: Z, M <- SphericalKMeans(H, K);  P <- ProxyAttn(Z), all layers
+                K = p.n_clusters
+                self.labels[l] = spherical_kmeans(self.Hc[l], K, p.kmeans_iters)
+                self.Z[l], self.zpos[l], self.zcnt[l] = cluster_proxies(self.Hc[l], win, self.labels[l], K)
+                live = np.nonzero(self.zcnt[l] > 0)[0]
+                self.Pprev[l] = np.zeros((K, m.n_heads, self.N), F64)
+                if len(live):
+                    qz, _, _ = self._qkv(l, self.Z[l][live], self.zpos[l][live])
+                    self.Pprev[l][live] = attn_logp_rows(qz, self.Kc[l], self.rowwise)
+            else:
+                self.Pprev[l] = logp[wi].copy()
             if l == m.n_layers - 1:
                 self.Aprev = logp[ai].copy()
             x = self._finish(l, x, logp)
+        tr["labels"] = [None if a is None else a.copy() for a in self.labels]
         tr["x_act"].append(x[ai].copy())
         self.tok_at_h0 = self.y[win].copy()
         self.win, self.act, self.n_pre = win, act, len(pre)
@@ -397,6 +475,11 @@ class _Seq:
             tr["x_act"].append(x.copy())
             # 1. patch the caches from the update packet of the previous layer
             if refresh and len(U_idx):
+                if p.select_mode == SELECT_CLUSTER_TOPK:
+                    # the centroid follows its refreshed members (Sec. 4.1: "updated incrementally")
+                    for t, i in enumerate(U_idx):
+                        c = self.labels[l][i]
+                        self.Z[l][c] = self.Z[l][c] + (U_val[t] - self.Hc[l][i]) / self.zcnt[l][c]
                 self.Hc[l][U_idx] = U_val
                 _, k, v = self._qkv(l, U_val, win[U_idx])
                 self.Kc[l][win[U_idx]] = k
@@ -412,7 +495,35 @@ class _Seq:
                 self.Aprev = logpA.copy()
             x = self._finish(l, x, logpA)
             # 3. drift of the window rows, selection, sparse forward -> next packet
-            if refresh:
+            if refresh and p.select_mode == SELECT_CLUSTER_TOPK:
+                # proxy attention of the centroids, drift per cluster, top-k clusters -> their member rows
+                K = p.n_clusters
+                live = np.nonzero(self.zcnt[l] > 0)[0]
+                D = np.zeros(K, F64)
+                if len(live):
+                    qz, _, _ = self._qkv(l, self.Z[l][live], self.zpos[l][live])
+                    Pz = attn_logp_rows(qz, self.Kc[l], self.rowwise)
+                    D[live] = kl_rows(Pz, self.Pprev[l][live])
+                    self.Pprev[l][live] = Pz
+                if forced_sel is not None:
+                    S = np.asarray(forced_sel[l], np.int64)
+                    chosen = np.unique(self.labels[l][S]) if len(S) else np.zeros(0, np.int64)
+                else:
+                    # (clusters without members have drift 0 and are never candidates: drift_floor >= 0)
+                    chosen = select_rows(D, SELECT_TOPK_COUNT, k=p.cluster_k, floor=p.drift_floor)
+                    S = np.array([i for i in range(W) if self.labels[l][i] in set(chosen.tolist())], np.int64)
+                tr["D"].append(D)
+                tr["sel"].append(S)
+                tr.setdefault("clusters", []).append(chosen)
+                U_idx = S
+                if len(S):
+                    # the selected rows' own attention rows (each row's query from its cached hidden state)
+                    qs, _, _ = self._qkv(l, self.Hc[l][S], win[S])
+                    Ps = attn_logp_rows(qs, self.Kc[l], self.rowwise)
+                    U_val = self._finish(l, self.Hc[l][S], Ps)
+                else:
+                    U_val = np.zeros((0, m.d_model), F64)
+            elif refresh:
                 qw, _, _ = self._qkv(l, self.Hc[l], win)
                 P = attn_logp_rows(qw, self.Kc[l], self.rowwise)
                 D = kl_rows(P, self.Pprev[l])

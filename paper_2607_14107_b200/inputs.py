@@ -38,6 +38,7 @@ SELECT_TOPK_COUNT = 1
 SELECT_THRESHOLD = 2
 SELECT_ALL = 3
 SELECT_NONE = 4
+SELECT_CLUSTER_TOPK = 5
 
 FLAG_DRIFT_COMMIT = 1 << 0
 FLAG_SUFFIX_COMMIT = 1 << 1
@@ -101,6 +102,11 @@ class Params:
     tau_suffix: float = 0.9
     logit_scale: float = 1.0
     flags: int = FLAG_DEFAULT
+    # centroid proxies (select_mode = SELECT_CLUSTER_TOPK): K clusters of the window's hidden states per layer,
+    # the cluster_k clusters with the largest drift are refreshed; Lloyd iterations of the spherical K-means
+    n_clusters: int = 8
+    cluster_k: int = 4
+    kmeans_iters: int = 4
 
     @property
     def seq_len(self) -> int:

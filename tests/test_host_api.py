@@ -96,7 +96,7 @@ def test_confidence_entry_points_check_alignment_and_empty_input(lib):
 
 def test_kernel_entry_points_validate(lib):
     assert lib.polestar_k_select(None, 1, 96, 0, 1, 0.0, 0.0, None, None, None) == Bd.E_INVAL
-    assert lib.polestar_k_attention(None, None, None, None, None, None, 1, 1, 1, 1, 64, 0, None) == Bd.E_INVAL
+    assert lib.polestar_k_attention(None, None, None, None, None, None, None, 1, 1, 1, 1, 64, 0, None) == Bd.E_INVAL
     assert lib.polestar_k_hidden_delta(None, None, None, 1, 8, 0, None) == Bd.E_INVAL
     assert lib.polestar_k_refresh_scratch_bytes(0, 1, 1, 1, 1, 1) == 0
     assert lib.polestar_k_refresh_scratch_bytes(1, 128, 4096, 32, 32, 128) > 128 * 4096 * 2

@@ -242,3 +242,81 @@ def test_bf16_emulation_changes_little():
     a.step(); b.step()
     xa, xb = a.seqs[0].trace["x_act"][-1], b.seqs[0].trace["x_act"][-1]
     assert 0 < np.abs(xa - xb).max() < 2e-2 * np.abs(xa).max()
+
+
+# ---------------------------------------------------------------- centroid proxies (Sec. 4.1)
+def test_singleton_clusters_equal_per_position_mode():
+    # With at least as many clusters as window rows every cluster is one row: its proxy is the row itself at the
+    # row's position, so cluster drift is row drift and "top-k clusters" is "top-k rows": the whole decode must be
+    # that of the per-position mode with the same budget: the same refresh sets and tokens, and the same numbers
+    # up to the rounding of the incremental centroid update (old + (new - old) instead of new).
+    m, p, w, prompt = tiny(logit_scale=3.0, tau_upd=-1, tau_suffix=0.7)
+    pa = dataclasses.replace(p, select_mode=I.SELECT_TOPK_COUNT, select_k=5)
+    pb = dataclasses.replace(p, select_mode=I.SELECT_CLUSTER_TOPK, n_clusters=64, cluster_k=5)
+    a, b = O.PolestarOracle(m, w, pa, prompt, rowwise=True), O.PolestarOracle(m, w, pb, prompt, rowwise=True)
+    n_ref = 0
+    while not a.done:
+        a.step(); b.step()
+        ta, tb = a.seqs[0].trace, b.seqs[0].trace
+        assert np.allclose(ta["logits"], tb["logits"], rtol=1e-9, atol=1e-9)
+        if ta["kind"] == "within" and ta["refresh"]:
+            n_ref += 1
+            W = len(a.seqs[0].win)
+            for l in range(m.n_layers):
+                assert np.array_equal(ta["sel"][l], tb["sel"][l])
+                assert np.allclose(ta["D"][l], tb["D"][l][:W], rtol=1e-9, atol=1e-12)
+                assert np.allclose(a.seqs[0].Kc[l], b.seqs[0].Kc[l], rtol=1e-9, atol=1e-9)
+        a.commit(); b.commit()
+        assert np.array_equal(a.tokens(), b.tokens())
+    assert b.done and n_ref > 5
+
+
+def test_all_clusters_selected_equals_nocache_bitwise():
+    m, p, w, prompt = tiny(select_mode=I.SELECT_CLUSTER_TOPK, n_clusters=4, cluster_k=4, tau_upd=-1,
+                           win_prefix_blocks=100, win_suffix_blocks=100, tau_suffix=0.4)
+    a = O.PolestarOracle(m, w, p, prompt, rowwise=True)
+    b = O.NoCacheOracle(m, w, dataclasses.replace(p, select_mode=I.SELECT_ALL), prompt, rowwise=True)
+    while not a.done:
+        a.step(); b.step()
+        assert np.array_equal(a.seqs[0].trace["logits"], b.seqs[0].trace["logits"])
+        a.commit(); b.commit()
+        assert np.array_equal(a.tokens(), b.tokens())
+
+
+def test_cluster_mode_invariants():
+    m, p, w, prompt = tiny(select_mode=I.SELECT_CLUSTER_TOPK, n_clusters=4, cluster_k=2, tau_upd=-1, logit_scale=3.0)
+    a = O.PolestarOracle(m, w, p, prompt)
+    n_ref = 0
+    while not a.done:
+        a.step()
+        s = a.seqs[0]
+        tr = s.trace
+        if tr["kind"] == "within" and tr["refresh"]:
+            n_ref += 1
+            for l in range(m.n_layers):
+                D, S, chosen = tr["D"][l], tr["sel"][l], tr["clusters"][l]
+                assert D.shape == (p.n_clusters,) and (D >= -1e-12).all()
+                assert len(chosen) <= p.cluster_k
+                # the refreshed rows are exactly the members of the chosen clusters, ascending
+                assert S.tolist() == [i for i in range(len(s.win)) if s.labels[l][i] in chosen.tolist()]
+                # the chosen clusters are the ones with the largest positive drift
+                rest = [c for c in range(p.n_clusters) if c not in chosen.tolist() and D[c] > 0]
+                if len(chosen) and rest:
+                    assert D[chosen].min() >= max(D[c] for c in rest)
+                # incremental centroid update == mean of the members' current hidden rows
+                Z, _, cnt = O.cluster_proxies(s.Hc[l], s.win, s.labels[l], p.n_clusters)
+                assert np.allclose(Z, s.Z[l], rtol=1e-11, atol=1e-12) and np.array_equal(cnt, s.zcnt[l])
+        a.commit()
+    assert n_ref > 5
+
+
+def test_cluster_mode_zero_drift_refreshes_nothing():
+    m, p, w, prompt = tiny(select_mode=I.SELECT_CLUSTER_TOPK, n_clusters=4, cluster_k=2, tau_upd=-1)
+    a = O.PolestarOracle(m, w, p, prompt)
+    a.step()
+    a.commit(forced=[{"commit": np.zeros(p.block, bool), "suffix": ()}])      # nothing committed: nothing changes
+    a.step()
+    tr = a.seqs[0].trace
+    assert tr["kind"] == "within" and tr["refresh"]
+    for l in range(m.n_layers):
+        assert not tr["D"][l].any() and len(tr["sel"][l]) == 0

@@ -376,3 +376,49 @@ def test_refresh_chain_rows_equal_full_recompute():
     # unchanged hidden row => unchanged K/V (Cor. 1 with dH = 0): refreshing twice changes nothing
     _, _, K3, V3 = O.refresh_chain(H, drift, k, wq, wk, wv, gain, 1e-5, theta, nh, nkv, dh, K2, V2, emulate_bf16=False)
     assert np.array_equal(K3, K2) and np.array_equal(V3, V2)
+
+
+# ---------------------------------------------------------------- centroid proxies (Sec. 4.1)
+def test_spherical_kmeans_pins():
+    # well separated directions are recovered whatever the rows' lengths (cosine similarity: "spherical")
+    d, K = 16, 4
+    dirs = np.linalg.qr(rng.standard_normal((d, d)))[0][:K]              # orthonormal centres
+    truth = np.array([0, 1, 2, 3] * 6)                                     # evenly spread, so every start row differs
+    H = dirs[truth] + 0.05 * rng.standard_normal((len(truth), d))
+    scale = 10.0 ** rng.uniform(-3, 3, size=(len(truth), 1))
+    lab = O.spherical_kmeans(H * scale, K, 4)
+    assert np.array_equal(lab, O.spherical_kmeans(H, K, 4))                # row scale does not matter
+    # same partition as the truth (cluster ids are a permutation)
+    assert len(set(zip(lab.tolist(), truth.tolist()))) == K
+    # no more rows than clusters: every row its own cluster
+    assert sorted(O.spherical_kmeans(H[:3], 8, 4).tolist()) == [0, 1, 2]
+    assert O.spherical_kmeans(np.zeros((0, d)), 8, 4).shape == (0,)
+    # brute force on random data: the returned labels are the nearest centres of the centres that the
+    # previous iteration produced, and the objective (sum of cosines to the own centre) never decreases
+    X = rng.standard_normal((40, 6))
+    U = X / np.linalg.norm(X, axis=1, keepdims=True)
+    Ke = 5
+    C = np.stack([U[int(np.floor((j + 0.5) * 40 / Ke))] for j in range(Ke)])
+    obj_prev = -np.inf
+    for it in range(1, 5):
+        lab_it = np.array([int(np.argmax([U[i] @ C[j] for j in range(Ke)])) for i in range(40)])
+        assert np.array_equal(lab_it, O.spherical_kmeans(X, Ke, it))
+        for j in range(Ke):
+            mem = U[lab_it == j]
+            if len(mem):
+                C[j] = mem.sum(0) / np.linalg.norm(mem.sum(0))
+        obj = sum(U[i] @ C[lab_it[i]] for i in range(40))
+        assert obj >= obj_prev - 1e-12
+        obj_prev = obj
+
+
+def test_cluster_proxies_pins():
+    H = rng.standard_normal((7, 5))
+    pos = np.array([3, 4, 5, 6, 20, 21, 22])
+    lab = np.array([0, 0, 2, 2, 2, 4, 0])
+    Z, zp, cnt = O.cluster_proxies(H, pos, lab, 6)
+    assert cnt.tolist() == [3, 0, 3, 0, 1, 0]
+    assert np.allclose(Z[0], (H[0] + H[1] + H[6]) / 3) and np.allclose(Z[2], H[2:5].mean(0))
+    assert np.array_equal(Z[4], H[5]) and zp[4] == 21                      # a cluster of one row is that row
+    assert zp[0] == int(np.floor((3 + 4 + 22) / 3 + 0.5)) and zp[2] == 10   # rounded mean position
+    assert not Z[1].any() and not Z[3].any()
