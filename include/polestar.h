@@ -79,6 +79,9 @@ extern "C" {
 #define POLESTAR_SELECT_THRESHOLD 2   /* drift > select_thresh                              */
 #define POLESTAR_SELECT_ALL 3         /* every window row (full refresh)                    */
 #define POLESTAR_SELECT_NONE 4        /* never refresh rows (drift still measured)          */
+#define POLESTAR_SELECT_CLUSTER_TOPK 5 /* centroid proxies (the paper's default policy): drift is measured on
+                                         n_clusters proxy rows per layer and the member rows of the cluster_k
+                                         clusters with the largest drift are refreshed                       */
 
 #define POLESTAR_FLAG_DRIFT_COMMIT  (1u << 0) /* drift-event clause of the commit rule (Sec. 4.2)  */
 #define POLESTAR_FLAG_SUFFIX_COMMIT (1u << 1) /* suffix-block commit from the final packet          */
@@ -142,6 +145,14 @@ typedef struct {
     int32_t tau_upd /*3; <0: refresh every step; INT32_MAX: never*/, hist /*5*/;
     float   tau_s /*0.9*/, alpha /*10*/, tau_suffix /*0.9*/, logit_scale /*1*/;
     uint32_t flags /*DRIFT_COMMIT|SUFFIX_COMMIT|GE_COMPARE*/;
+    /* Centroid proxies (Sec. 4.1 "Cluster and Quantize Hidden States", "Measuring Drift and Layer-wise KV
+     * Updates"; Sec. 5.1: K = 8, k = 4), used by POLESTAR_SELECT_CLUSTER_TOPK only.  What the paper leaves open is
+     * fixed as follows: spherical K-means of the window's layer-input hidden rows at every block entry, per layer,
+     * centre j starting at the unit vector of window row floor((j + 1/2) W / K), kmeans_iters Lloyd iterations
+     * (largest cosine, lowest cluster on ties; an empty cluster keeps its centre; no more rows than clusters:
+     * every row its own cluster); a cluster's proxy is the mean of its members' hidden rows, queried at the
+     * rounded mean of their positions, and follows its members when they are refreshed. */
+    int32_t n_clusters /*8; 1..16*/, cluster_k /*4*/, kmeans_iters /*4; 1..16*/;
 } polestar_params;
 
 typedef struct {
@@ -229,6 +240,10 @@ int polestar_tokens(polestar_ctx *c, int32_t *out_host);
 #define POLESTAR_READ_THETA_COUNT 18 /* int32 [batch] vectors pushed since the block was entered  */
 #define POLESTAR_READ_OWN_COMMIT 19  /* int32 [batch][block] the rule's own decision (bits as in
                                         READ_COMMIT), also when a forced decision replaced it    */
+#define POLESTAR_READ_LABELS     20  /* int32 [batch][W_max] cluster of every window row at `layer`
+                                        (centroid proxies; -1 beyond the window)                 */
+/* With POLESTAR_SELECT_CLUSTER_TOPK, READ_DRIFT holds the drift of the n_clusters proxies in its first
+ * n_clusters entries and READ_PPREV has the shape [batch][n_clusters][n_heads][N]. */
 /* Libraries built with -DPOLESTAR_TRACE only (time stamps, see csrc/common.cuh): */
 #define POLESTAR_READ_TRACE_KERNELS 98 /* int64 [8192]: next slot, then (kernel id, ns) pairs      */
 #define POLESTAR_READ_TRACE_GEMM 99  /* int64 [CTAs][12] stamps of the traced GEMM kind            */
@@ -246,6 +261,9 @@ int polestar_read(polestar_ctx *c, int32_t what, int32_t layer, void *dst_host, 
 #define POLESTAR_FORCE_TOKENS 4  /* after FORCE_COMMIT with the same n: token ids written at those
                                     positions ([batch][n]) instead of the library's own argmax (two
                                     near-equal logits may rank differently in another arithmetic)  */
+#define POLESTAR_FORCE_LABELS 5  /* centroid proxies: cluster labels of the window rows at `layer` for the next
+                                    block-entry forward, instead of the library's own K-means ([batch][n],
+                                    n = window rows; a near-tie between two centres may fall either way)  */
 int polestar_force(polestar_ctx *c, int32_t what, int32_t layer, const int32_t *idx_host, int32_t n);
 
 /* Per-family device time of the forwards so far (context created with POLESTAR_FLAG_PROFILE;

@@ -227,7 +227,9 @@ def spherical_kmeans(H: np.ndarray, K: int, iters: int) -> np.ndarray:
     C = np.stack([U[int(math.floor((j + 0.5) * W / Ke))] for j in range(Ke)])
     labels = np.zeros(W, np.int64)
     for _ in range(max(1, int(iters))):
-        sims = U @ C.T                                   # [W, Ke] cosines
+        # cosines [W, Ke], one centre at a time: coinciding centres (rows that are equal, e.g. still masked
+        # positions) then give bit-identical columns, so "lowest cluster id on ties" is well defined
+        sims = np.stack([U @ C[j] for j in range(Ke)], axis=1)
         labels = np.argmax(sims, axis=1)                 # first maximum: lowest cluster id on ties
         for j in range(Ke):
             mem = np.nonzero(labels == j)[0]

@@ -23,9 +23,9 @@ OK, E_INVAL, E_STATE, E_NOSPACE, E_CUDA, E_NONFINITE, E_TIMEOUT, E_DONE = 0, -1,
 
 READ_LOGITS, READ_CONF, READ_YHAT, READ_DELTA, READ_DRIFT, READ_SEL_COUNT, READ_SEL_IDX = 1, 2, 3, 4, 5, 6, 7
 READ_HIDDEN, READ_KCACHE, READ_VCACHE, READ_HCACHE, READ_COMMIT, READ_PPREV, READ_SUFFIX = 8, 9, 10, 11, 12, 13, 14
-READ_DRIFT_DELTA, READ_TAU_D, READ_THETA, READ_THETA_COUNT, READ_OWN_COMMIT = 15, 16, 17, 18, 19
+READ_DRIFT_DELTA, READ_TAU_D, READ_THETA, READ_THETA_COUNT, READ_OWN_COMMIT, READ_LABELS = 15, 16, 17, 18, 19, 20
 READ_TRACE_KERNELS, READ_TRACE_GEMM = 98, 99
-FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR, FORCE_TOKENS = 1, 2, 3, 4
+FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR, FORCE_TOKENS, FORCE_LABELS = 1, 2, 3, 4, 5
 FLAG_SIMT_GEMM, FLAG_PROMPT_DEVICE, FLAG_PROFILE = 1 << 5, 1 << 6, 1 << 7
 PROF_FAMILIES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head", "attention", "stage", "select",
                  "confidence", "commit", "misc"]
@@ -65,7 +65,8 @@ class CParams(C.Structure):
                 ("full_entry_period", C.c_int32), ("select_mode", C.c_int32), ("select_frac", C.c_float),
                 ("select_k", C.c_int32), ("select_thresh", C.c_float), ("drift_floor", C.c_float),
                 ("tau_upd", C.c_int32), ("hist", C.c_int32), ("tau_s", C.c_float), ("alpha", C.c_float),
-                ("tau_suffix", C.c_float), ("logit_scale", C.c_float), ("flags", C.c_uint32)]
+                ("tau_suffix", C.c_float), ("logit_scale", C.c_float), ("flags", C.c_uint32),
+                ("n_clusters", C.c_int32), ("cluster_k", C.c_int32), ("kmeans_iters", C.c_int32)]
 
 
 class CStepInfo(C.Structure):
@@ -159,7 +160,8 @@ def c_model(m: I.ModelCfg) -> CModel:
 def c_params(p: I.Params) -> CParams:
     return CParams(p.batch, p.prompt_len, p.gen_len, p.block, p.max_steps, p.win_prefix_blocks, p.win_suffix_blocks,
                    p.full_entry_period, p.select_mode, p.select_frac, p.select_k, p.select_thresh, p.drift_floor,
-                   p.tau_upd, p.hist, p.tau_s, p.alpha, p.tau_suffix, p.logit_scale, p.flags)
+                   p.tau_upd, p.hist, p.tau_s, p.alpha, p.tau_suffix, p.logit_scale, p.flags,
+                   p.n_clusters, p.cluster_k, p.kmeans_iters)
 
 
 def polestar_workspace_bytes(m: I.ModelCfg, p: I.Params) -> int:
@@ -314,7 +316,8 @@ class Polestar:
                   READ_SEL_IDX: ((bs, Wm), np.int32), READ_HIDDEN: ((bs, B, m.d_model), np.float32),
                   READ_KCACHE: ((bs, N, dkv), el), READ_VCACHE: ((bs, N, dkv), el),
                   READ_HCACHE: ((bs, Wm, m.d_model), np.float32), READ_COMMIT: ((bs, B), np.int32),
-                  READ_PPREV: ((bs, Wm, m.n_heads, N), np.float32), READ_SUFFIX: ((bs, Wm), np.int32),
+                  READ_PPREV: ((bs, p.n_clusters if p.select_mode == I.SELECT_CLUSTER_TOPK else Wm, m.n_heads, N), np.float32),
+                  READ_SUFFIX: ((bs, Wm), np.int32), READ_LABELS: ((bs, Wm), np.int32),
                   READ_DRIFT_DELTA: ((bs, B), np.float32), READ_TAU_D: ((bs, B), np.float32),
                   READ_THETA: ((bs, max(1, p.hist), B), np.float32), READ_THETA_COUNT: ((bs,), np.int32),
                   READ_OWN_COMMIT: ((bs, B), np.int32),
@@ -348,6 +351,10 @@ class Polestar:
             tok = np.ascontiguousarray(np.asarray(tokens, np.int32).reshape(self.p.batch, -1))
             _check(load().polestar_force(self.ctx, FORCE_TOKENS, 0, tok.ctypes.data_as(C.POINTER(C.c_int32)),
                                          tok.shape[1]))
+
+    def force_labels(self, layer: int, labels) -> None:
+        lab = np.ascontiguousarray(np.asarray(labels, np.int32).reshape(self.p.batch, -1))
+        _check(load().polestar_force(self.ctx, FORCE_LABELS, layer, lab.ctypes.data_as(C.POINTER(C.c_int32)), lab.shape[1]))
 
     def force_clear(self) -> None:
         _check(load().polestar_force(self.ctx, FORCE_CLEAR, 0, None, 0))

@@ -298,8 +298,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     const int4 rw = __ldg(reinterpret_cast<const int4*>(a.rows) + r);      // {seq, pos, widx, aidx}
                     if (rw.y >= 0) {
                         valid = 1;
-                        if (rw.z >= 0 && a.pprev) {
-                            const size_t i = ((size_t)rw.x * a.W_max + rw.z) * a.n_heads + h;
+                        if (a.cluster_K > 0 ? (row_is_proxy(rw.z) && a.pprev != nullptr) : (rw.z >= 0 && a.pprev != nullptr)) {
+                            // recorded drift rows: the window rows, or (centroid proxies) the clusters' proxy rows
+                            const size_t i = a.cluster_K > 0 ? ((size_t)rw.x * a.cluster_K + row_cluster(rw.z)) * a.n_heads + h
+                                                             : ((size_t)rw.x * a.W_max + rw.z) * a.n_heads + h;
                             prev = a.pprev + i * a.N; lsep = a.pprev_lse + i;
                         } else if (rw.w >= 0 && a.aprev) {
                             const size_t i = ((size_t)rw.x * a.B + rw.w) * a.n_heads + h;

@@ -86,9 +86,14 @@ __device__ __forceinline__ void trace_stamp(int, int = 0) {}
 struct Row {
     int seq;   // sequence in the batch
     int pos;   // absolute position in the sequence, -1 = unused
-    int widx;  // index in the local window, -1 = not a window row
+    int widx;  // index in the local window, -1 = not a window row; <= -2: proxy row of cluster -2 - widx
     int aidx;  // index in the active block, -1 = not an active row
 };
+// Proxy rows (centroid proxies, Sec. 4.1 "Cluster and Quantize Hidden States") follow the ordinary rows of a
+// sequence.  Their rotary position and emptiness differ from layer to layer (the clustering is per layer), so the
+// row table only marks them; kernels look both up in the layer's cluster tables.
+__device__ __forceinline__ bool row_is_proxy(int widx) { return widx <= -2; }
+__device__ __forceinline__ int row_cluster(int widx) { return -2 - widx; }
 
 struct SeqFlags { unsigned char v[64]; };
 
@@ -105,6 +110,7 @@ struct StepDesc {
     int e0;            // entry steps: first forwarded position
     int within;        // 1: window rows live in the hidden cache (within-block step)
     int record_kl;     // 1: drift of recorded rows is measured against the stored rows
+    int K;             // centroid proxies per sequence appended to the rows (0: per-position drift)
     SeqFlags refresh;  // within-block: which sequences refresh their cache this step
 };
 
@@ -210,6 +216,8 @@ struct EpiArgs {
     float scale;              // LOGITS
     // QKV_REFRESH (stand-alone refresh kernel): row r of sequence s = r / max_rows
     const int* idx; const int* counts; int max_rows; int P;
+    // QKV with proxy rows: rotary position of cluster c of sequence s at zpos[s * n_clusters + c] (< 0: empty cluster)
+    const int* zpos; int n_clusters;
     // RMSNorm folded into two GEMMs (steps whose rows all come straight from the previous GEMM): the producing
     // epilogue (RESID / DOWN) also stores a = x * gain in the model dtype and adds the row's sum of squares to
     // fold_ss (64-bit fixed point, 2^16: integer additions commute, so the sum is reproducible); the consuming
@@ -235,6 +243,17 @@ __device__ __forceinline__ float fold_inv(const EpiArgs& e, int m) {
     return rsqrtf(ss / (float)e.in_d + e.in_eps);
 }
 
+// Cluster tables of ONE layer (centroid proxies; all null / 0 in the per-position mode).
+struct ClusterTabs {
+    const int* labels;     // [batch][W_max] cluster of every window row
+    const int* zpos;       // [batch][K] rotary position of the proxy (rounded mean of the members' positions), -1 = empty
+    const int* zcnt;       // [batch][K] members
+    const int* members;    // [batch][W_max] window indices grouped by cluster, ascending inside a cluster
+    const int* moff;       // [batch][K + 1] start of every cluster's group
+    float* zbuf;           // [batch][K][d] the proxy rows (member means), rebuilt whenever they are needed
+    int K;
+};
+
 // Row-wise work appended to a GEMM whose output rows are the input of the next normalisation: once every CTA
 // of the grid has stored its outputs (a counter all CTAs add to), the CTAs share out the rows and stage the
 // next GEMM's operand, which saves a kernel boundary per normalisation.
@@ -249,6 +268,7 @@ struct PostArgs {
     const int* list; const int* m_count;       // kind 1
     const Row* rows; float* hc; const float* packet; const unsigned char* patch; unsigned char* kvflag;   // kind 2
     StepDesc sd;                               // kind 2
+    ClusterTabs ct;                            // kind 2: cluster tables of the layer being staged
     unsigned* counter;                         // never reset: `expect` is the running total after this launch
     unsigned expect;
 };
@@ -262,6 +282,7 @@ __device__ __forceinline__ void epilogue_pair(const EpiArgs& e, int m, int n, fl
             const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + m);   // {seq, pos, widx, aidx}
             if (rw.y < 0) return;
             seq = rw.x; pos = rw.y; kvf = __ldg(e.kvflag + m); qrow = m;
+            if (row_is_proxy(rw.z)) { pos = __ldg(e.zpos + seq * e.n_clusters + row_cluster(rw.z)); kvf = 0; if (pos < 0) return; }
         } else {
             seq = m / e.max_rows;
             const int i = m - seq * e.max_rows;
@@ -374,6 +395,7 @@ __device__ __forceinline__ void epilogue16(const EpiArgs& e, int m, int n, const
             const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + m);   // {seq, pos, widx, aidx}
             if (rw.y < 0) return;
             seq = rw.x; pos = rw.y; kvf = __ldg(e.kvflag + m);
+            if (row_is_proxy(rw.z)) { pos = __ldg(e.zpos + seq * e.n_clusters + row_cluster(rw.z)); kvf = 0; if (pos < 0) return; }
         } else {
             seq = m / e.max_rows;
             const int i = m - seq * e.max_rows;

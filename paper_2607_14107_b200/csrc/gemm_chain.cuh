@@ -469,7 +469,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                         prep_rows_row<T>(r, P.post.x, P.post.list, P.post.m_count, P.post.gain, P.post.eps, P.post.d, (T*)P.post.a_out, post_red);
                     else
                         prep_qkv_row<T>(P.post.sd, r, P.post.rows, P.post.x, P.post.hc, P.post.packet, P.post.patch, P.post.gain,
-                                        P.post.eps, P.post.d, (T*)P.post.a_out, P.post.kvflag, post_red);
+                                        P.post.eps, P.post.d, (T*)P.post.a_out, P.post.kvflag, post_red, P.post.ct);
                 }
             }
             arrive();

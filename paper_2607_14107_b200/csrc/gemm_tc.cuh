@@ -667,7 +667,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             prep_rows_row<T>(r, post.x, post.list, post.m_count, post.gain, post.eps, post.d, (T*)post.a_out, post_red);
                         else
                             prep_qkv_row<T>(post.sd, r, post.rows, post.x, post.hc, post.packet, post.patch, post.gain, post.eps,
-                                            post.d, (T*)post.a_out, post.kvflag, post_red);
+                                            post.d, (T*)post.a_out, post.kvflag, post_red, post.ct);
                     }
                 }
             }

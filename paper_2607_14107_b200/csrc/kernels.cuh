@@ -17,7 +17,11 @@ __global__ void build_rows_kernel(StepDesc sd, Row* rows) {
     const int s = i / sd.rows_per_seq, j = i - s * sd.rows_per_seq;
     Row r;
     r.seq = s; r.pos = -1; r.widx = -1; r.aidx = -1;
-    if (sd.kind == 2) {
+    const int n_plain = sd.rows_per_seq - sd.K;      // the proxy rows of the clusters come last
+    if (j >= n_plain) {
+        // proxy row: position and emptiness are per layer (cluster tables); unused on steps without refresh
+        if (sd.kind != 2 || sd.refresh.v[s]) { r.pos = 0; r.widx = -2 - (j - n_plain); }
+    } else if (sd.kind == 2) {
         if (j < sd.B) {
             r.pos = sd.act_start + j; r.aidx = j;
         } else {
@@ -46,7 +50,7 @@ __global__ void embed_rows_kernel(StepDesc sd, const Row* rows, const int* y, co
     KERNEL_PROLOGUE(2);   // embed_rows_kernel
     const int r = blockIdx.x;
     const Row rw = rows[r];
-    if (rw.pos < 0) return;
+    if (rw.pos < 0 || row_is_proxy(rw.widx)) return;
     const int tok = y[rw.seq * sd.N + rw.pos];
     const T* e = emb + (size_t)tok * d;
     if (sd.within && rw.widx >= 0) {
@@ -132,12 +136,40 @@ __device__ __forceinline__ void zero_row(T* a, int d) {
 template <typename T>
 __device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Row* rows, float* x, float* hc, const float* packet,
                                              const unsigned char* patch, const float* gain, float eps, int d,
-                                             T* a_out, unsigned char* kvflag, float* red) {
+                                             T* a_out, unsigned char* kvflag, float* red, const ClusterTabs& ct) {
     const Row rw = rows[r];
     T* a = a_out + (size_t)r * d;
     if (rw.pos < 0) {
         zero_row<T>(a, d);
         if (threadIdx.x == 0) kvflag[r] = 0;
+        return;
+    }
+    if (row_is_proxy(rw.widx)) {
+        // Proxy of a cluster = mean of its members' current hidden rows (Sec. 4.1: the centroid follows its refreshed
+        // members; rebuilding the mean from the cache is that incremental update without its rounding drift).
+        // Members are added in ascending window order by every thread for its own columns: deterministic.
+        const int c = row_cluster(rw.widx);
+        const int n = ct.zcnt[rw.seq * ct.K + c];
+        if (threadIdx.x == 0) kvflag[r] = 0;
+        if (n <= 0) { zero_row<T>(a, d); return; }
+        const int* mem = ct.members + (size_t)rw.seq * sd.W_max + ct.moff[rw.seq * (ct.K + 1) + c];
+        float* z = ct.zbuf + ((size_t)rw.seq * ct.K + c) * d;
+        const float inv_n = 1.f / (float)n;
+        for (int c4 = threadIdx.x; c4 < (d >> 2); c4 += blockDim.x) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int t = 0; t < n; ++t) {
+                const int w = mem[t];
+                const size_t o = (size_t)rw.seq * sd.W_max + w;
+                const float* src;
+                if (sd.within) src = patch[o] ? packet + o * d : hc + o * d;
+                else src = x + ((size_t)rw.seq * sd.rows_per_seq + (window_pos(sd, w) - sd.e0)) * d;      // entry: this forward's row
+                const float4 v = __ldcg(reinterpret_cast<const float4*>(src) + c4);
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            reinterpret_cast<float4*>(z)[c4] = make_float4(acc.x * inv_n, acc.y * inv_n, acc.z * inv_n, acc.w * inv_n);
+        }
+        __syncthreads();
+        norm_row<T>(z, gain, eps, d, a, nullptr, nullptr, red);
         return;
     }
     float* xr = x + (size_t)r * d;
@@ -162,10 +194,10 @@ __device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Ro
 template <typename T>
 __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* hc, const float* packet,
                                 const unsigned char* patch, const float* gain, float eps, int d,
-                                T* a_out, unsigned char* kvflag) {
+                                T* a_out, unsigned char* kvflag, ClusterTabs ct) {
     KERNEL_PROLOGUE(3);   // prep_qkv_kernel
     __shared__ float red[33];
-    prep_qkv_row<T>(sd, blockIdx.x, rows, x, hc, packet, patch, gain, eps, d, a_out, kvflag, red);
+    prep_qkv_row<T>(sd, blockIdx.x, rows, x, hc, packet, patch, gain, eps, d, a_out, kvflag, red, ct);
 }
 
 // RMSNorm of a compacted list of rows (FFN input, LM-head input).
@@ -225,6 +257,127 @@ __global__ void prep_refresh_kernel(const T* h, const int* idx, const int* count
     ss = block_sum(ss, red);
     const float inv = rsqrtf(ss / (float)d + eps);
     for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(to_f<T>(src[c]) * inv * gain[c]);
+}
+
+// ---------------------------------------------------------------------------------------
+// Spherical K-means of the window's hidden rows at block entry (Sec. 4.1 "Cluster and Quantize Hidden States";
+// Algorithm 1 "SphericalKMeans"), one CTA per sequence, and the cluster tables that follow from the labels.
+// Deterministic reading: centre j starts at the unit vector of window row floor((j + 1/2) W / K); `iters` Lloyd
+// iterations (assign to the largest cosine, lowest cluster on ties; centre = normalised sum of the members' unit
+// vectors, an empty cluster keeps its centre); no more rows than clusters: every row its own cluster.
+// All sums run in a fixed order.  K <= KM_MAX_K, W <= KM_MAX_W.
+// ---------------------------------------------------------------------------------------
+constexpr int KM_MAX_K = 16, KM_MAX_W = 1024, KM_THREADS = 512;
+struct KmeansArgs {
+    const float* x;            // entry forward: residual-stream rows of this layer [rows][d]
+    int d, K, iters;
+    int* labels; int* zpos; int* zcnt; int* members; int* moff;      // this layer's tables (see ClusterTabs)
+    const int* forced_labels;  // [batch][W_max], first entry < 0: not forced (parity replay of another clustering)
+    float* cent;               // scratch [batch][2][K][d]: the centres, and the member sums of the running update
+};
+__global__ void __launch_bounds__(KM_THREADS) kmeans_kernel(StepDesc sd, KmeansArgs a) {
+    KERNEL_PROLOGUE(18);   // kmeans_kernel
+    __shared__ float inv_norm[KM_MAX_W];
+    __shared__ int lab[KM_MAX_W];
+    __shared__ float red[33];
+    __shared__ int cnt[KM_MAX_K + 1];
+    const int s = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5, nw = KM_THREADS / 32;
+    const int W = sd.W, K = a.K, d = a.d;
+    auto row = [&](int w) { return a.x + ((size_t)s * sd.rows_per_seq + (window_pos(sd, w) - sd.e0)) * d; };
+    float* C = a.cent + (size_t)s * 2 * K * d;
+    float* Cn = C + (size_t)K * d;
+    const int* forced = a.forced_labels ? a.forced_labels + (size_t)s * sd.W_max : nullptr;
+    if (forced && forced[0] >= 0) {
+        for (int w = t; w < W; w += KM_THREADS) lab[w] = min(max(forced[w], 0), K - 1);
+    } else if (W <= K) {
+        for (int w = t; w < W; w += KM_THREADS) lab[w] = w;
+    } else {
+        for (int w = warp; w < W; w += nw) {
+            float ss = 0.f;
+            const float* h = row(w);
+            for (int c = lane; c < d; c += 32) { const float v = h[c]; ss = fmaf(v, v, ss); }
+            ss = warp_sum(ss);
+            if (lane == 0) inv_norm[w] = ss > 0.f ? rsqrtf(ss) : 0.f;
+        }
+        __syncthreads();
+        for (int j = 0; j < K; ++j) {
+            const int w0 = (int)(((2 * j + 1) * (long long)W) / (2 * K));       // floor((j + 1/2) W / K)
+            const float* h = row(w0);
+            const float inv = inv_norm[w0];
+            for (int c = t; c < d; c += KM_THREADS) C[(size_t)j * d + c] = h[c] * inv;
+        }
+        __syncthreads();
+        for (int it = 0; it < a.iters; ++it) {
+            // assignment: a warp per row, the row's dot product with every centre
+            for (int w = warp; w < W; w += nw) {
+                const float* h = row(w);
+                float best = -INFINITY;
+                int bj = 0;
+                for (int j = 0; j < K; ++j) {
+                    const float* cj = C + (size_t)j * d;
+                    float dot = 0.f;
+                    for (int c = lane; c < d; c += 32) dot = fmaf(h[c], cj[c], dot);
+                    dot = warp_sum(dot) * inv_norm[w];
+                    if (dot > best) { best = dot; bj = j; }
+                }
+                if (lane == 0) lab[w] = bj;
+            }
+            __syncthreads();
+            if (it + 1 == a.iters) break;          // the centres of the last update are never used
+            // update: every thread owns columns; members are added in ascending row order
+            if (t <= K) cnt[t] = 0;
+            __syncthreads();
+            if (t < K) { int n = 0; for (int w = 0; w < W; ++w) n += lab[w] == t; cnt[t] = n; }
+            __syncthreads();
+            float ssq[KM_MAX_K];
+#pragma unroll
+            for (int j = 0; j < KM_MAX_K; ++j) ssq[j] = 0.f;
+            for (int c = t; c < d; c += KM_THREADS) {
+                float acc[KM_MAX_K];
+#pragma unroll
+                for (int j = 0; j < KM_MAX_K; ++j) acc[j] = 0.f;
+                for (int w = 0; w < W; ++w) {
+                    const float v = row(w)[c] * inv_norm[w];
+                    const int lw = lab[w];
+#pragma unroll
+                    for (int j = 0; j < KM_MAX_K; ++j) acc[j] += (lw == j) ? v : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < KM_MAX_K; ++j)
+                    if (j < K && cnt[j] > 0) { Cn[(size_t)j * d + c] = acc[j]; ssq[j] = fmaf(acc[j], acc[j], ssq[j]); }
+            }
+            for (int j = 0; j < K; ++j) {
+                const float n2 = block_sum(ssq[j], red);
+                if (cnt[j] > 0 && n2 > 0.f) {        // (an empty cluster, or one whose unit vectors cancel, keeps its centre)
+                    const float inv = rsqrtf(n2);
+                    for (int c = t; c < d; c += KM_THREADS) C[(size_t)j * d + c] = Cn[(size_t)j * d + c] * inv;
+                }
+            }
+            __syncthreads();
+        }
+    }
+    __syncthreads();
+    // tables: labels, member counts, groups of members, rotary position of every proxy
+    for (int w = t; w < sd.W_max; w += KM_THREADS) a.labels[(size_t)s * sd.W_max + w] = w < W ? lab[w] : -1;
+    if (t < K) {
+        int n = 0;
+        long long sp = 0;
+        for (int w = 0; w < W; ++w) if (lab[w] == t) { ++n; sp += window_pos(sd, w); }
+        cnt[t] = n;
+        a.zcnt[s * K + t] = n;
+        a.zpos[s * K + t] = n > 0 ? (int)((2 * sp + n) / (2 * n)) : -1;       // floor(mean + 1/2)
+    }
+    __syncthreads();
+    if (t == 0) {
+        int off = 0;
+        for (int j = 0; j < K; ++j) { a.moff[s * (K + 1) + j] = off; off += cnt[j]; }
+        a.moff[s * (K + 1) + K] = off;
+    }
+    __syncthreads();
+    if (t < K) {
+        int o = a.moff[s * (K + 1) + t];
+        for (int w = 0; w < W; ++w) if (lab[w] == t) a.members[(size_t)s * sd.W_max + o++] = w;
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -302,6 +455,8 @@ struct AttnArgs {
     int N, n_heads, n_kv, head_dim, W_max, B, record_kl;
     int rows_per_seq, batch;   // layout of the forward's rows (stand-alone: n_rows, 1)
     float scale;
+    int cluster_K;             // > 0: centroid proxies: pprev / pprev_lse hold [batch][cluster_K] proxy rows per head and
+                               // window rows are not recorded
     int dirty_lo, dirty_hi;    // key positions [lo, hi) of every sequence that the kernel running just before may have
                                // written; all other K/V rows were complete before this forward was launched
     // stand-alone form: rows == null, row r belongs to sequence 0 and records into pprev[r]
@@ -320,7 +475,11 @@ __global__ void attention_simt_kernel(AttnArgs a) {
         const Row rw = a.rows[r];
         if (rw.pos < 0) return;
         seq = rw.seq;
-        if (rw.widx >= 0 && a.pprev) prev = a.pprev + (((size_t)seq * a.W_max + rw.widx) * a.n_heads + h) * a.N;
+        if (a.cluster_K > 0) {
+            if (row_is_proxy(rw.widx) && a.pprev) prev = a.pprev + (((size_t)seq * a.cluster_K + row_cluster(rw.widx)) * a.n_heads + h) * a.N;
+            else if (rw.aidx >= 0 && a.aprev) prev = a.aprev + (((size_t)seq * a.B + rw.aidx) * a.n_heads + h) * a.N;
+        }
+        else if (rw.widx >= 0 && a.pprev) prev = a.pprev + (((size_t)seq * a.W_max + rw.widx) * a.n_heads + h) * a.N;
         else if (rw.aidx >= 0 && a.aprev) prev = a.aprev + (((size_t)seq * a.B + rw.aidx) * a.n_heads + h) * a.N;
     } else if (a.pprev) {
         prev = a.pprev + ((size_t)r * a.n_heads + h) * a.N;
@@ -568,6 +727,8 @@ struct StepSelArgs {
     int* stats;                 // [0] += refreshed rows
     int n_heads, mode, k, W_max;
     float thresh, floor_;
+    ClusterTabs ct;             // centroid proxies (ct.K > 0): drift per cluster, the top cluster_k clusters' members
+    int cluster_k;
 };
 
 // The same work for a batch of one sequence with a window of at most SEL_SMALL_W rows, done by `nthr` >= W threads
@@ -629,7 +790,41 @@ __global__ void __launch_bounds__(SEL_THREADS) step_select_kernel(StepDesc sd, S
     const int t = threadIdx.x;
     const int sq = blockIdx.x;
     int cnt = 0;
-    if (sd.refresh.v[sq]) {
+    if (sd.refresh.v[sq] && a.ct.K > 0) {
+        // ---- centroid proxies (Sec. 4.1; Algorithm 1 "KL", "TopK", M[K]): drift of the K proxy rows, the
+        // cluster_k clusters with the largest drift, then their member rows in ascending order
+        __shared__ int csel[KM_MAX_K], ctmp[KM_MAX_K];
+        const int K = a.ct.K;
+        if (t < K) {
+            const float* kr = a.kl + (size_t)(sq * sd.rows_per_seq + sd.B + sd.W + t) * a.n_heads;
+            float acc = 0.f;
+            for (int h = 0; h < a.n_heads; ++h) acc += __ldg(kr + h);
+            const float dv = a.ct.zcnt[sq * K + t] > 0 ? acc / (float)a.n_heads : 0.f;       // an empty cluster never drifts
+            dsh[t] = dv;
+            a.drift[sq * a.W_max + t] = dv;
+        }
+        __syncthreads();
+        int* idx = a.sel_idx + sq * a.W_max;
+        unsigned char* fl = a.flag_next + sq * a.W_max;
+        const int fc = a.forced_cnt ? a.forced_cnt[sq] : -1;
+        if (fc >= 0) {
+            for (int w = t; w < sd.W; w += blockDim.x) fl[w] = 0;
+            __syncthreads();
+            for (int i = t; i < fc; i += blockDim.x) { const int w = a.forced_idx[sq * a.W_max + i]; idx[i] = w; fl[w] = 1; }
+            cnt = fc;
+        } else {
+            select_small(dsh, K, 1 /* top-k count */, a.cluster_k, a.thresh, a.floor_, ctmp, nullptr, sel_sh);
+            if (t < K) csel[t] = sel_sh[t];
+            __syncthreads();
+            const bool sel = t < sd.W && csel[a.ct.labels[(size_t)sq * a.W_max + t]] != 0;
+            if (t < SEL_SMALL_W) sel_sh[t] = sel ? 1 : 0;
+            __syncthreads();
+            int pos = 0, total = 0;
+            for (int j = 0; j < sd.W; ++j) { const int f = sel_sh[j]; total += f; pos += (j < t) ? f : 0; }
+            if (t < sd.W) { fl[t] = sel ? 1 : 0; if (sel) idx[pos] = t; }
+            cnt = total;
+        }
+    } else if (sd.refresh.v[sq]) {
         // head mean of the per-head drift (Eq. 4): eight lanes per row, all loads of a row in flight at once;
         // the partial sums are combined in a fixed order
         for (int w0 = 0; w0 < sd.W; w0 += blockDim.x / 8) {

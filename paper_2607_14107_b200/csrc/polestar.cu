@@ -326,6 +326,7 @@ struct Buffers {
     int* forced_commit; int* forced_tok; float* conf; int* yhat; float* delta; float* Delta; float* taud; int* commit_flags;
     int* own_flags; int* suffix_flags; int* seq_info; int* head_count; int* suf_seq; int* suf_w; int* stats; int* status;
     int* list_count; float* hidden_keep;
+    int* labels; int* zpos; int* zcnt; int* members; int* moff; int* forced_labels; float* zbuf; float* kcent;   // centroid proxies
     // scratch
     Row* rows; unsigned char* kvflag; float* x; float* x1; float* packet; char* a_buf; char* q_buf; char* o_buf;
     char* g_buf; float* kl; int* list; long long* fold_ss; HeadSrc* head_list; char* a_head; float* logits; ConfPart* conf_part;
@@ -417,7 +418,7 @@ struct polestar_ctx {
     std::vector<int> cum;
     StepDesc last_sd;
     int last_act_row_off = 0;
-    bool forced_select = false, forced_commit = false, forced_tokens = false;
+    bool forced_select = false, forced_commit = false, forced_tokens = false, forced_labels = false;
     int forced_commit_n = 0;
     int* seq_info_host = nullptr;          // pinned: bs * 8 + 8 words
     // launch accounting and optional per-family device timing (POLESTAR_FLAG_PROFILE)
@@ -467,12 +468,22 @@ static bool valid_cfg(const polestar_model* m, const polestar_params* p) {
     if (p->prompt_len < 0 || p->gen_len <= 0 || p->block <= 0 || p->block > 256) return false;
     if (p->gen_len % p->block) return false;
     if (p->max_steps <= 0 || p->win_prefix_blocks < 0 || p->win_suffix_blocks < 0 || p->full_entry_period <= 0) return false;
-    if (p->select_mode < 0 || p->select_mode > 4 || p->hist < 0 || p->hist > 64) return false;
+    if (p->select_mode < 0 || p->select_mode > POLESTAR_SELECT_CLUSTER_TOPK || p->hist < 0 || p->hist > 64) return false;
     const long long N = (long long)p->prompt_len + p->gen_len;
     if (N > 65536) return false;
     const long long wmax = std::min<long long>((long long)(p->win_prefix_blocks + p->win_suffix_blocks) * p->block, N - p->block);
     if (wmax > 1024) return false;
+    if (p->select_mode == POLESTAR_SELECT_CLUSTER_TOPK) {
+        // proxies ride behind the window rows; their drift shares the window's drift row; selection by rank counting
+        if (p->n_clusters < 1 || p->n_clusters > KM_MAX_K || p->cluster_k < 0 || p->kmeans_iters < 1 || p->kmeans_iters > 16) return false;
+        if (wmax > SEL_SMALL_W || p->n_clusters > std::max<long long>(wmax, 1) || m->d_model % 4) return false;
+    }
     return true;
+}
+
+// proxy rows per sequence (the full-recompute baseline has no cache to calibrate, hence no proxies)
+static int n_proxies(const polestar_params* p) {
+    return (p->select_mode == POLESTAR_SELECT_CLUSTER_TOPK && !(p->flags & POLESTAR_FLAG_NOCACHE)) ? p->n_clusters : 0;
 }
 
 static int window_max(const polestar_params* p) {
@@ -489,7 +500,9 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     const size_t F = m->d_ffn, V = m->vocab, nh = m->n_heads;
     const size_t Wm = window_max(p);
     const size_t n_suf = std::min<size_t>((size_t)p->win_suffix_blocks * B, Wm);
-    const size_t Mmax = bs * std::max(N, B + Wm);
+    const size_t Kp = n_proxies(p);                    // proxy rows per sequence (centroid proxies)
+    const size_t rec = Kp ? Kp : Wm;                   // recorded drift rows per sequence and layer
+    const size_t Mmax = bs * (std::max(N, B + Wm) + Kp);
     const size_t rows_lm = bs * (B + n_suf);
 #define TAKE(field, type, count)                                  \
     do {                                                          \
@@ -501,9 +514,9 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(kc, char, L * bs * N * dkv * es);
     TAKE(vc, char, L * bs * N * dkv * es);
     TAKE(hc, float, L * bs * Wm * d);
-    TAKE(pprev, float, L * bs * Wm * nh * N);
+    TAKE(pprev, float, L * bs * rec * nh * N);
     TAKE(aprev, float, bs * B * nh * N);
-    TAKE(pprev_lse, float, L * bs * Wm * nh);
+    TAKE(pprev_lse, float, L * bs * rec * nh);
     TAKE(aprev_lse, float, bs * B * nh);
     TAKE(theta, float, bs * std::max<size_t>(1, p->hist) * B);
     TAKE(theta_cnt, int, bs);
@@ -532,6 +545,14 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(status, int, 1);
     TAKE(list_count, int, 1);
     TAKE(hidden_keep, float, (p->flags & POLESTAR_FLAG_KEEP_HIDDEN) ? (L + 1) * bs * B * d : 1);
+    TAKE(labels, int, Kp ? L * bs * Wm : 1);
+    TAKE(zpos, int, Kp ? L * bs * Kp : 1);
+    TAKE(zcnt, int, Kp ? L * bs * Kp : 1);
+    TAKE(members, int, Kp ? L * bs * Wm : 1);
+    TAKE(moff, int, Kp ? L * bs * (Kp + 1) : 1);
+    TAKE(forced_labels, int, Kp ? L * bs * Wm : 1);
+    TAKE(zbuf, float, Kp ? bs * Kp * d : 1);
+    TAKE(kcent, float, Kp ? bs * 2 * Kp * d : 1);
     TAKE(rows, Row, Mmax);
     TAKE(kvflag, unsigned char, Mmax);
     TAKE(x, float, Mmax * d);
@@ -640,9 +661,11 @@ struct Path {
             const bool few_rows = !records && a.rows_per_seq <= 64 && a.N <= 1024 && c->sw.attn_kernel == 0;
             if ((c->sw.attn_kernel == 0 || c->sw.attn_kernel == 8) && attention_tc_applies(a) && !few_rows)
                 return launch_attention_tc(c->maps, a, c->st, c->b.status);
+            if (a.cluster_K > 0 && (a.pprev || a.aprev)) goto simt;      // the warp-level kernels do not know proxy rows
             CK(launch_attention_mma(a, c->st, c->sms, c->sw.attn_kernel));
             return POLESTAR_OK;
         }
+    simt:
         const int wpb = 4;
         const size_t smem = (size_t)wpb * a.N * sizeof(float);
         if (smem > SIMT_ATTN_SMEM_MAX) return POLESTAR_E_INVAL;
@@ -694,6 +717,24 @@ struct Path {
             float* hc = b.hc + (size_t)l * bs * Wm * d;
             float* pprev = b.pprev + (size_t)l * bs * Wm * m.n_heads * N;
             const bool last = l == L - 1;
+            // centroid proxies: this layer's cluster tables; at block entry they are made here, from the layer's input rows
+            ClusterTabs ct;
+            memset(&ct, 0, sizeof(ct));
+            const int Kp = sd.K;
+            if (Kp > 0) {
+                ct.labels = b.labels + (size_t)l * bs * Wm; ct.zpos = b.zpos + (size_t)l * bs * Kp; ct.zcnt = b.zcnt + (size_t)l * bs * Kp;
+                ct.members = b.members + (size_t)l * bs * Wm; ct.moff = b.moff + (size_t)l * bs * (Kp + 1); ct.zbuf = b.zbuf; ct.K = Kp;
+                if (!within) {
+                    Scope sc(c, POLESTAR_PROF_SELECT, (double)bs * sd.W * d * 4 * 2 * p.kmeans_iters, 0, 1);
+                    KmeansArgs ka;
+                    memset(&ka, 0, sizeof(ka));
+                    ka.x = b.x; ka.d = d; ka.K = Kp; ka.iters = p.kmeans_iters;
+                    ka.labels = b.labels + (size_t)l * bs * Wm; ka.zpos = b.zpos + (size_t)l * bs * Kp; ka.zcnt = b.zcnt + (size_t)l * bs * Kp;
+                    ka.members = b.members + (size_t)l * bs * Wm; ka.moff = b.moff + (size_t)l * bs * (Kp + 1);
+                    ka.forced_labels = b.forced_labels + (size_t)l * bs * Wm; ka.cent = b.kcent;
+                    CK(launch_k(kmeans_kernel, dim3(bs), dim3(KM_THREADS), 0, st, sd, ka));
+                }
+            }
             if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
                 Scope sc(c, POLESTAR_PROF_MISC, 0, 0, 1);
                 CK(launch_k(keep_hidden_kernel, dim3(bs * B), dim3(256), 0, st, sd, b.x, act_off, d, b.hidden_keep + (size_t)l * bs * B * d));
@@ -702,7 +743,7 @@ struct Path {
             if (!qkv_done && !qkv_staged) {      // (else: staged by the previous layer's down projection or chained kernel)
                 Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
                 CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
-                                                     c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag));
+                                                     c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag, ct));
                 CK(cudaGetLastError());
             }
             qkv_staged = false;
@@ -714,13 +755,14 @@ struct Path {
                 e.rows = b.rows; e.kvflag = b.kvflag; e.rope = b.rope; e.q_out = b.q_buf; e.kc = kc; e.vc = vc;
                 e.N_seq = N; e.n_heads = m.n_heads; e.n_kv = m.n_kv_heads; e.head_dim = m.head_dim; e.W_max = Wm;
                 e.within = within; e.ld_out = dq;
+                e.zpos = ct.zpos; e.n_clusters = Kp;
                 if (fold && l > 0) { e.in_ss = b.fold_ss + (size_t)(2 * l) * Mm; e.in_eps = m.rms_eps; e.in_d = d; }
                 if ((rc = gemm<EPI_QKV>(c, b.a_buf, c->wqkv[l], M, dq + 2 * dkv, d, e))) return rc;
             }
             qkv_done = false;
             {
                 const bool rec_w = sparse || !within;
-                const double rec_rows = (rec_w ? (double)bs * sd.W : 0.0) + (last ? (double)bs * B : 0.0);
+                const double rec_rows = (rec_w ? (double)bs * (Kp ? Kp : sd.W) : 0.0) + (last ? (double)bs * B : 0.0);
                 Scope sc(c, POLESTAR_PROF_ATTENTION,
                          2.0 * bs * N * dkv * esd + 2.0 * M * dq * esd + (sd.record_kl ? 2.0 : 1.0) * rec_rows * m.n_heads * N * 4,
                          4.0 * M * (double)N * dq, 1);
@@ -729,7 +771,13 @@ struct Path {
                 a.rows = b.rows; a.n_rows = M; a.q = b.q_buf; a.kc = kc; a.vc = vc; a.out = b.o_buf;
                 a.pprev = rec_w ? pprev : nullptr;
                 a.aprev = last ? b.aprev : nullptr;
-                a.pprev_lse = b.pprev_lse + (size_t)l * bs * Wm * m.n_heads;
+                if (Kp > 0 || n_proxies(&p) > 0) {
+                    // centroid proxies: [batch][K] recorded rows per layer (a step without refresh records none)
+                    const size_t Kall = (size_t)n_proxies(&p);
+                    a.pprev = rec_w ? b.pprev + (size_t)l * bs * Kall * m.n_heads * N : nullptr;
+                    a.cluster_K = (int)Kall;
+                }
+                a.pprev_lse = b.pprev_lse + (size_t)l * bs * (n_proxies(&p) ? (size_t)n_proxies(&p) : (size_t)Wm) * m.n_heads;
                 a.aprev_lse = b.aprev_lse;
                 a.kl = b.kl; a.N = N; a.n_heads = m.n_heads; a.n_kv = m.n_kv_heads; a.head_dim = m.head_dim;
                 a.W_max = Wm; a.B = B; a.record_kl = sd.record_kl; a.rows_per_seq = sd.rows_per_seq; a.batch = bs;
@@ -748,7 +796,7 @@ struct Path {
             // One sequence with a small window on the tensor-core path: the selection rides on the O projection
             // (idle warps of its first CTA), off the critical path; otherwise it is a kernel of its own.
             const bool sel_in_gemm = sparse && bs == 1 && sd.W <= SEL_SMALL_W && is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) &&
-                                     dq % 64 == 0 && d % 256 == 0 && c->sw.fuse_select;
+                                     dq % 64 == 0 && d % 256 == 0 && c->sw.fuse_select && Kp == 0;
             tc::SelFuse sf;
             memset(&sf, 0, sizeof(sf));
             if (sparse) {
@@ -762,6 +810,7 @@ struct Path {
                 s.mode = p.select_mode;
                 s.k = p.select_mode == POLESTAR_SELECT_TOPK_FRAC ? (int)floorf(p.select_frac * (float)sd.W + 0.5f) : p.select_k;
                 s.W_max = Wm; s.thresh = p.select_thresh; s.floor_ = p.drift_floor;
+                s.ct = ct; s.cluster_k = p.cluster_k;
                 if (sel_in_gemm) { sf.on = 1; sf.sd = sd; sf.a = s; }
                 else {
                     CK(launch_k(step_select_kernel, dim3(bs), dim3(SEL_THREADS), 0, st, sd, s));
@@ -796,7 +845,8 @@ struct Path {
                 int n_chain = 3;
                 double by4 = 0, fl4 = 0;
                 // (off by default: measured 1 % slower than launching that projection on its own)
-                if (l + 1 < L && !fold && c->sw.chain_qkv) {
+                if (l + 1 < L && !fold && c->sw.chain_qkv && n_proxies(&p) == 0) {      // (proxy rows are staged from the next
+                                                                                          // layer's cluster tables, made after this point)
                     n_chain = 4;
                     sp[2].norm_after = 2;
                     PostArgs& po = sp[2].post;
@@ -855,7 +905,7 @@ struct Path {
                 if (fold && l + 1 < L) { e.fold_a = b.a_buf; e.fold_gain = c->n1[l + 1]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 2) * Mm; }
                 PostArgs po;
                 memset(&po, 0, sizeof(po));
-                if (l + 1 < L) {
+                if (l + 1 < L && n_proxies(&p) == 0) {
                     po.kind = 2; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n1[l + 1]; po.a_out = b.a_buf;
                     po.x = b.x; po.rows = b.rows; po.hc = b.hc + (size_t)(l + 1) * bs * Wm * d; po.packet = b.packet;
                     po.patch = b.patch + (size_t)(l + 1) * bs * Wm; po.kvflag = b.kvflag; po.sd = sd;
@@ -907,20 +957,22 @@ static StepDesc make_step_desc(polestar_ctx* c, bool* any_refresh) {
     StepDesc sd;
     memset(&sd, 0, sizeof(sd));
     const int N = c->N, B = c->B;
+    const bool nocache = (p.flags & POLESTAR_FLAG_NOCACHE) != 0;
     const int start = p.prompt_len + c->block * B, end = start + B;
     sd.batch = p.batch; sd.N = N; sd.B = B; sd.act_start = start; sd.W_max = c->W_max;
+    const int Kp = n_proxies(&p);
     sd.pre_start = (int)std::max<long long>(0, (long long)start - (long long)p.win_prefix_blocks * B);
     sd.n_pre = start - sd.pre_start;
     sd.suf_start = end;
     const int n_suf = (int)(std::min<long long>(N, (long long)end + (long long)p.win_suffix_blocks * B) - end);
     sd.W = sd.n_pre + n_suf;
-    const bool nocache = (p.flags & POLESTAR_FLAG_NOCACHE) != 0;
     *any_refresh = false;
     if (c->need_entry || nocache) {
         const bool full = nocache || (c->block % p.full_entry_period == 0);
         sd.kind = full ? 0 : 1;
         sd.e0 = full ? 0 : sd.pre_start;
-        sd.rows_per_seq = full ? N : (sd.n_pre + B + n_suf);
+        sd.rows_per_seq = (full ? N : (sd.n_pre + B + n_suf)) + Kp;
+        sd.K = Kp;
         sd.within = 0;
         sd.record_kl = (nocache && !c->need_entry) ? 1 : 0;
     } else {
@@ -932,7 +984,8 @@ static StepDesc make_step_desc(polestar_ctx* c, bool* any_refresh) {
             sd.refresh.v[s] = r ? 1 : 0;
             if (r) { *any_refresh = true; c->cum[s] = 0; }
         }
-        sd.rows_per_seq = *any_refresh ? B + sd.W : B;
+        sd.K = *any_refresh ? Kp : 0;
+        sd.rows_per_seq = *any_refresh ? B + sd.W + Kp : B;
     }
     return sd;
 }
@@ -950,6 +1003,10 @@ extern "C" int polestar_step(polestar_ctx* c, polestar_step_info* info) {
     if (c->forced_select) {
         CK(cudaMemsetAsync(c->b.forced_cnt, 0xFF, (size_t)c->m.n_layers * c->p.batch * sizeof(int), c->st));
         c->forced_select = false;
+    }
+    if (c->forced_labels && sd.kind != 2) {       // forced labels serve one block-entry forward
+        CK(cudaMemsetAsync(c->b.forced_labels, 0xFF, (size_t)c->m.n_layers * c->p.batch * c->W_max * sizeof(int), c->st));
+        c->forced_labels = false;
     }
     c->last_sd = sd;
     c->pending = true;
@@ -1100,7 +1157,7 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     c->es = m->dtype == POLESTAR_BF16 ? 2 : 4;
     c->N = p->prompt_len + p->gen_len; c->B = p->block; c->W_max = window_max(p);
     c->n_blocks = p->gen_len / p->block;
-    c->M_max = p->batch * std::max(c->N, c->B + c->W_max);
+    c->M_max = p->batch * (std::max(c->N, c->B + c->W_max) + n_proxies(p));
     c->rows_lm = p->batch * (c->B + std::min(p->win_suffix_blocks * c->B, c->W_max));
     c->cum.assign(p->batch, 0);
     c->gws.partial = c->b.gemm_partial; c->gws.partial_bytes = GEMM_PARTIAL_BYTES;
@@ -1117,6 +1174,8 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     if (cudaMemsetAsync(c->b.forced_cnt, 0xFF, (size_t)m->n_layers * p->batch * sizeof(int), c->st) != cudaSuccess)
         return fail(POLESTAR_E_CUDA);
     if (cudaMemsetAsync(c->b.gemm_counters, 0, GEMM_COUNTERS * sizeof(int), c->st) != cudaSuccess) return fail(POLESTAR_E_CUDA);
+    if (n_proxies(p) && cudaMemsetAsync(c->b.forced_labels, 0xFF, (size_t)m->n_layers * p->batch * c->W_max * sizeof(int), c->st) != cudaSuccess)
+        return fail(POLESTAR_E_CUDA);
     if (prompt_dev) {
         init_tokens_kernel<<<(p->batch * c->N + 255) / 256, 256, 0, c->st>>>(c->b.y, prompt, p->batch, p->prompt_len, c->N,
                                                                             m->mask_id, m->vocab);
@@ -1200,7 +1259,7 @@ extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void*
         case POLESTAR_READ_COMMIT: src = c->b.commit_flags; sz = bs * B * 4; break;
         case POLESTAR_READ_PPREV: {
             // stored as (row, lse) with log-probability = row - lse: put together on the host
-            const size_t n_rows = bs * Wm * m.n_heads;
+            const size_t n_rows = bs * (n_proxies(&c->p) ? (size_t)n_proxies(&c->p) : Wm) * m.n_heads;
             std::vector<float> rows(n_rows * N), lse(n_rows);
             CK(cudaMemcpyAsync(rows.data(), c->b.pprev + layer * n_rows * N, rows.size() * 4, cudaMemcpyDeviceToHost, c->st));
             CK(cudaMemcpyAsync(lse.data(), c->b.pprev_lse + layer * n_rows, lse.size() * 4, cudaMemcpyDeviceToHost, c->st));
@@ -1216,6 +1275,9 @@ extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void*
         case POLESTAR_READ_THETA: src = c->b.theta; sz = bs * std::max<size_t>(1, c->p.hist) * B * 4; break;
         case POLESTAR_READ_THETA_COUNT: src = c->b.theta_cnt; sz = bs * 4; break;
         case POLESTAR_READ_OWN_COMMIT: src = c->b.own_flags; sz = bs * B * 4; break;
+        case POLESTAR_READ_LABELS:
+            if (!n_proxies(&c->p) || layer < 0 || layer >= (int)L) return POLESTAR_E_INVAL;
+            src = c->b.labels + layer * bs * Wm; sz = bs * Wm * 4; break;
 #ifdef POLESTAR_TRACE
         case POLESTAR_READ_TRACE_KERNELS: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384 - 65536; sz = 65536; break;
         case POLESTAR_READ_TRACE_GEMM: src = (char*)c->b.gemm_partial + GEMM_PARTIAL_BYTES - 16384; sz = 16384; break;
@@ -1253,6 +1315,15 @@ extern "C" int polestar_force(polestar_ctx* c, int32_t what, int32_t layer, cons
         CK(cudaMemcpyAsync(c->b.forced_cnt + (size_t)layer * bs, cnt.data(), bs * sizeof(int), cudaMemcpyHostToDevice, c->st));
         CK(cudaStreamSynchronize(c->st));
         c->forced_select = true;
+        return POLESTAR_OK;
+    }
+    if (what == POLESTAR_FORCE_LABELS) {
+        if (!n_proxies(&c->p) || layer < 0 || layer >= L || n <= 0 || n > Wm) return POLESTAR_E_INVAL;
+        for (int s = 0; s < bs; ++s)
+            CK(cudaMemcpyAsync(c->b.forced_labels + ((size_t)layer * bs + s) * Wm, idx + (size_t)s * n, n * sizeof(int),
+                               cudaMemcpyHostToDevice, c->st));
+        CK(cudaStreamSynchronize(c->st));
+        c->forced_labels = true;
         return POLESTAR_OK;
     }
     if (what == POLESTAR_FORCE_COMMIT) {

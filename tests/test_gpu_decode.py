@@ -26,7 +26,7 @@ def setup(name, std=0.02, **kw):
     return m, p, gpu, ora
 
 
-def run_forced(name, n_steps, std=0.02, **kw):
+def run_forced(name, n_steps, std=0.02, force_labels=True, **kw):
     """The CUDA path replays the oracle's refresh sets and commits; every step's numbers are compared."""
     m, p, gpu, ora = setup(name, std, **kw)
     tol = TOL[m.dtype]
@@ -39,7 +39,16 @@ def run_forced(name, n_steps, std=0.02, **kw):
             break
         ora.step()     # oracle first, so that its refresh sets can be imposed on the CUDA step
         tr = ora.seqs[0].trace
+        cluster = p.select_mode == I.SELECT_CLUSTER_TOPK
         if step > 0:
+            if cluster and tr["kind"] != "within" and force_labels:
+                # replay the oracle's clustering at later block entries (a near-tie between two centres may fall
+                # either way in fp32); the first entry, inside polestar_init, is the library's own K-means
+                for l in range(L):
+                    lab = np.full((p.batch, gpu.W_max), 0, np.int32)
+                    for s in range(p.batch):
+                        lab[s, :len(ora.seqs[s].labels[l])] = ora.seqs[s].labels[l]
+                    gpu.force_labels(l, lab[:, :len(ora.seqs[0].labels[l])])
             if tr["kind"] == "within" and tr["refresh"]:
                 for l in range(L):
                     sel = np.full((p.batch, gpu.W_max), -1, np.int32)
@@ -62,11 +71,17 @@ def run_forced(name, n_steps, std=0.02, **kw):
                     seen["refresh"] += 1
                     W = len(ora.seqs[s].win)
                     for l in range(L):
-                        close(gpu.read(Bd.READ_DRIFT, l)[s, :W], trs["D"][l], tol, f"step {step} drift l{l}")
+                        nD = len(trs["D"][l])          # window rows, or clusters (centroid proxies)
+                        close(gpu.read(Bd.READ_DRIFT, l)[s, :nD], trs["D"][l], tol, f"step {step} drift l{l}")
                         n = gpu.read(Bd.READ_SEL_COUNT, l)[s]
                         assert list(gpu.read(Bd.READ_SEL_IDX, l)[s, :n]) == list(trs["sel"][l])
             elif trs["kind"] == "entry_window":
                 seen["entry_window"] += 1
+            if cluster and trs["kind"] != "within":
+                for l in range(L):          # the clustering of this block entry
+                    W = len(ora.seqs[s].win)
+                    assert np.array_equal(gpu.read(Bd.READ_LABELS, l)[s, :W], ora.seqs[s].labels[l]), f"step {step} labels l{l}"
+                seen["clusterings"] = seen.get("clusterings", 0) + 1
             for l in range(L):
                 close_h(gpu.read(Bd.READ_KCACHE, l)[s].reshape(ora.seqs[s].Kc[l].shape), ora.seqs[s].Kc[l], tol,
                         f"step {step} K l{l}", depth=l)
@@ -128,6 +143,24 @@ def test_c1b_commit_quantities_match_oracle():
     seen = run_forced("c1b", 12, **C1B_COMMIT)
     assert seen["own_by_conf"] > 0 and seen["own_suffix"] > 0, seen
     assert seen["delta_rows"] > 0 and seen["theta_vectors"] > 5, seen
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("c1", dict(tau_upd=-1, logit_scale=12.0, tau_suffix=0.5)),                      # fp32, CUDA-core attention
+    ("c1b", dict(tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)),        # bf16, tensor-core attention
+    ("c1b", dict(tau_upd=2, logit_scale=24.0, tau_suffix=0.5, batch=3, n_clusters=5, cluster_k=2)),
+    ("c1b", dict(tau_upd=-1, logit_scale=24.0, n_clusters=16, cluster_k=16, block=8, gen_len=32, max_steps=16)),   # W = 24: ragged clusters
+])
+def test_centroid_proxy_mode_matches_oracle(name, kw):
+    # Sec. 4.1 default policy: K-means at block entry, proxy attention of the centroids, cluster top-k -> member rows
+    seen = run_forced(name, 24, select_mode=I.SELECT_CLUSTER_TOPK, **kw)
+    assert seen["refresh"] >= 2 and seen["clusterings"] >= 2, seen
+
+
+def test_centroid_proxy_own_clustering_matches_oracle():
+    # the library's own K-means at every block entry (nothing replayed): labels equal the oracle's
+    seen = run_forced("c1", 40, force_labels=False, select_mode=I.SELECT_CLUSTER_TOPK, tau_upd=2, logit_scale=12.0)
+    assert seen["clusterings"] >= 2, seen
 
 
 def test_c1_refresh_every_step_with_scaled_logits():
