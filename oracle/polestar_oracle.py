@@ -63,6 +63,7 @@ F64 = np.float64
 
 SELECT_TOPK_FRAC, SELECT_TOPK_COUNT, SELECT_THRESHOLD, SELECT_ALL, SELECT_NONE, SELECT_CLUSTER_TOPK = range(6)
 FLAG_DRIFT_COMMIT, FLAG_SUFFIX_COMMIT, FLAG_GE_COMPARE, FLAG_NOCACHE = 1, 2, 4, 8
+FLAG_NVFP4_HCACHE = 1 << 8
 
 
 # --------------------------------------------------------------------------
@@ -259,6 +260,69 @@ def cluster_proxies(H: np.ndarray, positions: np.ndarray, labels: np.ndarray, K:
     return Z, pos, cnt
 
 
+# --------------------------------------------------------------------------
+# NVFP4 residual codec of the hidden-state cache (Sec. 4.1 "Cluster and Quantize
+# Hidden States"; Appendix "Quantization Format")
+# --------------------------------------------------------------------------
+# A value is 1 sign bit, 2 exponent bits, 1 mantissa bit (E2M1): magnitudes
+# {0, 0.5, 1, 1.5, 2, 3, 4, 6}; every group of 16 values along the channel
+# dimension shares an FP8 E4M3 scale.  The format decides integers (codes), so the
+# codec is carried out in float32, the precision the kernel uses: the same inputs
+# give the same codes.  Readings where the paper is silent: scale = E4M3(amax / 6)
+# rounded to nearest even and saturated at 448; codes round to the nearest grid
+# value, ties to the even code, saturating at 6; an all-zero group has scale 0.
+
+E2M1_GRID = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0], np.float32)
+_E2M1_MID = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], np.float32)     # midpoints between grid values
+_E2M1_TIE_UP = np.array([False, True, False, True, False, True, False])       # a tie goes to the even code
+
+
+def e4m3_round(x) -> np.ndarray:
+    """Nearest FP8 E4M3 value (4 exponent bits, bias 7, 3 mantissa bits, no infinities; largest
+    448, smallest subnormal 2^-9), ties to even, saturating; x >= 0, float32 in and out."""
+    x = np.minimum(np.asarray(x, np.float32), np.float32(448.0))
+    out = np.zeros_like(x)
+    pos = x > 0
+    e = np.floor(np.log2(x, where=pos, out=np.zeros_like(x))).astype(np.int32)
+    e = np.clip(e, -6, 8)
+    step = np.ldexp(np.float32(1.0), e - 3).astype(np.float32)                # spacing of the grid around x
+    q = (np.rint(x / step) * step).astype(np.float32)                         # rint: ties to even; exact in float32
+    out[pos] = q[pos]
+    return np.minimum(out, np.float32(448.0))
+
+
+def nvfp4_quantize(r):
+    """r [..., d] (d a multiple of 16) -> (codes int8 [..., d]: bit 3 sign, bits 0-2 grid index;
+    scales float32 [..., d/16] on the E4M3 grid)."""
+    r = np.asarray(r, np.float32)
+    g = r.reshape(r.shape[:-1] + (r.shape[-1] // 16, 16))
+    amax = np.max(np.abs(g), axis=-1)
+    scale = e4m3_round(amax / np.float32(6.0))
+    safe = np.where(scale > 0, scale, np.float32(1.0)).astype(np.float32)
+    y = (np.abs(g) / safe[..., None]).astype(np.float32)
+    idx = np.zeros(y.shape, np.int8)
+    for k in range(7):                                    # count the midpoints passed (ties by the even-code rule)
+        idx += ((y > _E2M1_MID[k]) | ((y == _E2M1_MID[k]) & _E2M1_TIE_UP[k])).astype(np.int8)
+    idx = np.where(scale[..., None] > 0, idx, 0).astype(np.int8)
+    codes = (idx | ((g < 0).astype(np.int8) << 3)).astype(np.int8)
+    return codes.reshape(r.shape), scale
+
+
+def nvfp4_dequantize(codes, scale) -> np.ndarray:
+    codes = np.asarray(codes, np.int8)
+    g = codes.reshape(codes.shape[:-1] + (codes.shape[-1] // 16, 16))
+    mag = E2M1_GRID[g & 7] * np.asarray(scale, np.float32)[..., None]
+    return np.where((g & 8) != 0, -mag, mag).astype(np.float32).reshape(codes.shape)
+
+
+def residual_nvfp4_roundtrip(h, ref) -> np.ndarray:
+    """What the quantised cache holds for row(s) h with reference row(s) ref (the block-entry
+    centroid of the row's cluster): ref + dequant(quant(h - ref)), all in float32."""
+    h32, r32 = np.asarray(h, np.float32), np.asarray(ref, np.float32)
+    codes, scale = nvfp4_quantize((h32 - r32).astype(np.float32))
+    return (r32 + nvfp4_dequantize(codes, scale)).astype(np.float32).astype(F64)
+
+
 def confidence_rows(logits: np.ndarray, mask_id: int):
     """Eq. 1 and the confidence of Sec. 2: y_hat = argmax over v != [MASK] (lowest id
     on ties), c = softmax(logits over the whole vocabulary)[y_hat]."""
@@ -369,6 +433,7 @@ class _Seq:
         self.Z: List[Optional[np.ndarray]] = [None] * L
         self.zpos: List[Optional[np.ndarray]] = [None] * L
         self.zcnt: List[Optional[np.ndarray]] = [None] * L
+        self.Z0: List[Optional[np.ndarray]] = [None] * L      # block-entry centroids: reference of the NVFP4 residuals
         self.Aprev = None
         self.theta: List[np.ndarray] = []
         self.tok_at_h0 = None
@@ -432,6 +497,12 @@ class _Seq:
                 # Algorithm 1 block entry: Z, M <- SphericalKMeans(H, K);  P <- ProxyAttn(Z), all layers
                 K = p.n_clusters
                 self.labels[l] = spherical_kmeans(self.Hc[l], K, p.kmeans_iters)
+                if p.flags & FLAG_NVFP4_HCACHE:
+                    # the cache keeps NVFP4 residuals against the block-entry centroid of the row's cluster; the
+                    # reference stays fixed for the block, the drift proxy below follows the (dequantised) members
+                    self.Z0[l], _, _ = cluster_proxies(self.Hc[l], win, self.labels[l], K)
+                    self.Z0[l] = self.Z0[l].astype(np.float32).astype(F64)
+                    self.Hc[l] = residual_nvfp4_roundtrip(self.Hc[l], self.Z0[l][self.labels[l]])
                 self.Z[l], self.zpos[l], self.zcnt[l] = cluster_proxies(self.Hc[l], win, self.labels[l], K)
                 live = np.nonzero(self.zcnt[l] > 0)[0]
                 self.Pprev[l] = np.zeros((K, m.n_heads, self.N), F64)
@@ -477,6 +548,10 @@ class _Seq:
             tr["x_act"].append(x.copy())
             # 1. patch the caches from the update packet of the previous layer
             if refresh and len(U_idx):
+                if p.select_mode == SELECT_CLUSTER_TOPK and (p.flags & FLAG_NVFP4_HCACHE):
+                    # a refreshed row enters the cache through the codec; everything that follows (its K / V, its
+                    # query, the proxy, the residual input of the sparse forward) sees the stored value
+                    U_val = residual_nvfp4_roundtrip(U_val, self.Z0[l][self.labels[l][U_idx]])
                 if p.select_mode == SELECT_CLUSTER_TOPK:
                     # the centroid follows its refreshed members (Sec. 4.1: "updated incrementally")
                     for t, i in enumerate(U_idx):

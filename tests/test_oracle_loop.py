@@ -332,3 +332,30 @@ def test_cluster_mode_zero_drift_refreshes_nothing():
     assert tr["kind"] == "within" and tr["refresh"]
     for l in range(m.n_layers):
         assert not tr["D"][l].any() and len(tr["sel"][l]) == 0
+
+
+def test_nvfp4_hidden_cache_is_lossy_but_close():
+    # Sec. 4.1 "Cluster and Quantize Hidden States": the cached hidden rows are NVFP4 residuals against their
+    # cluster's centroid.  Every cached row lies on the codec's grid around its reference, the decode still
+    # terminates, and the logits stay close to the unquantised cluster mode (the paper's quantisation ablation
+    # reports the same ordering: a small loss).
+    kw = dict(select_mode=I.SELECT_CLUSTER_TOPK, n_clusters=4, cluster_k=2, tau_upd=-1, logit_scale=3.0)
+    m, p, w, prompt = tiny(**kw)
+    m = dataclasses.replace(m)            # (d_model 64: a multiple of the group size 16)
+    pq = dataclasses.replace(p, flags=p.flags | O.FLAG_NVFP4_HCACHE)
+    a, b = O.PolestarOracle(m, w, p, prompt), O.PolestarOracle(m, w, pq, prompt)
+    a.step(); b.step()
+    errs = []
+    for _ in range(2):       # the entry forward and the first step (later steps may already take other decisions)
+        sb = b.seqs[0]
+        for l in range(m.n_layers):
+            ref = sb.Z0[l][sb.labels[l]]
+            assert np.array_equal(O.residual_nvfp4_roundtrip(sb.Hc[l], ref), sb.Hc[l])        # on the grid: idempotent
+        errs.append(np.abs(a.seqs[0].trace["logits"] - b.seqs[0].trace["logits"]).max())
+        forced = [dict(commit=i["commit"], suffix=tuple(i["suffix_committed"])) for i in a.commit()]
+        b.commit(forced)
+        a.step(); b.step()
+    assert errs[0] == 0.0 and 0 < errs[1] < 0.1 * np.abs(a.seqs[0].trace["logits"]).max()
+    b2 = O.PolestarOracle(m, w, pq, prompt)
+    b2.decode()
+    assert b2.done and not (b2.tokens() == m.mask_id).any()

@@ -422,3 +422,48 @@ def test_cluster_proxies_pins():
     assert np.array_equal(Z[4], H[5]) and zp[4] == 21                      # a cluster of one row is that row
     assert zp[0] == int(np.floor((3 + 4 + 22) / 3 + 0.5)) and zp[2] == 10   # rounded mean position
     assert not Z[1].any() and not Z[3].any()
+
+
+# ---------------------------------------------------------------- NVFP4 residual codec (Appendix "Quantization Format")
+def test_e4m3_scale_rounding_matches_library_cast():
+    x = np.abs(rng.standard_normal(200000)).astype(np.float32) * np.float32(10.0) ** rng.integers(-5, 3, 200000).astype(np.float32)
+    x = np.concatenate([x, np.float32([0.0, 2.0 ** -9, 2.0 ** -10, 1.5 * 2.0 ** -9, 448.0, 1000.0, 0.0625 * 1.0625])])
+    ref = torch.tensor(np.minimum(x, np.float32(448.0))).to(torch.float8_e4m3fn).float().numpy()     # library: RNE; saturation by the clamp
+    assert np.array_equal(O.e4m3_round(x), ref)
+
+
+def test_e2m1_grid_is_the_formats_value_set():
+    # 1 sign, 2 exponent (bias 1), 1 mantissa bit: subnormals m/2, normals (1 + m/2) 2^(e-1)
+    vals = sorted({(m / 2.0) if e == 0 else (1 + m / 2.0) * 2.0 ** (e - 1) for e in range(4) for m in range(2)})
+    assert vals == O.E2M1_GRID.tolist() == [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+
+
+def test_nvfp4_quantize_pins():
+    r = (rng.standard_normal((64, 128)) * 10.0 ** rng.integers(-3, 2, (64, 1))).astype(np.float32)
+    r[3, 16:32] = 0.0                                            # an all-zero group
+    r[5, 0] = 1e4                                                # an outlier: the rest of its group rounds to zero
+    codes, scale = O.nvfp4_quantize(r)
+    dq = O.nvfp4_dequantize(codes, scale)
+    g, gq = r.reshape(64, 8, 16), dq.reshape(64, 8, 16)
+    amax = np.abs(g).max(-1)
+    assert np.array_equal(scale, O.e4m3_round(amax / np.float32(6.0))) and (scale[3, 1] == 0) and not gq[3, 1].any()
+    # brute force: every code is a nearest grid point of |x| / s (saturating), sign kept
+    for i, j, k in [(a, b, c) for a in range(0, 64, 7) for b in range(8) for c in range(16)]:
+        if scale[i, j] == 0:
+            continue
+        y = abs(g[i, j, k]) / scale[i, j]
+        best = np.abs(O.E2M1_GRID - min(y, np.float32(6.0))).min()
+        assert abs(abs(gq[i, j, k]) / scale[i, j] - min(y, 6.0)) <= best + 1e-6
+        assert gq[i, j, k] == 0 or np.sign(gq[i, j, k]) == np.sign(g[i, j, k])
+    # ties go to the even code: 0.25 -> 0, 0.75 -> 1, 1.25 -> 1, 1.75 -> 2, 2.5 -> 2, 3.5 -> 4, 5 -> 4 (scale 1: amax 6)
+    t = np.zeros((1, 16), np.float32)
+    t[0, :8] = [6.0, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0]
+    c, s1 = O.nvfp4_quantize(t)
+    assert s1[0, 0] == 1.0 and O.nvfp4_dequantize(c, s1)[0, :8].tolist() == [6.0, 0.0, 1.0, 1.0, 2.0, 2.0, 4.0, 4.0]
+    # error bound: half the coarsest grid step (2) times the scale; idempotent (grid points stay put)
+    assert (np.abs(g - gq) <= scale[..., None] * 1.0 + np.maximum(np.abs(g) - 6 * scale[..., None], 0) + 1e-12).all()
+    c2, s2 = O.nvfp4_quantize(dq)
+    assert np.array_equal(O.nvfp4_dequantize(c2, s2), dq)
+    # the residual round trip keeps the reference exactly when the row equals it
+    ref = rng.standard_normal((4, 32)).astype(np.float32)
+    assert np.array_equal(O.residual_nvfp4_roundtrip(ref, ref), ref.astype(np.float64))
