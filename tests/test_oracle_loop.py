@@ -347,10 +347,13 @@ def test_nvfp4_hidden_cache_is_lossy_but_close():
     a.step(); b.step()
     errs = []
     for _ in range(2):       # the entry forward and the first step (later steps may already take other decisions)
-        sb = b.seqs[0]
+        sa, sb = a.seqs[0], b.seqs[0]
         for l in range(m.n_layers):
-            ref = sb.Z0[l][sb.labels[l]]
-            assert np.array_equal(O.residual_nvfp4_roundtrip(sb.Hc[l], ref), sb.Hc[l])        # on the grid: idempotent
+            # every cached row is its reference plus a float32 grid value, within the codec's error of the plain row
+            assert np.array_equal(sb.Hc[l].astype(np.float32).astype(np.float64), sb.Hc[l])
+            if _ == 0:
+                res = np.abs(sa.Hc[l] - sb.Z0[l][sb.labels[l]]).reshape(len(sb.win), -1, 16).max(-1, keepdims=True)
+                assert (np.abs(sa.Hc[l] - sb.Hc[l]).reshape(len(sb.win), -1, 16) <= res / 6 * 1.07 + 1e-6).all()
         errs.append(np.abs(a.seqs[0].trace["logits"] - b.seqs[0].trace["logits"]).max())
         forced = [dict(commit=i["commit"], suffix=tuple(i["suffix_committed"])) for i in a.commit()]
         b.commit(forced)

@@ -460,10 +460,12 @@ def test_nvfp4_quantize_pins():
     t[0, :8] = [6.0, 0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0]
     c, s1 = O.nvfp4_quantize(t)
     assert s1[0, 0] == 1.0 and O.nvfp4_dequantize(c, s1)[0, :8].tolist() == [6.0, 0.0, 1.0, 1.0, 2.0, 2.0, 4.0, 4.0]
-    # error bound: half the coarsest grid step (2) times the scale; idempotent (grid points stay put)
+    # error bound: half the coarsest grid step (2) times the scale, plus what saturation at 6 s cuts off
     assert (np.abs(g - gq) <= scale[..., None] * 1.0 + np.maximum(np.abs(g) - 6 * scale[..., None], 0) + 1e-12).all()
+    # a group whose largest code is 6 keeps its scale, so its grid points stay put when quantised again
+    top = np.abs(gq).max(-1) == 6 * scale
     c2, s2 = O.nvfp4_quantize(dq)
-    assert np.array_equal(O.nvfp4_dequantize(c2, s2), dq)
+    assert top.any() and np.array_equal(O.nvfp4_dequantize(c2, s2).reshape(64, 8, 16)[top], gq[top])
     # the residual round trip keeps the reference exactly when the row equals it
     ref = rng.standard_normal((4, 32)).astype(np.float32)
     assert np.array_equal(O.residual_nvfp4_roundtrip(ref, ref), ref.astype(np.float64))
