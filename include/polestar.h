@@ -91,6 +91,13 @@ extern "C" {
 #define POLESTAR_FLAG_SIMT_GEMM     (1u << 5) /* bf16 models: plain CUDA-core GEMMs (debug aid)     */
 #define POLESTAR_FLAG_PROMPT_DEVICE (1u << 6) /* polestar_init: prompt ids are a DEVICE array       */
 #define POLESTAR_FLAG_PROFILE       (1u << 7) /* bracket kernel families with CUDA events           */
+#define POLESTAR_FLAG_NVFP4_HCACHE  (1u << 8) /* window hidden cache as NVFP4 residuals against the row's cluster
+                                                 centroid (Sec. 4.1 "Cluster and Quantize Hidden States"; Appendix
+                                                 "Quantization Format"): E2M1 codes, one E4M3 scale per 16 channels;
+                                                 needs POLESTAR_SELECT_CLUSTER_TOPK and d_model % 128 == 0.  The
+                                                 reference is the cluster's centroid at block entry (fixed for the
+                                                 block); a row is encoded when it enters the cache (block entry, or
+                                                 a packet row), and every later reader sees the decoded value.  */
 
 /* kernel families reported by polestar_profile */
 #define POLESTAR_PROF_GEMM_QKV     0
@@ -264,6 +271,12 @@ int polestar_read(polestar_ctx *c, int32_t what, int32_t layer, void *dst_host, 
 #define POLESTAR_FORCE_LABELS 5  /* centroid proxies: cluster labels of the window rows at `layer` for the next
                                     block-entry forward, instead of the library's own K-means ([batch][n],
                                     n = window rows; a near-tie between two centres may fall either way)  */
+#define POLESTAR_FORCE_HCODES 6  /* NVFP4 hidden cache (context created with POLESTAR_FLAG_KEEP_HIDDEN too): codes
+                                    of window rows at `layer`.  idx_host is a byte blob: mask uint8 [batch][n],
+                                    codes uint8 [batch][n][d/2], scales uint8 [batch][n][d/16] (n = window rows).
+                                    Rows with a non-zero mask take these codes now (the cache is rewritten), and
+                                    again in place of the codec's own decision if the NEXT step encodes them
+                                    (a value next to a code boundary may fall either way in another arithmetic) */
 int polestar_force(polestar_ctx *c, int32_t what, int32_t layer, const int32_t *idx_host, int32_t n);
 
 /* Per-family device time of the forwards so far (context created with POLESTAR_FLAG_PROFILE;
@@ -339,6 +352,15 @@ int polestar_k_refresh(const void *h_dev, const int32_t *idx_dev, const int32_t 
  * rows of that call are then incomplete). */
 int polestar_k_refresh_status(const void *scratch_dev, size_t scratch_bytes, int32_t batch, int32_t max_rows,
                               int32_t d, int32_t head_dim, void *cuda_stream);
+
+/* The NVFP4 residual codec on its own (Appendix "Quantization Format"): for every row, codes and scales of
+ * x - ref and the stored value ref + decode(...).  float32 arithmetic: scale = E4M3(amax / 6) (nearest even,
+ * saturating), codes to the nearest E2M1 value (ties to the even code, saturating at 6).
+ *   x_dev, ref_dev, deq_dev float [rows][d] (16-byte aligned), d % 128 == 0
+ *   codes_dev uint8 [rows][d/2] (channel 2i in the low nibble: bit 3 sign, bits 0-2 grid index)
+ *   scales_dev uint8 [rows][d/16] (E4M3 bit patterns). */
+int polestar_k_nvfp4_residual(const float *x_dev, const float *ref_dev, int32_t rows, int32_t d,
+                              uint8_t *codes_dev, uint8_t *scales_dev, float *deq_dev, void *cuda_stream);
 
 /* Confidence of logits rows (Eq. 1; Sec. 2 sampler set): per row, y_hat = argmax over v != mask_id
  * (lowest id on ties), conf = softmax(logits)[y_hat].  logits_dev float [rows][vocab], 16-byte aligned

@@ -315,12 +315,17 @@ def nvfp4_dequantize(codes, scale) -> np.ndarray:
     return np.where((g & 8) != 0, -mag, mag).astype(np.float32).reshape(codes.shape)
 
 
-def residual_nvfp4_roundtrip(h, ref) -> np.ndarray:
-    """What the quantised cache holds for row(s) h with reference row(s) ref (the block-entry
-    centroid of the row's cluster): ref + dequant(quant(h - ref)), all in float32."""
+def residual_nvfp4_encode(h, ref):
+    """Row(s) h with reference row(s) ref (the block-entry centroid of the row's cluster) ->
+    (codes, scales, stored value ref + dequant(quant(h - ref))), all in float32."""
     h32, r32 = np.asarray(h, np.float32), np.asarray(ref, np.float32)
     codes, scale = nvfp4_quantize((h32 - r32).astype(np.float32))
-    return (r32 + nvfp4_dequantize(codes, scale)).astype(np.float32).astype(F64)
+    return codes, scale, (r32 + nvfp4_dequantize(codes, scale)).astype(np.float32).astype(F64)
+
+
+def residual_nvfp4_roundtrip(h, ref) -> np.ndarray:
+    """What the quantised cache holds for row(s) h."""
+    return residual_nvfp4_encode(h, ref)[2]
 
 
 def confidence_rows(logits: np.ndarray, mask_id: int):
@@ -502,7 +507,8 @@ class _Seq:
                     # reference stays fixed for the block, the drift proxy below follows the (dequantised) members
                     self.Z0[l], _, _ = cluster_proxies(self.Hc[l], win, self.labels[l], K)
                     self.Z0[l] = self.Z0[l].astype(np.float32).astype(F64)
-                    self.Hc[l] = residual_nvfp4_roundtrip(self.Hc[l], self.Z0[l][self.labels[l]])
+                    cq, sq, self.Hc[l] = residual_nvfp4_encode(self.Hc[l], self.Z0[l][self.labels[l]])
+                    tr.setdefault("hcodes", {})[l] = (np.arange(len(win)), cq, sq)
                 self.Z[l], self.zpos[l], self.zcnt[l] = cluster_proxies(self.Hc[l], win, self.labels[l], K)
                 live = np.nonzero(self.zcnt[l] > 0)[0]
                 self.Pprev[l] = np.zeros((K, m.n_heads, self.N), F64)
@@ -551,7 +557,8 @@ class _Seq:
                 if p.select_mode == SELECT_CLUSTER_TOPK and (p.flags & FLAG_NVFP4_HCACHE):
                     # a refreshed row enters the cache through the codec; everything that follows (its K / V, its
                     # query, the proxy, the residual input of the sparse forward) sees the stored value
-                    U_val = residual_nvfp4_roundtrip(U_val, self.Z0[l][self.labels[l][U_idx]])
+                    cq, sq, U_val = residual_nvfp4_encode(U_val, self.Z0[l][self.labels[l][U_idx]])
+                    tr.setdefault("hcodes", {})[l] = (U_idx.copy(), cq, sq)
                 if p.select_mode == SELECT_CLUSTER_TOPK:
                     # the centroid follows its refreshed members (Sec. 4.1: "updated incrementally")
                     for t, i in enumerate(U_idx):

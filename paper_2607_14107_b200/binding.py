@@ -25,15 +25,15 @@ READ_LOGITS, READ_CONF, READ_YHAT, READ_DELTA, READ_DRIFT, READ_SEL_COUNT, READ_
 READ_HIDDEN, READ_KCACHE, READ_VCACHE, READ_HCACHE, READ_COMMIT, READ_PPREV, READ_SUFFIX = 8, 9, 10, 11, 12, 13, 14
 READ_DRIFT_DELTA, READ_TAU_D, READ_THETA, READ_THETA_COUNT, READ_OWN_COMMIT, READ_LABELS = 15, 16, 17, 18, 19, 20
 READ_TRACE_KERNELS, READ_TRACE_GEMM = 98, 99
-FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR, FORCE_TOKENS, FORCE_LABELS = 1, 2, 3, 4, 5
-FLAG_SIMT_GEMM, FLAG_PROMPT_DEVICE, FLAG_PROFILE = 1 << 5, 1 << 6, 1 << 7
+FORCE_SELECT, FORCE_COMMIT, FORCE_CLEAR, FORCE_TOKENS, FORCE_LABELS, FORCE_HCODES = 1, 2, 3, 4, 5, 6
+FLAG_SIMT_GEMM, FLAG_PROMPT_DEVICE, FLAG_PROFILE, FLAG_NVFP4_HCACHE = 1 << 5, 1 << 6, 1 << 7, 1 << 8
 PROF_FAMILIES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head", "attention", "stage", "select",
                  "confidence", "commit", "misc"]
 
 EXPORTS = [
     "polestar_workspace_bytes", "polestar_init", "polestar_step", "polestar_commit", "polestar_tokens",
     "polestar_read", "polestar_force", "polestar_profile", "polestar_destroy", "polestar_strerror",
-    "polestar_reload_env", "polestar_k_refresh_status",
+    "polestar_reload_env", "polestar_k_refresh_status", "polestar_k_nvfp4_residual",
     "polestar_k_attention", "polestar_k_hidden_delta", "polestar_k_select",
     "polestar_k_refresh_scratch_bytes", "polestar_k_refresh", "polestar_k_confidence",
     "polestar_k_confidence_noalloc", "polestar_sm_count",
@@ -131,6 +131,8 @@ def load():
     lib.polestar_k_confidence_noalloc.argtypes = [vp, i32, i32, i32, vp, vp, vp]
     lib.polestar_sm_count.restype = C.c_int
     lib.polestar_sm_count.argtypes = []
+    lib.polestar_k_nvfp4_residual.restype = C.c_int
+    lib.polestar_k_nvfp4_residual.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     lib.polestar_reload_env.restype = C.c_int
     lib.polestar_reload_env.argtypes = []
     lib.polestar_k_refresh_status.restype = C.c_int
@@ -356,6 +358,15 @@ class Polestar:
         lab = np.ascontiguousarray(np.asarray(labels, np.int32).reshape(self.p.batch, -1))
         _check(load().polestar_force(self.ctx, FORCE_LABELS, layer, lab.ctypes.data_as(C.POINTER(C.c_int32)), lab.shape[1]))
 
+    def force_hcodes(self, layer: int, mask, codes, scales) -> None:
+        """mask uint8 [batch][n], codes uint8 [batch][n][d/2], scales uint8 [batch][n][d/16] (E4M3 bit patterns)."""
+        mask = np.ascontiguousarray(mask, np.uint8)
+        blob = np.concatenate([mask.ravel(), np.ascontiguousarray(codes, np.uint8).ravel(),
+                               np.ascontiguousarray(scales, np.uint8).ravel()])
+        pad = np.zeros((-len(blob)) % 4, np.uint8)
+        blob = np.ascontiguousarray(np.concatenate([blob, pad]))
+        _check(load().polestar_force(self.ctx, FORCE_HCODES, layer, blob.ctypes.data_as(C.POINTER(C.c_int32)), mask.shape[1]))
+
     def force_clear(self) -> None:
         _check(load().polestar_force(self.ctx, FORCE_CLEAR, 0, None, 0))
 
@@ -412,6 +423,12 @@ def polestar_k_refresh(h, idx, counts, wqkv, norm, kc, vc, q_out, max_rows, n_he
                                      _ptr(q_out), batch, P, max_rows, d, n_heads, n_kv_heads, head_dim, rms_eps,
                                      rope_theta, _dtype_code(h), _ptr(scratch), scratch.numel() * scratch.element_size(),
                                      C.c_void_p(_stream())))
+
+
+def polestar_k_nvfp4_residual(x, ref, codes, scales, deq):
+    rows, d = x.shape
+    _check(load().polestar_k_nvfp4_residual(_ptr(x), _ptr(ref), rows, d, _ptr(codes), _ptr(scales), _ptr(deq),
+                                            C.c_void_p(_stream())))
 
 
 def polestar_reload_env() -> None:

@@ -252,7 +252,69 @@ struct ClusterTabs {
     const int* moff;       // [batch][K + 1] start of every cluster's group
     float* zbuf;           // [batch][K][d] the proxy rows (member means), rebuilt whenever they are needed
     int K;
+    // NVFP4 residual cache (null: the hidden cache holds plain fp32 rows): codes [batch][W_max][d/2] (two E2M1 values
+    // per byte, low nibble first), E4M3 scale bytes [batch][W_max][d/16], reference rows [batch][K][d] = the
+    // block-entry centroids
+    unsigned char* hq; unsigned char* hs; float* z0;
+    // imposed codes (null: none kept): rows whose mask byte is set take fq / fs (laid out like hq / hs) when encoded
+    const unsigned char* fmask; const unsigned char* fq; const unsigned char* fs;
 };
+
+// ---- NVFP4 residual codec (Sec. 4.1 "Cluster and Quantize Hidden States"; Appendix "Quantization Format") ----
+// E2M1 values {0, .5, 1, 1.5, 2, 3, 4, 6} with one FP8 E4M3 scale per 16 channels; float32 arithmetic throughout
+// (the codes are integers decided by it): scale = E4M3(amax / 6), round to nearest even, saturating at 448; codes
+// round to the nearest grid value, ties to the even code, saturating at 6.
+__device__ __forceinline__ float e4m3_round_pos(float x) {          // x >= 0 -> nearest E4M3 value
+    x = fminf(x, 448.f);
+    if (!(x > 0.f)) return 0.f;
+    int ex;
+    frexpf(x, &ex);                                                  // x = f 2^ex, f in [0.5, 1)
+    const int e = min(max(ex - 1, -6), 8);
+    const float step = ldexpf(1.f, e - 3);
+    return fminf(rintf(x / step) * step, 448.f);                     // (division by a power of two: exact)
+}
+__device__ __forceinline__ unsigned e4m3_bits(float q) {            // q on the E4M3 grid, >= 0
+    if (!(q > 0.f)) return 0u;
+    if (q < 0.015625f) return (unsigned)(q * 512.f);                 // subnormal: m 2^-9
+    int ex;
+    const float f = frexpf(q, &ex);                                  // q = f 2^ex
+    return ((unsigned)(ex - 1 + 7) << 3) | (unsigned)((f * 2.f - 1.f) * 8.f);
+}
+__device__ __forceinline__ float e4m3_value(unsigned b) {
+    const unsigned e = (b >> 3) & 15u, m = b & 7u;
+    return e == 0 ? (float)m * 0.001953125f : ldexpf(1.f + (float)m * 0.125f, (int)e - 7);
+}
+__device__ __forceinline__ unsigned e2m1_code(float r, float s) {   // residual r, group scale s > 0 -> sign | index
+    const float y = __fdiv_rn(fabsf(r), s);
+    unsigned i = (y > 0.25f) + (y >= 0.75f) + (y > 1.25f) + (y >= 1.75f) + (y > 2.5f) + (y >= 3.5f) + (y > 5.f);
+    return i | (r < 0.f ? 8u : 0u);
+}
+__device__ __forceinline__ float e2m1_value(unsigned code, float s) {
+    const unsigned i = code & 7u;
+    const float g = i < 4 ? 0.5f * (float)i : (i == 4 ? 2.f : (i == 5 ? 3.f : (i == 6 ? 4.f : 6.f)));
+    const float v = g * s;
+    return (code & 8u) ? -v : v;
+}
+// One 16-byte chunk (4 channels) of a row; the 4 lanes that hold a group of 16 channels call together (lane % 4 =
+// position in the group; every lane of the warp takes part).  Returns the stored value ref + dequant(quant(v - ref));
+// *codes = the chunk's four codes (4 bits each, channel 0 lowest), *scale_bits = the group's E4M3 byte.
+__device__ __forceinline__ float4 nvfp4_residual_chunk(float4 v, float4 ref, unsigned* codes, unsigned* scale_bits) {
+    const float4 r = make_float4(v.x - ref.x, v.y - ref.y, v.z - ref.z, v.w - ref.w);
+    float am = fmaxf(fmaxf(fabsf(r.x), fabsf(r.y)), fmaxf(fabsf(r.z), fabsf(r.w)));
+    am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, 1));
+    am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, 2));
+    const float s = e4m3_round_pos(__fdiv_rn(am, 6.f));
+    *scale_bits = e4m3_bits(s);
+    if (!(s > 0.f)) { *codes = 0u; return ref; }
+    const unsigned c0 = e2m1_code(r.x, s), c1 = e2m1_code(r.y, s), c2 = e2m1_code(r.z, s), c3 = e2m1_code(r.w, s);
+    *codes = c0 | (c1 << 4) | (c2 << 8) | (c3 << 12);
+    return make_float4(ref.x + e2m1_value(c0, s), ref.y + e2m1_value(c1, s), ref.z + e2m1_value(c2, s), ref.w + e2m1_value(c3, s));
+}
+__device__ __forceinline__ float4 nvfp4_dequant_chunk(unsigned codes, unsigned scale_bits, float4 ref) {
+    const float s = e4m3_value(scale_bits);
+    return make_float4(ref.x + e2m1_value(codes & 15u, s), ref.y + e2m1_value((codes >> 4) & 15u, s),
+                       ref.z + e2m1_value((codes >> 8) & 15u, s), ref.w + e2m1_value((codes >> 12) & 15u, s));
+}
 
 // Row-wise work appended to a GEMM whose output rows are the input of the next normalisation: once every CTA
 // of the grid has stored its outputs (a counter all CTAs add to), the CTAs share out the rows and stage the

@@ -155,18 +155,37 @@ __device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Ro
         const int* mem = ct.members + (size_t)rw.seq * sd.W_max + ct.moff[rw.seq * (ct.K + 1) + c];
         float* z = ct.zbuf + ((size_t)rw.seq * ct.K + c) * d;
         const float inv_n = 1.f / (float)n;
-        for (int c4 = threadIdx.x; c4 < (d >> 2); c4 += blockDim.x) {
+        const int n4 = d >> 2;
+        for (int c0 = 0; c0 < n4; c0 += blockDim.x) {            // (uniform trip count: the codec's lanes act together)
+            const int c4 = c0 + threadIdx.x;
+            const bool in = c4 < n4;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            const float4 rf = (ct.hq && in) ? __ldg(reinterpret_cast<const float4*>(ct.z0 + ((size_t)rw.seq * ct.K + c) * d) + c4)
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
             for (int t = 0; t < n; ++t) {
                 const int w = mem[t];
                 const size_t o = (size_t)rw.seq * sd.W_max + w;
-                const float* src;
-                if (sd.within) src = patch[o] ? packet + o * d : hc + o * d;
-                else src = x + ((size_t)rw.seq * sd.rows_per_seq + (window_pos(sd, w) - sd.e0)) * d;      // entry: this forward's row
-                const float4 v = __ldcg(reinterpret_cast<const float4*>(src) + c4);
+                const bool fresh = !sd.within || patch[o];       // a row that enters the cache now: plain values
+                const float* src = !sd.within ? x + ((size_t)rw.seq * sd.rows_per_seq + (window_pos(sd, w) - sd.e0)) * d
+                                              : (patch[o] ? packet + o * d : hc + o * d);
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (ct.hq) {
+                    // the member's STORED value: what the codec makes of a fresh row, or the codes already in the cache
+                    if (fresh) {
+                        if (in) v = __ldcg(reinterpret_cast<const float4*>(src) + c4);
+                        unsigned cd, sb;
+                        v = nvfp4_residual_chunk(v, rf, &cd, &sb);
+                        if (in && ct.fmask && ct.fmask[o])
+                            v = nvfp4_dequant_chunk(*reinterpret_cast<const unsigned short*>(ct.fq + o * (size_t)(d >> 1) + 2 * c4),
+                                                    ct.fs[o * (size_t)(d >> 4) + (c4 >> 2)], rf);
+                    } else if (in) {
+                        const unsigned cd = *reinterpret_cast<const unsigned short*>(ct.hq + o * (size_t)(d >> 1) + 2 * c4);
+                        v = nvfp4_dequant_chunk(cd, ct.hs[o * (size_t)(d >> 4) + (c4 >> 2)], rf);
+                    }
+                } else if (in) v = __ldcg(reinterpret_cast<const float4*>(src) + c4);
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
             }
-            reinterpret_cast<float4*>(z)[c4] = make_float4(acc.x * inv_n, acc.y * inv_n, acc.z * inv_n, acc.w * inv_n);
+            if (in) reinterpret_cast<float4*>(z)[c4] = make_float4(acc.x * inv_n, acc.y * inv_n, acc.z * inv_n, acc.w * inv_n);
         }
         __syncthreads();
         norm_row<T>(z, gain, eps, d, a, nullptr, nullptr, red);
@@ -174,7 +193,59 @@ __device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Ro
     }
     float* xr = x + (size_t)r * d;
     bool kv = true;
-    if (rw.widx >= 0) {
+    if (rw.widx >= 0 && ct.hq) {
+        // ---- NVFP4 residual cache: the row's codes against its cluster's block-entry centroid
+        const size_t o = (size_t)rw.seq * sd.W_max + rw.widx;
+        const float* ref = ct.z0 + ((size_t)rw.seq * ct.K + ct.labels[o]) * d;
+        unsigned char* cq = ct.hq + o * (size_t)(d >> 1);
+        unsigned char* cs = ct.hs + o * (size_t)(d >> 4);
+        const bool patched = sd.within && patch[o] != 0;
+        const bool fresh = !sd.within || patched;              // block entry records the row; a packet row replaces it
+        const bool imposed = fresh && ct.fmask && ct.fmask[o];
+        kv = fresh;
+        const float* src = !sd.within ? xr : packet + o * d;
+        const int n4 = d >> 2;
+        float4 v[NORM_VPT];
+        float ss = 0.f;
+#pragma unroll
+        for (int u = 0; u < NORM_VPT; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            const bool in = c4 < n4;
+            const float4 rf = in ? __ldg(reinterpret_cast<const float4*>(ref) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (fresh) {
+                const float4 raw = in ? __ldcg(reinterpret_cast<const float4*>(src) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+                unsigned cd, sb;
+                float4 q = nvfp4_residual_chunk(raw, rf, &cd, &sb);
+                if (in && imposed) {
+                    cd = *reinterpret_cast<const unsigned short*>(ct.fq + o * (size_t)(d >> 1) + 2 * c4);
+                    sb = ct.fs[o * (size_t)(d >> 4) + (c4 >> 2)];
+                    q = nvfp4_dequant_chunk(cd, sb, rf);
+                }
+                if (in) {
+                    *reinterpret_cast<unsigned short*>(cq + 2 * c4) = (unsigned short)cd;
+                    if ((c4 & 3) == 0) cs[c4 >> 2] = (unsigned char)sb;
+                    // a block-entry forward goes on with the plain row (only later steps read the cache); a refreshed
+                    // row is what the cache now holds
+                    v[u] = sd.within ? q : raw;
+                }
+            } else if (in) {
+                v[u] = nvfp4_dequant_chunk(*reinterpret_cast<const unsigned short*>(cq + 2 * c4), cs[c4 >> 2], rf);
+            }
+            ss += v[u].x * v[u].x + v[u].y * v[u].y + v[u].z * v[u].z + v[u].w * v[u].w;
+        }
+        ss = block_sum(ss, red);
+        const float inv = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+        for (int u = 0; u < NORM_VPT; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            if (c4 < n4) {
+                const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + c4);
+                store4<T>(a + 4 * c4, v[u].x * inv * g.x, v[u].y * inv * g.y, v[u].z * inv * g.z, v[u].w * inv * g.w);
+                if (sd.within) reinterpret_cast<float4*>(xr)[c4] = v[u];
+            }
+        }
+    } else if (rw.widx >= 0) {
         const size_t o = (size_t)rw.seq * sd.W_max + rw.widx;
         float* h = hc + o * d;
         if (sd.within) {
@@ -191,6 +262,15 @@ __device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Ro
     }
     if (threadIdx.x == 0) kvflag[r] = kv ? 1 : 0;
 }
+// Imposed NVFP4 codes written straight into the cache: one block per window row of one layer.
+__global__ void impose_codes_kernel(const unsigned char* fmask, const unsigned char* fq, const unsigned char* fs, unsigned char* hq,
+                                    unsigned char* hs, int d) {
+    const size_t o = blockIdx.x;
+    if (!fmask[o]) return;
+    for (int i = threadIdx.x; i < (d >> 1); i += blockDim.x) hq[o * (size_t)(d >> 1) + i] = fq[o * (size_t)(d >> 1) + i];
+    for (int i = threadIdx.x; i < (d >> 4); i += blockDim.x) hs[o * (size_t)(d >> 4) + i] = fs[o * (size_t)(d >> 4) + i];
+}
+
 template <typename T>
 __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* hc, const float* packet,
                                 const unsigned char* patch, const float* gain, float eps, int d,
@@ -273,6 +353,7 @@ struct KmeansArgs {
     int d, K, iters;
     int* labels; int* zpos; int* zcnt; int* members; int* moff;      // this layer's tables (see ClusterTabs)
     const int* forced_labels;  // [batch][W_max], first entry < 0: not forced (parity replay of another clustering)
+    float* z0;                 // NVFP4 residual cache: [batch][K][d] member means of the plain rows (null: not kept)
     float* cent;               // scratch [batch][2][K][d]: the centres, and the member sums of the running update
 };
 __global__ void __launch_bounds__(KM_THREADS) kmeans_kernel(StepDesc sd, KmeansArgs a) {
@@ -377,6 +458,37 @@ __global__ void __launch_bounds__(KM_THREADS) kmeans_kernel(StepDesc sd, KmeansA
     if (t < K) {
         int o = a.moff[s * (K + 1) + t];
         for (int w = 0; w < W; ++w) if (lab[w] == t) a.members[(size_t)s * sd.W_max + o++] = w;
+    }
+    if (a.z0) {
+        // reference rows of the residual codec: the clusters' centroids as this block entry sees them
+        for (int j = 0; j < K; ++j) {
+            const float inv_n = cnt[j] > 0 ? 1.f / (float)cnt[j] : 0.f;
+            for (int c = t; c < d; c += KM_THREADS) {
+                float acc = 0.f;
+                for (int w = 0; w < W; ++w) if (lab[w] == j) acc += row(w)[c];
+                a.z0[((size_t)s * K + j) * d + c] = acc * inv_n;
+            }
+        }
+    }
+}
+
+// The codec on its own: codes, scales and stored values of rows x against reference rows ref (one CTA per row).
+__global__ void nvfp4_residual_kernel(const float* x, const float* ref, int d, unsigned char* codes, unsigned char* scales, float* deq) {
+    KERNEL_PROLOGUE(19);   // nvfp4_residual_kernel
+    const size_t r = blockIdx.x;
+    const int n4 = d >> 2;
+    for (int c0 = 0; c0 < n4; c0 += blockDim.x) {
+        const int c4 = c0 + threadIdx.x;
+        const bool in = c4 < n4;
+        const float4 v = in ? reinterpret_cast<const float4*>(x + r * d)[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 rf = in ? reinterpret_cast<const float4*>(ref + r * d)[c4] : make_float4(0.f, 0.f, 0.f, 0.f);
+        unsigned cd, sb;
+        const float4 q = nvfp4_residual_chunk(v, rf, &cd, &sb);
+        if (in) {
+            *reinterpret_cast<unsigned short*>(codes + r * (size_t)(d >> 1) + 2 * c4) = (unsigned short)cd;
+            if ((c4 & 3) == 0) scales[r * (size_t)(d >> 4) + (c4 >> 2)] = (unsigned char)sb;
+            reinterpret_cast<float4*>(deq + r * d)[c4] = q;
+        }
     }
 }
 

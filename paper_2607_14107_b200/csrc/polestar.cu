@@ -327,6 +327,8 @@ struct Buffers {
     int* own_flags; int* suffix_flags; int* seq_info; int* head_count; int* suf_seq; int* suf_w; int* stats; int* status;
     int* list_count; float* hidden_keep;
     int* labels; int* zpos; int* zcnt; int* members; int* moff; int* forced_labels; float* zbuf; float* kcent;   // centroid proxies
+    unsigned char* hq; unsigned char* hs; float* z0;                                                             // NVFP4 residual cache
+    unsigned char* fmask; unsigned char* fq; unsigned char* fs;                                                  // imposed codes (checking only)
     // scratch
     Row* rows; unsigned char* kvflag; float* x; float* x1; float* packet; char* a_buf; char* q_buf; char* o_buf;
     char* g_buf; float* kl; int* list; long long* fold_ss; HeadSrc* head_list; char* a_head; float* logits; ConfPart* conf_part;
@@ -418,7 +420,7 @@ struct polestar_ctx {
     std::vector<int> cum;
     StepDesc last_sd;
     int last_act_row_off = 0;
-    bool forced_select = false, forced_commit = false, forced_tokens = false, forced_labels = false;
+    bool forced_select = false, forced_commit = false, forced_tokens = false, forced_labels = false, forced_codes = false;
     int forced_commit_n = 0;
     int* seq_info_host = nullptr;          // pinned: bs * 8 + 8 words
     // launch accounting and optional per-family device timing (POLESTAR_FLAG_PROFILE)
@@ -478,6 +480,10 @@ static bool valid_cfg(const polestar_model* m, const polestar_params* p) {
         if (p->n_clusters < 1 || p->n_clusters > KM_MAX_K || p->cluster_k < 0 || p->kmeans_iters < 1 || p->kmeans_iters > 16) return false;
         if (wmax > SEL_SMALL_W || p->n_clusters > std::max<long long>(wmax, 1) || m->d_model % 4) return false;
     }
+    if (p->flags & POLESTAR_FLAG_NVFP4_HCACHE) {
+        // residuals are taken against cluster centroids; whole warps work on a row's 16-channel groups
+        if (p->select_mode != POLESTAR_SELECT_CLUSTER_TOPK || (p->flags & POLESTAR_FLAG_NOCACHE) || m->d_model % 128) return false;
+    }
     return true;
 }
 
@@ -513,7 +519,8 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(rope, float2, N * (m->head_dim / 2));
     TAKE(kc, char, L * bs * N * dkv * es);
     TAKE(vc, char, L * bs * N * dkv * es);
-    TAKE(hc, float, L * bs * Wm * d);
+    const bool quant = (p->flags & POLESTAR_FLAG_NVFP4_HCACHE) != 0;
+    TAKE(hc, float, quant ? 1 : L * bs * Wm * d);
     TAKE(pprev, float, L * bs * rec * nh * N);
     TAKE(aprev, float, bs * B * nh * N);
     TAKE(pprev_lse, float, L * bs * rec * nh);
@@ -553,6 +560,13 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(forced_labels, int, Kp ? L * bs * Wm : 1);
     TAKE(zbuf, float, Kp ? bs * Kp * d : 1);
     TAKE(kcent, float, Kp ? bs * 2 * Kp * d : 1);
+    TAKE(hq, unsigned char, quant ? L * bs * Wm * (d / 2) : 1);
+    TAKE(hs, unsigned char, quant ? L * bs * Wm * (d / 16) : 1);
+    TAKE(z0, float, quant ? L * bs * Kp * d : 1);
+    const bool imposed = quant && (p->flags & POLESTAR_FLAG_KEEP_HIDDEN);
+    TAKE(fmask, unsigned char, imposed ? L * bs * Wm : 1);
+    TAKE(fq, unsigned char, imposed ? L * bs * Wm * (d / 2) : 1);
+    TAKE(fs, unsigned char, imposed ? L * bs * Wm * (d / 16) : 1);
     TAKE(rows, Row, Mmax);
     TAKE(kvflag, unsigned char, Mmax);
     TAKE(x, float, Mmax * d);
@@ -714,7 +728,7 @@ struct Path {
         for (int l = 0; l < L; ++l) {
             char* kc = b.kc + (size_t)l * bs * N * dkv * es;
             char* vc = b.vc + (size_t)l * bs * N * dkv * es;
-            float* hc = b.hc + (size_t)l * bs * Wm * d;
+            float* hc = (p.flags & POLESTAR_FLAG_NVFP4_HCACHE) ? b.hc : b.hc + (size_t)l * bs * Wm * d;     // (unused with the NVFP4 cache)
             float* pprev = b.pprev + (size_t)l * bs * Wm * m.n_heads * N;
             const bool last = l == L - 1;
             // centroid proxies: this layer's cluster tables; at block entry they are made here, from the layer's input rows
@@ -724,6 +738,14 @@ struct Path {
             if (Kp > 0) {
                 ct.labels = b.labels + (size_t)l * bs * Wm; ct.zpos = b.zpos + (size_t)l * bs * Kp; ct.zcnt = b.zcnt + (size_t)l * bs * Kp;
                 ct.members = b.members + (size_t)l * bs * Wm; ct.moff = b.moff + (size_t)l * bs * (Kp + 1); ct.zbuf = b.zbuf; ct.K = Kp;
+                if (p.flags & POLESTAR_FLAG_NVFP4_HCACHE) {
+                    ct.hq = b.hq + (size_t)l * bs * Wm * (d / 2); ct.hs = b.hs + (size_t)l * bs * Wm * (d / 16);
+                    ct.z0 = b.z0 + (size_t)l * bs * Kp * d;
+                    if (c->forced_codes) {
+                        ct.fmask = b.fmask + (size_t)l * bs * Wm; ct.fq = b.fq + (size_t)l * bs * Wm * (d / 2);
+                        ct.fs = b.fs + (size_t)l * bs * Wm * (d / 16);
+                    }
+                }
                 if (!within) {
                     Scope sc(c, POLESTAR_PROF_SELECT, (double)bs * sd.W * d * 4 * 2 * p.kmeans_iters, 0, 1);
                     KmeansArgs ka;
@@ -731,7 +753,7 @@ struct Path {
                     ka.x = b.x; ka.d = d; ka.K = Kp; ka.iters = p.kmeans_iters;
                     ka.labels = b.labels + (size_t)l * bs * Wm; ka.zpos = b.zpos + (size_t)l * bs * Kp; ka.zcnt = b.zcnt + (size_t)l * bs * Kp;
                     ka.members = b.members + (size_t)l * bs * Wm; ka.moff = b.moff + (size_t)l * bs * (Kp + 1);
-                    ka.forced_labels = b.forced_labels + (size_t)l * bs * Wm; ka.cent = b.kcent;
+                    ka.forced_labels = b.forced_labels + (size_t)l * bs * Wm; ka.cent = b.kcent; ka.z0 = ct.z0;
                     CK(launch_k(kmeans_kernel, dim3(bs), dim3(KM_THREADS), 0, st, sd, ka));
                 }
             }
@@ -1004,6 +1026,10 @@ extern "C" int polestar_step(polestar_ctx* c, polestar_step_info* info) {
         CK(cudaMemsetAsync(c->b.forced_cnt, 0xFF, (size_t)c->m.n_layers * c->p.batch * sizeof(int), c->st));
         c->forced_select = false;
     }
+    if (c->forced_codes) {                        // imposed codes serve one forward
+        CK(cudaMemsetAsync(c->b.fmask, 0, (size_t)c->m.n_layers * c->p.batch * c->W_max, c->st));
+        c->forced_codes = false;
+    }
     if (c->forced_labels && sd.kind != 2) {       // forced labels serve one block-entry forward
         CK(cudaMemsetAsync(c->b.forced_labels, 0xFF, (size_t)c->m.n_layers * c->p.batch * c->W_max * sizeof(int), c->st));
         c->forced_labels = false;
@@ -1255,7 +1281,33 @@ extern "C" int polestar_read(polestar_ctx* c, int32_t what, int32_t layer, void*
             src = c->b.hidden_keep + layer * bs * B * d; sz = bs * B * d * 4; break;
         case POLESTAR_READ_KCACHE: src = c->b.kc + layer * bs * N * dkv * c->es; sz = bs * N * dkv * c->es; break;
         case POLESTAR_READ_VCACHE: src = c->b.vc + layer * bs * N * dkv * c->es; sz = bs * N * dkv * c->es; break;
-        case POLESTAR_READ_HCACHE: src = c->b.hc + layer * bs * Wm * d; sz = bs * Wm * d * 4; break;
+        case POLESTAR_READ_HCACHE:
+            if (c->p.flags & POLESTAR_FLAG_NVFP4_HCACHE) {
+                // NVFP4 residual cache: reference row of the row's cluster + decoded residual, put together on the host
+                const size_t Kp = (size_t)n_proxies(&c->p), n_rows = bs * Wm;
+                std::vector<unsigned char> hq(n_rows * (d / 2)), hs(n_rows * (d / 16));
+                std::vector<float> z0(bs * Kp * d);
+                std::vector<int> lab(n_rows);
+                CK(cudaMemcpyAsync(hq.data(), c->b.hq + layer * hq.size(), hq.size(), cudaMemcpyDeviceToHost, c->st));
+                CK(cudaMemcpyAsync(hs.data(), c->b.hs + layer * hs.size(), hs.size(), cudaMemcpyDeviceToHost, c->st));
+                CK(cudaMemcpyAsync(z0.data(), c->b.z0 + layer * z0.size(), z0.size() * 4, cudaMemcpyDeviceToHost, c->st));
+                CK(cudaMemcpyAsync(lab.data(), c->b.labels + layer * n_rows, n_rows * 4, cudaMemcpyDeviceToHost, c->st));
+                CK(cudaStreamSynchronize(c->st));
+                static const float grid[8] = {0.f, 0.5f, 1.f, 1.5f, 2.f, 3.f, 4.f, 6.f};
+                float* o = (float*)dst;
+                const size_t n_out = std::min(n_rows * d, bytes / 4);
+                for (size_t i = 0; i < n_out; ++i) {
+                    const size_t r = i / d, ch = i % d, sq = r / Wm;
+                    if (lab[r] < 0) { o[i] = 0.f; continue; }
+                    const unsigned sb = hs[r * (d / 16) + ch / 16], e = (sb >> 3) & 15u, mm = sb & 7u;
+                    const float sc = e == 0 ? (float)mm * 0.001953125f : ldexpf(1.f + (float)mm * 0.125f, (int)e - 7);
+                    const unsigned code = (hq[r * (d / 2) + ch / 2] >> (4 * (ch & 1))) & 15u;
+                    const float v = grid[code & 7u] * sc;
+                    o[i] = z0[(sq * Kp + (size_t)lab[r]) * d + ch] + ((code & 8u) ? -v : v);
+                }
+                return POLESTAR_OK;
+            }
+            src = c->b.hc + layer * bs * Wm * d; sz = bs * Wm * d * 4; break;
         case POLESTAR_READ_COMMIT: src = c->b.commit_flags; sz = bs * B * 4; break;
         case POLESTAR_READ_PPREV: {
             // stored as (row, lse) with log-probability = row - lse: put together on the host
@@ -1324,6 +1376,28 @@ extern "C" int polestar_force(polestar_ctx* c, int32_t what, int32_t layer, cons
                                cudaMemcpyHostToDevice, c->st));
         CK(cudaStreamSynchronize(c->st));
         c->forced_labels = true;
+        return POLESTAR_OK;
+    }
+    if (what == POLESTAR_FORCE_HCODES) {
+        const unsigned want = POLESTAR_FLAG_NVFP4_HCACHE | POLESTAR_FLAG_KEEP_HIDDEN;
+        if ((c->p.flags & want) != want) return POLESTAR_E_STATE;
+        if (layer < 0 || layer >= L || n <= 0 || n > Wm || !idx) return POLESTAR_E_INVAL;
+        const size_t d = (size_t)c->m.d_model, W = (size_t)Wm;
+        const unsigned char* blob = (const unsigned char*)idx;
+        const unsigned char* hm = blob; const unsigned char* hq = hm + (size_t)bs * n; const unsigned char* hs = hq + (size_t)bs * n * (d / 2);
+        if (!c->forced_codes) CK(cudaMemsetAsync(c->b.fmask, 0, (size_t)L * bs * W, c->st));
+        for (int s = 0; s < bs; ++s) {
+            const size_t o = ((size_t)layer * bs + s) * W;
+            CK(cudaMemcpyAsync(c->b.fmask + o, hm + (size_t)s * n, n, cudaMemcpyHostToDevice, c->st));
+            CK(cudaMemcpyAsync(c->b.fq + o * (d / 2), hq + (size_t)s * n * (d / 2), (size_t)n * (d / 2), cudaMemcpyHostToDevice, c->st));
+            CK(cudaMemcpyAsync(c->b.fs + o * (d / 16), hs + (size_t)s * n * (d / 16), (size_t)n * (d / 16), cudaMemcpyHostToDevice, c->st));
+        }
+        const size_t o = (size_t)layer * bs * W;
+        impose_codes_kernel<<<(unsigned)(bs * W), 128, 0, c->st>>>(c->b.fmask + o, c->b.fq + o * (d / 2), c->b.fs + o * (d / 16),
+                                                                  c->b.hq + o * (d / 2), c->b.hs + o * (d / 16), (int)d);
+        CK(cudaGetLastError());
+        CK(cudaStreamSynchronize(c->st));
+        c->forced_codes = true;
         return POLESTAR_OK;
     }
     if (what == POLESTAR_FORCE_COMMIT) {
@@ -1505,6 +1579,17 @@ extern "C" int polestar_k_refresh_status(const void* scratch, size_t scratch_byt
     CK(cudaMemcpyAsync(&status, (const char*)scratch + off_status, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     CK(cudaStreamSynchronize((cudaStream_t)stream));
     return status ? POLESTAR_E_TIMEOUT : POLESTAR_OK;
+}
+
+extern "C" int polestar_k_nvfp4_residual(const float* x, const float* ref, int32_t rows, int32_t d, uint8_t* codes,
+                                         uint8_t* scales, float* deq, void* stream) {
+    if (rows < 0 || d <= 0 || d % 128) return POLESTAR_E_INVAL;
+    if (rows == 0) return POLESTAR_OK;
+    if (!x || !ref || !codes || !scales || !deq) return POLESTAR_E_INVAL;
+    if ((((uintptr_t)x | (uintptr_t)ref | (uintptr_t)deq) & 15) || ((uintptr_t)codes & 1)) return POLESTAR_E_INVAL;
+    nvfp4_residual_kernel<<<rows, 256, 0, (cudaStream_t)stream>>>(x, ref, d, codes, scales, deq);
+    CK(cudaGetLastError());
+    return POLESTAR_OK;
 }
 
 // The confidence kernel reads rows with 16-byte loads when the vocabulary is a multiple of four: the base must

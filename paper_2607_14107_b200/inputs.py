@@ -45,6 +45,7 @@ FLAG_SUFFIX_COMMIT = 1 << 1
 FLAG_GE_COMPARE = 1 << 2
 FLAG_NOCACHE = 1 << 3
 FLAG_KEEP_HIDDEN = 1 << 4
+FLAG_NVFP4_HCACHE = 1 << 8
 FLAG_DEFAULT = FLAG_DRIFT_COMMIT | FLAG_SUFFIX_COMMIT | FLAG_GE_COMPARE
 
 TAU_UPD_NEVER = 2**31 - 1

@@ -26,6 +26,43 @@ def setup(name, std=0.02, **kw):
     return m, p, gpu, ora
 
 
+def check_quantised_rows(h_gpu, seq, l, tol, seen, what):
+    """Rows of the NVFP4 residual cache (Appendix "Quantization Format").  The codes are integer decisions taken on
+    hidden states that agree with the oracle's only within the tolerance, so a value next to a decision boundary may
+    land on the neighbouring code (and a group maximum next to an E4M3 boundary on the neighbouring scale).  Hence:
+    every element within the tolerance plus one code step (2 * scale, with 15% for a neighbouring scale) of the
+    oracle's stored value, and all but a small share of them within the tolerance itself."""
+    ref = seq.Z0[l][seq.labels[l]]
+    res = (np.asarray(seq.Hc[l]) - ref).reshape(len(ref), -1, 16)
+    step = np.repeat(np.abs(res).max(axis=2) / 6.0 * 2.0 * 1.15, 16, axis=1)
+    err = np.abs(h_gpu - seq.Hc[l])
+    base = tol + tol * np.abs(seq.Hc[l])
+    assert (err <= base + step).all(), f"{what}: max abs err {err.max():.3e}"
+    seen["q_elems"] = seen.get("q_elems", 0) + err.size
+    seen["q_off"] = seen.get("q_off", 0) + int((err > base).sum())
+
+
+def impose_codes(gpu, ora, p, m):
+    """The oracle's NVFP4 codes of the rows its last step encoded, imposed on the CUDA path: a value next to a code
+    boundary may fall either way when the two sides' hidden states differ in the last places."""
+    d, Wm = m.d_model, gpu.W_max
+    for l in range(m.n_layers):
+        mask = np.zeros((p.batch, Wm), np.uint8)
+        codes = np.zeros((p.batch, Wm, d // 2), np.uint8)
+        scales = np.zeros((p.batch, Wm, d // 16), np.uint8)
+        for s in range(p.batch):
+            hc = ora.seqs[s].trace.get("hcodes", {}).get(l)
+            if hc is None or len(hc[0]) == 0:
+                continue
+            idx, cq, sq = hc
+            cq = np.asarray(cq).astype(np.uint8) & 15
+            mask[s, idx] = 1
+            codes[s, idx] = cq[:, 0::2] | (cq[:, 1::2] << 4)
+            scales[s, idx] = torch.from_numpy(np.ascontiguousarray(sq, np.float32)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+        if mask.any():
+            gpu.force_hcodes(l, mask, codes, scales)
+
+
 def run_forced(name, n_steps, std=0.02, force_labels=True, **kw):
     """The CUDA path replays the oracle's refresh sets and commits; every step's numbers are compared."""
     m, p, gpu, ora = setup(name, std, **kw)
@@ -49,6 +86,8 @@ def run_forced(name, n_steps, std=0.02, force_labels=True, **kw):
                     for s in range(p.batch):
                         lab[s, :len(ora.seqs[s].labels[l])] = ora.seqs[s].labels[l]
                     gpu.force_labels(l, lab[:, :len(ora.seqs[0].labels[l])])
+            if p.flags & I.FLAG_NVFP4_HCACHE:
+                impose_codes(gpu, ora, p, m)
             if tr["kind"] == "within" and tr["refresh"]:
                 for l in range(L):
                     sel = np.full((p.batch, gpu.W_max), -1, np.int32)
@@ -58,6 +97,13 @@ def run_forced(name, n_steps, std=0.02, force_labels=True, **kw):
                     gpu.force_select(l, sel)
             info = gpu.step()
             assert {0: "entry_full", 1: "entry_window", 2: "within"}[info.kind] == tr["kind"]
+        if step == 0 and (p.flags & I.FLAG_NVFP4_HCACHE):
+            # the first block entry ran inside polestar_init: bring its codes in line before anything reads the cache
+            for s in range(p.batch):
+                for l in range(L):
+                    W = len(ora.seqs[s].win)
+                    check_quantised_rows(gpu.read(Bd.READ_HCACHE, l)[s, :W], ora.seqs[s], l, tol, seen, f"entry H l{l}")
+            impose_codes(gpu, ora, p, m)
         for s in range(p.batch):
             trs = ora.seqs[s].trace
             for l in range(L + 1):
@@ -88,7 +134,11 @@ def run_forced(name, n_steps, std=0.02, force_labels=True, **kw):
                 close_h(gpu.read(Bd.READ_VCACHE, l)[s].reshape(ora.seqs[s].Vc[l].shape), ora.seqs[s].Vc[l], tol,
                         f"step {step} V l{l}", depth=l)
                 W = len(ora.seqs[s].win)
-                close_h(gpu.read(Bd.READ_HCACHE, l)[s, :W], ora.seqs[s].Hc[l], tol, f"step {step} H l{l}", depth=l)
+                if p.flags & I.FLAG_NVFP4_HCACHE:
+                    # (codes imposed: only the reference rows' last-place rounding separates the stored values)
+                    close(gpu.read(Bd.READ_HCACHE, l)[s, :W], ora.seqs[s].Hc[l], 1e-5, f"step {step} H l{l}")
+                else:
+                    close_h(gpu.read(Bd.READ_HCACHE, l)[s, :W], ora.seqs[s].Hc[l], tol, f"step {step} H l{l}", depth=l)
             _, conf = O.confidence_rows(trs["logits"], m.mask_id)
             close(gpu.read(Bd.READ_CONF)[s], conf, tol, f"step {step} conf")
         y_before = ora.tokens().copy()
@@ -155,6 +205,20 @@ def test_centroid_proxy_mode_matches_oracle(name, kw):
     # Sec. 4.1 default policy: K-means at block entry, proxy attention of the centroids, cluster top-k -> member rows
     seen = run_forced(name, 24, select_mode=I.SELECT_CLUSTER_TOPK, **kw)
     assert seen["refresh"] >= 2 and seen["clusterings"] >= 2, seen
+
+
+@pytest.mark.parametrize("name,kw,max_off", [
+    ("c1", dict(tau_upd=2, logit_scale=12.0), 2e-3),
+    ("c1b", dict(tau_upd=-1, logit_scale=24.0, tau_suffix=0.5, batch=3, n_clusters=5, cluster_k=2), 5e-2),
+])
+def test_nvfp4_hidden_cache_matches_oracle(name, kw, max_off):
+    # Sec. 4.1: the window's hidden rows kept as NVFP4 residuals against the block-entry centroids; every reader
+    # (proxies, recomputed rows' inputs, the next layer's packet) sees the decoded values on both sides
+    m, p0 = I.config(name)
+    seen = run_forced(name, 24, select_mode=I.SELECT_CLUSTER_TOPK, flags=p0.flags | I.FLAG_NVFP4_HCACHE, **kw)
+    # q_off: elements of the library's own first encoding (inside polestar_init) that landed on a neighbouring code
+    assert seen["refresh"] >= 2 and seen["clusterings"] >= 2 and seen["q_elems"] > 0, seen
+    assert seen["q_off"] <= max_off * seen["q_elems"], seen
 
 
 def test_centroid_proxy_own_clustering_matches_oracle():

@@ -281,3 +281,38 @@ def test_refresh_with_zero_selected_rows_touches_nothing():
                           m.rms_eps, m.rope_theta, scratch[off:])
     torch.cuda.synchronize()
     assert torch.equal(kc.cpu(), kc0) and torch.equal(vc.cpu(), kc0)
+
+
+@pytest.mark.parametrize("rows,d", [(1, 128), (37, 256), (300, 4096)])
+def test_nvfp4_residual_codec_bit_exact(rows, d):
+    # Appendix "Quantization Format": E2M1 codes with one E4M3 scale per 16 channels, float32 arithmetic on both
+    # sides, identical inputs -> identical codes, scales and stored values
+    g = torch.Generator().manual_seed(rows * 131 + d)
+    ref = torch.randn(rows, d, generator=g)
+    mag = torch.exp(torch.randn(rows, d // 16, 1, generator=g) * 3.0).expand(rows, d // 16, 16).reshape(rows, d)
+    x = ref + torch.randn(rows, d, generator=g) * mag * 0.05
+    x[0, :16] = ref[0, :16]                                   # an all-zero group
+    x[0, 16:32] = ref[0, 16:32] + 1e-7                         # below the smallest subnormal scale
+    x[0, 32:48] = ref[0, 32:48] + 1e5                          # saturates the E4M3 scale at 448
+    grid = torch.tensor([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+    mids = torch.tensor([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0])
+    ref[0, 48:64] = 0.0                                        # exact grid points and midpoints at scale 1
+    x[0, 48:56], x[0, 56:64] = grid, -mids
+    xd, rd = x.cuda(), ref.cuda()
+    codes = torch.empty(rows, d // 2, dtype=torch.uint8, device="cuda")
+    scales = torch.empty(rows, d // 16, dtype=torch.uint8, device="cuda")
+    deq = torch.empty(rows, d, device="cuda")
+    Bd.polestar_k_nvfp4_residual(xd, rd, codes, scales, deq)
+    torch.cuda.synchronize()
+    res = (x - ref).numpy()
+    o_codes, o_scale = O.nvfp4_quantize(res)
+    c = codes.cpu().numpy()
+    got = np.stack([c & 15, c >> 4], axis=-1).reshape(rows, d)
+    o_mag = (o_codes & 7)
+    # the sign bit of a zero magnitude carries no information
+    assert np.array_equal(got & 7, o_mag)
+    nz = o_mag > 0
+    assert np.array_equal((got & 8)[nz], (o_codes & 8)[nz])
+    sc = scales.cpu().view(torch.float8_e4m3fn).float().numpy()
+    assert np.array_equal(sc, o_scale)
+    assert np.array_equal(deq.cpu().numpy().astype(np.float64), O.residual_nvfp4_roundtrip(x.numpy(), ref.numpy()))

@@ -6,6 +6,7 @@ import re
 
 import pytest
 
+from oracle import polestar_oracle as O
 from paper_2607_14107_b200 import binding as Bd
 from paper_2607_14107_b200 import build as build_mod
 from paper_2607_14107_b200 import inputs as I
@@ -44,6 +45,25 @@ def test_workspace_bytes(lib):
     m, p = I.config("c1")
     m.n_heads = 3                       # not a multiple of the kv heads
     assert Bd.polestar_workspace_bytes(m, p) == 0
+
+
+def test_workspace_shrinks_with_centroid_proxies_and_the_nvfp4_cache(lib):
+    # Sec. 4.1: stored attention rows per cluster instead of per window row, hidden rows as 4-bit residuals with one
+    # scale byte per 16 channels (9/64 of the fp32 bytes)
+    import dataclasses
+    m, p = I.config("c4")
+    plain = Bd.polestar_workspace_bytes(m, p)
+    pc = dataclasses.replace(p, select_mode=I.SELECT_CLUSTER_TOPK)
+    proxies = Bd.polestar_workspace_bytes(m, pc)
+    assert plain - proxies > 10e9, (plain, proxies)
+    pq = dataclasses.replace(pc, flags=pc.flags | I.FLAG_NVFP4_HCACHE)
+    quantised = Bd.polestar_workspace_bytes(m, pq)
+    W_max = max(sum(len(part) for part in O.window_positions(p, b)) for b in range(p.gen_len // p.block))
+    rows = m.n_layers * p.batch * W_max
+    saved = rows * m.d_model * 4 * (1 - 9 / 64) - m.n_layers * p.batch * pc.n_clusters * m.d_model * 4
+    assert abs((proxies - quantised) - saved) < 0.02 * saved + 4096, (proxies - quantised, saved)
+    # the flag needs the cluster mode (the residuals' reference rows are the centroids)
+    assert Bd.polestar_workspace_bytes(m, dataclasses.replace(p, flags=p.flags | I.FLAG_NVFP4_HCACHE)) == 0
 
 
 def test_init_rejects_bad_arguments_before_using_the_device(lib):
