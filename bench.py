@@ -1,8 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the Polestar decoding hot path on B200.
 
-A "step" is one complete decode of one batch of synthetic prompts at the LLaDA-8B shape
-(prompt 256 + 256 generated tokens, block 32, one token per forward by default), i.e. every
+A "step" is one complete decode of one batch of synthetic prompts (default workload c2: the
+LLaDA-8B shape, prompt 256 + 256 generated tokens, block 32), i.e. every
 row of the hot path: block-entry forwards, within-block steps with drift / select / gathered
 K-V refresh / scatter / attention, and the confidence + drift-event commit.
 
@@ -27,7 +27,9 @@ sys.path.insert(0, ROOT)
 
 METRIC = "tokens/sec at LLaDA-8B shape (1xB200), tokens/forward"
 UNIT = "tokens/s"
-TRAFFIC_OVER_ALGORITHMIC = 1.004   # measured with ncu, see profiles/gemm_sk_kernel_c2.md
+# DRAM traffic of the projection kernels over their algorithmic bytes: NOT measured in this run, scaled from an ncu
+# capture of the same kernels on a 2-layer model at the c2 widths (profiles/gemm_sk_kernel_c2.md: 0.999)
+TRAFFIC_OVER_ALGORITHMIC = 0.999
 
 
 def parse():
@@ -39,6 +41,9 @@ def parse():
     ap.add_argument("--config", default="c2")
     ap.add_argument("--max-steps", type=int, default=0, help="denoising step budget (0: config default)")
     ap.add_argument("--tau-upd", type=int, default=None)
+    ap.add_argument("--select", default="config", choices=["config", "cluster"],
+                    help="cluster: centroid-proxy drift (Sec. 4.1), K = 8 clusters, top 4 refreshed")
+    ap.add_argument("--nvfp4", action="store_true", help="with --select cluster: NVFP4 residual hidden cache")
     ap.add_argument("--layers", type=int, default=0, help="debug: fewer layers (result marked invalid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-profile", action="store_true")
@@ -162,6 +167,9 @@ def run_ours(args):
         p = dataclasses.replace(p, max_steps=args.max_steps)
     if args.tau_upd is not None:
         p = dataclasses.replace(p, tau_upd=args.tau_upd)
+    if args.select == "cluster":
+        p = dataclasses.replace(p, select_mode=I.SELECT_CLUSTER_TOPK,
+                                flags=p.flags | (I.FLAG_NVFP4_HCACHE if args.nvfp4 else 0))
     packed = Bd.make_packed_weights(m, seed=0, device="cuda")
     # one batch of prompts per replica: independent sequences, no exchange between ranks (weak scaling)
     prompt = I.make_prompt(m, p, seed=R.replica_prompt_seed(1, rank))
@@ -226,15 +234,21 @@ def run_ours(args):
 
     (ms, ms2), (gen, gen2, fwd, launches) = R.aggregate([ms, ms2], [gen, gen2, fwd, launches], device="cuda")
 
+    esz = 2 if m.dtype == I.DTYPE_BF16 else 4
+    weight_gb = (m.n_layers * (m.d_model * (m.n_heads + 2 * m.n_kv_heads) * m.head_dim + m.n_heads * m.head_dim * m.d_model
+                               + 3 * m.d_model * m.d_ffn) + m.vocab * m.d_model) * esz / 1e9
     if rank == 0:
         hbm, tf, which = measured_peaks()
         out = {
             "metric": METRIC, "value": R.whole_job_rate(gen, ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if m.dtype == I.DTYPE_BF16 else "f32", "data": "synthetic",
-            "config": {"workload": f"{args.config}: LLaDA-8B shape, batch {p.batch}, prompt {p.prompt_len} + gen {p.gen_len}, "
-                                   f"block {p.block}, {p.max_steps} denoising steps, tau_upd {p.tau_upd}; one replica per GPU",
-                       "layers": m.n_layers, "l2": "inputs larger than L2 (16 GB of weights streamed per forward)",
+            "config": {"workload": f"{args.config}: {I.SHAPES.get(args.config, '?')}, batch {p.batch}, prompt {p.prompt_len} + gen {p.gen_len}, "
+                                   f"block {p.block}, {p.max_steps} denoising steps, tau_upd {p.tau_upd}, "
+                                   f"{'centroid proxies' + (' + NVFP4 hidden cache' if args.nvfp4 else '') if args.select == 'cluster' else 'per-position drift'}"
+                                   f"; one replica per GPU",
+                       "layers": m.n_layers,
+                       "l2": f"inputs larger than L2 ({weight_gb:.1f} GB of weights streamed per forward)",
                        "step": "one full decode of the batch"},
             "tokens_per_forward": gen / max(fwd, 1), "forwards_per_step": fwd / args.steps / world,
             "e2e": {"value": gen2 / (ms2 / 1e3), "unit": UNIT, "h2d_bytes_per_step": p.batch * p.prompt_len * 4,
@@ -258,15 +272,25 @@ def run_ours(args):
             ach_pipe = g_b / (g_ms_timed / 1e3) / 1e9 if g_ms_timed > 0 else 0.0
             # DRAM traffic per launch: ncu (dram__bytes_read + write) over the GEMM launches of one forward gives
             # 1.004 x the algorithmic bytes at these shapes (profiles/gemm_sk_kernel_c2.md); per-launch average.
-            out["roofline"] = {"bound": "hbm", "achieved": ach, "peak": hbm, "unit": "GB/s", "frac": ach / hbm,
+            # which roof binds the projections of this workload: the larger of the two fractions (few rows per
+            # forward stream the weights: HBM; hundreds of rows per forward: the tensor pipe)
+            tfl = g_f / (g_ms / 1e3) / 1e12 if g_ms > 0 else 0.0
+            tensor_bound = tfl / tf > ach / hbm
+            out["roofline"] = {"bound": "tensor" if tensor_bound else "hbm",
+                               "achieved": tfl if tensor_bound else ach, "peak": tf if tensor_bound else hbm,
+                               "unit": "TFLOP/s" if tensor_bound else "GB/s",
+                               "frac": tfl / tf if tensor_bound else ach / hbm,
                                "traffic": TRAFFIC_OVER_ALGORITHMIC * g_b / max(g_calls, 1),
+                               "traffic_source": "scaled from an ncu capture of the same kernels on 2 layers of the c2 widths "
+                                                 "(0.999 x algorithmic), not measured in this run",
                                "algorithmic_bytes_per_launch": g_b / max(g_calls, 1),
-                               "peak_source": which + " (copy bandwidth)",
+                               "hbm_GBps": ach, "hbm_frac": ach / hbm,
+                               "peak_source": which + (" (cuBLAS bf16, sustained)" if tensor_bound else " (copy bandwidth)"),
                                "kernel": "gemm_sk_kernel / gemm_chain_kernel (the five projections of a forward: one stream-K tcgen05 design)",
                                "launches": g_calls, "avg_launch_us": 1e3 * g_ms / max(g_calls, 1),
                                "avg_launch_us_in_pipeline": 1e3 * g_ms_timed / max(g_calls, 1),
-                               "frac_in_pipeline": ach_pipe / hbm,
-                               "tensor_tflops": g_f / (g_ms / 1e3) / 1e12 if g_ms > 0 else 0.0,
+                               "frac_in_pipeline": (tfl * g_ms / g_ms_timed / tf if g_ms_timed > 0 else 0.0) if tensor_bound else ach_pipe / hbm,
+                               "tensor_tflops": tfl, "tensor_frac": tfl / tf,
                                "share_of_device_time": g_ms / total_ms if total_ms > 0 else None}
             out["kernel_families"] = {k: {"ms": round(v["ms"], 3), "calls": int(v["calls"]),
                                           "GBps": round(v["bytes"] / (v["ms"] / 1e3) / 1e9, 1) if v["ms"] > 0 else None}
@@ -300,7 +324,7 @@ def run_reference(args):
     out = {"impl": "reference", "metric": METRIC, "value": best["value"], "unit": UNIT,
            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": steps, "warmup": 0, "ms_per_step": ms,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": f"{args.config}: LLaDA-8B shape, bounded sample on host cores (see cpu_baseline.sample)"},
+           "config": {"workload": f"{args.config}: {I.SHAPES.get(args.config, '?')}, bounded sample on host cores (see cpu_baseline.sample)"},
            "cpu_baseline": best,
            "e2e": {"value": best["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}

@@ -266,23 +266,20 @@ struct ClusterTabs {
 // round to the nearest grid value, ties to the even code, saturating at 6.
 __device__ __forceinline__ float e4m3_round_pos(float x) {          // x >= 0 -> nearest E4M3 value
     x = fminf(x, 448.f);
-    if (!(x > 0.f)) return 0.f;
-    int ex;
-    frexpf(x, &ex);                                                  // x = f 2^ex, f in [0.5, 1)
-    const int e = min(max(ex - 1, -6), 8);
-    const float step = ldexpf(1.f, e - 3);
-    return fminf(rintf(x / step) * step, 448.f);                     // (division by a power of two: exact)
+    if (x < 0.015625f) return rintf(x * 512.f) * 0.001953125f;       // below 2^-6: multiples of 2^-9 (both products exact)
+    // normal range: keep 3 mantissa bits, round to nearest even (a carry moves on to the exponent)
+    unsigned b = __float_as_uint(x);
+    b += 0x7FFFFu + ((b >> 20) & 1u);
+    return fminf(__uint_as_float(b & 0xFFF00000u), 448.f);
 }
 __device__ __forceinline__ unsigned e4m3_bits(float q) {            // q on the E4M3 grid, >= 0
-    if (!(q > 0.f)) return 0u;
     if (q < 0.015625f) return (unsigned)(q * 512.f);                 // subnormal: m 2^-9
-    int ex;
-    const float f = frexpf(q, &ex);                                  // q = f 2^ex
-    return ((unsigned)(ex - 1 + 7) << 3) | (unsigned)((f * 2.f - 1.f) * 8.f);
+    const unsigned b = __float_as_uint(q);
+    return (((b >> 23) - 120u) << 3) | ((b >> 20) & 7u);             // exponent bias 127 -> 7
 }
 __device__ __forceinline__ float e4m3_value(unsigned b) {
     const unsigned e = (b >> 3) & 15u, m = b & 7u;
-    return e == 0 ? (float)m * 0.001953125f : ldexpf(1.f + (float)m * 0.125f, (int)e - 7);
+    return e == 0 ? (float)m * 0.001953125f : __uint_as_float(((e + 120u) << 23) | (m << 20));
 }
 __device__ __forceinline__ unsigned e2m1_code(float r, float s) {   // residual r, group scale s > 0 -> sign | index
     const float y = __fdiv_rn(fabsf(r), s);
@@ -290,10 +287,10 @@ __device__ __forceinline__ unsigned e2m1_code(float r, float s) {   // residual 
     return i | (r < 0.f ? 8u : 0u);
 }
 __device__ __forceinline__ float e2m1_value(unsigned code, float s) {
-    const unsigned i = code & 7u;
-    const float g = i < 4 ? 0.5f * (float)i : (i == 4 ? 2.f : (i == 5 ? 3.f : (i == 6 ? 4.f : 6.f)));
-    const float v = g * s;
-    return (code & 8u) ? -v : v;
+    // index = 2 bits of exponent, 1 of mantissa: 0, .5 | (1 + m / 2) 2^(e - 1)
+    const unsigned e = (code >> 1) & 3u, m = code & 1u;
+    const float g = e == 0 ? 0.5f * (float)m : __uint_as_float(((e + 126u) << 23) | (m << 22));
+    return __uint_as_float(__float_as_uint(g * s) | ((code & 8u) << 28));
 }
 // One 16-byte chunk (4 channels) of a row; the 4 lanes that hold a group of 16 channels call together (lane % 4 =
 // position in the group; every lane of the warp takes part).  Returns the stored value ref + dequant(quant(v - ref));

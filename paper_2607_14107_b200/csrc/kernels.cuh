@@ -156,39 +156,104 @@ __device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Ro
         float* z = ct.zbuf + ((size_t)rw.seq * ct.K + c) * d;
         const float inv_n = 1.f / (float)n;
         const int n4 = d >> 2;
-        for (int c0 = 0; c0 < n4; c0 += blockDim.x) {            // (uniform trip count: the codec's lanes act together)
-            const int c4 = c0 + threadIdx.x;
-            const bool in = c4 < n4;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            const float4 rf = (ct.hq && in) ? __ldg(reinterpret_cast<const float4*>(ct.z0 + ((size_t)rw.seq * ct.K + c) * d) + c4)
-                                            : make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int t = 0; t < n; ++t) {
-                const int w = mem[t];
-                const size_t o = (size_t)rw.seq * sd.W_max + w;
-                const bool fresh = !sd.within || patch[o];       // a row that enters the cache now: plain values
-                const float* src = !sd.within ? x + ((size_t)rw.seq * sd.rows_per_seq + (window_pos(sd, w) - sd.e0)) * d
-                                              : (patch[o] ? packet + o * d : hc + o * d);
-                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (ct.hq) {
-                    // the member's STORED value: what the codec makes of a fresh row, or the codes already in the cache
-                    if (fresh) {
-                        if (in) v = __ldcg(reinterpret_cast<const float4*>(src) + c4);
-                        unsigned cd, sb;
-                        v = nvfp4_residual_chunk(v, rf, &cd, &sb);
-                        if (in && ct.fmask && ct.fmask[o])
-                            v = nvfp4_dequant_chunk(*reinterpret_cast<const unsigned short*>(ct.fq + o * (size_t)(d >> 1) + 2 * c4),
-                                                    ct.fs[o * (size_t)(d >> 4) + (c4 >> 2)], rf);
-                    } else if (in) {
-                        const unsigned cd = *reinterpret_cast<const unsigned short*>(ct.hq + o * (size_t)(d >> 1) + 2 * c4);
-                        v = nvfp4_dequant_chunk(cd, ct.hs[o * (size_t)(d >> 4) + (c4 >> 2)], rf);
-                    }
-                } else if (in) v = __ldcg(reinterpret_cast<const float4*>(src) + c4);
-                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-            }
-            if (in) reinterpret_cast<float4*>(z)[c4] = make_float4(acc.x * inv_n, acc.y * inv_n, acc.z * inv_n, acc.w * inv_n);
+        // the members' row tables go through shared memory in groups, so that the loads of the rows themselves do not
+        // wait on a chain of dependent index loads
+        constexpr int GROUP = 64;
+        __shared__ const float* s_src[GROUP];
+        __shared__ int s_o[GROUP];                               // row of the cache; bit 30: the row enters the cache now
+        float4 acc[NORM_VPT], rf[NORM_VPT];
+#pragma unroll
+        for (int u = 0; u < NORM_VPT; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            rf[u] = (ct.hq && c4 < n4) ? __ldg(reinterpret_cast<const float4*>(ct.z0 + ((size_t)rw.seq * ct.K + c) * d) + c4)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        __syncthreads();
-        norm_row<T>(z, gain, eps, d, a, nullptr, nullptr, red);
+        for (int t0 = 0; t0 < n; t0 += GROUP) {
+            __syncthreads();
+            if (threadIdx.x < GROUP && t0 + threadIdx.x < n) {
+                const int w = mem[t0 + threadIdx.x];
+                const int o = rw.seq * sd.W_max + w;
+                const bool pt = sd.within && patch[o];
+                s_src[threadIdx.x] = !sd.within ? x + ((size_t)rw.seq * sd.rows_per_seq + (window_pos(sd, w) - sd.e0)) * d
+                                                : (pt ? packet + (size_t)o * d : hc + (size_t)o * d);
+                s_o[threadIdx.x] = o | ((!sd.within || pt) ? (1 << 30) : 0);
+            }
+            __syncthreads();
+            const int nb = min(GROUP, n - t0);
+#pragma unroll
+            for (int u = 0; u < NORM_VPT; ++u) {
+                const int c4 = threadIdx.x + u * blockDim.x;
+                const bool in = c4 < n4;
+                if (u * (int)blockDim.x >= n4) continue;         // (the whole block is past the row)
+                // members in ascending window order for every column (deterministic), four at a time: all loads of a
+                // group are issued before the first of them is used
+                for (int t = 0; t < nb; t += 4) {
+                    float4 v[4];
+                    unsigned cd[4], sb[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        cd[k] = sb[k] = 0;
+                        if (t + k < nb && in) {
+                            const int so = s_o[t + k];
+                            const size_t o = (size_t)(so & ~(1 << 30));
+                            const bool fresh = (so >> 30) & 1;
+                            if (!ct.hq || fresh) v[k] = __ldcg(reinterpret_cast<const float4*>(s_src[t + k]) + c4);
+                            if (ct.hq) {
+                                // the member's STORED value: the codes in the cache, or (a row that enters the cache in this
+                                // step) what the codec makes of the plain row, or the codes imposed on it
+                                const bool imposed = fresh && ct.fmask && ct.fmask[o];
+                                const unsigned char* q = imposed ? ct.fq : ct.hq;
+                                const unsigned char* sc = imposed ? ct.fs : ct.hs;
+                                if (!fresh || imposed) {
+                                    cd[k] = *reinterpret_cast<const unsigned short*>(q + o * (size_t)(d >> 1) + 2 * c4);
+                                    sb[k] = sc[o * (size_t)(d >> 4) + (c4 >> 2)];
+                                }
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        if (t + k < nb) {                        // (uniform: the codec's lanes act together)
+                            if (ct.hq) {
+                                const int so = s_o[t + k];
+                                const bool fresh = (so >> 30) & 1;
+                                const bool imposed = fresh && ct.fmask && ct.fmask[(size_t)(so & ~(1 << 30))];
+                                if (fresh && !imposed) {
+                                    unsigned c_, s_;
+                                    v[k] = nvfp4_residual_chunk(v[k], rf[u], &c_, &s_);
+                                } else if (in) {
+                                    v[k] = nvfp4_dequant_chunk(cd[k], sb[k], rf[u]);
+                                }
+                            }
+                            acc[u].x += v[k].x; acc[u].y += v[k].y; acc[u].z += v[k].z; acc[u].w += v[k].w;
+                        }
+                    }
+                }
+            }
+        }
+        // the mean row (kept for read-back) and its RMSNorm, straight from the registers
+        float ss = 0.f;
+#pragma unroll
+        for (int u = 0; u < NORM_VPT; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            acc[u] = make_float4(acc[u].x * inv_n, acc[u].y * inv_n, acc[u].z * inv_n, acc[u].w * inv_n);
+            if (c4 < n4) {
+                reinterpret_cast<float4*>(z)[c4] = acc[u];
+                ss += acc[u].x * acc[u].x + acc[u].y * acc[u].y + acc[u].z * acc[u].z + acc[u].w * acc[u].w;
+            }
+        }
+        ss = block_sum(ss, red);
+        const float inv = rsqrtf(ss / (float)d + eps);
+#pragma unroll
+        for (int u = 0; u < NORM_VPT; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            if (c4 < n4) {
+                const float4 g = __ldg(reinterpret_cast<const float4*>(gain) + c4);
+                store4<T>(a + 4 * c4, acc[u].x * inv * g.x, acc[u].y * inv * g.y, acc[u].z * inv * g.z, acc[u].w * inv * g.w);
+            }
+        }
         return;
     }
     float* xr = x + (size_t)r * d;
@@ -213,6 +278,7 @@ __device__ __forceinline__ void prep_qkv_row(const StepDesc& sd, int r, const Ro
             const bool in = c4 < n4;
             const float4 rf = in ? __ldg(reinterpret_cast<const float4*>(ref) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
             v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (u * (int)blockDim.x >= n4) continue;           // (the whole block is past the row)
             if (fresh) {
                 const float4 raw = in ? __ldcg(reinterpret_cast<const float4*>(src) + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
                 unsigned cd, sb;
@@ -347,126 +413,166 @@ __global__ void prep_refresh_kernel(const T* h, const int* idx, const int* count
 // vectors, an empty cluster keeps its centre); no more rows than clusters: every row its own cluster.
 // All sums run in a fixed order.  K <= KM_MAX_K, W <= KM_MAX_W.
 // ---------------------------------------------------------------------------------------
-constexpr int KM_MAX_K = 16, KM_MAX_W = 1024, KM_THREADS = 512;
+constexpr int KM_MAX_K = 16, KM_MAX_W = 1024, KM_THREADS = 512, KM_CL = 8, KM_SMEM_BYTES = 160 * 1024;
 struct KmeansArgs {
     const float* x;            // entry forward: residual-stream rows of this layer [rows][d]
     int d, K, iters;
+    int chunk;                 // columns of the centres staged in shared memory at a time (multiple of 128; K * chunk floats)
     int* labels; int* zpos; int* zcnt; int* members; int* moff;      // this layer's tables (see ClusterTabs)
     const int* forced_labels;  // [batch][W_max], first entry < 0: not forced (parity replay of another clustering)
     float* z0;                 // NVFP4 residual cache: [batch][K][d] member means of the plain rows (null: not kept)
-    float* cent;               // scratch [batch][2][K][d]: the centres, and the member sums of the running update
+    float* cent;               // scratch [batch][K * d + W_max]: the centres (member sums, not normalised), the rows' 1 / norm
 };
-__global__ void __launch_bounds__(KM_THREADS) kmeans_kernel(StepDesc sd, KmeansArgs a) {
+// A cluster of KM_CL CTAs per sequence: the rows are split over the CTAs for the assignment, the columns for the
+// centre update; cluster barriers (release / acquire) separate the phases, data of other CTAs is read through L2.
+__device__ __forceinline__ void km_cluster_sync() {
+    __syncthreads();
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__global__ void __cluster_dims__(KM_CL, 1, 1) __launch_bounds__(KM_THREADS) kmeans_kernel(StepDesc sd, KmeansArgs a) {
     KERNEL_PROLOGUE(18);   // kmeans_kernel
-    __shared__ float inv_norm[KM_MAX_W];
+    extern __shared__ __align__(16) float Cs[];             // [K][chunk]
+    const int KM_CHUNK = a.chunk;
+    __shared__ float invn[KM_MAX_W];
     __shared__ int lab[KM_MAX_W];
-    __shared__ float red[33];
-    __shared__ int cnt[KM_MAX_K + 1];
-    const int s = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5, nw = KM_THREADS / 32;
+    __shared__ float inv_c[KM_MAX_K];
+    __shared__ int cnt[KM_MAX_K + 1], off[KM_MAX_K + 1];
+    __shared__ unsigned short ord[KM_MAX_W];                 // window rows grouped by cluster, ascending inside a cluster
+    const int s = blockIdx.y, rk = blockIdx.x, t = threadIdx.x, lane = t & 31, warp = t >> 5, nw = KM_THREADS / 32;
     const int W = sd.W, K = a.K, d = a.d;
     auto row = [&](int w) { return a.x + ((size_t)s * sd.rows_per_seq + (window_pos(sd, w) - sd.e0)) * d; };
-    float* C = a.cent + (size_t)s * 2 * K * d;
-    float* Cn = C + (size_t)K * d;
+    // lab[] -> cnt[], off[], ord[] (the whole block calls)
+    auto group_rows = [&]() {
+        __syncthreads();
+        if (t < K) { int n = 0; for (int w = 0; w < W; ++w) n += lab[w] == t; cnt[t] = n; }
+        __syncthreads();
+        if (t == 0) { int o = 0; for (int j = 0; j < K; ++j) { off[j] = o; o += cnt[j]; } off[K] = o; }
+        __syncthreads();
+        if (t < K) { int o = off[t]; for (int w = 0; w < W; ++w) if (lab[w] == t) ord[o++] = (unsigned short)w; }
+        __syncthreads();
+    };
+    float* C = a.cent + (size_t)s * ((size_t)K * d + sd.W_max);
+    float* invn_g = C + (size_t)K * d;
+    int* labels = a.labels + (size_t)s * sd.W_max;
+    const int per = (W + KM_CL - 1) / KM_CL, w_lo = min(W, rk * per), w_hi = min(W, w_lo + per);     // this CTA's rows
+    const int dper = (((d + KM_CL - 1) / KM_CL) + 3) & ~3, c_lo = min(d, rk * dper), c_hi = min(d, c_lo + dper);   // ... and columns
     const int* forced = a.forced_labels ? a.forced_labels + (size_t)s * sd.W_max : nullptr;
     if (forced && forced[0] >= 0) {
-        for (int w = t; w < W; w += KM_THREADS) lab[w] = min(max(forced[w], 0), K - 1);
+        for (int w = w_lo + t; w < w_hi; w += KM_THREADS) labels[w] = min(max(forced[w], 0), K - 1);
     } else if (W <= K) {
-        for (int w = t; w < W; w += KM_THREADS) lab[w] = w;
+        for (int w = w_lo + t; w < w_hi; w += KM_THREADS) labels[w] = w;
     } else {
-        for (int w = warp; w < W; w += nw) {
+        for (int w = w_lo + warp; w < w_hi; w += nw) {
             float ss = 0.f;
             const float* h = row(w);
             for (int c = lane; c < d; c += 32) { const float v = h[c]; ss = fmaf(v, v, ss); }
             ss = warp_sum(ss);
-            if (lane == 0) inv_norm[w] = ss > 0.f ? rsqrtf(ss) : 0.f;
+            if (lane == 0) invn_g[w] = ss > 0.f ? rsqrtf(ss) : 0.f;
         }
-        __syncthreads();
-        for (int j = 0; j < K; ++j) {
+        for (int j = rk; j < K; j += KM_CL) {                                  // starting centres: rows of the window
             const int w0 = (int)(((2 * j + 1) * (long long)W) / (2 * K));       // floor((j + 1/2) W / K)
             const float* h = row(w0);
-            const float inv = inv_norm[w0];
-            for (int c = t; c < d; c += KM_THREADS) C[(size_t)j * d + c] = h[c] * inv;
+            for (int c = t; c < d; c += KM_THREADS) C[(size_t)j * d + c] = h[c];
         }
-        __syncthreads();
+        km_cluster_sync();
+        for (int w = t; w < W; w += KM_THREADS) invn[w] = __ldcg(invn_g + w);
         for (int it = 0; it < a.iters; ++it) {
-            // assignment: a warp per row, the row's dot product with every centre
-            for (int w = warp; w < W; w += nw) {
-                const float* h = row(w);
-                float best = -INFINITY;
-                int bj = 0;
-                for (int j = 0; j < K; ++j) {
-                    const float* cj = C + (size_t)j * d;
-                    float dot = 0.f;
-                    for (int c = lane; c < d; c += 32) dot = fmaf(h[c], cj[c], dot);
-                    dot = warp_sum(dot) * inv_norm[w];
-                    if (dot > best) { best = dot; bj = j; }
+            // ---- assignment of this CTA's rows: a warp per row, the centres through shared memory in column chunks
+            for (int w_base = w_lo; w_base < w_hi || w_base == w_lo; w_base += nw) {
+                const int w = w_base + warp;
+                const bool live = w < w_hi;
+                const float* h = live ? row(w) : a.x;
+                float dot[KM_MAX_K];
+#pragma unroll
+                for (int j = 0; j < KM_MAX_K; ++j) dot[j] = 0.f;
+                float n2 = 0.f;                                                 // warp j: |centre j|^2 (first round only)
+                for (int c0 = 0; c0 < d; c0 += KM_CHUNK) {
+                    const int cw = min(KM_CHUNK, d - c0);
+                    __syncthreads();
+#pragma unroll 8
+                    for (int e = t; e < K * (KM_CHUNK / 4); e += KM_THREADS) {
+                        const int j = e / (KM_CHUNK / 4), q = e - j * (KM_CHUNK / 4);
+                        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (4 * q < cw) v = __ldcg(reinterpret_cast<const float4*>(C + (size_t)j * d + c0) + q);
+                        reinterpret_cast<float4*>(Cs + (size_t)j * KM_CHUNK)[q] = v;
+                    }
+                    __syncthreads();
+                    if (w_base == w_lo && warp < K)
+                        for (int q = lane; q < KM_CHUNK; q += 32) n2 = fmaf(Cs[warp * KM_CHUNK + q], Cs[warp * KM_CHUNK + q], n2);
+                    if (live) {
+#pragma unroll 4
+                        for (int q = lane * 4; q < cw; q += 128) {
+                            const float4 hv = *reinterpret_cast<const float4*>(h + c0 + q);
+#pragma unroll
+                            for (int j = 0; j < KM_MAX_K; ++j) {
+                                if (j < K) {
+                                    const float4 cv = *reinterpret_cast<const float4*>(Cs + j * KM_CHUNK + q);
+                                    dot[j] = fmaf(hv.x, cv.x, fmaf(hv.y, cv.y, fmaf(hv.z, cv.z, fmaf(hv.w, cv.w, dot[j]))));
+                                }
+                            }
+                        }
+                    }
                 }
-                if (lane == 0) lab[w] = bj;
+                if (w_base == w_lo) {
+                    n2 = warp_sum(n2);
+                    if (warp < K && lane == 0) inv_c[warp] = n2 > 0.f ? rsqrtf(n2) : 0.f;
+                }
+                __syncthreads();
+                if (live) {
+                    float best = -INFINITY;
+                    int bj = 0;
+#pragma unroll
+                    for (int j = 0; j < KM_MAX_K; ++j) {
+                        if (j < K) {
+                            const float cs = warp_sum(dot[j]) * inv_c[j] * invn[w];
+                            if (cs > best) { best = cs; bj = j; }          // (lowest cluster on ties)
+                        }
+                    }
+                    if (lane == 0) labels[w] = bj;
+                }
+                if (w_hi <= w_lo) break;
             }
-            __syncthreads();
+            km_cluster_sync();
             if (it + 1 == a.iters) break;          // the centres of the last update are never used
-            // update: every thread owns columns; members are added in ascending row order
-            if (t <= K) cnt[t] = 0;
-            __syncthreads();
-            if (t < K) { int n = 0; for (int w = 0; w < W; ++w) n += lab[w] == t; cnt[t] = n; }
-            __syncthreads();
-            float ssq[KM_MAX_K];
-#pragma unroll
-            for (int j = 0; j < KM_MAX_K; ++j) ssq[j] = 0.f;
-            for (int c = t; c < d; c += KM_THREADS) {
-                float acc[KM_MAX_K];
-#pragma unroll
-                for (int j = 0; j < KM_MAX_K; ++j) acc[j] = 0.f;
-                for (int w = 0; w < W; ++w) {
-                    const float v = row(w)[c] * inv_norm[w];
-                    const int lw = lab[w];
-#pragma unroll
-                    for (int j = 0; j < KM_MAX_K; ++j) acc[j] += (lw == j) ? v : 0.f;
-                }
-#pragma unroll
-                for (int j = 0; j < KM_MAX_K; ++j)
-                    if (j < K && cnt[j] > 0) { Cn[(size_t)j * d + c] = acc[j]; ssq[j] = fmaf(acc[j], acc[j], ssq[j]); }
-            }
-            for (int j = 0; j < K; ++j) {
-                const float n2 = block_sum(ssq[j], red);
-                if (cnt[j] > 0 && n2 > 0.f) {        // (an empty cluster, or one whose unit vectors cancel, keeps its centre)
-                    const float inv = rsqrtf(n2);
-                    for (int c = t; c < d; c += KM_THREADS) C[(size_t)j * d + c] = Cn[(size_t)j * d + c] * inv;
+            // ---- update of this CTA's columns: members added in ascending row order; an empty cluster keeps its centre
+            for (int w = t; w < W; w += KM_THREADS) lab[w] = __ldcg(labels + w);
+            group_rows();
+            for (int c = c_lo + t; c < c_hi; c += KM_THREADS) {
+                for (int j = 0; j < K; ++j) {
+                    if (cnt[j] == 0) continue;
+                    float acc = 0.f;
+#pragma unroll 8
+                    for (int i = off[j]; i < off[j + 1]; ++i) { const int w = ord[i]; acc += row(w)[c] * invn[w]; }
+                    C[(size_t)j * d + c] = acc;
                 }
             }
-            __syncthreads();
+            km_cluster_sync();
         }
     }
-    __syncthreads();
-    // tables: labels, member counts, groups of members, rotary position of every proxy
-    for (int w = t; w < sd.W_max; w += KM_THREADS) a.labels[(size_t)s * sd.W_max + w] = w < W ? lab[w] : -1;
-    if (t < K) {
-        int n = 0;
-        long long sp = 0;
-        for (int w = 0; w < W; ++w) if (lab[w] == t) { ++n; sp += window_pos(sd, w); }
-        cnt[t] = n;
-        a.zcnt[s * K + t] = n;
-        a.zpos[s * K + t] = n > 0 ? (int)((2 * sp + n) / (2 * n)) : -1;       // floor(mean + 1/2)
-    }
-    __syncthreads();
-    if (t == 0) {
-        int off = 0;
-        for (int j = 0; j < K; ++j) { a.moff[s * (K + 1) + j] = off; off += cnt[j]; }
-        a.moff[s * (K + 1) + K] = off;
-    }
-    __syncthreads();
-    if (t < K) {
-        int o = a.moff[s * (K + 1) + t];
-        for (int w = 0; w < W; ++w) if (lab[w] == t) a.members[(size_t)s * sd.W_max + o++] = w;
+    km_cluster_sync();
+    // ---- tables: member counts, groups of members, rotary position of every proxy (first CTA); labels of the unused rows
+    for (int w = t; w < W; w += KM_THREADS) lab[w] = __ldcg(labels + w);
+    group_rows();
+    if (rk == 0) {
+        for (int w = W + t; w < sd.W_max; w += KM_THREADS) labels[w] = -1;
+        if (t < K) {
+            const int n = cnt[t];
+            long long sp = 0;
+            for (int i = off[t]; i < off[t + 1]; ++i) sp += window_pos(sd, ord[i]);
+            a.zcnt[s * K + t] = n;
+            a.zpos[s * K + t] = n > 0 ? (int)((2 * sp + n) / (2 * n)) : -1;       // floor(mean + 1/2)
+        }
+        if (t <= K) a.moff[s * (K + 1) + t] = off[t];
+        for (int i = t; i < W; i += KM_THREADS) a.members[(size_t)s * sd.W_max + i] = ord[i];
     }
     if (a.z0) {
-        // reference rows of the residual codec: the clusters' centroids as this block entry sees them
-        for (int j = 0; j < K; ++j) {
-            const float inv_n = cnt[j] > 0 ? 1.f / (float)cnt[j] : 0.f;
-            for (int c = t; c < d; c += KM_THREADS) {
+        // reference rows of the residual codec: the clusters' centroids as this block entry sees them (this CTA's columns)
+        for (int c = c_lo + t; c < c_hi; c += KM_THREADS) {
+            for (int j = 0; j < K; ++j) {
                 float acc = 0.f;
-                for (int w = 0; w < W; ++w) if (lab[w] == j) acc += row(w)[c];
-                a.z0[((size_t)s * K + j) * d + c] = acc * inv_n;
+#pragma unroll 8
+                for (int i = off[j]; i < off[j + 1]; ++i) acc += row(ord[i])[c];
+                a.z0[((size_t)s * K + j) * d + c] = cnt[j] > 0 ? acc * (1.f / (float)cnt[j]) : 0.f;
             }
         }
     }

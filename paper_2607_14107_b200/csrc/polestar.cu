@@ -559,7 +559,7 @@ static size_t make_plan(const polestar_model* m, const polestar_params* p, Buffe
     TAKE(moff, int, Kp ? L * bs * (Kp + 1) : 1);
     TAKE(forced_labels, int, Kp ? L * bs * Wm : 1);
     TAKE(zbuf, float, Kp ? bs * Kp * d : 1);
-    TAKE(kcent, float, Kp ? bs * 2 * Kp * d : 1);
+    TAKE(kcent, float, Kp ? bs * (Kp * d + Wm) : 1);
     TAKE(hq, unsigned char, quant ? L * bs * Wm * (d / 2) : 1);
     TAKE(hs, unsigned char, quant ? L * bs * Wm * (d / 16) : 1);
     TAKE(z0, float, quant ? L * bs * Kp * d : 1);
@@ -635,6 +635,7 @@ static cudaError_t set_kernel_attributes() {
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV_REFRESH>), gemm_smem);
     PS_ATTR(tc::gemm_chain_kernel<__nv_bfloat16>, gemm_smem);
     PS_ATTR(atc::attention_tc_kernel, (int)atc::smem_bytes(atc::MAX_KT));
+    PS_ATTR(kmeans_kernel, KM_SMEM_BYTES);
     PS_ATTR(attention_simt_kernel<float>, (int)SIMT_ATTN_SMEM_MAX);
     PS_ATTR(attention_simt_kernel<__nv_bfloat16>, (int)SIMT_ATTN_SMEM_MAX);
 #undef PS_ATTR
@@ -754,7 +755,8 @@ struct Path {
                     ka.labels = b.labels + (size_t)l * bs * Wm; ka.zpos = b.zpos + (size_t)l * bs * Kp; ka.zcnt = b.zcnt + (size_t)l * bs * Kp;
                     ka.members = b.members + (size_t)l * bs * Wm; ka.moff = b.moff + (size_t)l * bs * (Kp + 1);
                     ka.forced_labels = b.forced_labels + (size_t)l * bs * Wm; ka.cent = b.kcent; ka.z0 = ct.z0;
-                    CK(launch_k(kmeans_kernel, dim3(bs), dim3(KM_THREADS), 0, st, sd, ka));
+                    ka.chunk = std::min((d + 127) & ~127, (KM_SMEM_BYTES / (Kp * 4)) & ~127);
+                    CK(launch_k(kmeans_kernel, dim3(KM_CL, bs), dim3(KM_THREADS), (size_t)Kp * ka.chunk * 4, st, sd, ka));
                 }
             }
             if (p.flags & POLESTAR_FLAG_KEEP_HIDDEN) {
@@ -842,12 +844,15 @@ struct Path {
             }
             // O projection -> RMSNorm -> gate/up -> down as one persistent kernel when the step is small enough
             bool chained = false;
-            if (is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && M <= tc::BLOCK_T && c->sw.chain) {
+            // (one sequence: its proxy rows are the last rows of the step and need nothing after the attention scores,
+            // so a refresh step with proxies still fits the chained kernel's single row tile)
+            const int Mc = (bs == 1 && Kp > 0 && list) ? M - Kp : M;
+            if (is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && Mc <= tc::BLOCK_T && c->sw.chain) {
                 ChainSpec sp[4];
                 memset(sp, 0, sizeof(sp));
                 sp[0].A = b.o_buf; sp[0].W = c->wo[l]; sp[0].N_out = d; sp[0].K = dq; sp[0].epi = EPI_RESID; sp[0].norm_after = 1;
                 sp[0].e.resid = b.x; sp[0].e.out_f32 = b.x1; sp[0].e.ld_out = d;
-                sp[0].post.kind = 1; sp[0].post.n_rows = M; sp[0].post.d = d; sp[0].post.eps = m.rms_eps; sp[0].post.gain = c->n2[l];
+                sp[0].post.kind = 1; sp[0].post.n_rows = Mc; sp[0].post.d = d; sp[0].post.eps = m.rms_eps; sp[0].post.gain = c->n2[l];
                 sp[0].post.a_out = b.a_buf; sp[0].post.x = b.x1; sp[0].post.list = list; sp[0].post.m_count = m2_count;
                 sp[1].A = b.a_buf; sp[1].W = c->wgu[l]; sp[1].N_out = 2 * F; sp[1].K = d; sp[1].epi = EPI_SWIGLU;
                 sp[1].e.out_t = b.g_buf; sp[1].e.ld_out = F; sp[1].e.m_count = m2_count;
@@ -862,7 +867,7 @@ struct Path {
                         sp[2].e.fold_a = b.a_buf; sp[2].e.fold_gain = c->n1[l + 1]; sp[2].e.fold_ss = b.fold_ss + (size_t)(2 * l + 2) * Mm;
                     }
                 }
-                const double by = ((double)d * dq + 3.0 * F * d) * esd, fl = 2.0 * M * d * (double)dq + 6.0 * Mlive * F * (double)d;
+                const double by = ((double)d * dq + 3.0 * F * d) * esd, fl = 2.0 * Mc * d * (double)dq + 6.0 * Mlive * F * (double)d;
                 // ... and, behind it, the next layer's input staging and QKV projection
                 int n_chain = 3;
                 double by4 = 0, fl4 = 0;
@@ -885,11 +890,11 @@ struct Path {
                 }
                 {
                     Scope sc(c, POLESTAR_PROF_GEMM_GATE_UP, by + (n_chain == 4 ? by4 : 0), fl + (n_chain == 4 ? fl4 : 0), 0);
-                    if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, n_chain, M, st, sf.on ? &sf : nullptr, &chained))) return rc;
+                    if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, n_chain, Mc, st, sf.on ? &sf : nullptr, &chained))) return rc;
                     if (!chained && n_chain == 4) {
                         n_chain = 3;
                         sp[2].norm_after = 0;
-                        if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, 3, M, st, sf.on ? &sf : nullptr, &chained))) return rc;
+                        if ((rc = launch_gemm_chain<__nv_bfloat16>(c->maps, c->gws, sp, 3, Mc, st, sf.on ? &sf : nullptr, &chained))) return rc;
                     }
                 }
                 if (chained) { c->launches += 1; qkv_done = (n_chain == 4); }

@@ -126,6 +126,8 @@ def config(name: str):
     c2  LLaDA-8B shape, batch 1, prompt 256 + gen 256, block 32
     c3  Dream-7B shape (GQA 28/4), batch 4, prompt 512 + gen 512
     c4  long generation on the LLaDA-8B shape, batch 8, 1024 + 1024, block 64
+    c6  short generations on the LLaDA-8B shape (Sec. 5.2, hard-to-parallelise tasks: generation length 32,
+        block 8), batch 1, prompt 128
     """
     if name == "c1":
         m = ModelCfg(2, 256, 4, 4, 64, 1024, 1024, DTYPE_F32, 1e-5, 10000.0)
@@ -142,9 +144,16 @@ def config(name: str):
     elif name == "c4":
         m = ModelCfg(32, 4096, 32, 32, 128, 12288, 126464, DTYPE_BF16, 1e-5, 500000.0)
         p = Params(batch=8, prompt_len=1024, gen_len=1024, block=64, max_steps=1024)
+    elif name == "c6":
+        m = ModelCfg(32, 4096, 32, 32, 128, 12288, 126464, DTYPE_BF16, 1e-5, 500000.0)
+        p = Params(batch=1, prompt_len=128, gen_len=32, block=8, max_steps=32)
     else:
         raise KeyError(name)
     return m, p
+
+
+SHAPES = {"c1": "tiny fp32 model", "c1b": "tiny bf16 model", "c2": "LLaDA-8B shape", "c3": "Dream-7B shape (GQA 28/4)",
+          "c4": "LLaDA-8B shape, long generation", "c6": "LLaDA-8B shape, short generation"}
 
 
 def reduced_depth(m: ModelCfg, n_layers: int) -> ModelCfg:

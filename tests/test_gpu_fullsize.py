@@ -92,9 +92,10 @@ def compare_step(gpu, ora, m, p, step):
         for l in range(L):
             Kc = gpu.read(Bd.READ_KCACHE, l)[s].reshape(ora.seqs[s].Kc[l].shape)
             Vc = gpu.read(Bd.READ_VCACHE, l)[s].reshape(ora.seqs[s].Vc[l].shape)
-            close(Kc, ora.seqs[s].Kc[l], TOL, f"step {step} K l{l}")
-            close(Vc, ora.seqs[s].Vc[l], TOL, f"step {step} V l{l}")
-            close(gpu.read(Bd.READ_HCACHE, l)[s, :W], ora.seqs[s].Hc[l], TOL, f"step {step} H l{l}")
+            # K / V of layer l: the layer's input (l layers deep) through one more normalisation + projection
+            close(Kc, ora.seqs[s].Kc[l], TOL, f"step {step} K l{l}", depth=l + 1)
+            close(Vc, ora.seqs[s].Vc[l], TOL, f"step {step} V l{l}", depth=l + 1)
+            close(gpu.read(Bd.READ_HCACHE, l)[s, :W], ora.seqs[s].Hc[l], TOL, f"step {step} H l{l}", depth=l)
 
 
 def run_reduced_depth(m, p, n_within):
@@ -157,6 +158,16 @@ def test_c4_shape_reduced_depth_matches_oracle():
     p = dataclasses.replace(p, batch=2, max_steps=48, tau_upd=25, flags=p.flags | I.FLAG_KEEP_HIDDEN)
     kinds = run_reduced_depth(m, p, n_within=3)
     assert kinds == ["entry_full", "within", "within_refresh", "entry_window"], kinds
+
+
+def test_c6_short_generation_shape_matches_oracle():
+    # Sec. 5.2 (hard-to-parallelise tasks): generation length 32 with block 8 at the LLaDA-8B widths, depth 2: a
+    # window of 16 + 8 rows, eight active rows per step, a block entry every few forwards
+    m, p = I.config("c6")
+    m = I.reduced_depth(m, 2)
+    p = dataclasses.replace(p, tau_upd=-1, flags=p.flags | I.FLAG_KEEP_HIDDEN)
+    kinds = run_reduced_depth(m, p, n_within=9)
+    assert kinds[0] == "entry_full" and "entry_window" in kinds and "within_refresh" in kinds, kinds
 
 
 @pytest.fixture(scope="module")
