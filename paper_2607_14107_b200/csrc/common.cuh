@@ -224,6 +224,11 @@ struct EpiArgs {
     // epilogue (SWIGLU / QKV) multiplies its rows by rsqrt(ss / d + eps), which commutes with the matrix product.
     void* fold_a; const float* fold_gain; long long* fold_ss;
     const long long* in_ss; float in_eps; int in_d;
+    // RESID / DOWN whose output rows ARE the residual rows (out_f32 == resid, no packet rows in the step): every CTA
+    // adds its part of the product straight onto them with vector reductions in L2 (red.global.add.v4.f32) -- no
+    // published partial tiles, no wait for the other contributors, no reduction pass.  The order of the fp32
+    // additions is then the order of arrival (results agree to rounding, not bit for bit).
+    int accumulate;
 };
 
 constexpr float FOLD_SCALE = 65536.f;

@@ -58,6 +58,10 @@ __device__ __forceinline__ void epi4_dyn(int kind, const EpiArgs& e, int m, int 
     else epilogue4<T, EPI_DOWN>(e, m, n, v);
 }
 __device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+__device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)),
+                 "f"(__uint_as_float(c)), "f"(__uint_as_float(d)) : "memory");
+}
 
 // One word counts the arrivals of the whole grid (spreading it over several words made every poll several
 // dependent acquire loads and was slower).
@@ -134,7 +138,7 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             range(p, kb_total, U, u_begin, u_end);
             const int Gp = ca.p[p].G;
             int n_fix = 0;
-            if (u_end > u_begin) {
+            if (u_end > u_begin && !ca.p[p].e.accumulate) {
                 const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;
                 const bool head_cut = u_begin != tb * kb_total, tail_cut = u_end != (te + 1) * kb_total;
                 int fix_tile[2] = {0, 0};
@@ -286,7 +290,30 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                     warp_live = q * 32 < Mv;
                 }
                 const uint32_t taddr = taddr0 + (uint32_t)((seg & 1) * BLOCK_F);
-                if (whole) {
+                if (P.e.accumulate) {
+                    // this segment's part of the product goes straight onto the residual rows (whole or partial alike)
+                    bool row_ok = live;
+                    if (live && P.epi == EPI_DOWN) row_ok = __ldg(reinterpret_cast<const int4*>(P.e.rows) + t_local).y >= 0;
+                    float* dst = P.e.out_f32 + (size_t)t_local * P.e.ld_out + n0;
+                    if (warp_live) {
+                        for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
+                            uint32_t r[4][16];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * j), r[j]);
+                            tmem_ld_wait();
+                            if (row_ok) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                                    for (int c = 0; c < 16; c += 4)
+                                        red_add_v4(dst + c0 + 16 * j + c, r[j][c], r[j][c + 1], r[j][c + 2], r[j][c + 3]);
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
+                } else if (whole) {
                     if (warp_live) {
                         for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
                             float v[16];

@@ -50,6 +50,8 @@ struct Switches {
     int refresh_simt = 0;    // POLESTAR_REFRESH_SIMT
     int fuse_prep = 0;       // POLESTAR_FUSE_PREP (measured negative result, kept with its test)
     int fold_norm = 0;       // POLESTAR_FOLD_NORM (same)
+    int accumulate = 1;      // POLESTAR_GEMM_ACCUMULATE: O / down projections of the chained kernel add their parts onto
+                             // the residual rows in L2 (0: ordered reduction of published partial tiles, bit-reproducible)
     int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
     int l2promo = (int)CU_TENSOR_MAP_L2_PROMOTION_L2_128B;   // POLESTAR_TMA_L2PROMO
     int gemm_trace = -1;     // POLESTAR_GEMM_TRACE (POLESTAR_TRACE builds)
@@ -73,6 +75,7 @@ static Switches read_switches() {
     w.refresh_simt = env_int("POLESTAR_REFRESH_SIMT", w.refresh_simt);
     w.fuse_prep = env_int("POLESTAR_FUSE_PREP", w.fuse_prep);
     w.fold_norm = env_int("POLESTAR_FOLD_NORM", w.fold_norm);
+    w.accumulate = env_int("POLESTAR_GEMM_ACCUMULATE", w.accumulate);
     w.chain_qkv = env_int("POLESTAR_CHAIN_QKV", w.chain_qkv);
     w.l2promo = env_int("POLESTAR_TMA_L2PROMO", w.l2promo);
     w.gemm_trace = env_int("POLESTAR_GEMM_TRACE", w.gemm_trace);
@@ -850,14 +853,18 @@ struct Path {
             if (is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && Mc <= tc::BLOCK_T && c->sw.chain) {
                 ChainSpec sp[4];
                 memset(sp, 0, sizeof(sp));
+                // (in-place variant: the product is added onto the residual rows themselves, x doubles as x1)
+                const bool acc = c->sw.accumulate && !fold;
+                float* x1 = acc ? b.x : b.x1;
                 sp[0].A = b.o_buf; sp[0].W = c->wo[l]; sp[0].N_out = d; sp[0].K = dq; sp[0].epi = EPI_RESID; sp[0].norm_after = 1;
-                sp[0].e.resid = b.x; sp[0].e.out_f32 = b.x1; sp[0].e.ld_out = d;
+                sp[0].e.resid = b.x; sp[0].e.out_f32 = x1; sp[0].e.ld_out = d; sp[0].e.accumulate = acc ? 1 : 0;
                 sp[0].post.kind = 1; sp[0].post.n_rows = Mc; sp[0].post.d = d; sp[0].post.eps = m.rms_eps; sp[0].post.gain = c->n2[l];
-                sp[0].post.a_out = b.a_buf; sp[0].post.x = b.x1; sp[0].post.list = list; sp[0].post.m_count = m2_count;
+                sp[0].post.a_out = b.a_buf; sp[0].post.x = x1; sp[0].post.list = list; sp[0].post.m_count = m2_count;
                 sp[1].A = b.a_buf; sp[1].W = c->wgu[l]; sp[1].N_out = 2 * F; sp[1].K = d; sp[1].epi = EPI_SWIGLU;
                 sp[1].e.out_t = b.g_buf; sp[1].e.ld_out = F; sp[1].e.m_count = m2_count;
                 sp[2].A = b.g_buf; sp[2].W = c->wd[l]; sp[2].N_out = d; sp[2].K = F; sp[2].epi = EPI_DOWN;
-                sp[2].e.rows = b.rows; sp[2].e.list = list; sp[2].e.m_count = m2_count; sp[2].e.resid = b.x1; sp[2].e.out_f32 = b.x;
+                sp[2].e.rows = b.rows; sp[2].e.list = list; sp[2].e.m_count = m2_count; sp[2].e.resid = x1; sp[2].e.out_f32 = b.x;
+                sp[2].e.accumulate = (acc && !list) ? 1 : 0;      // (steps with packet rows keep the ordered epilogue)
                 sp[2].e.packet = b.packet; sp[2].e.W_max = Wm; sp[2].e.within = within; sp[2].e.ld_out = d;
                 if (fold) {
                     sp[0].norm_after = 0;
