@@ -20,6 +20,7 @@
 #include "attn_mma.cuh"
 #include "gemm_tc.cuh"
 #include "attn_tc.cuh"
+#include "attn_stream.cuh"
 #include "gemm_chain.cuh"
 #include "kernels.cuh"
 
@@ -306,6 +307,40 @@ static int launch_attention_tc(MapCache& maps, const AttnArgs& a, cudaStream_t s
     const size_t smem = atc::smem_bytes(g.kt);
     // (always a cluster launch, also for a single key range: the kernel addresses its own CTA through the cluster window)
     CK(launch_k_cluster(atc::attention_tc_kernel, grid, dim3(atc::THREADS), smem, st, (unsigned)g.cl, *mq, *mk, *mv, g));
+    return POLESTAR_OK;
+}
+
+// The streaming form (attn_stream.cuh): one CTA per (128 rows, head) walks all key tiles; any number of keys.
+static bool attention_stream_applies(const AttnArgs& a) {
+    return a.head_dim == ast::DH && a.N > 0 && (a.n_heads * a.head_dim) % 64 == 0 && (a.n_kv * a.head_dim) % 64 == 0;
+}
+// Which of the two tensor-core kernels: the streaming one as soon as its grid (row tiles x heads x sequences) fills a
+// good part of the GPU -- block entries, batches, long sequences (measured: 512 x 512 keys 43 us against 80 us,
+// 2048 x 2048 keys 0.6 ms against 1.4 ms) -- or the keys exceed what a cluster of key ranges covers; the cluster
+// kernel for the small steps of one short sequence, where spreading the keys over SMs wins (128 x 512: 20 us against 37 us).
+static bool attention_prefers_stream(const AttnArgs& a) {
+    const int batch = a.batch > 0 ? a.batch : 1;
+    const int rps = a.rows_per_seq > 0 ? a.rows_per_seq : a.n_rows;
+    const long long ctas = (long long)((rps + ast::ROWS - 1) / ast::ROWS) * batch * a.n_heads;
+    return ctas >= 64 || a.N > atc::MAX_N;
+}
+static int launch_attention_stream(MapCache& maps, const AttnArgs& a, cudaStream_t st, int* status) {
+    if (a.n_rows <= 0) return POLESTAR_OK;
+    ast::Args g;
+    memset(&g, 0, sizeof(g));
+    g.a = a;
+    const int batch = a.batch > 0 ? a.batch : 1;
+    g.rows_per_seq = a.rows_per_seq > 0 ? a.rows_per_seq : a.n_rows;
+    g.tiles_per_seq = (g.rows_per_seq + ast::ROWS - 1) / ast::ROWS;
+    g.status = status;
+    const int dq = a.n_heads * a.head_dim, dkv = a.n_kv * a.head_dim;
+    const int kv_batch = a.rows ? batch : 1;
+    const CUtensorMap* mq = maps.get(a.q, (uint64_t)a.n_rows, (uint64_t)dq, ast::ROWS);
+    const CUtensorMap* mk = maps.get3(a.kc, (uint64_t)kv_batch, (uint64_t)a.N, (uint64_t)dkv);
+    const CUtensorMap* mv = maps.get3(a.vc, (uint64_t)kv_batch, (uint64_t)a.N, (uint64_t)dkv);
+    if (!mq || !mk || !mv) return POLESTAR_E_CUDA;
+    dim3 grid((unsigned)(g.tiles_per_seq * batch), (unsigned)a.n_heads);
+    CK(launch_k(ast::attention_stream_kernel, grid, dim3(ast::THREADS), ast::smem_bytes(), st, *mq, *mk, *mv, g));
     return POLESTAR_OK;
 }
 
@@ -639,6 +674,7 @@ static cudaError_t set_kernel_attributes() {
     PS_ATTR(tc::gemm_chain_kernel<__nv_bfloat16>, gemm_smem);
     PS_ATTR(atc::attention_tc_kernel, (int)atc::smem_bytes(atc::MAX_KT));
     PS_ATTR(kmeans_kernel, KM_SMEM_BYTES);
+    PS_ATTR(ast::attention_stream_kernel, (int)ast::smem_bytes());
     PS_ATTR(attention_simt_kernel<float>, (int)SIMT_ATTN_SMEM_MAX);
     PS_ATTR(attention_simt_kernel<__nv_bfloat16>, (int)SIMT_ATTN_SMEM_MAX);
 #undef PS_ATTR
@@ -677,6 +713,9 @@ struct Path {
             // layer at the 8B shape), everywhere else the tensor-core kernel does.
             const bool records = a.pprev != nullptr || a.aprev != nullptr;
             const bool few_rows = !records && a.rows_per_seq <= 64 && a.N <= 1024 && c->sw.attn_kernel == 0;
+            if (attention_stream_applies(a) && !few_rows &&
+                (c->sw.attn_kernel == 9 || (c->sw.attn_kernel == 0 && attention_prefers_stream(a))))
+                return launch_attention_stream(c->maps, a, c->st, c->b.status);
             if ((c->sw.attn_kernel == 0 || c->sw.attn_kernel == 8) && attention_tc_applies(a) && !few_rows)
                 return launch_attention_tc(c->maps, a, c->st, c->b.status);
             if (a.cluster_K > 0 && (a.pprev || a.aprev)) goto simt;      // the warp-level kernels do not know proxy rows
@@ -1455,6 +1494,12 @@ extern "C" int polestar_k_attention(const void* q, const void* k, const void* v,
     if (rc) return rc;
     const Switches sw = stand_alone_switches();
     if (dtype == POLESTAR_BF16 && head_dim == 128 && !sw.attn_simt) {
+        if (attention_stream_applies(a) && (sw.attn_kernel == 9 || (sw.attn_kernel == 0 && attention_prefers_stream(a))) &&
+            !((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v)) & 15)) {
+            MapCache maps;
+            maps.l2promo = sw.l2promo;
+            return launch_attention_stream(maps, a, st, nullptr);
+        }
         if ((sw.attn_kernel == 0 || sw.attn_kernel == 8) && attention_tc_applies(a) &&
             !((((uintptr_t)q | (uintptr_t)k | (uintptr_t)v)) & 15)) {
             MapCache maps;                 // the three tensor maps of this call

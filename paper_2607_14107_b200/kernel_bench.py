@@ -128,9 +128,12 @@ def bench_hidden_delta(quick):
 
 
 def bench_drift(quick):
-    # window rows of one layer of the 8B shape (W = 96, N = 512) and of the long config (W = 192, N = 2048)
+    # window rows of one layer of the 8B shape (W = 96, N = 512) and of the long config (W = 192, N = 2048);
+    # --quick: the 8B-shape cases only (a small case for profiler captures)
     for name, R, N, nh, n_copy in (("c2", 96, 512, 32, 24), ("c2 window+block", 128, 512, 32, 24), ("c2 block entry", 512, 512, 32, 8),
                                    ("c4 per sequence", 192, 2048, 32, 4), ("c4 block entry", 2048, 2048, 32, 2)):
+        if quick and not name.startswith("c2"):
+            continue
         dh = 128
         q = [I.normal_tensor(I.tensor_key(5, c, 1), (R, nh * dh), 1.0, torch.bfloat16, "cuda") for c in range(n_copy)]
         k = [I.normal_tensor(I.tensor_key(5, c, 2), (N, nh * dh), 1.0, torch.bfloat16, "cuda") for c in range(n_copy)]

@@ -244,7 +244,7 @@ def test_c1b_bf16_norm_staging_inside_the_gemm_tail(monkeypatch):
     assert seen["refresh"] > 3
 
 
-@pytest.mark.parametrize("variant", ["0", "5"])
+@pytest.mark.parametrize("variant", ["0", "5", "9"])
 def test_c1b_long_ragged_sequence(monkeypatch, variant):
     # N = 1100 + 64 > 1024 keys: the two-pass attention kernel (automatic choice) and the 64-row-tile kernel
     # (forced) inside the decoding loop; the prompt length is not a multiple of the block size
@@ -273,6 +273,18 @@ def test_c1b_bf16_separate_launches(monkeypatch):
     monkeypatch.setenv("POLESTAR_CHAIN", "0")
     seen = run_forced("c1b", 10, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5)
     assert seen["refresh"] > 3
+
+
+@pytest.mark.parametrize("kw", [
+    dict(tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5, batch=3),
+    dict(tau_upd=-1, logit_scale=24.0, tau_suffix=0.5, batch=2, select_mode=I.SELECT_CLUSTER_TOPK, n_clusters=5, cluster_k=2),
+])
+def test_c1b_streaming_attention_kernel(monkeypatch, kw):
+    # the streaming tensor-core attention kernel (one CTA per row tile and head, two passes over the key tiles) on every
+    # step of a decode: block entries (recorded rows), plain steps, refresh steps with stored rows / proxy rows
+    monkeypatch.setenv("POLESTAR_ATTN_KERNEL", "9")
+    seen = run_forced("c1b", 12, **kw)
+    assert seen["refresh"] > 3 and seen["entry_window"] >= 0
 
 
 def test_c1b_bf16_simt_gemm_path():

@@ -52,6 +52,14 @@ def test_attention_drift_matches_oracle(dtype, R, N, nh, nkv, dh):
     (8, 200, 2048, 8, 8),          # the long-sequence shape: 2 x 8 key tiles
     (8, 130, 1024, 2, 2),          # eight key ranges of one tile
     (8, 64, 402, 2, 1),            # key count not a multiple of four (scalar access to the stored rows)
+    # streaming tensor-core kernel (one CTA per row tile and head walks the key tiles twice)
+    (9, 5, 37, 2, 2),              # fewer rows and keys than one tile
+    (9, 128, 512, 2, 2),           # one full row tile, four key tiles
+    (9, 37, 200, 4, 2),            # ragged rows and keys, GQA
+    (9, 150, 1100, 2, 1),          # two row tiles, nine key tiles (odd count: the accumulators swap roles between the passes)
+    (9, 200, 2048, 8, 8),          # the long-sequence shape
+    (9, 64, 402, 2, 1),            # key count not a multiple of four
+    (9, 70, 3000, 2, 2),           # more keys than the cluster kernel takes
 ])
 def test_attention_kernel_variants(monkeypatch, variant, R, N, nh, nkv):
     monkeypatch.setenv("POLESTAR_ATTN_KERNEL", str(variant))
