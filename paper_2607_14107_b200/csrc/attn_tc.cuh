@@ -441,9 +441,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const bool in = valid && (k16 + i < a.N);
-                        const float t = __uint_as_float(r[u][i]) * scale2;
+                        const float t = __fmul_rn(__uint_as_float(r[u][i]), scale2);     // (rounded products, never fused into the
+                                                                                         // subtraction from the stored value below)
                         const float p = in ? ex2(t - lse2) : 0.f;      // rows that are not valid hand zeros to the tensor core
-                        s_nat[i] = t * LN2_F;
+                        s_nat[i] = __fmul_rn(t, LN2_F);
                         if (use_old && in) A = fmaf(p, s_nat[i] - old[16 * u + i], A);
                         pr[i] = p;
                     }
