@@ -145,6 +145,112 @@ def oracle_sample(m, p, device_for_inputs):
                        f"extrapolated to {m.n_layers} layers: {t_full:.1f}s per forward, {tpf:.1f} tokens per forward")}
 
 
+# ----------------------------------------------------------------------------- refresh microbench (c5)
+C5_METRIC = "refreshed rows/s, refresh microbench on the LLaDA-8B layer shape (4096 x 4096 cache, batch 1)"
+C5_FRACS = (0.01, 0.05)
+
+
+def c5_oracle(dev):
+    """The oracle's select -> gather -> QKV projection -> RoPE -> scatter chain on the microbench's inputs, timed
+    once at refresh fractions 1 % and 5 % (larger fractions are the same matmul with more rows)."""
+    import numpy as np
+    import torch
+    from oracle import polestar_oracle as O
+    from paper_2607_14107_b200 import inputs as I
+    d, nh, dh, P = 4096, 32, 128, 4096
+    m = I.ModelCfg(1, d, nh, nh, dh, 64, 1024, I.DTYPE_BF16, 1e-5, 500000.0)
+    w = I.make_weights(m, seed=10, device=dev, with_globals=False)["layers"][0]
+    wl = {n: w[n].detach().to("cpu", torch.float32).numpy() for n in ("wq", "wk", "wv")}
+    norm = np.ones(d)
+    h, drift = I.make_refresh_inputs(1, P, d, device=dev)
+    hn = h[0].detach().to("cpu", torch.float32).numpy().astype(np.float64)
+    kc = np.zeros((P, nh, dh)); vc = np.zeros((P, nh, dh))
+    cores = os.cpu_count() or 1
+    torch.set_num_threads(cores)
+    out = {}
+    for frac in C5_FRACS:
+        k = I.refresh_count(frac)
+        t0 = time.perf_counter()
+        O.refresh_chain(hn, drift[0].cpu().numpy(), k, wl["wq"], wl["wk"], wl["wv"], norm, 1e-5, 500000.0, nh, nh, dh, kc, vc)
+        out[frac] = (k, time.perf_counter() - t0)
+    return out, cores
+
+
+def run_c5(args):
+    """`--config c5`: the stand-alone refresh chain (polestar_k_select + polestar_k_refresh) at 1 % and 5 % of a
+    4096-position cache, with the oracle's chain on the host cores beside it.  One step = one chain call."""
+    import torch
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2607_14107_b200 import inputs as I
+    if args.impl == "reference":
+        res, cores = c5_oracle("cuda" if torch.cuda.is_available() else "cpu")
+        k, t = res[0.05]
+        sample = "; ".join(f"{int(f * 100)} %: {kk} rows in {tt:.2f} s" for f, (kk, tt) in res.items())
+        print(json.dumps({"impl": "reference", "metric": C5_METRIC, "value": k / t, "unit": "rows/s", "n_gpus": 1, "steps": 1,
+                          "warmup": 0, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                          "dtype": "f64", "data": "synthetic", "config": {"workload": "c5: refresh fraction 5 % (205 rows), batch 1"},
+                          "cpu_baseline": {"value": k / t, "unit": "rows/s", "cores": cores, "kind": "oracle", "sample": sample},
+                          "e2e": {"value": k / t, "unit": "rows/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}), flush=True)
+        return
+    from paper_2607_14107_b200 import binding as Bd
+    d, nh, dh, P = 4096, 32, 128, 4096
+    m = I.ModelCfg(1, d, nh, nh, dh, 64, 1024, I.DTYPE_BF16, 1e-5, 500000.0)
+    n_w = 4                                          # rotating weight copies: 4 x 100 MB > L2
+    wq = []
+    for c in range(n_w):
+        w = I.make_weights(m, seed=10 + c, device="cuda", with_globals=False)["layers"][0]
+        perm = Bd.rope_interleave_index(dh).cuda()
+        q = w["wq"].view(nh, dh, d)[:, perm].reshape(nh * dh, d)
+        kk = w["wk"].view(nh, dh, d)[:, perm].reshape(nh * dh, d)
+        wq.append(Bd.tile_major(torch.cat([q, kk, w["wv"]], 0)))
+    norm = torch.ones(d, device="cuda")
+    h, drift = I.make_refresh_inputs(1, P, d, device="cuda")
+    kc = torch.zeros((1, P, nh * dh), dtype=torch.bfloat16, device="cuda")
+    vc = torch.zeros_like(kc)
+    full_idx = torch.zeros((1, P), dtype=torch.int32, device="cuda")
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    hbm, tf, which = measured_peaks()
+    res = {}
+    for frac in C5_FRACS:
+        k = I.refresh_count(frac)
+        idx = torch.zeros((1, k), dtype=torch.int32, device="cuda")
+        scratch = torch.empty(Bd.polestar_k_refresh_scratch_bytes(1, k, d, nh, nh, dh) + 1024, dtype=torch.uint8, device="cuda")
+        scratch = scratch[(-scratch.data_ptr()) % 1024:]
+
+        def chain(i):
+            Bd.polestar_k_select(drift, I.SELECT_TOPK_COUNT, k, 0.0, 0.0, full_idx, cnt)
+            idx.copy_(full_idx[:, :k])
+            Bd.polestar_k_refresh(h, idx, cnt, wq[i % n_w], norm, kc, vc, None, k, nh, nh, dh, 1e-5, 500000.0, scratch)
+        for i in range(max(3, args.warmup)):
+            chain(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps * 10):
+            chain(i)
+        e1.record()
+        torch.cuda.synchronize()
+        res[frac] = (k, e0.elapsed_time(e1) / (args.steps * 10))
+    k, ms = res[0.05]
+    by = 3 * d * d * 2 + k * d * 2 + 2 * k * d * 2
+    out = {"metric": C5_METRIC, "value": k / (ms / 1e3), "unit": "rows/s", "n_gpus": 1, "steps": args.steps * 10, "warmup": max(3, args.warmup),
+           "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": "c5: refresh fraction 5 % (205 rows), batch 1", "l2": "four rotating 100 MB weight copies (> L2)",
+                      "other_fractions": {f"{int(f * 100)}%": {"rows": kk, "us": round(t * 1e3, 2)} for f, (kk, t) in res.items()}},
+           "roofline": {"bound": "hbm", "achieved": by / (ms / 1e3) / 1e9, "peak": hbm, "unit": "GB/s", "frac": by / (ms / 1e3) / 1e9 / hbm,
+                        "traffic": None, "peak_source": which + " (copy bandwidth)", "kernel": "select + prep_refresh + gemm_sk_kernel<EPI_QKV_REFRESH>"},
+           "e2e": None, "gpu_launches": args.steps * 10 * 3}
+    if not args.no_cpu_baseline:
+        cres, cores = c5_oracle("cuda")
+        ck, ct = cres[0.05]
+        out["cpu_baseline"] = {"value": ck / ct, "unit": "rows/s", "cores": cores, "kind": "oracle",
+                               "sample": "; ".join(f"{int(f * 100)} %: {kk} rows in {tt:.2f} s" for f, (kk, tt) in cres.items())}
+    print(json.dumps(out), flush=True)
+
+
 # ----------------------------------------------------------------------------- our arm
 def run_ours(args):
     import numpy as np
@@ -333,7 +439,9 @@ def run_reference(args):
 
 if __name__ == "__main__":
     a = parse()
-    if a.impl == "reference":
+    if a.config == "c5":
+        run_c5(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         run_ours(a)
