@@ -173,7 +173,7 @@ __host__ __device__ inline uint32_t instr_desc_bf16(int m, int n) {
 struct SkArgs {
     int M, N_out, K, stages;
     int tiles_f, tiles_t;
-    float* partial;     // [2 * gridDim.x][BLOCK_T][BLOCK_F] fp32
+    float* partial;     // [2 * gridDim.x][tokens per CTA tile][BLOCK_F] fp32
     int* tile_counter;  // arrivals [tile] and, done_offset further on, finished shares [tile]; zero before
                         // launch, zero again after
     int done_offset;
@@ -238,7 +238,11 @@ struct SelFuse {
     StepSelArgs a;
 };
 
-template <typename T, int EPI>
+// TT = 128-row halves of a token tile.  TT = 2 (steps of several hundred rows, where the operands come from L2 and
+// the tensor pipe is the limit): a CTA tile is 256 tokens x 256 features, two MMAs per k step share one weight tile, so
+// a k block costs 64 KB of operands for twice the work of the 48 KB of TT = 1; both accumulators (2 x 256 columns) fill
+// the tensor memory, so the epilogue of a segment no longer overlaps the next segment's MMAs.
+template <typename T, int EPI, int TT = 1>
 __global__ void __launch_bounds__(FIX_THREADS, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                SkArgs g, EpiArgs e, PostArgs post, SelFuse sf) {
@@ -251,6 +255,9 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     __shared__ int fx_n;
     __shared__ volatile int fx_ready;
 
+    constexpr int BT = BLOCK_T * TT;                       // tokens per CTA tile
+    constexpr uint32_t A_BYTES_T = A_BYTES * TT;           // activations of a stage: TT boxes of [128][64]
+    constexpr uint32_t STAGE_T = A_BYTES_T + W_BYTES;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int G = gridDim.x, cta = blockIdx.x;
     if (threadIdx.x == 0) SK_STAMP(0);
@@ -372,27 +379,31 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             };
             It iw = start();
             for (int i = 0; i < pre; ++i, advance(iw)) {
-                mbar_expect_tx(full0 + 8 * i, STAGE_BYTES);
-                if (g.w_stream) tma_load_2d_hint(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0,
+                mbar_expect_tx(full0 + 8 * i, STAGE_T);
+                if (g.w_stream) tma_load_2d_hint(smem_base + i * STAGE_T + A_BYTES_T, &map_w, full0 + 8 * i, 0,
                                                  (iw.f * kb_total + iw.kb) * BLOCK_F, pol);
-                else tma_load_2d(smem_base + i * STAGE_BYTES + A_BYTES, &map_w, full0 + 8 * i, 0, (iw.f * kb_total + iw.kb) * BLOCK_F);
+                else tma_load_2d(smem_base + i * STAGE_T + A_BYTES_T, &map_w, full0 + 8 * i, 0, (iw.f * kb_total + iw.kb) * BLOCK_F);
             }
             pdl_wait();
             SK_STAMP(2);
             {
                 It ia = start();
                 for (int i = 0; i < pre; ++i, advance(ia))
-                    tma_load_2d(smem_base + i * STAGE_BYTES, &map_a, full0 + 8 * i, ia.kb * BLOCK_K, ia.t * BLOCK_T);
+#pragma unroll
+                    for (int hh = 0; hh < TT; ++hh)
+                        tma_load_2d(smem_base + i * STAGE_T + hh * A_BYTES, &map_a, full0 + 8 * i, ia.kb * BLOCK_K, ia.t * BT + hh * BLOCK_T);
             }
             for (int i = pre; i < n_units; ++i, advance(iw)) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
-                const uint32_t dst = smem_base + s * STAGE_BYTES;
-                mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
-                if (g.w_stream) tma_load_2d_hint(dst + A_BYTES, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F, pol);
-                else tma_load_2d(dst + A_BYTES, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F);
-                tma_load_2d(dst, &map_a, full0 + 8 * s, iw.kb * BLOCK_K, iw.t * BLOCK_T);
+                const uint32_t dst = smem_base + s * STAGE_T;
+                mbar_expect_tx(full0 + 8 * s, STAGE_T);
+                if (g.w_stream) tma_load_2d_hint(dst + A_BYTES_T, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F, pol);
+                else tma_load_2d(dst + A_BYTES_T, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F);
+#pragma unroll
+                for (int hh = 0; hh < TT; ++hh)
+                    tma_load_2d(dst + hh * A_BYTES, &map_a, full0 + 8 * s, iw.kb * BLOCK_K, iw.t * BT + hh * BLOCK_T);
             }
         }
     } else if (warp == 1) {
@@ -406,24 +417,31 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             for (int i = 0; i < n_units; ++i, kb = (i == dp_units) ? tail_kb0 : ((kb + 1 == kb_total) ? 0 : kb + 1)) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
-                if (seg_start && seg > 1) {
+                if (TT == 1 && seg_start && seg > 1) {
                     // the epilogue must have drained this buffer's previous segment (seg - 2)
                     if (!mbar_wait(accum_empty + 8 * (seg & 1), (uint32_t)((seg >> 1) - 1) & 1u, abort_flag)) break;
+                    tc_fence_after();
+                }
+                if (TT == 2 && seg_start && seg > 0) {
+                    // one pair of accumulators: the epilogue must have drained the previous segment
+                    if (!mbar_wait(accum_empty, (uint32_t)(seg - 1) & 1u, abort_flag)) break;
                     tc_fence_after();
                 }
                 if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) break;
                 if (i == 0) SK_STAMP(3);
                 tc_fence_after();
-                const uint32_t sa = smem_base + s * STAGE_BYTES;
-                const uint64_t da = smem_desc_sw128(sa), dw = smem_desc_sw128(sa + A_BYTES);
+                const uint32_t sa = smem_base + s * STAGE_T;
+                const uint64_t dw = smem_desc_sw128(sa + A_BYTES_T);
 #pragma unroll
                 for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                    umma_bf16(tmem_base + (uint32_t)((seg & 1) * BLOCK_F), da + (uint64_t)(k * 2), dw + (uint64_t)(k * 2), idesc,
-                              (!seg_start || k > 0) ? 1u : 0u);
+#pragma unroll
+                    for (int hh = 0; hh < TT; ++hh)
+                        umma_bf16(tmem_base + (uint32_t)((TT == 1 ? (seg & 1) : hh) * BLOCK_F), smem_desc_sw128(sa + hh * A_BYTES) + (uint64_t)(k * 2),
+                                  dw + (uint64_t)(k * 2), idesc, (!seg_start || k > 0) ? 1u : 0u);
                 umma_commit(empty0 + 8 * s);
                 seg_start = false;
                 if (kb == kb_total - 1 || i == n_units - 1) {
-                    umma_commit(accum_full + 8 * (seg & 1));
+                    umma_commit(accum_full + (TT == 1 ? 8 * (seg & 1) : 0));
                     if (i == n_units - 1) SK_STAMP(4);
                     ++seg;
                     seg_start = true;
@@ -455,51 +473,53 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
             int tile_f, tile_t;
             tile_ft(tile, g.tiles_f, g.tiles_t, tile_f, tile_t);
-            const int m = tile_t * BLOCK_T + t_local;
             const int n0 = tile_f * BLOCK_F;
-            const bool live = m < Mv;
-            const bool warp_live = tile_t * BLOCK_T + q * 32 < Mv;      // any live token in this warp's quarter
             const bool whole = (k0 == 0 && k1 == kb_total);
-            if (!mbar_wait(accum_full + 8 * (seg & 1), (uint32_t)(seg >> 1) & 1u, abort_flag)) break;
+            if (!mbar_wait(accum_full + (TT == 1 ? 8 * (seg & 1) : 0), (uint32_t)(TT == 1 ? (seg >> 1) : seg) & 1u, abort_flag)) break;
             tc_fence_after();
-            const uint32_t taddr = taddr0 + (uint32_t)((seg & 1) * BLOCK_F);
-            if (whole) {
-                if (warp_live) {
-                    for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
-                        float v[16];
-                        tmem_ld16(taddr + (uint32_t)c0, v);
-                        if (live) {
-                            epilogue16<T, EPI>(e, m, n0 + c0, v);
+            const int which = (k0 == 0) ? 1 : 0;     // slot 0: my range starts inside this tile
+#pragma unroll
+            for (int hh = 0; hh < TT; ++hh) {
+                const int m = tile_t * BT + hh * BLOCK_T + t_local;
+                const bool live = m < Mv;
+                const bool warp_live = tile_t * BT + hh * BLOCK_T + q * 32 < Mv;      // any live token in this warp's quarter
+                const uint32_t taddr = taddr0 + (uint32_t)((TT == 1 ? (seg & 1) : hh) * BLOCK_F);
+                if (whole) {
+                    if (warp_live) {
+                        for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
+                            float v[16];
+                            tmem_ld16(taddr + (uint32_t)c0, v);
+                            if (live) {
+                                epilogue16<T, EPI>(e, m, n0 + c0, v);
+                            }
+                        }
+                    }
+                } else {
+                    // partial segment: publish it now, reduce later (pass 2), so that publishing never
+                    // waits on another CTA
+                    float* part = g.partial + ((size_t)(2 * cta + which) * BT + hh * BLOCK_T + t_local) * BLOCK_F;
+                    if (warp_live) {
+                        // 64 columns per round trip to TMEM (four loads in flight, one wait)
+                        for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
+                            uint32_t r[4][16];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * j), r[j]);
+                            tmem_ld_wait();
+                            if (live) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                                    for (int c = 0; c < 16; c += 4)
+                                        *reinterpret_cast<uint4*>(part + c0 + 16 * j + c) = make_uint4(r[j][c], r[j][c + 1], r[j][c + 2], r[j][c + 3]);
+                            }
                         }
                     }
                 }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
-            } else {
-                // partial segment: publish it now, reduce later (pass 2), so that publishing never
-                // waits on another CTA
-                const int which = (k0 == 0) ? 1 : 0;     // slot 0: my range starts inside this tile
-                float* part = g.partial + ((size_t)(2 * cta + which) * BLOCK_T + t_local) * BLOCK_F;
-                if (warp_live) {
-                    // 64 columns per round trip to TMEM (four loads in flight, one wait)
-                    for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
-                        uint32_t r[4][16];
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * j), r[j]);
-                        tmem_ld_wait();
-                        if (live) {
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-#pragma unroll
-                                for (int c = 0; c < 16; c += 4)
-                                    *reinterpret_cast<uint4*>(part + c0 + 16 * j + c) = make_uint4(r[j][c], r[j][c + 1], r[j][c + 2], r[j][c + 3]);
-                        }
-                    }
-                }
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(accum_empty + 8 * (seg & 1));
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(accum_empty + (TT == 1 ? 8 * (seg & 1) : 0));
+            if (!whole) {
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile], 1);
@@ -531,7 +551,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     const int before = fx_par[f][3], mine = fx_par[f][4], w_all = fx_par[f][5];
                     f_tf[f] = fx_par[f][6]; f_tt[f] = fx_par[f][7];
                     const int tile_t = f_tt[f];
-                    const int n_live = max(0, min(BLOCK_T, Mv - tile_t * BLOCK_T));
+                    const int n_live = max(0, min(BT, Mv - tile_t * BT));
                     const int n_items = n_live * (BLOCK_F / 16);
                     f_lo[f] = (n_items * before) / w_all;
                     f_n[f] = (n_items * (before + mine)) / w_all - f_lo[f];
@@ -543,7 +563,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int f = (int)threadIdx.x < f_n[0] ? 0 : 1;
                 const int item = f_lo[f] + (int)threadIdx.x - (f ? f_n[0] : 0);
                 const int tile = fix_tile[f];
-                epilogue_prefetch<T, EPI>(e, f_tt[f] * BLOCK_T + item / (BLOCK_F / 16), f_tf[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
+                epilogue_prefetch<T, EPI>(e, f_tt[f] * BT + item / (BLOCK_F / 16), f_tf[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
             }
             if (threadIdx.x == 64) {
                 // bounded wait until all contributors have published their partial tiles
@@ -578,13 +598,13 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             const int cc = c_lo + sg0 + j;
                             const int wsl = (cc == c_lo) ? 1 : 0;
                             tv[j] = (sg0 + j < nseg)
-                                        ? __ldcg(reinterpret_cast<const float4*>(g.partial + ((size_t)(2 * cc + wsl) * BLOCK_T + tl) * BLOCK_F + c0))
+                                        ? __ldcg(reinterpret_cast<const float4*>(g.partial + ((size_t)(2 * cc + wsl) * BT + tl) * BLOCK_F + c0))
                                         : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
 #pragma unroll
                         for (int j = 0; j < 16; ++j) { acc.x += tv[j].x; acc.y += tv[j].y; acc.z += tv[j].z; acc.w += tv[j].w; }
                     }
-                    epilogue4<T, EPI>(e, f_tt[f] * BLOCK_T + tl, f_tf[f] * BLOCK_F + c0, acc);
+                    epilogue4<T, EPI>(e, f_tt[f] * BT + tl, f_tf[f] * BLOCK_F + c0, acc);
                 }
             } else if (last_sh) {
                 for (int i = (int)threadIdx.x; i < total; i += FIX_THREADS) {
@@ -606,7 +626,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 // (only the tile's first contributor can start at or before the tile's first unit)
                                 const int wsl = (cc == c_lo) ? 1 : 0;
                                 const float4* ps = reinterpret_cast<const float4*>(
-                                    g.partial + ((size_t)(2 * cc + wsl) * BLOCK_T + tl) * BLOCK_F + c0);
+                                    g.partial + ((size_t)(2 * cc + wsl) * BT + tl) * BLOCK_F + c0);
 #pragma unroll
                                 for (int x = 0; x < 4; ++x) tv[j][x] = __ldcg(ps + x);
                             } else {
@@ -622,7 +642,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
                             }
                     }
-                    const int mm = f_tt[f] * BLOCK_T + tl;
+                    const int mm = f_tt[f] * BT + tl;
                     const int n0 = f_tf[f] * BLOCK_F;
                     epilogue16<T, EPI>(e, mm, n0 + c0, acc);
                 }

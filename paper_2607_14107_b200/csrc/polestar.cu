@@ -51,6 +51,10 @@ struct Switches {
     int refresh_simt = 0;    // POLESTAR_REFRESH_SIMT
     int fuse_prep = 0;       // POLESTAR_FUSE_PREP (measured negative result, kept with its test)
     int fold_norm = 0;       // POLESTAR_FOLD_NORM (same)
+    int tall_rows = 3072;    // POLESTAR_GEMM_TALL_ROWS: projections of at least this many rows use 256-token CTA tiles
+                             // (measured on the 4096-wide QKV projection: 4096 rows 0.72 -> 0.75 of the bf16 peak, 8192 rows
+                             // 0.70 -> 0.79, 16384 rows 0.66 -> 0.78; below ~3000 rows the coarser tiles balance worse:
+                             // 1024 rows 0.56 -> 0.51, 2048 rows 0.67 -> 0.64)
     int accumulate = 1;      // POLESTAR_GEMM_ACCUMULATE: O / down projections of the chained kernel add their parts onto
                              // the residual rows in L2 (0: ordered reduction of published partial tiles, bit-reproducible)
     int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
@@ -77,6 +81,7 @@ static Switches read_switches() {
     w.fuse_prep = env_int("POLESTAR_FUSE_PREP", w.fuse_prep);
     w.fold_norm = env_int("POLESTAR_FOLD_NORM", w.fold_norm);
     w.accumulate = env_int("POLESTAR_GEMM_ACCUMULATE", w.accumulate);
+    w.tall_rows = env_int("POLESTAR_GEMM_TALL_ROWS", w.tall_rows);
     w.chain_qkv = env_int("POLESTAR_CHAIN_QKV", w.chain_qkv);
     w.l2promo = env_int("POLESTAR_TMA_L2PROMO", w.l2promo);
     w.gemm_trace = env_int("POLESTAR_GEMM_TRACE", w.gemm_trace);
@@ -219,8 +224,8 @@ static int launch_gemm_simt(const void* A, const void* W, int M, int N_out, int 
 }
 
 // stream-K grid of a GEMM with M rows: G CTAs over U units
-static void sk_grid(const GemmWs& ws, int M, int N_out, int K, long long* U, long long* G) {
-    const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + tc::BLOCK_T - 1) / tc::BLOCK_T;
+static void sk_grid(const GemmWs& ws, int M, int N_out, int K, long long* U, long long* G, int BT = tc::BLOCK_T) {
+    const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + BT - 1) / BT;
     const int sms = ws.sms;
     *U = (long long)tiles_f * tiles_t * (K / 64);
     long long g = std::min<long long>((long long)sms, *U);
@@ -247,12 +252,16 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     const CUtensorMap* mw = maps.get(W, (uint64_t)N_out * (uint64_t)(K / 64), 64, tc::BLOCK_F);
     const CUtensorMap* ma = maps.get(A, (uint64_t)M, (uint64_t)K, tc::BLOCK_T);
     if (!mw || !ma) return POLESTAR_E_CUDA;
-    const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + tc::BLOCK_T - 1) / tc::BLOCK_T;
+    // Steps of several hundred rows (operands from L2, tensor-bound): CTA tiles of 256 tokens, two MMAs per k step on
+    // one weight tile (64 KB of operands per k block for twice the work of 48 KB)
+    const int TT = (M >= ws.sw.tall_rows) ? 2 : 1;
+    const int BT = tc::BLOCK_T * TT;
+    const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + BT - 1) / BT;
     // When a multiple of the tile count fits on >= 85 % of the SMs, the grid takes it: CTA ranges then never
     // cross a tile boundary, so every CTA has one segment (one fix-up instead of two, or none at all).
     long long U, G;
-    sk_grid(ws, M, N_out, K, &U, &G);
-    while (G > 1 && ((size_t)2 * G * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
+    sk_grid(ws, M, N_out, K, &U, &G, BT);
+    while (G > 1 && ((size_t)2 * G * BT * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
     if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
     tc::SkArgs g;
     g.M = M; g.N_out = N_out; g.K = K; g.tiles_f = tiles_f; g.tiles_t = tiles_t;
@@ -260,12 +269,13 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     // flight, and less shared memory per block leaves room for the next kernel's blocks to become resident early); two
     // stages are 4 % slower.  Four stages when operands come from L2 (several token tiles).
     g.stages = std::max(2, std::min(4, ws.sw.stages > 0 ? ws.sw.stages : (tiles_t == 1 ? 3 : 4)));
+    if (TT == 2) g.stages = std::min(g.stages, 3);          // 64 KB per stage
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
     g.w_stream = (g.tiles_t == 1 && ws.sw.evict_first) ? 1 : 0;
     // POLESTAR_TRACE builds: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
     g.trace = (ws.sw.gemm_trace == EPI) ? (long long*)((char*)ws.partial + ws.partial_bytes - 16384) : nullptr;
-    const size_t smem = (size_t)g.stages * tc::STAGE_BYTES + 1024;
-    auto kern = tc::gemm_sk_kernel<__nv_bfloat16, EPI>;
+    const size_t smem = (size_t)g.stages * (tc::STAGE_BYTES + (TT - 1) * tc::A_BYTES) + 1024;
+    auto kern = TT == 2 ? tc::gemm_sk_kernel<__nv_bfloat16, EPI, 2> : tc::gemm_sk_kernel<__nv_bfloat16, EPI, 1>;
     PostArgs pa;
     memset(&pa, 0, sizeof(pa));
     if (post && post->kind && ws.post_counter) {
@@ -375,7 +385,7 @@ struct Buffers {
 
 static const int CONF_CHUNKS = 32;
 static const int FORCED_COMMIT_MAX = 512;
-static const size_t GEMM_PARTIAL_BYTES = ((size_t)40 << 20) + 16384 + 65536;   // 2 slots x 148 CTAs x 128 x 256 fp32
+static const size_t GEMM_PARTIAL_BYTES = ((size_t)80 << 20) + 16384 + 65536;   // 2 slots x 148 CTAs x 256 x 256 fp32
 // One projection of a chained launch (gemm_chain.cuh): A [M, K] x W [N_out, K]^T with epilogue `epi`.
 struct ChainSpec {
     const void* A; const void* W;
@@ -671,6 +681,12 @@ static cudaError_t set_kernel_attributes() {
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_DOWN>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_LOGITS>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV_REFRESH>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_RESID, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_SWIGLU, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_DOWN, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_LOGITS, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV_REFRESH, 2>), gemm_smem);
     PS_ATTR(tc::gemm_chain_kernel<__nv_bfloat16>, gemm_smem);
     PS_ATTR(atc::attention_tc_kernel, (int)atc::smem_bytes(atc::MAX_KT));
     PS_ATTR(kmeans_kernel, KM_SMEM_BYTES);

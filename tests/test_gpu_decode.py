@@ -287,6 +287,15 @@ def test_c1b_streaming_attention_kernel(monkeypatch, kw):
     assert seen["refresh"] > 3 and seen["entry_window"] >= 0
 
 
+def test_c1b_tall_gemm_tiles(monkeypatch):
+    # 256-token CTA tiles (two MMAs per k step on one weight tile) for every projection of more than 129 rows: block
+    # entries of a batch (ragged: 3 x 146 and 3 x 90 rows), refresh steps (3 x 72 rows), whole and split tiles
+    monkeypatch.setenv("POLESTAR_GEMM_TALL_ROWS", "130")
+    seen = run_forced("c1b", 12, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5, batch=3, prompt_len=50, gen_len=96, block=24,
+                      max_steps=16)
+    assert seen["refresh"] > 3 and seen["entry_window"] > 0
+
+
 def test_c1b_bf16_simt_gemm_path():
     run_forced("c1b", 6, tau_upd=-1, flags=I.FLAG_DEFAULT | Bd.FLAG_SIMT_GEMM)
 
