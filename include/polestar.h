@@ -353,6 +353,13 @@ int polestar_k_refresh(const void *h_dev, const int32_t *idx_dev, const int32_t 
 int polestar_k_refresh_status(const void *scratch_dev, size_t scratch_bytes, int32_t batch, int32_t max_rows,
                               int32_t d, int32_t head_dim, void *cuda_stream);
 
+/* The bounded device-side wait on its own (every wait of the library on a counter, flag or mbarrier has a limit; the
+ * paper has no counterpart).  One thread waits until *counter_dev (uint32, wrap-safe comparison) reaches `expect` or
+ * `limit_cycles` SM clock cycles (1 .. 2e9) have passed; synchronises the stream.  Returns POLESTAR_OK, or
+ * POLESTAR_E_TIMEOUT when the wait gave up (*status_dev = 1): the CUDA context stays usable, nothing was trapped. */
+int polestar_k_wait_probe(const uint32_t *counter_dev, uint32_t expect, int64_t limit_cycles, int32_t *status_dev,
+                          void *cuda_stream);
+
 /* The NVFP4 residual codec on its own (Appendix "Quantization Format"): for every row, codes and scales of
  * x - ref and the stored value ref + decode(...).  float32 arithmetic: scale = E4M3(amax / 6) (nearest even,
  * saturating), codes to the nearest E2M1 value (ties to the even code, saturating at 6).

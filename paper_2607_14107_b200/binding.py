@@ -33,7 +33,7 @@ PROF_FAMILIES = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_hea
 EXPORTS = [
     "polestar_workspace_bytes", "polestar_init", "polestar_step", "polestar_commit", "polestar_tokens",
     "polestar_read", "polestar_force", "polestar_profile", "polestar_destroy", "polestar_strerror",
-    "polestar_reload_env", "polestar_k_refresh_status", "polestar_k_nvfp4_residual",
+    "polestar_reload_env", "polestar_k_refresh_status", "polestar_k_nvfp4_residual", "polestar_k_wait_probe",
     "polestar_k_attention", "polestar_k_hidden_delta", "polestar_k_select",
     "polestar_k_refresh_scratch_bytes", "polestar_k_refresh", "polestar_k_confidence",
     "polestar_k_confidence_noalloc", "polestar_sm_count",
@@ -133,6 +133,8 @@ def load():
     lib.polestar_sm_count.argtypes = []
     lib.polestar_k_nvfp4_residual.restype = C.c_int
     lib.polestar_k_nvfp4_residual.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    lib.polestar_k_wait_probe.restype = C.c_int
+    lib.polestar_k_wait_probe.argtypes = [vp, C.c_uint32, C.c_int64, vp, vp]
     lib.polestar_reload_env.restype = C.c_int
     lib.polestar_reload_env.argtypes = []
     lib.polestar_k_refresh_status.restype = C.c_int
@@ -429,6 +431,11 @@ def polestar_k_nvfp4_residual(x, ref, codes, scales, deq):
     rows, d = x.shape
     _check(load().polestar_k_nvfp4_residual(_ptr(x), _ptr(ref), rows, d, _ptr(codes), _ptr(scales), _ptr(deq),
                                             C.c_void_p(_stream())))
+
+
+def polestar_k_wait_probe(counter, expect: int, limit_cycles: int, status) -> int:
+    """Returns the library's code (OK or E_TIMEOUT) instead of raising: the time-out is the expected outcome."""
+    return load().polestar_k_wait_probe(_ptr(counter), expect, limit_cycles, _ptr(status), C.c_void_p(_stream()))
 
 
 def polestar_reload_env() -> None:

@@ -70,13 +70,24 @@ __device__ __forceinline__ void grid_counter_arrive(unsigned* counter, int cta) 
     atomicAdd(counter, 1u);
 }
 // one thread: wait until the grid-wide counter has reached `expect` (wrap-safe), bounded
-__device__ __forceinline__ bool grid_counter_wait(const unsigned* counter, unsigned expect, volatile int* abort_flag) {
+__device__ __forceinline__ bool grid_counter_wait(const unsigned* counter, unsigned expect, volatile int* abort_flag,
+                                                  long long limit_cycles = WAIT_LIMIT_CYCLES) {
     const long long t0 = clock64();
     while ((int)((unsigned)ld_acquire_gpu(reinterpret_cast<const int*>(counter)) - expect) < 0) {
-        if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+        if (*abort_flag || clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
         __nanosleep(32);
     }
     return true;
+}
+
+// The bounded wait on its own: one thread waits until *counter reaches `expect` or `limit_cycles` have passed, and
+// reports which (status 1 = gave up).  No TMA, no mbarrier, nothing else in flight: what a caller uses to check that a
+// wait nobody satisfies ends in an error code and leaves the context usable.
+__global__ void wait_probe_kernel(const unsigned* counter, unsigned expect, long long limit_cycles, int* status) {
+    __shared__ int abort_sh;
+    abort_sh = 0;
+    const bool ok = grid_counter_wait(counter, expect, &abort_sh, limit_cycles);
+    *status = ok ? 0 : 1;
 }
 
 template <typename T>

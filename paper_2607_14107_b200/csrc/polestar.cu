@@ -1654,6 +1654,16 @@ extern "C" int polestar_k_refresh_status(const void* scratch, size_t scratch_byt
     return status ? POLESTAR_E_TIMEOUT : POLESTAR_OK;
 }
 
+extern "C" int polestar_k_wait_probe(const uint32_t* counter, uint32_t expect, int64_t limit_cycles, int32_t* status, void* stream) {
+    if (!counter || !status || limit_cycles <= 0 || limit_cycles > 2000000000LL) return POLESTAR_E_INVAL;
+    tc::wait_probe_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(counter, expect, (long long)limit_cycles, status);
+    CK(cudaGetLastError());
+    int h = 0;
+    CK(cudaMemcpyAsync(&h, status, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    return h ? POLESTAR_E_TIMEOUT : POLESTAR_OK;
+}
+
 extern "C" int polestar_k_nvfp4_residual(const float* x, const float* ref, int32_t rows, int32_t d, uint8_t* codes,
                                          uint8_t* scales, float* deq, void* stream) {
     if (rows < 0 || d <= 0 || d % 128) return POLESTAR_E_INVAL;

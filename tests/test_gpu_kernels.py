@@ -324,3 +324,17 @@ def test_nvfp4_residual_codec_bit_exact(rows, d):
     sc = scales.cpu().view(torch.float8_e4m3fn).float().numpy()
     assert np.array_equal(sc, o_scale)
     assert np.array_equal(deq.cpu().numpy().astype(np.float64), O.residual_nvfp4_roundtrip(x.numpy(), ref.numpy()))
+
+
+def test_bounded_wait_gives_up_with_an_error_code():
+    # every device-side wait of the library is bounded; this is that wait alone, on a counter nobody advances: it
+    # ends after its limit (~1 ms here) with E_TIMEOUT, and the context goes on working
+    counter = torch.zeros(1, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert Bd.polestar_k_wait_probe(counter, 1, 2_000_000, status) == Bd.E_TIMEOUT
+    assert int(status.item()) == 1
+    counter += 1
+    assert Bd.polestar_k_wait_probe(counter, 1, 2_000_000, status) == Bd.OK
+    assert int(status.item()) == 0
+    x = torch.arange(8, device="cuda").sum().item()              # the context is intact
+    assert x == 28
