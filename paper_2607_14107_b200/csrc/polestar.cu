@@ -290,6 +290,13 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     return POLESTAR_OK;
 }
 
+// Block size of the row-wise staging kernels (one CTA per row, the row in registers): 512 threads for the few rows of a
+// decoding step (latency: every thread has one or two 16-byte loads in flight), 128 threads when a step has hundreds of
+// rows, so that several rows share an SM instead of queueing one 512-thread CTA after the other.
+static int norm_threads(int rows, int d) {
+    return (rows >= 256 && d <= 4 * NORM_VPT * 128) ? 128 : NORM_THREADS;
+}
+
 // Attention + drift on tensor cores (attn_tc.cuh): bf16, head_dim 128, at most atc::MAX_N keys.
 static bool attention_tc_applies(const AttnArgs& a) {
     return a.head_dim == atc::DH && a.N <= atc::MAX_N && a.N > 0 && (a.n_heads * a.head_dim) % 64 == 0 &&
@@ -824,7 +831,7 @@ struct Path {
             if (fold && l > 0) qkv_staged = true;      // the previous down projection stored x * gain and the sums of squares
             if (!qkv_done && !qkv_staged) {      // (else: staged by the previous layer's down projection or chained kernel)
                 Scope sc(c, POLESTAR_PROF_STAGE, (double)M * d * (4 + esd), 0, 1);
-                CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
+                CK(launch_k(prep_qkv_kernel<T>, dim3(M), dim3(norm_threads(M, d)), 0, st, sd, b.rows, b.x, hc, b.packet, b.patch + (size_t)l * bs * Wm,
                                                      c->n1[l], m.rms_eps, d, (T*)b.a_buf, b.kvflag, ct));
                 CK(cudaGetLastError());
             }
@@ -976,7 +983,7 @@ struct Path {
             if (fold) ffn_staged = true;
             if (!ffn_staged) {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
-                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(NORM_THREADS), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
+                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(norm_threads(M, d)), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
                 CK(cudaGetLastError());
             }
             {
@@ -1016,7 +1023,7 @@ struct Path {
             CK(launch_k(build_head_list_kernel, dim3(1), dim3(256), 0, st, sd, b.y, m.mask_id, b.sel_idx + (size_t)(L - 1) * bs * Wm,
                                                       b.sel_cnt + (size_t)(L - 1) * bs, use_suffix, 0, b.head_list,
                                                       b.head_count, b.suf_seq, b.suf_w));
-            CK(launch_k(prep_head_kernel<T>, dim3(Mh), dim3(NORM_THREADS), 0, st, b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
+            CK(launch_k(prep_head_kernel<T>, dim3(Mh), dim3(norm_threads(Mh, d)), 0, st, b.x, b.packet, b.head_list, b.head_count, c->final_norm, m.rms_eps, d,
                                                    (T*)b.a_head));
             CK(cudaGetLastError());
         }
