@@ -58,10 +58,7 @@ __device__ __forceinline__ void epi4_dyn(int kind, const EpiArgs& e, int m, int 
     else epilogue4<T, EPI_DOWN>(e, m, n, v);
 }
 __device__ __forceinline__ void fence_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
-__device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)),
-                 "f"(__uint_as_float(c)), "f"(__uint_as_float(d)) : "memory");
-}
+
 
 // One word counts the arrivals of the whole grid (spreading it over several words made every poll several
 // dependent acquire loads and was slower).

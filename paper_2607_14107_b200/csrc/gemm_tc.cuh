@@ -238,6 +238,12 @@ struct SelFuse {
     StepSelArgs a;
 };
 
+// four fp32 values added onto dst in L2 (16-byte aligned)
+__device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(__uint_as_float(a)), "f"(__uint_as_float(b)),
+                 "f"(__uint_as_float(c)), "f"(__uint_as_float(d)) : "memory");
+}
+
 // TT = 128-row halves of a token tile.  TT = 2 (steps of several hundred rows, where the operands come from L2 and
 // the tensor pipe is the limit): a CTA tile is 256 tokens x 256 features, two MMAs per k step share one weight tile, so
 // a k block costs 64 KB of operands for twice the work of the 48 KB of TT = 1; both accumulators (2 x 256 columns) fill
@@ -314,7 +320,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         // A tile's items (one row x 16 columns each) are dealt to its contributors in contiguous shares; a CTA that
         // contributes to two tiles takes half a share of each, so that every CTA reduces about as many items.
         int n_fix = 0;
-        if (n_tail > 0) {
+        if (n_tail > 0 && !((EPI == EPI_RESID || EPI == EPI_DOWN) && e.accumulate)) {
             const long long tb = u_begin / kb_total, te = (u_end - 1) / kb_total;       // (stream-K part's own numbering)
             const bool head_cut = u_begin != tb * kb_total, tail_cut = u_end != (te + 1) * kb_total;
             int fix_tile[2] = {0, 0};
@@ -494,6 +500,26 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             }
                         }
                     }
+                } else if ((EPI == EPI_RESID || EPI == EPI_DOWN) && e.accumulate) {
+                    // partial segment of a projection whose output rows are the residual rows: add it onto them in L2
+                    bool row_ok = live;
+                    if (EPI == EPI_DOWN && live) row_ok = __ldg(reinterpret_cast<const int4*>(e.rows) + m).y >= 0;
+                    float* dst = e.out_f32 + (size_t)m * e.ld_out + n0;
+                    if (warp_live) {
+                        for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
+                            uint32_t r[4][16];
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * j), r[j]);
+                            tmem_ld_wait();
+                            if (row_ok) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                                    for (int c = 0; c < 16; c += 4)
+                                        red_add_v4(dst + c0 + 16 * j + c, r[j][c], r[j][c + 1], r[j][c + 2], r[j][c + 3]);
+                            }
+                        }
+                    }
                 } else {
                     // partial segment: publish it now, reduce later (pass 2), so that publishing never
                     // waits on another CTA
@@ -519,7 +545,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(accum_empty + (TT == 1 ? 8 * (seg & 1) : 0));
-            if (!whole) {
+            if (!whole && !((EPI == EPI_RESID || EPI == EPI_DOWN) && e.accumulate)) {
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile], 1);

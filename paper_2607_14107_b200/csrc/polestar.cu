@@ -968,22 +968,25 @@ struct Path {
                 }
                 if (chained) { c->launches += 1; qkv_done = (n_chain == 4); }
             }
+            // (separate launches, tensor-core path: the same in-place accumulation of the split tiles as in the chained kernel)
+            const bool acc_sk = c->sw.accumulate && !fold && is_bf16 && !(p.flags & POLESTAR_FLAG_SIMT_GEMM) && d % 256 == 0 && dq % 64 == 0 && F % 64 == 0;
+            float* const x1s = acc_sk ? b.x : b.x1;
             if (!chained) {
             {
                 Scope sc(c, POLESTAR_PROF_GEMM_O, (double)d * dq * esd + (double)M * dq * esd + 2.0 * M * d * 4, 2.0 * M * d * (double)dq, 1);
                 memset(&e, 0, sizeof(e));
-                e.resid = b.x; e.out_f32 = b.x1; e.ld_out = d;
+                e.resid = b.x; e.out_f32 = x1s; e.ld_out = d; e.accumulate = acc_sk ? 1 : 0;
                 if (fold) { e.fold_a = b.a_buf; e.fold_gain = c->n2[l]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 1) * Mm; }
                 PostArgs po;
                 memset(&po, 0, sizeof(po));
                 po.kind = 1; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n2[l]; po.a_out = b.a_buf;
-                po.x = b.x1; po.list = list; po.m_count = m2_count;
+                po.x = x1s; po.list = list; po.m_count = m2_count;
                 if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->wo[l], M, d, dq, e, &po, &ffn_staged, sf.on ? &sf : nullptr))) return rc;
             }
             if (fold) ffn_staged = true;
             if (!ffn_staged) {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
-                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(norm_threads(M, d)), 0, st, b.x1, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
+                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(norm_threads(M, d)), 0, st, x1s, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
                 CK(cudaGetLastError());
             }
             {
@@ -996,8 +999,8 @@ struct Path {
             {
                 Scope sc(c, POLESTAR_PROF_GEMM_DOWN, ((double)F * d + Mlive * F) * esd + 2.0 * Mlive * d * 4, 2.0 * Mlive * F * (double)d, 1);
                 memset(&e, 0, sizeof(e));
-                e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = b.x1; e.out_f32 = b.x; e.packet = b.packet;
-                e.W_max = Wm; e.within = within; e.ld_out = d;
+                e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = x1s; e.out_f32 = b.x; e.packet = b.packet;
+                e.W_max = Wm; e.within = within; e.ld_out = d; e.accumulate = (acc_sk && !list) ? 1 : 0;
                 if (fold && l + 1 < L) { e.fold_a = b.a_buf; e.fold_gain = c->n1[l + 1]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 2) * Mm; }
                 PostArgs po;
                 memset(&po, 0, sizeof(po));
