@@ -301,8 +301,16 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
                 if (P.e.accumulate) {
                     // this segment's part of the product goes straight onto the residual rows (whole or partial alike)
                     bool row_ok = live;
-                    if (live && P.epi == EPI_DOWN) row_ok = __ldg(reinterpret_cast<const int4*>(P.e.rows) + t_local).y >= 0;
                     float* dst = P.e.out_f32 + (size_t)t_local * P.e.ld_out + n0;
+                    if (live && P.epi == EPI_DOWN) {
+                        // compacted row -> forward row; a selected window row of a refresh step lands in its packet row
+                        // (which the RMSNorm staging before the gate/up projection has set to the residual row)
+                        const int r0 = P.e.list ? __ldcg(P.e.list + t_local) : t_local;
+                        const int4 rw = __ldg(reinterpret_cast<const int4*>(P.e.rows) + r0);       // {seq, pos, widx, aidx}
+                        row_ok = rw.y >= 0;
+                        dst = (P.e.within && rw.z >= 0) ? P.e.packet + ((size_t)rw.x * P.e.W_max + rw.z) * P.e.ld_out + n0
+                                                        : P.e.out_f32 + (size_t)r0 * P.e.ld_out + n0;
+                    }
                     if (warp_live) {
                         for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
                             uint32_t r[4][16];
@@ -501,7 +509,8 @@ gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant_
             if (post_ok) {
                 for (int r = cta; r < P.post.n_rows; r += G) {
                     if (P.norm_after == 1)
-                        prep_rows_row<T>(r, P.post.x, P.post.list, P.post.m_count, P.post.gain, P.post.eps, P.post.d, (T*)P.post.a_out, post_red);
+                        prep_rows_row<T>(r, P.post.x, P.post.list, P.post.m_count, P.post.gain, P.post.eps, P.post.d, (T*)P.post.a_out, post_red,
+                                         P.post.rows, const_cast<float*>(P.post.packet), P.post.sd.W_max);
                     else
                         prep_qkv_row<T>(P.post.sd, r, P.post.rows, P.post.x, P.post.hc, P.post.packet, P.post.patch, P.post.gain,
                                         P.post.eps, P.post.d, (T*)P.post.a_out, P.post.kvflag, post_red, P.post.ct);

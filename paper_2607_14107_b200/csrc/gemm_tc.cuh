@@ -503,8 +503,14 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 } else if ((EPI == EPI_RESID || EPI == EPI_DOWN) && e.accumulate) {
                     // partial segment of a projection whose output rows are the residual rows: add it onto them in L2
                     bool row_ok = live;
-                    if (EPI == EPI_DOWN && live) row_ok = __ldg(reinterpret_cast<const int4*>(e.rows) + m).y >= 0;
                     float* dst = e.out_f32 + (size_t)m * e.ld_out + n0;
+                    if (EPI == EPI_DOWN && live) {
+                        const int r0 = e.list ? __ldcg(e.list + m) : m;
+                        const int4 rw = __ldg(reinterpret_cast<const int4*>(e.rows) + r0);       // {seq, pos, widx, aidx}
+                        row_ok = rw.y >= 0;
+                        dst = (e.within && rw.z >= 0) ? e.packet + ((size_t)rw.x * e.W_max + rw.z) * e.ld_out + n0
+                                                      : e.out_f32 + (size_t)r0 * e.ld_out + n0;
+                    }
                     if (warp_live) {
                         for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
                             uint32_t r[4][16];
@@ -710,7 +716,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (post_ok) {
                     for (int r = cta; r < post.n_rows; r += G) {
                         if (post.kind == 1)
-                            prep_rows_row<T>(r, post.x, post.list, post.m_count, post.gain, post.eps, post.d, (T*)post.a_out, post_red);
+                            prep_rows_row<T>(r, post.x, post.list, post.m_count, post.gain, post.eps, post.d, (T*)post.a_out, post_red,
+                                             post.rows, const_cast<float*>(post.packet), post.sd.W_max);
                         else
                             prep_qkv_row<T>(post.sd, r, post.rows, post.x, post.hc, post.packet, post.patch, post.gain, post.eps,
                                             post.d, (T*)post.a_out, post.kvflag, post_red, post.ct);

@@ -348,23 +348,31 @@ __global__ void prep_qkv_kernel(StepDesc sd, const Row* rows, float* x, float* h
 
 // RMSNorm of a compacted list of rows (FFN input, LM-head input).
 //   src row = list ? list[i] : i;  packet_rows: rows flagged as window rows read the packet
+//   packet != null (steps whose down projection adds onto its output rows): the residual row of a selected window row is
+//   also copied to its packet row, where that projection's parts then land
 template <typename T>
 __device__ __forceinline__ void prep_rows_row(int i, const float* x, const int* list, const int* m_count, const float* gain,
-                                              float eps, int d, T* a_out, float* red) {
+                                              float eps, int d, T* a_out, float* red, const Row* rows = nullptr,
+                                              float* packet = nullptr, int W_max = 0) {
     T* a = a_out + (size_t)i * d;
     if (m_count && i >= *m_count) {
         for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
         return;
     }
     const int r = list ? list[i] : i;
-    norm_row<T>(x + (size_t)r * d, gain, eps, d, a, nullptr, nullptr, red);
+    float* copy = nullptr;
+    if (packet && rows) {
+        const Row rw = rows[r];
+        if (rw.pos >= 0 && rw.widx >= 0) copy = packet + ((size_t)rw.seq * W_max + rw.widx) * d;
+    }
+    norm_row<T>(x + (size_t)r * d, gain, eps, d, a, copy, nullptr, red);
 }
 template <typename T>
 __global__ void prep_rows_kernel(const float* x, const int* list, const int* m_count, const float* gain,
-                                 float eps, int d, T* a_out) {
+                                 float eps, int d, T* a_out, const Row* rows, float* packet, int W_max) {
     KERNEL_PROLOGUE(4);   // prep_rows_kernel
     __shared__ float red[33];
-    prep_rows_row<T>(blockIdx.x, x, list, m_count, gain, eps, d, a_out, red);
+    prep_rows_row<T>(blockIdx.x, x, list, m_count, gain, eps, d, a_out, red, rows, packet, W_max);
 }
 
 // LM-head input rows: entry i < n_act reads x[act_rows...]; later entries read packet rows.

@@ -922,11 +922,12 @@ struct Path {
                 sp[0].e.resid = b.x; sp[0].e.out_f32 = x1; sp[0].e.ld_out = d; sp[0].e.accumulate = acc ? 1 : 0;
                 sp[0].post.kind = 1; sp[0].post.n_rows = Mc; sp[0].post.d = d; sp[0].post.eps = m.rms_eps; sp[0].post.gain = c->n2[l];
                 sp[0].post.a_out = b.a_buf; sp[0].post.x = x1; sp[0].post.list = list; sp[0].post.m_count = m2_count;
+                if (acc && list) { sp[0].post.rows = b.rows; sp[0].post.packet = b.packet; sp[0].post.sd = sd; }     // packet rows <- residual rows
                 sp[1].A = b.a_buf; sp[1].W = c->wgu[l]; sp[1].N_out = 2 * F; sp[1].K = d; sp[1].epi = EPI_SWIGLU;
                 sp[1].e.out_t = b.g_buf; sp[1].e.ld_out = F; sp[1].e.m_count = m2_count;
                 sp[2].A = b.g_buf; sp[2].W = c->wd[l]; sp[2].N_out = d; sp[2].K = F; sp[2].epi = EPI_DOWN;
                 sp[2].e.rows = b.rows; sp[2].e.list = list; sp[2].e.m_count = m2_count; sp[2].e.resid = x1; sp[2].e.out_f32 = b.x;
-                sp[2].e.accumulate = (acc && !list) ? 1 : 0;      // (steps with packet rows keep the ordered epilogue)
+                sp[2].e.accumulate = acc ? 1 : 0;
                 sp[2].e.packet = b.packet; sp[2].e.W_max = Wm; sp[2].e.within = within; sp[2].e.ld_out = d;
                 if (fold) {
                     sp[0].norm_after = 0;
@@ -981,12 +982,14 @@ struct Path {
                 memset(&po, 0, sizeof(po));
                 po.kind = 1; po.n_rows = M; po.d = d; po.eps = m.rms_eps; po.gain = c->n2[l]; po.a_out = b.a_buf;
                 po.x = x1s; po.list = list; po.m_count = m2_count;
+                if (acc_sk && list) { po.rows = b.rows; po.packet = b.packet; po.sd = sd; }
                 if ((rc = gemm<EPI_RESID>(c, b.o_buf, c->wo[l], M, d, dq, e, &po, &ffn_staged, sf.on ? &sf : nullptr))) return rc;
             }
             if (fold) ffn_staged = true;
             if (!ffn_staged) {
                 Scope sc(c, POLESTAR_PROF_STAGE, Mlive * d * (4 + esd), 0, 1);
-                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(norm_threads(M, d)), 0, st, x1s, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf));
+                CK(launch_k(prep_rows_kernel<T>, dim3(M), dim3(norm_threads(M, d)), 0, st, x1s, list, m2_count, c->n2[l], m.rms_eps, d, (T*)b.a_buf,
+                            (acc_sk && list) ? b.rows : (const Row*)nullptr, (acc_sk && list) ? b.packet : (float*)nullptr, Wm));
                 CK(cudaGetLastError());
             }
             {
@@ -1000,7 +1003,7 @@ struct Path {
                 Scope sc(c, POLESTAR_PROF_GEMM_DOWN, ((double)F * d + Mlive * F) * esd + 2.0 * Mlive * d * 4, 2.0 * Mlive * F * (double)d, 1);
                 memset(&e, 0, sizeof(e));
                 e.rows = b.rows; e.list = list; e.m_count = m2_count; e.resid = x1s; e.out_f32 = b.x; e.packet = b.packet;
-                e.W_max = Wm; e.within = within; e.ld_out = d; e.accumulate = (acc_sk && !list) ? 1 : 0;
+                e.W_max = Wm; e.within = within; e.ld_out = d; e.accumulate = acc_sk ? 1 : 0;
                 if (fold && l + 1 < L) { e.fold_a = b.a_buf; e.fold_gain = c->n1[l + 1]; e.fold_ss = b.fold_ss + (size_t)(2 * l + 2) * Mm; }
                 PostArgs po;
                 memset(&po, 0, sizeof(po));
