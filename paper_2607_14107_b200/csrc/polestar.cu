@@ -51,10 +51,11 @@ struct Switches {
     int refresh_simt = 0;    // POLESTAR_REFRESH_SIMT
     int fuse_prep = 0;       // POLESTAR_FUSE_PREP (measured negative result, kept with its test)
     int fold_norm = 0;       // POLESTAR_FOLD_NORM (same)
-    int tall_rows = 3072;    // POLESTAR_GEMM_TALL_ROWS: projections of at least this many rows use 256-token CTA tiles
-                             // (measured on the 4096-wide QKV projection: 4096 rows 0.72 -> 0.75 of the bf16 peak, 8192 rows
-                             // 0.70 -> 0.79, 16384 rows 0.66 -> 0.78; below ~3000 rows the coarser tiles balance worse:
-                             // 1024 rows 0.56 -> 0.51, 2048 rows 0.67 -> 0.64)
+    int tall_rows = 2048;    // POLESTAR_GEMM_TALL_ROWS: projections of at least this many rows use 256-token CTA tiles
+                             // (measured on the 4096-wide QKV projection alone: 4096 rows 0.72 -> 0.75 of the bf16 peak, 8192
+                             // rows 0.70 -> 0.79, 16384 rows 0.66 -> 0.78, 2048 rows 0.67 -> 0.64, 1024 rows 0.56 -> 0.51; in
+                             // the long-generation decode, whose refresh steps have 2048 rows, 335 -> 339 tokens/s with the
+                             // threshold at 2048, no change at 512)
     int accumulate = 1;      // POLESTAR_GEMM_ACCUMULATE: O / down projections of the chained kernel add their parts onto
                              // the residual rows in L2 (0: ordered reduction of published partial tiles, bit-reproducible)
     int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
