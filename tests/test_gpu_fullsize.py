@@ -20,6 +20,7 @@ from paper_2607_14107_b200 import binding as Bd
 from paper_2607_14107_b200 import inputs as I
 
 from parity import check_commit_quantities, new_stats, outside_fraction
+from test_gpu_decode import impose_codes
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
@@ -86,7 +87,8 @@ def compare_step(gpu, ora, m, p, step):
             close(gpu.read(Bd.READ_DELTA)[s], tr["delta"], TOL, f"step {step} delta")
             if tr["refresh"]:
                 for l in range(L):
-                    close(gpu.read(Bd.READ_DRIFT, l)[s, :W], tr["D"][l], TOL, f"step {step} drift l{l}")
+                    nD = len(tr["D"][l])            # window rows, or clusters (centroid proxies)
+                    close(gpu.read(Bd.READ_DRIFT, l)[s, :nD], tr["D"][l], TOL, f"step {step} drift l{l}")
                     n = gpu.read(Bd.READ_SEL_COUNT, l)[s]
                     assert list(gpu.read(Bd.READ_SEL_IDX, l)[s, :n]) == list(tr["sel"][l])
         for l in range(L):
@@ -107,6 +109,15 @@ def run_reduced_depth(m, p, n_within):
     gpu = Bd.Polestar(m, packed, p, prompt)
     ora = O.PolestarOracle(m, wn, p, prompt)
     ora.step()
+    cluster = p.select_mode == I.SELECT_CLUSTER_TOPK
+    quant = bool(p.flags & I.FLAG_NVFP4_HCACHE)
+    if cluster:
+        for s in range(p.batch):        # the library's own K-means of the first block entry (inside polestar_init)
+            for l in range(m.n_layers):
+                W = len(ora.seqs[s].win)
+                assert np.array_equal(gpu.read(Bd.READ_LABELS, l)[s, :W], ora.seqs[s].labels[l]), f"labels l{l}"
+    if quant:
+        impose_codes(gpu, ora, p, m)    # a value next to a code boundary may have fallen the other way: same codes from here on
     compare_step(gpu, ora, m, p, 0)
     kinds = [ora.seqs[0].trace["kind"]]
     stats = new_stats()
@@ -116,6 +127,14 @@ def run_reduced_depth(m, p, n_within):
         assert np.array_equal(gpu.tokens(), ora.tokens())
         ora.step()
         tr = ora.seqs[0].trace
+        if cluster and tr["kind"] != "within":
+            for l in range(m.n_layers):
+                lab = np.zeros((p.batch, len(ora.seqs[0].labels[l])), np.int32)
+                for s in range(p.batch):
+                    lab[s] = ora.seqs[s].labels[l]
+                gpu.force_labels(l, lab)
+        if quant:
+            impose_codes(gpu, ora, p, m)
         if tr["kind"] == "within" and tr["refresh"]:
             for l in range(m.n_layers):
                 sel = np.full((p.batch, gpu.W_max), -1, np.int32)
@@ -158,6 +177,18 @@ def test_c4_shape_reduced_depth_matches_oracle():
     p = dataclasses.replace(p, batch=2, max_steps=48, tau_upd=25, flags=p.flags | I.FLAG_KEEP_HIDDEN)
     kinds = run_reduced_depth(m, p, n_within=3)
     assert kinds == ["entry_full", "within", "within_refresh", "entry_window"], kinds
+
+
+def test_c2_shape_centroid_proxies_and_nvfp4_cache_match_oracle():
+    # Sec. 4.1 default policy at the LLaDA-8B widths, depth 2: K-means over 4096-wide rows (the library's own labels
+    # against the oracle's at the first entry), proxy rows through the staging kernel and the attention kernels, cluster
+    # top-k, the hidden cache as NVFP4 residuals (the library's own codes replaced by the oracle's after every encode)
+    m, p = I.config("c2")
+    m = I.reduced_depth(m, 2)
+    p = dataclasses.replace(p, tau_upd=-1, select_mode=I.SELECT_CLUSTER_TOPK,
+                            flags=p.flags | I.FLAG_KEEP_HIDDEN | I.FLAG_NVFP4_HCACHE)
+    kinds = run_reduced_depth(m, p, n_within=2)
+    assert kinds == ["entry_full", "within_refresh", "within_refresh"], kinds
 
 
 def test_c6_short_generation_shape_matches_oracle():
