@@ -208,11 +208,17 @@ def c2_full():
     return m, p, packed
 
 
-def test_c2_full_depth_full_refresh_equals_nocache(c2_full):
+@pytest.mark.parametrize("mode", ["every row", "every cluster"])
+def test_c2_full_depth_full_refresh_equals_nocache(c2_full, mode):
+    # Sec. 4.1 / Sec. 3.1: refreshing everything (all window rows; or, with centroid proxies, all eight clusters of a
+    # window that spans the sequence) reproduces decoding without a cache, here over the full 32 layers
     m, p, packed = c2_full
+    if mode == "every cluster":          # (the cluster mode takes windows of up to 256 rows: a 128 + 128 sequence)
+        p = dataclasses.replace(p, prompt_len=128, gen_len=128)
     prompt = I.make_prompt(m, p).numpy()
-    pa = dataclasses.replace(p, select_mode=I.SELECT_ALL, tau_upd=-1, win_prefix_blocks=16, win_suffix_blocks=16,
-                             flags=(I.FLAG_DEFAULT | I.FLAG_KEEP_HIDDEN) & ~I.FLAG_SUFFIX_COMMIT, max_steps=64)
+    sel = dict(select_mode=I.SELECT_ALL) if mode == "every row" else dict(select_mode=I.SELECT_CLUSTER_TOPK, n_clusters=8, cluster_k=8)
+    pa = dataclasses.replace(p, tau_upd=-1, win_prefix_blocks=16, win_suffix_blocks=16,
+                             flags=(I.FLAG_DEFAULT | I.FLAG_KEEP_HIDDEN) & ~I.FLAG_SUFFIX_COMMIT, max_steps=64, **sel)
     pb = dataclasses.replace(pa, flags=pa.flags | I.FLAG_NOCACHE)
     a, b = Bd.Polestar(m, packed, pa, prompt), Bd.Polestar(m, packed, pb, prompt)
     for step in range(5):
