@@ -362,3 +362,51 @@ def test_nvfp4_hidden_cache_is_lossy_but_close():
     b2 = O.PolestarOracle(m, w, pq, prompt)
     b2.decode()
     assert b2.done and not (b2.tokens() == m.mask_id).any()
+
+
+@pytest.mark.parametrize("nkv", [1, 2])
+def test_entry_forward_matches_a_transformer_built_from_library_primitives(nkv):
+    # The composition of the pieces (pre-norm residual wiring, which gain goes where, GQA head mapping, the order of
+    # gate and up in SwiGLU, rotary positions, final norm + LM head + logit scale) against the same model written
+    # with the tensor library's own primitives: rms_norm, linear, non-causal scaled_dot_product_attention (Eq. 3), and
+    # the rotation done as a complex multiplication.  The first forward of a decode is a full-sequence forward.
+    import torch
+    import torch.nn.functional as F
+    m, p, w, prompt = tiny(nkv=nkv, logit_scale=3.0)
+    ora = O.PolestarOracle(m, w, p, prompt)
+    y = torch.from_numpy(ora.seqs[0].y.copy()).long()
+    ora.step()
+    tr = ora.seqs[0].trace
+    assert tr["kind"] == "entry_full"
+    act = torch.from_numpy(np.asarray(ora.seqs[0].act)).long()
+    N, nh, dh = len(y), m.n_heads, m.head_dim
+    t = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    pos = torch.arange(N, dtype=torch.float64)
+    inv = m.rope_theta ** (-torch.arange(0, dh, 2, dtype=torch.float64) / dh)
+    rot = torch.polar(torch.ones(N, dh // 2, dtype=torch.float64), pos[:, None] * inv[None, :])[:, None, :]
+
+    def rotate(u):          # [N, H, dh]: pair i = (u[i], u[i + dh/2]) as one complex number
+        c = torch.complex(u[..., :dh // 2], u[..., dh // 2:]) * rot
+        return torch.cat([c.real, c.imag], -1)
+
+    x = t(w["embed"])[y]
+    hidden = [x[act]]
+    for wl in w["layers"]:
+        a = F.rms_norm(x, (m.d_model,), t(wl["norm1"]), m.rms_eps)
+        q = rotate(F.linear(a, t(wl["wq"])).view(N, nh, dh))
+        k = rotate(F.linear(a, t(wl["wk"])).view(N, nkv, dh)).repeat_interleave(nh // nkv, dim=1)
+        v = F.linear(a, t(wl["wv"])).view(N, nkv, dh).repeat_interleave(nh // nkv, dim=1)
+        o = F.scaled_dot_product_attention(q.transpose(0, 1)[None], k.transpose(0, 1)[None], v.transpose(0, 1)[None])[0]
+        x1 = x + F.linear(o.transpose(0, 1).reshape(N, nh * dh), t(wl["wo"]))
+        f = F.rms_norm(x1, (m.d_model,), t(wl["norm2"]), m.rms_eps)
+        x = x1 + F.linear(F.silu(F.linear(f, t(wl["wg"]))) * F.linear(f, t(wl["wu"])), t(wl["wd"]))
+        hidden.append(x[act])
+    logits = F.linear(F.rms_norm(x[act], (m.d_model,), t(w["final_norm"]), m.rms_eps), t(w["lm_head"])) * p.logit_scale
+    for l, h in enumerate(hidden):
+        assert np.allclose(tr["x_act"][l], h.numpy(), atol=1e-10, rtol=1e-9), f"hidden l{l}"
+    assert np.allclose(tr["logits"], logits.numpy(), atol=1e-9, rtol=1e-9)
+    # a mistake in the wiring would show: swapping gate and up moves the logits far beyond that
+    wl = w["layers"][0]
+    f0 = F.rms_norm(hidden[0], (m.d_model,), t(wl["norm2"]), m.rms_eps)
+    assert not np.allclose((F.silu(F.linear(f0, t(wl["wg"]))) * F.linear(f0, t(wl["wu"]))).numpy(),
+                           (F.silu(F.linear(f0, t(wl["wu"]))) * F.linear(f0, t(wl["wg"]))).numpy(), atol=1e-3)
