@@ -393,17 +393,32 @@ __global__ void prep_head_kernel(const float* x, const float* packet, const Head
 }
 
 // Gather + RMSNorm for the stand-alone refresh kernel: row (s, i) <- h[s][idx[s][i]].
+// The same launch also prepares what the projection behind it needs (one launch instead of four): the rotary entries
+// of the row's position (rope_tab[pos][half], when rope_tab is given) and, in its first block, zeroed split-tile
+// counters and status word of the caller's scratch.
 template <typename T>
 __global__ void prep_refresh_kernel(const T* h, const int* idx, const int* counts, int max_rows, int P,
-                                    const float* gain, float eps, int d, T* a_out) {
+                                    const float* gain, float eps, int d, T* a_out, float2* rope_tab, int half, double theta,
+                                    int* counters, int n_counters, int* status) {
     KERNEL_PROLOGUE(6);   // prep_refresh_kernel
     __shared__ float red[33];
     const int m = blockIdx.x;
     const int s = m / max_rows, i = m - s * max_rows;
     T* a = a_out + (size_t)m * d;
+    if (m == 0 && counters) {
+        for (int c = threadIdx.x; c < n_counters; c += blockDim.x) counters[c] = 0;
+        if (threadIdx.x == 0 && status) *status = 0;
+    }
     if (i >= counts[s]) {
         for (int c = threadIdx.x; c < d; c += blockDim.x) a[c] = from_f<T>(0.f);
         return;
+    }
+    if (rope_tab) {
+        const int pos = idx[s * max_rows + i];
+        for (int k = threadIdx.x; k < half; k += blockDim.x) {
+            const double ang = (double)pos * pow(theta, -(double)k / (double)half);
+            rope_tab[(size_t)pos * half + k] = make_float2((float)cos(ang), (float)sin(ang));
+        }
     }
     const T* src = h + ((size_t)s * P + idx[s * max_rows + i]) * d;
     float ss = 0.f;
@@ -1441,20 +1456,6 @@ __global__ void rope_table_kernel(float2* tab, int N, int half, double theta) {
     const double inv = pow(theta, -(double)k / (double)half);
     const double ang = (double)pos * inv;
     tab[i] = make_float2((float)cos(ang), (float)sin(ang));
-}
-
-// the same entries for the listed positions only: row i < counts[s] of sequence s fills tab[idx[s][i]]
-__global__ void rope_rows_kernel(float2* tab, const int* idx, const int* counts, int max_rows, int n_rows, int half, double theta) {
-    KERNEL_PROLOGUE(17);   // rope_rows_kernel
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n_rows * half) return;
-    const int m = i / half, k = i - m * half;
-    const int s = m / max_rows, r = m - s * max_rows;
-    if (r >= counts[s]) return;
-    const int pos = idx[s * max_rows + r];
-    const double inv = pow(theta, -(double)k / (double)half);
-    const double ang = (double)pos * inv;
-    tab[(size_t)pos * half + k] = make_float2((float)cos(ang), (float)sin(ang));
 }
 
 }  // namespace ps

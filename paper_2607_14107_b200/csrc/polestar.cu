@@ -1637,15 +1637,14 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     const long long tiles = (long long)((dq + 2 * dkv + tc::BLOCK_F - 1) / tc::BLOCK_F) * ((M + tc::BLOCK_T - 1) / tc::BLOCK_T);
     const int n_cnt = (int)std::min<long long>(GEMM_COUNTERS, 2 * (tiles + 1));
     ws.counters = (int*)(sc + off_cnt); ws.n_counters = n_cnt; ws.status = (int*)(sc + off_status);
-    CK(cudaMemsetAsync(ws.counters, 0, (size_t)n_cnt * sizeof(int), st));
-    CK(cudaMemsetAsync(ws.status, 0, sizeof(int), st));       // read back by polestar_k_refresh_status
     const int half = head_dim / 2;
-    // launched back to back with programmatic stream serialization: each kernel starts while its predecessor drains
-    // rotary entries: of the selected positions only when these are fewer than the whole table
-    if (M < P) CK(launch_k(rope_rows_kernel, dim3((M * half + 255) / 256), dim3(256), 0, st, rope, idx, counts, max_rows, M, half, (double)rope_theta));
-    else CK(launch_k(rope_table_kernel, dim3((P * half + 255) / 256), dim3(256), 0, st, rope, P, half, (double)rope_theta));
+    // Two launches with programmatic stream serialization (the projection starts while the gather drains).  The gather
+    // kernel also clears the counters and the status word (read back by polestar_k_refresh_status) and writes the rotary
+    // entries of the selected positions; only a refresh of (nearly) every position fills the whole table instead.
+    const bool table = M >= P;
+    if (table) CK(launch_k(rope_table_kernel, dim3((P * half + 255) / 256), dim3(256), 0, st, rope, P, half, (double)rope_theta));
     CK(launch_k(prep_refresh_kernel<__nv_bfloat16>, dim3(M), dim3(256), 0, st, (const __nv_bfloat16*)h, idx, counts, max_rows, P, norm,
-                rms_eps, d, a_buf));
+                rms_eps, d, a_buf, table ? (float2*)nullptr : rope, half, (double)rope_theta, ws.counters, n_cnt, ws.status));
     CK(cudaGetLastError());
     EpiArgs e;
     memset(&e, 0, sizeof(e));
