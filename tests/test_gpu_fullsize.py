@@ -191,6 +191,17 @@ def test_c2_shape_centroid_proxies_and_nvfp4_cache_match_oracle():
     assert kinds == ["entry_full", "within_refresh", "within_refresh"], kinds
 
 
+def test_c3_widths_centroid_proxies_and_nvfp4_cache_match_oracle():
+    # the same policy at the Dream-7B widths (d 3584 = 28 x 128: not a power of two; GQA 28 / 4), batch 2, short
+    # sequences: K-means, proxy staging and the codec with 3584-wide rows, proxy rows of two sequences in one forward
+    m, _ = I.config("c3")
+    m = I.reduced_depth(m, 1)
+    p = I.Params(batch=2, prompt_len=64, gen_len=64, block=32, max_steps=64, tau_upd=-1, select_mode=I.SELECT_CLUSTER_TOPK,
+                 n_clusters=6, cluster_k=3, flags=I.FLAG_DEFAULT | I.FLAG_KEEP_HIDDEN | I.FLAG_NVFP4_HCACHE)
+    kinds = run_reduced_depth(m, p, n_within=2)
+    assert kinds == ["entry_full", "within_refresh", "within_refresh"], kinds
+
+
 def test_c6_short_generation_shape_matches_oracle():
     # Sec. 5.2 (hard-to-parallelise tasks): generation length 32 with block 8 at the LLaDA-8B widths, depth 2: a
     # window of 16 + 8 rows, eight active rows per step, a block entry every few forwards
