@@ -350,7 +350,7 @@ constexpr int SP_SLOT_BYTES = AT_BN * AT_DH * 2;     // one K or V tile: 8 KB
 // (max, sum), partial KL and partial outputs through distributed shared memory; rank 0 writes the results.
 template <int NW, int TPW, int CL>
 __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
-    KERNEL_PROLOGUE(7);   // __launch_bounds__
+    pdl_trigger();        // (the wait for the kernel before this one comes after the first loads of untouched key tiles)
     extern __shared__ uint8_t at_smem_raw[];
     __shared__ float red_m[NW][AT_BM], red_l[NW][AT_BM], red_kl[NW][AT_BM];
     __shared__ float lse_sh[AT_BM];
@@ -399,8 +399,24 @@ __global__ void __launch_bounds__(NW * 32) attention_sp_kernel(AttnMmaArgs g) {
         }
         cp_async_commit();
     };
-    if (n_loads > 0) issue(0);
-    if (n_loads > 1) issue(1);
+    // Key tiles outside [dirty_lo, dirty_hi) were last written by an earlier forward, which the host has waited for:
+    // their K / V can be on their way while the projection before this kernel still runs.  q, the row table and
+    // the rows that projection writes come after the wait.
+    auto load_clean = [&](int j) {
+        const bool is_v = j >= my_tiles;
+        const int lo = (warp + ((is_v ? j - my_tiles : j) * CL + rank) * NW) * AT_BN;
+        return lo + AT_BN <= a.dirty_lo || lo >= a.dirty_hi;
+    };
+    int issued = 0;
+    if (n_loads > 0 && load_clean(0)) {
+        issue(0);
+        issued = 1;
+        if (n_loads > 1 && load_clean(1)) { issue(1); issued = 2; }
+    }
+    pdl_wait();
+    trace_stamp(7);
+    if (issued < 1 && n_loads > 0) issue(0);
+    if (issued < 2 && n_loads > 1) issue(1);
 
     // ---- row bookkeeping + Q tile (overlap the first K loads; neither waits for the other) ----------
     // Rows without a valid descriptor may hold stale q values: they only ever affect their own row of
