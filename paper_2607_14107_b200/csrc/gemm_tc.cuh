@@ -179,6 +179,8 @@ struct SkArgs {
     int done_offset;
     int* status;        // set to 1 on a wait time-out
     int w_stream;       // 1: every weight byte is read once by this launch: load it with the evict_first L2 policy
+    int epi_groups;     // 1..3 groups of four warps drain an accumulator (groups beyond the first: warps 8-11, 12-15,
+                        // which otherwise idle until the reduction pass); the 16-column chunks are dealt round-robin
     long long* trace;   // POLESTAR_TRACE builds: [gridDim.x][12] nanosecond stamps of this launch (null: off): 0 start,
                         // 1 set-up done, 2 dependencies resolved, 3 first stage full, 4 last MMA issued, 5 partial tiles
                         // published, 6 other contributors arrived, 8 share reduced, 7 end
@@ -295,7 +297,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         for (int s = 0; s < g.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int b2 = 0; b2 < 2; ++b2) {
             mbar_init(accum_full + 8 * b2, 1);
-            mbar_init(accum_empty + 8 * b2, 4);      // one arrival per epilogue warp
+            mbar_init(accum_empty + 8 * b2, 4 * g.epi_groups);      // one arrival per epilogue warp
         }
         abort_sh = 0;
         last_sh = 0;
@@ -454,11 +456,12 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
             }
         }
-    } else if (warp < 6) {
+    } else if (warp < 6 || (warp >= 8 && warp < 4 + 4 * g.epi_groups)) {
         // ---- epilogue warps: TMEM lane = token, column = feature ------------------------------------
         pdl_wait();
         trace_stamp(100 + EPI, 64);
-        const int q = warp & 3;
+        const int q = warp & 3;                      // a warp reaches the 32 lanes of its quarter only
+        const int groups = g.epi_groups, gi = warp < 6 ? 0 : (warp - 4) >> 2;
         const int t_local = q * 32 + lane;
         const uint32_t taddr0 = tmem_base + ((uint32_t)(q * 32) << 16);
         const int Mv = e.m_count ? min(g.M, __ldg(e.m_count)) : g.M;
@@ -493,6 +496,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 if (whole) {
                     if (warp_live) {
                         for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
+                            if ((hh * (BLOCK_F / 16) + (c0 >> 4)) % groups != gi) continue;
                             float v[16];
                             tmem_ld16(taddr + (uint32_t)c0, v);
                             if (live) {
@@ -513,6 +517,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     }
                     if (warp_live) {
                         for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
+                            if ((hh * (BLOCK_F / 64) + (c0 >> 6)) % groups != gi) continue;
                             uint32_t r[4][16];
 #pragma unroll
                             for (int j = 0; j < 4; ++j) tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * j), r[j]);
@@ -533,6 +538,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     if (warp_live) {
                         // 64 columns per round trip to TMEM (four loads in flight, one wait)
                         for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
+                            if ((hh * (BLOCK_F / 64) + (c0 >> 6)) % groups != gi) continue;
                             uint32_t r[4][16];
 #pragma unroll
                             for (int j = 0; j < 4; ++j) tmem_ld16_issue(taddr + (uint32_t)(c0 + 16 * j), r[j]);
@@ -553,7 +559,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (lane == 0) mbar_arrive(accum_empty + (TT == 1 ? 8 * (seg & 1) : 0));
             if (!whole && !((EPI == EPI_RESID || EPI == EPI_DOWN) && e.accumulate)) {
                 __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, %0;" ::"r"(128 * groups) : "memory");
                 if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile], 1);
             }
             ++seg;

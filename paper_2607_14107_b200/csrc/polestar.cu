@@ -59,6 +59,8 @@ struct Switches {
     int accumulate = 1;      // POLESTAR_GEMM_ACCUMULATE: O / down projections of the chained kernel add their parts onto
                              // the residual rows in L2 (0: ordered reduction of published partial tiles, bit-reproducible)
     int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
+    int epi_groups = 3;      // POLESTAR_GEMM_EPI_GROUPS: groups of four warps that drain an accumulator when a projection
+                             // has several token tiles (1: the four epilogue warps alone)
     int l2promo = (int)CU_TENSOR_MAP_L2_PROMOTION_L2_128B;   // POLESTAR_TMA_L2PROMO
     int gemm_trace = -1;     // POLESTAR_GEMM_TRACE (POLESTAR_TRACE builds)
     int kernel_trace = 0;    // POLESTAR_KERNEL_TRACE (POLESTAR_TRACE builds)
@@ -74,6 +76,7 @@ static Switches read_switches() {
     w.fuse_select = env_int("POLESTAR_FUSE_SELECT", w.fuse_select);
     w.chain = env_int("POLESTAR_CHAIN", w.chain);
     w.stages = env_int("POLESTAR_GEMM_STAGES", w.stages);
+    w.epi_groups = env_int("POLESTAR_GEMM_EPI_GROUPS", w.epi_groups);
     w.align_pct = env_int("POLESTAR_GEMM_ALIGN_PCT", w.align_pct);
     w.half_align = env_int("POLESTAR_GEMM_HALF_ALIGN", w.half_align);
     w.attn_kernel = env_int("POLESTAR_ATTN_KERNEL", w.attn_kernel);
@@ -273,6 +276,7 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     if (TT == 2) g.stages = std::min(g.stages, 3);          // 64 KB per stage
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
     g.w_stream = (g.tiles_t == 1 && ws.sw.evict_first) ? 1 : 0;
+    g.epi_groups = g.tiles_t > 1 ? std::max(1, std::min(3, ws.sw.epi_groups)) : 1;
     // POLESTAR_TRACE builds: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
     g.trace = (ws.sw.gemm_trace == EPI) ? (long long*)((char*)ws.partial + ws.partial_bytes - 16384) : nullptr;
     const size_t smem = (size_t)g.stages * (tc::STAGE_BYTES + (TT - 1) * tc::A_BYTES) + 1024;
@@ -287,6 +291,7 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     }
     tc::SelFuse sfz;
     if (sel) sfz = *sel; else memset(&sfz, 0, sizeof(sfz));
+    if (sfz.on) g.epi_groups = 1;          // the selection runs on warps 6-13 of the first CTA
     CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e, pa, sfz));
     return POLESTAR_OK;
 }
