@@ -56,6 +56,8 @@ struct Switches {
                              // rows 0.70 -> 0.79, 16384 rows 0.66 -> 0.78, 2048 rows 0.67 -> 0.64, 1024 rows 0.56 -> 0.51; in
                              // the long-generation decode, whose refresh steps have 2048 rows, 335 -> 339 tokens/s with the
                              // threshold at 2048, no change at 512)
+    int tall_rows_ffn = 512; // POLESTAR_GEMM_TALL_ROWS_FFN: the same threshold for the gate/up projection, whose epilogue is short
+                             // enough for the tall tile to pay from 512 rows on (follows POLESTAR_GEMM_TALL_ROWS when only that is set)
     int accumulate = 1;      // POLESTAR_GEMM_ACCUMULATE: O / down projections of the chained kernel add their parts onto
                              // the residual rows in L2 (0: ordered reduction of published partial tiles, bit-reproducible)
     int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
@@ -86,6 +88,7 @@ static Switches read_switches() {
     w.fold_norm = env_int("POLESTAR_FOLD_NORM", w.fold_norm);
     w.accumulate = env_int("POLESTAR_GEMM_ACCUMULATE", w.accumulate);
     w.tall_rows = env_int("POLESTAR_GEMM_TALL_ROWS", w.tall_rows);
+    w.tall_rows_ffn = env_int("POLESTAR_GEMM_TALL_ROWS_FFN", getenv("POLESTAR_GEMM_TALL_ROWS") ? w.tall_rows : w.tall_rows_ffn);
     w.chain_qkv = env_int("POLESTAR_CHAIN_QKV", w.chain_qkv);
     w.l2promo = env_int("POLESTAR_TMA_L2PROMO", w.l2promo);
     w.gemm_trace = env_int("POLESTAR_GEMM_TRACE", w.gemm_trace);
@@ -258,7 +261,7 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     if (!mw || !ma) return POLESTAR_E_CUDA;
     // Steps of several hundred rows (operands from L2, tensor-bound): CTA tiles of 256 tokens, two MMAs per k step on
     // one weight tile (64 KB of operands per k block for twice the work of 48 KB)
-    const int TT = (M >= ws.sw.tall_rows) ? 2 : 1;
+    const int TT = (M >= (EPI == EPI_SWIGLU ? ws.sw.tall_rows_ffn : ws.sw.tall_rows)) ? 2 : 1;
     const int BT = tc::BLOCK_T * TT;
     const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + BT - 1) / BT;
     // When a multiple of the tile count fits on >= 85 % of the SMs, the grid takes it: CTA ranges then never
