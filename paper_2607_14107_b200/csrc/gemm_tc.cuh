@@ -128,6 +128,36 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// ---- CTA pairs (cluster of two): one tcgen05.mma, issued by the even CTA, runs on both SMs' tensor cores -----------------
+// address of the same shared-memory variable in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// load into this CTA's shared memory; the bytes are counted on a barrier of either CTA of the pair
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(x), "r"(y)
+        : "memory");
+}
+// D (256 x N, 128 rows in each CTA's tensor memory) += A (128 rows per CTA) x B (N / 2 rows per CTA); descriptors are
+// the issuing CTA's, the peer's operands sit at the same shared-memory offsets
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives on the barrier at this offset in both CTAs once the MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
 // 16 consecutive accumulator columns of this thread's TMEM lane
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
     uint32_t r[16];
@@ -188,7 +218,7 @@ struct SkArgs {
 
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #ifdef POLESTAR_TRACE
-#define SK_STAMP(i) do { if (g.trace) g.trace[(size_t)cta * 12 + (i)] = gtime(); } while (0)
+#define SK_STAMP(i) do { if (g.trace) g.trace[(size_t)blockIdx.x * 12 + (i)] = gtime(); } while (0)
 #else
 #define SK_STAMP(i) do { } while (0)
 #endif
@@ -250,7 +280,15 @@ __device__ __forceinline__ void red_add_v4(float* dst, uint32_t a, uint32_t b, u
 // the tensor pipe is the limit): a CTA tile is 256 tokens x 256 features, two MMAs per k step share one weight tile, so
 // a k block costs 64 KB of operands for twice the work of the 48 KB of TT = 1; both accumulators (2 x 256 columns) fill
 // the tensor memory, so the epilogue of a segment no longer overlaps the next segment's MMAs.
-template <typename T, int EPI, int TT = 1>
+//
+// CG = 2 (with TT = 1; launched as clusters of two CTAs): a CTA pair works on a tile of 256 tokens x 256 features.  Each
+// CTA loads its 128 tokens and HALF of the weight tile (128 features), the even CTA issues one MMA for both tensor cores
+// (tcgen05.mma.cta_group::2, M = 256), and each CTA ends up with its 128 tokens x 256 features in its own tensor memory:
+// 32 KB of operands per CTA and k block instead of 48, so six stages fit and the operand supply (bytes in flight against
+// the load latency) no longer limits the MMA rate, while the two accumulators keep the epilogue overlapped.  The schedule
+// treats the pair as one CTA (stream-K ranges, whole tiles first); everything after the MMAs (epilogue, partial tiles,
+// reduction pass) is per CTA on its own 128 rows, with partial-tile slots and tile counters of its own.
+template <typename T, int EPI, int TT = 1, int CG = 1>
 __global__ void __launch_bounds__(FIX_THREADS, 1)
 gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_a,
                SkArgs g, EpiArgs e, PostArgs post, SelFuse sf) {
@@ -265,9 +303,15 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 
     constexpr int BT = BLOCK_T * TT;                       // tokens per CTA tile
     constexpr uint32_t A_BYTES_T = A_BYTES * TT;           // activations of a stage: TT boxes of [128][64]
-    constexpr uint32_t STAGE_T = A_BYTES_T + W_BYTES;
+    constexpr uint32_t W_BYTES_C = W_BYTES / CG;           // weights of a stage in this CTA's shared memory
+    constexpr uint32_t STAGE_T = A_BYTES_T + W_BYTES_C;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = gridDim.x, cta = blockIdx.x;
+    constexpr bool PAIR = CG == 2;
+    static_assert(!PAIR || TT == 1, "CTA pairs take 128-token halves");
+    const int rank = PAIR ? (int)(blockIdx.x & 1u) : 0;                  // CTA within its pair (cluster of two along x)
+    // scheduling unit: a CTA, or a CTA pair (both CTAs of a pair run the same schedule)
+    const int G = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x, cta = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int slot_cta = (int)blockIdx.x;                                // owner index of partial-tile slots
     if (threadIdx.x == 0) SK_STAMP(0);
     const int kb_total = g.K / BLOCK_K;
     // Schedule: with more tiles than CTAs, CTA c first takes the whole tiles c, c + G, c + 2G, ... (`dp` of them:
@@ -297,7 +341,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         for (int s = 0; s < g.stages; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
         for (int b2 = 0; b2 < 2; ++b2) {
             mbar_init(accum_full + 8 * b2, 1);
-            mbar_init(accum_empty + 8 * b2, 4 * g.epi_groups);      // one arrival per epilogue warp
+            mbar_init(accum_empty + 8 * b2, 4 * g.epi_groups * CG);      // one arrival per epilogue warp (of both CTAs)
         }
         abort_sh = 0;
         last_sh = 0;
@@ -307,7 +351,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_sh), ncols);
     tc_fence_before();
-    __syncthreads();
+    if (PAIR) cluster_sync_all(); else __syncthreads();      // (pairs: the peer's barriers are initialised before anything arrives on them)
     tc_fence_after();
     pdl_trigger();
     if (threadIdx.x == 0) SK_STAMP(1);
@@ -386,7 +430,15 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
             };
             It iw = start();
+            // pairs: the bytes of both CTAs' loads are counted on the even CTA's barrier, which alone expects them
+            const uint32_t full_pair = PAIR ? mapa_u32(full0, 0) : 0u;
             for (int i = 0; i < pre; ++i, advance(iw)) {
+                if (PAIR) {
+                    if (rank == 0) mbar_expect_tx(full0 + 8 * i, 2 * STAGE_T);
+                    tma_load_2d_pair(smem_base + i * STAGE_T + A_BYTES_T, &map_w, full_pair + 8 * i, 0,
+                                     (iw.f * kb_total + iw.kb) * BLOCK_F + rank * (BLOCK_F / 2));
+                    continue;
+                }
                 mbar_expect_tx(full0 + 8 * i, STAGE_T);
                 if (g.w_stream) tma_load_2d_hint(smem_base + i * STAGE_T + A_BYTES_T, &map_w, full0 + 8 * i, 0,
                                                  (iw.f * kb_total + iw.kb) * BLOCK_F, pol);
@@ -396,16 +448,27 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             SK_STAMP(2);
             {
                 It ia = start();
-                for (int i = 0; i < pre; ++i, advance(ia))
+                for (int i = 0; i < pre; ++i, advance(ia)) {
+                    if (PAIR) {
+                        tma_load_2d_pair(smem_base + i * STAGE_T, &map_a, full_pair + 8 * i, ia.kb * BLOCK_K, (ia.t * CG + rank) * BT);
+                        continue;
+                    }
 #pragma unroll
                     for (int hh = 0; hh < TT; ++hh)
                         tma_load_2d(smem_base + i * STAGE_T + hh * A_BYTES, &map_a, full0 + 8 * i, ia.kb * BLOCK_K, ia.t * BT + hh * BLOCK_T);
+                }
             }
             for (int i = pre; i < n_units; ++i, advance(iw)) {
                 const int s = i % g.stages;
                 const uint32_t ph = (uint32_t)(i / g.stages) & 1u;
                 if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) break;
                 const uint32_t dst = smem_base + s * STAGE_T;
+                if (PAIR) {
+                    if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * STAGE_T);
+                    tma_load_2d_pair(dst + A_BYTES_T, &map_w, full_pair + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F + rank * (BLOCK_F / 2));
+                    tma_load_2d_pair(dst, &map_a, full_pair + 8 * s, iw.kb * BLOCK_K, (iw.t * CG + rank) * BT);
+                    continue;
+                }
                 mbar_expect_tx(full0 + 8 * s, STAGE_T);
                 if (g.w_stream) tma_load_2d_hint(dst + A_BYTES_T, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F, pol);
                 else tma_load_2d(dst + A_BYTES_T, &map_w, full0 + 8 * s, 0, (iw.f * kb_total + iw.kb) * BLOCK_F);
@@ -415,8 +478,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(BLOCK_T, BLOCK_F);
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_bf16(BLOCK_T * CG, BLOCK_F);
             int seg = 0;
             bool seg_start = true;
             const int tail_kb0 = (int)(u_begin % kb_total);
@@ -443,13 +506,18 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                 for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
 #pragma unroll
-                    for (int hh = 0; hh < TT; ++hh)
-                        umma_bf16(tmem_base + (uint32_t)((TT == 1 ? (seg & 1) : hh) * BLOCK_F), smem_desc_sw128(sa + hh * A_BYTES) + (uint64_t)(k * 2),
-                                  dw + (uint64_t)(k * 2), idesc, (!seg_start || k > 0) ? 1u : 0u);
-                umma_commit(empty0 + 8 * s);
+                    for (int hh = 0; hh < TT; ++hh) {
+                        if (PAIR)
+                            umma_bf16_pair(tmem_base + (uint32_t)((seg & 1) * BLOCK_F), smem_desc_sw128(sa) + (uint64_t)(k * 2),
+                                           dw + (uint64_t)(k * 2), idesc, (!seg_start || k > 0) ? 1u : 0u);
+                        else
+                            umma_bf16(tmem_base + (uint32_t)((TT == 1 ? (seg & 1) : hh) * BLOCK_F), smem_desc_sw128(sa + hh * A_BYTES) + (uint64_t)(k * 2),
+                                      dw + (uint64_t)(k * 2), idesc, (!seg_start || k > 0) ? 1u : 0u);
+                    }
+                if (PAIR) umma_commit_pair(empty0 + 8 * s); else umma_commit(empty0 + 8 * s);
                 seg_start = false;
                 if (kb == kb_total - 1 || i == n_units - 1) {
-                    umma_commit(accum_full + (TT == 1 ? 8 * (seg & 1) : 0));
+                    if (PAIR) umma_commit_pair(accum_full + 8 * (seg & 1)); else umma_commit(accum_full + (TT == 1 ? 8 * (seg & 1) : 0));
                     if (i == n_units - 1) SK_STAMP(4);
                     ++seg;
                     seg_start = true;
@@ -489,9 +557,9 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int which = (k0 == 0) ? 1 : 0;     // slot 0: my range starts inside this tile
 #pragma unroll
             for (int hh = 0; hh < TT; ++hh) {
-                const int m = tile_t * BT + hh * BLOCK_T + t_local;
+                const int m = (tile_t * CG + rank) * BT + hh * BLOCK_T + t_local;
                 const bool live = m < Mv;
-                const bool warp_live = tile_t * BT + hh * BLOCK_T + q * 32 < Mv;      // any live token in this warp's quarter
+                const bool warp_live = (tile_t * CG + rank) * BT + hh * BLOCK_T + q * 32 < Mv;      // any live token in this warp's quarter
                 const uint32_t taddr = taddr0 + (uint32_t)((TT == 1 ? (seg & 1) : hh) * BLOCK_F);
                 if (whole) {
                     if (warp_live) {
@@ -534,7 +602,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 } else {
                     // partial segment: publish it now, reduce later (pass 2), so that publishing never
                     // waits on another CTA
-                    float* part = g.partial + ((size_t)(2 * cta + which) * BT + hh * BLOCK_T + t_local) * BLOCK_F;
+                    float* part = g.partial + ((size_t)(2 * slot_cta + which) * BT + hh * BLOCK_T + t_local) * BLOCK_F;
                     if (warp_live) {
                         // 64 columns per round trip to TMEM (four loads in flight, one wait)
                         for (int c0 = 0; c0 < BLOCK_F; c0 += 64) {
@@ -556,11 +624,14 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(accum_empty + (TT == 1 ? 8 * (seg & 1) : 0));
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(mapa_u32(accum_empty + 8 * (seg & 1), 0));      // the even CTA issues the MMAs
+                else mbar_arrive(accum_empty + (TT == 1 ? 8 * (seg & 1) : 0));
+            }
             if (!whole && !((EPI == EPI_RESID || EPI == EPI_DOWN) && e.accumulate)) {
                 __threadfence();
                 asm volatile("bar.sync 1, %0;" ::"r"(128 * groups) : "memory");
-                if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile], 1);
+                if (threadIdx.x == 64) atomicAdd(&g.tile_counter[tile * CG + rank], 1);
             }
             ++seg;
         }
@@ -589,7 +660,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     const int before = fx_par[f][3], mine = fx_par[f][4], w_all = fx_par[f][5];
                     f_tf[f] = fx_par[f][6]; f_tt[f] = fx_par[f][7];
                     const int tile_t = f_tt[f];
-                    const int n_live = max(0, min(BT, Mv - tile_t * BT));
+                    const int n_live = max(0, min(BT, Mv - (tile_t * CG + rank) * BT));
                     const int n_items = n_live * (BLOCK_F / 16);
                     f_lo[f] = (n_items * before) / w_all;
                     f_n[f] = (n_items * (before + mine)) / w_all - f_lo[f];
@@ -601,14 +672,14 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const int f = (int)threadIdx.x < f_n[0] ? 0 : 1;
                 const int item = f_lo[f] + (int)threadIdx.x - (f ? f_n[0] : 0);
                 const int tile = fix_tile[f];
-                epilogue_prefetch<T, EPI>(e, f_tt[f] * BT + item / (BLOCK_F / 16), f_tf[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
+                epilogue_prefetch<T, EPI>(e, (f_tt[f] * CG + rank) * BT + item / (BLOCK_F / 16), f_tf[f] * BLOCK_F + (item % (BLOCK_F / 16)) * 16);
             }
             if (threadIdx.x == 64) {
                 // bounded wait until all contributors have published their partial tiles
                 const long long t0 = clock64();
                 int ok = 1;
                 for (int f = 0; f < n_fix && ok; ++f) {
-                    while (ld_acquire_gpu(&g.tile_counter[fix_tile[f]]) < f_nseg[f]) {
+                    while (ld_acquire_gpu(&g.tile_counter[fix_tile[f] * CG + rank]) < f_nseg[f]) {
                         if (*abort_flag || clock64() - t0 > WAIT_LIMIT_CYCLES) { ok = 0; *abort_flag = 1; break; }
                         __nanosleep(64);
                     }
@@ -636,13 +707,13 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                             const int cc = c_lo + sg0 + j;
                             const int wsl = (cc == c_lo) ? 1 : 0;
                             tv[j] = (sg0 + j < nseg)
-                                        ? __ldcg(reinterpret_cast<const float4*>(g.partial + ((size_t)(2 * cc + wsl) * BT + tl) * BLOCK_F + c0))
+                                        ? __ldcg(reinterpret_cast<const float4*>(g.partial + ((size_t)(2 * (cc * CG + rank) + wsl) * BT + tl) * BLOCK_F + c0))
                                         : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
 #pragma unroll
                         for (int j = 0; j < 16; ++j) { acc.x += tv[j].x; acc.y += tv[j].y; acc.z += tv[j].z; acc.w += tv[j].w; }
                     }
-                    epilogue4<T, EPI>(e, f_tt[f] * BT + tl, f_tf[f] * BLOCK_F + c0, acc);
+                    epilogue4<T, EPI>(e, (f_tt[f] * CG + rank) * BT + tl, f_tf[f] * BLOCK_F + c0, acc);
                 }
             } else if (last_sh) {
                 for (int i = (int)threadIdx.x; i < total; i += FIX_THREADS) {
@@ -664,7 +735,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 // (only the tile's first contributor can start at or before the tile's first unit)
                                 const int wsl = (cc == c_lo) ? 1 : 0;
                                 const float4* ps = reinterpret_cast<const float4*>(
-                                    g.partial + ((size_t)(2 * cc + wsl) * BT + tl) * BLOCK_F + c0);
+                                    g.partial + ((size_t)(2 * (cc * CG + rank) + wsl) * BT + tl) * BLOCK_F + c0);
 #pragma unroll
                                 for (int x = 0; x < 4; ++x) tv[j][x] = __ldcg(ps + x);
                             } else {
@@ -680,7 +751,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                                 acc[4 * x + 2] += tv[j][x].z; acc[4 * x + 3] += tv[j][x].w;
                             }
                     }
-                    const int mm = f_tt[f] * BT + tl;
+                    const int mm = (f_tt[f] * CG + rank) * BT + tl;
                     const int n0 = f_tf[f] * BLOCK_F;
                     epilogue16<T, EPI>(e, mm, n0 + c0, acc);
                 }
@@ -690,7 +761,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             if (threadIdx.x == 64 && last_sh) {
                 // the last contributor to finish its share re-arms the tile's counters for the next launch
                 for (int f = 0; f < n_fix; ++f) {
-                    const int tile = fix_tile[f];
+                    const int tile = fix_tile[f] * CG + rank;
                     const int prev = atomicAdd(&g.tile_counter[g.done_offset + tile], 1);
                     if (prev == f_nseg[f] - 1) { g.tile_counter[tile] = 0; g.tile_counter[g.done_offset + tile] = 0; }
                 }
@@ -699,7 +770,8 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     }
 
     tc_fence_before();
-    __syncthreads();
+    // (pairs: neither CTA leaves while the other may still arrive on its barriers or its MMAs read this shared memory)
+    if (PAIR) cluster_sync_all(); else __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, ncols);
     if constexpr (EPI == EPI_RESID || EPI == EPI_DOWN) {
         if (post.kind != 0) {
@@ -708,7 +780,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             __shared__ float post_red[33];
             __shared__ int post_ok;
             if (threadIdx.x == 0) { __threadfence(); atomicAdd(post.counter, 1u); }
-            if (cta < post.n_rows) {
+            if ((int)blockIdx.x < post.n_rows) {
                 if (threadIdx.x == 0) {
                     const long long t0 = clock64();
                     int ok = 1;
@@ -720,7 +792,7 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 }
                 __syncthreads();
                 if (post_ok) {
-                    for (int r = cta; r < post.n_rows; r += G) {
+                    for (int r = (int)blockIdx.x; r < post.n_rows; r += (int)gridDim.x) {
                         if (post.kind == 1)
                             prep_rows_row<T>(r, post.x, post.list, post.m_count, post.gain, post.eps, post.d, (T*)post.a_out, post_red,
                                              post.rows, const_cast<float*>(post.packet), post.sd.W_max);

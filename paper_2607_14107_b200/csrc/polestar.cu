@@ -61,6 +61,7 @@ struct Switches {
     int accumulate = 1;      // POLESTAR_GEMM_ACCUMULATE: O / down projections of the chained kernel add their parts onto
                              // the residual rows in L2 (0: ordered reduction of published partial tiles, bit-reproducible)
     int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
+    int pair_rows = 1 << 30; // POLESTAR_GEMM_PAIR_ROWS: projections of at least this many rows run on CTA pairs (tcgen05 cta_group::2)
     int epi_groups = 3;      // POLESTAR_GEMM_EPI_GROUPS: groups of four warps that drain an accumulator when a projection
                              // has several token tiles (1: the four epilogue warps alone)
     int l2promo = (int)CU_TENSOR_MAP_L2_PROMOTION_L2_128B;   // POLESTAR_TMA_L2PROMO
@@ -78,6 +79,7 @@ static Switches read_switches() {
     w.fuse_select = env_int("POLESTAR_FUSE_SELECT", w.fuse_select);
     w.chain = env_int("POLESTAR_CHAIN", w.chain);
     w.stages = env_int("POLESTAR_GEMM_STAGES", w.stages);
+    w.pair_rows = env_int("POLESTAR_GEMM_PAIR_ROWS", w.pair_rows);
     w.epi_groups = env_int("POLESTAR_GEMM_EPI_GROUPS", w.epi_groups);
     w.align_pct = env_int("POLESTAR_GEMM_ALIGN_PCT", w.align_pct);
     w.half_align = env_int("POLESTAR_GEMM_HALF_ALIGN", w.half_align);
@@ -107,12 +109,13 @@ static Switches stand_alone_switches() {
 // ------------------------------------------------------------------------------------------
 // per-device facts: SM count, dynamic shared-memory attributes of the kernels, built-in scratch
 // ------------------------------------------------------------------------------------------
-struct DevInfo { bool ready = false; int sm_count = 0; };
+struct DevInfo { bool ready = false; int sm_count = 0; int gemm_pairs = 0; };
 static const int MAX_DEVICES = 64;
 static DevInfo g_dev[MAX_DEVICES];
 static int g_last_sm_count = 0;
 
 static cudaError_t set_kernel_attributes();
+static int resident_gemm_pairs();
 // Facts of the CURRENT device; the first call on a device queries it and raises the shared-memory limits of
 // every kernel that needs more than the default there (function attributes are per device).
 static int device_info(DevInfo* out) {
@@ -124,6 +127,7 @@ static int device_info(DevInfo* out) {
     if (!di.ready) {
         CK(cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev));
         CK(set_kernel_attributes());
+        di.gemm_pairs = resident_gemm_pairs();
         di.ready = true;
     }
     g_last_sm_count = di.sm_count;
@@ -214,6 +218,7 @@ struct GemmWs {
     unsigned* chain_counter = nullptr;     // the same for chained launches
     mutable unsigned chain_total = 0;
     int sms = 148;                         // SMs of the device the launches go to
+    int pairs = 0;                         // CTA pairs (clusters of two) of the pair GEMM that are resident at once; 0: pairs unavailable
     Switches sw;
 };
 
@@ -231,9 +236,9 @@ static int launch_gemm_simt(const void* A, const void* W, int M, int N_out, int 
 }
 
 // stream-K grid of a GEMM with M rows: G CTAs over U units
-static void sk_grid(const GemmWs& ws, int M, int N_out, int K, long long* U, long long* G, int BT = tc::BLOCK_T) {
+static void sk_grid(const GemmWs& ws, int M, int N_out, int K, long long* U, long long* G, int BT = tc::BLOCK_T, int units = 0) {
     const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + BT - 1) / BT;
-    const int sms = ws.sms;
+    const int sms = units > 0 ? units : ws.sms;           // scheduling units: SMs, or resident CTA pairs
     *U = (long long)tiles_f * tiles_t * (K / 64);
     long long g = std::min<long long>((long long)sms, *U);
     const long long tiles = (long long)tiles_f * tiles_t;
@@ -256,20 +261,29 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     if (M <= 0) return POLESTAR_OK;
     // weights: tile-major [chunks * 256][64]; activations: exactly M rows, so that the rows of a token tile
     // beyond M are out of bounds and arrive as zeros without being read
-    const CUtensorMap* mw = maps.get(W, (uint64_t)N_out * (uint64_t)(K / 64), 64, tc::BLOCK_F);
-    const CUtensorMap* ma = maps.get(A, (uint64_t)M, (uint64_t)K, tc::BLOCK_T);
-    if (!mw || !ma) return POLESTAR_E_CUDA;
     // Steps of several hundred rows (operands from L2, tensor-bound): CTA tiles of 256 tokens, two MMAs per k step on
     // one weight tile (64 KB of operands per k block for twice the work of 48 KB)
-    const int TT = (M >= (EPI == EPI_SWIGLU ? ws.sw.tall_rows_ffn : ws.sw.tall_rows)) ? 2 : 1;
-    const int BT = tc::BLOCK_T * TT;
+    // From POLESTAR_GEMM_PAIR_ROWS rows on: CTA pairs on tiles of 256 tokens (one MMA over both SMs, half a weight tile each)
+    const bool pair = ws.pairs > 0 && M >= ws.sw.pair_rows && !(sel && sel->on);
+    const int TT = (!pair && M >= (EPI == EPI_SWIGLU ? ws.sw.tall_rows_ffn : ws.sw.tall_rows)) ? 2 : 1;
+    const int BT = tc::BLOCK_T * (pair ? 2 : TT);          // tokens per scheduling unit's tile
     const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + BT - 1) / BT;
     // When a multiple of the tile count fits on >= 85 % of the SMs, the grid takes it: CTA ranges then never
     // cross a tile boundary, so every CTA has one segment (one fix-up instead of two, or none at all).
+    const CUtensorMap* mw = maps.get(W, (uint64_t)N_out * (uint64_t)(K / 64), 64, pair ? tc::BLOCK_F / 2 : tc::BLOCK_F);
+    const CUtensorMap* ma = maps.get(A, (uint64_t)M, (uint64_t)K, tc::BLOCK_T);
+    if (!mw || !ma) return POLESTAR_E_CUDA;
     long long U, G;
-    sk_grid(ws, M, N_out, K, &U, &G, BT);
-    while (G > 1 && ((size_t)2 * G * BT * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
-    if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
+    if (pair) {
+        // the pair is the scheduling unit: G counts pairs here, the launch has twice as many CTAs
+        sk_grid(ws, M, N_out, K, &U, &G, BT, ws.pairs);
+        while (G > 1 && ((size_t)4 * G * tc::BLOCK_T * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
+        if (2 * tiles_f * tiles_t + 2 > ws.n_counters / 2) return POLESTAR_E_INVAL;
+    } else {
+        sk_grid(ws, M, N_out, K, &U, &G, BT, ws.sms);
+        while (G > 1 && ((size_t)2 * G * BT * tc::BLOCK_F * 4 + 16384 + 65536 > ws.partial_bytes)) --G;
+        if (tiles_f * tiles_t > ws.n_counters / 2) return POLESTAR_E_INVAL;
+    }
     tc::SkArgs g;
     g.M = M; g.N_out = N_out; g.K = K; g.tiles_f = tiles_f; g.tiles_t = tiles_t;
     // Three stages (145 KB) for the weight-bound steps: measured +2 % tokens/s over four (the HBM stream needs no more in
@@ -277,24 +291,31 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     // stages are 4 % slower.  Four stages when operands come from L2 (several token tiles).
     g.stages = std::max(2, std::min(4, ws.sw.stages > 0 ? ws.sw.stages : (tiles_t == 1 ? 3 : 4)));
     if (TT == 2) g.stages = std::min(g.stages, 3);          // 64 KB per stage
+    if (pair) g.stages = 6;                                 // 32 KB per stage and CTA
     g.partial = ws.partial; g.tile_counter = ws.counters; g.done_offset = ws.n_counters / 2; g.status = ws.status;
     g.w_stream = (g.tiles_t == 1 && ws.sw.evict_first) ? 1 : 0;
     g.epi_groups = g.tiles_t > 1 ? std::max(1, std::min(3, ws.sw.epi_groups)) : 1;
     // POLESTAR_TRACE builds: nanosecond stamps of the launches of one epilogue kind, kept in the tail of the partial workspace
     g.trace = (ws.sw.gemm_trace == EPI) ? (long long*)((char*)ws.partial + ws.partial_bytes - 16384) : nullptr;
-    const size_t smem = (size_t)g.stages * (tc::STAGE_BYTES + (TT - 1) * tc::A_BYTES) + 1024;
+    const size_t smem = pair ? (size_t)g.stages * (tc::A_BYTES + tc::W_BYTES / 2) + 1024
+                             : (size_t)g.stages * (tc::STAGE_BYTES + (TT - 1) * tc::A_BYTES) + 1024;
     auto kern = TT == 2 ? tc::gemm_sk_kernel<__nv_bfloat16, EPI, 2> : tc::gemm_sk_kernel<__nv_bfloat16, EPI, 1>;
+    const unsigned n_ctas = (unsigned)(pair ? 2 * G : G);
     PostArgs pa;
     memset(&pa, 0, sizeof(pa));
     if (post && post->kind && ws.post_counter) {
         pa = *post;
         pa.counter = ws.post_counter;
-        ws.post_total += (unsigned)G;
+        ws.post_total += n_ctas;
         pa.expect = ws.post_total;
     }
     tc::SelFuse sfz;
     if (sel) sfz = *sel; else memset(&sfz, 0, sizeof(sfz));
     if (sfz.on) g.epi_groups = 1;          // the selection runs on warps 6-13 of the first CTA
+    if (pair) {
+        CK(launch_k_cluster(tc::gemm_sk_kernel<__nv_bfloat16, EPI, 1, 2>, dim3(n_ctas), dim3(tc::FIX_THREADS), smem, st, 2u, *mw, *ma, g, e, pa, sfz));
+        return POLESTAR_OK;
+    }
     CK(launch_k(kern, dim3((unsigned)G), dim3(tc::FIX_THREADS), smem, st, *mw, *ma, g, e, pa, sfz));
     return POLESTAR_OK;
 }
@@ -687,6 +708,21 @@ extern "C" const char* polestar_strerror(int code) {
 }
 
 static const size_t SIMT_ATTN_SMEM_MAX = 200 * 1024;
+// How many clusters of two CTAs of the pair GEMM the device holds at once (its grid-wide counters need every CTA resident)
+static int resident_gemm_pairs() {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(2 * 148); cfg.blockDim = dim3(tc::FIX_THREADS);
+    cfg.dynamicSmemBytes = 6 * (tc::A_BYTES + tc::W_BYTES / 2) + 1024;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV, 1, 2>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
 static cudaError_t set_kernel_attributes() {
     cudaError_t e;
     const int gemm_smem = 4 * (int)tc::STAGE_BYTES + 1024;    // four stages of 48 KB + alignment slack
@@ -697,6 +733,12 @@ static cudaError_t set_kernel_attributes() {
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_DOWN>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_LOGITS>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV_REFRESH>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV, 1, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_RESID, 1, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_SWIGLU, 1, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_DOWN, 1, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_LOGITS, 1, 2>), gemm_smem);
+    PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV_REFRESH, 1, 2>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_QKV, 2>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_RESID, 2>), gemm_smem);
     PS_ATTR((tc::gemm_sk_kernel<__nv_bfloat16, EPI_SWIGLU, 2>), gemm_smem);
@@ -1280,7 +1322,7 @@ extern "C" int polestar_init(polestar_ctx** out, const polestar_model* m, const 
     c->gws.counters = c->b.gemm_counters; c->gws.n_counters = GEMM_COUNTERS - 512; c->gws.status = c->b.status;
     c->gws.post_counter = reinterpret_cast<unsigned*>(c->b.gemm_counters + GEMM_COUNTERS - 1); c->gws.post_total = 0;
     c->gws.chain_counter = reinterpret_cast<unsigned*>(c->b.gemm_counters + GEMM_COUNTERS - 512); c->gws.chain_total = 0;
-    c->gws.sms = c->sms; c->gws.sw = c->sw;
+    c->gws.sms = c->sms; c->gws.sw = c->sw; c->gws.pairs = di.gemm_pairs;
 
     auto fail = [&](int code) { delete c; return code; };
     // zero the persistent state (everything in front of the scratch rows)
@@ -1635,7 +1677,7 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     float2* rope = (float2*)(sc + off_rope);
     MapCache maps;                     // the two tensor maps of this call (built per call: no shared state)
     GemmWs ws;
-    ws.sms = di.sm_count; ws.sw = stand_alone_switches();
+    ws.sms = di.sm_count; ws.sw = stand_alone_switches(); ws.pairs = di.gemm_pairs;
     maps.l2promo = ws.sw.l2promo;
     ws.partial = (float*)(sc + off_part); ws.partial_bytes = GEMM_PARTIAL_BYTES;
     const int M = batch * max_rows;
@@ -1643,7 +1685,8 @@ extern "C" int polestar_k_refresh(const void* h, const int32_t* idx, const int32
     // The scratch is caller memory with unknown contents: the split-K tile counters must start at zero.  Only the
     // counters of this GEMM's output tiles (arrivals, then finished shares) are used, so only those are cleared.
     const long long tiles = (long long)((dq + 2 * dkv + tc::BLOCK_F - 1) / tc::BLOCK_F) * ((M + tc::BLOCK_T - 1) / tc::BLOCK_T);
-    const int n_cnt = (int)std::min<long long>(GEMM_COUNTERS, 2 * (tiles + 1));
+    // (CTA pairs count per 128-row half of their 256-row tiles: up to one more half per feature tile)
+    const int n_cnt = (int)std::min<long long>(GEMM_COUNTERS, 2 * (tiles + (dq + 2 * dkv) / tc::BLOCK_F + 2));
     ws.counters = (int*)(sc + off_cnt); ws.n_counters = n_cnt; ws.status = (int*)(sc + off_status);
     const int half = head_dim / 2;
     // Two launches with programmatic stream serialization (the projection starts while the gather drains).  The gather

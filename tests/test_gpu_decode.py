@@ -296,6 +296,16 @@ def test_c1b_tall_gemm_tiles(monkeypatch):
     assert seen["refresh"] > 3 and seen["entry_window"] > 0
 
 
+def test_c1b_gemm_cta_pairs(monkeypatch):
+    # CTA pairs (tcgen05 cta_group::2: one MMA over two SMs, each loading half of the weight tile) for every projection of
+    # more than 129 rows: ragged block entries of a batch (a pair tile's second half partly or wholly empty), refresh
+    # steps, whole and split tiles, in-place L2 reductions of the O / down projections
+    monkeypatch.setenv("POLESTAR_GEMM_PAIR_ROWS", "130")
+    seen = run_forced("c1b", 12, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5, batch=3, prompt_len=50, gen_len=96, block=24,
+                      max_steps=16)
+    assert seen["refresh"] > 3 and seen["entry_window"] > 0
+
+
 def test_c1b_bf16_simt_gemm_path():
     run_forced("c1b", 6, tau_upd=-1, flags=I.FLAG_DEFAULT | Bd.FLAG_SIMT_GEMM)
 

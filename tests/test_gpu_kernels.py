@@ -194,6 +194,22 @@ def test_select_zero_drift_and_nan():
     (4096, 4096, 32, 32, 41, 1), (4096, 4096, 32, 32, 1024, 1), (4096, 4096, 32, 32, 410, 8),
 ])
 def test_refresh_chain_matches_oracle(P, d, nh, nkv, k, batch):
+    check_refresh_chain(P, d, nh, nkv, k, batch)
+
+
+@pytest.mark.parametrize("P,d,nh,nkv,k,batch", [
+    (300, 256, 2, 2, 300, 1),          # 300 rows: the second pair tile's second half is empty
+    (3400, 256, 2, 2, 3300, 4),        # more pair tiles than pairs: whole tiles round-robin + stream-K tail
+    (4096, 4096, 32, 32, 410, 8),      # the micro-benchmark's shape, 3280 rows
+])
+def test_refresh_chain_on_cta_pairs(monkeypatch, P, d, nh, nkv, k, batch):
+    # the same projection on CTA pairs (tcgen05 cta_group::2): each CTA of a pair loads half of the weight tile
+    monkeypatch.setenv("POLESTAR_GEMM_PAIR_ROWS", "200")
+    Bd.polestar_reload_env()           # the stand-alone calls read the switches once, not per launch
+    check_refresh_chain(P, d, nh, nkv, k, batch)
+
+
+def check_refresh_chain(P, d, nh, nkv, k, batch):
     dh = 128
     big = d >= 2048
     dev = "cuda" if big else "cpu"                      # large inputs are generated on the device (same values)
