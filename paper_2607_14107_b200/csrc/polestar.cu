@@ -786,7 +786,11 @@ struct Path {
             // single block of rows the warp-level kernel's shorter dependency chain wins (11 us against 16 us per
             // layer at the 8B shape), everywhere else the tensor-core kernel does.
             const bool records = a.pprev != nullptr || a.aprev != nullptr;
-            const bool few_rows = !records && a.rows_per_seq <= 64 && a.N <= 1024 && c->sw.attn_kernel == 0;
+            // Beyond 1024 keys the warp-level family has a 64-row kernel: it wins where (sequences x heads) fill the GPU (a
+            // batch of long sequences, 64 rows each: 85 us against 111 us for the streaming kernel, whose 128-row tiles are half empty).
+            const bool fills = (long long)(a.batch > 0 ? a.batch : 1) * a.n_heads >= c->sms;
+            const bool few_rows = !records && a.rows_per_seq <= 64 && c->sw.attn_kernel == 0 &&
+                                  (a.N <= 1024 || (a.rows_per_seq >= 48 && fills));
             if (attention_stream_applies(a) && !few_rows &&
                 (c->sw.attn_kernel == 9 || (c->sw.attn_kernel == 0 && attention_prefers_stream(a))))
                 return launch_attention_stream(c->maps, a, c->st, c->b.status);
