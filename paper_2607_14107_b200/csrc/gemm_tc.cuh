@@ -182,6 +182,13 @@ __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// the same wait for registers that arithmetic consumes: they are operands of the wait, so nothing that uses them moves above it
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t* r) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+                 :: "memory");
+}
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 
@@ -563,12 +570,30 @@ gemm_sk_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                 const uint32_t taddr = taddr0 + (uint32_t)((TT == 1 ? (seg & 1) : hh) * BLOCK_F);
                 if (whole) {
                     if (warp_live) {
-                        for (int c0 = 0; c0 < BLOCK_F; c0 += 16) {
-                            if ((hh * (BLOCK_F / 16) + (c0 >> 4)) % groups != gi) continue;
-                            float v[16];
-                            tmem_ld16(taddr + (uint32_t)c0, v);
+                        // this warp's 16-column chunks of the half (dealt round-robin over the groups); the tensor-memory load
+                        // of the next chunk is in flight during the epilogue of the current one
+                        const int step = 16 * groups;
+                        int c0 = 16 * (((gi - hh * (BLOCK_F / 16)) % groups + groups) % groups);
+                        uint32_t ra[16], rb[16];
+                        float v[16];
+                        if (c0 < BLOCK_F) tmem_ld16_issue(taddr + (uint32_t)c0, ra);
+                        while (c0 < BLOCK_F) {
+                            const int c1 = c0 + step;
+                            tmem_ld_wait16(ra);
+                            if (c1 < BLOCK_F) tmem_ld16_issue(taddr + (uint32_t)c1, rb);
                             if (live) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(ra[i]);
                                 epilogue16<T, EPI>(e, m, n0 + c0, v);
+                            }
+                            if (c1 >= BLOCK_F) break;
+                            c0 = c1 + step;
+                            tmem_ld_wait16(rb);
+                            if (c0 < BLOCK_F) tmem_ld16_issue(taddr + (uint32_t)c0, ra);
+                            if (live) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(rb[i]);
+                                epilogue16<T, EPI>(e, m, n0 + c1, v);
                             }
                         }
                     }
