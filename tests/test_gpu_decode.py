@@ -296,6 +296,15 @@ def test_c1b_tall_gemm_tiles(monkeypatch):
     assert seen["refresh"] > 3 and seen["entry_window"] > 0
 
 
+@pytest.mark.parametrize("groups", [1, 2])
+def test_c1b_epilogue_warp_groups(monkeypatch, groups):
+    # projections with several token tiles drain their accumulators with four, eight or (the default) twelve warps
+    monkeypatch.setenv("POLESTAR_GEMM_EPI_GROUPS", str(groups))
+    seen = run_forced("c1b", 8, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5, batch=3, prompt_len=50, gen_len=96, block=24,
+                      max_steps=16)
+    assert seen["refresh"] > 2
+
+
 def test_c1b_gemm_cta_pairs(monkeypatch):
     # CTA pairs (tcgen05 cta_group::2: one MMA over two SMs, each loading half of the weight tile) for every projection of
     # more than 129 rows: ragged block entries of a batch (a pair tile's second half partly or wholly empty), refresh
