@@ -16,6 +16,9 @@ pytestmark = pytest.mark.gpu
 
 def setup(name, std=0.02, **kw):
     m, p = I.config(name)
+    model_kw = kw.pop("model", None)        # overrides of the model's shape
+    if model_kw:
+        m = dataclasses.replace(m, **model_kw)
     kw["flags"] = kw.get("flags", p.flags) | I.FLAG_KEEP_HIDDEN
     p = dataclasses.replace(p, **kw)
     w = I.make_weights(m, seed=0, std=std)
@@ -294,6 +297,14 @@ def test_c1b_tall_gemm_tiles(monkeypatch):
     seen = run_forced("c1b", 12, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5, batch=3, prompt_len=50, gen_len=96, block=24,
                       max_steps=16)
     assert seen["refresh"] > 3 and seen["entry_window"] > 0
+
+
+def test_c1b_batch_of_long_sequences_plain_steps():
+    # 19 sequences x 8 heads fill the GPU's SMs, more than 1024 keys, 64-row blocks: the layers of a plain step that record
+    # nothing take the 64-row warp-level attention kernel, the last layer and the refresh steps the streaming kernel
+    seen = run_forced("c1b", 7, model=dict(d_model=1024, n_heads=8, n_kv_heads=8), batch=19, prompt_len=1040, gen_len=64, block=64,
+                      max_steps=16, tau_upd=5, logit_scale=12.0, alpha=0.001, tau_suffix=0.5)
+    assert seen["within"] > seen["refresh"] > 0
 
 
 @pytest.mark.parametrize("groups", [1, 2])
