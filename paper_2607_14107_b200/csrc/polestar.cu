@@ -58,6 +58,7 @@ struct Switches {
                              // threshold at 2048, no change at 512)
     int tall_rows_ffn = 512; // POLESTAR_GEMM_TALL_ROWS_FFN: the same threshold for the gate/up projection, whose epilogue is short
                              // enough for the tall tile to pay from 512 rows on (follows POLESTAR_GEMM_TALL_ROWS when only that is set)
+    int one_tall = 1;        // POLESTAR_GEMM_ONE_TALL: projections of 129 - 256 rows run as one 256-token tile
     int accumulate = 1;      // POLESTAR_GEMM_ACCUMULATE: O / down projections of the chained kernel add their parts onto
                              // the residual rows in L2 (0: ordered reduction of published partial tiles, bit-reproducible)
     int chain_qkv = 0;       // POLESTAR_CHAIN_QKV (same)
@@ -89,6 +90,7 @@ static Switches read_switches() {
     w.fuse_prep = env_int("POLESTAR_FUSE_PREP", w.fuse_prep);
     w.fold_norm = env_int("POLESTAR_FOLD_NORM", w.fold_norm);
     w.accumulate = env_int("POLESTAR_GEMM_ACCUMULATE", w.accumulate);
+    w.one_tall = env_int("POLESTAR_GEMM_ONE_TALL", w.one_tall);
     w.tall_rows = env_int("POLESTAR_GEMM_TALL_ROWS", w.tall_rows);
     w.tall_rows_ffn = env_int("POLESTAR_GEMM_TALL_ROWS_FFN", getenv("POLESTAR_GEMM_TALL_ROWS") ? w.tall_rows : w.tall_rows_ffn);
     w.chain_qkv = env_int("POLESTAR_CHAIN_QKV", w.chain_qkv);
@@ -265,7 +267,10 @@ static int launch_gemm_tc(MapCache& maps, const GemmWs& ws, const void* A, const
     // one weight tile (64 KB of operands per k block for twice the work of 48 KB)
     // From POLESTAR_GEMM_PAIR_ROWS rows on: CTA pairs on tiles of 256 tokens (one MMA over both SMs, half a weight tile each)
     const bool pair = ws.pairs > 0 && M >= ws.sw.pair_rows && !(sel && sel->on);
-    const int TT = (!pair && M >= (EPI == EPI_SWIGLU ? ws.sw.tall_rows_ffn : ws.sw.tall_rows)) ? 2 : 1;
+    // (129 - 256 rows, e.g. a refresh step plus its proxy rows: one 256-token tile keeps the step a single token tile, so
+    // every weight byte is still read once and streamed with evict_first, instead of two token tiles sharing the weights)
+    const bool one_tall = M > tc::BLOCK_T && M <= 2 * tc::BLOCK_T && ws.sw.one_tall;
+    const int TT = (!pair && (one_tall || M >= (EPI == EPI_SWIGLU ? ws.sw.tall_rows_ffn : ws.sw.tall_rows))) ? 2 : 1;
     const int BT = tc::BLOCK_T * (pair ? 2 : TT);          // tokens per scheduling unit's tile
     const int tiles_f = N_out / tc::BLOCK_F, tiles_t = (M + BT - 1) / BT;
     // When a multiple of the tile count fits on >= 85 % of the SMs, the grid takes it: CTA ranges then never
