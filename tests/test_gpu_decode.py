@@ -299,6 +299,15 @@ def test_c1b_tall_gemm_tiles(monkeypatch):
     assert seen["refresh"] > 3 and seen["entry_window"] > 0
 
 
+@pytest.mark.parametrize("pre,suf", [(3, 1), (2, 2)])
+def test_c1b_wide_windows(pre, suf):
+    # refresh steps of 160 rows (32 active + 128 window rows): every projection runs as one 256-token tile, the selection
+    # rides on the O projection
+    seen = run_forced("c1b", 12, tau_upd=-1, logit_scale=24.0, alpha=0.001, tau_suffix=0.5, prompt_len=128, gen_len=128, block=32,
+                      max_steps=16, win_prefix_blocks=pre, win_suffix_blocks=suf)
+    assert seen["refresh"] > 3 and seen["entry_window"] > 0
+
+
 def test_c1b_batch_of_long_sequences_plain_steps():
     # 19 sequences x 8 heads fill the GPU's SMs, more than 1024 keys, 64-row blocks: the layers of a plain step that record
     # nothing take the 64-row warp-level attention kernel, the last layer and the refresh steps the streaming kernel
